@@ -1,0 +1,313 @@
+"""CPU oracle for the Structured Recurrent Mixer (SRM): TEST INFRASTRUCTURE ONLY.
+
+A plain, slow, obviously-correct numpy implementation (fp64 by default) of what the
+CUDA path computes: the sequence-parallel form (explicit token-mixing matrices), the
+recurrent form (constant-size per-sample state), the channel-mixing feed-forward,
+the LM head and the two token-selection rules. Only the tests, the smoke check and
+the benchmark's CPU-baseline leg may import it. It shares no code with the CUDA path
+and does not import it; inputs (weights, prompts) are passed in as numpy arrays.
+
+Notation follows the paper's Method section: X, Y in R^{d x n} hold one column per
+position, Y = X M + B with M in R^{n x n} upper-triangular (entry [i, j] weights
+input position i in output position j, so i <= j), alpha the repeated weight vector,
+lambda the decay constant, beta the per-position bias, and the "cache" is the sum
+term of Eq. 2 / Eq. 3. Arrays here are stored position-major, Z[n, d] = X^T.
+
+Parity status of each function (what pins it, see tests/test_oracle_*.py):
+  mixing_matrix            pinned: printed 3x3 matrix of Eq. 1, printed pattern of Eq. 3
+  mixer_parallel           pinned: brute-force loops, cumulative-sum special cases
+  mixer_recurrent_step     pinned: closed forms of Eq. 2 / Eq. 3, equality with the
+                           parallel form to 1e-9, op count, cache size d per layer
+  layer_norm, gelu_erf     pinned: moments / identities / tabulated erf values
+  philox4x32_10            pinned: cuRAND's host Philox4_32_10 generator, bijectivity
+  select_greedy, select_topk  pinned: brute-force sort, frequency test
+  SRMOracle (full model logits)  PARITY UNPINNED beyond self-consistency (parallel ==
+                           recurrent, causality): the paper prints no activations and
+                           its architecture figure is missing, so the block structure
+                           (pre-norm residual blocks, LayerNorm, erf-GELU FFN with
+                           biases, untied bias-free LM head) is a stated reading.
+"""
+from __future__ import annotations
+
+import numpy as np
+from scipy.special import erf as _erf
+
+
+# --------------------------------------------------------------------------------------
+# Token mixing (Method / Architecture: Eq. 1, Eq. 2, Eq. 3)
+# --------------------------------------------------------------------------------------
+
+def mixing_matrix(kind: str, alpha, lam: float, n: int, dtype=np.float64) -> np.ndarray:
+    """Explicit n x n token-mixing matrix M of one head.
+
+    kind "row"   : row i repeats alpha[i], decayed by lam per diagonal (Eq. 1):
+                   M[i, j] = lam^(j-i) * alpha[i]  for i <= j, else 0.
+    kind "col"   : column j repeats alpha[j] (Eq. 3):
+                   M[i, j] = lam^(j-i) * alpha[j]  for i <= j, else 0.
+    Built with scalar loops on purpose (brute-force definition).
+    """
+    M = np.zeros((n, n), dtype=dtype)
+    for i in range(n):
+        for j in range(i, n):
+            a = alpha[i] if kind == "row" else alpha[j]
+            M[i, j] = dtype(lam) ** (j - i) * dtype(a)
+    return M
+
+
+def head_kinds(n_heads: int):
+    """'Mixed' heads: the first half of the heads are row-repeat, the second half
+    column-repeat; outputs are concatenated (Architecture, mixed heads)."""
+    return ["row" if g < n_heads // 2 else "col" for g in range(n_heads)]
+
+
+def mixer_parallel(Z: np.ndarray, alpha: np.ndarray, beta: np.ndarray, lam: np.ndarray,
+                   n_heads: int):
+    """Sequence-parallel token mixing of one layer for one sample.
+
+    Z[n, d] are the (normed) inputs, one row per position. For head g with channel
+    slice c, Y[:, c]^T = Z[:, c]^T M_g + beta[:n, c]^T   (Y = X M + B).
+    Also returns the hand-off cache S_n[d], i.e. the sum term of Eq. 2 / Eq. 3 that
+    position n would use:  row heads  S_n = sum_{m<n} lam^(n-m) alpha[m] z_m,
+                           col heads  S_n = sum_{m<n} lam^(n-m) z_m.
+    """
+    n, d = Z.shape
+    dh = d // n_heads
+    dt = Z.dtype.type
+    Y = np.empty_like(Z)
+    S = np.zeros(d, dtype=Z.dtype)
+    for g, kind in enumerate(head_kinds(n_heads)):
+        c = slice(g * dh, (g + 1) * dh)
+        M = mixing_matrix(kind, alpha[g], lam[g], n, dtype=dt)
+        X = Z[:, c].T                               # d_h x n, columns = positions
+        Y[:, c] = (X @ M).T + beta[:n, c]
+        for m in range(n):
+            w = dt(lam[g]) ** (n - m)
+            if kind == "row":
+                w = w * dt(alpha[g][m])
+            S[c] += w * Z[m, c]
+    return Y, S
+
+
+def mixer_recurrent_step(z: np.ndarray, S: np.ndarray, t: int, alpha: np.ndarray,
+                         beta: np.ndarray, lam: np.ndarray, n_heads: int):
+    """One recurrent token-mixing step at absolute position t (batched over rows).
+
+    z[..., d] normed input of position t, S[..., d] the cache (sum term) for position t.
+    row heads (Eq. 2):  y = alpha_t z + beta_t + S ;      S' = lam (S + alpha_t z)
+    col heads (Eq. 3):  y = alpha_t (z + S) + beta_t ;    S' = lam (S + z)
+    so that S'(t+1) = sum_{m<=t} lam^(t+1-m) [alpha_m] z_m is the sum term of t+1.
+    """
+    d = z.shape[-1]
+    dh = d // n_heads
+    dt = z.dtype.type
+    y = np.empty_like(z)
+    S_new = np.empty_like(S)
+    for g, kind in enumerate(head_kinds(n_heads)):
+        c = slice(g * dh, (g + 1) * dh)
+        a, l = dt(alpha[g][t]), dt(lam[g])
+        if kind == "row":
+            u = a * z[..., c]
+            y[..., c] = u + beta[t, c] + S[..., c]
+            S_new[..., c] = l * (S[..., c] + u)
+        else:
+            v = z[..., c] + S[..., c]
+            y[..., c] = a * v + beta[t, c]
+            S_new[..., c] = l * v
+    return y, S_new
+
+
+# --------------------------------------------------------------------------------------
+# Channel mixing and norms (stated reading: pre-norm residual block, LayerNorm with
+# affine parameters and biased variance, Linear -> exact erf GELU -> Linear, with biases)
+# --------------------------------------------------------------------------------------
+
+def layer_norm(x: np.ndarray, g: np.ndarray, b: np.ndarray, eps: float) -> np.ndarray:
+    mu = x.mean(axis=-1, keepdims=True)
+    var = ((x - mu) ** 2).mean(axis=-1, keepdims=True)
+    return (x - mu) / np.sqrt(var + x.dtype.type(eps)) * g + b
+
+
+def gelu_erf(x: np.ndarray) -> np.ndarray:
+    return (0.5 * x * (1.0 + _erf(x / np.sqrt(2.0)))).astype(x.dtype)
+
+
+def feed_forward(a: np.ndarray, W1, b1, W2, b2) -> np.ndarray:
+    """FFN(a) = W2 gelu(W1 a + b1) + b2, weights stored [out, in]."""
+    return gelu_erf(a @ W1.T + b1) @ W2.T + b2
+
+
+# --------------------------------------------------------------------------------------
+# Token selection
+# --------------------------------------------------------------------------------------
+
+_M0, _M1 = 0xD2511F53, 0xCD9E8D57
+_W0, _W1 = 0x9E3779B9, 0xBB67AE85
+_MASK = 0xFFFFFFFF
+
+
+def philox4x32_10(counter, key):
+    """Philox4x32 with 10 rounds (Salmon et al., 'Parallel random numbers: as easy as
+    1, 2, 3', SC'11). counter = 4 uint32 words, key = 2 uint32 words -> 4 uint32 words."""
+    c0, c1, c2, c3 = (int(v) & _MASK for v in counter)
+    k0, k1 = (int(v) & _MASK for v in key)
+    for _ in range(10):
+        p0 = _M0 * c0
+        p1 = _M1 * c2
+        c0, c1, c2, c3 = ((p1 >> 32) ^ c1 ^ k0) & _MASK, p1 & _MASK, \
+                         ((p0 >> 32) ^ c3 ^ k1) & _MASK, p0 & _MASK
+        k0 = (k0 + _W0) & _MASK
+        k1 = (k1 + _W1) & _MASK
+    return c0, c1, c2, c3
+
+
+def philox_uniform(seed: int, sample_idx: int, step: int) -> float:
+    """u in [0,1) for (seed, sample, step): the first output word of Philox4x32-10 with
+    key (seed low word, seed high word) and counter (sample_idx, step, 0, 0), keeping
+    its top 24 bits: u = (r >> 8) * 2^-24 (exactly representable in fp32)."""
+    r = philox4x32_10((sample_idx, step, 0, 0), (seed & _MASK, (seed >> 32) & _MASK))[0]
+    return (r >> 8) * (1.0 / 16777216.0)
+
+
+def select_greedy(logits: np.ndarray) -> np.ndarray:
+    """argmax over the vocabulary; among equal maxima the smallest id wins."""
+    return np.argmax(logits, axis=-1).astype(np.int32)   # numpy returns the first maximum
+
+
+def topk_order(row: np.ndarray, k: int) -> np.ndarray:
+    """ids of the k largest logits ordered by (logit descending, id ascending)."""
+    ids = np.lexsort((np.arange(row.shape[0]), -row))     # primary -row, secondary id
+    return ids[:k]
+
+
+def select_topk(logits: np.ndarray, k: int, temperature: float, seed: int,
+                sample_idx: np.ndarray, step: int, return_detail: bool = False):
+    """Temperature + top-k sampling by inverse CDF.
+
+    For each row: keep the k largest logits in (logit desc, id asc) order,
+    w_i = exp((l_i - l_0) / T), c_i = w_0 + ... + w_i, u = philox_uniform(...);
+    the token is the first i with c_i > u * c_{k-1} (the last one if none).
+    """
+    B = logits.shape[0]
+    out = np.empty(B, dtype=np.int32)
+    detail = []
+    for b in range(B):
+        row = logits[b].astype(np.float64)
+        ids = topk_order(row, k)
+        w = np.exp((row[ids] - row[ids[0]]) / temperature)
+        c = np.cumsum(w)
+        u = philox_uniform(seed, int(sample_idx[b]), step)
+        thr = u * c[-1]
+        pick = len(ids) - 1
+        for i in range(len(ids)):
+            if c[i] > thr:
+                pick = i
+                break
+        out[b] = ids[pick]
+        if return_detail:
+            detail.append(dict(ids=ids, cdf=c, thr=thr, pick=pick, u=u))
+    return (out, detail) if return_detail else out
+
+
+# --------------------------------------------------------------------------------------
+# The model
+# --------------------------------------------------------------------------------------
+
+class SRMOracle:
+    """Whole-model oracle. `W` is the parameter dict of srm_inputs.make_weights (any dict
+    of numpy arrays with those names works); all arithmetic runs in `dtype`."""
+
+    def __init__(self, n_layers, d_model, vocab, n_ctx, W, n_heads=4, ln_eps=1e-5,
+                 dtype=np.float64):
+        self.L, self.d, self.V, self.n_ctx, self.h = n_layers, d_model, vocab, n_ctx, n_heads
+        self.eps, self.dt = ln_eps, dtype
+        cv = lambda a: np.asarray(a, dtype=dtype)
+        self.E, self.W_lm = cv(W["E"]), cv(W["W_lm"])
+        self.lnf_g, self.lnf_b = cv(W["lnf_g"]), cv(W["lnf_b"])
+        self.layers = [{k: cv(v) for k, v in lw.items()} for lw in W["layers"]]
+        assert len(self.layers) == n_layers
+
+    # -- sequence-parallel form --------------------------------------------------------
+    def forward_parallel(self, tokens: np.ndarray, keep_x: bool = False):
+        """tokens int[B, n] -> logits[B, n, V] for every position, hand-off cache
+        state[L, B, d] (what position n would read). Token mixing uses the explicit
+        matrices of Eq. 1 / Eq. 3 per head."""
+        B, n = tokens.shape
+        assert n <= self.n_ctx
+        x = self.E[tokens]                                   # [B, n, d]; no positional embedding
+        state = np.zeros((self.L, B, self.d), dtype=self.dt)
+        xs = []
+        for l, lw in enumerate(self.layers):
+            z = layer_norm(x, lw["ln1_g"], lw["ln1_b"], self.eps)
+            y = np.empty_like(z)
+            for b in range(B):
+                y[b], state[l, b] = mixer_parallel(z[b], lw["alpha"], lw["beta"], lw["lam"], self.h)
+            x = x + y
+            a = layer_norm(x, lw["ln2_g"], lw["ln2_b"], self.eps)
+            x = x + feed_forward(a, lw["W1"], lw["b1"], lw["W2"], lw["b2"])
+            if keep_x:
+                xs.append(x.copy())
+        logits = layer_norm(x, self.lnf_g, self.lnf_b, self.eps) @ self.W_lm.T
+        return (logits, state, xs) if keep_x else (logits, state)
+
+    # -- recurrent form ----------------------------------------------------------------
+    def init_state(self, B: int) -> np.ndarray:
+        return np.zeros((self.L, B, self.d), dtype=self.dt)
+
+    def decode_step(self, state: np.ndarray, tok: np.ndarray, pos: int, keep_x: bool = False):
+        """Consume tok[B] at absolute position `pos`: returns logits[B, V] (predicting
+        position pos+1) and the updated cache state'[L, B, d]."""
+        assert 0 <= pos < self.n_ctx
+        x = self.E[tok]                                      # [B, d]
+        new_state = np.empty_like(state)
+        xs = []
+        for l, lw in enumerate(self.layers):
+            z = layer_norm(x, lw["ln1_g"], lw["ln1_b"], self.eps)
+            y, new_state[l] = mixer_recurrent_step(z, state[l], pos, lw["alpha"], lw["beta"],
+                                                   lw["lam"], self.h)
+            x = x + y
+            a = layer_norm(x, lw["ln2_g"], lw["ln2_b"], self.eps)
+            x = x + feed_forward(a, lw["W1"], lw["b1"], lw["W2"], lw["b2"])
+            if keep_x:
+                xs.append(x.copy())
+        logits = layer_norm(x, self.lnf_g, self.lnf_b, self.eps) @ self.W_lm.T
+        return (logits, new_state, xs) if keep_x else (logits, new_state)
+
+    def prefill_recurrent(self, tokens: np.ndarray):
+        """The recurrent form applied position by position to a prompt:
+        logits[B, n, V] and the cache after n tokens."""
+        B, n = tokens.shape
+        state = self.init_state(B)
+        out = np.empty((B, n, self.V), dtype=self.dt)
+        for t in range(n):
+            out[:, t], state = self.decode_step(state, tokens[:, t], t)
+        return out, state
+
+    # -- generation --------------------------------------------------------------------
+    def generate(self, prompts: np.ndarray, gen: int, sampling: dict | None = None,
+                 sample_idx: np.ndarray | None = None, parallel_prefill: bool = True):
+        """Prefill the prompts, then produce `gen` tokens per sample. Generated token k
+        is selected from the logits of position n-1+k and uses Philox step k.
+        Returns tokens[B, gen], the per-step logits[gen, B, V] and the final state."""
+        B, n = prompts.shape
+        sampling = sampling or {"mode": "greedy"}
+        sidx = np.arange(B) if sample_idx is None else sample_idx
+        if parallel_prefill:
+            lg, state = self.forward_parallel(prompts)
+        else:
+            lg, state = self.prefill_recurrent(prompts)
+        logits = lg[:, -1]
+        toks = np.empty((B, gen), dtype=np.int32)
+        all_logits = np.empty((gen, B, self.V), dtype=self.dt)
+        for k in range(gen):
+            all_logits[k] = logits
+            toks[:, k] = self.select(logits, sampling, sidx, k)
+            if k + 1 < gen:
+                logits, state = self.decode_step(state, toks[:, k], n + k)
+        return toks, all_logits, state
+
+    @staticmethod
+    def select(logits, sampling, sample_idx, step):
+        if sampling.get("mode", "greedy") == "greedy":
+            return select_greedy(logits)
+        return select_topk(logits, sampling["top_k"], sampling["temperature"],
+                           sampling["seed"], sample_idx, step)
