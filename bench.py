@@ -1,0 +1,441 @@
+#!/usr/bin/env python
+"""Benchmark of the SRM decode hot path on B200: generated tokens/s at a given batch.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload mid] [--batch B]
+    python bench.py --impl reference ...      # the CPU oracle on the host cores, same metric
+    python bench.py --sweep                   # tokens/s-vs-batch curve + maximum concurrency
+
+A "step" is one recurrent decode step of the whole batch: embedding, L x (fused token-mixer
+state update + feed-forward up/down GEMMs), final norm, LM head, token selection. The
+sequence-parallel prefill that builds the cache runs once before the timed region and is timed
+and reported separately ("prefill"). One JSON line is printed by rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC, UNIT = "generated_tokens_per_s", "tokens/s"
+L2_BYTES = 126e6
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# DRAM traffic of the dominant kernel per launch (bytes), from the ncu capture summarised in
+# profiles/; None until a capture exists for the benchmarked shape.
+GEMM_DRAM_TRAFFIC_PER_STEP = None
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return d, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def __exit__(self, *a):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=2)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        for r in self.rows:
+            if len(r) < 8:
+                continue
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def step_flops(shape):
+    d, L, V = shape.d_model, shape.n_layers, shape.vocab
+    return 16 * L * d * d + 2 * d * V            # per generated token
+
+
+def step_roofline_s(shape, B, state_bytes, peaks):
+    """Slower of the step's FLOPs at the tensor peak and its weight + state bytes at HBM bandwidth."""
+    d, L, V = shape.d_model, shape.n_layers, shape.vocab
+    t_tc = B * step_flops(shape) / (peaks["bf16_tflops_sustained"] * 1e12)
+    bytes_ = 2 * (8 * L * d * d + d * V) + B * 2 * L * d * state_bytes
+    t_hbm = bytes_ / (peaks["hbm_gbs"] * 1e9)
+    return max(t_tc, t_hbm), ("tensor" if t_tc >= t_hbm else "hbm"), t_tc, t_hbm
+
+
+# ----------------------------------------------------------------------------------------------
+def run_reference(args):
+    """The CPU oracle (numpy fp64, as it stands) on the host cores: same metric and config, each
+    step a bounded sample of the batch."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import numpy as np
+    import srm_inputs as I
+    from oracle import srm_oracle as O
+    w = I.WORKLOADS[args.workload]
+    shape = I.CONFIGS[w["model"]]
+    B_full = args.batch or w["batch"] or 4096
+    sample = min(B_full, args.ref_samples)
+    W = I.make_weights(shape)
+    orc = O.SRMOracle(shape.n_layers, shape.d_model, shape.vocab, shape.n_ctx, W, n_heads=shape.n_heads,
+                      ln_eps=shape.ln_eps)
+    rng = np.random.default_rng(0)
+    state = rng.normal(size=(shape.n_layers, sample, shape.d_model))
+    tok = I.make_prompts(args.workload, batch=sample)[:, 0]
+    pos = w["prompt_len"]
+    for _ in range(args.warmup):
+        lg, state = orc.decode_step(state, tok, pos); tok = O.select_greedy(lg); pos += 1
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        lg, state = orc.decode_step(state, tok, pos); tok = O.select_greedy(lg)
+        pos = pos + 1 if pos + 1 < shape.n_ctx else w["prompt_len"]
+    dt = time.perf_counter() - t0
+    value = sample * args.steps / dt
+    cores = _blas_threads()
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": _config_dict(args, shape, w, B_full, extra={"sample": f"{sample} of {B_full} samples per step"}),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": f"{sample} samples x {args.steps} decode steps (numpy fp64 oracle)"},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def _blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 0) for p in threadpool_info() if p.get("user_api") == "blas"]
+        if n:
+            return max(n)
+    except Exception:
+        pass
+    return os.cpu_count()
+
+
+def _config_dict(args, shape, w, B, extra=None):
+    c = {"workload": f"{args.workload}: SRM L{shape.n_layers} d{shape.d_model} F{shape.d_ffn} V{shape.vocab} "
+                     f"n_ctx{shape.n_ctx} {shape.dtype}, batch {B}, prompts {w['prompt_len']} tokens ({w['prompts']}), "
+                     f"{w['sampling']} selection",
+         "batch_per_gpu": B, "prompt_len": w["prompt_len"], "selection": w["sampling"],
+         "parallelism": "independent replicas, no collective"}
+    if extra:
+        c.update(extra)
+    return c
+
+
+def cpu_baseline(shape, W, workload, w, seconds_target=12.0):
+    """Times the oracle's decode step on a bounded sample on the host cores."""
+    import numpy as np
+    import srm_inputs as I
+    from oracle import srm_oracle as O
+    orc = O.SRMOracle(shape.n_layers, shape.d_model, shape.vocab, shape.n_ctx, W, n_heads=shape.n_heads,
+                      ln_eps=shape.ln_eps)
+    sample = 32
+    state = np.random.default_rng(0).normal(size=(shape.n_layers, sample, shape.d_model))
+    tok = I.make_prompts(workload, batch=sample)[:, 0]
+    pos = w["prompt_len"]
+    lg, state = orc.decode_step(state, tok, pos)            # warm-up (BLAS threads, page faults)
+    steps, t0 = 0, time.perf_counter()
+    while True:
+        lg, state = orc.decode_step(state, tok, pos + 1 + steps % 8)
+        tok = O.select_greedy(lg)
+        steps += 1
+        dt = time.perf_counter() - t0
+        if dt > seconds_target or steps >= 64:
+            break
+    return {"value": sample * steps / dt, "unit": UNIT, "cores": _blas_threads(), "kind": "oracle",
+            "sample": f"{sample} samples x {steps} decode steps of the same model (numpy fp64 oracle, {dt:.1f} s)"}
+
+
+# ----------------------------------------------------------------------------------------------
+def run_ours(args):
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+
+    import paper_2605_08696_b200 as P
+    import srm_inputs as I
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+
+    w = I.WORKLOADS[args.workload]
+    shape = I.CONFIGS[w["model"]]
+    B = args.batch or w["batch"] or 4096
+    n = w["prompt_len"]
+    peaks, peak_src = measured_peaks()
+
+    W = I.make_weights(shape)
+    model = P.SRM(shape, W, device=dev, state_dtype=args.state_dtype)
+    samp = P.Sampling("greedy") if w["sampling"] == "greedy" else \
+        P.Sampling("topk", w["top_k"], w["temperature"], seed=shape.seed, sample_idx_base=rank * B)
+    prompts = torch.from_numpy(I.make_prompts(args.workload, batch=B)).to(dev)
+    chunk = min(B, args.chunk)
+    st = model.new_state(B)
+    ws = model.new_workspace(chunk, n, prefill_samples=max(1, min(B, args.prefill_rows // n)))
+    sbytes = 2 if args.state_dtype == "bf16" else 4
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    # ---- prefill (once; timed separately) ----
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sync_all()
+    e0.record()
+    model.prefill(st, prompts, samp, ws)
+    e1.record()
+    torch.cuda.synchronize()
+    prefill_ms = e0.elapsed_time(e1)
+
+    step_no = [1]
+
+    def one_step():
+        if st.pos >= shape.n_ctx:            # timing-only wrap: keep alpha/beta indices in range
+            st.pos = n
+        model.decode_step(st, None, samp, step_no[0], ws)
+        step_no[0] += 1
+
+    for _ in range(max(args.warmup, 3)):
+        one_step()
+    # ---- timed region: exactly K steps ----
+    sync_all()
+    launches0 = model.kernel_launches()
+    with ClockSampler(local) as clk:
+        e0.record()
+        for _ in range(args.steps):
+            one_step()
+        e1.record()
+        torch.cuda.synchronize()
+    t_ms = e0.elapsed_time(e1)
+    launches = model.kernel_launches() - launches0
+    t = torch.tensor([t_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.barrier()
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    t_ms_max = t.item()
+    value = world * B * args.steps / (t_ms_max / 1e3)
+
+    # ---- per-kernel durations, CUDA events on the launching stream, same workload ----
+    model.profile_reset()
+    model.profile(True)
+    for _ in range(args.steps):
+        one_step()
+    torch.cuda.synchronize()
+    model.profile(False)
+    prof = model.profile_read()
+    d, L, V, F = shape.d_model, shape.n_layers, shape.vocab, shape.d_ffn
+    gemm_ms = sum(prof[k][1] for k in ("gemm_up", "gemm_down", "gemm_lm"))
+    gemm_launches = sum(prof[k][0] for k in ("gemm_up", "gemm_down", "gemm_lm"))
+    gemm_flops = args.steps * B * step_flops(shape)
+    achieved_tf = gemm_flops / (gemm_ms / 1e3) / 1e12 if gemm_ms > 0 else 0.0
+    prof_total = sum(v[1] for v in prof.values())
+    peak_tf = peaks["bf16_tflops_sustained"]
+    t_roof, bound, t_tc, t_hbm = step_roofline_s(shape, B, sbytes, peaks)
+    mixer_bytes = args.steps * L * B * d * (4 + 4 + 2 * sbytes + 2)       # x r/w, cache r/w, bf16 activation
+    kernels = {k: {"launches": v[0], "ms_total": round(v[1], 3), "share": round(v[1] / prof_total, 4) if prof_total else 0}
+               for k, v in prof.items() if v[0]}
+    kernels["gemm_up"]["tflops"] = round(args.steps * L * B * 2 * d * F / (prof["gemm_up"][1] / 1e3) / 1e12, 1)
+    kernels["gemm_down"]["tflops"] = round(args.steps * L * B * 2 * d * F / (prof["gemm_down"][1] / 1e3) / 1e12, 1)
+    kernels["gemm_lm"]["tflops"] = round(args.steps * B * 2 * d * V / (prof["gemm_lm"][1] / 1e3) / 1e12, 1)
+    kernels["mixer"]["gbs"] = round(mixer_bytes / (prof["mixer"][1] / 1e3) / 1e9, 1)
+    kernels["select"]["gbs"] = round(args.steps * B * V * 4 / (prof["select"][1] / 1e3) / 1e9, 1)
+
+    # ---- end to end through the host-buffer call: H2D tokens in, D2H tokens out, every step ----
+    h_in = st.last_token().cpu().pin_memory()
+    h_out = torch.empty_like(h_in).pin_memory()
+    for _ in range(2):
+        if st.pos >= shape.n_ctx:
+            st.pos = n
+        model.decode_step_host(st, h_in, samp, step_no[0], h_out, ws); step_no[0] += 1
+        torch.cuda.synchronize(); h_in.copy_(h_out)
+    sync_all()
+    e0.record()
+    for _ in range(args.steps):
+        if st.pos >= shape.n_ctx:
+            st.pos = n
+        model.decode_step_host(st, h_in, samp, step_no[0], h_out, ws); step_no[0] += 1
+        torch.cuda.current_stream().synchronize()      # the next step's input is this step's output
+        h_in.copy_(h_out)
+    e1.record()
+    torch.cuda.synchronize()
+    te = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.barrier()
+        dist.all_reduce(te, op=dist.ReduceOp.MAX)
+    e2e_value = world * B * args.steps / (te.item() / 1e3)
+    status = st.status()
+
+    if rank == 0:
+        free_b, total_b = torch.cuda.mem_get_info()
+        per_sample = L * d * sbytes + 4 * w["gen"] + 4
+        fixed = model.blob.numel() + ws.numel()
+        max_conc = int((total_b * 0.97 - fixed) // per_sample)
+        clocks = clk.summary()
+        cpu = cpu_baseline(shape, W, args.workload, w) if world == 1 and not args.no_cpu_baseline else None
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": t_ms_max / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if shape.dtype == "bf16" else "f32",
+            "data": "synthetic",
+            "config": _config_dict(args, shape, w, B, extra={
+                "state_dtype": args.state_dtype, "chunk_rows": chunk,
+                "l2": f"inputs larger than L2: per-step working set (cache {L * B * d * sbytes / 1e6:.0f} MB + weights "
+                      f"{model.blob.numel() / 1e6:.0f} MB + logits {chunk * V * 4 / 1e6:.0f} MB) vs 126 MB L2; no flush"}),
+            "gpu_launches": int(launches),
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": B * 4, "d2h_bytes_per_step": B * 4},
+            "roofline": {"bound": "tensor", "kernel": "gemm_tc_kernel (feed-forward up/down + LM head)",
+                         "achieved": round(achieved_tf, 1), "peak": peak_tf, "unit": "TFLOP/s",
+                         "frac": round(achieved_tf / peak_tf, 4), "peak_source": f"bf16_tflops_sustained, {peak_src}",
+                         "frac_of_burst_peak": round(achieved_tf / peaks["bf16_tflops"], 4),
+                         "launches": int(gemm_launches), "traffic": GEMM_DRAM_TRAFFIC_PER_STEP,
+                         "flops_per_step": B * step_flops(shape)},
+            "step_roofline": {"bound": bound, "t_roof_ms": round(t_roof * 1e3, 4), "t_tensor_ms": round(t_tc * 1e3, 4),
+                              "t_hbm_ms": round(t_hbm * 1e3, 4), "frac": round(t_roof * 1e3 / (t_ms_max / args.steps), 4),
+                              "peaks": f"{peak_src}: {peak_tf} TFLOP/s sustained bf16, {peaks['hbm_gbs']} GB/s HBM"},
+            "kernels": kernels,
+            "prefill": {"ms": round(prefill_ms, 2), "prompt_tokens_per_s": round(B * n / (prefill_ms / 1e3), 1)},
+            "state_bytes_per_sample": L * d * sbytes,
+            "max_concurrent_samples": max_conc,
+            "device_status": status,
+            "cpu_baseline": cpu,
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def run_sweep(args):
+    """tokens/s vs batch on the mid model plus the largest batch that fits (128-token prompts,
+    256 generated tokens per sample budgeted in the token store)."""
+    import torch
+    import paper_2605_08696_b200 as P
+    import srm_inputs as I
+    w = I.WORKLOADS["sweep"]
+    shape = I.CONFIGS[w["model"]]
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    W = I.make_weights(shape)
+    model = P.SRM(shape, W, device=dev, state_dtype=args.state_dtype)
+    g = P.Sampling("greedy")
+    sbytes = 2 if args.state_dtype == "bf16" else 4
+    L, d = shape.n_layers, shape.d_model
+    chunk = args.chunk
+    ws = model.new_workspace(chunk, w["prompt_len"], prefill_samples=max(1, args.prefill_rows // w["prompt_len"]))
+    free_b, total_b = torch.cuda.mem_get_info()
+    per_sample = L * d * sbytes + 4 * w["gen"] + 4 + 4 * w["prompt_len"]
+    max_conc = int((free_b * 0.97) // per_sample)
+    batches = [1, 64, 1024, 8192, 32768]
+    while batches[-1] * 2 <= max_conc:
+        batches.append(batches[-1] * 2)
+    if args.sweep_max:
+        batches = [b for b in batches if b <= args.sweep_max]
+    curve = []
+    for B in batches:
+        st = model.new_state(B)
+        prompts = torch.from_numpy(I.uniform_prompts(min(B, 65536), w["prompt_len"], shape.vocab, shape.seed)).to(dev)
+        if B > prompts.shape[0]:
+            prompts = prompts.repeat((B + prompts.shape[0] - 1) // prompts.shape[0], 1)[:B].contiguous()
+        model.prefill(st, prompts, g, ws)
+        steps = 8 if B >= 262144 else 24
+        for _ in range(3):
+            model.decode_step(st, None, g, 1, ws)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(steps):
+            model.decode_step(st, None, g, 1, ws)
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / steps
+        curve.append({"batch": B, "ms_per_step": round(ms, 4), "tokens_per_s": round(B / (ms / 1e3), 1),
+                      "state_bytes_per_sample": L * d * sbytes, "status": st.status()})
+        print(json.dumps(curve[-1]), file=sys.stderr, flush=True)
+        del st, prompts
+        torch.cuda.empty_cache()
+    line = {"metric": METRIC, "unit": UNIT, "n_gpus": 1, "sweep": curve, "max_concurrent_samples": max_conc,
+            "state_dtype": args.state_dtype, "config": {"workload": "sweep: mid SRM, 128-token uniform prompts"}}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=64)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="mid", choices=["tiny", "small", "mid", "rl"])
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's batch per GPU")
+    ap.add_argument("--chunk", type=int, default=8192, help="samples per decode pass (workspace size)")
+    ap.add_argument("--prefill-rows", type=int, default=65536, help="prompt rows per prefill pass")
+    ap.add_argument("--state-dtype", default="fp32", choices=["fp32", "bf16"])
+    ap.add_argument("--ref-samples", type=int, default=32)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true")
+    ap.add_argument("--sweep-max", type=int, default=0)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    elif args.sweep:
+        run_sweep(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,242 @@
+/*
+ * srm.h — C ABI of the B200-native Structured Recurrent Mixer (SRM) decode library.
+ *
+ * What the library computes (paper sections in brackets):
+ *   - the recurrent-form decode step over a batch of B independent samples: per layer a
+ *     token-mixer cache update [Method/Architecture, Eq. 2 (row-repeat heads) and Eq. 3
+ *     (column-repeat heads), "mixed" heads], then the channel-mixing feed-forward, then
+ *     the LM head and token selection [Recurrent Throughput and Concurrency];
+ *   - the sequence-parallel form over a prompt, which yields the same cache
+ *     [Method/Architecture, Eq. 1 and Eq. 3; "either recurrent or sequence parallel
+ *     operations without any change to the underlying cache structure"].
+ *
+ * Conventions
+ *   - Every pointer named d_* is a DEVICE pointer, 16-byte aligned unless stated; h_* is a
+ *     HOST pointer. The library allocates no device memory: weights, state, workspace and
+ *     token buffers are allocated by the caller and only borrowed. They must stay valid
+ *     until the handle that borrowed them is destroyed (weights: srm_destroy; state buffer:
+ *     srm_state_destroy; workspace and token buffers: until the stream work of the call ends).
+ *   - `stream` is a cudaStream_t passed as void*. All device work is enqueued on it and the
+ *     calls return without synchronising, except where stated.
+ *   - All functions return 0 (SRM_OK) or a negative srm_error. No exceptions, no global
+ *     mutable state besides the last CUDA error code. Handles are not thread-safe; distinct
+ *     handles may be used from distinct threads.
+ *   - Matrices are row-major [out, in]. Positions are absolute, 0-based; all samples of a
+ *     state share one position counter.
+ *   - The CUDA device current at srm_create is the one the handles belong to.
+ */
+#ifndef SRM_H_
+#define SRM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct srm_model srm_model;   /* opaque host object; borrows the weight blob      */
+typedef struct srm_state srm_state;   /* opaque host object; borrows the state buffer     */
+
+enum srm_error {
+  SRM_OK = 0,
+  SRM_ERR_INVALID_ARG = -1,          /* null pointer, non-positive size, bad enum          */
+  SRM_ERR_UNSUPPORTED = -2,          /* shape outside what the kernels support             */
+  SRM_ERR_ALIGNMENT = -3,            /* a device pointer is not 16-byte (blob: 256) aligned */
+  SRM_ERR_BUFFER_TOO_SMALL = -4,     /* weights / state / workspace smaller than required  */
+  SRM_ERR_CTX_OVERFLOW = -5,         /* position would reach n_ctx (alpha, beta end there) */
+  SRM_ERR_CUDA = -6,                 /* a CUDA call failed; see srm_last_cuda_error        */
+  SRM_ERR_DEVICE_STATUS = -7         /* srm_status found device-side flags set             */
+};
+
+/* Bits of the device status word (srm_status). Kernels never trap: they clamp, flag, go on. */
+enum srm_status_bits {
+  SRM_STATUS_TOKEN_RANGE = 1u,       /* a token id was outside [0, vocab); it was clamped  */
+  SRM_STATUS_WAIT_TIMEOUT = 2u,      /* a bounded pipeline wait inside a GEMM gave up      */
+  SRM_STATUS_NONFINITE = 4u          /* the sampler met a non-finite logit                 */
+};
+
+enum { SRM_DTYPE_FP32 = 0, SRM_DTYPE_BF16 = 1 };
+enum { SRM_SELECT_GREEDY = 0, SRM_SELECT_TOPK = 1 };
+enum { SRM_FLAG_SIMT_GEMM = 1 };     /* debug: run the bf16 GEMMs on the plain SIMT kernel  */
+
+/* Model description. Heads g < n_heads/2 are row-repeat, the rest column-repeat. */
+typedef struct {
+  int32_t n_layers;      /* L >= 1                                                        */
+  int32_t d_model;       /* d, multiple of 64, <= 2048                                    */
+  int32_t n_heads;       /* h, even, d % (4h) == 0                                        */
+  int32_t ffn_mult;      /* F = ffn_mult * d                                              */
+  int32_t vocab;         /* V, multiple of 8                                              */
+  int32_t n_ctx;         /* positions for which alpha/beta exist                          */
+  int32_t dtype;         /* SRM_DTYPE_FP32: fp32 weights, plain fp32 FMA everywhere;
+                            SRM_DTYPE_BF16: bf16 matrices and GEMM inputs, fp32 accumulate,
+                            fp32 residual stream, norms and mixer arithmetic              */
+  int32_t state_dtype;   /* storage type of the cache: SRM_DTYPE_FP32 or SRM_DTYPE_BF16    */
+  float   ln_eps;        /* LayerNorm epsilon                                             */
+  int32_t flags;         /* SRM_FLAG_* (0 in production)                                  */
+} srm_config;
+
+/* Token selection. Greedy: smallest id among the maxima. Top-k: keep the top_k largest logits
+ * ordered by (logit desc, id asc), weights exp((l - l_max)/temperature), inverse-CDF draw with
+ * u = (r >> 8) * 2^-24 where r is the first word of Philox4x32-10 with key (seed lo, seed hi)
+ * and counter (sample_idx_base + b, step, 0, 0); 1 <= top_k <= 256. */
+typedef struct {
+  int32_t  mode;             /* SRM_SELECT_*                                               */
+  int32_t  top_k;
+  float    temperature;
+  int32_t  reserved;
+  uint64_t seed;
+  uint64_t sample_idx_base;  /* Philox sample index of row 0 of the state                  */
+} srm_sampling;
+
+/* ---- sizes and weight-blob layout ------------------------------------------------------- */
+
+/* Tensors of the weight blob, in blob order. Small vectors are always fp32; the four matrices
+ * (E, W1, W2, W_LM) are fp32 or bf16 per config.dtype. Every tensor starts 256-byte aligned. */
+enum srm_tensor {
+  SRM_T_E = 0,        /* [V, d]    embedding (global: layer = -1)                          */
+  SRM_T_LN1_G, SRM_T_LN1_B,          /* [d]  norm before the token mixer                   */
+  SRM_T_ALPHA,        /* [h, n_ctx] repeated mixing weights alpha                          */
+  SRM_T_BETA,         /* [n_ctx, d] per-position bias beta                                 */
+  SRM_T_LAMBDA,       /* [h]       decay constants in (0.9, 1]                             */
+  SRM_T_LN2_G, SRM_T_LN2_B,          /* [d]  norm before the feed-forward                  */
+  SRM_T_W1,           /* [F, d]    up projection                                           */
+  SRM_T_B1,           /* [F]                                                               */
+  SRM_T_W2,           /* [d, F]    down projection                                         */
+  SRM_T_B2,           /* [d]                                                               */
+  SRM_T_LNF_G, SRM_T_LNF_B,          /* [d]  final norm (global)                           */
+  SRM_T_W_LM,         /* [V, d]    LM head, no bias (global)                               */
+  SRM_T_COUNT
+};
+
+/* Total bytes of the weight blob, 0 if the config is invalid. */
+size_t srm_weights_bytes(const srm_config* cfg);
+/* Byte offset, byte size and element size of one tensor inside the blob (layer ignored for
+ * the global tensors). Lets a caller fill the blob without knowing the layout rule. */
+int srm_weight_slot(const srm_config* cfg, int32_t layer, int32_t tensor,
+                    size_t* offset, size_t* nbytes, int32_t* elem_bytes);
+/* Bytes of the state buffer for B samples: a 256-byte header (status word, counters), the
+ * last selected token int32[B], then the cache [L, B, d] in state_dtype. */
+size_t srm_state_bytes(const srm_config* cfg, int64_t B);
+/* Workspace bytes so that decode processes `B_chunk` samples per pass and prefill handles
+ * prompts of up to `n_prefill_max` tokens in one pass of at least one sample. Calls accept any
+ * workspace at least this large for B_chunk = 1 and split the batch into as many passes as
+ * the given workspace requires. */
+size_t srm_workspace_bytes(const srm_config* cfg, int64_t B_chunk, int32_t n_prefill_max);
+
+/* ---- handles ------------------------------------------------------------------------------ */
+
+/* Validates cfg, records tensor addresses inside the caller's blob (256-byte aligned,
+ * nbytes >= srm_weights_bytes) and prepares TMA descriptors for the weight matrices. */
+int srm_create(const srm_config* cfg, const void* d_weights, size_t nbytes, srm_model** out);
+int srm_destroy(srm_model* m);
+
+/* Binds a caller buffer of >= srm_state_bytes(cfg, B) bytes as the state of B samples and
+ * enqueues its zero-fill (cache = 0, position = 0) on `stream`. */
+int srm_state_create(srm_model* m, int64_t B, void* d_state, size_t nbytes, void* stream,
+                     srm_state** out);
+int srm_state_destroy(srm_state* s);
+int srm_state_reset(srm_state* s, void* stream);
+/* Position bookkeeping (host side): number of tokens consumed so far. */
+int64_t srm_state_pos(const srm_state* s);
+int srm_state_set_pos(srm_state* s, int64_t pos);
+/* Device address of the cache slab of one layer, [B, d] in state_dtype (for checkpointing
+ * and tests), and of the last-token vector int32[B]. */
+void* srm_state_layer_ptr(const srm_state* s, int32_t layer);
+int32_t* srm_state_last_token_ptr(const srm_state* s);
+/* Synchronises `stream`, copies the device status word to *flags and clears it.
+ * Returns SRM_ERR_DEVICE_STATUS when any bit was set. */
+int srm_status(srm_state* s, void* stream, uint32_t* flags);
+
+/* ---- the hot path ------------------------------------------------------------------------- */
+
+/* Sequence-parallel prefill [Eq. 1, Eq. 3]: consumes d_tokens[B, n] (row-major int32) at
+ * positions 0..n-1 of a freshly reset state, leaves the cache that position n reads and
+ * pos = n, and selects generated token 0 from the logits of position n-1 (Philox step 0).
+ * d_first_tok int32[B] and d_logits_last float[B, V] may be NULL. */
+int srm_prefill(srm_model* m, srm_state* s, const int32_t* d_tokens, int32_t n,
+                const srm_sampling* sampling, int32_t* d_first_tok, float* d_logits_last,
+                void* d_ws, size_t ws_bytes, void* stream);
+
+/* One recurrent decode step [Eq. 2, Eq. 3]: consumes d_tok_in[B] (NULL: the token selected
+ * by the previous call) at position pos, updates the cache, pos += 1, and selects the next
+ * token with Philox step `step`. d_tok_out int32[B] and d_logits_out float[B, V] may be NULL. */
+int srm_decode_step(srm_model* m, srm_state* s, const int32_t* d_tok_in,
+                    const srm_sampling* sampling, int32_t step, int32_t* d_tok_out,
+                    float* d_logits_out, void* d_ws, size_t ws_bytes, void* stream);
+
+/* Generation loop: `steps` decode steps, each consuming the previously selected token
+ * (the one left by srm_prefill or the previous step). Step j (0-based) writes its selection
+ * to d_out[b * out_stride + j] and uses Philox step first_step + j. No host synchronisation
+ * between steps. Fails with SRM_ERR_CTX_OVERFLOW before enqueuing anything if
+ * pos + steps > n_ctx. */
+int srm_generate(srm_model* m, srm_state* s, int32_t steps, int32_t first_step,
+                 const srm_sampling* sampling, int32_t* d_out, int64_t out_stride,
+                 void* d_ws, size_t ws_bytes, void* stream);
+
+/* Same step as srm_decode_step with HOST token buffers (pinned memory recommended):
+ * copies h_tok_in[B] to the device, runs the step, copies the selection to h_tok_out[B], all
+ * on `stream`; the caller synchronises the stream before reading h_tok_out. */
+int srm_decode_step_host(srm_model* m, srm_state* s, const int32_t* h_tok_in,
+                         const srm_sampling* sampling, int32_t step, int32_t* h_tok_out,
+                         void* d_ws, size_t ws_bytes, void* stream);
+
+/* ---- single kernels, exported for unit parity tests and profiling ------------------------- */
+
+/* Fused token-mixer step of one layer on R rows at position t [Eq. 2, Eq. 3]:
+ *   x <- (d_tok != NULL ? E[tok] : x);  z = LN1(x);  y, S' = mixer(z, S, t);  x <- x + y;
+ *   a = LN2(x) in the activation type of cfg.dtype.
+ * d_x float[R, d] in/out, d_S [R, d] in state_dtype in/out, d_a [R, d] out. */
+int srm_k_mixer_step(srm_model* m, int32_t layer, int32_t t, int64_t R, const int32_t* d_tok,
+                     float* d_x, void* d_S, void* d_a, uint32_t* d_status, void* stream);
+/* out = LN_f(x) in the activation type: d_x float[R, d] -> d_a [R, d]. */
+int srm_k_final_norm(srm_model* m, int64_t R, const float* d_x, void* d_a, void* stream);
+/* Dense projection D[M, N] = A[M, K] * W[N, K]^T with one of three epilogues:
+ *   0: out_act[M, N] = gelu_erf(D + bias)      (activation type)
+ *   1: out_f32[M, N] += D + bias               (fp32 residual stream)
+ *   2: out_f32[M, N] = D                       (fp32 logits)
+ * A, W in the activation type of cfg.dtype; bf16 runs on the tcgen05 tensor-core kernel
+ * (or the SIMT kernel when cfg.flags has SRM_FLAG_SIMT_GEMM), fp32 on the SIMT kernel. */
+int srm_k_gemm(srm_model* m, int32_t epilogue, int64_t M, int64_t N, int64_t K, const void* d_A,
+               const void* d_W, const float* d_bias, void* d_out, uint32_t* d_status,
+               void* stream);
+/* Token selection on d_logits float[R, V] -> d_tok int32[R]; row r uses sample index
+ * sampling->sample_idx_base + r. */
+int srm_k_select(srm_model* m, int64_t R, const float* d_logits, const srm_sampling* sampling,
+                 int32_t step, int32_t* d_tok, uint32_t* d_status, void* stream);
+/* Sequence-parallel token mixing of one layer for Bp samples of n positions [Eq. 1, Eq. 3]:
+ * x[Bp*n, d] in/out (row = b*n + position), a[Bp*n, d] out, cache S[Bp, d] out (the sum term
+ * position n reads). d_tok (int32[Bp*n]) non-NULL: rows start from the embedding. */
+int srm_k_prefill_mixer(srm_model* m, int32_t layer, int64_t Bp, int32_t n, const int32_t* d_tok,
+                        float* d_x, void* d_S, void* d_a, uint32_t* d_status, void* stream);
+
+/* ---- measurement -------------------------------------------------------------------------- */
+enum srm_kernel_class {
+  SRM_KERNEL_MIXER = 0,          /* fused recurrent token-mixer step                           */
+  SRM_KERNEL_GEMM_UP,            /* feed-forward up projection (+bias, GELU)                   */
+  SRM_KERNEL_GEMM_DOWN,          /* feed-forward down projection (+bias, residual)             */
+  SRM_KERNEL_GEMM_LM,            /* LM head                                                    */
+  SRM_KERNEL_NORM,               /* final norm                                                 */
+  SRM_KERNEL_SELECT,             /* token selection                                            */
+  SRM_KERNEL_PREFILL_MIXER,      /* sequence-parallel token mixing                             */
+  SRM_KERNEL_CLASS_COUNT
+};
+/* While enabled, every kernel launch of this model is bracketed by two CUDA events recorded on the
+ * launching stream (events are created on first need and reused; no device memory). */
+int srm_profile_enable(srm_model* m, int on);
+/* Waits for the recorded events, folds them into per-class totals and returns the number of
+ * launches and the summed device time (ms) of one class since the last reset. */
+int srm_profile_read(srm_model* m, int32_t kernel_class, uint64_t* launches, double* total_ms);
+int srm_profile_reset(srm_model* m);
+/* Number of kernels this library has launched since it was loaded (all models). */
+uint64_t srm_kernel_launches(void);
+
+/* ---- diagnostics -------------------------------------------------------------------------- */
+const char* srm_strerror(int code);
+int srm_last_cuda_error(void);        /* cudaError_t of the most recent SRM_ERR_CUDA       */
+const char* srm_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SRM_H_ */

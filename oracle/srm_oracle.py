@@ -61,7 +61,7 @@ def head_kinds(n_heads: int):
 
 
 def mixer_parallel(Z: np.ndarray, alpha: np.ndarray, beta: np.ndarray, lam: np.ndarray,
-                   n_heads: int):
+                   n_heads: int, matrices=None):
     """Sequence-parallel token mixing of one layer for one sample.
 
     Z[n, d] are the (normed) inputs, one row per position. For head g with channel
@@ -69,6 +69,8 @@ def mixer_parallel(Z: np.ndarray, alpha: np.ndarray, beta: np.ndarray, lam: np.n
     Also returns the hand-off cache S_n[d], i.e. the sum term of Eq. 2 / Eq. 3 that
     position n would use:  row heads  S_n = sum_{m<n} lam^(n-m) alpha[m] z_m,
                            col heads  S_n = sum_{m<n} lam^(n-m) z_m.
+    `matrices` may hold the per-head M already built by mixing_matrix for this n (they do
+    not depend on the sample).
     """
     n, d = Z.shape
     dh = d // n_heads
@@ -77,7 +79,7 @@ def mixer_parallel(Z: np.ndarray, alpha: np.ndarray, beta: np.ndarray, lam: np.n
     S = np.zeros(d, dtype=Z.dtype)
     for g, kind in enumerate(head_kinds(n_heads)):
         c = slice(g * dh, (g + 1) * dh)
-        M = mixing_matrix(kind, alpha[g], lam[g], n, dtype=dt)
+        M = matrices[g] if matrices is not None else mixing_matrix(kind, alpha[g], lam[g], n, dtype=dt)
         X = Z[:, c].T                               # d_h x n, columns = positions
         Y[:, c] = (X @ M).T + beta[:n, c]
         for m in range(n):
@@ -239,8 +241,10 @@ class SRMOracle:
         for l, lw in enumerate(self.layers):
             z = layer_norm(x, lw["ln1_g"], lw["ln1_b"], self.eps)
             y = np.empty_like(z)
+            Ms = [mixing_matrix(kind, lw["alpha"][g], lw["lam"][g], n, dtype=self.dt)
+                  for g, kind in enumerate(head_kinds(self.h))]
             for b in range(B):
-                y[b], state[l, b] = mixer_parallel(z[b], lw["alpha"], lw["beta"], lw["lam"], self.h)
+                y[b], state[l, b] = mixer_parallel(z[b], lw["alpha"], lw["beta"], lw["lam"], self.h, Ms)
             x = x + y
             a = layer_norm(x, lw["ln2_g"], lw["ln2_b"], self.eps)
             x = x + feed_forward(a, lw["W1"], lw["b1"], lw["W2"], lw["b2"])

@@ -1,0 +1,8 @@
+"""B200-native (sm_100a) Structured Recurrent Mixer decode path.
+
+`binding` is a thin ctypes layer over the C-ABI library libsrm.so (include/srm.h): it marshals
+torch device buffers and streams into the calls, nothing else. All arithmetic of the path runs
+in the CUDA kernels under csrc/.
+"""
+from .binding import (SRM, SRMState, Sampling, SRMError, load_library, lib_path,  # noqa: F401
+                      EPI_BIAS_GELU, EPI_BIAS_RESIDUAL, EPI_PLAIN)

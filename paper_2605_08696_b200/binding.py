@@ -1,0 +1,346 @@
+"""ctypes binding of libsrm.so. Argument marshalling only.
+
+Device memory and streams come from torch; every function below passes raw pointers and sizes
+to the C ABI declared in include/srm.h and raises SRMError on a non-zero return code.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+import numpy as np
+import torch
+
+from . import build as _build
+
+EPI_BIAS_GELU, EPI_BIAS_RESIDUAL, EPI_PLAIN = 0, 1, 2
+DTYPE_FP32, DTYPE_BF16 = 0, 1
+FLAG_SIMT_GEMM = 1
+
+# enum srm_tensor
+T_E, T_LN1_G, T_LN1_B, T_ALPHA, T_BETA, T_LAMBDA, T_LN2_G, T_LN2_B, T_W1, T_B1, T_W2, T_B2, \
+    T_LNF_G, T_LNF_B, T_W_LM = range(15)
+_LAYER_TENSORS = {"ln1_g": T_LN1_G, "ln1_b": T_LN1_B, "alpha": T_ALPHA, "beta": T_BETA, "lam": T_LAMBDA,
+                  "ln2_g": T_LN2_G, "ln2_b": T_LN2_B, "W1": T_W1, "b1": T_B1, "W2": T_W2, "b2": T_B2}
+_GLOBAL_TENSORS = {"E": T_E, "lnf_g": T_LNF_G, "lnf_b": T_LNF_B, "W_lm": T_W_LM}
+
+
+class SRMError(RuntimeError):
+    def __init__(self, code, where):
+        self.code = code
+        msg = _lib().srm_strerror(code).decode() if _LIB is not None else "?"
+        extra = f" (cudaError {_lib().srm_last_cuda_error()})" if code == -6 else ""
+        super().__init__(f"{where}: {msg}{extra} [{code}]")
+
+
+class _Config(C.Structure):
+    _fields_ = [("n_layers", C.c_int32), ("d_model", C.c_int32), ("n_heads", C.c_int32),
+                ("ffn_mult", C.c_int32), ("vocab", C.c_int32), ("n_ctx", C.c_int32),
+                ("dtype", C.c_int32), ("state_dtype", C.c_int32), ("ln_eps", C.c_float),
+                ("flags", C.c_int32)]
+
+
+class _Sampling(C.Structure):
+    _fields_ = [("mode", C.c_int32), ("top_k", C.c_int32), ("temperature", C.c_float),
+                ("reserved", C.c_int32), ("seed", C.c_uint64), ("sample_idx_base", C.c_uint64)]
+
+
+@dataclass
+class Sampling:
+    mode: str = "greedy"          # "greedy" or "topk"
+    top_k: int = 50
+    temperature: float = 1.0
+    seed: int = 0
+    sample_idx_base: int = 0
+
+    def c(self) -> _Sampling:
+        return _Sampling(0 if self.mode == "greedy" else 1, self.top_k, self.temperature, 0,
+                         self.seed & 0xFFFFFFFFFFFFFFFF, self.sample_idx_base)
+
+
+_LIB = None
+
+# every symbol include/srm.h declares: (name, restype, argtypes)
+_P, _I32, _I64, _SZ = C.c_void_p, C.c_int32, C.c_int64, C.c_size_t
+SYMBOLS = {
+    "srm_weights_bytes": (_SZ, [C.POINTER(_Config)]),
+    "srm_weight_slot": (C.c_int, [C.POINTER(_Config), _I32, _I32, C.POINTER(_SZ), C.POINTER(_SZ), C.POINTER(_I32)]),
+    "srm_state_bytes": (_SZ, [C.POINTER(_Config), _I64]),
+    "srm_workspace_bytes": (_SZ, [C.POINTER(_Config), _I64, _I32]),
+    "srm_create": (C.c_int, [C.POINTER(_Config), _P, _SZ, C.POINTER(_P)]),
+    "srm_destroy": (C.c_int, [_P]),
+    "srm_state_create": (C.c_int, [_P, _I64, _P, _SZ, _P, C.POINTER(_P)]),
+    "srm_state_destroy": (C.c_int, [_P]),
+    "srm_state_reset": (C.c_int, [_P, _P]),
+    "srm_state_pos": (_I64, [_P]),
+    "srm_state_set_pos": (C.c_int, [_P, _I64]),
+    "srm_state_layer_ptr": (_P, [_P, _I32]),
+    "srm_state_last_token_ptr": (_P, [_P]),
+    "srm_status": (C.c_int, [_P, _P, C.POINTER(C.c_uint32)]),
+    "srm_prefill": (C.c_int, [_P, _P, _P, _I32, C.POINTER(_Sampling), _P, _P, _P, _SZ, _P]),
+    "srm_decode_step": (C.c_int, [_P, _P, _P, C.POINTER(_Sampling), _I32, _P, _P, _P, _SZ, _P]),
+    "srm_generate": (C.c_int, [_P, _P, _I32, _I32, C.POINTER(_Sampling), _P, _I64, _P, _SZ, _P]),
+    "srm_decode_step_host": (C.c_int, [_P, _P, _P, C.POINTER(_Sampling), _I32, _P, _P, _SZ, _P]),
+    "srm_k_mixer_step": (C.c_int, [_P, _I32, _I32, _I64, _P, _P, _P, _P, _P, _P]),
+    "srm_k_final_norm": (C.c_int, [_P, _I64, _P, _P, _P]),
+    "srm_k_gemm": (C.c_int, [_P, _I32, _I64, _I64, _I64, _P, _P, _P, _P, _P, _P]),
+    "srm_k_select": (C.c_int, [_P, _I64, _P, C.POINTER(_Sampling), _I32, _P, _P, _P]),
+    "srm_k_prefill_mixer": (C.c_int, [_P, _I32, _I64, _I32, _P, _P, _P, _P, _P, _P]),
+    "srm_profile_enable": (C.c_int, [_P, C.c_int]),
+    "srm_profile_read": (C.c_int, [_P, _I32, C.POINTER(C.c_uint64), C.POINTER(C.c_double)]),
+    "srm_profile_reset": (C.c_int, [_P]),
+    "srm_kernel_launches": (C.c_uint64, []),
+    "srm_strerror": (C.c_char_p, [C.c_int]),
+    "srm_last_cuda_error": (C.c_int, []),
+    "srm_version": (C.c_char_p, []),
+}
+
+
+def lib_path() -> str:
+    return _build.LIB_PATH
+
+
+def load_library(build_if_missing: bool = True):
+    """Load libsrm.so (building it with nvcc when absent or stale). There is no fallback:
+    without the CUDA library nothing in this package can run."""
+    global _LIB
+    if _LIB is not None:
+        return _LIB
+    if build_if_missing and _build.needs_build():
+        _build.build_library()
+    if not os.path.exists(_build.LIB_PATH):
+        raise ImportError(f"{_build.LIB_PATH} is missing; run paper_2605_08696_b200/build.py")
+    lib = C.CDLL(_build.LIB_PATH)
+    for name, (res, args) in SYMBOLS.items():
+        fn = getattr(lib, name)          # AttributeError if the symbol is not exported
+        fn.restype, fn.argtypes = res, args
+    _LIB = lib
+    return lib
+
+
+def _lib():
+    return load_library()
+
+
+def _check(code, where):
+    if code != 0:
+        raise SRMError(code, where)
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    assert t.is_contiguous(), "tensor must be contiguous"
+    return C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _shape_get(shape, key):
+    return shape[key] if isinstance(shape, dict) else getattr(shape, key)
+
+
+class SRMState:
+    """Cache of B samples (device buffer owned here as a torch tensor, borrowed by the library)."""
+
+    def __init__(self, model: "SRM", B: int):
+        self.model, self.B = model, B
+        nbytes = _lib().srm_state_bytes(C.byref(model.cfg), B)
+        if nbytes == 0:
+            raise SRMError(-1, "srm_state_bytes")
+        self.buf = torch.empty(nbytes, dtype=torch.uint8, device=model.device)
+        self.handle = C.c_void_p()
+        _check(_lib().srm_state_create(model.handle, B, _ptr(self.buf), nbytes, _stream(), C.byref(self.handle)),
+               "srm_state_create")
+
+    def __del__(self):
+        if getattr(self, "handle", None) and _LIB is not None:
+            _LIB.srm_state_destroy(self.handle)
+            self.handle = None
+
+    @property
+    def pos(self) -> int:
+        return _lib().srm_state_pos(self.handle)
+
+    @pos.setter
+    def pos(self, v: int):
+        _check(_lib().srm_state_set_pos(self.handle, v), "srm_state_set_pos")
+
+    def reset(self):
+        _check(_lib().srm_state_reset(self.handle, _stream()), "srm_state_reset")
+
+    def status(self) -> int:
+        """Synchronises, returns and clears the device status word."""
+        f = C.c_uint32(0)
+        rc = _lib().srm_status(self.handle, _stream(), C.byref(f))
+        if rc not in (0, -7):
+            raise SRMError(rc, "srm_status")
+        return f.value
+
+    def layer(self, l: int) -> torch.Tensor:
+        """View of the cache slab of one layer, [B, d] in the state dtype."""
+        m = self.model
+        ptr = _lib().srm_state_layer_ptr(self.handle, l)
+        off = ptr - self.buf.data_ptr()
+        es = 2 if m.cfg.state_dtype == DTYPE_BF16 else 4
+        dt = torch.bfloat16 if es == 2 else torch.float32
+        n = self.B * m.cfg.d_model
+        return self.buf[off: off + n * es].view(dt).view(self.B, m.cfg.d_model)
+
+    def cache(self) -> torch.Tensor:
+        """[L, B, d] copy of the whole cache in fp32."""
+        return torch.stack([self.layer(l).float() for l in range(self.model.cfg.n_layers)])
+
+    def last_token(self) -> torch.Tensor:
+        off = _lib().srm_state_last_token_ptr(self.handle) - self.buf.data_ptr()
+        return self.buf[off: off + 4 * self.B].view(torch.int32)
+
+
+class SRM:
+    """Model handle: packs the weight dict into the library's blob layout and owns the blob."""
+
+    def __init__(self, shape, weights: dict, device: str = "cuda:0", state_dtype: str = "fp32", flags: int = 0):
+        lib = _lib()
+        dt = _shape_get(shape, "dtype")
+        self.cfg = _Config(_shape_get(shape, "n_layers"), _shape_get(shape, "d_model"), _shape_get(shape, "n_heads"),
+                           _shape_get(shape, "ffn_mult"), _shape_get(shape, "vocab"), _shape_get(shape, "n_ctx"),
+                           DTYPE_BF16 if dt == "bf16" else DTYPE_FP32,
+                           DTYPE_BF16 if state_dtype == "bf16" else DTYPE_FP32,
+                           _shape_get(shape, "ln_eps"), flags)
+        self.device = torch.device(device)
+        self.act_dtype = torch.bfloat16 if dt == "bf16" else torch.float32
+        nbytes = lib.srm_weights_bytes(C.byref(self.cfg))
+        if nbytes == 0:
+            raise SRMError(-2, "srm_weights_bytes")
+        host = torch.zeros(nbytes, dtype=torch.uint8)
+        self._slots = {}
+
+        def put(layer, tid, arr):
+            off, nb, eb = _SZ(), _SZ(), _I32()
+            _check(lib.srm_weight_slot(C.byref(self.cfg), layer, tid, C.byref(off), C.byref(nb), C.byref(eb)),
+                   "srm_weight_slot")
+            t = torch.from_numpy(np.ascontiguousarray(arr, dtype=np.float32))
+            t = t.to(torch.bfloat16) if eb.value == 2 else t
+            raw = t.contiguous().view(torch.uint8).reshape(-1)
+            assert raw.numel() == nb.value, (layer, tid, raw.numel(), nb.value)
+            host[off.value: off.value + nb.value] = raw
+            self._slots[(layer, tid)] = (off.value, nb.value, eb.value, tuple(t.shape))
+
+        for name, tid in _GLOBAL_TENSORS.items():
+            put(-1, tid, weights[name])
+        for l, lw in enumerate(weights["layers"]):
+            for name, tid in _LAYER_TENSORS.items():
+                put(l, tid, lw[name])
+        with torch.cuda.device(self.device):
+            self.blob = host.to(self.device)
+            self.handle = C.c_void_p()
+            _check(lib.srm_create(C.byref(self.cfg), _ptr(self.blob), nbytes, C.byref(self.handle)), "srm_create")
+
+    def __del__(self):
+        if getattr(self, "handle", None) and _LIB is not None:
+            _LIB.srm_destroy(self.handle)
+            self.handle = None
+
+    # ---- buffers ----
+    def tensor(self, layer: int, tid: int) -> torch.Tensor:
+        """Device view of one tensor of the blob."""
+        off, nb, eb, shp = self._slots[(layer, tid)]
+        dt = torch.bfloat16 if eb == 2 else torch.float32
+        return self.blob[off: off + nb].view(dt).view(shp)
+
+    def new_state(self, B: int) -> SRMState:
+        return SRMState(self, B)
+
+    def workspace_bytes(self, B_chunk: int, n_prefill: int = 0) -> int:
+        return _lib().srm_workspace_bytes(C.byref(self.cfg), B_chunk, n_prefill)
+
+    def new_workspace(self, B_chunk: int, n_prefill: int = 0, prefill_samples: int = 1) -> torch.Tensor:
+        nb = max(self.workspace_bytes(B_chunk, 0), prefill_samples * self.workspace_bytes(1, n_prefill) if n_prefill else 0)
+        return torch.empty(nb, dtype=torch.uint8, device=self.device)
+
+    # ---- hot path ----
+    def prefill(self, state: SRMState, tokens: torch.Tensor, sampling: Sampling, ws: torch.Tensor,
+                want_logits: bool = False):
+        B, n = tokens.shape
+        assert B == state.B and tokens.dtype == torch.int32
+        first = torch.empty(B, dtype=torch.int32, device=self.device)
+        logits = torch.empty(B, self.cfg.vocab, dtype=torch.float32, device=self.device) if want_logits else None
+        s = sampling.c()
+        _check(_lib().srm_prefill(self.handle, state.handle, _ptr(tokens), n, C.byref(s), _ptr(first), _ptr(logits),
+                                  _ptr(ws), ws.numel(), _stream()), "srm_prefill")
+        return (first, logits) if want_logits else first
+
+    def decode_step(self, state: SRMState, tok_in, sampling: Sampling, step: int, ws: torch.Tensor,
+                    want_logits: bool = False, tok_out: torch.Tensor | None = None):
+        if tok_out is None:
+            tok_out = torch.empty(state.B, dtype=torch.int32, device=self.device)
+        logits = torch.empty(state.B, self.cfg.vocab, dtype=torch.float32, device=self.device) if want_logits else None
+        s = sampling.c()
+        _check(_lib().srm_decode_step(self.handle, state.handle, _ptr(tok_in), C.byref(s), step, _ptr(tok_out),
+                                      _ptr(logits), _ptr(ws), ws.numel(), _stream()), "srm_decode_step")
+        return (tok_out, logits) if want_logits else tok_out
+
+    def generate(self, state: SRMState, steps: int, first_step: int, sampling: Sampling, ws: torch.Tensor,
+                 out: torch.Tensor | None = None) -> torch.Tensor:
+        if out is None:
+            out = torch.empty(state.B, steps, dtype=torch.int32, device=self.device)
+        s = sampling.c()
+        _check(_lib().srm_generate(self.handle, state.handle, steps, first_step, C.byref(s), _ptr(out), out.stride(0),
+                                   _ptr(ws), ws.numel(), _stream()), "srm_generate")
+        return out
+
+    def decode_step_host(self, state: SRMState, h_tok_in: torch.Tensor, sampling: Sampling, step: int,
+                         h_tok_out: torch.Tensor, ws: torch.Tensor):
+        """Host-buffer variant: h_tok_in / h_tok_out are CPU int32 tensors (pinned for async copies)."""
+        assert not h_tok_in.is_cuda and not h_tok_out.is_cuda
+        s = sampling.c()
+        _check(_lib().srm_decode_step_host(self.handle, state.handle, _ptr(h_tok_in), C.byref(s), step,
+                                           _ptr(h_tok_out), _ptr(ws), ws.numel(), _stream()), "srm_decode_step_host")
+
+    # ---- measurement ----
+    KERNEL_CLASSES = ("mixer", "gemm_up", "gemm_down", "gemm_lm", "norm", "select", "prefill_mixer")
+
+    def profile(self, on: bool):
+        _check(_lib().srm_profile_enable(self.handle, int(on)), "srm_profile_enable")
+
+    def profile_reset(self):
+        _check(_lib().srm_profile_reset(self.handle), "srm_profile_reset")
+
+    def profile_read(self) -> dict:
+        """{class name: (launches, total device ms)} since the last reset."""
+        out = {}
+        for i, name in enumerate(self.KERNEL_CLASSES):
+            n, ms = C.c_uint64(), C.c_double()
+            _check(_lib().srm_profile_read(self.handle, i, C.byref(n), C.byref(ms)), "srm_profile_read")
+            out[name] = (n.value, ms.value)
+        return out
+
+    @staticmethod
+    def kernel_launches() -> int:
+        return _lib().srm_kernel_launches()
+
+    # ---- single kernels ----
+    def k_mixer_step(self, layer, t, x, S, a, tok=None, status=None):
+        _check(_lib().srm_k_mixer_step(self.handle, layer, t, x.shape[0], _ptr(tok), _ptr(x), _ptr(S), _ptr(a),
+                                       _ptr(status), _stream()), "srm_k_mixer_step")
+
+    def k_final_norm(self, x, a):
+        _check(_lib().srm_k_final_norm(self.handle, x.shape[0], _ptr(x), _ptr(a), _stream()), "srm_k_final_norm")
+
+    def k_gemm(self, epilogue, A, W, bias, out, status=None):
+        M, K = A.shape
+        N = W.shape[0]
+        _check(_lib().srm_k_gemm(self.handle, epilogue, M, N, K, _ptr(A), _ptr(W), _ptr(bias), _ptr(out),
+                                 _ptr(status), _stream()), "srm_k_gemm")
+
+    def k_select(self, logits, sampling: Sampling, step, tok, status=None):
+        s = sampling.c()
+        _check(_lib().srm_k_select(self.handle, logits.shape[0], _ptr(logits), C.byref(s), step, _ptr(tok),
+                                   _ptr(status), _stream()), "srm_k_select")
+
+    def k_prefill_mixer(self, layer, Bp, n, x, S, a, tok=None, status=None):
+        _check(_lib().srm_k_prefill_mixer(self.handle, layer, Bp, n, _ptr(tok), _ptr(x), _ptr(S), _ptr(a),
+                                          _ptr(status), _stream()), "srm_k_prefill_mixer")

@@ -1,0 +1,61 @@
+"""Builds libsrm.so (the C-ABI CUDA library) in-tree with nvcc for sm_100a."""
+from __future__ import annotations
+
+import os
+import shutil
+import subprocess
+import sys
+
+PKG_DIR = os.path.dirname(os.path.abspath(__file__))
+CSRC = os.path.join(PKG_DIR, "csrc")
+LIB_PATH = os.path.join(PKG_DIR, "libsrm.so")
+
+NVCC_FLAGS = [
+    "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+    "-Xptxas=-v",
+    "-shared", "-Xcompiler", "-fPIC", "-cudart", "static",
+]
+
+
+def _sources():
+    return sorted(os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cu", ".cuh")))
+
+
+def _source_hash() -> str:
+    import hashlib
+    h = hashlib.sha256()
+    for s in _sources() + [os.path.join(os.path.dirname(PKG_DIR), "include", "srm.h")]:
+        with open(s, "rb") as f:
+            h.update(f.read())
+    h.update(" ".join(NVCC_FLAGS).encode())
+    return h.hexdigest()
+
+
+def needs_build() -> bool:
+    """True when libsrm.so is missing or was built from different sources."""
+    if not os.path.exists(LIB_PATH) or not os.path.exists(LIB_PATH + ".srchash"):
+        return True
+    with open(LIB_PATH + ".srchash") as f:
+        return f.read().strip() != _source_hash()
+
+
+def build_library(force: bool = False, verbose: bool = False) -> str:
+    """Compile csrc/srm_api.cu (which includes every kernel header) into libsrm.so."""
+    if not force and not needs_build():
+        return LIB_PATH
+    nvcc = shutil.which("nvcc") or "/usr/local/cuda/bin/nvcc"
+    cmd = [nvcc] + NVCC_FLAGS + ["-o", LIB_PATH, os.path.join(CSRC, "srm_api.cu")]
+    res = subprocess.run(cmd, capture_output=True, text=True)
+    if verbose or res.returncode != 0:
+        sys.stderr.write(res.stdout + res.stderr)
+    if res.returncode != 0:
+        raise RuntimeError("nvcc failed building libsrm.so")
+    with open(os.path.join(PKG_DIR, "ptxas_report.txt"), "w") as f:
+        f.write(res.stderr)
+    with open(LIB_PATH + ".srchash", "w") as f:
+        f.write(_source_hash())
+    return LIB_PATH
+
+
+if __name__ == "__main__":
+    print(build_library(force=True, verbose="-v" in sys.argv))

@@ -1,0 +1,163 @@
+// Sequence-parallel token mixing over a prompt (Method/Architecture, Eq. 1 and Eq. 3).
+//
+// One CTA owns one sample and walks its n positions in tiles of T positions. Inside a tile the
+// mixing is the explicit matrix product Y = Z M + B with the T x T diagonal block of M built
+// from alpha and lambda (row-repeat: M[i][j] = lambda^(j-i) alpha_i, column-repeat:
+// lambda^(j-i) alpha_j, i <= j). The blocks of M above the diagonal are rank one, so their
+// contribution is carried between tiles as the d-vector sum term of Eq. 2 / Eq. 3, which after
+// the last tile is exactly the cache the recurrent form continues from. With T >= n this is the
+// paper's full n x n product. LN1, the residual add and LN2 are fused around the mixing, so each
+// row of the residual stream is read once and written once per layer.
+#pragma once
+
+#include "common.cuh"
+#include "mixer.cuh"
+
+namespace srm {
+
+constexpr int kPrefillThreads = 256;
+constexpr int kPrefillTile = 16;     // T
+constexpr int kPrefillMaxHeads = 8;
+constexpr int kPrefillMaxCPT = 8;    // channels per thread: d <= 2048
+
+struct PrefillParams {
+  float* x;              // [Bp*n, d] in/out
+  const int32_t* tok;    // [Bp*n] or nullptr
+  const void* E;
+  void* S;               // [Bp, d] out (state type)
+  void* a;               // [Bp*n, d] out (activation type)
+  const float* ln1_g; const float* ln1_b;
+  const float* ln2_g; const float* ln2_b;
+  const float* alpha; const float* beta; const float* lam;
+  int64_t Bp;
+  int n, d, h, n_ctx, vocab;
+  float eps;
+  uint32_t* status;
+};
+
+template <typename WT, typename ST>
+__global__ void __launch_bounds__(kPrefillThreads) prefill_mixer_kernel(const PrefillParams p) {
+  constexpr int T = kPrefillTile;
+  extern __shared__ float xs[];                       // [T][d] tile of the residual stream
+  __shared__ float Mt[kPrefillMaxHeads][T][T];        // diagonal block of M per head
+  __shared__ float pw[kPrefillMaxHeads][T + 1];       // lambda^k
+  __shared__ float al[kPrefillMaxHeads][T];           // alpha of the tile's positions
+  __shared__ float mu[T], rs[T];                      // LN1 statistics of the tile's rows
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int d = p.d, n = p.n, h = p.h, dh = d / h, h_row = h >> 1;
+  const int64_t b = blockIdx.x;
+  if (b >= p.Bp) return;
+
+  for (int i = tid; i < h * (T + 1); i += kPrefillThreads) {
+    const int g = i / (T + 1), k = i % (T + 1);
+    pw[g][k] = powf(__ldg(p.lam + g), (float)k);
+  }
+  float carry[kPrefillMaxCPT];
+#pragma unroll
+  for (int q = 0; q < kPrefillMaxCPT; ++q) carry[q] = 0.f;
+
+  for (int j0 = 0; j0 < n; j0 += T) {
+    const int rows = min(T, n - j0);
+    const int64_t row0 = b * n + j0;
+    __syncthreads();     // previous tile fully written back before xs / Mt are overwritten
+    // ---- load the tile (embedding rows for the first layer) ----
+    if (p.tok != nullptr) {
+      for (int r = warp; r < rows; r += kPrefillThreads / 32) {
+        int tk = p.tok[row0 + r];
+        if (tk < 0 || tk >= p.vocab) {
+          if (lane == 0) raise_status(p.status, kStatusTokenRange);
+          tk = tk < 0 ? 0 : p.vocab - 1;
+        }
+        const WT* e = reinterpret_cast<const WT*>(p.E) + (int64_t)tk * d;
+        for (int c = lane * 4; c < d; c += 128) st4(xs + r * d + c, ldg4(e + c));
+      }
+    } else {
+      const float* src = p.x + row0 * d;
+      for (int i = tid * 4; i < rows * d; i += kPrefillThreads * 4) st4(xs + i, ld4(src + i));
+    }
+    for (int i = tid; i < h * T; i += kPrefillThreads) {
+      const int g = i / T, r = i % T;
+      al[g][r] = (r < rows) ? __ldg(p.alpha + (int64_t)g * p.n_ctx + j0 + r) : 0.f;
+    }
+    __syncthreads();
+    // ---- diagonal block of M, and LN1 statistics (one warp per row) ----
+    for (int i = tid; i < h * T * T; i += kPrefillThreads) {
+      const int g = i / (T * T), r = (i / T) % T, c = i % T;     // M[r][c]: input r -> output c
+      float m = 0.f;
+      if (r <= c) m = pw[g][c - r] * (g < h_row ? al[g][r] : al[g][c]);
+      Mt[g][r][c] = m;
+    }
+    for (int r = warp; r < rows; r += kPrefillThreads / 32) {
+      const float* xr = xs + r * d;
+      float s = 0.f;
+      for (int c = lane; c < d; c += 32) s += xr[c];
+      const float mean = warp_sum(s) / (float)d;
+      float q = 0.f;
+      for (int c = lane; c < d; c += 32) { const float t = xr[c] - mean; q += t * t; }
+      const float rstd = rsqrtf(warp_sum(q) / (float)d + p.eps);
+      if (lane == 0) { mu[r] = mean; rs[r] = rstd; }
+    }
+    __syncthreads();
+    // ---- mixing: one thread per channel; z_i recomputed from x, mean, rstd ----
+#pragma unroll
+    for (int q = 0; q < kPrefillMaxCPT; ++q) {
+      const int c = tid + q * kPrefillThreads;
+      if (c < d) {
+        const int g = c / dh;
+        const bool is_row = g < h_row;
+        const float gg = __ldg(p.ln1_g + c), bb = __ldg(p.ln1_b + c);
+        float z[T];
+#pragma unroll
+        for (int i = 0; i < T; ++i) z[i] = (i < rows) ? (xs[i * d + c] - mu[i]) * rs[i] * gg + bb : 0.f;
+        const float S0 = carry[q];
+#pragma unroll
+        for (int j = 0; j < T; ++j) {
+          if (j < rows) {
+            float acc = 0.f;
+#pragma unroll
+            for (int i = 0; i <= j; ++i) acc = fmaf(z[i], Mt[g][i][j], acc);
+            // rank-one blocks above the diagonal, folded into the carried sum term
+            const float tail = pw[g][j] * S0;
+            acc += is_row ? tail : al[g][j] * tail;
+            acc += __ldg(p.beta + (int64_t)(j0 + j) * d + c);
+            xs[j * d + c] += acc;
+          }
+        }
+        // sum term for the position after this tile
+        float sn = pw[g][rows] * S0;
+#pragma unroll
+        for (int i = 0; i < T; ++i) {
+          if (i < rows) sn = fmaf(pw[g][rows - i] * (is_row ? al[g][i] : 1.f), z[i], sn);
+        }
+        carry[q] = sn;
+      }
+    }
+    __syncthreads();
+    // ---- LN2 and write-back (one warp per row) ----
+    for (int r = warp; r < rows; r += kPrefillThreads / 32) {
+      const float* xr = xs + r * d;
+      float s = 0.f;
+      for (int c = lane; c < d; c += 32) s += xr[c];
+      const float mean = warp_sum(s) / (float)d;
+      float q = 0.f;
+      for (int c = lane; c < d; c += 32) { const float t = xr[c] - mean; q += t * t; }
+      const float rstd = rsqrtf(warp_sum(q) / (float)d + p.eps);
+      float* xo = p.x + (row0 + r) * d;
+      WT* ao = reinterpret_cast<WT*>(p.a) + (row0 + r) * d;
+      for (int c = lane * 4; c < d; c += 128) {
+        const float4 v = ld4(xr + c);
+        st4(xo + c, v);
+        st4(ao + c, norm4(v, mean, rstd, ldg4(p.ln2_g + c), ldg4(p.ln2_b + c)));
+      }
+    }
+  }
+  ST* So = reinterpret_cast<ST*>(p.S) + b * d;
+#pragma unroll
+  for (int q = 0; q < kPrefillMaxCPT; ++q) {
+    const int c = tid + q * kPrefillThreads;
+    if (c < d) So[c] = from_float<ST>(carry[q]);
+  }
+}
+
+}  // namespace srm

@@ -1,0 +1,220 @@
+// Token selection over the vocabulary: greedy argmax (lowest id among ties) and
+// temperature / top-k sampling keyed by Philox4x32-10(seed; sample, step).
+// One 256-thread block per sample row; warp-shuffle reductions; the row is streamed with
+// 128-bit loads (and staged once in shared memory for the multi-pass top-k selection).
+#pragma once
+
+#include "common.cuh"
+
+namespace srm {
+
+constexpr int kSelThreads = 256;
+constexpr int kTopKMax = 256;
+
+struct SelectOut {
+  int32_t* last_tok;    // [R] always written (state's "previous selection")
+  int32_t* tok_out;     // [R] or nullptr
+  int32_t* store;       // token store base or nullptr: store[row * store_stride + store_col]
+  int64_t store_stride;
+  int64_t store_col;
+};
+
+__device__ __forceinline__ void write_token(const SelectOut& o, int64_t row, int tok) {
+  o.last_tok[row] = tok;
+  if (o.tok_out != nullptr) o.tok_out[row] = tok;
+  if (o.store != nullptr) o.store[row * o.store_stride + o.store_col] = tok;
+}
+
+// ---- greedy -------------------------------------------------------------------------------
+__device__ __forceinline__ void argmax_take(float v, int i, float& bv, int& bi) {
+  if (v > bv || (v == bv && i < bi)) { bv = v; bi = i; }
+}
+
+__global__ void __launch_bounds__(kSelThreads)
+select_greedy_kernel(const float* __restrict__ logits, int64_t R, int V, SelectOut out, uint32_t* status) {
+  const int64_t row = blockIdx.x;
+  if (row >= R) return;
+  const float* lr = logits + row * (int64_t)V;
+  float bv = -INFINITY;
+  int bi = 0x7fffffff;
+  bool bad = false;
+  for (int i = threadIdx.x * 4; i < V; i += kSelThreads * 4) {
+    const float4 v = *reinterpret_cast<const float4*>(lr + i);
+    bad |= !(v.x == v.x) | !(v.y == v.y) | !(v.z == v.z) | !(v.w == v.w);
+    argmax_take(v.x, i, bv, bi); argmax_take(v.y, i + 1, bv, bi);
+    argmax_take(v.z, i + 2, bv, bi); argmax_take(v.w, i + 3, bv, bi);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+    const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+    argmax_take(ov, oi, bv, bi);
+  }
+  __shared__ float sv[kSelThreads / 32];
+  __shared__ int si[kSelThreads / 32];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (lane == 0) { sv[warp] = bv; si[warp] = bi; }
+  if (bad) raise_status(status, kStatusNonFinite);
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < kSelThreads / 32; ++w) argmax_take(sv[w], si[w], bv, bi);
+    if (bi < 0 || bi >= V) bi = 0;       // all-NaN row
+    write_token(out, row, bi);
+  }
+}
+
+// ---- Philox4x32-10 (Salmon et al., SC'11) ---------------------------------------------------
+__device__ __forceinline__ uint32_t philox4x32_10_word0(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                                        uint32_t k0, uint32_t k1) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+    c0 = hi1 ^ c1 ^ k0; c1 = lo1; c2 = hi0 ^ c3 ^ k1; c3 = lo0;
+    k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+  }
+  return c0;
+}
+
+// order-preserving map float -> uint32 (larger float, larger key) and back
+__device__ __forceinline__ uint32_t order_key(float f) {
+  const uint32_t u = __float_as_uint(f);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float key_value(uint32_t k) {
+  return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
+
+// ---- top-k + temperature + inverse-CDF draw ------------------------------------------------
+// 1. radix-select (4 passes of 8 bits) the key of the k-th largest logit;
+// 2. collect everything above it, plus the lowest ids among the ties at it;
+// 3. bitonic-sort the <= 256 candidates by (logit desc, id asc);
+// 4. one thread accumulates w_i = exp((l_i - l_0)/T) in that order and picks the first
+//    cumulative weight exceeding u * total.
+template <bool ROW_IN_SMEM>
+__global__ void __launch_bounds__(kSelThreads)
+select_topk_kernel(const float* __restrict__ logits, int64_t R, int V, int k, float inv_temp, uint64_t seed,
+                   uint64_t sample_base, int step, SelectOut out, uint32_t* status) {
+  extern __shared__ float srow[];
+  __shared__ uint32_t hist[256];
+  __shared__ unsigned long long cand[kTopKMax];
+  __shared__ uint32_t sh_prefix, sh_need, sh_ties, sh_count, sh_running;
+  __shared__ uint32_t warp_cnt[kSelThreads / 32];
+
+  const int64_t row = blockIdx.x;
+  if (row >= R) return;
+  const float* lr = logits + row * (int64_t)V;
+  const int tid = threadIdx.x;
+  bool bad = false;
+  if (ROW_IN_SMEM) {
+    for (int i = tid * 4; i < V; i += kSelThreads * 4) {
+      const float4 v = *reinterpret_cast<const float4*>(lr + i);
+      bad |= !(v.x == v.x) | !(v.y == v.y) | !(v.z == v.z) | !(v.w == v.w);
+      *reinterpret_cast<float4*>(srow + i) = v;
+    }
+  }
+  if (bad) raise_status(status, kStatusNonFinite);
+  const float* src = ROW_IN_SMEM ? srow : lr;
+  if (tid == 0) { sh_prefix = 0; sh_need = (uint32_t)k; sh_count = 0; sh_running = 0; }
+  __syncthreads();
+
+  uint32_t mask = 0;
+  for (int shift = 24; shift >= 0; shift -= 8) {
+    hist[tid] = 0;
+    __syncthreads();
+    const uint32_t prefix = sh_prefix;
+    for (int i = tid; i < V; i += kSelThreads) {
+      const uint32_t key = order_key(src[i]);
+      if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+    }
+    __syncthreads();
+    if (tid == 0) {
+      uint32_t need = sh_need, cum = 0;
+      int digit = 0;
+      for (int b = 255; b >= 0; --b) {
+        if (cum + hist[b] >= need) { digit = b; break; }
+        cum += hist[b];
+      }
+      sh_need = need - cum;              // how many still to take inside this digit
+      sh_prefix = prefix | ((uint32_t)digit << shift);
+      sh_ties = hist[digit];             // after the last pass: number of keys equal to the threshold
+    }
+    mask |= 255u << shift;
+    __syncthreads();
+  }
+  const uint32_t thr = sh_prefix, need_ties = sh_need, ties = sh_ties;
+  const uint32_t n_above = (uint32_t)k - need_ties;
+
+  // keys strictly above the threshold: order does not matter (sorted below)
+  for (int i = tid; i < V; i += kSelThreads) {
+    const uint32_t key = order_key(src[i]);
+    if (key > thr || (key == thr && ties == need_ties)) {
+      const uint32_t slot = atomicAdd(&sh_count, 1u);
+      if (slot < (uint32_t)kTopKMax) cand[slot] = ((unsigned long long)(~key) << 32) | (uint32_t)i;
+    }
+  }
+  if (ties != need_ties) {
+    // more ties than places: take the lowest ids, found by a block-wide ordered scan
+    const int warp = tid >> 5, lane = tid & 31;
+    for (int base = 0; base < V; base += kSelThreads) {
+      const int i = base + tid;
+      const bool f = (i < V) && (order_key(src[i]) == thr);
+      const uint32_t bal = __ballot_sync(0xffffffffu, f);
+      if (lane == 0) warp_cnt[warp] = __popc(bal);
+      __syncthreads();
+      uint32_t off = sh_running;
+      for (int w = 0; w < warp; ++w) off += warp_cnt[w];
+      off += __popc(bal & ((1u << lane) - 1u));
+      if (f && off < need_ties) cand[n_above + off] = ((unsigned long long)(~thr) << 32) | (uint32_t)i;
+      __syncthreads();
+      if (tid == 0) {
+        uint32_t t = 0;
+        for (int w = 0; w < kSelThreads / 32; ++w) t += warp_cnt[w];
+        sh_running += t;
+      }
+      __syncthreads();
+      if (sh_running >= need_ties) break;
+    }
+  }
+  __syncthreads();
+  // pad to a power of two and sort ascending by (~key, id) = (logit desc, id asc)
+  int P = 1;
+  while (P < k) P <<= 1;
+  if (tid >= k && tid < P) cand[tid] = ~0ull;
+  __syncthreads();
+  for (int size = 2; size <= P; size <<= 1) {
+    for (int stride = size >> 1; stride > 0; stride >>= 1) {
+      if (tid < P) {
+        const int j = tid ^ stride;
+        if (j > tid) {
+          const unsigned long long a = cand[tid], b = cand[j];
+          const bool up = (tid & size) == 0;
+          if ((a > b) == up) { cand[tid] = b; cand[j] = a; }
+        }
+      }
+      __syncthreads();
+    }
+  }
+  if (tid == 0) {
+    const float l0 = key_value(~(uint32_t)(cand[0] >> 32));
+    float* cdf = reinterpret_cast<float*>(hist);     // reuse: k <= 256 floats
+    float c = 0.f;
+    for (int i = 0; i < k; ++i) {
+      const float li = key_value(~(uint32_t)(cand[i] >> 32));
+      c += expf((li - l0) * inv_temp);
+      cdf[i] = c;
+    }
+    const uint64_t sidx = sample_base + (uint64_t)row;
+    const uint32_t r = philox4x32_10_word0((uint32_t)sidx, (uint32_t)step, 0u, 0u, (uint32_t)seed,
+                                           (uint32_t)(seed >> 32));
+    const float u = (float)(r >> 8) * (1.0f / 16777216.0f);
+    const float target = u * c;
+    int pick = k - 1;
+    for (int i = 0; i < k; ++i) {
+      if (cdf[i] > target) { pick = i; break; }
+    }
+    write_token(out, row, (int)(uint32_t)(cand[pick] & 0xffffffffull));
+  }
+}
+
+}  // namespace srm

@@ -1,0 +1,782 @@
+// Host runtime and C ABI of the SRM decode library (see include/srm.h for the contract).
+// Everything here is argument checking, buffer carving and kernel launches; all arithmetic
+// of the path runs in the kernels included below.
+#include "../../include/srm.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+#include <new>
+#include <vector>
+
+#include "common.cuh"
+#include "gemm_simt.cuh"
+#include "gemm_tc.cuh"
+#include "mixer.cuh"
+#include "prefill.cuh"
+#include "select.cuh"
+
+using namespace srm;
+
+namespace {
+
+int g_last_cuda_error = 0;
+
+#define SRM_CUDA(expr)                                  \
+  do {                                                  \
+    cudaError_t e__ = (expr);                           \
+    if (e__ != cudaSuccess) {                           \
+      g_last_cuda_error = (int)e__;                     \
+      return SRM_ERR_CUDA;                              \
+    }                                                   \
+  } while (0)
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+struct Slot { size_t off = 0, bytes = 0; int elem = 4; };
+
+struct Layout {
+  Slot global[SRM_T_COUNT];
+  std::vector<Slot> layer;     // [L][SRM_T_COUNT]
+  size_t total = 0;
+};
+
+bool is_global_tensor(int t) { return t == SRM_T_E || t == SRM_T_LNF_G || t == SRM_T_LNF_B || t == SRM_T_W_LM; }
+
+bool config_ok(const srm_config* c) {
+  if (c == nullptr) return false;
+  if (c->n_layers < 1 || c->d_model < 64 || c->d_model > 2048 || c->d_model % 64) return false;
+  if (c->n_heads < 2 || c->n_heads > kPrefillMaxHeads || c->n_heads % 2 || c->d_model % (4 * c->n_heads)) return false;
+  if (c->ffn_mult < 1 || c->vocab < 8 || c->vocab % 8 || c->n_ctx < 1) return false;
+  if (c->dtype != SRM_DTYPE_FP32 && c->dtype != SRM_DTYPE_BF16) return false;
+  if (c->state_dtype != SRM_DTYPE_FP32 && c->state_dtype != SRM_DTYPE_BF16) return false;
+  if (!(c->ln_eps > 0.f)) return false;
+  return true;
+}
+
+size_t tensor_elems(const srm_config& c, int t) {
+  const size_t d = c.d_model, F = (size_t)c.ffn_mult * d, V = c.vocab, n = c.n_ctx, h = c.n_heads;
+  switch (t) {
+    case SRM_T_E: case SRM_T_W_LM: return V * d;
+    case SRM_T_ALPHA: return h * n;
+    case SRM_T_BETA: return n * d;
+    case SRM_T_LAMBDA: return h;
+    case SRM_T_W1: case SRM_T_W2: return F * d;
+    case SRM_T_B1: return F;
+    default: return d;
+  }
+}
+
+Layout make_layout(const srm_config& c) {
+  Layout L;
+  const int wbytes = c.dtype == SRM_DTYPE_BF16 ? 2 : 4;
+  auto is_matrix = [](int t) { return t == SRM_T_E || t == SRM_T_W1 || t == SRM_T_W2 || t == SRM_T_W_LM; };
+  size_t off = 0;
+  auto place = [&](int t) {
+    Slot s;
+    s.elem = is_matrix(t) ? wbytes : 4;
+    s.bytes = tensor_elems(c, t) * s.elem;
+    s.off = off;
+    off = align_up(off + s.bytes, 256);
+    return s;
+  };
+  L.global[SRM_T_E] = place(SRM_T_E);
+  L.layer.resize((size_t)c.n_layers * SRM_T_COUNT);
+  for (int l = 0; l < c.n_layers; ++l)
+    for (int t = SRM_T_LN1_G; t <= SRM_T_B2; ++t) L.layer[(size_t)l * SRM_T_COUNT + t] = place(t);
+  L.global[SRM_T_LNF_G] = place(SRM_T_LNF_G);
+  L.global[SRM_T_LNF_B] = place(SRM_T_LNF_B);
+  L.global[SRM_T_W_LM] = place(SRM_T_W_LM);
+  L.total = off;
+  return L;
+}
+
+// ---- TMA descriptors ------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  });
+  return fn;
+}
+
+// bf16 row-major [rows, cols] matrix, box = 64 columns (128 bytes, the swizzle span) x box_rows.
+int make_tmap_bf16(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int box_rows) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (fn == nullptr) { g_last_cuda_error = (int)cudaErrorNotSupported; return SRM_ERR_CUDA; }
+  cuuint64_t gdim[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t gstride[1] = {(cuuint64_t)cols * 2};
+  cuuint32_t box[2] = {(cuuint32_t)tc::BK, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstride, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) { g_last_cuda_error = 10000 + (int)r; return SRM_ERR_CUDA; }
+  return SRM_OK;
+}
+
+struct TmapCacheEntry { const void* base; int64_t rows, cols; int box_rows; CUtensorMap map; };
+
+unsigned long long g_kernel_launches = 0;     // kernels launched by this library since load
+
+struct ProfRecord { cudaEvent_t start, stop; int cls; };
+
+}  // namespace
+
+struct srm_model {
+  srm_config cfg;
+  const uint8_t* w;
+  Layout layout;
+  int device = 0;
+  int num_sms = 0;
+  bool tc_ready = false;                 // smem attribute set for the tensor-core kernels
+  std::vector<TmapCacheEntry> tmaps;     // weight and activation descriptors, built on first use
+  bool profiling = false;                // bracket every launch with CUDA events on its stream
+  std::vector<ProfRecord> prof;          // open records, folded into the totals by srm_profile_read
+  std::vector<cudaEvent_t> event_pool;
+  unsigned long long prof_launches[SRM_KERNEL_CLASS_COUNT] = {};
+  double prof_ms[SRM_KERNEL_CLASS_COUNT] = {};
+
+  const void* ptr(int layer, int t) const {
+    const Slot& s = is_global_tensor(t) ? layout.global[t] : layout.layer[(size_t)layer * SRM_T_COUNT + t];
+    return w + s.off;
+  }
+  const float* fptr(int layer, int t) const { return reinterpret_cast<const float*>(ptr(layer, t)); }
+  int act_bytes() const { return cfg.dtype == SRM_DTYPE_BF16 ? 2 : 4; }
+  int state_bytes() const { return cfg.state_dtype == SRM_DTYPE_BF16 ? 2 : 4; }
+  int64_t F() const { return (int64_t)cfg.ffn_mult * cfg.d_model; }
+
+  int tmap(const void* base, int64_t rows, int64_t cols, int box_rows, const CUtensorMap** out) {
+    for (auto& e : tmaps)
+      if (e.base == base && e.rows == rows && e.cols == cols && e.box_rows == box_rows) { *out = &e.map; return SRM_OK; }
+    if (tmaps.size() >= 4096) tmaps.clear();
+    TmapCacheEntry e{base, rows, cols, box_rows, {}};
+    int rc = make_tmap_bf16(&e.map, base, rows, cols, box_rows);
+    if (rc != SRM_OK) return rc;
+    tmaps.push_back(e);
+    *out = &tmaps.back().map;
+    return SRM_OK;
+  }
+};
+
+struct srm_state {
+  srm_model* m;
+  int64_t B;
+  uint8_t* base;
+  size_t nbytes;
+  uint32_t* status;       // device status word (header)
+  int32_t* last_tok;      // [B]
+  uint8_t* S;             // [L, B, d] in state dtype
+  int64_t pos;
+
+  void* layer_ptr(int l) const { return S + (size_t)l * B * m->cfg.d_model * m->state_bytes(); }
+};
+
+namespace {
+
+// Counts the launch and, when profiling is on, records an event before and after it.
+struct LaunchScope {
+  srm_model* m; cudaStream_t st; cudaEvent_t stop = nullptr;
+  LaunchScope(const srm_model& model, int cls, cudaStream_t stream) : m(const_cast<srm_model*>(&model)), st(stream) {
+    ++g_kernel_launches;
+    if (!m->profiling) return;
+    cudaEvent_t ev[2];
+    for (auto& e : ev) {
+      if (!m->event_pool.empty()) { e = m->event_pool.back(); m->event_pool.pop_back(); }
+      else if (cudaEventCreate(&e) != cudaSuccess) return;
+    }
+    cudaEventRecord(ev[0], st);
+    stop = ev[1];
+    m->prof.push_back(ProfRecord{ev[0], ev[1], cls});
+  }
+  ~LaunchScope() { if (stop != nullptr) cudaEventRecord(stop, st); }
+};
+
+constexpr size_t kStateHeader = 256;
+
+size_t state_bytes_for(const srm_config& c, int64_t B) {
+  const size_t sb = c.state_dtype == SRM_DTYPE_BF16 ? 2 : 4;
+  return kStateHeader + align_up((size_t)B * 4, 256) + (size_t)c.n_layers * B * c.d_model * sb;
+}
+
+// ---- workspace carving ----------------------------------------------------------------------
+struct DecodeWs { float* x; void* a; void* H; float* logits; int64_t rows; };
+struct PrefillWs { float* x; void* a; void* H; void* a_last; float* logits; int64_t samples; };
+
+size_t decode_ws_bytes(const srm_model& m, int64_t rows) {
+  const size_t d = m.cfg.d_model, F = m.F(), V = m.cfg.vocab, ab = m.act_bytes();
+  return align_up(rows * d * 4, 256) + align_up(rows * d * ab, 256) + align_up(rows * F * ab, 256) +
+         align_up(rows * V * 4, 256);
+}
+size_t prefill_ws_bytes(const srm_model& m, int64_t samples, int n) {
+  const size_t d = m.cfg.d_model, F = m.F(), V = m.cfg.vocab, ab = m.act_bytes(), rows = (size_t)samples * n;
+  return align_up(rows * d * 4, 256) + align_up(rows * d * ab, 256) + align_up(rows * F * ab, 256) +
+         align_up(samples * d * ab, 256) + align_up(samples * V * 4, 256);
+}
+int64_t fit_rows(size_t ws_bytes, int64_t want, size_t (*need)(const srm_model&, int64_t, int), const srm_model& m, int n) {
+  if (need(m, 1, n) > ws_bytes) return 0;
+  int64_t lo = 1, hi = want;            // largest r in [1, want] with need(r) <= ws_bytes
+  while (lo < hi) {
+    const int64_t mid = lo + (hi - lo + 1) / 2;
+    if (need(m, mid, n) <= ws_bytes) lo = mid; else hi = mid - 1;
+  }
+  return lo;
+}
+size_t decode_need(const srm_model& m, int64_t r, int) { return decode_ws_bytes(m, r); }
+size_t prefill_need(const srm_model& m, int64_t r, int n) { return prefill_ws_bytes(m, r, n); }
+
+DecodeWs carve_decode(const srm_model& m, void* ws, int64_t rows) {
+  const size_t d = m.cfg.d_model, F = m.F(), ab = m.act_bytes();
+  uint8_t* p = static_cast<uint8_t*>(ws);
+  DecodeWs w;
+  w.rows = rows;
+  w.x = reinterpret_cast<float*>(p); p += align_up(rows * d * 4, 256);
+  w.a = p; p += align_up(rows * d * ab, 256);
+  w.H = p; p += align_up(rows * F * ab, 256);
+  w.logits = reinterpret_cast<float*>(p);
+  return w;
+}
+PrefillWs carve_prefill(const srm_model& m, void* ws, int64_t samples, int n) {
+  const size_t d = m.cfg.d_model, F = m.F(), ab = m.act_bytes(), rows = (size_t)samples * n;
+  uint8_t* p = static_cast<uint8_t*>(ws);
+  PrefillWs w;
+  w.samples = samples;
+  w.x = reinterpret_cast<float*>(p); p += align_up(rows * d * 4, 256);
+  w.a = p; p += align_up(rows * d * ab, 256);
+  w.H = p; p += align_up(rows * F * ab, 256);
+  w.a_last = p; p += align_up(samples * d * ab, 256);
+  w.logits = reinterpret_cast<float*>(p);
+  return w;
+}
+
+// ---- kernel launchers -------------------------------------------------------------------------
+template <typename WT, typename ST>
+int launch_mixer_nv(const MixerParams& p, cudaStream_t st) {
+  const int nv = (p.d + 127) / 128;
+  const unsigned grid = (unsigned)((p.R + kMixerWarps - 1) / kMixerWarps);
+  const dim3 blk(kMixerWarps * 32);
+  if (nv <= 1) mixer_step_kernel<1, WT, ST><<<grid, blk, 0, st>>>(p);
+  else if (nv <= 2) mixer_step_kernel<2, WT, ST><<<grid, blk, 0, st>>>(p);
+  else if (nv <= 4) mixer_step_kernel<4, WT, ST><<<grid, blk, 0, st>>>(p);
+  else if (nv <= 6) mixer_step_kernel<6, WT, ST><<<grid, blk, 0, st>>>(p);
+  else if (nv <= 8) mixer_step_kernel<8, WT, ST><<<grid, blk, 0, st>>>(p);
+  else if (nv <= 12) mixer_step_kernel<12, WT, ST><<<grid, blk, 0, st>>>(p);
+  else mixer_step_kernel<16, WT, ST><<<grid, blk, 0, st>>>(p);
+  SRM_CUDA(cudaGetLastError());
+  return SRM_OK;
+}
+
+int launch_mixer(const srm_model& m, int layer, int t, int64_t R, const int32_t* tok, float* x, void* S, void* a,
+                 uint32_t* status, cudaStream_t st) {
+  if (R <= 0) return SRM_OK;
+  LaunchScope scope(m, SRM_KERNEL_MIXER, st);
+  MixerParams p;
+  p.x = x; p.tok = tok; p.E = m.ptr(-1, SRM_T_E); p.S = S; p.a = a;
+  p.ln1_g = m.fptr(layer, SRM_T_LN1_G); p.ln1_b = m.fptr(layer, SRM_T_LN1_B);
+  p.ln2_g = m.fptr(layer, SRM_T_LN2_G); p.ln2_b = m.fptr(layer, SRM_T_LN2_B);
+  p.alpha = m.fptr(layer, SRM_T_ALPHA); p.beta = m.fptr(layer, SRM_T_BETA); p.lam = m.fptr(layer, SRM_T_LAMBDA);
+  p.R = R; p.d = m.cfg.d_model; p.h = m.cfg.n_heads; p.n_ctx = m.cfg.n_ctx; p.t = t; p.vocab = m.cfg.vocab;
+  p.eps = m.cfg.ln_eps; p.status = status;
+  const bool wb = m.cfg.dtype == SRM_DTYPE_BF16, sb = m.cfg.state_dtype == SRM_DTYPE_BF16;
+  if (wb && sb) return launch_mixer_nv<bf16, bf16>(p, st);
+  if (wb) return launch_mixer_nv<bf16, float>(p, st);
+  if (sb) return launch_mixer_nv<float, bf16>(p, st);
+  return launch_mixer_nv<float, float>(p, st);
+}
+
+template <typename WT>
+int launch_norm_t(const float* x, int64_t R, int64_t stride, int64_t offset, const float* g, const float* b, float eps,
+                  int d, void* out, cudaStream_t st) {
+  const int nv = (d + 127) / 128;
+  const unsigned grid = (unsigned)((R + kMixerWarps - 1) / kMixerWarps);
+  const dim3 blk(kMixerWarps * 32);
+  WT* o = reinterpret_cast<WT*>(out);
+  if (nv <= 1) norm_rows_kernel<1, WT><<<grid, blk, 0, st>>>(x, R, stride, offset, g, b, eps, d, o);
+  else if (nv <= 2) norm_rows_kernel<2, WT><<<grid, blk, 0, st>>>(x, R, stride, offset, g, b, eps, d, o);
+  else if (nv <= 4) norm_rows_kernel<4, WT><<<grid, blk, 0, st>>>(x, R, stride, offset, g, b, eps, d, o);
+  else if (nv <= 6) norm_rows_kernel<6, WT><<<grid, blk, 0, st>>>(x, R, stride, offset, g, b, eps, d, o);
+  else if (nv <= 8) norm_rows_kernel<8, WT><<<grid, blk, 0, st>>>(x, R, stride, offset, g, b, eps, d, o);
+  else if (nv <= 12) norm_rows_kernel<12, WT><<<grid, blk, 0, st>>>(x, R, stride, offset, g, b, eps, d, o);
+  else norm_rows_kernel<16, WT><<<grid, blk, 0, st>>>(x, R, stride, offset, g, b, eps, d, o);
+  SRM_CUDA(cudaGetLastError());
+  return SRM_OK;
+}
+
+int launch_final_norm(const srm_model& m, const float* x, int64_t R, int64_t stride, int64_t offset, void* out,
+                      cudaStream_t st) {
+  if (R <= 0) return SRM_OK;
+  LaunchScope scope(m, SRM_KERNEL_NORM, st);
+  const float* g = m.fptr(-1, SRM_T_LNF_G);
+  const float* b = m.fptr(-1, SRM_T_LNF_B);
+  if (m.cfg.dtype == SRM_DTYPE_BF16) return launch_norm_t<bf16>(x, R, stride, offset, g, b, m.cfg.ln_eps, m.cfg.d_model, out, st);
+  return launch_norm_t<float>(x, R, stride, offset, g, b, m.cfg.ln_eps, m.cfg.d_model, out, st);
+}
+
+template <typename T>
+int launch_gemm_simt(int epi, int64_t M, int64_t N, int64_t K, const void* A, const void* W, const float* bias,
+                     void* out, cudaStream_t st) {
+  const dim3 grid((unsigned)((N + kSimtBN - 1) / kSimtBN), (unsigned)((M + kSimtBM - 1) / kSimtBM));
+  const T* a = reinterpret_cast<const T*>(A);
+  const T* w = reinterpret_cast<const T*>(W);
+  if (epi == kEpiBiasGelu) gemm_simt_kernel<T, kEpiBiasGelu><<<grid, 256, 0, st>>>(a, w, bias, out, M, N, K);
+  else if (epi == kEpiBiasResidual) gemm_simt_kernel<T, kEpiBiasResidual><<<grid, 256, 0, st>>>(a, w, bias, out, M, N, K);
+  else gemm_simt_kernel<T, kEpiPlain><<<grid, 256, 0, st>>>(a, w, bias, out, M, N, K);
+  SRM_CUDA(cudaGetLastError());
+  return SRM_OK;
+}
+
+int ensure_tc_ready(srm_model& m) {
+  if (m.tc_ready) return SRM_OK;
+  SRM_CUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<kEpiBiasGelu>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes));
+  SRM_CUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<kEpiBiasResidual>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes));
+  SRM_CUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<kEpiPlain>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes));
+  m.tc_ready = true;
+  return SRM_OK;
+}
+
+int launch_gemm_tc(srm_model& m, int epi, int64_t M, int64_t N, int64_t K, const void* A, const void* W,
+                   const float* bias, void* out, uint32_t* status, cudaStream_t st) {
+  int rc = ensure_tc_ready(m);
+  if (rc != SRM_OK) return rc;
+  const CUtensorMap *ta, *tb;
+  if ((rc = m.tmap(A, M, K, tc::BM, &ta)) != SRM_OK) return rc;
+  CUtensorMap a_copy = *ta;             // the cache may reallocate on the next insertion
+  if ((rc = m.tmap(W, N, K, tc::BN, &tb)) != SRM_OK) return rc;
+  tc::GemmArgs g{M, N, K, bias, out, status};
+  const int64_t tiles = ((M + tc::BM - 1) / tc::BM) * ((N + tc::BN - 1) / tc::BN);
+  const unsigned grid = (unsigned)(tiles < m.num_sms ? tiles : m.num_sms);
+  if (epi == kEpiBiasGelu) tc::gemm_tc_kernel<kEpiBiasGelu><<<grid, tc::kThreads, tc::kSmemBytes, st>>>(a_copy, *tb, g);
+  else if (epi == kEpiBiasResidual) tc::gemm_tc_kernel<kEpiBiasResidual><<<grid, tc::kThreads, tc::kSmemBytes, st>>>(a_copy, *tb, g);
+  else tc::gemm_tc_kernel<kEpiPlain><<<grid, tc::kThreads, tc::kSmemBytes, st>>>(a_copy, *tb, g);
+  SRM_CUDA(cudaGetLastError());
+  return SRM_OK;
+}
+
+int launch_gemm(srm_model& m, int epi, int64_t M, int64_t N, int64_t K, const void* A, const void* W,
+                const float* bias, void* out, uint32_t* status, cudaStream_t st) {
+  if (M <= 0) return SRM_OK;
+  LaunchScope scope(m, epi == kEpiBiasGelu ? SRM_KERNEL_GEMM_UP : epi == kEpiBiasResidual ? SRM_KERNEL_GEMM_DOWN : SRM_KERNEL_GEMM_LM, st);
+  if (m.cfg.dtype == SRM_DTYPE_FP32) return launch_gemm_simt<float>(epi, M, N, K, A, W, bias, out, st);
+  if (m.cfg.flags & SRM_FLAG_SIMT_GEMM) return launch_gemm_simt<bf16>(epi, M, N, K, A, W, bias, out, st);
+  return launch_gemm_tc(m, epi, M, N, K, A, W, bias, out, status, st);
+}
+
+int check_sampling(const srm_model& m, const srm_sampling* s) {
+  if (s == nullptr) return SRM_ERR_INVALID_ARG;
+  if (s->mode == SRM_SELECT_GREEDY) return SRM_OK;
+  if (s->mode != SRM_SELECT_TOPK) return SRM_ERR_INVALID_ARG;
+  if (s->top_k < 1 || s->top_k > kTopKMax || s->top_k > m.cfg.vocab || !(s->temperature > 0.f)) return SRM_ERR_INVALID_ARG;
+  return SRM_OK;
+}
+
+int launch_select(const srm_model& m, int64_t R, const float* logits, const srm_sampling& s, uint64_t sample_base,
+                  int step, const SelectOut& out, uint32_t* status, cudaStream_t st) {
+  if (R <= 0) return SRM_OK;
+  LaunchScope scope(m, SRM_KERNEL_SELECT, st);
+  const int V = m.cfg.vocab;
+  if (s.mode == SRM_SELECT_GREEDY) {
+    select_greedy_kernel<<<(unsigned)R, kSelThreads, 0, st>>>(logits, R, V, out, status);
+  } else {
+    const size_t row_bytes = (size_t)V * 4;
+    const float inv_t = 1.0f / s.temperature;
+    if (row_bytes <= 160 * 1024) {
+      static bool attr_set = false;
+      if (!attr_set) {
+        SRM_CUDA(cudaFuncSetAttribute(select_topk_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024));
+        attr_set = true;
+      }
+      select_topk_kernel<true><<<(unsigned)R, kSelThreads, row_bytes, st>>>(logits, R, V, s.top_k, inv_t, s.seed,
+                                                                            sample_base, step, out, status);
+    } else {
+      select_topk_kernel<false><<<(unsigned)R, kSelThreads, 0, st>>>(logits, R, V, s.top_k, inv_t, s.seed,
+                                                                     sample_base, step, out, status);
+    }
+  }
+  SRM_CUDA(cudaGetLastError());
+  return SRM_OK;
+}
+
+int launch_prefill_mixer(const srm_model& m, int layer, int64_t Bp, int n, const int32_t* tok, float* x, void* S,
+                         void* a, uint32_t* status, cudaStream_t st) {
+  if (Bp <= 0) return SRM_OK;
+  LaunchScope scope(m, SRM_KERNEL_PREFILL_MIXER, st);
+  PrefillParams p;
+  p.x = x; p.tok = tok; p.E = m.ptr(-1, SRM_T_E); p.S = S; p.a = a;
+  p.ln1_g = m.fptr(layer, SRM_T_LN1_G); p.ln1_b = m.fptr(layer, SRM_T_LN1_B);
+  p.ln2_g = m.fptr(layer, SRM_T_LN2_G); p.ln2_b = m.fptr(layer, SRM_T_LN2_B);
+  p.alpha = m.fptr(layer, SRM_T_ALPHA); p.beta = m.fptr(layer, SRM_T_BETA); p.lam = m.fptr(layer, SRM_T_LAMBDA);
+  p.Bp = Bp; p.n = n; p.d = m.cfg.d_model; p.h = m.cfg.n_heads; p.n_ctx = m.cfg.n_ctx; p.vocab = m.cfg.vocab;
+  p.eps = m.cfg.ln_eps; p.status = status;
+  const size_t smem = (size_t)kPrefillTile * m.cfg.d_model * 4;
+  const bool wb = m.cfg.dtype == SRM_DTYPE_BF16, sb = m.cfg.state_dtype == SRM_DTYPE_BF16;
+  auto go = [&](auto kernel) -> int {
+    SRM_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    kernel<<<(unsigned)Bp, kPrefillThreads, smem, st>>>(p);
+    SRM_CUDA(cudaGetLastError());
+    return SRM_OK;
+  };
+  if (wb && sb) return go(prefill_mixer_kernel<bf16, bf16>);
+  if (wb) return go(prefill_mixer_kernel<bf16, float>);
+  if (sb) return go(prefill_mixer_kernel<float, bf16>);
+  return go(prefill_mixer_kernel<float, float>);
+}
+
+// One decode step for rows [b0, b0 + R) of the state.
+int decode_chunk(srm_model& m, srm_state& s, int64_t b0, int64_t R, const int32_t* tok_in, const srm_sampling& samp,
+                 int step, const SelectOut& out_all, float* logits_out, const DecodeWs& w, cudaStream_t st) {
+  const srm_config& c = m.cfg;
+  const int d = c.d_model;
+  const int64_t F = m.F();
+  const int t = (int)s.pos;
+  int rc;
+  for (int l = 0; l < c.n_layers; ++l) {
+    uint8_t* Sl = static_cast<uint8_t*>(s.layer_ptr(l)) + (size_t)b0 * d * m.state_bytes();
+    if ((rc = launch_mixer(m, l, t, R, l == 0 ? tok_in + b0 : nullptr, w.x, Sl, w.a, s.status, st))) return rc;
+    if ((rc = launch_gemm(m, kEpiBiasGelu, R, F, d, w.a, m.ptr(l, SRM_T_W1), m.fptr(l, SRM_T_B1), w.H, s.status, st))) return rc;
+    if ((rc = launch_gemm(m, kEpiBiasResidual, R, d, F, w.H, m.ptr(l, SRM_T_W2), m.fptr(l, SRM_T_B2), w.x, s.status, st))) return rc;
+  }
+  if ((rc = launch_final_norm(m, w.x, R, 1, 0, w.a, st))) return rc;
+  float* lg = logits_out != nullptr ? logits_out + b0 * c.vocab : w.logits;
+  if ((rc = launch_gemm(m, kEpiPlain, R, c.vocab, d, w.a, m.ptr(-1, SRM_T_W_LM), nullptr, lg, s.status, st))) return rc;
+  SelectOut o = out_all;
+  o.last_tok += b0;
+  if (o.tok_out) o.tok_out += b0;
+  if (o.store) o.store += b0 * o.store_stride;
+  return launch_select(m, R, lg, samp, samp.sample_idx_base + (uint64_t)b0, step, o, s.status, st);
+}
+
+int decode_step_impl(srm_model* m, srm_state* s, const int32_t* d_tok_in, const srm_sampling* samp, int step,
+                     int32_t* d_tok_out, int32_t* d_store, int64_t store_stride, int64_t store_col,
+                     float* d_logits_out, void* d_ws, size_t ws_bytes, cudaStream_t st) {
+  if (m == nullptr || s == nullptr || s->m != m || d_ws == nullptr) return SRM_ERR_INVALID_ARG;
+  int rc = check_sampling(*m, samp);
+  if (rc) return rc;
+  if (!aligned(d_ws, 256) || !aligned(d_tok_in, 4) || !aligned(d_tok_out, 4) || !aligned(d_logits_out, 16)) return SRM_ERR_ALIGNMENT;
+  if (s->pos >= m->cfg.n_ctx) return SRM_ERR_CTX_OVERFLOW;
+  const int64_t rows = fit_rows(ws_bytes, s->B, decode_need, *m, 0);
+  if (rows < 1) return SRM_ERR_BUFFER_TOO_SMALL;
+  const DecodeWs w = carve_decode(*m, d_ws, rows);
+  const int32_t* tok_in = d_tok_in != nullptr ? d_tok_in : s->last_tok;
+  SelectOut out{s->last_tok, d_tok_out, d_store, store_stride, store_col};
+  for (int64_t b0 = 0; b0 < s->B; b0 += rows) {
+    const int64_t R = (s->B - b0 < rows) ? s->B - b0 : rows;
+    if ((rc = decode_chunk(*m, *s, b0, R, tok_in, *samp, step, out, d_logits_out, w, st))) return rc;
+  }
+  s->pos += 1;
+  return SRM_OK;
+}
+
+}  // namespace
+
+// ================================ C ABI =========================================================
+extern "C" {
+
+size_t srm_weights_bytes(const srm_config* cfg) {
+  if (!config_ok(cfg)) return 0;
+  return make_layout(*cfg).total;
+}
+
+int srm_weight_slot(const srm_config* cfg, int32_t layer, int32_t tensor, size_t* offset, size_t* nbytes,
+                    int32_t* elem_bytes) {
+  if (!config_ok(cfg) || tensor < 0 || tensor >= SRM_T_COUNT) return SRM_ERR_INVALID_ARG;
+  const Layout L = make_layout(*cfg);
+  Slot s;
+  if (is_global_tensor(tensor)) {
+    s = L.global[tensor];
+  } else {
+    if (layer < 0 || layer >= cfg->n_layers) return SRM_ERR_INVALID_ARG;
+    s = L.layer[(size_t)layer * SRM_T_COUNT + tensor];
+  }
+  if (offset) *offset = s.off;
+  if (nbytes) *nbytes = s.bytes;
+  if (elem_bytes) *elem_bytes = s.elem;
+  return SRM_OK;
+}
+
+size_t srm_state_bytes(const srm_config* cfg, int64_t B) {
+  if (!config_ok(cfg) || B < 1) return 0;
+  return state_bytes_for(*cfg, B);
+}
+
+size_t srm_workspace_bytes(const srm_config* cfg, int64_t B_chunk, int32_t n_prefill_max) {
+  if (!config_ok(cfg) || B_chunk < 1 || n_prefill_max < 0) return 0;
+  srm_model tmp;
+  tmp.cfg = *cfg;
+  size_t need = decode_ws_bytes(tmp, B_chunk);
+  if (n_prefill_max > 0) {
+    const size_t p = prefill_ws_bytes(tmp, 1, n_prefill_max);
+    if (p > need) need = p;
+  }
+  return need;
+}
+
+int srm_create(const srm_config* cfg, const void* d_weights, size_t nbytes, srm_model** out) {
+  if (out == nullptr || d_weights == nullptr) return SRM_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (cfg == nullptr) return SRM_ERR_INVALID_ARG;
+  if (!config_ok(cfg)) return SRM_ERR_UNSUPPORTED;
+  if (!aligned(d_weights, 256)) return SRM_ERR_ALIGNMENT;
+  srm_model* m = new (std::nothrow) srm_model();
+  if (m == nullptr) return SRM_ERR_INVALID_ARG;
+  m->cfg = *cfg;
+  m->w = static_cast<const uint8_t*>(d_weights);
+  m->layout = make_layout(*cfg);
+  if (nbytes < m->layout.total) { delete m; return SRM_ERR_BUFFER_TOO_SMALL; }
+  cudaError_t e = cudaGetDevice(&m->device);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&m->num_sms, cudaDevAttrMultiProcessorCount, m->device);
+  if (e != cudaSuccess) { g_last_cuda_error = (int)e; delete m; return SRM_ERR_CUDA; }
+  m->tmaps.reserve(256);
+  *out = m;
+  return SRM_OK;
+}
+
+int srm_destroy(srm_model* m) {
+  if (m != nullptr) {
+    for (auto& r : m->prof) { cudaEventDestroy(r.start); cudaEventDestroy(r.stop); }
+    for (auto& e : m->event_pool) cudaEventDestroy(e);
+  }
+  delete m;
+  return SRM_OK;
+}
+
+int srm_profile_enable(srm_model* m, int on) {
+  if (m == nullptr) return SRM_ERR_INVALID_ARG;
+  m->profiling = on != 0;
+  return SRM_OK;
+}
+
+int srm_profile_read(srm_model* m, int32_t kernel_class, uint64_t* launches, double* total_ms) {
+  if (m == nullptr || kernel_class < 0 || kernel_class >= SRM_KERNEL_CLASS_COUNT) return SRM_ERR_INVALID_ARG;
+  for (auto& r : m->prof) {
+    SRM_CUDA(cudaEventSynchronize(r.stop));
+    float ms = 0.f;
+    SRM_CUDA(cudaEventElapsedTime(&ms, r.start, r.stop));
+    m->prof_launches[r.cls] += 1;
+    m->prof_ms[r.cls] += ms;
+    m->event_pool.push_back(r.start);
+    m->event_pool.push_back(r.stop);
+  }
+  m->prof.clear();
+  if (launches) *launches = m->prof_launches[kernel_class];
+  if (total_ms) *total_ms = m->prof_ms[kernel_class];
+  return SRM_OK;
+}
+
+int srm_profile_reset(srm_model* m) {
+  if (m == nullptr) return SRM_ERR_INVALID_ARG;
+  int rc = srm_profile_read(m, 0, nullptr, nullptr);
+  if (rc) return rc;
+  for (int i = 0; i < SRM_KERNEL_CLASS_COUNT; ++i) { m->prof_launches[i] = 0; m->prof_ms[i] = 0.0; }
+  return SRM_OK;
+}
+
+uint64_t srm_kernel_launches(void) { return g_kernel_launches; }
+
+int srm_state_create(srm_model* m, int64_t B, void* d_state, size_t nbytes, void* stream, srm_state** out) {
+  if (out == nullptr) return SRM_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (m == nullptr || d_state == nullptr || B < 1) return SRM_ERR_INVALID_ARG;
+  if (!aligned(d_state, 256)) return SRM_ERR_ALIGNMENT;
+  if (nbytes < state_bytes_for(m->cfg, B)) return SRM_ERR_BUFFER_TOO_SMALL;
+  srm_state* s = new (std::nothrow) srm_state();
+  if (s == nullptr) return SRM_ERR_INVALID_ARG;
+  s->m = m; s->B = B; s->base = static_cast<uint8_t*>(d_state); s->nbytes = state_bytes_for(m->cfg, B);
+  s->status = reinterpret_cast<uint32_t*>(s->base);
+  s->last_tok = reinterpret_cast<int32_t*>(s->base + kStateHeader);
+  s->S = s->base + kStateHeader + align_up((size_t)B * 4, 256);
+  s->pos = 0;
+  int rc = srm_state_reset(s, stream);
+  if (rc != SRM_OK) { delete s; return rc; }
+  *out = s;
+  return SRM_OK;
+}
+
+int srm_state_destroy(srm_state* s) {
+  delete s;
+  return SRM_OK;
+}
+
+int srm_state_reset(srm_state* s, void* stream) {
+  if (s == nullptr) return SRM_ERR_INVALID_ARG;
+  SRM_CUDA(cudaMemsetAsync(s->base, 0, s->nbytes, static_cast<cudaStream_t>(stream)));
+  s->pos = 0;
+  return SRM_OK;
+}
+
+int64_t srm_state_pos(const srm_state* s) { return s ? s->pos : -1; }
+
+int srm_state_set_pos(srm_state* s, int64_t pos) {
+  if (s == nullptr || pos < 0 || pos > s->m->cfg.n_ctx) return SRM_ERR_INVALID_ARG;
+  s->pos = pos;
+  return SRM_OK;
+}
+
+void* srm_state_layer_ptr(const srm_state* s, int32_t layer) {
+  if (s == nullptr || layer < 0 || layer >= s->m->cfg.n_layers) return nullptr;
+  return s->layer_ptr(layer);
+}
+
+int32_t* srm_state_last_token_ptr(const srm_state* s) { return s ? s->last_tok : nullptr; }
+
+int srm_status(srm_state* s, void* stream, uint32_t* flags) {
+  if (s == nullptr) return SRM_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint32_t f = 0;
+  SRM_CUDA(cudaMemcpyAsync(&f, s->status, 4, cudaMemcpyDeviceToHost, st));
+  SRM_CUDA(cudaMemsetAsync(s->status, 0, 4, st));
+  SRM_CUDA(cudaStreamSynchronize(st));
+  if (flags) *flags = f;
+  return f ? SRM_ERR_DEVICE_STATUS : SRM_OK;
+}
+
+int srm_prefill(srm_model* m, srm_state* s, const int32_t* d_tokens, int32_t n, const srm_sampling* samp,
+                int32_t* d_first_tok, float* d_logits_last, void* d_ws, size_t ws_bytes, void* stream) {
+  if (m == nullptr || s == nullptr || s->m != m || d_tokens == nullptr || d_ws == nullptr || n < 1) return SRM_ERR_INVALID_ARG;
+  int rc = check_sampling(*m, samp);
+  if (rc) return rc;
+  if (!aligned(d_ws, 256) || !aligned(d_tokens, 4) || !aligned(d_first_tok, 4) || !aligned(d_logits_last, 16)) return SRM_ERR_ALIGNMENT;
+  if (s->pos != 0) return SRM_ERR_INVALID_ARG;           // the parallel form starts from an empty cache
+  if (n > m->cfg.n_ctx) return SRM_ERR_CTX_OVERFLOW;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int64_t Bp = fit_rows(ws_bytes, s->B, prefill_need, *m, n);
+  if (Bp < 1) return SRM_ERR_BUFFER_TOO_SMALL;
+  const PrefillWs w = carve_prefill(*m, d_ws, Bp, n);
+  const srm_config& c = m->cfg;
+  const int d = c.d_model;
+  const int64_t F = m->F();
+  for (int64_t b0 = 0; b0 < s->B; b0 += Bp) {
+    const int64_t nb = (s->B - b0 < Bp) ? s->B - b0 : Bp;
+    const int64_t rows = nb * n;
+    for (int l = 0; l < c.n_layers; ++l) {
+      uint8_t* Sl = static_cast<uint8_t*>(s->layer_ptr(l)) + (size_t)b0 * d * m->state_bytes();
+      if ((rc = launch_prefill_mixer(*m, l, nb, n, l == 0 ? d_tokens + b0 * n : nullptr, w.x, Sl, w.a, s->status, st))) return rc;
+      if ((rc = launch_gemm(*m, kEpiBiasGelu, rows, F, d, w.a, m->ptr(l, SRM_T_W1), m->fptr(l, SRM_T_B1), w.H, s->status, st))) return rc;
+      if ((rc = launch_gemm(*m, kEpiBiasResidual, rows, d, F, w.H, m->ptr(l, SRM_T_W2), m->fptr(l, SRM_T_B2), w.x, s->status, st))) return rc;
+    }
+    // LM head and selection on the last prompt position only
+    if ((rc = launch_final_norm(*m, w.x, nb, n, n - 1, w.a_last, st))) return rc;
+    float* lg = d_logits_last != nullptr ? d_logits_last + b0 * c.vocab : w.logits;
+    if ((rc = launch_gemm(*m, kEpiPlain, nb, c.vocab, d, w.a_last, m->ptr(-1, SRM_T_W_LM), nullptr, lg, s->status, st))) return rc;
+    SelectOut o{s->last_tok + b0, d_first_tok ? d_first_tok + b0 : nullptr, nullptr, 0, 0};
+    if ((rc = launch_select(*m, nb, lg, *samp, samp->sample_idx_base + (uint64_t)b0, 0, o, s->status, st))) return rc;
+  }
+  s->pos = n;
+  return SRM_OK;
+}
+
+int srm_decode_step(srm_model* m, srm_state* s, const int32_t* d_tok_in, const srm_sampling* samp, int32_t step,
+                    int32_t* d_tok_out, float* d_logits_out, void* d_ws, size_t ws_bytes, void* stream) {
+  return decode_step_impl(m, s, d_tok_in, samp, step, d_tok_out, nullptr, 0, 0, d_logits_out, d_ws, ws_bytes,
+                          static_cast<cudaStream_t>(stream));
+}
+
+int srm_generate(srm_model* m, srm_state* s, int32_t steps, int32_t first_step, const srm_sampling* samp,
+                 int32_t* d_out, int64_t out_stride, void* d_ws, size_t ws_bytes, void* stream) {
+  if (m == nullptr || s == nullptr || steps < 0 || (d_out != nullptr && out_stride < steps)) return SRM_ERR_INVALID_ARG;
+  if (s->pos + steps > m->cfg.n_ctx) return SRM_ERR_CTX_OVERFLOW;
+  for (int j = 0; j < steps; ++j) {
+    int rc = decode_step_impl(m, s, nullptr, samp, first_step + j, nullptr, d_out, out_stride, j, nullptr, d_ws,
+                              ws_bytes, static_cast<cudaStream_t>(stream));
+    if (rc) return rc;
+  }
+  return SRM_OK;
+}
+
+int srm_decode_step_host(srm_model* m, srm_state* s, const int32_t* h_tok_in, const srm_sampling* samp, int32_t step,
+                         int32_t* h_tok_out, void* d_ws, size_t ws_bytes, void* stream) {
+  if (m == nullptr || s == nullptr || h_tok_in == nullptr || h_tok_out == nullptr) return SRM_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // the state's own last-token vector doubles as the device staging buffer
+  SRM_CUDA(cudaMemcpyAsync(s->last_tok, h_tok_in, (size_t)s->B * 4, cudaMemcpyHostToDevice, st));
+  int rc = decode_step_impl(m, s, nullptr, samp, step, nullptr, nullptr, 0, 0, nullptr, d_ws, ws_bytes, st);
+  if (rc) return rc;
+  SRM_CUDA(cudaMemcpyAsync(h_tok_out, s->last_tok, (size_t)s->B * 4, cudaMemcpyDeviceToHost, st));
+  return SRM_OK;
+}
+
+// ---- single kernels ---------------------------------------------------------------------------
+int srm_k_mixer_step(srm_model* m, int32_t layer, int32_t t, int64_t R, const int32_t* d_tok, float* d_x, void* d_S,
+                     void* d_a, uint32_t* d_status, void* stream) {
+  if (m == nullptr || R < 0) return SRM_ERR_INVALID_ARG;
+  if (R == 0) return SRM_OK;
+  if (d_x == nullptr || d_S == nullptr || d_a == nullptr) return SRM_ERR_INVALID_ARG;
+  if (layer < 0 || layer >= m->cfg.n_layers || t < 0) return SRM_ERR_INVALID_ARG;
+  if (t >= m->cfg.n_ctx) return SRM_ERR_CTX_OVERFLOW;
+  if (!aligned(d_x, 16) || !aligned(d_S, 16) || !aligned(d_a, 16)) return SRM_ERR_ALIGNMENT;
+  return launch_mixer(*m, layer, t, R, d_tok, d_x, d_S, d_a, d_status, static_cast<cudaStream_t>(stream));
+}
+
+int srm_k_final_norm(srm_model* m, int64_t R, const float* d_x, void* d_a, void* stream) {
+  if (m == nullptr || R < 0) return SRM_ERR_INVALID_ARG;
+  if (R == 0) return SRM_OK;
+  if (d_x == nullptr || d_a == nullptr) return SRM_ERR_INVALID_ARG;
+  if (!aligned(d_x, 16) || !aligned(d_a, 16)) return SRM_ERR_ALIGNMENT;
+  return launch_final_norm(*m, d_x, R, 1, 0, d_a, static_cast<cudaStream_t>(stream));
+}
+
+int srm_k_gemm(srm_model* m, int32_t epilogue, int64_t M, int64_t N, int64_t K, const void* d_A, const void* d_W,
+               const float* d_bias, void* d_out, uint32_t* d_status, void* stream) {
+  if (m == nullptr || M < 0 || N < 1 || K < 1) return SRM_ERR_INVALID_ARG;
+  if (M == 0) return SRM_OK;
+  if (d_A == nullptr || d_W == nullptr || d_out == nullptr) return SRM_ERR_INVALID_ARG;
+  if (epilogue < 0 || epilogue > 2 || (epilogue != kEpiPlain && d_bias == nullptr)) return SRM_ERR_INVALID_ARG;
+  if (K % 64 || N % 8) return SRM_ERR_UNSUPPORTED;
+  if (!aligned(d_A, 16) || !aligned(d_W, 16) || !aligned(d_out, 16) || !aligned(d_bias, 16)) return SRM_ERR_ALIGNMENT;
+  return launch_gemm(*m, epilogue, M, N, K, d_A, d_W, d_bias, d_out, d_status, static_cast<cudaStream_t>(stream));
+}
+
+int srm_k_select(srm_model* m, int64_t R, const float* d_logits, const srm_sampling* samp, int32_t step,
+                 int32_t* d_tok, uint32_t* d_status, void* stream) {
+  if (m == nullptr || R < 0) return SRM_ERR_INVALID_ARG;
+  if (R == 0) return SRM_OK;
+  if (d_logits == nullptr || d_tok == nullptr) return SRM_ERR_INVALID_ARG;
+  int rc = check_sampling(*m, samp);
+  if (rc) return rc;
+  if (!aligned(d_logits, 16)) return SRM_ERR_ALIGNMENT;
+  SelectOut o{d_tok, nullptr, nullptr, 0, 0};
+  return launch_select(*m, R, d_logits, *samp, samp->sample_idx_base, step, o, d_status, static_cast<cudaStream_t>(stream));
+}
+
+int srm_k_prefill_mixer(srm_model* m, int32_t layer, int64_t Bp, int32_t n, const int32_t* d_tok, float* d_x, void* d_S,
+                        void* d_a, uint32_t* d_status, void* stream) {
+  if (m == nullptr || Bp < 0 || n < 1) return SRM_ERR_INVALID_ARG;
+  if (Bp == 0) return SRM_OK;
+  if (d_x == nullptr || d_S == nullptr || d_a == nullptr) return SRM_ERR_INVALID_ARG;
+  if (layer < 0 || layer >= m->cfg.n_layers) return SRM_ERR_INVALID_ARG;
+  if (n > m->cfg.n_ctx) return SRM_ERR_CTX_OVERFLOW;
+  if (!aligned(d_x, 16) || !aligned(d_S, 16) || !aligned(d_a, 16)) return SRM_ERR_ALIGNMENT;
+  return launch_prefill_mixer(*m, layer, Bp, n, d_tok, d_x, d_S, d_a, d_status, static_cast<cudaStream_t>(stream));
+}
+
+const char* srm_strerror(int code) {
+  switch (code) {
+    case SRM_OK: return "ok";
+    case SRM_ERR_INVALID_ARG: return "invalid argument";
+    case SRM_ERR_UNSUPPORTED: return "unsupported shape or configuration";
+    case SRM_ERR_ALIGNMENT: return "misaligned device pointer";
+    case SRM_ERR_BUFFER_TOO_SMALL: return "buffer too small";
+    case SRM_ERR_CTX_OVERFLOW: return "position would exceed n_ctx";
+    case SRM_ERR_CUDA: return "CUDA call failed (see srm_last_cuda_error)";
+    case SRM_ERR_DEVICE_STATUS: return "device status flags set";
+    default: return "unknown error";
+  }
+}
+
+int srm_last_cuda_error(void) { return g_last_cuda_error; }
+
+const char* srm_version(void) { return "srm-b200 0.1 (sm_100a)"; }
+
+}  // extern "C"

@@ -1,0 +1,230 @@
+"""Parity of each CUDA kernel, called through the C ABI, against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+import srm_inputs as I
+from helpers import custom_shape, rel_err_rows
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda:0"
+
+
+def _model(shape, W=None, **kw):
+    import paper_2605_08696_b200 as P
+    W = W if W is not None else I.make_weights(shape, alpha_std=0.5, beta_std=0.5)
+    return P.SRM(shape, W, device=DEV, **kw), W
+
+
+def _t(a, dtype=torch.float32):
+    return torch.from_numpy(np.ascontiguousarray(a)).to(DEV).to(dtype).contiguous()
+
+
+# ---- fused token-mixer step (Eq. 2, Eq. 3) --------------------------------------------------
+
+@pytest.mark.parametrize("d,dtype,state_dtype", [(64, "fp32", "fp32"), (512, "bf16", "fp32"), (1024, "bf16", "fp32"),
+                                                 (1536, "bf16", "fp32"), (1024, "bf16", "bf16"), (2048, "fp32", "fp32"),
+                                                 (192, "fp32", "bf16")])
+@pytest.mark.parametrize("embed", [False, True])
+def test_mixer_step_matches_oracle(d, dtype, state_dtype, embed):
+    from oracle import srm_oracle as O
+    shape = custom_shape(n_layers=2, d_model=d, vocab=512, n_ctx=40, dtype=dtype, seed=7)
+    m, W = _model(shape, state_dtype=state_dtype)
+    rng = np.random.default_rng(d)
+    R, layer, t = 37, 1, 17                       # ragged row count (not a multiple of the 4 rows per block)
+    lw = {k: np.asarray(v, np.float64) for k, v in W["layers"][layer].items()}
+    tok = rng.integers(0, shape.vocab, size=R).astype(np.int32)
+    x0 = W["E"][tok].astype(np.float64) if embed else rng.normal(size=(R, d))
+    S0 = rng.normal(size=(R, d))
+    sdt = torch.bfloat16 if state_dtype == "bf16" else torch.float32
+    S0 = _t(S0, sdt).float().cpu().numpy().astype(np.float64)      # what the device really holds
+    x = _t(rng.normal(size=(R, d)) if embed else x0)
+    x_in = x.clone()
+    S = _t(S0, sdt)
+    a = torch.zeros(R, d, dtype=m.act_dtype, device=DEV)
+    m.k_mixer_step(layer, t, x, S, a, tok=_t(tok, torch.int32) if embed else None)
+    torch.cuda.synchronize()
+    x0 = x0 if embed else x_in.cpu().numpy().astype(np.float64)
+    z = O.layer_norm(x0, lw["ln1_g"], lw["ln1_b"], shape.ln_eps)
+    y, S1 = O.mixer_recurrent_step(z, S0, t, lw["alpha"], lw["beta"], lw["lam"], shape.n_heads)
+    x1 = x0 + y
+    a1 = O.layer_norm(x1, lw["ln2_g"], lw["ln2_b"], shape.ln_eps)
+    assert rel_err_rows(x.cpu().numpy(), x1) < 1e-5
+    assert rel_err_rows(S.float().cpu().numpy(), S1) < (1e-5 if state_dtype == "fp32" else 6e-3)
+    assert rel_err_rows(a.float().cpu().numpy(), a1) < (1e-5 if dtype == "fp32" else 6e-3)
+
+
+def test_mixer_step_zero_rows_and_token_clamp():
+    shape = custom_shape(d_model=64, vocab=256)
+    m, W = _model(shape)
+    x = torch.zeros(0, 64, device=DEV); S = torch.zeros(0, 64, device=DEV); a = torch.zeros(0, 64, device=DEV)
+    m.k_mixer_step(0, 0, x, S, a)                   # empty batch: a no-op, no launch error
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    x = torch.zeros(3, 64, device=DEV); S = torch.zeros(3, 64, device=DEV); a = torch.zeros(3, 64, device=DEV)
+    m.k_mixer_step(0, 0, x, S, a, tok=torch.tensor([5, 999, -2], dtype=torch.int32, device=DEV), status=status)
+    torch.cuda.synchronize()
+    assert status.item() & 1                        # SRM_STATUS_TOKEN_RANGE, ids clamped not trapped
+    assert torch.isfinite(x).all()
+
+
+def test_final_norm_matches_oracle():
+    from oracle import srm_oracle as O
+    for d, dtype in [(64, "fp32"), (1024, "bf16")]:
+        shape = custom_shape(d_model=d, dtype=dtype)
+        m, W = _model(shape)
+        x = np.random.default_rng(1).normal(1.0, 2.0, size=(11, d))
+        xg = _t(x)
+        a = torch.zeros(11, d, dtype=m.act_dtype, device=DEV)
+        m.k_final_norm(xg, a)
+        want = O.layer_norm(xg.cpu().numpy().astype(np.float64), W["lnf_g"].astype(np.float64),
+                            W["lnf_b"].astype(np.float64), shape.ln_eps)
+        assert rel_err_rows(a.float().cpu().numpy(), want) < (1e-5 if dtype == "fp32" else 6e-3)
+
+
+# ---- projections ---------------------------------------------------------------------------------
+
+def _gemm_case(m, M, N, K, epi, act, seed=0):
+    from oracle import srm_oracle as O
+    rng = np.random.default_rng(seed)
+    A = _t(rng.normal(size=(M, K)), act)
+    W = _t(rng.normal(size=(N, K)) * 0.05, act)
+    bias = _t(rng.normal(size=N))
+    A64, W64 = A.float().cpu().numpy().astype(np.float64), W.float().cpu().numpy().astype(np.float64)
+    D = A64 @ W64.T
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    if epi == 0:
+        out = torch.zeros(M, N, dtype=act, device=DEV)
+        want = O.gelu_erf(D + bias.cpu().numpy().astype(np.float64))
+    elif epi == 1:
+        out0 = rng.normal(size=(M, N)).astype(np.float32)
+        out = _t(out0)
+        want = out0.astype(np.float64) + D + bias.cpu().numpy().astype(np.float64)
+    else:
+        out = torch.full((M, N), float("nan"), dtype=torch.float32, device=DEV)
+        want = D
+    m.k_gemm(epi, A, W, bias, out, status=status)
+    torch.cuda.synchronize()
+    assert status.item() == 0, f"device status {status.item()}"
+    return out.float().cpu().numpy(), want
+
+
+@pytest.mark.parametrize("M,N,K", [(128, 256, 64), (256, 512, 128), (1, 256, 64), (300, 1000, 192),
+                                   (77, 8000, 512), (520, 264, 1024), (4096, 1024, 4096)])
+@pytest.mark.parametrize("epi", [0, 1, 2])
+def test_tensor_core_gemm_matches_fp64_matmul(M, N, K, epi):
+    shape = custom_shape(d_model=64, dtype="bf16")
+    m, _ = _model(shape)
+    got, want = _gemm_case(m, M, N, K, epi, torch.bfloat16, seed=M + N + K + epi)
+    tol = 6e-3 if epi == 0 else 2e-5          # bf16 output rounding vs fp32 accumulation error
+    assert rel_err_rows(got, want) < tol
+
+
+def test_tensor_core_gemm_equals_simt_gemm_on_device():
+    """Same bf16 inputs through the SIMT kernel and the tcgen05 kernel: fp32 accumulation in a
+    different order only."""
+    shape = custom_shape(d_model=64, dtype="bf16")
+    m_tc, _ = _model(shape)
+    m_simt, _ = _model(shape, flags=1)
+    for epi in (0, 2):
+        a, _ = _gemm_case(m_tc, 333, 520, 256, epi, torch.bfloat16, seed=3)
+        b, _ = _gemm_case(m_simt, 333, 520, 256, epi, torch.bfloat16, seed=3)
+        assert rel_err_rows(a, b) < (8e-3 if epi == 0 else 1e-5)
+
+
+@pytest.mark.parametrize("M,N,K", [(4, 256, 64), (70, 130 * 8, 256), (129, 64, 128)])
+@pytest.mark.parametrize("epi", [0, 1, 2])
+def test_fp32_simt_gemm_matches_fp64_matmul(M, N, K, epi):
+    shape = custom_shape(d_model=64, dtype="fp32")
+    m, _ = _model(shape)
+    got, want = _gemm_case(m, M, N, K, epi, torch.float32, seed=M + epi)
+    assert rel_err_rows(got, want) < 2e-6
+
+
+# ---- token selection -------------------------------------------------------------------------------
+
+def test_greedy_selection_bit_exact():
+    from oracle import srm_oracle as O
+    import paper_2605_08696_b200 as P
+    for V in (256, 8000, 32000):
+        shape = custom_shape(vocab=V)
+        m, _ = _model(shape)
+        rng = np.random.default_rng(V)
+        lg = rng.normal(size=(33, V)).astype(np.float32)
+        lg[0, :] = 1.5                               # all equal: id 0
+        lg[1, [7, V - 1, 100]] = 9.0                 # ties: lowest id
+        lg[2, V - 1] = 50.0                          # maximum in the last slot
+        tok = torch.zeros(33, dtype=torch.int32, device=DEV)
+        m.k_select(_t(lg), P.Sampling("greedy"), 0, tok)
+        assert np.array_equal(tok.cpu().numpy(), O.select_greedy(lg))
+
+
+@pytest.mark.parametrize("V,k", [(256, 50), (8000, 50), (32000, 50), (32000, 1), (1024, 256), (48000, 17)])
+def test_topk_sampling_matches_oracle(V, k):
+    from oracle import srm_oracle as O
+    import paper_2605_08696_b200 as P
+    shape = custom_shape(vocab=V)
+    m, _ = _model(shape)
+    rng = np.random.default_rng(V + k)
+    R, T, seed, step, base = 48, 0.8, 0x1234567887654321, 11, 1000
+    lg = (rng.normal(size=(R, V)) * 2).astype(np.float32)
+    lg[0] = np.round(lg[0], 0)                       # heavy ties, also across the k-th place
+    lg[1, :] = 0.25                                  # all equal: the k lowest ids
+    tok = torch.zeros(R, dtype=torch.int32, device=DEV)
+    samp = P.Sampling("topk", top_k=k, temperature=T, seed=seed, sample_idx_base=base)
+    m.k_select(_t(lg), samp, step, tok)
+    got = tok.cpu().numpy()
+    want, det = O.select_topk(lg, k, T, seed, base + np.arange(R), step, return_detail=True)
+    exempt = 0
+    for r in range(R):
+        assert got[r] in det[r]["ids"]               # always one of the oracle's top-k ids
+        if got[r] != want[r]:
+            # only allowed when u*total sits within 1e-6*total of a CDF edge (fp32 vs fp64 sums)
+            c, thr = det[r]["cdf"], det[r]["thr"]
+            assert np.min(np.abs(c - thr)) < 1e-6 * c[-1], (r, got[r], want[r])
+            exempt += 1
+    assert exempt <= 1
+
+
+def test_topk_sampling_stream_is_keyed_by_sample_and_step():
+    import paper_2605_08696_b200 as P
+    shape = custom_shape(vocab=8000)
+    m, _ = _model(shape)
+    lg = _t(np.tile(np.random.default_rng(0).normal(size=(1, 8000)).astype(np.float32), (64, 1)))
+    outs = []
+    for base, step in [(0, 0), (0, 1), (64, 0), (0, 0)]:
+        tok = torch.zeros(64, dtype=torch.int32, device=DEV)
+        m.k_select(lg, P.Sampling("topk", 50, 0.8, seed=5, sample_idx_base=base), step, tok)
+        outs.append(tok.cpu().numpy())
+    assert np.array_equal(outs[0], outs[3])          # deterministic
+    assert not np.array_equal(outs[0], outs[1]) and not np.array_equal(outs[0], outs[2])
+    assert len(np.unique(outs[0])) > 5
+
+
+# ---- sequence-parallel token mixing (Eq. 1, Eq. 3) -----------------------------------------------
+
+@pytest.mark.parametrize("d,dtype,n", [(64, "fp32", 8), (64, "fp32", 32), (64, "fp32", 37), (512, "bf16", 128),
+                                       (1024, "bf16", 50), (1536, "bf16", 33)])
+@pytest.mark.parametrize("embed", [False, True])
+def test_prefill_mixer_matches_oracle_parallel_form(d, dtype, n, embed):
+    from oracle import srm_oracle as O
+    shape = custom_shape(n_layers=1, d_model=d, vocab=512, n_ctx=max(n, 40), dtype=dtype, seed=9)
+    m, W = _model(shape)
+    lw = {k: np.asarray(v, np.float64) for k, v in W["layers"][0].items()}
+    rng = np.random.default_rng(n)
+    Bp = 3
+    tok = rng.integers(0, shape.vocab, size=(Bp, n)).astype(np.int32)
+    x0 = W["E"][tok].astype(np.float64) if embed else rng.normal(size=(Bp, n, d)).astype(np.float32).astype(np.float64)
+    x = _t(np.zeros((Bp * n, d)) if embed else x0.reshape(Bp * n, d))
+    S = torch.full((Bp, d), float("nan"), device=DEV)
+    a = torch.zeros(Bp * n, d, dtype=m.act_dtype, device=DEV)
+    m.k_prefill_mixer(0, Bp, n, x, S, a, tok=_t(tok.reshape(-1), torch.int32) if embed else None)
+    torch.cuda.synchronize()
+    for b in range(Bp):
+        z = O.layer_norm(x0[b], lw["ln1_g"], lw["ln1_b"], shape.ln_eps)
+        y, Sn = O.mixer_parallel(z, lw["alpha"], lw["beta"], lw["lam"], shape.n_heads)
+        x1 = x0[b] + y
+        a1 = O.layer_norm(x1, lw["ln2_g"], lw["ln2_b"], shape.ln_eps)
+        assert rel_err_rows(x[b * n:(b + 1) * n].cpu().numpy(), x1) < 2e-5
+        assert rel_err_rows(S[b].cpu().numpy(), Sn) < 2e-5
+        assert rel_err_rows(a[b * n:(b + 1) * n].float().cpu().numpy(), a1) < (2e-5 if dtype == "fp32" else 6e-3)
