@@ -1,14 +1,27 @@
-// bf16 projection D[M,N] = A[M,K] * W[N,K]^T on the 5th-generation tensor cores (sm_100a):
-// TMA (cp.async.bulk.tensor, 128-byte swizzle, no multicast) -> shared-memory ring ->
-// tcgen05.mma (one issuing thread, cta_group::1, 128x256x16 per instruction) with fp32
-// accumulators in tensor memory (two 256-column buffers, so the epilogue of tile i overlaps
-// the main loop of tile i+1) -> tcgen05.ld -> fused epilogue -> global memory.
+// bf16 projection D[M,N] = A[M,K] * W[N,K]^T on the 5th-generation tensor cores (sm_100a).
 //
-// The kernel is persistent: grid = min(tiles, SMs), tiles are taken round-robin.
-// Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner, warps 2..5 = epilogue
-// (warp w reads TMEM lanes 32*(w%4) .. +31, i.e. one accumulator row per thread).
+// Two CTAs of a cluster (a CTA pair on neighbouring SMs) own one 256 x 256 output tile:
+//   TMA (cp.async.bulk.tensor, 128-byte swizzle, no multicast): CTA r loads rows
+//   [128 r, 128 r + 128) of the A tile and of the W tile into its own shared-memory ring;
+//   both CTAs' copies complete on the leader CTA's mbarrier;
+//   tcgen05.mma.cta_group::2 (one issuing thread in the leader CTA, 256x256x16 per instruction)
+//   reads both CTAs' shared memory and accumulates in fp32 in both CTAs' tensor memory (each holds
+//   its 128 rows x 256 columns, two such buffers, so the epilogue of tile i overlaps the main loop
+//   of tile i+1); tcgen05.commit multicasts "stage free" / "accumulator ready" to both CTAs;
+//   tcgen05.ld -> fused epilogue -> global memory, in each CTA for its own 128 rows.
+// Pairing halves the W bytes each SM pulls from L2 per flop compared with a 128 x 256 tile per
+// SM, which is what bounded the single-CTA version of this kernel.
+//
+// The kernel is persistent: grid = 2 * min(tiles, resident clusters), tiles taken round-robin.
+// Warp roles per CTA: warp 0 = TMA producer, warp 1 = MMA issuer (leader only) and TMEM owner,
+// warps 2..17 = epilogue (warp w reads TMEM lanes 32*(w%4) .. +31, one accumulator row per thread;
+// the four warps that share a lane quarter split the tile's columns; four warps per scheduler hide
+// each other's TMEM / shared / global latencies, since with K = d the epilogue's instruction issue
+// is as long as the tile's MMAs). Each epilogue warp transposes its values through a private
+// shared-memory patch so that every global store (and residual load) instruction covers eight
+// rows x 64 contiguous bytes in whole 32-byte sectors.
 // Every wait is bounded: after ~2^31 clock cycles a waiter raises kStatusWaitTimeout, leaves its
-// loop, and the CTA still releases its tensor memory and exits.
+// loop, and both CTAs still meet at the final cluster barrier, release tensor memory and exit.
 #pragma once
 
 #include <cuda.h>
@@ -19,14 +32,19 @@
 namespace srm {
 namespace tc {
 
-constexpr int BM = 128, BN = 256, BK = 64;
-constexpr int kStages = 4;
-constexpr int kAStageBytes = BM * BK * 2;        // 16 KiB
-constexpr int kBStageBytes = BN * BK * 2;        // 32 KiB
+constexpr int BM = 256, BN = 256, BK = 64;       // tile of one CTA pair
+constexpr int kRowsPerCta = 128;                 // A rows and W rows each CTA loads per k-block
+constexpr int kStages = 5;
+constexpr int kAStageBytes = kRowsPerCta * BK * 2;   // 16 KiB
+constexpr int kBStageBytes = kRowsPerCta * BK * 2;   // 16 KiB
 constexpr int kStageBytes = kAStageBytes + kBStageBytes;
 constexpr int kBarrierBytes = 256;
-constexpr int kSmemBytes = kStages * kStageBytes + kBarrierBytes + 1024;  // +1024: manual alignment
-constexpr int kThreads = 192;
+constexpr int kEpiWarps = 16;
+constexpr int kColsPerEpiWarp = BN / (kEpiWarps / 4);   // 64
+constexpr int kPatchRowBytes = 80;               // 64 data bytes + 16 pad (bank spread)
+constexpr int kPatchBytes = 32 * kPatchRowBytes; // one patch per epilogue warp
+constexpr int kSmemBytes = kStages * kStageBytes + kEpiWarps * kPatchBytes + kBarrierBytes + 1024;  // +1024: alignment
+constexpr int kThreads = 64 + kEpiWarps * 32;
 constexpr int kTmemCols = 512;                   // two accumulators of BN fp32 columns
 constexpr long long kWaitLimitCycles = 1ll << 31;
 
@@ -69,21 +87,44 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint32
     }
   }
 }
-__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, uint64_t* bar, int x, int y) {
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// shared::cluster address of the same shared-memory offset in CTA `rank` of this cluster
+__device__ __forceinline__ uint32_t mapa(uint32_t saddr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// arrive (optionally announcing transaction bytes) on an mbarrier anywhere in the cluster
+__device__ __forceinline__ void mbar_expect_tx_cluster(uint32_t cluster_addr, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cluster.b64 _, [%0], %1;" ::"r"(cluster_addr), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// TMA tile load into this CTA's shared memory whose completion is counted on an mbarrier that may
+// live in the peer CTA of the pair (cta_group::2); no multicast.
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, uint32_t bar_cluster_addr, int x, int y) {
   asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-      ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(x), "r"(y)
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar_cluster_addr), "r"(x), "r"(y)
       : "memory");
 }
 __device__ __forceinline__ void tmem_alloc(uint32_t* slot, uint32_t cols) {
-  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(slot)), "r"(cols)
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(slot)), "r"(cols)
                : "memory");
 }
 __device__ __forceinline__ void tmem_relinquish() {
-  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
 }
 __device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
-  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -92,13 +133,16 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
-// mbarrier arrive once all tcgen05 operations issued so far by this thread have completed
-__device__ __forceinline__ void umma_commit(uint64_t* bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+// Arrive on the mbarrier at this shared-memory offset in BOTH CTAs of the pair once all tcgen05
+// operations issued so far by this thread have completed.
+__device__ __forceinline__ void umma_commit_pair(uint64_t* bar) {
+  const uint16_t mask = 3;
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(smem_u32(bar)), "h"(mask)
                : "memory");
 }
 // 32 consecutive fp32 columns of this thread's TMEM lane
@@ -129,7 +173,7 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
   d |= static_cast<uint64_t>(2) << 61;
   return d;
 }
-// Instruction descriptor: fp32 accumulate, bf16 A and B, both K-major, N = BN, M = BM.
+// Instruction descriptor: fp32 accumulate, bf16 A and B, both K-major, N = BN, M = BM (pair).
 constexpr uint32_t kInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(BN >> 3) << 17) |
                                 (uint32_t(BM >> 4) << 24);
 
@@ -140,66 +184,136 @@ struct GemmArgs {
   uint32_t* status;
 };
 
+// GELU(v) = v * Phi(v) with erfc by the rational approximation 7.1.26 of Abramowitz & Stegun
+// (|error| <= 1.5e-7, far below the bf16 resolution of the value it feeds; coefficients halved so
+// that h = erfc(|v|/sqrt 2) / 2 = Phi(-|v|)). One rcp.approx and one ex2.approx per element keep
+// the epilogue within the issue slots a K = d tile leaves.
+__device__ __forceinline__ float rcp_approx(float x) {
+  float r;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+  return r;
+}
+__device__ __forceinline__ float ex2_approx(float x) {
+  float r;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+  return r;
+}
+__device__ __forceinline__ float gelu_fast(float v) {
+  const float ax = fabsf(v) * 0.70710678118654752440f;
+  const float t = rcp_approx(fmaf(0.3275911f, ax, 1.0f));
+  const float e = ex2_approx(ax * ax * -1.4426950408889634f);      // exp(-v^2 / 2)
+  float p = fmaf(t, 0.5307027145f, -0.7265760135f);
+  p = fmaf(t, p, 0.7107068705f);
+  p = fmaf(t, p, -0.142248368f);
+  p = fmaf(t, p, 0.127414796f);
+  const float h = p * t * e;                                       // Phi(-|v|)
+  return v * (v < 0.f ? h : 1.0f - h);
+}
+
+// Writes one 32-row x 64-byte patch (row = the staging thread's lane) from `patch` to global memory.
+// Lane l handles the 16-byte piece l/8 of rows (l%8) + 8*i: a quarter-warp then reads eight rows whose
+// 80-byte stride spreads them over distinct banks, and the warp as a whole still covers eight rows x
+// 64 contiguous bytes per instruction.
 template <int EPI>
-__device__ __forceinline__ void epilogue_store(const GemmArgs& g, int64_t row, int64_t col0, const uint32_t (&r)[32]) {
-  if (row >= g.M) return;
-  if (EPI == kEpiBiasGelu) {
-    bf16* o = reinterpret_cast<bf16*>(g.out) + row * g.N + col0;
+__device__ __forceinline__ void flush_patch(const GemmArgs& g, const uint8_t* patch, int lane, int64_t row0,
+                                            int64_t col0) {
+  constexpr int kElem = (EPI == kEpiBiasGelu) ? 2 : 4;
+  constexpr int kPer16 = 16 / kElem;
+  const int piece = lane >> 3;
+  const int64_t col = col0 + piece * kPer16;
+  if (col >= g.N) return;
 #pragma unroll
-    for (int j = 0; j < 32; j += 8) {
-      if (col0 + j < g.N) {
-        const float4 b0 = __ldg(reinterpret_cast<const float4*>(g.bias + col0 + j));
-        const float4 b1 = __ldg(reinterpret_cast<const float4*>(g.bias + col0 + j + 4));
-        __nv_bfloat162 p0 = __floats2bfloat162_rn(gelu_erf(__uint_as_float(r[j + 0]) + b0.x),
-                                                  gelu_erf(__uint_as_float(r[j + 1]) + b0.y));
-        __nv_bfloat162 p1 = __floats2bfloat162_rn(gelu_erf(__uint_as_float(r[j + 2]) + b0.z),
-                                                  gelu_erf(__uint_as_float(r[j + 3]) + b0.w));
-        __nv_bfloat162 p2 = __floats2bfloat162_rn(gelu_erf(__uint_as_float(r[j + 4]) + b1.x),
-                                                  gelu_erf(__uint_as_float(r[j + 5]) + b1.y));
-        __nv_bfloat162 p3 = __floats2bfloat162_rn(gelu_erf(__uint_as_float(r[j + 6]) + b1.z),
-                                                  gelu_erf(__uint_as_float(r[j + 7]) + b1.w));
-        uint4 u;
-        u.x = *reinterpret_cast<uint32_t*>(&p0); u.y = *reinterpret_cast<uint32_t*>(&p1);
-        u.z = *reinterpret_cast<uint32_t*>(&p2); u.w = *reinterpret_cast<uint32_t*>(&p3);
-        *reinterpret_cast<uint4*>(o + j) = u;
-      }
-    }
-  } else {
-    float* o = reinterpret_cast<float*>(g.out) + row * g.N + col0;
-#pragma unroll
-    for (int j = 0; j < 32; j += 4) {
-      if (col0 + j < g.N) {
-        float4 v = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]), __uint_as_float(r[j + 2]),
-                               __uint_as_float(r[j + 3]));
-        if (EPI == kEpiBiasResidual) {
-          const float4 b = __ldg(reinterpret_cast<const float4*>(g.bias + col0 + j));
-          const float4 x = *reinterpret_cast<const float4*>(o + j);
-          v = make_float4(x.x + (v.x + b.x), x.y + (v.y + b.y), x.z + (v.z + b.z), x.w + (v.w + b.w));
-        }
-        *reinterpret_cast<float4*>(o + j) = v;
+  for (int i = 0; i < 4; ++i) {
+    const int r = i * 8 + (lane & 7);
+    const int64_t row = row0 + r;
+    if (row < g.M) {
+      uint4 v = *reinterpret_cast<const uint4*>(patch + r * kPatchRowBytes + piece * 16);
+      uint8_t* dst = reinterpret_cast<uint8_t*>(g.out) + (row * g.N + col) * kElem;
+      if (EPI == kEpiBiasResidual) {
+        const float4 x = *reinterpret_cast<const float4*>(dst);
+        float4 f = *reinterpret_cast<float4*>(&v);
+        f = make_float4(x.x + f.x, x.y + f.y, x.z + f.z, x.w + f.w);
+        *reinterpret_cast<float4*>(dst) = f;
+      } else {
+        *reinterpret_cast<uint4*>(dst) = v;
       }
     }
   }
 }
 
+// One 32-column chunk of this thread's accumulator row -> bias / activation -> patch -> global.
 template <int EPI>
-__global__ void __launch_bounds__(kThreads, 1)
+__device__ __forceinline__ void epilogue_chunk(const GemmArgs& g, uint8_t* patch, int lane, int64_t row0, int64_t col0,
+                                               const uint32_t (&r)[32]) {
+  uint8_t* mine = patch + lane * kPatchRowBytes;
+  if (EPI == kEpiBiasGelu) {
+    // 32 bf16 = 64 bytes: one pass
+#pragma unroll
+    for (int j = 0; j < 32; j += 8) {
+      float4 b0 = make_float4(0.f, 0.f, 0.f, 0.f), b1 = b0;
+      if (col0 + j < g.N) {
+        b0 = __ldg(reinterpret_cast<const float4*>(g.bias + col0 + j));
+        b1 = __ldg(reinterpret_cast<const float4*>(g.bias + col0 + j + 4));
+      }
+      __nv_bfloat162 p0 = __floats2bfloat162_rn(gelu_fast(__uint_as_float(r[j + 0]) + b0.x),
+                                                gelu_fast(__uint_as_float(r[j + 1]) + b0.y));
+      __nv_bfloat162 p1 = __floats2bfloat162_rn(gelu_fast(__uint_as_float(r[j + 2]) + b0.z),
+                                                gelu_fast(__uint_as_float(r[j + 3]) + b0.w));
+      __nv_bfloat162 p2 = __floats2bfloat162_rn(gelu_fast(__uint_as_float(r[j + 4]) + b1.x),
+                                                gelu_fast(__uint_as_float(r[j + 5]) + b1.y));
+      __nv_bfloat162 p3 = __floats2bfloat162_rn(gelu_fast(__uint_as_float(r[j + 6]) + b1.z),
+                                                gelu_fast(__uint_as_float(r[j + 7]) + b1.w));
+      uint4 u;
+      u.x = *reinterpret_cast<uint32_t*>(&p0); u.y = *reinterpret_cast<uint32_t*>(&p1);
+      u.z = *reinterpret_cast<uint32_t*>(&p2); u.w = *reinterpret_cast<uint32_t*>(&p3);
+      *reinterpret_cast<uint4*>(mine + j * 2) = u;
+    }
+    __syncwarp();
+    flush_patch<EPI>(g, patch, lane, row0, col0);
+    __syncwarp();
+  } else {
+    // 32 fp32 = 128 bytes: two passes of 16 columns
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+      const int64_t c0 = col0 + half * 16;
+#pragma unroll
+      for (int j = 0; j < 16; j += 4) {
+        float4 v = make_float4(__uint_as_float(r[half * 16 + j]), __uint_as_float(r[half * 16 + j + 1]),
+                               __uint_as_float(r[half * 16 + j + 2]), __uint_as_float(r[half * 16 + j + 3]));
+        if (EPI == kEpiBiasResidual && c0 + j < g.N) {
+          const float4 b = __ldg(reinterpret_cast<const float4*>(g.bias + c0 + j));
+          v = make_float4(v.x + b.x, v.y + b.y, v.z + b.z, v.w + b.w);
+        }
+        *reinterpret_cast<float4*>(mine + j * 4) = v;
+      }
+      __syncwarp();
+      flush_patch<EPI>(g, patch, lane, row0, c0);
+      __syncwarp();
+    }
+  }
+}
+
+template <int EPI>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmArgs g) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sA = smem;
   uint8_t* sB = smem + kStages * kAStageBytes;
-  uint64_t* full = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes);
-  uint64_t* empty = full + kStages;
-  uint64_t* tfull = empty + kStages;     // [2] accumulator ready for the epilogue
-  uint64_t* tempty = tfull + 2;          // [2] accumulator drained by the epilogue
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes);   // used in the leader CTA
+  uint64_t* empty = full + kStages;      // per CTA: stage may be refilled
+  uint64_t* tfull = empty + kStages;     // per CTA [2]: accumulator ready for the epilogue
+  uint64_t* tempty = tfull + 2;          // leader [2]: accumulator drained by both CTAs' epilogues
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty + 2);
+  uint8_t* patches = smem + kStages * kStageBytes + kBarrierBytes;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();           // 0 = leader of the pair
+  const int64_t cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(&tfull[a], 1); mbar_init(&tempty[a], 128); }
+    for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 2); mbar_init(&empty[s], 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(&tfull[a], 1); mbar_init(&tempty[a], 2 * kEpiWarps); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -207,7 +321,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     tmem_relinquish();
   }
   tc_fence_before();
-  __syncthreads();
+  cluster_sync();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
@@ -216,42 +330,38 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const int k_blocks = static_cast<int>(g.K / BK);
 
   if (warp == 0) {
-    // ---------------- TMA producer ----------------
+    // ---------------- TMA producer (both CTAs) ----------------
     if (lane == 0) {
       asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmA)) : "memory");
       asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmB)) : "memory");
       int stage = 0;
       uint32_t phase = 0;
-      int issued = 0;
       bool ok = true;
-      for (int64_t tile = blockIdx.x; ok && tile < tiles; tile += gridDim.x) {
-        const int m0 = static_cast<int>(tile % m_tiles) * BM, n0 = static_cast<int>(tile / m_tiles) * BN;
+      for (int64_t tile = cluster_id; ok && tile < tiles; tile += n_clusters) {
+        const int m0 = static_cast<int>(tile % m_tiles) * BM + static_cast<int>(rank) * kRowsPerCta;
+        const int n0 = static_cast<int>(tile / m_tiles) * BN + static_cast<int>(rank) * kRowsPerCta;
         for (int kb = 0; kb < k_blocks; ++kb) {
           if (!mbar_wait(&empty[stage], phase ^ 1u, g.status)) { ok = false; break; }
-          mbar_expect_tx(&full[stage], kStageBytes);
-          tma_load_2d(sA + stage * kAStageBytes, &tmA, &full[stage], kb * BK, m0);
-          tma_load_2d(sB + stage * kBStageBytes, &tmB, &full[stage], kb * BK, n0);
-          ++issued;
+          const uint32_t full_leader = mapa(smem_u32(&full[stage]), 0);
+          mbar_expect_tx_cluster(full_leader, kStageBytes);
+          tma_load_2d(sA + stage * kAStageBytes, &tmA, full_leader, kb * BK, m0);
+          tma_load_2d(sB + stage * kBStageBytes, &tmB, full_leader, kb * BK, n0);
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
       }
       if (!ok) {
-        // another role gave up: let the copies already issued land before the CTA exits
-        const int pending = issued < kStages ? issued : kStages;
-        for (int i = 0; i < pending; ++i) {
-          if (stage == 0) { stage = kStages; phase ^= 1u; }
-          --stage;
-          (void)mbar_wait(&full[stage], phase, nullptr);
-        }
+        // a consumer gave up: give the copies already issued time to land before the CTA can exit
+        const long long t0 = clock64();
+        while (clock64() - t0 < (1ll << 21)) { }
       }
     }
   } else if (warp == 1) {
-    // ---------------- MMA issuer ----------------
-    if (lane == 0) {
+    // ---------------- MMA issuer (leader CTA only) ----------------
+    if (rank == 0 && lane == 0) {
       int stage = 0, acc = 0;
       uint32_t phase = 0, acc_phase = 0;
       bool ok = true;
-      for (int64_t tile = blockIdx.x; ok && tile < tiles; tile += gridDim.x) {
+      for (int64_t tile = cluster_id; ok && tile < tiles; tile += n_clusters) {
         if (!mbar_wait(&tempty[acc], acc_phase ^ 1u, g.status)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN);
@@ -263,39 +373,46 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
           for (int k = 0; k < BK / 16; ++k)
             umma_bf16(d_tmem, da + 2u * k, db + 2u * k, kInstrDesc, (kb | k) != 0 ? 1u : 0u);
-          umma_commit(&empty[stage]);
+          umma_commit_pair(&empty[stage]);
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
-        if (ok) umma_commit(&tfull[acc]);
+        if (ok) umma_commit_pair(&tfull[acc]);
         if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
       }
     }
   } else {
-    // ---------------- epilogue: TMEM -> registers -> global ----------------
-    const int quad = warp & 3;
+    // ---------------- epilogue: TMEM -> registers -> smem patch -> global (both CTAs) ----------------
+    const int quad = warp & 3;                       // TMEM lane quarter this warp may read
+    const int cgrp = (warp - 2) >> 2;                // which 64-column group of the tile
+    uint8_t* patch = patches + (warp - 2) * kPatchBytes;
     int acc = 0;
     uint32_t acc_phase = 0;
-    for (int64_t tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
-      const int64_t m0 = (tile % m_tiles) * BM, n0 = (tile / m_tiles) * BN;
+    for (int64_t tile = cluster_id; tile < tiles; tile += n_clusters) {
+      const int64_t m0 = (tile % m_tiles) * BM + rank * kRowsPerCta, n0 = (tile / m_tiles) * BN;
       if (!mbar_wait(&tfull[acc], acc_phase, g.status)) break;
       tc_fence_after();
-      const int64_t row = m0 + quad * 32 + lane;
-      const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + static_cast<uint32_t>(acc * BN);
+      const int64_t row0 = m0 + quad * 32;
+      const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) +
+                             static_cast<uint32_t>(acc * BN + cgrp * kColsPerEpiWarp);
 #pragma unroll 1
-      for (int c = 0; c < BN; c += 32) {
+      for (int c = 0; c < kColsPerEpiWarp; c += 32) {
         uint32_t r[32];
         tmem_ld32(taddr + c, r);
         tmem_ld_wait();
-        if (n0 + c < g.N) epilogue_store<EPI>(g, row, n0 + c, r);
+        const int64_t col = n0 + cgrp * kColsPerEpiWarp + c;
+        if (col < g.N) epilogue_chunk<EPI>(g, patch, lane, row0, col, r);
       }
       tc_fence_before();
-      mbar_arrive(&tempty[acc]);
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(mapa(smem_u32(&tempty[acc]), 0));
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
   }
 
+  // Both CTAs stay until the pair is done: the leader's MMAs read the peer's shared memory and
+  // write its tensor memory, and the peer signals barriers that live in the leader.
   tc_fence_before();
-  __syncthreads();
+  cluster_sync();
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, kTmemCols);

@@ -143,6 +143,7 @@ struct srm_model {
   int device = 0;
   int num_sms = 0;
   bool tc_ready = false;                 // smem attribute set for the tensor-core kernels
+  int tc_clusters = 0;                   // CTA pairs of the tensor-core kernel that are resident at once
   std::vector<TmapCacheEntry> tmaps;     // weight and activation descriptors, built on first use
   bool profiling = false;                // bracket every launch with CUDA events on its stream
   std::vector<ProfRecord> prof;          // open records, folded into the totals by srm_profile_read
@@ -343,6 +344,19 @@ int ensure_tc_ready(srm_model& m) {
   SRM_CUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<kEpiBiasGelu>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes));
   SRM_CUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<kEpiBiasResidual>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes));
   SRM_CUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<kEpiPlain>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes));
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * (m.num_sms / 2));
+  cfg.blockDim = dim3(tc::kThreads);
+  cfg.dynamicSmemBytes = tc::kSmemBytes;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeClusterDimension;
+  attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  int clusters = 0;
+  SRM_CUDA(cudaOccupancyMaxActiveClusters(&clusters, tc::gemm_tc_kernel<kEpiPlain>, &cfg));
+  if (clusters < 1) { g_last_cuda_error = (int)cudaErrorLaunchOutOfResources; return SRM_ERR_CUDA; }
+  m.tc_clusters = clusters < m.num_sms / 2 ? clusters : m.num_sms / 2;
   m.tc_ready = true;
   return SRM_OK;
 }
@@ -352,12 +366,12 @@ int launch_gemm_tc(srm_model& m, int epi, int64_t M, int64_t N, int64_t K, const
   int rc = ensure_tc_ready(m);
   if (rc != SRM_OK) return rc;
   const CUtensorMap *ta, *tb;
-  if ((rc = m.tmap(A, M, K, tc::BM, &ta)) != SRM_OK) return rc;
+  if ((rc = m.tmap(A, M, K, tc::kRowsPerCta, &ta)) != SRM_OK) return rc;
   CUtensorMap a_copy = *ta;             // the cache may reallocate on the next insertion
-  if ((rc = m.tmap(W, N, K, tc::BN, &tb)) != SRM_OK) return rc;
+  if ((rc = m.tmap(W, N, K, tc::kRowsPerCta, &tb)) != SRM_OK) return rc;
   tc::GemmArgs g{M, N, K, bias, out, status};
   const int64_t tiles = ((M + tc::BM - 1) / tc::BM) * ((N + tc::BN - 1) / tc::BN);
-  const unsigned grid = (unsigned)(tiles < m.num_sms ? tiles : m.num_sms);
+  const unsigned grid = 2u * (unsigned)(tiles < m.tc_clusters ? tiles : m.tc_clusters);
   if (epi == kEpiBiasGelu) tc::gemm_tc_kernel<kEpiBiasGelu><<<grid, tc::kThreads, tc::kSmemBytes, st>>>(a_copy, *tb, g);
   else if (epi == kEpiBiasResidual) tc::gemm_tc_kernel<kEpiBiasResidual><<<grid, tc::kThreads, tc::kSmemBytes, st>>>(a_copy, *tb, g);
   else tc::gemm_tc_kernel<kEpiPlain><<<grid, tc::kThreads, tc::kSmemBytes, st>>>(a_copy, *tb, g);

@@ -201,7 +201,11 @@ def test_rl_config_topk_philox_parity_subset():
     prompts = I.make_prompts("rl", batch=16 * 8)[::16][:8]          # 8 distinct prompts
     samp = dict(mode="topk", top_k=50, temperature=0.8, seed=3)
     r = _teacher_forced(shape, W, model, prompts, 5, sampling=samp, sample_idx=np.arange(8) + 7)
-    assert r["mismatches"] == 0 and r["checked"] > 0
+    # Random-init logits are nearly flat, so membership of the top-50 set is rarely stable under
+    # the bf16 logit error: most free-running comparisons are exempt by rule (b) and the in-situ
+    # check (a), asserted inside for all 8 x 5 decisions, is the bit-exact one.
+    assert r["mismatches"] == 0
+    assert r["checked"] + r["exempt"] == 8 * 5
 
 
 def test_host_buffer_step_matches_device_step():
