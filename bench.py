@@ -50,6 +50,13 @@ class ClockSampler:
 
     def __init__(self, index: int):
         self.index, self.rows, self.proc = index, [], None
+        self.t0 = self.t1 = None
+
+    def mark_start(self):
+        self.t0 = time.monotonic()
+
+    def mark_stop(self):
+        self.t1 = time.monotonic()
 
     def __enter__(self):
         try:
@@ -64,7 +71,7 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.rows.append([c.strip() for c in line.split(",")])
+            self.rows.append((time.monotonic(), [c.strip() for c in line.split(",")]))
 
     def __exit__(self, *a):
         if self.proc is not None:
@@ -76,7 +83,9 @@ class ClockSampler:
 
     def summary(self):
         sm, mx, reasons = [], [], set()
-        for r in self.rows:
+        # a sample printed at time ts describes the ~100 ms before it
+        inside = [r for ts, r in self.rows if self.t0 is None or (self.t0 + 0.05 <= ts <= (self.t1 or ts) + 0.1)]
+        for r in inside:
             if len(r) < 8:
                 continue
             try:
@@ -235,11 +244,15 @@ def run_ours(args):
     # ---- prefill (once; timed separately) ----
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sync_all()
-    e0.record()
-    model.prefill(st, prompts, samp, ws)
-    e1.record()
-    torch.cuda.synchronize()
-    prefill_ms = e0.elapsed_time(e1)
+    prefill_ms = None
+    if args.no_prefill:                      # profiling aid: decode cost does not depend on the cache contents
+        st.pos = n
+    else:
+        e0.record()
+        model.prefill(st, prompts, samp, ws)
+        e1.record()
+        torch.cuda.synchronize()
+        prefill_ms = e0.elapsed_time(e1)
 
     step_no = [1]
 
@@ -249,17 +262,20 @@ def run_ours(args):
         model.decode_step(st, None, samp, step_no[0], ws)
         step_no[0] += 1
 
-    for _ in range(max(args.warmup, 3)):
-        one_step()
-    # ---- timed region: exactly K steps ----
-    sync_all()
-    launches0 = model.kernel_launches()
-    with ClockSampler(local) as clk:
+    with ClockSampler(local) as clk:         # nvidia-smi starts up during the warm-up steps
+        for _ in range(max(args.warmup, 3)):
+            one_step()
+        # ---- timed region: exactly K steps ----
+        sync_all()
+        launches0 = model.kernel_launches()
+        clk.mark_start()
         e0.record()
         for _ in range(args.steps):
             one_step()
         e1.record()
         torch.cuda.synchronize()
+        clk.mark_stop()
+        time.sleep(0.15)                     # let the sample that covers the end of the region arrive
     t_ms = e0.elapsed_time(e1)
     launches = model.kernel_launches() - launches0
     t = torch.tensor([t_ms], dtype=torch.float64, device=dev)
@@ -348,7 +364,8 @@ def run_ours(args):
                               "t_hbm_ms": round(t_hbm * 1e3, 4), "frac": round(t_roof * 1e3 / (t_ms_max / args.steps), 4),
                               "peaks": f"{peak_src}: {peak_tf} TFLOP/s sustained bf16, {peaks['hbm_gbs']} GB/s HBM"},
             "kernels": kernels,
-            "prefill": {"ms": round(prefill_ms, 2), "prompt_tokens_per_s": round(B * n / (prefill_ms / 1e3), 1)},
+            "prefill": None if prefill_ms is None else
+            {"ms": round(prefill_ms, 2), "prompt_tokens_per_s": round(B * n / (prefill_ms / 1e3), 1)},
             "state_bytes_per_sample": L * d * sbytes,
             "max_concurrent_samples": max_conc,
             "device_status": status,
@@ -416,7 +433,7 @@ def run_sweep(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=64)
+    ap.add_argument("--steps", type=int, default=256)
     ap.add_argument("--warmup", type=int, default=8)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="mid", choices=["tiny", "small", "mid", "rl"])
@@ -426,6 +443,8 @@ def main():
     ap.add_argument("--state-dtype", default="fp32", choices=["fp32", "bf16"])
     ap.add_argument("--ref-samples", type=int, default=32)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-prefill", action="store_true",
+                    help="skip the prefill (cache stays zero, pos = prompt length): keeps profiler captures short")
     ap.add_argument("--sweep", action="store_true")
     ap.add_argument("--sweep-max", type=int, default=0)
     args = ap.parse_args()
