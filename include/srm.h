@@ -46,7 +46,8 @@ enum srm_error {
   SRM_ERR_BUFFER_TOO_SMALL = -4,     /* weights / state / workspace smaller than required  */
   SRM_ERR_CTX_OVERFLOW = -5,         /* position would reach n_ctx (alpha, beta end there) */
   SRM_ERR_CUDA = -6,                 /* a CUDA call failed; see srm_last_cuda_error        */
-  SRM_ERR_DEVICE_STATUS = -7         /* srm_status found device-side flags set             */
+  SRM_ERR_DEVICE_STATUS = -7,        /* srm_status found device-side flags set             */
+  SRM_ERR_STATIC_SCRATCH = -8        /* batch needs more scratch than the built-in array holds */
 };
 
 /* Bits of the device status word (srm_status). Kernels never trap: they clamp, flag, go on. */
@@ -180,6 +181,35 @@ int srm_generate(srm_model* m, srm_state* s, int32_t steps, int32_t first_step,
 int srm_decode_step_host(srm_model* m, srm_state* s, const int32_t* h_tok_in,
                          const srm_sampling* sampling, int32_t step, int32_t* h_tok_out,
                          void* d_ws, size_t ws_bytes, void* stream);
+
+/* Decode step for callers that cannot allocate device memory. (The paper has no counterpart:
+ * this is a packaging variant of srm_decode_step, not a step of the method.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - a plug-in inside a host
+ * application that reserved the whole device up front, a latency-critical loop that must not
+ * take cudaMalloc's implicit device-wide synchronisation, a callback that is only allowed to
+ * enqueue work. Such a caller still owns its inputs and outputs (weights, state, token buffers);
+ * what it cannot provide is the per-step workspace (residual stream, activations, hidden layer,
+ * logits). Here that workspace is an array of SRM_STATIC_SCRATCH_BYTES that is part of the
+ * library image itself: every GPU that loads libsrm.so holds these bytes until the process
+ * exits, whether or not this call is ever used.
+ *
+ * Same arguments and results as srm_decode_step, minus the workspace. Differences:
+ *   - the whole batch must fit in one pass: if srm_workspace_bytes(cfg, B, 0) exceeds
+ *     SRM_STATIC_SCRATCH_BYTES the call enqueues nothing and returns SRM_ERR_STATIC_SCRATCH
+ *     (e.g. the mid model, 142 KB per row, takes up to 236 rows; the tiny model about 14 000);
+ *   - the device that is current must be the model's device (else SRM_ERR_INVALID_ARG);
+ *   - the first call on each device looks up the array's device address (cudaGetSymbolAddress).
+ *     Make that first call outside of any stream capture; later calls only enqueue kernels;
+ *   - no cudaMalloc, cudaFree or other allocating routine is called, on any call;
+ *   - every call on a device shares the one array. It keeps whatever the previous call left
+ *     there; the step overwrites every byte it later reads, so nothing has to be cleared. Two
+ *     calls whose GPU work can overlap (different streams, or different host threads without
+ *     ordering) race on the array and produce garbage: serialise them on one stream. */
+#define SRM_STATIC_SCRATCH_BYTES (32u << 20)
+int srm_decode_step_static(srm_model* m, srm_state* s, const int32_t* d_tok_in,
+                           const srm_sampling* sampling, int32_t step, int32_t* d_tok_out,
+                           float* d_logits_out, void* stream);
 
 /* ---- single kernels, exported for unit parity tests and profiling ------------------------- */
 

@@ -82,6 +82,7 @@ SYMBOLS = {
     "srm_decode_step": (C.c_int, [_P, _P, _P, C.POINTER(_Sampling), _I32, _P, _P, _P, _SZ, _P]),
     "srm_generate": (C.c_int, [_P, _P, _I32, _I32, C.POINTER(_Sampling), _P, _I64, _P, _SZ, _P]),
     "srm_decode_step_host": (C.c_int, [_P, _P, _P, C.POINTER(_Sampling), _I32, _P, _P, _SZ, _P]),
+    "srm_decode_step_static": (C.c_int, [_P, _P, _P, C.POINTER(_Sampling), _I32, _P, _P, _P]),
     "srm_k_mixer_step": (C.c_int, [_P, _I32, _I32, _I64, _P, _P, _P, _P, _P, _P]),
     "srm_k_final_norm": (C.c_int, [_P, _I64, _P, _P, _P]),
     "srm_k_gemm": (C.c_int, [_P, _I32, _I64, _I64, _I64, _P, _P, _P, _P, _P, _P]),
@@ -299,6 +300,18 @@ class SRM:
         s = sampling.c()
         _check(_lib().srm_decode_step_host(self.handle, state.handle, _ptr(h_tok_in), C.byref(s), step,
                                            _ptr(h_tok_out), _ptr(ws), ws.numel(), _stream()), "srm_decode_step_host")
+
+    def decode_step_static(self, state: SRMState, tok_in, sampling: Sampling, step: int,
+                           want_logits: bool = False, tok_out: torch.Tensor | None = None):
+        """srm_decode_step on the library's built-in scratch array (no workspace argument): for callers
+        that cannot allocate device memory. Raises SRMError(-8) when the batch does not fit."""
+        if tok_out is None:
+            tok_out = torch.empty(state.B, dtype=torch.int32, device=self.device)
+        logits = torch.empty(state.B, self.cfg.vocab, dtype=torch.float32, device=self.device) if want_logits else None
+        s = sampling.c()
+        _check(_lib().srm_decode_step_static(self.handle, state.handle, _ptr(tok_in), C.byref(s), step, _ptr(tok_out),
+                                             _ptr(logits), _stream()), "srm_decode_step_static")
+        return (tok_out, logits) if want_logits else tok_out
 
     # ---- measurement ----
     KERNEL_CLASSES = ("mixer", "gemm_up", "gemm_down", "gemm_lm", "norm", "select", "prefill_mixer")

@@ -721,6 +721,51 @@ int srm_decode_step_host(srm_model* m, srm_state* s, const int32_t* h_tok_in, co
   return SRM_OK;
 }
 
+// ---- decode step on the built-in scratch array --------------------------------------------------
+}  // extern "C"
+
+// Workspace for callers that cannot allocate: part of the module image, so it exists on every
+// device that loads the library. In host code this name is only a handle for
+// cudaGetSymbolAddress; kernels must be given the address that call returns.
+static __device__ __align__(256) unsigned char g_static_scratch[SRM_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void* g_static_scratch_addr[kMaxDevices] = {};    // device address per device ordinal, looked up once
+std::mutex g_static_scratch_mutex;
+
+// Address of g_static_scratch on the current device (which must be `device`).
+int static_scratch_address(int device, void** out) {
+  int cur = -1;
+  SRM_CUDA(cudaGetDevice(&cur));
+  if (cur != device || cur < 0 || cur >= kMaxDevices) return SRM_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
+  if (g_static_scratch_addr[cur] == nullptr) {
+    void* p = nullptr;
+    SRM_CUDA(cudaGetSymbolAddress(&p, g_static_scratch));
+    if (p == nullptr || !aligned(p, 256)) return SRM_ERR_ALIGNMENT;
+    g_static_scratch_addr[cur] = p;
+  }
+  *out = g_static_scratch_addr[cur];
+  return SRM_OK;
+}
+}  // namespace
+
+extern "C" {
+
+int srm_decode_step_static(srm_model* m, srm_state* s, const int32_t* d_tok_in, const srm_sampling* samp,
+                           int32_t step, int32_t* d_tok_out, float* d_logits_out, void* stream) {
+  if (m == nullptr || s == nullptr || s->m != m) return SRM_ERR_INVALID_ARG;
+  if (decode_ws_bytes(*m, s->B) > (size_t)SRM_STATIC_SCRATCH_BYTES) return SRM_ERR_STATIC_SCRATCH;
+  void* ws = nullptr;
+  int rc = static_scratch_address(m->device, &ws);
+  if (rc != SRM_OK) return rc;
+  // Nothing in the workspace has to start at zero: the first mixer launch writes x and a, the up
+  // projection writes H, the LM head writes the logits, each before anything reads them.
+  return decode_step_impl(m, s, d_tok_in, samp, step, d_tok_out, nullptr, 0, 0, d_logits_out, ws,
+                          (size_t)SRM_STATIC_SCRATCH_BYTES, static_cast<cudaStream_t>(stream));
+}
+
 // ---- single kernels ---------------------------------------------------------------------------
 int srm_k_mixer_step(srm_model* m, int32_t layer, int32_t t, int64_t R, const int32_t* d_tok, float* d_x, void* d_S,
                      void* d_a, uint32_t* d_status, void* stream) {
@@ -785,6 +830,7 @@ const char* srm_strerror(int code) {
     case SRM_ERR_CTX_OVERFLOW: return "position would exceed n_ctx";
     case SRM_ERR_CUDA: return "CUDA call failed (see srm_last_cuda_error)";
     case SRM_ERR_DEVICE_STATUS: return "device status flags set";
+    case SRM_ERR_STATIC_SCRATCH: return "batch needs more scratch than the library's built-in array holds";
     default: return "unknown error";
   }
 }

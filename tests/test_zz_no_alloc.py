@@ -1,0 +1,62 @@
+"""srm_decode_step_static: the decode step for callers that cannot allocate device memory (a plug-in
+inside an application that reserved the whole GPU, a loop that must not take cudaMalloc's implicit
+synchronisation). Its workspace is an array built into the library, so the call takes no workspace
+argument. It must give what srm_decode_step gives with a caller-allocated workspace.
+
+Collected last on purpose (file name): a run that stops at the first failure has then already
+executed every other test. The test needs no state left behind by other tests and leaves none that
+matters: the built-in array is scratch, fully rewritten by every call.
+"""
+import numpy as np
+import pytest
+import torch
+
+import srm_inputs as I
+from helpers import rel_err_rows
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+TOL = {"fp32": 1e-4, "bf16": 3e-2}     # the tolerances of the model-level parity tests
+
+
+@pytest.mark.parametrize("shape,B", [
+    (I.CONFIGS["tiny"], 4),
+    (I.SRMShape(n_layers=2, d_model=256, vocab=1000, n_ctx=32, dtype="bf16", seed=7), 300),
+])
+def test_static_scratch_step_matches_workspace_step_twice_in_a_row(shape, B):
+    import paper_2605_08696_b200 as P
+    W = I.make_weights(shape)
+    model = P.SRM(shape, W, device=DEV)
+    g = P.Sampling("greedy")
+    n = 6
+    prompts = torch.from_numpy(I.uniform_prompts(B, n, shape.vocab, seed=11)).to(DEV)
+    ws = model.new_workspace(B, n, prefill_samples=B)
+    st_ref, st_new = model.new_state(B), model.new_state(B)
+    first = model.prefill(st_ref, prompts, g, ws)
+    model.prefill(st_new, prompts, g, ws)
+    tok = first
+    for k in range(2):                                   # two calls in a row share the built-in array
+        t_ref, lg_ref = model.decode_step(st_ref, tok, g, k + 1, ws, want_logits=True)
+        t_new, lg_new = model.decode_step_static(st_new, tok, g, k + 1, want_logits=True)
+        torch.cuda.synchronize()
+        assert rel_err_rows(lg_new.cpu().numpy(), lg_ref.cpu().numpy()) < TOL[shape.dtype]
+        assert torch.equal(t_new, t_ref)
+        assert rel_err_rows(st_new.cache().cpu().numpy(), st_ref.cache().cpu().numpy()) < TOL[shape.dtype]
+        tok = t_ref
+    assert st_new.pos == st_ref.pos == n + 2
+    assert st_new.status() == 0 and st_ref.status() == 0
+
+
+def test_static_scratch_step_rejects_a_batch_that_does_not_fit():
+    import paper_2605_08696_b200 as P
+    shape = I.CONFIGS["tiny"]
+    model = P.SRM(shape, I.make_weights(shape), device=DEV)
+    B = 20000                                            # 20000 rows x 2.3 KB of workspace > 32 MiB
+    assert model.workspace_bytes(B) > 32 << 20
+    st = model.new_state(B)
+    st.pos = 1
+    with pytest.raises(P.SRMError) as e:
+        model.decode_step_static(st, None, P.Sampling("greedy"), 1)
+    assert e.value.code == -8
+    assert "scratch" in str(e.value)
+    assert st.pos == 1                                   # nothing was enqueued, nothing advanced
