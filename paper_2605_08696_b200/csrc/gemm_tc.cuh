@@ -17,9 +17,12 @@
 // warps 2..17 = epilogue (warp w reads TMEM lanes 32*(w%4) .. +31, one accumulator row per thread;
 // the four warps that share a lane quarter split the tile's columns; four warps per scheduler hide
 // each other's TMEM / shared / global latencies, since with K = d the epilogue's instruction issue
-// is as long as the tile's MMAs). Each epilogue warp transposes its values through a private
-// shared-memory patch so that every global store (and residual load) instruction covers eight
-// rows x 64 contiguous bytes in whole 32-byte sectors.
+// is as long as the tile's MMAs). Each epilogue warp stages 32 rows x 128 bytes of finished
+// output in a private, 128-byte-swizzled shared-memory buffer and hands it to the TMA unit: a tiled
+// bulk store for the activation and logit epilogues, a tiled bulk reduce-add (fp32 add performed in
+// L2) for the residual epilogue, so no thread computes a global address, waits on a global load of
+// x, or holds a store in flight. Every element of x receives exactly one add per launch, so the
+// result does not depend on timing. Rows and columns beyond M, N are clipped by the TMA unit.
 // Every wait is bounded: after ~2^31 clock cycles a waiter raises kStatusWaitTimeout, leaves its
 // loop, and both CTAs still meet at the final cluster barrier, release tensor memory and exit.
 #pragma once
@@ -41,9 +44,9 @@ constexpr int kStageBytes = kAStageBytes + kBStageBytes;
 constexpr int kBarrierBytes = 256;
 constexpr int kEpiWarps = 16;
 constexpr int kColsPerEpiWarp = BN / (kEpiWarps / 4);   // 64
-constexpr int kPatchRowBytes = 80;               // 64 data bytes + 16 pad (bank spread)
-constexpr int kPatchBytes = 32 * kPatchRowBytes; // one patch per epilogue warp
-constexpr int kSmemBytes = kStages * kStageBytes + kEpiWarps * kPatchBytes + kBarrierBytes + 1024;  // +1024: alignment
+constexpr int kOutBoxRows = 32;                  // one epilogue warp's rows
+constexpr int kOutBoxBytes = kOutBoxRows * 128;  // staging buffer of one epilogue warp: 32 rows x 128 bytes
+constexpr int kSmemBytes = kStages * kStageBytes + kEpiWarps * kOutBoxBytes + kBarrierBytes + 1024;  // +1024: alignment
 constexpr int kThreads = 64 + kEpiWarps * 32;
 constexpr int kTmemCols = 512;                   // two accumulators of BN fp32 columns
 constexpr long long kWaitLimitCycles = 1ll << 31;
@@ -160,6 +163,34 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+// ---- bulk tensor stores (shared -> global), tracked per issuing thread in bulk async-groups ----
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, const void* src, int x, int y) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(src)), "r"(x), "r"(y)
+               : "memory");
+}
+// Same store, marked evict-first in L2: for output that is written once and not read again soon (the
+// logits), so that it does not push the operands the mainloop keeps re-reading out of L2.
+__device__ __forceinline__ void tma_store_2d_streaming(const CUtensorMap* map, const void* src, int x, int y) {
+  uint64_t policy;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group.L2::cache_hint [%0, {%2, %3}], [%1], %4;"
+               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(src)), "r"(x), "r"(y), "l"(policy)
+               : "memory");
+}
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* map, const void* src, int x, int y) {
+  asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(src)), "r"(x), "r"(y)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// the bulk operations committed by this thread have finished READING shared memory
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+// ... have completed altogether
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+// orders this thread's generic-proxy writes to shared memory before later async-proxy (TMA) reads
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
 // Shared-memory matrix descriptor of a K-major bf16 tile whose rows are 128 bytes (64 elements)
 // laid out by TMA with the 128-byte swizzle: 8-row groups are 1024 bytes apart (SBO), the
 // leading-dimension offset is not used by swizzled K-major layouts, descriptor version 1,
@@ -184,10 +215,13 @@ struct GemmArgs {
   uint32_t* status;
 };
 
-// GELU(v) = v * Phi(v) with erfc by the rational approximation 7.1.26 of Abramowitz & Stegun
-// (|error| <= 1.5e-7, far below the bf16 resolution of the value it feeds; coefficients halved so
-// that h = erfc(|v|/sqrt 2) / 2 = Phi(-|v|)). One rcp.approx and one ex2.approx per element keep
-// the epilogue within the issue slots a K = d tile leaves.
+// GELU(v) = v * Phi(v) with the normal CDF written as a logistic function of an odd polynomial,
+//   Phi(v) ~= 1 / (1 + exp(-v (a + b v^2 + c v^4))),   a = 1.59501055, b = 7.40160400e-2, c = -7.03804784e-4
+// (coefficients fitted to minimise the maximum error of v * Phi(v) over the real line; |error| <= 2.6e-5,
+// two orders below the bf16 resolution of the hidden activations it feeds). v^2 is clamped at 64 so the
+// polynomial stays positive; beyond |v| = 8 the logistic term is 0 or 1 to fp32 precision anyway.
+// Nine instructions per element, two of them on the special-function unit (ex2, rcp): the epilogue of a
+// K = d tile has about as many issue slots as the tile's MMAs take, so the erf route does not fit.
 __device__ __forceinline__ float rcp_approx(float x) {
   float r;
   asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
@@ -199,113 +233,101 @@ __device__ __forceinline__ float ex2_approx(float x) {
   return r;
 }
 __device__ __forceinline__ float gelu_fast(float v) {
-  const float ax = fabsf(v) * 0.70710678118654752440f;
-  const float t = rcp_approx(fmaf(0.3275911f, ax, 1.0f));
-  const float e = ex2_approx(ax * ax * -1.4426950408889634f);      // exp(-v^2 / 2)
-  float p = fmaf(t, 0.5307027145f, -0.7265760135f);
-  p = fmaf(t, p, 0.7107068705f);
-  p = fmaf(t, p, -0.142248368f);
-  p = fmaf(t, p, 0.127414796f);
-  const float h = p * t * e;                                       // Phi(-|v|)
-  return v * (v < 0.f ? h : 1.0f - h);
+  constexpr float kLog2e = 1.4426950408889634f;
+  const float s = fminf(v * v, 64.0f);
+  float q = fmaf(s, 7.03804784e-4f * kLog2e, -7.40160400e-2f * kLog2e);
+  q = fmaf(s, q, -1.59501055f * kLog2e);                 // -log2(e) * (a + b s + c s^2)
+  const float e = ex2_approx(q * v);                     // exp(-v (a + b s + c s^2))
+  return v * rcp_approx(e + 1.0f);
 }
 
-// Writes one 32-row x 64-byte patch (row = the staging thread's lane) from `patch` to global memory.
-// Lane l handles the 16-byte piece l/8 of rows (l%8) + 8*i: a quarter-warp then reads eight rows whose
-// 80-byte stride spreads them over distinct banks, and the warp as a whole still covers eight rows x
-// 64 contiguous bytes per instruction.
+// Hands this warp's 32 rows x 128 bytes (v = the 32 words of the lane's row) to the TMA unit.
+// The staging buffer uses the 128-byte swizzle of the output tensor map: the 16-byte piece q of row r
+// sits at piece q ^ (r % 8), which also makes the eight lanes of a quarter-warp hit distinct banks.
+// Lane 0 issues the bulk operation and is the only thread that tracks its completion.
 template <int EPI>
-__device__ __forceinline__ void flush_patch(const GemmArgs& g, const uint8_t* patch, int lane, int64_t row0,
-                                            int64_t col0) {
-  constexpr int kElem = (EPI == kEpiBiasGelu) ? 2 : 4;
-  constexpr int kPer16 = 16 / kElem;
-  const int piece = lane >> 3;
-  const int64_t col = col0 + piece * kPer16;
-  if (col >= g.N) return;
+__device__ __forceinline__ void emit_box(const CUtensorMap* tmD, uint8_t* buf, int lane, int col, int row,
+                                         const uint32_t (&v)[32]) {
+  if (lane == 0) bulk_wait_read();          // the previous box has left the buffer
+  __syncwarp();
+  uint8_t* mine = buf + lane * 128;
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const int r = i * 8 + (lane & 7);
-    const int64_t row = row0 + r;
-    if (row < g.M) {
-      uint4 v = *reinterpret_cast<const uint4*>(patch + r * kPatchRowBytes + piece * 16);
-      uint8_t* dst = reinterpret_cast<uint8_t*>(g.out) + (row * g.N + col) * kElem;
-      if (EPI == kEpiBiasResidual) {
-        const float4 x = *reinterpret_cast<const float4*>(dst);
-        float4 f = *reinterpret_cast<float4*>(&v);
-        f = make_float4(x.x + f.x, x.y + f.y, x.z + f.z, x.w + f.w);
-        *reinterpret_cast<float4*>(dst) = f;
-      } else {
-        *reinterpret_cast<uint4*>(dst) = v;
-      }
-    }
+  for (int q = 0; q < 8; ++q)
+    *reinterpret_cast<uint4*>(mine + ((q ^ (lane & 7)) << 4)) = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+  fence_async_smem();
+  __syncwarp();
+  if (lane == 0) {
+    if (EPI == kEpiBiasResidual) tma_reduce_add_2d(tmD, buf, col, row);
+    else if (EPI == kEpiPlain) tma_store_2d_streaming(tmD, buf, col, row);
+    else tma_store_2d(tmD, buf, col, row);
+    bulk_commit();
   }
 }
 
-// One 32-column chunk of this thread's accumulator row -> bias / activation -> patch -> global.
+// The 64 accumulator columns [col0, col0 + 64) of this warp's 32 rows: TMEM -> registers -> bias /
+// activation -> one (bf16) or two (fp32) boxes of 128 bytes per row.
 template <int EPI>
-__device__ __forceinline__ void epilogue_chunk(const GemmArgs& g, uint8_t* patch, int lane, int64_t row0, int64_t col0,
-                                               const uint32_t (&r)[32]) {
-  uint8_t* mine = patch + lane * kPatchRowBytes;
+__device__ __forceinline__ void epilogue_columns(const GemmArgs& g, const CUtensorMap* tmD, uint8_t* buf, int lane,
+                                                 uint32_t taddr, int row0, int col0) {
   if (EPI == kEpiBiasGelu) {
-    // 32 bf16 = 64 bytes: one pass
-#pragma unroll
-    for (int j = 0; j < 32; j += 8) {
-      float4 b0 = make_float4(0.f, 0.f, 0.f, 0.f), b1 = b0;
-      if (col0 + j < g.N) {
-        b0 = __ldg(reinterpret_cast<const float4*>(g.bias + col0 + j));
-        b1 = __ldg(reinterpret_cast<const float4*>(g.bias + col0 + j + 4));
-      }
-      __nv_bfloat162 p0 = __floats2bfloat162_rn(gelu_fast(__uint_as_float(r[j + 0]) + b0.x),
-                                                gelu_fast(__uint_as_float(r[j + 1]) + b0.y));
-      __nv_bfloat162 p1 = __floats2bfloat162_rn(gelu_fast(__uint_as_float(r[j + 2]) + b0.z),
-                                                gelu_fast(__uint_as_float(r[j + 3]) + b0.w));
-      __nv_bfloat162 p2 = __floats2bfloat162_rn(gelu_fast(__uint_as_float(r[j + 4]) + b1.x),
-                                                gelu_fast(__uint_as_float(r[j + 5]) + b1.y));
-      __nv_bfloat162 p3 = __floats2bfloat162_rn(gelu_fast(__uint_as_float(r[j + 6]) + b1.z),
-                                                gelu_fast(__uint_as_float(r[j + 7]) + b1.w));
-      uint4 u;
-      u.x = *reinterpret_cast<uint32_t*>(&p0); u.y = *reinterpret_cast<uint32_t*>(&p1);
-      u.z = *reinterpret_cast<uint32_t*>(&p2); u.w = *reinterpret_cast<uint32_t*>(&p3);
-      *reinterpret_cast<uint4*>(mine + j * 2) = u;
-    }
-    __syncwarp();
-    flush_patch<EPI>(g, patch, lane, row0, col0);
-    __syncwarp();
-  } else {
-    // 32 fp32 = 128 bytes: two passes of 16 columns
+    uint32_t v[32];
 #pragma unroll
     for (int half = 0; half < 2; ++half) {
-      const int64_t c0 = col0 + half * 16;
+      uint32_t r[32];
+      tmem_ld32(taddr + 32 * half, r);
+      tmem_ld_wait();
+      const int col = col0 + 32 * half;
 #pragma unroll
-      for (int j = 0; j < 16; j += 4) {
-        float4 v = make_float4(__uint_as_float(r[half * 16 + j]), __uint_as_float(r[half * 16 + j + 1]),
-                               __uint_as_float(r[half * 16 + j + 2]), __uint_as_float(r[half * 16 + j + 3]));
-        if (EPI == kEpiBiasResidual && c0 + j < g.N) {
-          const float4 b = __ldg(reinterpret_cast<const float4*>(g.bias + c0 + j));
-          v = make_float4(v.x + b.x, v.y + b.y, v.z + b.z, v.w + b.w);
-        }
-        *reinterpret_cast<float4*>(mine + j * 4) = v;
+      for (int j = 0; j < 32; j += 4) {
+        float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (col + j < g.N) b = __ldg(reinterpret_cast<const float4*>(g.bias + col + j));
+        __nv_bfloat162 p;
+        p = __floats2bfloat162_rn(gelu_fast(__uint_as_float(r[j + 0]) + b.x), gelu_fast(__uint_as_float(r[j + 1]) + b.y));
+        v[16 * half + j / 2] = *reinterpret_cast<uint32_t*>(&p);
+        p = __floats2bfloat162_rn(gelu_fast(__uint_as_float(r[j + 2]) + b.z), gelu_fast(__uint_as_float(r[j + 3]) + b.w));
+        v[16 * half + j / 2 + 1] = *reinterpret_cast<uint32_t*>(&p);
       }
-      __syncwarp();
-      flush_patch<EPI>(g, patch, lane, row0, c0);
-      __syncwarp();
+    }
+    emit_box<EPI>(tmD, buf, lane, col0, row0, v);
+  } else {
+#pragma unroll 1
+    for (int c = 0; c < kColsPerEpiWarp; c += 32) {
+      const int col = col0 + c;
+      if (col >= g.N) break;
+      uint32_t r[32];
+      tmem_ld32(taddr + c, r);
+      tmem_ld_wait();
+      if (EPI == kEpiBiasResidual) {
+#pragma unroll
+        for (int j = 0; j < 32; j += 4) {
+          if (col + j < g.N) {
+            const float4 b = __ldg(reinterpret_cast<const float4*>(g.bias + col + j));
+            r[j + 0] = __float_as_uint(__uint_as_float(r[j + 0]) + b.x);
+            r[j + 1] = __float_as_uint(__uint_as_float(r[j + 1]) + b.y);
+            r[j + 2] = __float_as_uint(__uint_as_float(r[j + 2]) + b.z);
+            r[j + 3] = __float_as_uint(__uint_as_float(r[j + 3]) + b.w);
+          }
+        }
+      }
+      emit_box<EPI>(tmD, buf, lane, col, row0, r);
     }
   }
 }
 
 template <int EPI>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmArgs g) {
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const __grid_constant__ CUtensorMap tmD, const GemmArgs g) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sA = smem;
   uint8_t* sB = smem + kStages * kAStageBytes;
-  uint64_t* full = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes);   // used in the leader CTA
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes + kEpiWarps * kOutBoxBytes);   // used in the leader CTA
   uint64_t* empty = full + kStages;      // per CTA: stage may be refilled
   uint64_t* tfull = empty + kStages;     // per CTA [2]: accumulator ready for the epilogue
   uint64_t* tempty = tfull + 2;          // leader [2]: accumulator drained by both CTAs' epilogues
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty + 2);
-  uint8_t* patches = smem + kStages * kStageBytes + kBarrierBytes;
+  uint8_t* boxes = smem + kStages * kStageBytes;      // 1024-byte aligned, one staging buffer per epilogue warp
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();           // 0 = leader of the pair
@@ -381,32 +403,28 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       }
     }
   } else {
-    // ---------------- epilogue: TMEM -> registers -> smem patch -> global (both CTAs) ----------------
+    // ---------------- epilogue: TMEM -> registers -> swizzled smem box -> TMA store / reduce (both CTAs) ----
     const int quad = warp & 3;                       // TMEM lane quarter this warp may read
     const int cgrp = (warp - 2) >> 2;                // which 64-column group of the tile
-    uint8_t* patch = patches + (warp - 2) * kPatchBytes;
+    uint8_t* buf = boxes + (warp - 2) * kOutBoxBytes;
+    if (lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmD)) : "memory");
     int acc = 0;
     uint32_t acc_phase = 0;
     for (int64_t tile = cluster_id; tile < tiles; tile += n_clusters) {
       const int64_t m0 = (tile % m_tiles) * BM + rank * kRowsPerCta, n0 = (tile / m_tiles) * BN;
       if (!mbar_wait(&tfull[acc], acc_phase, g.status)) break;
       tc_fence_after();
-      const int64_t row0 = m0 + quad * 32;
+      const int row0 = static_cast<int>(m0) + quad * 32;
+      const int col0 = static_cast<int>(n0) + cgrp * kColsPerEpiWarp;
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) +
                              static_cast<uint32_t>(acc * BN + cgrp * kColsPerEpiWarp);
-#pragma unroll 1
-      for (int c = 0; c < kColsPerEpiWarp; c += 32) {
-        uint32_t r[32];
-        tmem_ld32(taddr + c, r);
-        tmem_ld_wait();
-        const int64_t col = n0 + cgrp * kColsPerEpiWarp + c;
-        if (col < g.N) epilogue_chunk<EPI>(g, patch, lane, row0, col, r);
-      }
+      if (row0 < g.M && col0 < g.N) epilogue_columns<EPI>(g, &tmD, buf, lane, taddr, row0, col0);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(mapa(smem_u32(&tempty[acc]), 0));
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
+    if (lane == 0) bulk_wait_all();                  // the staged boxes must be out before shared memory goes away
   }
 
   // Both CTAs stay until the pair is done: the leader's MMAs read the peer's shared memory and

@@ -113,22 +113,23 @@ EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
-// bf16 row-major [rows, cols] matrix, box = 64 columns (128 bytes, the swizzle span) x box_rows.
-int make_tmap_bf16(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int box_rows) {
+// Row-major [rows, cols] matrix of 2-byte (bf16) or 4-byte (fp32) elements; the box is 128 bytes of
+// one row (the swizzle span) x box_rows rows.
+int make_tmap(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int box_rows, int elem_bytes) {
   EncodeTiledFn fn = encode_tiled_fn();
   if (fn == nullptr) { g_last_cuda_error = (int)cudaErrorNotSupported; return SRM_ERR_CUDA; }
   cuuint64_t gdim[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-  cuuint64_t gstride[1] = {(cuuint64_t)cols * 2};
-  cuuint32_t box[2] = {(cuuint32_t)tc::BK, (cuuint32_t)box_rows};
+  cuuint64_t gstride[1] = {(cuuint64_t)cols * (cuuint64_t)elem_bytes};
+  cuuint32_t box[2] = {(cuuint32_t)(128 / elem_bytes), (cuuint32_t)box_rows};
   cuuint32_t estr[2] = {1, 1};
-  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstride, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  CUresult r = fn(map, elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
+                  const_cast<void*>(base), gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) { g_last_cuda_error = 10000 + (int)r; return SRM_ERR_CUDA; }
   return SRM_OK;
 }
 
-struct TmapCacheEntry { const void* base; int64_t rows, cols; int box_rows; CUtensorMap map; };
+struct TmapCacheEntry { const void* base; int64_t rows, cols; int box_rows, elem_bytes; CUtensorMap map; };
 
 unsigned long long g_kernel_launches = 0;     // kernels launched by this library since load
 
@@ -160,15 +161,19 @@ struct srm_model {
   int state_bytes() const { return cfg.state_dtype == SRM_DTYPE_BF16 ? 2 : 4; }
   int64_t F() const { return (int64_t)cfg.ffn_mult * cfg.d_model; }
 
-  int tmap(const void* base, int64_t rows, int64_t cols, int box_rows, const CUtensorMap** out) {
+  // Copies the descriptor out: the cache may reallocate or be cleared by a later insertion.
+  int tmap(const void* base, int64_t rows, int64_t cols, int box_rows, int elem_bytes, CUtensorMap* out) {
     for (auto& e : tmaps)
-      if (e.base == base && e.rows == rows && e.cols == cols && e.box_rows == box_rows) { *out = &e.map; return SRM_OK; }
+      if (e.base == base && e.rows == rows && e.cols == cols && e.box_rows == box_rows && e.elem_bytes == elem_bytes) {
+        *out = e.map;
+        return SRM_OK;
+      }
     if (tmaps.size() >= 4096) tmaps.clear();
-    TmapCacheEntry e{base, rows, cols, box_rows, {}};
-    int rc = make_tmap_bf16(&e.map, base, rows, cols, box_rows);
+    TmapCacheEntry e{base, rows, cols, box_rows, elem_bytes, {}};
+    int rc = make_tmap(&e.map, base, rows, cols, box_rows, elem_bytes);
     if (rc != SRM_OK) return rc;
     tmaps.push_back(e);
-    *out = &tmaps.back().map;
+    *out = e.map;
     return SRM_OK;
   }
 };
@@ -365,16 +370,16 @@ int launch_gemm_tc(srm_model& m, int epi, int64_t M, int64_t N, int64_t K, const
                    const float* bias, void* out, uint32_t* status, cudaStream_t st) {
   int rc = ensure_tc_ready(m);
   if (rc != SRM_OK) return rc;
-  const CUtensorMap *ta, *tb;
-  if ((rc = m.tmap(A, M, K, tc::kRowsPerCta, &ta)) != SRM_OK) return rc;
-  CUtensorMap a_copy = *ta;             // the cache may reallocate on the next insertion
-  if ((rc = m.tmap(W, N, K, tc::kRowsPerCta, &tb)) != SRM_OK) return rc;
+  CUtensorMap ta, tb, td;
+  if ((rc = m.tmap(A, M, K, tc::kRowsPerCta, 2, &ta)) != SRM_OK) return rc;
+  if ((rc = m.tmap(W, N, K, tc::kRowsPerCta, 2, &tb)) != SRM_OK) return rc;
+  if ((rc = m.tmap(out, M, N, tc::kOutBoxRows, epi == kEpiBiasGelu ? 2 : 4, &td)) != SRM_OK) return rc;
   tc::GemmArgs g{M, N, K, bias, out, status};
   const int64_t tiles = ((M + tc::BM - 1) / tc::BM) * ((N + tc::BN - 1) / tc::BN);
   const unsigned grid = 2u * (unsigned)(tiles < m.tc_clusters ? tiles : m.tc_clusters);
-  if (epi == kEpiBiasGelu) tc::gemm_tc_kernel<kEpiBiasGelu><<<grid, tc::kThreads, tc::kSmemBytes, st>>>(a_copy, *tb, g);
-  else if (epi == kEpiBiasResidual) tc::gemm_tc_kernel<kEpiBiasResidual><<<grid, tc::kThreads, tc::kSmemBytes, st>>>(a_copy, *tb, g);
-  else tc::gemm_tc_kernel<kEpiPlain><<<grid, tc::kThreads, tc::kSmemBytes, st>>>(a_copy, *tb, g);
+  if (epi == kEpiBiasGelu) tc::gemm_tc_kernel<kEpiBiasGelu><<<grid, tc::kThreads, tc::kSmemBytes, st>>>(ta, tb, td, g);
+  else if (epi == kEpiBiasResidual) tc::gemm_tc_kernel<kEpiBiasResidual><<<grid, tc::kThreads, tc::kSmemBytes, st>>>(ta, tb, td, g);
+  else tc::gemm_tc_kernel<kEpiPlain><<<grid, tc::kThreads, tc::kSmemBytes, st>>>(ta, tb, td, g);
   SRM_CUDA(cudaGetLastError());
   return SRM_OK;
 }
