@@ -230,6 +230,15 @@ int srm_k_final_norm(srm_model* m, int64_t R, const float* d_x, void* d_a, void*
 int srm_k_gemm(srm_model* m, int32_t epilogue, int64_t M, int64_t N, int64_t K, const void* d_A,
                const void* d_W, const float* d_bias, void* d_out, uint32_t* d_status,
                void* stream);
+/* LM head with greedy selection fused into the GEMM epilogue (bf16 models only): d_tok[r] =
+ * argmax_v (a[r, :] . W_lm[v, :]), lowest id among equal maxima - the token srm_k_gemm (epilogue 2)
+ * followed by greedy srm_k_select gives, without writing the R x V logits. d_a [R, d] in the
+ * activation type; d_part is scratch of part_bytes >= ceil(V / 256) * 4 * R * 8 bytes, 16-byte aligned.
+ * This is the path srm_decode_step, srm_generate and srm_prefill take for greedy sampling when the
+ * caller does not ask for logits [Recurrent Throughput and Concurrency: finding the next tokens from the
+ * logits is the bottleneck the paper measures at large batch]. */
+int srm_k_lm_head_greedy(srm_model* m, int64_t R, const void* d_a, void* d_part, size_t part_bytes,
+                         int32_t* d_tok, uint32_t* d_status, void* stream);
 /* Token selection on d_logits float[R, V] -> d_tok int32[R]; row r uses sample index
  * sampling->sample_idx_base + r. */
 int srm_k_select(srm_model* m, int64_t R, const float* d_logits, const srm_sampling* sampling,

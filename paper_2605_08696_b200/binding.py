@@ -86,6 +86,7 @@ SYMBOLS = {
     "srm_k_mixer_step": (C.c_int, [_P, _I32, _I32, _I64, _P, _P, _P, _P, _P, _P]),
     "srm_k_final_norm": (C.c_int, [_P, _I64, _P, _P, _P]),
     "srm_k_gemm": (C.c_int, [_P, _I32, _I64, _I64, _I64, _P, _P, _P, _P, _P, _P]),
+    "srm_k_lm_head_greedy": (C.c_int, [_P, _I64, _P, _P, _SZ, _P, _P, _P]),
     "srm_k_select": (C.c_int, [_P, _I64, _P, C.POINTER(_Sampling), _I32, _P, _P, _P]),
     "srm_k_prefill_mixer": (C.c_int, [_P, _I32, _I64, _I32, _P, _P, _P, _P, _P, _P]),
     "srm_profile_enable": (C.c_int, [_P, C.c_int]),
@@ -348,6 +349,10 @@ class SRM:
         N = W.shape[0]
         _check(_lib().srm_k_gemm(self.handle, epilogue, M, N, K, _ptr(A), _ptr(W), _ptr(bias), _ptr(out),
                                  _ptr(status), _stream()), "srm_k_gemm")
+
+    def k_lm_head_greedy(self, a, part, tok, status=None):
+        _check(_lib().srm_k_lm_head_greedy(self.handle, a.shape[0], _ptr(a), _ptr(part), part.numel() * part.element_size(),
+                                           _ptr(tok), _ptr(status), _stream()), "srm_k_lm_head_greedy")
 
     def k_select(self, logits, sampling: Sampling, step, tok, status=None):
         s = sampling.c()

@@ -7,7 +7,12 @@
 
 namespace srm {
 
-enum GemmEpilogue { kEpiBiasGelu = 0, kEpiBiasResidual = 1, kEpiPlain = 2 };
+enum GemmEpilogue {
+  kEpiBiasGelu = 0,       // out = gelu(D + bias) in the activation type
+  kEpiBiasResidual = 1,   // out += D + bias (fp32)
+  kEpiPlain = 2,          // out = D (fp32)
+  kEpiArgmax = 3          // tensor-core kernel only: per-row (max, lowest column) of every 64-column slice of D
+};
 
 constexpr int kSimtBM = 64, kSimtBN = 64, kSimtBK = 16;
 

@@ -211,9 +211,13 @@ constexpr uint32_t kInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(B
 struct GemmArgs {
   int64_t M, N, K;
   const float* bias;   // [N] (epilogues 0, 1)
-  void* out;           // bf16 [M,N] (epilogue 0) or float [M,N] (epilogues 1, 2)
+  void* out;           // bf16 [M,N] (epilogue 0), float [M,N] (epilogues 1, 2), or for kEpiArgmax the partial
+                       // results uint2 [argmax_slots(N)][M] = (bits of the slice maximum, its column)
   uint32_t* status;
 };
+
+// kEpiArgmax: one partial result per row and per 64-column slice of the (256-column padded) output.
+__host__ __device__ inline int64_t argmax_slots(int64_t N) { return (N + BN - 1) / BN * (BN / 64); }
 
 // GELU(v) = v * Phi(v) with the normal CDF written as a logistic function of an odd polynomial,
 //   Phi(v) ~= 1 / (1 + exp(-v (a + b v^2 + c v^4))),   a = 1.59501055, b = 7.40160400e-2, c = -7.03804784e-4
@@ -269,6 +273,35 @@ __device__ __forceinline__ void emit_box(const CUtensorMap* tmD, uint8_t* buf, i
 template <int EPI>
 __device__ __forceinline__ void epilogue_columns(const GemmArgs& g, const CUtensorMap* tmD, uint8_t* buf, int lane,
                                                  uint32_t taddr, int row0, int col0) {
+  if (EPI == kEpiArgmax) {
+    // Greedy selection fused into the LM head: the logits never leave the SM. Each lane scans its row's
+    // 64 columns in ascending order and keeps the first maximum (strictly-greater test), which is the
+    // rule of the stand-alone selection kernel; a slice that lies wholly beyond N yields (-inf, INT_MAX).
+    float bv = -INFINITY;
+    int bi = 0x7fffffff;
+    bool bad = false;
+#pragma unroll 1
+    for (int c = 0; c < kColsPerEpiWarp; c += 32) {
+      const int col = col0 + c;
+      if (col >= g.N) break;
+      uint32_t r[32];
+      tmem_ld32(taddr + c, r);
+      tmem_ld_wait();
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        const float v = __uint_as_float(r[j]);
+        if (col + j < g.N) {
+          bad |= !(v == v);
+          if (v > bv || (v == bv && col + j < bi)) { bv = v; bi = col + j; }
+        }
+      }
+    }
+    if (bad) raise_status(g.status, kStatusNonFinite);
+    const int64_t slot = col0 / kColsPerEpiWarp;
+    const int64_t row = row0 + lane;
+    if (row < g.M) reinterpret_cast<uint2*>(g.out)[slot * g.M + row] = make_uint2(__float_as_uint(bv), (uint32_t)bi);
+    return;
+  }
   if (EPI == kEpiBiasGelu) {
     uint32_t v[32];
 #pragma unroll
@@ -418,7 +451,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int col0 = static_cast<int>(n0) + cgrp * kColsPerEpiWarp;
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) +
                              static_cast<uint32_t>(acc * BN + cgrp * kColsPerEpiWarp);
-      if (row0 < g.M && col0 < g.N) epilogue_columns<EPI>(g, &tmD, buf, lane, taddr, row0, col0);
+      if (row0 < g.M && (col0 < g.N || EPI == kEpiArgmax)) epilogue_columns<EPI>(g, &tmD, buf, lane, taddr, row0, col0);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(mapa(smem_u32(&tempty[acc]), 0));

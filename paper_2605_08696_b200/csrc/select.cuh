@@ -63,6 +63,34 @@ select_greedy_kernel(const float* __restrict__ logits, int64_t R, int V, SelectO
   }
 }
 
+// Second stage of the selection fused into the LM head: reduces the per-slice partial results
+// part[slot][row] = (bits of the slice maximum, its column) over the slots of each row with the same rule
+// (largest value, lowest column among equals). 32 rows x 8 slot lanes per block; every load instruction
+// of a warp covers 32 consecutive rows (256 contiguous bytes).
+constexpr int kArgmaxRows = 32, kArgmaxLanes = 8;
+__global__ void __launch_bounds__(kArgmaxRows * kArgmaxLanes)
+argmax_reduce_kernel(const uint2* __restrict__ part, int64_t R, int64_t slots, int V, SelectOut out) {
+  __shared__ float sv[kArgmaxLanes][kArgmaxRows];
+  __shared__ int si[kArgmaxLanes][kArgmaxRows];
+  const int rr = threadIdx.x & 31, sl = threadIdx.x >> 5;
+  const int64_t row = (int64_t)blockIdx.x * kArgmaxRows + rr;
+  float bv = -INFINITY;
+  int bi = 0x7fffffff;
+  if (row < R) {
+    for (int64_t s = sl; s < slots; s += kArgmaxLanes) {
+      const uint2 p = __ldg(part + s * R + row);
+      argmax_take(__uint_as_float(p.x), (int)p.y, bv, bi);
+    }
+  }
+  sv[sl][rr] = bv; si[sl][rr] = bi;
+  __syncthreads();
+  if (sl == 0 && row < R) {
+    for (int w = 1; w < kArgmaxLanes; ++w) argmax_take(sv[w][rr], si[w][rr], bv, bi);
+    if (bi < 0 || bi >= V) bi = 0;       // all-NaN row
+    write_token(out, row, bi);
+  }
+}
+
 // ---- Philox4x32-10 (Salmon et al., SC'11) ---------------------------------------------------
 __device__ __forceinline__ uint32_t philox4x32_10_word0(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
                                                         uint32_t k0, uint32_t k1) {

@@ -274,13 +274,20 @@ int launch_mixer_nv(const MixerParams& p, cudaStream_t st) {
   const int nv = (p.d + 127) / 128;
   const unsigned grid = (unsigned)((p.R + kMixerWarps - 1) / kMixerWarps);
   const dim3 blk(kMixerWarps * 32);
-  if (nv <= 1) mixer_step_kernel<1, WT, ST><<<grid, blk, 0, st>>>(p);
-  else if (nv <= 2) mixer_step_kernel<2, WT, ST><<<grid, blk, 0, st>>>(p);
-  else if (nv <= 4) mixer_step_kernel<4, WT, ST><<<grid, blk, 0, st>>>(p);
-  else if (nv <= 6) mixer_step_kernel<6, WT, ST><<<grid, blk, 0, st>>>(p);
-  else if (nv <= 8) mixer_step_kernel<8, WT, ST><<<grid, blk, 0, st>>>(p);
-  else if (nv <= 12) mixer_step_kernel<12, WT, ST><<<grid, blk, 0, st>>>(p);
-  else mixer_step_kernel<16, WT, ST><<<grid, blk, 0, st>>>(p);
+  // whole 128-channel vectors per lane, each inside one head: the lean path
+  const bool fast = p.d % 128 == 0 && (p.d / p.h) % 128 == 0 && (nv == 4 || nv == 8 || nv == 12 || nv == 16);
+  if (fast) {
+    if (nv == 4) mixer_step_kernel<4, true, WT, ST><<<grid, blk, 0, st>>>(p);
+    else if (nv == 8) mixer_step_kernel<8, true, WT, ST><<<grid, blk, 0, st>>>(p);
+    else if (nv == 12) mixer_step_kernel<12, true, WT, ST><<<grid, blk, 0, st>>>(p);
+    else mixer_step_kernel<16, true, WT, ST><<<grid, blk, 0, st>>>(p);
+  } else if (nv <= 1) mixer_step_kernel<1, false, WT, ST><<<grid, blk, 0, st>>>(p);
+  else if (nv <= 2) mixer_step_kernel<2, false, WT, ST><<<grid, blk, 0, st>>>(p);
+  else if (nv <= 4) mixer_step_kernel<4, false, WT, ST><<<grid, blk, 0, st>>>(p);
+  else if (nv <= 6) mixer_step_kernel<6, false, WT, ST><<<grid, blk, 0, st>>>(p);
+  else if (nv <= 8) mixer_step_kernel<8, false, WT, ST><<<grid, blk, 0, st>>>(p);
+  else if (nv <= 12) mixer_step_kernel<12, false, WT, ST><<<grid, blk, 0, st>>>(p);
+  else mixer_step_kernel<16, false, WT, ST><<<grid, blk, 0, st>>>(p);
   SRM_CUDA(cudaGetLastError());
   return SRM_OK;
 }
@@ -349,6 +356,7 @@ int ensure_tc_ready(srm_model& m) {
   SRM_CUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<kEpiBiasGelu>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes));
   SRM_CUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<kEpiBiasResidual>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes));
   SRM_CUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<kEpiPlain>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes));
+  SRM_CUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<kEpiArgmax>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes));
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2 * (m.num_sms / 2));
   cfg.blockDim = dim3(tc::kThreads);
@@ -373,12 +381,14 @@ int launch_gemm_tc(srm_model& m, int epi, int64_t M, int64_t N, int64_t K, const
   CUtensorMap ta, tb, td;
   if ((rc = m.tmap(A, M, K, tc::kRowsPerCta, 2, &ta)) != SRM_OK) return rc;
   if ((rc = m.tmap(W, N, K, tc::kRowsPerCta, 2, &tb)) != SRM_OK) return rc;
-  if ((rc = m.tmap(out, M, N, tc::kOutBoxRows, epi == kEpiBiasGelu ? 2 : 4, &td)) != SRM_OK) return rc;
+  if (epi == kEpiArgmax) td = ta;       // no output matrix: the descriptor is not used
+  else if ((rc = m.tmap(out, M, N, tc::kOutBoxRows, epi == kEpiBiasGelu ? 2 : 4, &td)) != SRM_OK) return rc;
   tc::GemmArgs g{M, N, K, bias, out, status};
   const int64_t tiles = ((M + tc::BM - 1) / tc::BM) * ((N + tc::BN - 1) / tc::BN);
   const unsigned grid = 2u * (unsigned)(tiles < m.tc_clusters ? tiles : m.tc_clusters);
   if (epi == kEpiBiasGelu) tc::gemm_tc_kernel<kEpiBiasGelu><<<grid, tc::kThreads, tc::kSmemBytes, st>>>(ta, tb, td, g);
   else if (epi == kEpiBiasResidual) tc::gemm_tc_kernel<kEpiBiasResidual><<<grid, tc::kThreads, tc::kSmemBytes, st>>>(ta, tb, td, g);
+  else if (epi == kEpiArgmax) tc::gemm_tc_kernel<kEpiArgmax><<<grid, tc::kThreads, tc::kSmemBytes, st>>>(ta, tb, td, g);
   else tc::gemm_tc_kernel<kEpiPlain><<<grid, tc::kThreads, tc::kSmemBytes, st>>>(ta, tb, td, g);
   SRM_CUDA(cudaGetLastError());
   return SRM_OK;
@@ -388,6 +398,7 @@ int launch_gemm(srm_model& m, int epi, int64_t M, int64_t N, int64_t K, const vo
                 const float* bias, void* out, uint32_t* status, cudaStream_t st) {
   if (M <= 0) return SRM_OK;
   LaunchScope scope(m, epi == kEpiBiasGelu ? SRM_KERNEL_GEMM_UP : epi == kEpiBiasResidual ? SRM_KERNEL_GEMM_DOWN : SRM_KERNEL_GEMM_LM, st);
+  if (epi == kEpiArgmax) return launch_gemm_tc(m, epi, M, N, K, A, W, bias, out, status, st);
   if (m.cfg.dtype == SRM_DTYPE_FP32) return launch_gemm_simt<float>(epi, M, N, K, A, W, bias, out, st);
   if (m.cfg.flags & SRM_FLAG_SIMT_GEMM) return launch_gemm_simt<bf16>(epi, M, N, K, A, W, bias, out, st);
   return launch_gemm_tc(m, epi, M, N, K, A, W, bias, out, status, st);
@@ -424,6 +435,30 @@ int launch_select(const srm_model& m, int64_t R, const float* logits, const srm_
                                                                      sample_base, step, out, status);
     }
   }
+  SRM_CUDA(cudaGetLastError());
+  return SRM_OK;
+}
+
+// True when token selection can be fused into the LM-head GEMM: greedy rule, tensor-core path, and the
+// caller does not ask for the logits.
+bool can_fuse_greedy(const srm_model& m, const srm_sampling& s, const float* logits_out) {
+  return s.mode == SRM_SELECT_GREEDY && logits_out == nullptr && m.cfg.dtype == SRM_DTYPE_BF16 &&
+         !(m.cfg.flags & SRM_FLAG_SIMT_GEMM);
+}
+
+// LM head with the argmax fused into its epilogue: `part` receives uint2 [argmax_slots(V)][R] partial
+// results (it needs argmax_slots(V) * R * 8 bytes, never more than the R x V fp32 logits would), a small
+// second kernel reduces them per row and writes the tokens.
+int launch_lm_head_greedy(srm_model& m, int64_t R, const void* a, void* part, const SelectOut& out, uint32_t* status,
+                          cudaStream_t st) {
+  if (R <= 0) return SRM_OK;
+  const int V = m.cfg.vocab;
+  int rc = launch_gemm(m, kEpiArgmax, R, V, m.cfg.d_model, a, m.ptr(-1, SRM_T_W_LM), nullptr, part, status, st);
+  if (rc != SRM_OK) return rc;
+  LaunchScope scope(m, SRM_KERNEL_SELECT, st);
+  const unsigned grid = (unsigned)((R + kArgmaxRows - 1) / kArgmaxRows);
+  argmax_reduce_kernel<<<grid, kArgmaxRows * kArgmaxLanes, 0, st>>>(reinterpret_cast<const uint2*>(part), R,
+                                                                   tc::argmax_slots(V), V, out);
   SRM_CUDA(cudaGetLastError());
   return SRM_OK;
 }
@@ -468,12 +503,13 @@ int decode_chunk(srm_model& m, srm_state& s, int64_t b0, int64_t R, const int32_
     if ((rc = launch_gemm(m, kEpiBiasResidual, R, d, F, w.H, m.ptr(l, SRM_T_W2), m.fptr(l, SRM_T_B2), w.x, s.status, st))) return rc;
   }
   if ((rc = launch_final_norm(m, w.x, R, 1, 0, w.a, st))) return rc;
-  float* lg = logits_out != nullptr ? logits_out + b0 * c.vocab : w.logits;
-  if ((rc = launch_gemm(m, kEpiPlain, R, c.vocab, d, w.a, m.ptr(-1, SRM_T_W_LM), nullptr, lg, s.status, st))) return rc;
   SelectOut o = out_all;
   o.last_tok += b0;
   if (o.tok_out) o.tok_out += b0;
   if (o.store) o.store += b0 * o.store_stride;
+  if (can_fuse_greedy(m, samp, logits_out)) return launch_lm_head_greedy(m, R, w.a, w.logits, o, s.status, st);
+  float* lg = logits_out != nullptr ? logits_out + b0 * c.vocab : w.logits;
+  if ((rc = launch_gemm(m, kEpiPlain, R, c.vocab, d, w.a, m.ptr(-1, SRM_T_W_LM), nullptr, lg, s.status, st))) return rc;
   return launch_select(m, R, lg, samp, samp.sample_idx_base + (uint64_t)b0, step, o, s.status, st);
 }
 
@@ -687,9 +723,13 @@ int srm_prefill(srm_model* m, srm_state* s, const int32_t* d_tokens, int32_t n, 
     }
     // LM head and selection on the last prompt position only
     if ((rc = launch_final_norm(*m, w.x, nb, n, n - 1, w.a_last, st))) return rc;
+    SelectOut o{s->last_tok + b0, d_first_tok ? d_first_tok + b0 : nullptr, nullptr, 0, 0};
+    if (can_fuse_greedy(*m, *samp, d_logits_last)) {
+      if ((rc = launch_lm_head_greedy(*m, nb, w.a_last, w.logits, o, s->status, st))) return rc;
+      continue;
+    }
     float* lg = d_logits_last != nullptr ? d_logits_last + b0 * c.vocab : w.logits;
     if ((rc = launch_gemm(*m, kEpiPlain, nb, c.vocab, d, w.a_last, m->ptr(-1, SRM_T_W_LM), nullptr, lg, s->status, st))) return rc;
-    SelectOut o{s->last_tok + b0, d_first_tok ? d_first_tok + b0 : nullptr, nullptr, 0, 0};
     if ((rc = launch_select(*m, nb, lg, *samp, samp->sample_idx_base + (uint64_t)b0, 0, o, s->status, st))) return rc;
   }
   s->pos = n;
@@ -800,6 +840,18 @@ int srm_k_gemm(srm_model* m, int32_t epilogue, int64_t M, int64_t N, int64_t K, 
   if (K % 64 || N % 8) return SRM_ERR_UNSUPPORTED;
   if (!aligned(d_A, 16) || !aligned(d_W, 16) || !aligned(d_out, 16) || !aligned(d_bias, 16)) return SRM_ERR_ALIGNMENT;
   return launch_gemm(*m, epilogue, M, N, K, d_A, d_W, d_bias, d_out, d_status, static_cast<cudaStream_t>(stream));
+}
+
+int srm_k_lm_head_greedy(srm_model* m, int64_t R, const void* d_a, void* d_part, size_t part_bytes, int32_t* d_tok,
+                         uint32_t* d_status, void* stream) {
+  if (m == nullptr || R < 0) return SRM_ERR_INVALID_ARG;
+  if (R == 0) return SRM_OK;
+  if (d_a == nullptr || d_part == nullptr || d_tok == nullptr) return SRM_ERR_INVALID_ARG;
+  if (m->cfg.dtype != SRM_DTYPE_BF16) return SRM_ERR_UNSUPPORTED;
+  if (!aligned(d_a, 16) || !aligned(d_part, 16)) return SRM_ERR_ALIGNMENT;
+  if (part_bytes < (size_t)tc::argmax_slots(m->cfg.vocab) * (size_t)R * 8) return SRM_ERR_BUFFER_TOO_SMALL;
+  SelectOut o{d_tok, nullptr, nullptr, 0, 0};
+  return launch_lm_head_greedy(*m, R, d_a, d_part, o, d_status, static_cast<cudaStream_t>(stream));
 }
 
 int srm_k_select(srm_model* m, int64_t R, const float* d_logits, const srm_sampling* samp, int32_t step,

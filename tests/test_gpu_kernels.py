@@ -159,6 +159,49 @@ def test_greedy_selection_bit_exact():
         assert np.array_equal(tok.cpu().numpy(), O.select_greedy(lg))
 
 
+@pytest.mark.parametrize("R,V,d", [(1, 256, 64), (300, 1000, 192), (513, 8000, 512), (96, 32000, 1024)])
+def test_lm_head_with_fused_greedy_selection(R, V, d):
+    """The LM head that selects inside its epilogue picks (i) exactly the token that the plain LM head
+    followed by the selection kernel picks on the device (same fp32 accumulators, same tie rule: W_lm rows
+    are duplicated so that exact ties occur, also across 64-column slices and 256-column tiles), and
+    (ii) the oracle's argmax of the fp64 logits wherever its top-2 margin exceeds the bf16 GEMM error."""
+    from oracle import srm_oracle as O
+    import paper_2605_08696_b200 as P
+    from helpers import top2_margin
+    shape = custom_shape(n_layers=1, d_model=d, vocab=V, dtype="bf16", seed=V)
+    W = I.make_weights(shape)
+    rng = np.random.default_rng(R + V)
+    W["W_lm"] = I.round_to_bf16(rng.normal(size=(V, d)).astype(np.float32) * 0.05)
+    W["W_lm"][V - 1] = W["W_lm"][3]                  # tie between the first and the last tile
+    W["W_lm"][70] = W["W_lm"][3]                     # ... and the next slice of the same tile
+    W["W_lm"][11] = W["W_lm"][10]                    # tie inside one slice
+    m, _ = _model(shape, W)
+    a_np = rng.normal(size=(R, d)).astype(np.float32)
+    a_np[0] = 8.0 * W["W_lm"][3] / np.linalg.norm(W["W_lm"][3])      # row 0: ids 3, 70, V-1 tie for the maximum
+    if R > 2:
+        a_np[2] = 8.0 * W["W_lm"][10] / np.linalg.norm(W["W_lm"][10])  # row 2: ids 10, 11 tie
+    a = _t(a_np, torch.bfloat16)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    slots = (V + 255) // 256 * 4
+    part = torch.empty(slots * R * 2, dtype=torch.int32, device=DEV)
+    tok_fused = torch.full((R,), -1, dtype=torch.int32, device=DEV)
+    m.k_lm_head_greedy(a, part, tok_fused, status=status)
+    logits = torch.full((R, V), float("nan"), dtype=torch.float32, device=DEV)
+    m.k_gemm(P.EPI_PLAIN, a, m.tensor(-1, 14), None, logits, status=status)
+    tok_plain = torch.full((R,), -1, dtype=torch.int32, device=DEV)
+    m.k_select(logits, P.Sampling("greedy"), 0, tok_plain, status=status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    got = tok_fused.cpu().numpy()
+    assert np.array_equal(got, tok_plain.cpu().numpy())
+    assert got[0] == 3 and (R <= 2 or got[2] == 10)
+    lg64 = a.float().cpu().numpy().astype(np.float64) @ W["W_lm"].astype(np.float64).T
+    want = O.select_greedy(lg64)
+    strict = top2_margin(lg64) > 1e-2
+    assert strict.sum() > 0.5 * R or R < 8
+    assert np.array_equal(got[strict], want[strict])
+
+
 @pytest.mark.parametrize("V,k", [(256, 50), (8000, 50), (32000, 50), (32000, 1), (1024, 256), (48000, 17)])
 def test_topk_sampling_matches_oracle(V, k):
     from oracle import srm_oracle as O

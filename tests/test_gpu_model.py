@@ -166,6 +166,27 @@ def test_small_config_batch_invariance_and_chunking():
     assert np.array_equal(outs[0][:16], outs[2])
 
 
+def test_fused_greedy_head_equals_logits_then_selection_on_device():
+    """srm_generate / srm_prefill select inside the LM-head epilogue when no logits are requested; asking
+    for the logits takes the LM head + selection-kernel route. Free-running, both must emit the same ids."""
+    import paper_2605_08696_b200 as P
+    shape, W, model = _build("small")
+    B, n, gen = 70, 128, 10
+    prompts = torch.from_numpy(I.make_prompts("small")[:B]).to(DEV)
+    g = P.Sampling("greedy")
+    ws = model.new_workspace(B, n, prefill_samples=B)
+    st_a, st_b = model.new_state(B), model.new_state(B)
+    first_a = model.prefill(st_a, prompts, g, ws)                        # fused
+    rest_a = model.generate(st_a, gen, 1, g, ws)                         # fused
+    first_b, _ = model.prefill(st_b, prompts, g, ws, want_logits=True)   # logits + selection kernel
+    toks_b, tok = [first_b], first_b
+    for k in range(gen):
+        tok, _ = model.decode_step(st_b, tok, g, k + 1, ws, want_logits=True)
+        toks_b.append(tok.clone())
+    assert torch.equal(torch.cat([first_a[:, None], rest_a], 1), torch.stack(toks_b, 1))
+    assert st_a.status() == 0 and st_b.status() == 0
+
+
 def test_resume_from_exported_cache():
     """generate(2k) == generate(k), copy the state buffer, generate(k) on the copy."""
     import paper_2605_08696_b200 as P
