@@ -17,6 +17,14 @@ __device__ __forceinline__ void raise_status(uint32_t* status, uint32_t bit) {
   if (status != nullptr) atomicOr(status, bit);
 }
 
+// Programmatic dependent launch. Every kernel of this library is launched with the programmatic
+// stream-serialization attribute: it may start while its predecessor in the stream is still draining,
+// runs whatever does not touch global memory, and calls pdl_wait() before its first global access
+// (the wait returns once the predecessor grid has completed and its writes are visible). pdl_trigger()
+// lets the successor start launching; it only affects when that grid is scheduled, never its ordering.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);

@@ -20,6 +20,8 @@ template <typename T, int EPI>
 __global__ void __launch_bounds__(256)
 gemm_simt_kernel(const T* __restrict__ A, const T* __restrict__ W, const float* __restrict__ bias,
                  void* __restrict__ out, int64_t M, int64_t N, int64_t K) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ float sA[kSimtBK][kSimtBM + 4];
   __shared__ float sW[kSimtBK][kSimtBN + 4];
   const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;

@@ -77,6 +77,8 @@ __device__ __forceinline__ void row_stats_full(const float4 (&v)[NV], float inv_
 template <int NV, bool FAST, typename WT, typename ST>
 __global__ void __launch_bounds__(kMixerWarps * 32, (FAST && NV <= 8) ? kMixerFastMinBlocks : 1)
 mixer_step_kernel(const MixerParams p) {
+  pdl_trigger();
+  pdl_wait();
   const int lane = threadIdx.x & 31;
   const int64_t row = (int64_t)blockIdx.x * kMixerWarps + (threadIdx.x >> 5);
   if (row >= p.R) return;
@@ -233,6 +235,8 @@ __global__ void __launch_bounds__(kMixerWarps * 32)
 norm_rows_kernel(const float* __restrict__ x, int64_t R, int64_t src_stride, int64_t src_offset,
                  const float* __restrict__ g, const float* __restrict__ b, float eps, int d,
                  WT* __restrict__ out) {
+  pdl_trigger();
+  pdl_wait();
   const int lane = threadIdx.x & 31;
   const int64_t row = (int64_t)blockIdx.x * kMixerWarps + (threadIdx.x >> 5);
   if (row >= R) return;

@@ -37,6 +37,8 @@ struct PrefillParams {
 
 template <typename WT, typename ST>
 __global__ void __launch_bounds__(kPrefillThreads) prefill_mixer_kernel(const PrefillParams p) {
+  pdl_trigger();
+  pdl_wait();
   constexpr int T = kPrefillTile;
   extern __shared__ float xs[];                       // [T][d] tile of the residual stream
   __shared__ float Mt[kPrefillMaxHeads][T][T];        // diagonal block of M per head

@@ -32,6 +32,8 @@ __device__ __forceinline__ void argmax_take(float v, int i, float& bv, int& bi) 
 
 __global__ void __launch_bounds__(kSelThreads)
 select_greedy_kernel(const float* __restrict__ logits, int64_t R, int V, SelectOut out, uint32_t* status) {
+  pdl_trigger();
+  pdl_wait();
   const int64_t row = blockIdx.x;
   if (row >= R) return;
   const float* lr = logits + row * (int64_t)V;
@@ -70,6 +72,8 @@ select_greedy_kernel(const float* __restrict__ logits, int64_t R, int V, SelectO
 constexpr int kArgmaxRows = 32, kArgmaxLanes = 8;
 __global__ void __launch_bounds__(kArgmaxRows * kArgmaxLanes)
 argmax_reduce_kernel(const uint2* __restrict__ part, int64_t R, int64_t slots, int V, SelectOut out) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ float sv[kArgmaxLanes][kArgmaxRows];
   __shared__ int si[kArgmaxLanes][kArgmaxRows];
   const int rr = threadIdx.x & 31, sl = threadIdx.x >> 5;
@@ -123,6 +127,8 @@ template <bool ROW_IN_SMEM>
 __global__ void __launch_bounds__(kSelThreads)
 select_topk_kernel(const float* __restrict__ logits, int64_t R, int V, int k, float inv_temp, uint64_t seed,
                    uint64_t sample_base, int step, SelectOut out, uint32_t* status) {
+  pdl_trigger();
+  pdl_wait();
   extern __shared__ float srow[];
   __shared__ uint32_t hist[256];
   __shared__ unsigned long long cand[kTopKMax];

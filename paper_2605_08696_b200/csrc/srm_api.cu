@@ -10,6 +10,7 @@
 #include <cstring>
 #include <mutex>
 #include <new>
+#include <utility>
 #include <vector>
 
 #include "common.cuh"
@@ -269,6 +270,23 @@ PrefillWs carve_prefill(const srm_model& m, void* ws, int64_t samples, int n) {
 }
 
 // ---- kernel launchers -------------------------------------------------------------------------
+// Every kernel goes through here: programmatic stream serialization lets the next kernel's blocks be
+// scheduled and run their set-up while this one drains; each kernel orders itself with pdl_wait().
+template <typename... KArgs, typename... Args>
+cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+
 template <typename WT, typename ST>
 int launch_mixer_nv(const MixerParams& p, cudaStream_t st) {
   const int nv = (p.d + 127) / 128;
@@ -277,17 +295,17 @@ int launch_mixer_nv(const MixerParams& p, cudaStream_t st) {
   // whole 128-channel vectors per lane, each inside one head: the lean path
   const bool fast = p.d % 128 == 0 && (p.d / p.h) % 128 == 0 && (nv == 4 || nv == 8 || nv == 12 || nv == 16);
   if (fast) {
-    if (nv == 4) mixer_step_kernel<4, true, WT, ST><<<grid, blk, 0, st>>>(p);
-    else if (nv == 8) mixer_step_kernel<8, true, WT, ST><<<grid, blk, 0, st>>>(p);
-    else if (nv == 12) mixer_step_kernel<12, true, WT, ST><<<grid, blk, 0, st>>>(p);
-    else mixer_step_kernel<16, true, WT, ST><<<grid, blk, 0, st>>>(p);
-  } else if (nv <= 1) mixer_step_kernel<1, false, WT, ST><<<grid, blk, 0, st>>>(p);
-  else if (nv <= 2) mixer_step_kernel<2, false, WT, ST><<<grid, blk, 0, st>>>(p);
-  else if (nv <= 4) mixer_step_kernel<4, false, WT, ST><<<grid, blk, 0, st>>>(p);
-  else if (nv <= 6) mixer_step_kernel<6, false, WT, ST><<<grid, blk, 0, st>>>(p);
-  else if (nv <= 8) mixer_step_kernel<8, false, WT, ST><<<grid, blk, 0, st>>>(p);
-  else if (nv <= 12) mixer_step_kernel<12, false, WT, ST><<<grid, blk, 0, st>>>(p);
-  else mixer_step_kernel<16, false, WT, ST><<<grid, blk, 0, st>>>(p);
+    if (nv == 4) SRM_CUDA(launch_kernel(mixer_step_kernel<4, true, WT, ST>, dim3(grid), dim3(blk), 0, st, p));
+    else if (nv == 8) SRM_CUDA(launch_kernel(mixer_step_kernel<8, true, WT, ST>, dim3(grid), dim3(blk), 0, st, p));
+    else if (nv == 12) SRM_CUDA(launch_kernel(mixer_step_kernel<12, true, WT, ST>, dim3(grid), dim3(blk), 0, st, p));
+    else SRM_CUDA(launch_kernel(mixer_step_kernel<16, true, WT, ST>, dim3(grid), dim3(blk), 0, st, p));
+  } else if (nv <= 1) SRM_CUDA(launch_kernel(mixer_step_kernel<1, false, WT, ST>, dim3(grid), dim3(blk), 0, st, p));
+  else if (nv <= 2) SRM_CUDA(launch_kernel(mixer_step_kernel<2, false, WT, ST>, dim3(grid), dim3(blk), 0, st, p));
+  else if (nv <= 4) SRM_CUDA(launch_kernel(mixer_step_kernel<4, false, WT, ST>, dim3(grid), dim3(blk), 0, st, p));
+  else if (nv <= 6) SRM_CUDA(launch_kernel(mixer_step_kernel<6, false, WT, ST>, dim3(grid), dim3(blk), 0, st, p));
+  else if (nv <= 8) SRM_CUDA(launch_kernel(mixer_step_kernel<8, false, WT, ST>, dim3(grid), dim3(blk), 0, st, p));
+  else if (nv <= 12) SRM_CUDA(launch_kernel(mixer_step_kernel<12, false, WT, ST>, dim3(grid), dim3(blk), 0, st, p));
+  else SRM_CUDA(launch_kernel(mixer_step_kernel<16, false, WT, ST>, dim3(grid), dim3(blk), 0, st, p));
   SRM_CUDA(cudaGetLastError());
   return SRM_OK;
 }
@@ -317,13 +335,13 @@ int launch_norm_t(const float* x, int64_t R, int64_t stride, int64_t offset, con
   const unsigned grid = (unsigned)((R + kMixerWarps - 1) / kMixerWarps);
   const dim3 blk(kMixerWarps * 32);
   WT* o = reinterpret_cast<WT*>(out);
-  if (nv <= 1) norm_rows_kernel<1, WT><<<grid, blk, 0, st>>>(x, R, stride, offset, g, b, eps, d, o);
-  else if (nv <= 2) norm_rows_kernel<2, WT><<<grid, blk, 0, st>>>(x, R, stride, offset, g, b, eps, d, o);
-  else if (nv <= 4) norm_rows_kernel<4, WT><<<grid, blk, 0, st>>>(x, R, stride, offset, g, b, eps, d, o);
-  else if (nv <= 6) norm_rows_kernel<6, WT><<<grid, blk, 0, st>>>(x, R, stride, offset, g, b, eps, d, o);
-  else if (nv <= 8) norm_rows_kernel<8, WT><<<grid, blk, 0, st>>>(x, R, stride, offset, g, b, eps, d, o);
-  else if (nv <= 12) norm_rows_kernel<12, WT><<<grid, blk, 0, st>>>(x, R, stride, offset, g, b, eps, d, o);
-  else norm_rows_kernel<16, WT><<<grid, blk, 0, st>>>(x, R, stride, offset, g, b, eps, d, o);
+  if (nv <= 1) SRM_CUDA(launch_kernel(norm_rows_kernel<1, WT>, dim3(grid), dim3(blk), 0, st, x, R, stride, offset, g, b, eps, d, o));
+  else if (nv <= 2) SRM_CUDA(launch_kernel(norm_rows_kernel<2, WT>, dim3(grid), dim3(blk), 0, st, x, R, stride, offset, g, b, eps, d, o));
+  else if (nv <= 4) SRM_CUDA(launch_kernel(norm_rows_kernel<4, WT>, dim3(grid), dim3(blk), 0, st, x, R, stride, offset, g, b, eps, d, o));
+  else if (nv <= 6) SRM_CUDA(launch_kernel(norm_rows_kernel<6, WT>, dim3(grid), dim3(blk), 0, st, x, R, stride, offset, g, b, eps, d, o));
+  else if (nv <= 8) SRM_CUDA(launch_kernel(norm_rows_kernel<8, WT>, dim3(grid), dim3(blk), 0, st, x, R, stride, offset, g, b, eps, d, o));
+  else if (nv <= 12) SRM_CUDA(launch_kernel(norm_rows_kernel<12, WT>, dim3(grid), dim3(blk), 0, st, x, R, stride, offset, g, b, eps, d, o));
+  else SRM_CUDA(launch_kernel(norm_rows_kernel<16, WT>, dim3(grid), dim3(blk), 0, st, x, R, stride, offset, g, b, eps, d, o));
   SRM_CUDA(cudaGetLastError());
   return SRM_OK;
 }
@@ -344,9 +362,9 @@ int launch_gemm_simt(int epi, int64_t M, int64_t N, int64_t K, const void* A, co
   const dim3 grid((unsigned)((N + kSimtBN - 1) / kSimtBN), (unsigned)((M + kSimtBM - 1) / kSimtBM));
   const T* a = reinterpret_cast<const T*>(A);
   const T* w = reinterpret_cast<const T*>(W);
-  if (epi == kEpiBiasGelu) gemm_simt_kernel<T, kEpiBiasGelu><<<grid, 256, 0, st>>>(a, w, bias, out, M, N, K);
-  else if (epi == kEpiBiasResidual) gemm_simt_kernel<T, kEpiBiasResidual><<<grid, 256, 0, st>>>(a, w, bias, out, M, N, K);
-  else gemm_simt_kernel<T, kEpiPlain><<<grid, 256, 0, st>>>(a, w, bias, out, M, N, K);
+  if (epi == kEpiBiasGelu) SRM_CUDA(launch_kernel(gemm_simt_kernel<T, kEpiBiasGelu>, dim3(grid), dim3(256), 0, st, a, w, bias, out, M, N, K));
+  else if (epi == kEpiBiasResidual) SRM_CUDA(launch_kernel(gemm_simt_kernel<T, kEpiBiasResidual>, dim3(grid), dim3(256), 0, st, a, w, bias, out, M, N, K));
+  else SRM_CUDA(launch_kernel(gemm_simt_kernel<T, kEpiPlain>, dim3(grid), dim3(256), 0, st, a, w, bias, out, M, N, K));
   SRM_CUDA(cudaGetLastError());
   return SRM_OK;
 }
@@ -386,10 +404,10 @@ int launch_gemm_tc(srm_model& m, int epi, int64_t M, int64_t N, int64_t K, const
   tc::GemmArgs g{M, N, K, bias, out, status};
   const int64_t tiles = ((M + tc::BM - 1) / tc::BM) * ((N + tc::BN - 1) / tc::BN);
   const unsigned grid = 2u * (unsigned)(tiles < m.tc_clusters ? tiles : m.tc_clusters);
-  if (epi == kEpiBiasGelu) tc::gemm_tc_kernel<kEpiBiasGelu><<<grid, tc::kThreads, tc::kSmemBytes, st>>>(ta, tb, td, g);
-  else if (epi == kEpiBiasResidual) tc::gemm_tc_kernel<kEpiBiasResidual><<<grid, tc::kThreads, tc::kSmemBytes, st>>>(ta, tb, td, g);
-  else if (epi == kEpiArgmax) tc::gemm_tc_kernel<kEpiArgmax><<<grid, tc::kThreads, tc::kSmemBytes, st>>>(ta, tb, td, g);
-  else tc::gemm_tc_kernel<kEpiPlain><<<grid, tc::kThreads, tc::kSmemBytes, st>>>(ta, tb, td, g);
+  if (epi == kEpiBiasGelu) SRM_CUDA(launch_kernel(tc::gemm_tc_kernel<kEpiBiasGelu>, dim3(grid), dim3(tc::kThreads), tc::kSmemBytes, st, ta, tb, td, g));
+  else if (epi == kEpiBiasResidual) SRM_CUDA(launch_kernel(tc::gemm_tc_kernel<kEpiBiasResidual>, dim3(grid), dim3(tc::kThreads), tc::kSmemBytes, st, ta, tb, td, g));
+  else if (epi == kEpiArgmax) SRM_CUDA(launch_kernel(tc::gemm_tc_kernel<kEpiArgmax>, dim3(grid), dim3(tc::kThreads), tc::kSmemBytes, st, ta, tb, td, g));
+  else SRM_CUDA(launch_kernel(tc::gemm_tc_kernel<kEpiPlain>, dim3(grid), dim3(tc::kThreads), tc::kSmemBytes, st, ta, tb, td, g));
   SRM_CUDA(cudaGetLastError());
   return SRM_OK;
 }
@@ -418,7 +436,7 @@ int launch_select(const srm_model& m, int64_t R, const float* logits, const srm_
   LaunchScope scope(m, SRM_KERNEL_SELECT, st);
   const int V = m.cfg.vocab;
   if (s.mode == SRM_SELECT_GREEDY) {
-    select_greedy_kernel<<<(unsigned)R, kSelThreads, 0, st>>>(logits, R, V, out, status);
+    SRM_CUDA(launch_kernel(select_greedy_kernel, dim3((unsigned)R), dim3(kSelThreads), 0, st, logits, R, V, out, status));
   } else {
     const size_t row_bytes = (size_t)V * 4;
     const float inv_t = 1.0f / s.temperature;
@@ -428,11 +446,11 @@ int launch_select(const srm_model& m, int64_t R, const float* logits, const srm_
         SRM_CUDA(cudaFuncSetAttribute(select_topk_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024));
         attr_set = true;
       }
-      select_topk_kernel<true><<<(unsigned)R, kSelThreads, row_bytes, st>>>(logits, R, V, s.top_k, inv_t, s.seed,
-                                                                            sample_base, step, out, status);
+      SRM_CUDA(launch_kernel(select_topk_kernel<true>, dim3((unsigned)R), dim3(kSelThreads), row_bytes, st, logits, R, V, s.top_k, inv_t, s.seed,
+                                                                            sample_base, step, out, status));
     } else {
-      select_topk_kernel<false><<<(unsigned)R, kSelThreads, 0, st>>>(logits, R, V, s.top_k, inv_t, s.seed,
-                                                                     sample_base, step, out, status);
+      SRM_CUDA(launch_kernel(select_topk_kernel<false>, dim3((unsigned)R), dim3(kSelThreads), 0, st, logits, R, V, s.top_k, inv_t, s.seed,
+                                                                     sample_base, step, out, status));
     }
   }
   SRM_CUDA(cudaGetLastError());
@@ -457,8 +475,8 @@ int launch_lm_head_greedy(srm_model& m, int64_t R, const void* a, void* part, co
   if (rc != SRM_OK) return rc;
   LaunchScope scope(m, SRM_KERNEL_SELECT, st);
   const unsigned grid = (unsigned)((R + kArgmaxRows - 1) / kArgmaxRows);
-  argmax_reduce_kernel<<<grid, kArgmaxRows * kArgmaxLanes, 0, st>>>(reinterpret_cast<const uint2*>(part), R,
-                                                                   tc::argmax_slots(V), V, out);
+  SRM_CUDA(launch_kernel(argmax_reduce_kernel, dim3(grid), dim3(kArgmaxRows * kArgmaxLanes), 0, st, reinterpret_cast<const uint2*>(part), R,
+                                                                   tc::argmax_slots(V), V, out));
   SRM_CUDA(cudaGetLastError());
   return SRM_OK;
 }
@@ -478,7 +496,7 @@ int launch_prefill_mixer(const srm_model& m, int layer, int64_t Bp, int n, const
   const bool wb = m.cfg.dtype == SRM_DTYPE_BF16, sb = m.cfg.state_dtype == SRM_DTYPE_BF16;
   auto go = [&](auto kernel) -> int {
     SRM_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    kernel<<<(unsigned)Bp, kPrefillThreads, smem, st>>>(p);
+    SRM_CUDA(launch_kernel(kernel, dim3((unsigned)Bp), dim3(kPrefillThreads), smem, st, p));
     SRM_CUDA(cudaGetLastError());
     return SRM_OK;
   };
