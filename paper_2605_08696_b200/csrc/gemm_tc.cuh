@@ -214,6 +214,7 @@ struct GemmArgs {
   void* out;           // bf16 [M,N] (epilogue 0), float [M,N] (epilogues 1, 2), or for kEpiArgmax the partial
                        // results uint2 [argmax_slots(N)][M] = (bits of the slice maximum, its column)
   uint32_t* status;
+  int w_static;        // W is constant data (model weights): its first tiles may be fetched before pdl_wait()
 };
 
 // kEpiArgmax: one partial result per row and per 64-column slice of the (256-column padded) output.
@@ -381,7 +382,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   // Barriers, tensor memory and the cluster handshake are set up; from here on global memory is touched.
-  pdl_wait();
+  // The producer thread orders itself (it may fetch weights, which no kernel writes, ahead of the wait).
+  if (threadIdx.x != 0) pdl_wait();
 
   const int64_t m_tiles = (g.M + BM - 1) / BM, n_tiles = (g.N + BN - 1) / BN;
   const int64_t tiles = m_tiles * n_tiles;
@@ -395,10 +397,31 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
+      // While the predecessor kernel drains: start the first tile's W loads (the ring is empty, so
+      // the first kStages stages need no wait), then order against the predecessor and add the A loads.
+      int pre = 0;
+      if (cluster_id < tiles) {
+        const int m0 = static_cast<int>(cluster_id % m_tiles) * BM + static_cast<int>(rank) * kRowsPerCta;
+        const int n0 = static_cast<int>(cluster_id / m_tiles) * BN + static_cast<int>(rank) * kRowsPerCta;
+        pre = k_blocks < kStages ? k_blocks : kStages;
+        if (!g.w_static) pdl_wait();
+        for (int kb = 0; kb < pre; ++kb) {
+          const uint32_t full_leader = mapa(smem_u32(&full[kb]), 0);
+          mbar_expect_tx_cluster(full_leader, kStageBytes);
+          tma_load_2d(sB + kb * kBStageBytes, &tmB, full_leader, kb * BK, n0);
+        }
+        if (g.w_static) pdl_wait();
+        for (int kb = 0; kb < pre; ++kb)
+          tma_load_2d(sA + kb * kAStageBytes, &tmA, mapa(smem_u32(&full[kb]), 0), kb * BK, m0);
+        stage = pre;
+        if (stage == kStages) { stage = 0; phase ^= 1u; }
+      } else {
+        pdl_wait();
+      }
       for (int64_t tile = cluster_id; ok && tile < tiles; tile += n_clusters) {
         const int m0 = static_cast<int>(tile % m_tiles) * BM + static_cast<int>(rank) * kRowsPerCta;
         const int n0 = static_cast<int>(tile / m_tiles) * BN + static_cast<int>(rank) * kRowsPerCta;
-        for (int kb = 0; kb < k_blocks; ++kb) {
+        for (int kb = (tile == cluster_id ? pre : 0); kb < k_blocks; ++kb) {
           if (!mbar_wait(&empty[stage], phase ^ 1u, g.status)) { ok = false; break; }
           const uint32_t full_leader = mapa(smem_u32(&full[stage]), 0);
           mbar_expect_tx_cluster(full_leader, kStageBytes);

@@ -401,7 +401,9 @@ int launch_gemm_tc(srm_model& m, int epi, int64_t M, int64_t N, int64_t K, const
   if ((rc = m.tmap(W, N, K, tc::kRowsPerCta, 2, &tb)) != SRM_OK) return rc;
   if (epi == kEpiArgmax) td = ta;       // no output matrix: the descriptor is not used
   else if ((rc = m.tmap(out, M, N, tc::kOutBoxRows, epi == kEpiBiasGelu ? 2 : 4, &td)) != SRM_OK) return rc;
-  tc::GemmArgs g{M, N, K, bias, out, status};
+  const uint8_t* wb = static_cast<const uint8_t*>(W);
+  const int w_static = wb >= m.w && wb < m.w + m.layout.total;      // inside the weight blob
+  tc::GemmArgs g{M, N, K, bias, out, status, w_static};
   const int64_t tiles = ((M + tc::BM - 1) / tc::BM) * ((N + tc::BN - 1) / tc::BN);
   const unsigned grid = 2u * (unsigned)(tiles < m.tc_clusters ? tiles : m.tc_clusters);
   if (epi == kEpiBiasGelu) SRM_CUDA(launch_kernel(tc::gemm_tc_kernel<kEpiBiasGelu>, dim3(grid), dim3(tc::kThreads), tc::kSmemBytes, st, ta, tb, td, g));
