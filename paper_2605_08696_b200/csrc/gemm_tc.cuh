@@ -161,6 +161,16 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
       : "r"(taddr)
       : "memory");
 }
+// 16 consecutive fp32 columns of this thread's TMEM lane
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // ---- bulk tensor stores (shared -> global), tracked per issuing thread in bulk async-groups ----
@@ -222,28 +232,24 @@ __host__ __device__ inline int64_t argmax_slots(int64_t N) { return (N + BN - 1)
 
 // GELU(v) = v * Phi(v) with the normal CDF written as a logistic function of an odd polynomial,
 //   Phi(v) ~= 1 / (1 + exp(-v (a + b v^2 + c v^4))),   a = 1.59501055, b = 7.40160400e-2, c = -7.03804784e-4
-// (coefficients fitted to minimise the maximum error of v * Phi(v) over the real line; |error| <= 2.6e-5,
-// two orders below the bf16 resolution of the hidden activations it feeds). v^2 is clamped at 64 so the
-// polynomial stays positive; beyond |v| = 8 the logistic term is 0 or 1 to fp32 precision anyway.
-// Nine instructions per element, two of them on the special-function unit (ex2, rcp): the epilogue of a
-// K = d tile has about as many issue slots as the tile's MMAs take, so the erf route does not fit.
-__device__ __forceinline__ float rcp_approx(float x) {
+// (coefficients fitted to minimise the maximum error of v * Phi(v) over the real line: 2.6e-5), evaluated
+// through 1 / (1 + exp(-w)) = (1 + tanh(w / 2)) / 2 with the hardware tanh (absolute error below 2^-10.9),
+// so |error| <= 2.6e-5 + |v| / 2 * 5.2e-4: below a quarter of the bf16 spacing of the hidden activation it
+// produces. v^2 is clamped at 64 so the polynomial stays positive; beyond |v| = 8 tanh is +-1 anyway.
+// Eight instructions per element, one on the special-function unit: the epilogue shares the SM with the
+// next tile's MMAs, and with erf, or with ex2 + rcp, the special-function unit alone took half a tile time.
+__device__ __forceinline__ float tanh_approx(float x) {
   float r;
-  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
-  return r;
-}
-__device__ __forceinline__ float ex2_approx(float x) {
-  float r;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+  asm("tanh.approx.f32 %0, %1;" : "=f"(r) : "f"(x));
   return r;
 }
 __device__ __forceinline__ float gelu_fast(float v) {
-  constexpr float kLog2e = 1.4426950408889634f;
   const float s = fminf(v * v, 64.0f);
-  float q = fmaf(s, 7.03804784e-4f * kLog2e, -7.40160400e-2f * kLog2e);
-  q = fmaf(s, q, -1.59501055f * kLog2e);                 // -log2(e) * (a + b s + c s^2)
-  const float e = ex2_approx(q * v);                     // exp(-v (a + b s + c s^2))
-  return v * rcp_approx(e + 1.0f);
+  float q = fmaf(s, -0.5f * 7.03804784e-4f, 0.5f * 7.40160400e-2f);
+  q = fmaf(s, q, 0.5f * 1.59501055f);                    // (a + b s + c s^2) / 2
+  const float t = tanh_approx(q * v);
+  const float hv = 0.5f * v;
+  return fmaf(hv, t, hv);
 }
 
 // Hands this warp's 32 rows x 128 bytes (v = the 32 words of the lane's row) to the TMA unit.
@@ -269,82 +275,104 @@ __device__ __forceinline__ void emit_box(const CUtensorMap* tmD, uint8_t* buf, i
   }
 }
 
+// max(a, b, c) that returns NaN when any input is NaN
+__device__ __forceinline__ float max3_nan(float a, float b, float c) {
+  float r;
+  asm("max.NaN.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
+
+// Greedy selection over 16 consecutive logits r[0..15] of columns col .. col+15, folded into the running
+// (bv, bi) with the rule of the stand-alone selection kernel: largest value, lowest column among equals,
+// NaN never wins. The chunk maximum costs half an instruction per element; the column search runs only in
+// lanes whose chunk beats their running maximum.
+__device__ __forceinline__ void argmax_chunk16(const uint32_t (&r)[16], int col, int64_t N, float& bv, int& bi, bool& bad) {
+  float f[16];
+#pragma unroll
+  for (int j = 0; j < 16; ++j) f[j] = __uint_as_float(r[j]);
+  if (col + 16 <= N) {
+    const float m = max3_nan(max3_nan(max3_nan(f[0], f[1], f[2]), max3_nan(f[3], f[4], f[5]), max3_nan(f[6], f[7], f[8])),
+                             max3_nan(max3_nan(f[9], f[10], f[11]), max3_nan(f[12], f[13], f[14]), f[15]), -INFINITY);
+    if (m == m) {                       // no NaN in the chunk
+      if (m > bv) {
+        int idx = 15;
+#pragma unroll
+        for (int j = 14; j >= 0; --j) idx = (f[j] == m) ? j : idx;
+        bv = m;
+        bi = col + idx;
+      }
+      return;
+    }
+  }
+  // a NaN somewhere, or the ragged end of the row: the element-by-element rule
+#pragma unroll
+  for (int j = 0; j < 16; ++j) {
+    if (col + j < N) {
+      bad |= !(f[j] == f[j]);
+      if (f[j] > bv || (f[j] == bv && col + j < bi)) { bv = f[j]; bi = col + j; }
+    }
+  }
+}
+
 // The 64 accumulator columns [col0, col0 + 64) of this warp's 32 rows: TMEM -> registers -> bias /
-// activation -> one (bf16) or two (fp32) boxes of 128 bytes per row.
+// activation -> one (bf16) or two (fp32) boxes of 128 bytes per row, or the fused greedy selection.
+// The columns come in four chunks of 16; the load of chunk i+1 is in flight while chunk i is processed
+// (tcgen05.wait::ld waits for every load of the thread, so it is placed after the processing).
 template <int EPI>
 __device__ __forceinline__ void epilogue_columns(const GemmArgs& g, const CUtensorMap* tmD, uint8_t* buf, int lane,
                                                  uint32_t taddr, int row0, int col0) {
-  if (EPI == kEpiArgmax) {
-    // Greedy selection fused into the LM head: the logits never leave the SM. Each lane scans its row's
-    // 64 columns in ascending order and keeps the first maximum (strictly-greater test), which is the
-    // rule of the stand-alone selection kernel; a slice that lies wholly beyond N yields (-inf, INT_MAX).
-    float bv = -INFINITY;
-    int bi = 0x7fffffff;
-    bool bad = false;
-#pragma unroll 1
-    for (int c = 0; c < kColsPerEpiWarp; c += 32) {
-      const int col = col0 + c;
-      if (col >= g.N) break;
-      uint32_t r[32];
-      tmem_ld32(taddr + c, r);
-      tmem_ld_wait();
+  constexpr int kChunks = kColsPerEpiWarp / 16;
+  uint32_t ra[16], rb[16];
+  uint32_t v[32];                        // staged output words of the lane's row (not used by kEpiArgmax)
+  float bv = -INFINITY;                  // kEpiArgmax: running maximum and its column
+  int bi = 0x7fffffff;
+  bool bad = false;
+  tmem_ld16(taddr, ra);
+  tmem_ld_wait();
 #pragma unroll
-      for (int j = 0; j < 32; ++j) {
-        const float v = __uint_as_float(r[j]);
-        if (col + j < g.N) {
-          bad |= !(v == v);
-          if (v > bv || (v == bv && col + j < bi)) { bv = v; bi = col + j; }
+  for (int c = 0; c < kChunks; ++c) {
+    uint32_t (&cur)[16] = (c & 1) ? rb : ra;
+    uint32_t (&nxt)[16] = (c & 1) ? ra : rb;
+    if (c + 1 < kChunks) tmem_ld16(taddr + 16 * (c + 1), nxt);
+    const int col = col0 + 16 * c;
+    if (EPI == kEpiArgmax) {
+      if (col < g.N) argmax_chunk16(cur, col, g.N, bv, bi, bad);
+    } else if (EPI == kEpiBiasGelu) {
+#pragma unroll
+      for (int j = 0; j < 16; j += 4) {
+        float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (col + j < g.N) b = __ldg(reinterpret_cast<const float4*>(g.bias + col + j));
+        __nv_bfloat162 p;
+        p = __floats2bfloat162_rn(gelu_fast(__uint_as_float(cur[j + 0]) + b.x), gelu_fast(__uint_as_float(cur[j + 1]) + b.y));
+        v[8 * c + j / 2] = *reinterpret_cast<uint32_t*>(&p);
+        p = __floats2bfloat162_rn(gelu_fast(__uint_as_float(cur[j + 2]) + b.z), gelu_fast(__uint_as_float(cur[j + 3]) + b.w));
+        v[8 * c + j / 2 + 1] = *reinterpret_cast<uint32_t*>(&p);
+      }
+      if (c == kChunks - 1) emit_box<EPI>(tmD, buf, lane, col0, row0, v);
+    } else {
+#pragma unroll
+      for (int j = 0; j < 16; j += 4) {
+        if (EPI == kEpiBiasResidual && col + j < g.N) {
+          const float4 b = __ldg(reinterpret_cast<const float4*>(g.bias + col + j));
+          v[16 * (c & 1) + j + 0] = __float_as_uint(__uint_as_float(cur[j + 0]) + b.x);
+          v[16 * (c & 1) + j + 1] = __float_as_uint(__uint_as_float(cur[j + 1]) + b.y);
+          v[16 * (c & 1) + j + 2] = __float_as_uint(__uint_as_float(cur[j + 2]) + b.z);
+          v[16 * (c & 1) + j + 3] = __float_as_uint(__uint_as_float(cur[j + 3]) + b.w);
+        } else {
+          v[16 * (c & 1) + j + 0] = cur[j + 0]; v[16 * (c & 1) + j + 1] = cur[j + 1];
+          v[16 * (c & 1) + j + 2] = cur[j + 2]; v[16 * (c & 1) + j + 3] = cur[j + 3];
         }
       }
+      // two chunks make one box of 32 fp32 columns; a box that starts beyond N is not emitted
+      if ((c & 1) && col - 16 < g.N) emit_box<EPI>(tmD, buf, lane, col - 16, row0, v);
     }
+    if (c + 1 < kChunks) tmem_ld_wait();
+  }
+  if (EPI == kEpiArgmax) {
     if (bad) raise_status(g.status, kStatusNonFinite);
     const int64_t slot = col0 / kColsPerEpiWarp;
     const int64_t row = row0 + lane;
     if (row < g.M) reinterpret_cast<uint2*>(g.out)[slot * g.M + row] = make_uint2(__float_as_uint(bv), (uint32_t)bi);
-    return;
-  }
-  if (EPI == kEpiBiasGelu) {
-    uint32_t v[32];
-#pragma unroll
-    for (int half = 0; half < 2; ++half) {
-      uint32_t r[32];
-      tmem_ld32(taddr + 32 * half, r);
-      tmem_ld_wait();
-      const int col = col0 + 32 * half;
-#pragma unroll
-      for (int j = 0; j < 32; j += 4) {
-        float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (col + j < g.N) b = __ldg(reinterpret_cast<const float4*>(g.bias + col + j));
-        __nv_bfloat162 p;
-        p = __floats2bfloat162_rn(gelu_fast(__uint_as_float(r[j + 0]) + b.x), gelu_fast(__uint_as_float(r[j + 1]) + b.y));
-        v[16 * half + j / 2] = *reinterpret_cast<uint32_t*>(&p);
-        p = __floats2bfloat162_rn(gelu_fast(__uint_as_float(r[j + 2]) + b.z), gelu_fast(__uint_as_float(r[j + 3]) + b.w));
-        v[16 * half + j / 2 + 1] = *reinterpret_cast<uint32_t*>(&p);
-      }
-    }
-    emit_box<EPI>(tmD, buf, lane, col0, row0, v);
-  } else {
-#pragma unroll 1
-    for (int c = 0; c < kColsPerEpiWarp; c += 32) {
-      const int col = col0 + c;
-      if (col >= g.N) break;
-      uint32_t r[32];
-      tmem_ld32(taddr + c, r);
-      tmem_ld_wait();
-      if (EPI == kEpiBiasResidual) {
-#pragma unroll
-        for (int j = 0; j < 32; j += 4) {
-          if (col + j < g.N) {
-            const float4 b = __ldg(reinterpret_cast<const float4*>(g.bias + col + j));
-            r[j + 0] = __float_as_uint(__uint_as_float(r[j + 0]) + b.x);
-            r[j + 1] = __float_as_uint(__uint_as_float(r[j + 1]) + b.y);
-            r[j + 2] = __float_as_uint(__uint_as_float(r[j + 2]) + b.z);
-            r[j + 3] = __float_as_uint(__uint_as_float(r[j + 3]) + b.w);
-          }
-        }
-      }
-      emit_box<EPI>(tmD, buf, lane, col, row0, r);
-    }
   }
 }
 
