@@ -126,9 +126,11 @@ __device__ __forceinline__ float key_value(uint32_t k) {
 template <bool ROW_IN_SMEM>
 __global__ void __launch_bounds__(kSelThreads)
 select_topk_kernel(const float* __restrict__ logits, int64_t R, int V, int k, float inv_temp, uint64_t seed,
-                   uint64_t sample_base, int step, SelectOut out, uint32_t* status) {
+                   uint64_t sample_base, int step, SelectOut out, uint32_t* status, int only_marked) {
   pdl_trigger();
   pdl_wait();
+  // second stage of the streaming kernel below: only the rows it marked (-1) are processed here
+  if (only_marked && out.last_tok[blockIdx.x < R ? blockIdx.x : 0] != -1) return;
   extern __shared__ float srow[];
   __shared__ uint32_t hist[256];
   __shared__ unsigned long long cand[kTopKMax];
@@ -243,6 +245,130 @@ select_topk_kernel(const float* __restrict__ logits, int64_t R, int V, int k, fl
                                            (uint32_t)(seed >> 32));
     const float u = (float)(r >> 8) * (1.0f / 16777216.0f);
     const float target = u * c;
+    int pick = k - 1;
+    for (int i = 0; i < k; ++i) {
+      if (cdf[i] > target) { pick = i; break; }
+    }
+    write_token(out, row, (int)(uint32_t)(cand[pick] & 0xffffffffull));
+  }
+}
+
+// ---- top-k, streaming version ------------------------------------------------------------------
+// The radix selection above makes four histogram passes over a row held in shared memory; with logits
+// that share their leading bits almost all of its shared-memory atomics land in one or two bins. This
+// kernel instead (1) streams the row once for mean and standard deviation, (2) streams it again (an L2
+// hit) collecting every logit >= t = mean + z * sd, and accepts the candidate set when it holds at least
+// k and at most kTopkCap entries: any set {x >= t} with >= k members contains the k largest logits and all
+// ties at the k-th place, so sorting it by (logit desc, id asc) gives exactly the order the radix version
+// gives. z starts at the normal quantile for an expected 2.5 k candidates (z0, from the host) and is
+// bisected when the count misses the window. Rows that still miss it after kTopkRounds (constant rows,
+// infinities, more than kTopkCap ties) are marked with token -1 and redone by select_topk_kernel.
+// Little shared memory, so several rows are in flight per SM and the row never has to fit on chip.
+constexpr int kTopkCap = 1024;
+constexpr int kTopkRounds = 6;
+
+__global__ void __launch_bounds__(kSelThreads)
+select_topk_stream_kernel(const float* __restrict__ logits, int64_t R, int V, int k, float inv_temp, float z0,
+                          uint64_t seed, uint64_t sample_base, int step, SelectOut out, uint32_t* status) {
+  pdl_trigger();
+  pdl_wait();
+  __shared__ unsigned long long cand[kTopkCap];
+  __shared__ float red_s[kSelThreads / 32], red_q[kSelThreads / 32];
+  __shared__ float sh_mean, sh_sd;
+  __shared__ uint32_t sh_count;
+  __shared__ float cdf[kTopKMax];
+
+  const int64_t row = blockIdx.x;
+  if (row >= R) return;
+  const float* lr = logits + row * (int64_t)V;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+  // ---- pass 1: moments ----
+  float sum = 0.f, sq = 0.f;
+  bool bad = false;
+  for (int i = tid * 4; i < V; i += kSelThreads * 4) {
+    const float4 v = *reinterpret_cast<const float4*>(lr + i);
+    bad |= !(v.x == v.x) | !(v.y == v.y) | !(v.z == v.z) | !(v.w == v.w);
+    sum += (v.x + v.y) + (v.z + v.w);
+    sq = fmaf(v.x, v.x, sq); sq = fmaf(v.y, v.y, sq); sq = fmaf(v.z, v.z, sq); sq = fmaf(v.w, v.w, sq);
+  }
+  if (bad) raise_status(status, kStatusNonFinite);
+  sum = warp_sum(sum); sq = warp_sum(sq);
+  if (lane == 0) { red_s[warp] = sum; red_q[warp] = sq; }
+  __syncthreads();
+  if (tid == 0) {
+    float a = 0.f, b = 0.f;
+    for (int w = 0; w < kSelThreads / 32; ++w) { a += red_s[w]; b += red_q[w]; }
+    const float mean = a / (float)V;
+    sh_mean = mean;
+    sh_sd = sqrtf(fmaxf(b / (float)V - mean * mean, 0.f));
+    sh_count = 0;
+  }
+  __syncthreads();
+  const float mean = sh_mean, sd = sh_sd;
+
+  // ---- pass 2 (repeated while the count misses [k, kTopkCap]): collect everything >= t ----
+  float z = z0, lo = -INFINITY, hi = INFINITY;       // lo: a z that gave too many, hi: one that gave too few
+  uint32_t c = 0;
+  bool found = false;
+  for (int round = 0; round < kTopkRounds; ++round) {
+    const float t = fmaf(z, sd, mean);
+    for (int i = tid * 4; i < V; i += kSelThreads * 4) {
+      const float4 v = *reinterpret_cast<const float4*>(lr + i);
+      const float e[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        if (e[j] >= t) {
+          const uint32_t slot = atomicAdd(&sh_count, 1u);
+          if (slot < (uint32_t)kTopkCap) cand[slot] = ((unsigned long long)(~order_key(e[j])) << 32) | (uint32_t)(i + j);
+        }
+      }
+    }
+    __syncthreads();
+    c = sh_count;
+    __syncthreads();
+    if (c >= (uint32_t)k && c <= (uint32_t)kTopkCap) { found = true; break; }
+    if (tid == 0) sh_count = 0;
+    if (c < (uint32_t)k) hi = z; else lo = z;
+    z = (lo > -INFINITY && hi < INFINITY) ? 0.5f * (lo + hi) : (c < (uint32_t)k ? z - 1.0f : z + 0.75f);
+    __syncthreads();
+  }
+  if (!found) {                                      // block-uniform
+    if (tid == 0) out.last_tok[row] = -1;
+    return;
+  }
+
+  // ---- sort the c candidates ascending by (~key, id) = (logit desc, id asc) ----
+  int P = 2;
+  while (P < (int)c) P <<= 1;
+  for (int i = (int)c + tid; i < P; i += kSelThreads) cand[i] = ~0ull;
+  __syncthreads();
+  for (int size = 2; size <= P; size <<= 1) {
+    for (int stride = size >> 1; stride > 0; stride >>= 1) {
+      for (int i = tid; i < P; i += kSelThreads) {
+        const int j = i ^ stride;
+        if (j > i) {
+          const unsigned long long a = cand[i], b = cand[j];
+          const bool up = (i & size) == 0;
+          if ((a > b) == up) { cand[i] = b; cand[j] = a; }
+        }
+      }
+      __syncthreads();
+    }
+  }
+  if (tid == 0) {
+    const float l0 = key_value(~(uint32_t)(cand[0] >> 32));
+    float acc = 0.f;
+    for (int i = 0; i < k; ++i) {
+      const float li = key_value(~(uint32_t)(cand[i] >> 32));
+      acc += expf((li - l0) * inv_temp);
+      cdf[i] = acc;
+    }
+    const uint64_t sidx = sample_base + (uint64_t)row;
+    const uint32_t r = philox4x32_10_word0((uint32_t)sidx, (uint32_t)step, 0u, 0u, (uint32_t)seed,
+                                           (uint32_t)(seed >> 32));
+    const float u = (float)(r >> 8) * (1.0f / 16777216.0f);
+    const float target = u * acc;
     int pick = k - 1;
     for (int i = 0; i < k; ++i) {
       if (cdf[i] > target) { pick = i; break; }

@@ -6,6 +6,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <cmath>
 #include <cstdio>
 #include <cstring>
 #include <mutex>
@@ -440,20 +441,21 @@ int launch_select(const srm_model& m, int64_t R, const float* logits, const srm_
   if (s.mode == SRM_SELECT_GREEDY) {
     SRM_CUDA(launch_kernel(select_greedy_kernel, dim3((unsigned)R), dim3(kSelThreads), 0, st, logits, R, V, out, status));
   } else {
-    const size_t row_bytes = (size_t)V * 4;
     const float inv_t = 1.0f / s.temperature;
-    if (row_bytes <= 160 * 1024) {
-      static bool attr_set = false;
-      if (!attr_set) {
-        SRM_CUDA(cudaFuncSetAttribute(select_topk_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024));
-        attr_set = true;
-      }
-      SRM_CUDA(launch_kernel(select_topk_kernel<true>, dim3((unsigned)R), dim3(kSelThreads), row_bytes, st, logits, R, V, s.top_k, inv_t, s.seed,
-                                                                            sample_base, step, out, status));
-    } else {
-      SRM_CUDA(launch_kernel(select_topk_kernel<false>, dim3((unsigned)R), dim3(kSelThreads), 0, st, logits, R, V, s.top_k, inv_t, s.seed,
-                                                                     sample_base, step, out, status));
-    }
+    // threshold start: the normal quantile that leaves about 2.5 k of the V logits above it
+    // (rational approximation 26.2.23 of Abramowitz & Stegun; only a starting point, the kernel adapts)
+    double pr = 2.5 * s.top_k / (double)V;
+    if (pr > 0.45) pr = 0.45;
+    const double tt = std::sqrt(-2.0 * std::log(pr));
+    const float z0 = (float)(tt - (2.515517 + 0.802853 * tt + 0.010328 * tt * tt) /
+                                      (1.0 + 1.432788 * tt + 0.189269 * tt * tt + 0.001308 * tt * tt * tt));
+    SRM_CUDA(launch_kernel(select_topk_stream_kernel, dim3((unsigned)R), dim3(kSelThreads), 0, st, logits, R, V, s.top_k,
+                           inv_t, z0, s.seed, sample_base, step, out, status));
+    // rows the streaming kernel could not settle (marked -1): the radix selection, reading the row from
+    // global memory; every other block exits at once
+    SRM_CUDA(launch_kernel(select_topk_kernel<false>, dim3((unsigned)R), dim3(kSelThreads), 0, st, logits, R, V, s.top_k,
+                           inv_t, s.seed, sample_base, step, out, status, 1));
+    ++g_kernel_launches;
   }
   SRM_CUDA(cudaGetLastError());
   return SRM_OK;
