@@ -26,7 +26,6 @@ struct MixerParams {
 };
 
 constexpr int kMixerWarps = 4;
-constexpr int kMixerFastMinBlocks = 4;   // register cap of the lean path: 128 per thread, 16 warps per SM
 
 // LayerNorm statistics of a register-resident row: two passes (mean, then centred variance).
 template <int NV>
@@ -71,12 +70,10 @@ __device__ __forceinline__ void row_stats_full(const float4 (&v)[NV], float inv_
 }
 
 // NV = ceil(d / 128): float4 vectors per lane. WT: weight/activation type, ST: cache type.
-// FAST: d == NV * 128 and the head width is a multiple of 128, so every vector a warp touches lies inside
-// one head and inside the row: no bounds tests, no per-lane head arithmetic (the head index advances with
-// a warp-uniform counter). The general path covers every other supported shape.
-template <int NV, bool FAST, typename WT, typename ST>
-__global__ void __launch_bounds__(kMixerWarps * 32, (FAST && NV <= 8) ? kMixerFastMinBlocks : 1)
-mixer_step_kernel(const MixerParams p) {
+// General-shape version (any d that is a multiple of 4, any head width); shapes made of whole
+// 128-channel vectors per head take mixer_stream_kernel instead.
+template <int NV, typename WT, typename ST>
+__global__ void __launch_bounds__(kMixerWarps * 32) mixer_step_kernel(const MixerParams p) {
   pdl_trigger();
   pdl_wait();
   const int lane = threadIdx.x & 31;
@@ -85,80 +82,6 @@ mixer_step_kernel(const MixerParams p) {
   const int d = p.d;
   const int dh = d / p.h;
   const int h_row = p.h >> 1;
-
-  if (FAST) {
-    const int c0 = lane * 4;
-    float4 v[NV], s[NV];
-    ST* Sr = reinterpret_cast<ST*>(p.S) + row * d + c0;
-    float* xr = p.x + row * d + c0;
-    if (p.tok != nullptr) {
-      int tk = p.tok[row];
-      if (tk < 0 || tk >= p.vocab) {
-        if (lane == 0) raise_status(p.status, kStatusTokenRange);
-        tk = tk < 0 ? 0 : p.vocab - 1;
-      }
-      const WT* e = reinterpret_cast<const WT*>(p.E) + (int64_t)tk * d + c0;
-#pragma unroll
-      for (int i = 0; i < NV; ++i) v[i] = ldg4(e + i * 128);
-    } else {
-#pragma unroll
-      for (int i = 0; i < NV; ++i) v[i] = ld4(xr + i * 128);
-    }
-#pragma unroll
-    for (int i = 0; i < NV; ++i) s[i] = ld4(Sr + i * 128);
-
-    const float inv_d = 1.0f / (float)d;
-    float mean, rstd;
-    row_stats_full<NV>(v, inv_d, p.eps, mean, rstd);
-    const float nmr = -mean * rstd;                      // (x - mean) * rstd = x * rstd + nmr
-
-    const float* beta_t = p.beta + (int64_t)p.t * d + c0;
-    const float* g1 = p.ln1_g + c0;
-    const float* b1 = p.ln1_b + c0;
-    const int vph = dh >> 7;                             // vectors per head
-    int g = 0, left = vph;
-    float al = __ldg(p.alpha + p.t), lm = __ldg(p.lam);
-#pragma unroll
-    for (int i = 0; i < NV; ++i) {
-      const float4 gg = ldg4(g1 + i * 128), bb = ldg4(b1 + i * 128), bt = ldg4(beta_t + i * 128);
-      float4 z;
-      z.x = fmaf(fmaf(v[i].x, rstd, nmr), gg.x, bb.x); z.y = fmaf(fmaf(v[i].y, rstd, nmr), gg.y, bb.y);
-      z.z = fmaf(fmaf(v[i].z, rstd, nmr), gg.z, bb.z); z.w = fmaf(fmaf(v[i].w, rstd, nmr), gg.w, bb.w);
-      float4 y, sn;
-      if (g < h_row) {            // row-repeat head, Eq. 2: y = a z + b + S ; S' = l (S + a z)
-        const float4 u = make_float4(al * z.x, al * z.y, al * z.z, al * z.w);
-        y = make_float4(u.x + bt.x + s[i].x, u.y + bt.y + s[i].y, u.z + bt.z + s[i].z, u.w + bt.w + s[i].w);
-        sn = make_float4(lm * (s[i].x + u.x), lm * (s[i].y + u.y), lm * (s[i].z + u.z), lm * (s[i].w + u.w));
-      } else {                    // column-repeat head, Eq. 3: y = a (z + S) + b ; S' = l (z + S)
-        const float4 w = make_float4(z.x + s[i].x, z.y + s[i].y, z.z + s[i].z, z.w + s[i].w);
-        y = make_float4(al * w.x + bt.x, al * w.y + bt.y, al * w.z + bt.z, al * w.w + bt.w);
-        sn = make_float4(lm * w.x, lm * w.y, lm * w.z, lm * w.w);
-      }
-      st4(Sr + i * 128, sn);
-      v[i] = make_float4(v[i].x + y.x, v[i].y + y.y, v[i].z + y.z, v[i].w + y.w);
-      st4(xr + i * 128, v[i]);
-      if (--left == 0 && i + 1 < NV) {                   // next vector starts the next head
-        ++g; left = vph;
-        al = __ldg(p.alpha + (int64_t)g * p.n_ctx + p.t);
-        lm = __ldg(p.lam + g);
-      }
-    }
-
-    row_stats_full<NV>(v, inv_d, p.eps, mean, rstd);
-    const float nmr2 = -mean * rstd;
-    WT* ar = reinterpret_cast<WT*>(p.a) + row * d + c0;
-    const float* g2 = p.ln2_g + c0;
-    const float* b2 = p.ln2_b + c0;
-#pragma unroll
-    for (int i = 0; i < NV; ++i) {
-      const float4 gg = ldg4(g2 + i * 128), bb = ldg4(b2 + i * 128);
-      float4 o;
-      o.x = fmaf(fmaf(v[i].x, rstd, nmr2), gg.x, bb.x); o.y = fmaf(fmaf(v[i].y, rstd, nmr2), gg.y, bb.y);
-      o.z = fmaf(fmaf(v[i].z, rstd, nmr2), gg.z, bb.z); o.w = fmaf(fmaf(v[i].w, rstd, nmr2), gg.w, bb.w);
-      st4(ar + i * 128, o);
-    }
-    return;
-  }
 
   float4 v[NV];
   if (p.tok != nullptr) {

@@ -18,6 +18,7 @@
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
 #include "mixer.cuh"
+#include "mixer_stream.cuh"
 #include "prefill.cuh"
 #include "select.cuh"
 
@@ -288,26 +289,39 @@ cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_
   return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
 
+template <int NV, typename WT, typename ST>
+int launch_mixer_stream(const MixerParams& p, int num_sms, cudaStream_t st) {
+  const int warps = mixer_stream_warps(p.d, (int)sizeof(ST));
+  const size_t smem = mixer_stream_smem(p.d, (int)sizeof(ST), warps);
+  static bool attr_set = false;               // per instantiation
+  if (!attr_set) {
+    SRM_CUDA(cudaFuncSetAttribute(mixer_stream_kernel<NV, WT, ST>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  kStreamSmemBudget));
+    attr_set = true;
+  }
+  const unsigned grid = (unsigned)(p.R < num_sms ? p.R : num_sms);
+  SRM_CUDA(launch_kernel(mixer_stream_kernel<NV, WT, ST>, dim3(grid), dim3(warps * 32), smem, st, p));
+  return SRM_OK;
+}
+
 template <typename WT, typename ST>
-int launch_mixer_nv(const MixerParams& p, cudaStream_t st) {
+int launch_mixer_nv(const MixerParams& p, int num_sms, cudaStream_t st) {
   const int nv = (p.d + 127) / 128;
+  // whole 128-channel vectors per lane, each inside one head: the streaming kernel
+  const bool fast = p.d % 128 == 0 && (p.d / p.h) % 128 == 0 && p.h <= 8 && mixer_stream_warps(p.d, (int)sizeof(ST)) >= 1;
+  if (fast && nv == 4) return launch_mixer_stream<4, WT, ST>(p, num_sms, st);
+  if (fast && nv == 8) return launch_mixer_stream<8, WT, ST>(p, num_sms, st);
+  if (fast && nv == 12) return launch_mixer_stream<12, WT, ST>(p, num_sms, st);
+  if (fast && nv == 16) return launch_mixer_stream<16, WT, ST>(p, num_sms, st);
   const unsigned grid = (unsigned)((p.R + kMixerWarps - 1) / kMixerWarps);
   const dim3 blk(kMixerWarps * 32);
-  // whole 128-channel vectors per lane, each inside one head: the lean path
-  const bool fast = p.d % 128 == 0 && (p.d / p.h) % 128 == 0 && (nv == 4 || nv == 8 || nv == 12 || nv == 16);
-  if (fast) {
-    if (nv == 4) SRM_CUDA(launch_kernel(mixer_step_kernel<4, true, WT, ST>, dim3(grid), dim3(blk), 0, st, p));
-    else if (nv == 8) SRM_CUDA(launch_kernel(mixer_step_kernel<8, true, WT, ST>, dim3(grid), dim3(blk), 0, st, p));
-    else if (nv == 12) SRM_CUDA(launch_kernel(mixer_step_kernel<12, true, WT, ST>, dim3(grid), dim3(blk), 0, st, p));
-    else SRM_CUDA(launch_kernel(mixer_step_kernel<16, true, WT, ST>, dim3(grid), dim3(blk), 0, st, p));
-  } else if (nv <= 1) SRM_CUDA(launch_kernel(mixer_step_kernel<1, false, WT, ST>, dim3(grid), dim3(blk), 0, st, p));
-  else if (nv <= 2) SRM_CUDA(launch_kernel(mixer_step_kernel<2, false, WT, ST>, dim3(grid), dim3(blk), 0, st, p));
-  else if (nv <= 4) SRM_CUDA(launch_kernel(mixer_step_kernel<4, false, WT, ST>, dim3(grid), dim3(blk), 0, st, p));
-  else if (nv <= 6) SRM_CUDA(launch_kernel(mixer_step_kernel<6, false, WT, ST>, dim3(grid), dim3(blk), 0, st, p));
-  else if (nv <= 8) SRM_CUDA(launch_kernel(mixer_step_kernel<8, false, WT, ST>, dim3(grid), dim3(blk), 0, st, p));
-  else if (nv <= 12) SRM_CUDA(launch_kernel(mixer_step_kernel<12, false, WT, ST>, dim3(grid), dim3(blk), 0, st, p));
-  else SRM_CUDA(launch_kernel(mixer_step_kernel<16, false, WT, ST>, dim3(grid), dim3(blk), 0, st, p));
-  SRM_CUDA(cudaGetLastError());
+  if (nv <= 1) SRM_CUDA(launch_kernel(mixer_step_kernel<1, WT, ST>, dim3(grid), dim3(blk), 0, st, p));
+  else if (nv <= 2) SRM_CUDA(launch_kernel(mixer_step_kernel<2, WT, ST>, dim3(grid), dim3(blk), 0, st, p));
+  else if (nv <= 4) SRM_CUDA(launch_kernel(mixer_step_kernel<4, WT, ST>, dim3(grid), dim3(blk), 0, st, p));
+  else if (nv <= 6) SRM_CUDA(launch_kernel(mixer_step_kernel<6, WT, ST>, dim3(grid), dim3(blk), 0, st, p));
+  else if (nv <= 8) SRM_CUDA(launch_kernel(mixer_step_kernel<8, WT, ST>, dim3(grid), dim3(blk), 0, st, p));
+  else if (nv <= 12) SRM_CUDA(launch_kernel(mixer_step_kernel<12, WT, ST>, dim3(grid), dim3(blk), 0, st, p));
+  else SRM_CUDA(launch_kernel(mixer_step_kernel<16, WT, ST>, dim3(grid), dim3(blk), 0, st, p));
   return SRM_OK;
 }
 
@@ -323,10 +337,10 @@ int launch_mixer(const srm_model& m, int layer, int t, int64_t R, const int32_t*
   p.R = R; p.d = m.cfg.d_model; p.h = m.cfg.n_heads; p.n_ctx = m.cfg.n_ctx; p.t = t; p.vocab = m.cfg.vocab;
   p.eps = m.cfg.ln_eps; p.status = status;
   const bool wb = m.cfg.dtype == SRM_DTYPE_BF16, sb = m.cfg.state_dtype == SRM_DTYPE_BF16;
-  if (wb && sb) return launch_mixer_nv<bf16, bf16>(p, st);
-  if (wb) return launch_mixer_nv<bf16, float>(p, st);
-  if (sb) return launch_mixer_nv<float, bf16>(p, st);
-  return launch_mixer_nv<float, float>(p, st);
+  if (wb && sb) return launch_mixer_nv<bf16, bf16>(p, m.num_sms, st);
+  if (wb) return launch_mixer_nv<bf16, float>(p, m.num_sms, st);
+  if (sb) return launch_mixer_nv<float, bf16>(p, m.num_sms, st);
+  return launch_mixer_nv<float, float>(p, m.num_sms, st);
 }
 
 template <typename WT>
