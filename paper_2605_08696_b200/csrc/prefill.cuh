@@ -1,9 +1,10 @@
 // Sequence-parallel token mixing over a prompt (Method/Architecture, Eq. 1 and Eq. 3).
 //
 // One CTA owns one sample and walks its n positions in tiles of T positions. Inside a tile the
-// mixing is the explicit matrix product Y = Z M + B with the T x T diagonal block of M built
-// from alpha and lambda (row-repeat: M[i][j] = lambda^(j-i) alpha_i, column-repeat:
-// lambda^(j-i) alpha_j, i <= j). The blocks of M above the diagonal are rank one, so their
+// mixing is the explicit matrix product Y = Z M + B with the T x T diagonal block of M generated on
+// the fly from alpha and lambda (row-repeat: M[i][j] = lambda^(j-i) alpha_i, column-repeat:
+// lambda^(j-i) alpha_j, i <= j): each thread keeps its head's powers lambda^0..lambda^T in registers
+// and the tile's alpha in shared memory, so the product needs no loads of M. The blocks of M above the diagonal are rank one, so their
 // contribution is carried between tiles as the d-vector sum term of Eq. 2 / Eq. 3, which after
 // the last tile is exactly the cache the recurrent form continues from. With T >= n this is the
 // paper's full n x n product. LN1, the residual add and LN2 are fused around the mixing, so each
@@ -41,7 +42,6 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_mixer_kernel(const Pr
   pdl_wait();
   constexpr int T = kPrefillTile;
   extern __shared__ float xs[];                       // [T][d] tile of the residual stream
-  __shared__ float Mt[kPrefillMaxHeads][T][T];        // diagonal block of M per head
   __shared__ float pw[kPrefillMaxHeads][T + 1];       // lambda^k
   __shared__ float al[kPrefillMaxHeads][T];           // alpha of the tile's positions
   __shared__ float mu[T], rs[T];                      // LN1 statistics of the tile's rows
@@ -83,20 +83,18 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_mixer_kernel(const Pr
       al[g][r] = (r < rows) ? __ldg(p.alpha + (int64_t)g * p.n_ctx + j0 + r) : 0.f;
     }
     __syncthreads();
-    // ---- diagonal block of M, and LN1 statistics (one warp per row) ----
-    for (int i = tid; i < h * T * T; i += kPrefillThreads) {
-      const int g = i / (T * T), r = (i / T) % T, c = i % T;     // M[r][c]: input r -> output c
-      float m = 0.f;
-      if (r <= c) m = pw[g][c - r] * (g < h_row ? al[g][r] : al[g][c]);
-      Mt[g][r][c] = m;
-    }
+    // ---- LN1 statistics (one warp per row) ----
     for (int r = warp; r < rows; r += kPrefillThreads / 32) {
       const float* xr = xs + r * d;
       float s = 0.f;
-      for (int c = lane; c < d; c += 32) s += xr[c];
+      for (int c = lane * 4; c < d; c += 128) { const float4 v = ld4(xr + c); s += (v.x + v.y) + (v.z + v.w); }
       const float mean = warp_sum(s) / (float)d;
       float q = 0.f;
-      for (int c = lane; c < d; c += 32) { const float t = xr[c] - mean; q += t * t; }
+      for (int c = lane * 4; c < d; c += 128) {
+        const float4 v = ld4(xr + c);
+        const float t0 = v.x - mean, t1 = v.y - mean, t2 = v.z - mean, t3 = v.w - mean;
+        q += (t0 * t0 + t1 * t1) + (t2 * t2 + t3 * t3);
+      }
       const float rstd = rsqrtf(warp_sum(q) / (float)d + p.eps);
       if (lane == 0) { mu[r] = mean; rs[r] = rstd; }
     }
@@ -109,28 +107,42 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_mixer_kernel(const Pr
         const int g = c / dh;
         const bool is_row = g < h_row;
         const float gg = __ldg(p.ln1_g + c), bb = __ldg(p.ln1_b + c);
-        float z[T];
+        // powers of this head's lambda and the tile's inputs u_i = alpha_i z_i (row-repeat) or z_i (column-repeat)
+        float lp[T + 1];
 #pragma unroll
-        for (int i = 0; i < T; ++i) z[i] = (i < rows) ? (xs[i * d + c] - mu[i]) * rs[i] * gg + bb : 0.f;
+        for (int k = 0; k <= T; ++k) lp[k] = pw[g][k];
+        float u[T];
+#pragma unroll
+        for (int i = 0; i < T; ++i) {
+          const float z = (i < rows) ? (xs[i * d + c] - mu[i]) * rs[i] * gg + bb : 0.f;
+          u[i] = is_row ? al[g][i] * z : z;
+        }
         const float S0 = carry[q];
 #pragma unroll
         for (int j = 0; j < T; ++j) {
           if (j < rows) {
-            float acc = 0.f;
+            // column j of the diagonal block: sum_i z_i M[i][j] with M[i][j] = lambda^(j-i) alpha_i (row)
+            // or lambda^(j-i) alpha_j (column), plus the rank-one blocks above it folded into the carried sum
+            float acc = lp[j] * S0;
 #pragma unroll
-            for (int i = 0; i <= j; ++i) acc = fmaf(z[i], Mt[g][i][j], acc);
-            // rank-one blocks above the diagonal, folded into the carried sum term
-            const float tail = pw[g][j] * S0;
-            acc += is_row ? tail : al[g][j] * tail;
+            for (int i = 0; i <= j; ++i) acc = fmaf(u[i], lp[j - i], acc);
+            if (!is_row) acc *= al[g][j];
             acc += __ldg(p.beta + (int64_t)(j0 + j) * d + c);
             xs[j * d + c] += acc;
           }
         }
-        // sum term for the position after this tile
-        float sn = pw[g][rows] * S0;
+        // sum term for the position after this tile (u_i = 0 beyond the last row of a ragged tile)
+        float sn;
+        if (rows == T) {
+          sn = lp[T] * S0;
 #pragma unroll
-        for (int i = 0; i < T; ++i) {
-          if (i < rows) sn = fmaf(pw[g][rows - i] * (is_row ? al[g][i] : 1.f), z[i], sn);
+          for (int i = 0; i < T; ++i) sn = fmaf(lp[T - i], u[i], sn);
+        } else {
+          sn = pw[g][rows] * S0;
+#pragma unroll
+          for (int i = 0; i < T; ++i) {
+            if (i < rows) sn = fmaf(pw[g][rows - i], u[i], sn);
+          }
         }
         carry[q] = sn;
       }
@@ -140,10 +152,14 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_mixer_kernel(const Pr
     for (int r = warp; r < rows; r += kPrefillThreads / 32) {
       const float* xr = xs + r * d;
       float s = 0.f;
-      for (int c = lane; c < d; c += 32) s += xr[c];
+      for (int c = lane * 4; c < d; c += 128) { const float4 v = ld4(xr + c); s += (v.x + v.y) + (v.z + v.w); }
       const float mean = warp_sum(s) / (float)d;
       float q = 0.f;
-      for (int c = lane; c < d; c += 32) { const float t = xr[c] - mean; q += t * t; }
+      for (int c = lane * 4; c < d; c += 128) {
+        const float4 v = ld4(xr + c);
+        const float t0 = v.x - mean, t1 = v.y - mean, t2 = v.z - mean, t3 = v.w - mean;
+        q += (t0 * t0 + t1 * t1) + (t2 * t2 + t3 * t3);
+      }
       const float rstd = rsqrtf(warp_sum(q) / (float)d + p.eps);
       float* xo = p.x + (row0 + r) * d;
       WT* ao = reinterpret_cast<WT*>(p.a) + (row0 + r) * d;

@@ -45,7 +45,12 @@ def _teacher_forced(shape, W, model, prompts, gen, sampling=None, sample_idx=Non
         lg_np = lg.cpu().numpy()
         worst = max(worst, rel_err_rows(lg_np, logits_o[k]))
         if samp_o["mode"] == "greedy":
-            strict = top2_margin(logits_o[k]) > MARGIN
+            # Both of the top two logits can move by the row's device error eps, so a decision is only
+            # determined when the oracle's margin exceeds 2 eps. In fp32 mode eps ~ 1e-6 and the rule is the
+            # plain 1e-2 margin; in bf16 mode eps (bounded by the logit tolerance asserted below) reaches
+            # ~1e-2 on the 16- and 24-layer models, and the guard keeps a 0.0101 margin from counting.
+            eps_row = np.max(np.abs(lg_np - logits_o[k]), axis=-1)
+            strict = top2_margin(logits_o[k]) > np.maximum(MARGIN, 2.0 * eps_row)
             checked += int(strict.sum())
             mism += int(np.sum(tok_g[strict] != toks_o[strict, k]))
             exempt += int(np.sum(~strict))
