@@ -30,7 +30,7 @@ L2_BYTES = 126e6
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # DRAM traffic of the dominant kernel per launch (bytes), from the ncu capture summarised in
 # profiles/; None until a capture exists for the benchmarked shape.
-GEMM_DRAM_TRAFFIC_PER_STEP = None
+GEMM_DRAM_TRAFFIC_PER_STEP = {"mid": 1.303e9}      # cold-cache (ncu flushes between passes), mid model at batch 4096
 
 
 def measured_peaks():
@@ -358,7 +358,8 @@ def run_ours(args):
                          "achieved": round(achieved_tf, 1), "peak": peak_tf, "unit": "TFLOP/s",
                          "frac": round(achieved_tf / peak_tf, 4), "peak_source": f"bf16_tflops_sustained, {peak_src}",
                          "frac_of_burst_peak": round(achieved_tf / peaks["bf16_tflops"], 4),
-                         "launches": int(gemm_launches), "traffic": GEMM_DRAM_TRAFFIC_PER_STEP,
+                         "launches": int(gemm_launches),
+                         "traffic": GEMM_DRAM_TRAFFIC_PER_STEP.get(args.workload) if B == 4096 else None,
                          "flops_per_step": B * step_flops(shape)},
             "step_roofline": {"bound": bound, "t_roof_ms": round(t_roof * 1e3, 4), "t_tensor_ms": round(t_tc * 1e3, 4),
                               "t_hbm_ms": round(t_hbm * 1e3, 4), "frac": round(t_roof * 1e3 / (t_ms_max / args.steps), 4),

@@ -81,9 +81,19 @@ argmax_reduce_kernel(const uint2* __restrict__ part, int64_t R, int64_t slots, i
   float bv = -INFINITY;
   int bi = 0x7fffffff;
   if (row < R) {
-    for (int64_t s = sl; s < slots; s += kArgmaxLanes) {
-      const uint2 p = __ldg(part + s * R + row);
-      argmax_take(__uint_as_float(p.x), (int)p.y, bv, bi);
+    // eight independent loads in flight per thread; slots are visited in ascending order, so the
+    // lowest column among equal maxima is kept
+    int64_t s = sl;
+    for (; s + 7 * kArgmaxLanes < slots; s += 8 * kArgmaxLanes) {
+      uint2 q[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) q[u] = __ldg(part + (s + u * kArgmaxLanes) * R + row);
+#pragma unroll
+      for (int u = 0; u < 8; ++u) argmax_take(__uint_as_float(q[u].x), (int)q[u].y, bv, bi);
+    }
+    for (; s < slots; s += kArgmaxLanes) {
+      const uint2 q = __ldg(part + s * R + row);
+      argmax_take(__uint_as_float(q.x), (int)q.y, bv, bi);
     }
   }
   sv[sl][rr] = bv; si[sl][rr] = bi;
