@@ -21,6 +21,9 @@ Parity status of each function (what pins it, see tests/test_oracle_*.py):
   layer_norm, gelu_erf     pinned: moments / identities / tabulated erf values
   philox4x32_10            pinned: cuRAND's host Philox4_32_10 generator, bijectivity
   select_greedy, select_topk  pinned: brute-force sort, frequency test
+  token_mixer_parallel / _recurrent with head projections (Eq. 10)
+                           pinned: brute-force Eq. 10 in the paper's d x n orientation with explicit
+                           per-head I_g, identity projections == no projections, parallel == recurrent
   SRMOracle (full model logits)  PARITY UNPINNED beyond self-consistency (parallel ==
                            recurrent, causality): the paper prints no activations and
                            its architecture figure is missing, so the block structure
@@ -211,6 +214,32 @@ def select_topk(logits: np.ndarray, k: int, temperature: float, seed: int,
 
 
 # --------------------------------------------------------------------------------------
+# Head projections (Method / Architecture, Eq. 10): Y = P_out (concat_g [(I_g X) M_g + beta_g])
+# --------------------------------------------------------------------------------------
+
+def token_mixer_parallel(Z: np.ndarray, lw: dict, n_heads: int, matrices=None):
+    """Sequence-parallel token-mixing block of one layer for one sample, Z[n, d] (normed inputs).
+    Without projections this is mixer_parallel. With lw["W_in"] (rows g*d_h..(g+1)*d_h = I_g) and
+    lw["W_out"] (= P_out): every position is projected, Q = Z W_in^T, the heads of Q are mixed along
+    the sequence, and the concatenated result is projected back, Y = (.) W_out^T. The cache is the
+    sum term of the PROJECTED values."""
+    if "W_in" not in lw:
+        return mixer_parallel(Z, lw["alpha"], lw["beta"], lw["lam"], n_heads, matrices)
+    Q = Z @ lw["W_in"].T
+    Yh, S = mixer_parallel(Q, lw["alpha"], lw["beta"], lw["lam"], n_heads, matrices)
+    return Yh @ lw["W_out"].T, S
+
+
+def token_mixer_recurrent(z: np.ndarray, S: np.ndarray, t: int, lw: dict, n_heads: int):
+    """Recurrent counterpart of token_mixer_parallel for position t (batched over rows)."""
+    if "W_in" not in lw:
+        return mixer_recurrent_step(z, S, t, lw["alpha"], lw["beta"], lw["lam"], n_heads)
+    q = z @ lw["W_in"].T
+    yh, S_new = mixer_recurrent_step(q, S, t, lw["alpha"], lw["beta"], lw["lam"], n_heads)
+    return yh @ lw["W_out"].T, S_new
+
+
+# --------------------------------------------------------------------------------------
 # The model
 # --------------------------------------------------------------------------------------
 
@@ -244,7 +273,7 @@ class SRMOracle:
             Ms = [mixing_matrix(kind, lw["alpha"][g], lw["lam"][g], n, dtype=self.dt)
                   for g, kind in enumerate(head_kinds(self.h))]
             for b in range(B):
-                y[b], state[l, b] = mixer_parallel(z[b], lw["alpha"], lw["beta"], lw["lam"], self.h, Ms)
+                y[b], state[l, b] = token_mixer_parallel(z[b], lw, self.h, Ms)
             x = x + y
             a = layer_norm(x, lw["ln2_g"], lw["ln2_b"], self.eps)
             x = x + feed_forward(a, lw["W1"], lw["b1"], lw["W2"], lw["b2"])
@@ -266,8 +295,7 @@ class SRMOracle:
         xs = []
         for l, lw in enumerate(self.layers):
             z = layer_norm(x, lw["ln1_g"], lw["ln1_b"], self.eps)
-            y, new_state[l] = mixer_recurrent_step(z, state[l], pos, lw["alpha"], lw["beta"],
-                                                   lw["lam"], self.h)
+            y, new_state[l] = token_mixer_recurrent(z, state[l], pos, lw, self.h)
             x = x + y
             a = layer_norm(x, lw["ln2_g"], lw["ln2_b"], self.eps)
             x = x + feed_forward(a, lw["W1"], lw["b1"], lw["W2"], lw["b2"])

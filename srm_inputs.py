@@ -29,6 +29,7 @@ class SRMShape:
     dtype: str = "bf16"        # "fp32" or "bf16" (weights + GEMM inputs; fp32 accumulate)
     seed: int = 0
     ln_eps: float = 1e-5
+    head_proj: bool = False    # per-head input projections I_h (stacked: W_in[d,d]) and output projection W_out[d,d]
 
     @property
     def d_ffn(self) -> int:
@@ -77,11 +78,12 @@ def make_weights(shape: SRMShape, *, std: float = 0.02, alpha_std: float | None 
     Returns a dict of fp32 numpy arrays:
       E[V,d], lnf_g[d], lnf_b[d], W_lm[V,d], and a list "layers" of dicts with
       ln1_g, ln1_b, alpha[h,n_ctx], beta[n_ctx,d], lam[h], ln2_g, ln2_b,
-      W1[F,d], b1[F], W2[d,F], b2[d].
+      W1[F,d], b1[F], W2[d,F], b2[d], and with shape.head_proj also W_in[d,d] (rows g*d_h..(g+1)*d_h are
+      head g's input projection I_g) and W_out[d,d] (the output projection P_out).
     Norm gains are 1 + N(0,std^2) and norm shifts N(0,std^2) so that the affine part of
     every norm is exercised. The decay constants lam are uniform on (lam_lo, 1) except
     head 0 of each layer, which is exactly 1 (the closed end of the allowed interval).
-    In bf16 mode the matrices (E, W1, W2, W_lm) are rounded to bf16 once, here.
+    In bf16 mode the matrices (E, W1, W2, W_lm, W_in, W_out) are rounded to bf16 once, here.
     """
     rng = np.random.Generator(np.random.Philox(key=shape.seed))
     d, F, V, n, h = shape.d_model, shape.d_ffn, shape.vocab, shape.n_ctx, shape.n_heads
@@ -105,6 +107,9 @@ def make_weights(shape: SRMShape, *, std: float = 0.02, alpha_std: float | None 
             "ln2_g": (1.0 + nrm(d)).astype(np.float32), "ln2_b": nrm(d),
             "W1": mat(F, d), "b1": nrm(F), "W2": mat(d, F), "b2": nrm(d),
         })
+        if shape.head_proj:        # drawn last, so the tensors above do not depend on the switch within a layer
+            W["layers"][-1]["W_in"] = mat(d, d)
+            W["layers"][-1]["W_out"] = mat(d, d)
     W["lnf_g"] = (1.0 + nrm(d)).astype(np.float32)
     W["lnf_b"] = nrm(d)
     W["W_lm"] = mat(V, d)
