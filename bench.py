@@ -102,14 +102,15 @@ class ClockSampler:
 
 def step_flops(shape):
     d, L, V = shape.d_model, shape.n_layers, shape.vocab
-    return 16 * L * d * d + 2 * d * V            # per generated token
+    per_layer = 20 if shape.head_proj else 16    # FFN up + down (16 d^2), head projections W_in + W_out (4 d^2)
+    return per_layer * L * d * d + 2 * d * V     # per generated token
 
 
 def step_roofline_s(shape, B, state_bytes, peaks):
     """Slower of the step's FLOPs at the tensor peak and its weight + state bytes at HBM bandwidth."""
     d, L, V = shape.d_model, shape.n_layers, shape.vocab
     t_tc = B * step_flops(shape) / (peaks["bf16_tflops_sustained"] * 1e12)
-    bytes_ = 2 * (8 * L * d * d + d * V) + B * 2 * L * d * state_bytes
+    bytes_ = step_flops(shape) + B * 2 * L * d * state_bytes      # bf16 weights: as many bytes as flop per token
     t_hbm = bytes_ / (peaks["hbm_gbs"] * 1e9)
     return max(t_tc, t_hbm), ("tensor" if t_tc >= t_hbm else "hbm"), t_tc, t_hbm
 
@@ -126,6 +127,9 @@ def run_reference(args):
     from oracle import srm_oracle as O
     w = I.WORKLOADS[args.workload]
     shape = I.CONFIGS[w["model"]]
+    if args.head_proj:
+        import dataclasses
+        shape = dataclasses.replace(shape, head_proj=True)
     B_full = args.batch or w["batch"] or 4096
     sample = min(B_full, args.ref_samples)
     W = I.make_weights(shape)
@@ -166,7 +170,7 @@ def _blas_threads():
 
 
 def _config_dict(args, shape, w, B, extra=None):
-    c = {"workload": f"{args.workload}: SRM L{shape.n_layers} d{shape.d_model} F{shape.d_ffn} V{shape.vocab} "
+    c = {"workload": f"{args.workload}{' + head projections' if shape.head_proj else ''}: SRM L{shape.n_layers} d{shape.d_model} F{shape.d_ffn} V{shape.vocab} "
                      f"n_ctx{shape.n_ctx} {shape.dtype}, batch {B}, prompts {w['prompt_len']} tokens ({w['prompts']}), "
                      f"{w['sampling']} selection",
          "batch_per_gpu": B, "prompt_len": w["prompt_len"], "selection": w["sampling"],
@@ -221,6 +225,9 @@ def run_ours(args):
 
     w = I.WORKLOADS[args.workload]
     shape = I.CONFIGS[w["model"]]
+    if args.head_proj:
+        import dataclasses
+        shape = dataclasses.replace(shape, head_proj=True)
     B = args.batch or w["batch"] or 4096
     n = w["prompt_len"]
     peaks, peak_src = measured_peaks()
@@ -294,8 +301,8 @@ def run_ours(args):
     model.profile(False)
     prof = model.profile_read()
     d, L, V, F = shape.d_model, shape.n_layers, shape.vocab, shape.d_ffn
-    gemm_ms = sum(prof[k][1] for k in ("gemm_up", "gemm_down", "gemm_lm"))
-    gemm_launches = sum(prof[k][0] for k in ("gemm_up", "gemm_down", "gemm_lm"))
+    gemm_ms = sum(prof[k][1] for k in ("gemm_up", "gemm_down", "gemm_lm", "gemm_proj"))
+    gemm_launches = sum(prof[k][0] for k in ("gemm_up", "gemm_down", "gemm_lm", "gemm_proj"))
     gemm_flops = args.steps * B * step_flops(shape)
     achieved_tf = gemm_flops / (gemm_ms / 1e3) / 1e12 if gemm_ms > 0 else 0.0
     prof_total = sum(v[1] for v in prof.values())
@@ -307,6 +314,8 @@ def run_ours(args):
     kernels["gemm_up"]["tflops"] = round(args.steps * L * B * 2 * d * F / (prof["gemm_up"][1] / 1e3) / 1e12, 1)
     kernels["gemm_down"]["tflops"] = round(args.steps * L * B * 2 * d * F / (prof["gemm_down"][1] / 1e3) / 1e12, 1)
     kernels["gemm_lm"]["tflops"] = round(args.steps * B * 2 * d * V / (prof["gemm_lm"][1] / 1e3) / 1e12, 1)
+    if shape.head_proj:
+        kernels["gemm_proj"]["tflops"] = round(args.steps * L * B * 4 * d * d / (prof["gemm_proj"][1] / 1e3) / 1e12, 1)
     kernels["mixer"]["gbs"] = round(mixer_bytes / (prof["mixer"][1] / 1e3) / 1e9, 1)
     kernels["select"]["gbs"] = round(args.steps * B * V * 4 / (prof["select"][1] / 1e3) / 1e9, 1)
 
@@ -444,6 +453,8 @@ def main():
     ap.add_argument("--state-dtype", default="fp32", choices=["fp32", "bf16"])
     ap.add_argument("--ref-samples", type=int, default=32)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--head-proj", action="store_true",
+                    help="token mixer with head projections (Eq. 10): adds W_in, W_out [d, d] per layer")
     ap.add_argument("--no-prefill", action="store_true",
                     help="skip the prefill (cache stays zero, pos = prompt length): keeps profiler captures short")
     ap.add_argument("--sweep", action="store_true")

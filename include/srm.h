@@ -59,7 +59,13 @@ enum srm_status_bits {
 
 enum { SRM_DTYPE_FP32 = 0, SRM_DTYPE_BF16 = 1 };
 enum { SRM_SELECT_GREEDY = 0, SRM_SELECT_TOPK = 1 };
-enum { SRM_FLAG_SIMT_GEMM = 1 };     /* debug: run the bf16 GEMMs on the plain SIMT kernel  */
+enum {
+  SRM_FLAG_SIMT_GEMM = 1,            /* debug: run the bf16 GEMMs on the plain SIMT kernel  */
+  SRM_FLAG_HEAD_PROJ = 2             /* token mixer with head projections [Method/Architecture, Eq. 10]:
+                                        q = W_in LN1(x) (W_in stacks the per-head I_g), heads of q mixed, and
+                                        x += W_out (concatenated heads); the cache holds projected values.
+                                        Adds W_in, W_out [d, d] per layer to the blob and 4 L d^2 flop per token */
+};
 
 /* Model description. Heads g < n_heads/2 are row-repeat, the rest column-repeat. */
 typedef struct {
@@ -107,6 +113,9 @@ enum srm_tensor {
   SRM_T_B2,           /* [d]                                                               */
   SRM_T_LNF_G, SRM_T_LNF_B,          /* [d]  final norm (global)                           */
   SRM_T_W_LM,         /* [V, d]    LM head, no bias (global)                               */
+  SRM_T_W_IN,         /* [d, d]    per layer, only with SRM_FLAG_HEAD_PROJ: rows g*d_h.. are I_g; placed
+                                   after B2 in the layer's part of the blob                          */
+  SRM_T_W_OUT,        /* [d, d]    per layer, only with SRM_FLAG_HEAD_PROJ: P_out                   */
   SRM_T_COUNT
 };
 
@@ -223,7 +232,7 @@ int srm_k_mixer_step(srm_model* m, int32_t layer, int32_t t, int64_t R, const in
 int srm_k_final_norm(srm_model* m, int64_t R, const float* d_x, void* d_a, void* stream);
 /* Dense projection D[M, N] = A[M, K] * W[N, K]^T with one of three epilogues:
  *   0: out_act[M, N] = gelu_erf(D + bias)      (activation type)
- *   1: out_f32[M, N] += D + bias               (fp32 residual stream)
+ *   1: out_f32[M, N] += D + bias               (fp32 residual stream; d_bias may be NULL: no bias)
  *   2: out_f32[M, N] = D                       (fp32 logits)
  * A, W in the activation type of cfg.dtype; bf16 runs on the tcgen05 tensor-core kernel
  * (or the SIMT kernel when cfg.flags has SRM_FLAG_SIMT_GEMM), fp32 on the SIMT kernel. */
@@ -258,6 +267,7 @@ enum srm_kernel_class {
   SRM_KERNEL_NORM,               /* final norm                                                 */
   SRM_KERNEL_SELECT,             /* token selection                                            */
   SRM_KERNEL_PREFILL_MIXER,      /* sequence-parallel token mixing                             */
+  SRM_KERNEL_GEMM_PROJ,          /* head projections W_in, W_out (SRM_FLAG_HEAD_PROJ)          */
   SRM_KERNEL_CLASS_COUNT
 };
 /* While enabled, every kernel launch of this model is bracketed by two CUDA events recorded on the

@@ -17,10 +17,11 @@ from . import build as _build
 EPI_BIAS_GELU, EPI_BIAS_RESIDUAL, EPI_PLAIN = 0, 1, 2
 DTYPE_FP32, DTYPE_BF16 = 0, 1
 FLAG_SIMT_GEMM = 1
+FLAG_HEAD_PROJ = 2
 
 # enum srm_tensor
 T_E, T_LN1_G, T_LN1_B, T_ALPHA, T_BETA, T_LAMBDA, T_LN2_G, T_LN2_B, T_W1, T_B1, T_W2, T_B2, \
-    T_LNF_G, T_LNF_B, T_W_LM = range(15)
+    T_LNF_G, T_LNF_B, T_W_LM, T_W_IN, T_W_OUT = range(17)
 _LAYER_TENSORS = {"ln1_g": T_LN1_G, "ln1_b": T_LN1_B, "alpha": T_ALPHA, "beta": T_BETA, "lam": T_LAMBDA,
                   "ln2_g": T_LN2_G, "ln2_b": T_LN2_B, "W1": T_W1, "b1": T_B1, "W2": T_W2, "b2": T_B2}
 _GLOBAL_TENSORS = {"E": T_E, "lnf_g": T_LNF_G, "lnf_b": T_LNF_B, "W_lm": T_W_LM}
@@ -207,6 +208,8 @@ class SRM:
     def __init__(self, shape, weights: dict, device: str = "cuda:0", state_dtype: str = "fp32", flags: int = 0):
         lib = _lib()
         dt = _shape_get(shape, "dtype")
+        if (shape.get("head_proj", False) if isinstance(shape, dict) else getattr(shape, "head_proj", False)):
+            flags |= FLAG_HEAD_PROJ
         self.cfg = _Config(_shape_get(shape, "n_layers"), _shape_get(shape, "d_model"), _shape_get(shape, "n_heads"),
                            _shape_get(shape, "ffn_mult"), _shape_get(shape, "vocab"), _shape_get(shape, "n_ctx"),
                            DTYPE_BF16 if dt == "bf16" else DTYPE_FP32,
@@ -236,6 +239,9 @@ class SRM:
         for l, lw in enumerate(weights["layers"]):
             for name, tid in _LAYER_TENSORS.items():
                 put(l, tid, lw[name])
+            if flags & FLAG_HEAD_PROJ:
+                put(l, T_W_IN, lw["W_in"])
+                put(l, T_W_OUT, lw["W_out"])
         with torch.cuda.device(self.device):
             self.blob = host.to(self.device)
             self.handle = C.c_void_p()
@@ -315,7 +321,7 @@ class SRM:
         return (tok_out, logits) if want_logits else tok_out
 
     # ---- measurement ----
-    KERNEL_CLASSES = ("mixer", "gemm_up", "gemm_down", "gemm_lm", "norm", "select", "prefill_mixer")
+    KERNEL_CLASSES = ("mixer", "gemm_up", "gemm_down", "gemm_lm", "norm", "select", "prefill_mixer", "gemm_proj")
 
     def profile(self, on: bool):
         _check(_lib().srm_profile_enable(self.handle, int(on)), "srm_profile_enable")

@@ -61,7 +61,7 @@ gemm_simt_kernel(const T* __restrict__ A, const T* __restrict__ W, const float* 
         reinterpret_cast<T*>(out)[m * N + n] = from_float<T>(gelu_erf(v + bias[n]));
       } else if (EPI == kEpiBiasResidual) {
         float* o = reinterpret_cast<float*>(out) + m * N + n;
-        *o = *o + (v + bias[n]);
+        *o = *o + (bias != nullptr ? v + bias[n] : v);
       } else {
         reinterpret_cast<float*>(out)[m * N + n] = v;
       }

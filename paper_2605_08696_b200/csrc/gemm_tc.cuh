@@ -352,7 +352,7 @@ __device__ __forceinline__ void epilogue_columns(const GemmArgs& g, const CUtens
     } else {
 #pragma unroll
       for (int j = 0; j < 16; j += 4) {
-        if (EPI == kEpiBiasResidual && col + j < g.N) {
+        if (EPI == kEpiBiasResidual && g.bias != nullptr && col + j < g.N) {
           const float4 b = __ldg(reinterpret_cast<const float4*>(g.bias + col + j));
           v[16 * (c & 1) + j + 0] = __float_as_uint(__uint_as_float(cur[j + 0]) + b.x);
           v[16 * (c & 1) + j + 1] = __float_as_uint(__uint_as_float(cur[j + 1]) + b.y);

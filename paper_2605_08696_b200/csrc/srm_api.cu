@@ -19,6 +19,7 @@
 #include "gemm_tc.cuh"
 #include "mixer.cuh"
 #include "mixer_stream.cuh"
+#include "mixer_proj.cuh"
 #include "prefill.cuh"
 #include "select.cuh"
 
@@ -69,6 +70,7 @@ size_t tensor_elems(const srm_config& c, int t) {
     case SRM_T_BETA: return n * d;
     case SRM_T_LAMBDA: return h;
     case SRM_T_W1: case SRM_T_W2: return F * d;
+    case SRM_T_W_IN: case SRM_T_W_OUT: return d * d;
     case SRM_T_B1: return F;
     default: return d;
   }
@@ -77,7 +79,9 @@ size_t tensor_elems(const srm_config& c, int t) {
 Layout make_layout(const srm_config& c) {
   Layout L;
   const int wbytes = c.dtype == SRM_DTYPE_BF16 ? 2 : 4;
-  auto is_matrix = [](int t) { return t == SRM_T_E || t == SRM_T_W1 || t == SRM_T_W2 || t == SRM_T_W_LM; };
+  auto is_matrix = [](int t) {
+    return t == SRM_T_E || t == SRM_T_W1 || t == SRM_T_W2 || t == SRM_T_W_LM || t == SRM_T_W_IN || t == SRM_T_W_OUT;
+  };
   size_t off = 0;
   auto place = [&](int t) {
     Slot s;
@@ -90,7 +94,13 @@ Layout make_layout(const srm_config& c) {
   L.global[SRM_T_E] = place(SRM_T_E);
   L.layer.resize((size_t)c.n_layers * SRM_T_COUNT);
   for (int l = 0; l < c.n_layers; ++l)
+  {
     for (int t = SRM_T_LN1_G; t <= SRM_T_B2; ++t) L.layer[(size_t)l * SRM_T_COUNT + t] = place(t);
+    if (c.flags & SRM_FLAG_HEAD_PROJ) {
+      L.layer[(size_t)l * SRM_T_COUNT + SRM_T_W_IN] = place(SRM_T_W_IN);
+      L.layer[(size_t)l * SRM_T_COUNT + SRM_T_W_OUT] = place(SRM_T_W_OUT);
+    }
+  }
   L.global[SRM_T_LNF_G] = place(SRM_T_LNF_G);
   L.global[SRM_T_LNF_B] = place(SRM_T_LNF_B);
   L.global[SRM_T_W_LM] = place(SRM_T_W_LM);
@@ -146,6 +156,7 @@ struct srm_model {
   Layout layout;
   int device = 0;
   int num_sms = 0;
+  bool head_proj() const { return (cfg.flags & SRM_FLAG_HEAD_PROJ) != 0; }
   bool tc_ready = false;                 // smem attribute set for the tensor-core kernels
   int tc_clusters = 0;                   // CTA pairs of the tensor-core kernel that are resident at once
   std::vector<TmapCacheEntry> tmaps;     // weight and activation descriptors, built on first use
@@ -222,18 +233,19 @@ size_t state_bytes_for(const srm_config& c, int64_t B) {
 }
 
 // ---- workspace carving ----------------------------------------------------------------------
-struct DecodeWs { float* x; void* a; void* H; float* logits; int64_t rows; };
-struct PrefillWs { float* x; void* a; void* H; void* a_last; float* logits; int64_t samples; };
+struct DecodeWs { float* x; void* a; void* H; float* logits; float* q; int64_t rows; };     // q: head projections only
+struct PrefillWs { float* x; void* a; void* H; void* a_last; float* logits; float* q; int64_t samples; };
 
 size_t decode_ws_bytes(const srm_model& m, int64_t rows) {
   const size_t d = m.cfg.d_model, F = m.F(), V = m.cfg.vocab, ab = m.act_bytes();
   return align_up(rows * d * 4, 256) + align_up(rows * d * ab, 256) + align_up(rows * F * ab, 256) +
-         align_up(rows * V * 4, 256);
+         align_up(rows * V * 4, 256) + (m.head_proj() ? align_up(rows * d * 4, 256) : 0);
 }
 size_t prefill_ws_bytes(const srm_model& m, int64_t samples, int n) {
   const size_t d = m.cfg.d_model, F = m.F(), V = m.cfg.vocab, ab = m.act_bytes(), rows = (size_t)samples * n;
   return align_up(rows * d * 4, 256) + align_up(rows * d * ab, 256) + align_up(rows * F * ab, 256) +
-         align_up(samples * d * ab, 256) + align_up(samples * V * 4, 256);
+         align_up(samples * d * ab, 256) + align_up(samples * V * 4, 256) +
+         (m.head_proj() ? align_up(rows * d * 4, 256) : 0);
 }
 int64_t fit_rows(size_t ws_bytes, int64_t want, size_t (*need)(const srm_model&, int64_t, int), const srm_model& m, int n) {
   if (need(m, 1, n) > ws_bytes) return 0;
@@ -255,7 +267,8 @@ DecodeWs carve_decode(const srm_model& m, void* ws, int64_t rows) {
   w.x = reinterpret_cast<float*>(p); p += align_up(rows * d * 4, 256);
   w.a = p; p += align_up(rows * d * ab, 256);
   w.H = p; p += align_up(rows * F * ab, 256);
-  w.logits = reinterpret_cast<float*>(p);
+  w.logits = reinterpret_cast<float*>(p); p += align_up(rows * (size_t)m.cfg.vocab * 4, 256);
+  w.q = m.head_proj() ? reinterpret_cast<float*>(p) : nullptr;
   return w;
 }
 PrefillWs carve_prefill(const srm_model& m, void* ws, int64_t samples, int n) {
@@ -267,7 +280,8 @@ PrefillWs carve_prefill(const srm_model& m, void* ws, int64_t samples, int n) {
   w.a = p; p += align_up(rows * d * ab, 256);
   w.H = p; p += align_up(rows * F * ab, 256);
   w.a_last = p; p += align_up(samples * d * ab, 256);
-  w.logits = reinterpret_cast<float*>(p);
+  w.logits = reinterpret_cast<float*>(p); p += align_up(samples * (size_t)m.cfg.vocab * 4, 256);
+  w.q = m.head_proj() ? reinterpret_cast<float*>(p) : nullptr;
   return w;
 }
 
@@ -361,6 +375,15 @@ int launch_norm_t(const float* x, int64_t R, int64_t stride, int64_t offset, con
   return SRM_OK;
 }
 
+// out[r, :] = LN(x[r * stride + offset, :]; g, b) in the activation type
+int launch_norm(const srm_model& m, const float* x, int64_t R, int64_t stride, int64_t offset, const float* g,
+                const float* b, void* out, cudaStream_t st) {
+  if (R <= 0) return SRM_OK;
+  LaunchScope scope(m, SRM_KERNEL_NORM, st);
+  if (m.cfg.dtype == SRM_DTYPE_BF16) return launch_norm_t<bf16>(x, R, stride, offset, g, b, m.cfg.ln_eps, m.cfg.d_model, out, st);
+  return launch_norm_t<float>(x, R, stride, offset, g, b, m.cfg.ln_eps, m.cfg.d_model, out, st);
+}
+
 int launch_final_norm(const srm_model& m, const float* x, int64_t R, int64_t stride, int64_t offset, void* out,
                       cudaStream_t st) {
   if (R <= 0) return SRM_OK;
@@ -430,9 +453,10 @@ int launch_gemm_tc(srm_model& m, int epi, int64_t M, int64_t N, int64_t K, const
 }
 
 int launch_gemm(srm_model& m, int epi, int64_t M, int64_t N, int64_t K, const void* A, const void* W,
-                const float* bias, void* out, uint32_t* status, cudaStream_t st) {
+                const float* bias, void* out, uint32_t* status, cudaStream_t st, int cls = -1) {
   if (M <= 0) return SRM_OK;
-  LaunchScope scope(m, epi == kEpiBiasGelu ? SRM_KERNEL_GEMM_UP : epi == kEpiBiasResidual ? SRM_KERNEL_GEMM_DOWN : SRM_KERNEL_GEMM_LM, st);
+  if (cls < 0) cls = epi == kEpiBiasGelu ? SRM_KERNEL_GEMM_UP : epi == kEpiBiasResidual ? SRM_KERNEL_GEMM_DOWN : SRM_KERNEL_GEMM_LM;
+  LaunchScope scope(m, cls, st);
   if (epi == kEpiArgmax) return launch_gemm_tc(m, epi, M, N, K, A, W, bias, out, status, st);
   if (m.cfg.dtype == SRM_DTYPE_FP32) return launch_gemm_simt<float>(epi, M, N, K, A, W, bias, out, st);
   if (m.cfg.flags & SRM_FLAG_SIMT_GEMM) return launch_gemm_simt<bf16>(epi, M, N, K, A, W, bias, out, st);
@@ -524,6 +548,53 @@ int launch_prefill_mixer(const srm_model& m, int layer, int64_t Bp, int n, const
   return go(prefill_mixer_kernel<float, float>);
 }
 
+// Token-mixing block with head projections (Eq. 10) on `rows` rows of the residual stream:
+//   [x = E[tok]];  a = LN1(x);  q = a W_in^T;  y, S' = mixer(q, S);  x += y W_out^T;  a = LN2(x).
+// Decode: t >= 0, one position, S [rows, d] in/out. Prefill: t < 0, `samples` prompts of n positions
+// (rows = samples * n), sequence-parallel mixing, S [samples, d] out.
+template <typename WT, typename ST>
+int launch_mix_proj_t(bool prefill, const MixProjParams& p, int64_t vecs, cudaStream_t st) {
+  const unsigned grid = (unsigned)((vecs + kMixProjThreads - 1) / kMixProjThreads);
+  if (prefill) SRM_CUDA(launch_kernel(mixer_proj_prefill_kernel<WT, ST>, dim3(grid), dim3(kMixProjThreads), 0, st, p));
+  else SRM_CUDA(launch_kernel(mixer_proj_step_kernel<WT, ST>, dim3(grid), dim3(kMixProjThreads), 0, st, p));
+  return SRM_OK;
+}
+
+int launch_mixer_block_proj(srm_model& m, int layer, int t, int64_t rows, int64_t samples, int n, const int32_t* tok,
+                            float* x, void* S, void* a, float* q, uint32_t* status, cudaStream_t st) {
+  if (rows <= 0) return SRM_OK;
+  const srm_config& c = m.cfg;
+  const int d = c.d_model;
+  const bool prefill = t < 0;
+  const bool wb = c.dtype == SRM_DTYPE_BF16, sb = c.state_dtype == SRM_DTYPE_BF16;
+  int rc;
+  if (tok != nullptr) {
+    LaunchScope scope(m, prefill ? SRM_KERNEL_PREFILL_MIXER : SRM_KERNEL_MIXER, st);
+    const unsigned grid = (unsigned)((rows * (d / 4) + kMixProjThreads - 1) / kMixProjThreads);
+    if (wb) SRM_CUDA(launch_kernel(embed_rows_kernel<bf16>, dim3(grid), dim3(kMixProjThreads), 0, st, tok,
+                                   reinterpret_cast<const bf16*>(m.ptr(-1, SRM_T_E)), x, rows, d, c.vocab, status));
+    else SRM_CUDA(launch_kernel(embed_rows_kernel<float>, dim3(grid), dim3(kMixProjThreads), 0, st, tok,
+                                reinterpret_cast<const float*>(m.ptr(-1, SRM_T_E)), x, rows, d, c.vocab, status));
+  }
+  if ((rc = launch_norm(m, x, rows, 1, 0, m.fptr(layer, SRM_T_LN1_G), m.fptr(layer, SRM_T_LN1_B), a, st))) return rc;
+  if ((rc = launch_gemm(m, kEpiPlain, rows, d, d, a, m.ptr(layer, SRM_T_W_IN), nullptr, q, status, st, SRM_KERNEL_GEMM_PROJ))) return rc;
+  {
+    LaunchScope scope(m, prefill ? SRM_KERNEL_PREFILL_MIXER : SRM_KERNEL_MIXER, st);
+    MixProjParams p;
+    p.q = q; p.S = S; p.y = a;
+    p.alpha = m.fptr(layer, SRM_T_ALPHA); p.beta = m.fptr(layer, SRM_T_BETA); p.lam = m.fptr(layer, SRM_T_LAMBDA);
+    p.R = prefill ? samples : rows; p.d = d; p.h = c.n_heads; p.n_ctx = c.n_ctx; p.t = prefill ? 0 : t; p.n = n;
+    const int64_t vecs = p.R * (d / 4);
+    if (wb && sb) rc = launch_mix_proj_t<bf16, bf16>(prefill, p, vecs, st);
+    else if (wb) rc = launch_mix_proj_t<bf16, float>(prefill, p, vecs, st);
+    else if (sb) rc = launch_mix_proj_t<float, bf16>(prefill, p, vecs, st);
+    else rc = launch_mix_proj_t<float, float>(prefill, p, vecs, st);
+    if (rc) return rc;
+  }
+  if ((rc = launch_gemm(m, kEpiBiasResidual, rows, d, d, a, m.ptr(layer, SRM_T_W_OUT), nullptr, x, status, st, SRM_KERNEL_GEMM_PROJ))) return rc;
+  return launch_norm(m, x, rows, 1, 0, m.fptr(layer, SRM_T_LN2_G), m.fptr(layer, SRM_T_LN2_B), a, st);
+}
+
 // One decode step for rows [b0, b0 + R) of the state.
 int decode_chunk(srm_model& m, srm_state& s, int64_t b0, int64_t R, const int32_t* tok_in, const srm_sampling& samp,
                  int step, const SelectOut& out_all, float* logits_out, const DecodeWs& w, cudaStream_t st) {
@@ -534,7 +605,9 @@ int decode_chunk(srm_model& m, srm_state& s, int64_t b0, int64_t R, const int32_
   int rc;
   for (int l = 0; l < c.n_layers; ++l) {
     uint8_t* Sl = static_cast<uint8_t*>(s.layer_ptr(l)) + (size_t)b0 * d * m.state_bytes();
-    if ((rc = launch_mixer(m, l, t, R, l == 0 ? tok_in + b0 : nullptr, w.x, Sl, w.a, s.status, st))) return rc;
+    if (m.head_proj()) {
+      if ((rc = launch_mixer_block_proj(m, l, t, R, R, 1, l == 0 ? tok_in + b0 : nullptr, w.x, Sl, w.a, w.q, s.status, st))) return rc;
+    } else if ((rc = launch_mixer(m, l, t, R, l == 0 ? tok_in + b0 : nullptr, w.x, Sl, w.a, s.status, st))) return rc;
     if ((rc = launch_gemm(m, kEpiBiasGelu, R, F, d, w.a, m.ptr(l, SRM_T_W1), m.fptr(l, SRM_T_B1), w.H, s.status, st))) return rc;
     if ((rc = launch_gemm(m, kEpiBiasResidual, R, d, F, w.H, m.ptr(l, SRM_T_W2), m.fptr(l, SRM_T_B2), w.x, s.status, st))) return rc;
   }
@@ -589,6 +662,7 @@ int srm_weight_slot(const srm_config* cfg, int32_t layer, int32_t tensor, size_t
     s = L.global[tensor];
   } else {
     if (layer < 0 || layer >= cfg->n_layers) return SRM_ERR_INVALID_ARG;
+    if ((tensor == SRM_T_W_IN || tensor == SRM_T_W_OUT) && !(cfg->flags & SRM_FLAG_HEAD_PROJ)) return SRM_ERR_INVALID_ARG;
     s = L.layer[(size_t)layer * SRM_T_COUNT + tensor];
   }
   if (offset) *offset = s.off;
@@ -753,7 +827,9 @@ int srm_prefill(srm_model* m, srm_state* s, const int32_t* d_tokens, int32_t n, 
     const int64_t rows = nb * n;
     for (int l = 0; l < c.n_layers; ++l) {
       uint8_t* Sl = static_cast<uint8_t*>(s->layer_ptr(l)) + (size_t)b0 * d * m->state_bytes();
-      if ((rc = launch_prefill_mixer(*m, l, nb, n, l == 0 ? d_tokens + b0 * n : nullptr, w.x, Sl, w.a, s->status, st))) return rc;
+      if (m->head_proj()) {
+        if ((rc = launch_mixer_block_proj(*m, l, -1, rows, nb, n, l == 0 ? d_tokens + b0 * n : nullptr, w.x, Sl, w.a, w.q, s->status, st))) return rc;
+      } else if ((rc = launch_prefill_mixer(*m, l, nb, n, l == 0 ? d_tokens + b0 * n : nullptr, w.x, Sl, w.a, s->status, st))) return rc;
       if ((rc = launch_gemm(*m, kEpiBiasGelu, rows, F, d, w.a, m->ptr(l, SRM_T_W1), m->fptr(l, SRM_T_B1), w.H, s->status, st))) return rc;
       if ((rc = launch_gemm(*m, kEpiBiasResidual, rows, d, F, w.H, m->ptr(l, SRM_T_W2), m->fptr(l, SRM_T_B2), w.x, s->status, st))) return rc;
     }
@@ -872,7 +948,7 @@ int srm_k_gemm(srm_model* m, int32_t epilogue, int64_t M, int64_t N, int64_t K, 
   if (m == nullptr || M < 0 || N < 1 || K < 1) return SRM_ERR_INVALID_ARG;
   if (M == 0) return SRM_OK;
   if (d_A == nullptr || d_W == nullptr || d_out == nullptr) return SRM_ERR_INVALID_ARG;
-  if (epilogue < 0 || epilogue > 2 || (epilogue != kEpiPlain && d_bias == nullptr)) return SRM_ERR_INVALID_ARG;
+  if (epilogue < 0 || epilogue > 2 || (epilogue == kEpiBiasGelu && d_bias == nullptr)) return SRM_ERR_INVALID_ARG;
   if (K % 64 || N % 8) return SRM_ERR_UNSUPPORTED;
   if (!aligned(d_A, 16) || !aligned(d_W, 16) || !aligned(d_out, 16) || !aligned(d_bias, 16)) return SRM_ERR_ALIGNMENT;
   return launch_gemm(*m, epilogue, M, N, K, d_A, d_W, d_bias, d_out, d_status, static_cast<cudaStream_t>(stream));
