@@ -204,6 +204,30 @@ def cpu_baseline(shape, W, workload, w, seconds_target=12.0):
             "sample": f"{sample} samples x {steps} decode steps of the same model (numpy fp64 oracle, {dt:.1f} s)"}
 
 
+# ---- multi-GPU: independent replicas, no collective in the step -------------------------------
+def rank_plan(rank: int, world: int, B: int) -> dict:
+    """What differs between the replicas: each rank owns B samples of the whole job, global sample
+    indices [rank*B, (rank+1)*B) (they key the Philox draws), and runs the same step on its own GPU."""
+    return {"sample_idx_base": rank * B, "first_sample": rank * B, "last_sample": (rank + 1) * B - 1,
+            "total_samples": world * B}
+
+
+def max_over_ranks(ms: float, world: int, device=None) -> float:
+    """Device-timed duration of the slowest rank (MAX all-reduce; identity for one rank)."""
+    if world == 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.item()
+
+
+def whole_job_value(world: int, B: int, steps: int, ms_max: float) -> float:
+    """tokens/s of the whole job: every rank generated B tokens per step, the job took the slowest rank's time."""
+    return world * B * steps / (ms_max / 1e3)
+
+
 # ----------------------------------------------------------------------------------------------
 def run_ours(args):
     import numpy as np
@@ -235,7 +259,8 @@ def run_ours(args):
     W = I.make_weights(shape)
     model = P.SRM(shape, W, device=dev, state_dtype=args.state_dtype)
     samp = P.Sampling("greedy") if w["sampling"] == "greedy" else \
-        P.Sampling("topk", w["top_k"], w["temperature"], seed=shape.seed, sample_idx_base=rank * B)
+        P.Sampling("topk", w["top_k"], w["temperature"], seed=shape.seed,
+                   sample_idx_base=rank_plan(rank, world, B)["sample_idx_base"])
     prompts = torch.from_numpy(I.make_prompts(args.workload, batch=B)).to(dev)
     chunk = min(B, args.chunk)
     st = model.new_state(B)
@@ -285,12 +310,10 @@ def run_ours(args):
         time.sleep(0.15)                     # let the sample that covers the end of the region arrive
     t_ms = e0.elapsed_time(e1)
     launches = model.kernel_launches() - launches0
-    t = torch.tensor([t_ms], dtype=torch.float64, device=dev)
     if world > 1:
         dist.barrier()
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    t_ms_max = t.item()
-    value = world * B * args.steps / (t_ms_max / 1e3)
+    t_ms_max = max_over_ranks(t_ms, world, dev)
+    value = whole_job_value(world, B, args.steps, t_ms_max)
 
     # ---- per-kernel durations, CUDA events on the launching stream, same workload ----
     model.profile_reset()
@@ -337,11 +360,9 @@ def run_ours(args):
         h_in.copy_(h_out)
     e1.record()
     torch.cuda.synchronize()
-    te = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
     if world > 1:
         dist.barrier()
-        dist.all_reduce(te, op=dist.ReduceOp.MAX)
-    e2e_value = world * B * args.steps / (te.item() / 1e3)
+    e2e_value = whole_job_value(world, B, args.steps, max_over_ranks(e0.elapsed_time(e1), world, dev))
     status = st.status()
 
     if rank == 0:
