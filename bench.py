@@ -280,8 +280,13 @@ def run_ours(args):
     if args.no_prefill:                      # profiling aid: decode cost does not depend on the cache contents
         st.pos = n
     else:
+        replicated = w["prompts"] == "replicated" and B % w["n_prompts"] == 0 and not args.no_prompt_dedup
         e0.record()
-        model.prefill(st, prompts, samp, ws)
+        if replicated:                       # each distinct prompt runs once, its cache is copied to its replicas
+            reps = B // w["n_prompts"]
+            model.prefill_replicated(st, prompts[::reps].contiguous(), reps, samp, ws)
+        else:
+            model.prefill(st, prompts, samp, ws)
         e1.record()
         torch.cuda.synchronize()
         prefill_ms = e0.elapsed_time(e1)
@@ -396,7 +401,8 @@ def run_ours(args):
                               "peaks": f"{peak_src}: {peak_tf} TFLOP/s sustained bf16, {peaks['hbm_gbs']} GB/s HBM"},
             "kernels": kernels,
             "prefill": None if prefill_ms is None else
-            {"ms": round(prefill_ms, 2), "prompt_tokens_per_s": round(B * n / (prefill_ms / 1e3), 1)},
+            {"ms": round(prefill_ms, 2), "prompt_tokens_per_s": round(B * n / (prefill_ms / 1e3), 1),
+             "distinct_prompts": w.get("n_prompts") if (w["prompts"] == "replicated" and not args.no_prompt_dedup) else B},
             "state_bytes_per_sample": L * d * sbytes,
             "max_concurrent_samples": max_conc,
             "device_status": status,
@@ -476,6 +482,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--head-proj", action="store_true",
                     help="token mixer with head projections (Eq. 10): adds W_in, W_out [d, d] per layer")
+    ap.add_argument("--no-prompt-dedup", action="store_true",
+                    help="rl workload: prefill all 16384 rows instead of the 16 distinct prompts")
     ap.add_argument("--no-prefill", action="store_true",
                     help="skip the prefill (cache stays zero, pos = prompt length): keeps profiler captures short")
     ap.add_argument("--sweep", action="store_true")

@@ -168,6 +168,18 @@ int srm_prefill(srm_model* m, srm_state* s, const int32_t* d_tokens, int32_t n,
                 const srm_sampling* sampling, int32_t* d_first_tok, float* d_logits_last,
                 void* d_ws, size_t ws_bytes, void* stream);
 
+/* Prefill for replicated prompts [Inference Compute Scaling: many samples per question, as in the
+ * GRPO rollouts]: d_tokens holds n_prompts DISTINCT prompts [n_prompts, n]; the state has
+ * B = n_prompts * replicas samples and sample p * replicas + j is replica j of prompt p. Every prompt runs
+ * through the sequence-parallel form once, its cache is copied to the rows of its replicas, and each
+ * replica selects its own first token from the prompt's last-position logits (Philox sample index
+ * sample_idx_base + state row, step 0), which is what srm_prefill on the replicated token matrix gives, bit
+ * for bit. d_first_tok int32[B] and d_logits_last float[n_prompts, V] may be NULL. Needs, on top of the
+ * prefill workspace, L * d * state element bytes (rounded up to 256) per prompt of a pass at the end of d_ws. */
+int srm_prefill_replicated(srm_model* m, srm_state* s, const int32_t* d_tokens, int32_t n_prompts, int32_t n,
+                           int32_t replicas, const srm_sampling* sampling, int32_t* d_first_tok,
+                           float* d_logits_last, void* d_ws, size_t ws_bytes, void* stream);
+
 /* One recurrent decode step [Eq. 2, Eq. 3]: consumes d_tok_in[B] (NULL: the token selected
  * by the previous call) at position pos, updates the cache, pos += 1, and selects the next
  * token with Philox step `step`. d_tok_out int32[B] and d_logits_out float[B, V] may be NULL. */

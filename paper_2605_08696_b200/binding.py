@@ -80,6 +80,7 @@ SYMBOLS = {
     "srm_state_last_token_ptr": (_P, [_P]),
     "srm_status": (C.c_int, [_P, _P, C.POINTER(C.c_uint32)]),
     "srm_prefill": (C.c_int, [_P, _P, _P, _I32, C.POINTER(_Sampling), _P, _P, _P, _SZ, _P]),
+    "srm_prefill_replicated": (C.c_int, [_P, _P, _P, _I32, _I32, _I32, C.POINTER(_Sampling), _P, _P, _P, _SZ, _P]),
     "srm_decode_step": (C.c_int, [_P, _P, _P, C.POINTER(_Sampling), _I32, _P, _P, _P, _SZ, _P]),
     "srm_generate": (C.c_int, [_P, _P, _I32, _I32, C.POINTER(_Sampling), _P, _I64, _P, _SZ, _P]),
     "srm_decode_step_host": (C.c_int, [_P, _P, _P, C.POINTER(_Sampling), _I32, _P, _P, _SZ, _P]),
@@ -279,6 +280,19 @@ class SRM:
         s = sampling.c()
         _check(_lib().srm_prefill(self.handle, state.handle, _ptr(tokens), n, C.byref(s), _ptr(first), _ptr(logits),
                                   _ptr(ws), ws.numel(), _stream()), "srm_prefill")
+        return (first, logits) if want_logits else first
+
+    def prefill_replicated(self, state: SRMState, tokens: torch.Tensor, replicas: int, sampling: Sampling,
+                           ws: torch.Tensor, want_logits: bool = False):
+        """tokens [P, n] distinct prompts; state.B == P * replicas; row p * replicas + j is replica j of prompt p."""
+        P_, n = tokens.shape
+        assert P_ * replicas == state.B and tokens.dtype == torch.int32
+        first = torch.empty(state.B, dtype=torch.int32, device=self.device)
+        logits = torch.empty(P_, self.cfg.vocab, dtype=torch.float32, device=self.device) if want_logits else None
+        s = sampling.c()
+        _check(_lib().srm_prefill_replicated(self.handle, state.handle, _ptr(tokens), P_, n, replicas, C.byref(s),
+                                             _ptr(first), _ptr(logits), _ptr(ws), ws.numel(), _stream()),
+               "srm_prefill_replicated")
         return (first, logits) if want_logits else first
 
     def decode_step(self, state: SRMState, tok_in, sampling: Sampling, step: int, ws: torch.Tensor,

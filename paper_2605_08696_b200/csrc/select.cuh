@@ -17,6 +17,7 @@ struct SelectOut {
   int32_t* store;       // token store base or nullptr: store[row * store_stride + store_col]
   int64_t store_stride;
   int64_t store_col;
+  int64_t row_div;      // output row r reads logits row r / row_div (replicas of one prompt share a row); >= 1
 };
 
 __device__ __forceinline__ void write_token(const SelectOut& o, int64_t row, int tok) {
@@ -36,7 +37,7 @@ select_greedy_kernel(const float* __restrict__ logits, int64_t R, int V, SelectO
   pdl_wait();
   const int64_t row = blockIdx.x;
   if (row >= R) return;
-  const float* lr = logits + row * (int64_t)V;
+  const float* lr = logits + (row / out.row_div) * (int64_t)V;
   float bv = -INFINITY;
   int bi = 0x7fffffff;
   bool bad = false;
@@ -149,7 +150,7 @@ select_topk_kernel(const float* __restrict__ logits, int64_t R, int V, int k, fl
 
   const int64_t row = blockIdx.x;
   if (row >= R) return;
-  const float* lr = logits + row * (int64_t)V;
+  const float* lr = logits + (row / out.row_div) * (int64_t)V;
   const int tid = threadIdx.x;
   bool bad = false;
   if (ROW_IN_SMEM) {
@@ -290,7 +291,7 @@ select_topk_stream_kernel(const float* __restrict__ logits, int64_t R, int V, in
 
   const int64_t row = blockIdx.x;
   if (row >= R) return;
-  const float* lr = logits + row * (int64_t)V;
+  const float* lr = logits + (row / out.row_div) * (int64_t)V;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
   // ---- pass 1: moments ----
@@ -385,6 +386,18 @@ select_topk_stream_kernel(const float* __restrict__ logits, int64_t R, int V, in
     }
     write_token(out, row, (int)(uint32_t)(cand[pick] & 0xffffffffull));
   }
+}
+
+// Cache rows of `replicas` consecutive samples = the row of their prompt:
+// dst[(p0 + p) * replicas + j, :] = src[p, :] for p < np, j < replicas (16-byte vectors; one layer).
+__global__ void __launch_bounds__(256)
+broadcast_rows_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, int64_t np, int64_t replicas, int64_t vec_per_row) {
+  pdl_trigger();
+  pdl_wait();
+  const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  if (i >= np * replicas * vec_per_row) return;
+  const int64_t row = i / vec_per_row, v = i % vec_per_row;
+  dst[i] = __ldg(src + (row / replicas) * vec_per_row + v);
 }
 
 }  // namespace srm

@@ -634,7 +634,7 @@ int decode_step_impl(srm_model* m, srm_state* s, const int32_t* d_tok_in, const 
   if (rows < 1) return SRM_ERR_BUFFER_TOO_SMALL;
   const DecodeWs w = carve_decode(*m, d_ws, rows);
   const int32_t* tok_in = d_tok_in != nullptr ? d_tok_in : s->last_tok;
-  SelectOut out{s->last_tok, d_tok_out, d_store, store_stride, store_col};
+  SelectOut out{s->last_tok, d_tok_out, d_store, store_stride, store_col, 1};
   for (int64_t b0 = 0; b0 < s->B; b0 += rows) {
     const int64_t R = (s->B - b0 < rows) ? s->B - b0 : rows;
     if ((rc = decode_chunk(*m, *s, b0, R, tok_in, *samp, step, out, d_logits_out, w, st))) return rc;
@@ -807,45 +807,95 @@ int srm_status(srm_state* s, void* stream, uint32_t* flags) {
   return f ? SRM_ERR_DEVICE_STATUS : SRM_OK;
 }
 
-int srm_prefill(srm_model* m, srm_state* s, const int32_t* d_tokens, int32_t n, const srm_sampling* samp,
-                int32_t* d_first_tok, float* d_logits_last, void* d_ws, size_t ws_bytes, void* stream) {
+}  // extern "C"
+
+namespace {
+
+// Sequence-parallel prefill of `P` prompts, each standing for `replicas` consecutive samples of the state
+// (replicas == 1: the plain prefill). A prompt is run once; with replicas > 1 its per-layer cache goes to a
+// staging area at the end of the workspace and is then copied to the rows of its replicas, and every replica
+// selects its own first token from the prompt's last-position logits.
+int prefill_impl(srm_model* m, srm_state* s, const int32_t* d_tokens, int64_t P, int32_t n, int64_t replicas,
+                 const srm_sampling* samp, int32_t* d_first_tok, float* d_logits_last, void* d_ws, size_t ws_bytes,
+                 cudaStream_t st) {
+  const srm_config& c = m->cfg;
+  const int d = c.d_model;
+  const int64_t F = m->F();
+  const size_t row_bytes = (size_t)d * m->state_bytes();
+  const size_t stage_per_prompt = replicas > 1 ? align_up((size_t)c.n_layers * row_bytes, 256) : 0;
+  // largest number of prompts per pass whose workspace and staging both fit
+  int64_t Bp = fit_rows(ws_bytes, P, prefill_need, *m, n);
+  while (Bp >= 1 && prefill_ws_bytes(*m, Bp, n) + (size_t)Bp * stage_per_prompt > ws_bytes) --Bp;
+  if (Bp < 1) return SRM_ERR_BUFFER_TOO_SMALL;
+  const PrefillWs w = carve_prefill(*m, d_ws, Bp, n);
+  uint8_t* stage = static_cast<uint8_t*>(d_ws) + align_up(prefill_ws_bytes(*m, Bp, n), 256);
+  int rc;
+  for (int64_t p0 = 0; p0 < P; p0 += Bp) {
+    const int64_t np = (P - p0 < Bp) ? P - p0 : Bp;
+    const int64_t rows = np * n;
+    const int64_t b0 = p0 * replicas, nb = np * replicas;          // state rows of this pass
+    for (int l = 0; l < c.n_layers; ++l) {
+      uint8_t* Sl = replicas > 1 ? stage + (size_t)l * np * row_bytes
+                                 : static_cast<uint8_t*>(s->layer_ptr(l)) + (size_t)b0 * row_bytes;
+      if (m->head_proj()) {
+        if ((rc = launch_mixer_block_proj(*m, l, -1, rows, np, n, l == 0 ? d_tokens + p0 * n : nullptr, w.x, Sl, w.a, w.q, s->status, st))) return rc;
+      } else if ((rc = launch_prefill_mixer(*m, l, np, n, l == 0 ? d_tokens + p0 * n : nullptr, w.x, Sl, w.a, s->status, st))) return rc;
+      if ((rc = launch_gemm(*m, kEpiBiasGelu, rows, F, d, w.a, m->ptr(l, SRM_T_W1), m->fptr(l, SRM_T_B1), w.H, s->status, st))) return rc;
+      if ((rc = launch_gemm(*m, kEpiBiasResidual, rows, d, F, w.H, m->ptr(l, SRM_T_W2), m->fptr(l, SRM_T_B2), w.x, s->status, st))) return rc;
+      if (replicas > 1) {
+        LaunchScope scope(*m, SRM_KERNEL_PREFILL_MIXER, st);
+        const int64_t vpr = (int64_t)row_bytes / 16, total = nb * vpr;
+        uint8_t* dst = static_cast<uint8_t*>(s->layer_ptr(l)) + (size_t)b0 * row_bytes;
+        SRM_CUDA(launch_kernel(broadcast_rows_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, st,
+                               reinterpret_cast<const uint4*>(Sl), reinterpret_cast<uint4*>(dst), np, replicas, vpr));
+      }
+    }
+    // LM head on the last prompt position only; selection per state row
+    if ((rc = launch_final_norm(*m, w.x, np, n, n - 1, w.a_last, st))) return rc;
+    SelectOut o{s->last_tok + b0, d_first_tok ? d_first_tok + b0 : nullptr, nullptr, 0, 0, replicas};
+    if (replicas == 1 && can_fuse_greedy(*m, *samp, d_logits_last)) {
+      if ((rc = launch_lm_head_greedy(*m, np, w.a_last, w.logits, o, s->status, st))) return rc;
+      continue;
+    }
+    float* lg = d_logits_last != nullptr ? d_logits_last + p0 * c.vocab : w.logits;
+    if ((rc = launch_gemm(*m, kEpiPlain, np, c.vocab, d, w.a_last, m->ptr(-1, SRM_T_W_LM), nullptr, lg, s->status, st))) return rc;
+    if ((rc = launch_select(*m, nb, lg, *samp, samp->sample_idx_base + (uint64_t)b0, 0, o, s->status, st))) return rc;
+  }
+  s->pos = n;
+  return SRM_OK;
+}
+
+int prefill_check(srm_model* m, srm_state* s, const int32_t* d_tokens, int32_t n, const srm_sampling* samp,
+                  const int32_t* d_first_tok, const float* d_logits_last, const void* d_ws) {
   if (m == nullptr || s == nullptr || s->m != m || d_tokens == nullptr || d_ws == nullptr || n < 1) return SRM_ERR_INVALID_ARG;
   int rc = check_sampling(*m, samp);
   if (rc) return rc;
   if (!aligned(d_ws, 256) || !aligned(d_tokens, 4) || !aligned(d_first_tok, 4) || !aligned(d_logits_last, 16)) return SRM_ERR_ALIGNMENT;
   if (s->pos != 0) return SRM_ERR_INVALID_ARG;           // the parallel form starts from an empty cache
   if (n > m->cfg.n_ctx) return SRM_ERR_CTX_OVERFLOW;
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
-  const int64_t Bp = fit_rows(ws_bytes, s->B, prefill_need, *m, n);
-  if (Bp < 1) return SRM_ERR_BUFFER_TOO_SMALL;
-  const PrefillWs w = carve_prefill(*m, d_ws, Bp, n);
-  const srm_config& c = m->cfg;
-  const int d = c.d_model;
-  const int64_t F = m->F();
-  for (int64_t b0 = 0; b0 < s->B; b0 += Bp) {
-    const int64_t nb = (s->B - b0 < Bp) ? s->B - b0 : Bp;
-    const int64_t rows = nb * n;
-    for (int l = 0; l < c.n_layers; ++l) {
-      uint8_t* Sl = static_cast<uint8_t*>(s->layer_ptr(l)) + (size_t)b0 * d * m->state_bytes();
-      if (m->head_proj()) {
-        if ((rc = launch_mixer_block_proj(*m, l, -1, rows, nb, n, l == 0 ? d_tokens + b0 * n : nullptr, w.x, Sl, w.a, w.q, s->status, st))) return rc;
-      } else if ((rc = launch_prefill_mixer(*m, l, nb, n, l == 0 ? d_tokens + b0 * n : nullptr, w.x, Sl, w.a, s->status, st))) return rc;
-      if ((rc = launch_gemm(*m, kEpiBiasGelu, rows, F, d, w.a, m->ptr(l, SRM_T_W1), m->fptr(l, SRM_T_B1), w.H, s->status, st))) return rc;
-      if ((rc = launch_gemm(*m, kEpiBiasResidual, rows, d, F, w.H, m->ptr(l, SRM_T_W2), m->fptr(l, SRM_T_B2), w.x, s->status, st))) return rc;
-    }
-    // LM head and selection on the last prompt position only
-    if ((rc = launch_final_norm(*m, w.x, nb, n, n - 1, w.a_last, st))) return rc;
-    SelectOut o{s->last_tok + b0, d_first_tok ? d_first_tok + b0 : nullptr, nullptr, 0, 0};
-    if (can_fuse_greedy(*m, *samp, d_logits_last)) {
-      if ((rc = launch_lm_head_greedy(*m, nb, w.a_last, w.logits, o, s->status, st))) return rc;
-      continue;
-    }
-    float* lg = d_logits_last != nullptr ? d_logits_last + b0 * c.vocab : w.logits;
-    if ((rc = launch_gemm(*m, kEpiPlain, nb, c.vocab, d, w.a_last, m->ptr(-1, SRM_T_W_LM), nullptr, lg, s->status, st))) return rc;
-    if ((rc = launch_select(*m, nb, lg, *samp, samp->sample_idx_base + (uint64_t)b0, 0, o, s->status, st))) return rc;
-  }
-  s->pos = n;
   return SRM_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int srm_prefill(srm_model* m, srm_state* s, const int32_t* d_tokens, int32_t n, const srm_sampling* samp,
+                int32_t* d_first_tok, float* d_logits_last, void* d_ws, size_t ws_bytes, void* stream) {
+  int rc = prefill_check(m, s, d_tokens, n, samp, d_first_tok, d_logits_last, d_ws);
+  if (rc) return rc;
+  return prefill_impl(m, s, d_tokens, s->B, n, 1, samp, d_first_tok, d_logits_last, d_ws, ws_bytes,
+                      static_cast<cudaStream_t>(stream));
+}
+
+int srm_prefill_replicated(srm_model* m, srm_state* s, const int32_t* d_tokens, int32_t n_prompts, int32_t n,
+                           int32_t replicas, const srm_sampling* samp, int32_t* d_first_tok, float* d_logits_last,
+                           void* d_ws, size_t ws_bytes, void* stream) {
+  int rc = prefill_check(m, s, d_tokens, n, samp, d_first_tok, d_logits_last, d_ws);
+  if (rc) return rc;
+  if (n_prompts < 1 || replicas < 1 || (int64_t)n_prompts * replicas != s->B) return SRM_ERR_INVALID_ARG;
+  return prefill_impl(m, s, d_tokens, n_prompts, n, replicas, samp, d_first_tok, d_logits_last, d_ws, ws_bytes,
+                      static_cast<cudaStream_t>(stream));
 }
 
 int srm_decode_step(srm_model* m, srm_state* s, const int32_t* d_tok_in, const srm_sampling* samp, int32_t step,
@@ -962,7 +1012,7 @@ int srm_k_lm_head_greedy(srm_model* m, int64_t R, const void* d_a, void* d_part,
   if (m->cfg.dtype != SRM_DTYPE_BF16) return SRM_ERR_UNSUPPORTED;
   if (!aligned(d_a, 16) || !aligned(d_part, 16)) return SRM_ERR_ALIGNMENT;
   if (part_bytes < (size_t)tc::argmax_slots(m->cfg.vocab) * (size_t)R * 8) return SRM_ERR_BUFFER_TOO_SMALL;
-  SelectOut o{d_tok, nullptr, nullptr, 0, 0};
+  SelectOut o{d_tok, nullptr, nullptr, 0, 0, 1};
   return launch_lm_head_greedy(*m, R, d_a, d_part, o, d_status, static_cast<cudaStream_t>(stream));
 }
 
@@ -974,7 +1024,7 @@ int srm_k_select(srm_model* m, int64_t R, const float* d_logits, const srm_sampl
   int rc = check_sampling(*m, samp);
   if (rc) return rc;
   if (!aligned(d_logits, 16)) return SRM_ERR_ALIGNMENT;
-  SelectOut o{d_tok, nullptr, nullptr, 0, 0};
+  SelectOut o{d_tok, nullptr, nullptr, 0, 0, 1};
   return launch_select(*m, R, d_logits, *samp, samp->sample_idx_base, step, o, d_status, static_cast<cudaStream_t>(stream));
 }
 

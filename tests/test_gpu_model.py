@@ -192,6 +192,38 @@ def test_fused_greedy_head_equals_logits_then_selection_on_device():
     assert st_a.status() == 0 and st_b.status() == 0
 
 
+@pytest.mark.parametrize("mode", ["greedy", "topk"])
+def test_replicated_prefill_equals_prefill_of_the_replicated_prompts(mode):
+    """srm_prefill_replicated (each distinct prompt run once, cache copied to its replicas, one selection per
+    replica) leaves, bit for bit, what srm_prefill on the replicated token matrix leaves: cache, first tokens,
+    and the tokens of the following decode steps. Several passes (small workspace) included."""
+    import paper_2605_08696_b200 as P
+    shape, W, model = _build("small")
+    n_prompts, replicas, n = 5, 7, 40
+    B = n_prompts * replicas
+    base = torch.from_numpy(I.uniform_prompts(n_prompts, n, shape.vocab, seed=31)).to(DEV)
+    full = base.repeat_interleave(replicas, dim=0).contiguous()
+    samp = P.Sampling("greedy") if mode == "greedy" else P.Sampling("topk", 50, 0.8, seed=77, sample_idx_base=1000)
+    ws = model.new_workspace(B, n, prefill_samples=B + 8)
+    st_a, st_b, st_c = model.new_state(B), model.new_state(B), model.new_state(B)
+    first_a = model.prefill(st_a, full, samp, ws)
+    first_b, lg_b = model.prefill_replicated(st_b, base, replicas, samp, ws, want_logits=True)
+    ws_small = model.new_workspace(4, n, prefill_samples=3)                  # two prompts per pass at most
+    first_c = model.prefill_replicated(st_c, base, replicas, samp, ws_small)
+    assert torch.equal(first_a, first_b) and torch.equal(first_a, first_c)
+    assert torch.equal(st_a.cache(), st_b.cache()) and torch.equal(st_a.cache(), st_c.cache())
+    assert lg_b.shape == (n_prompts, shape.vocab)
+    if mode == "topk":
+        assert len(set(first_a[:replicas].tolist())) > 1                     # replicas of one prompt draw differently
+    else:
+        assert len(set(first_a[:replicas].tolist())) == 1
+    for k in range(1, 4):
+        ta = model.decode_step(st_a, None, samp, k, ws)
+        tb = model.decode_step(st_b, None, samp, k, ws)
+        assert torch.equal(ta, tb)
+    assert st_a.status() == 0 and st_b.status() == 0 and st_c.status() == 0 and st_b.pos == n + 3
+
+
 def test_resume_from_exported_cache():
     """generate(2k) == generate(k), copy the state buffer, generate(k) on the copy."""
     import paper_2605_08696_b200 as P
