@@ -281,12 +281,19 @@ def run_ours(args):
         st.pos = n
     else:
         replicated = w["prompts"] == "replicated" and B % w["n_prompts"] == 0 and not args.no_prompt_dedup
+
+        def do_prefill():
+            if replicated:                   # each distinct prompt runs once, its cache is copied to its replicas
+                reps = B // w["n_prompts"]
+                model.prefill_replicated(st, prompts[::reps].contiguous(), reps, samp, ws)
+            else:
+                model.prefill(st, prompts, samp, ws)
+
+        do_prefill()                         # untimed: first-use costs (module load, descriptor encoding)
+        st.reset()
+        torch.cuda.synchronize()
         e0.record()
-        if replicated:                       # each distinct prompt runs once, its cache is copied to its replicas
-            reps = B // w["n_prompts"]
-            model.prefill_replicated(st, prompts[::reps].contiguous(), reps, samp, ws)
-        else:
-            model.prefill(st, prompts, samp, ws)
+        do_prefill()
         e1.record()
         torch.cuda.synchronize()
         prefill_ms = e0.elapsed_time(e1)
@@ -476,7 +483,7 @@ def main():
     ap.add_argument("--workload", default="mid", choices=["tiny", "small", "mid", "rl"])
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch per GPU")
     ap.add_argument("--chunk", type=int, default=8192, help="samples per decode pass (workspace size)")
-    ap.add_argument("--prefill-rows", type=int, default=65536, help="prompt rows per prefill pass")
+    ap.add_argument("--prefill-rows", type=int, default=262144, help="prompt rows per prefill pass")
     ap.add_argument("--state-dtype", default="fp32", choices=["fp32", "bf16"])
     ap.add_argument("--ref-samples", type=int, default=32)
     ap.add_argument("--no-cpu-baseline", action="store_true")
