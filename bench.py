@@ -257,7 +257,8 @@ def run_ours(args):
     peaks, peak_src = measured_peaks()
 
     W = I.make_weights(shape)
-    model = P.SRM(shape, W, device=dev, state_dtype=args.state_dtype)
+    model = P.SRM(shape, W, device=dev, state_dtype=args.state_dtype,
+                  flags={"auto": 0, "on": P.FLAG_GRAPH, "off": P.FLAG_NO_GRAPH}[args.graph])
     samp = P.Sampling("greedy") if w["sampling"] == "greedy" else \
         P.Sampling("topk", w["top_k"], w["temperature"], seed=shape.seed,
                    sample_idx_base=rank_plan(rank, world, B)["sample_idx_base"])
@@ -299,23 +300,30 @@ def run_ours(args):
         prefill_ms = e0.elapsed_time(e1)
 
     step_no = [1]
+    store = torch.empty(B, shape.n_ctx - n, dtype=torch.int32, device=dev)       # generated-token store
 
-    def one_step():
-        if st.pos >= shape.n_ctx:            # timing-only wrap: keep alpha/beta indices in range
-            st.pos = n
-        model.decode_step(st, None, samp, step_no[0], ws)
-        step_no[0] += 1
+    def run_steps(k):
+        """k decode steps through the generation loop of the library (srm_generate: launch by launch, or a
+        replayed CUDA graph for launch-bound batches); the position wraps to the end of the prompt when the
+        context is exhausted (timing only: alpha/beta indices stay in range)."""
+        while k > 0:
+            room = shape.n_ctx - st.pos
+            if room == 0:
+                st.pos = n
+                continue
+            c = min(k, room)
+            model.generate(st, c, step_no[0], samp, ws, out=store)
+            step_no[0] += c
+            k -= c
 
     with ClockSampler(local) as clk:         # nvidia-smi starts up during the warm-up steps
-        for _ in range(max(args.warmup, 3)):
-            one_step()
+        run_steps(max(args.warmup, 3))
         # ---- timed region: exactly K steps ----
         sync_all()
         launches0 = model.kernel_launches()
         clk.mark_start()
         e0.record()
-        for _ in range(args.steps):
-            one_step()
+        run_steps(args.steps)
         e1.record()
         torch.cuda.synchronize()
         clk.mark_stop()
@@ -330,8 +338,7 @@ def run_ours(args):
     # ---- per-kernel durations, CUDA events on the launching stream, same workload ----
     model.profile_reset()
     model.profile(True)
-    for _ in range(args.steps):
-        one_step()
+    run_steps(args.steps)
     torch.cuda.synchronize()
     model.profile(False)
     prof = model.profile_read()
@@ -390,7 +397,7 @@ def run_ours(args):
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if shape.dtype == "bf16" else "f32",
             "data": "synthetic",
             "config": _config_dict(args, shape, w, B, extra={
-                "state_dtype": args.state_dtype, "chunk_rows": chunk,
+                "state_dtype": args.state_dtype, "chunk_rows": chunk, "graph": args.graph,
                 "l2": f"inputs larger than L2: per-step working set (cache {L * B * d * sbytes / 1e6:.0f} MB + weights "
                       f"{model.blob.numel() / 1e6:.0f} MB + logits {chunk * V * 4 / 1e6:.0f} MB) vs 126 MB L2; no flush"}),
             "gpu_launches": int(launches),
@@ -454,20 +461,19 @@ def run_sweep(args):
             prompts = prompts.repeat((B + prompts.shape[0] - 1) // prompts.shape[0], 1)[:B].contiguous()
         model.prefill(st, prompts, g, ws)
         steps = 8 if B >= 262144 else 24
-        for _ in range(3):
-            model.decode_step(st, None, g, 1, ws)
+        store = torch.empty(B, steps, dtype=torch.int32, device=dev)
+        model.generate(st, 4, 1, g, ws, out=store)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.cuda.synchronize()
         e0.record()
-        for _ in range(steps):
-            model.decode_step(st, None, g, 1, ws)
+        model.generate(st, steps, 5, g, ws, out=store)
         e1.record()
         torch.cuda.synchronize()
         ms = e0.elapsed_time(e1) / steps
         curve.append({"batch": B, "ms_per_step": round(ms, 4), "tokens_per_s": round(B / (ms / 1e3), 1),
                       "state_bytes_per_sample": L * d * sbytes, "status": st.status()})
         print(json.dumps(curve[-1]), file=sys.stderr, flush=True)
-        del st, prompts
+        del st, prompts, store
         torch.cuda.empty_cache()
     line = {"metric": METRIC, "unit": UNIT, "n_gpus": 1, "sweep": curve, "max_concurrent_samples": max_conc,
             "state_dtype": args.state_dtype, "config": {"workload": "sweep: mid SRM, 128-token uniform prompts"}}
@@ -489,6 +495,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--head-proj", action="store_true",
                     help="token mixer with head projections (Eq. 10): adds W_in, W_out [d, d] per layer")
+    ap.add_argument("--graph", default="auto", choices=["auto", "on", "off"],
+                    help="srm_generate replays a captured step: auto = only for launch-bound (small) batches")
     ap.add_argument("--no-prompt-dedup", action="store_true",
                     help="rl workload: prefill all 16384 rows instead of the 16 distinct prompts")
     ap.add_argument("--no-prefill", action="store_true",

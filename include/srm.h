@@ -60,6 +60,9 @@ enum srm_status_bits {
 enum { SRM_DTYPE_FP32 = 0, SRM_DTYPE_BF16 = 1 };
 enum { SRM_SELECT_GREEDY = 0, SRM_SELECT_TOPK = 1 };
 enum {
+  SRM_FLAG_NO_GRAPH = 4,             /* srm_generate never replays a captured step                     */
+  SRM_FLAG_GRAPH = 8,                /* srm_generate always replays a captured step (default: only for
+                                        batches small enough to be bound by the host's launch rate)     */
   SRM_FLAG_SIMT_GEMM = 1,            /* debug: run the bf16 GEMMs on the plain SIMT kernel  */
   SRM_FLAG_HEAD_PROJ = 2             /* token mixer with head projections [Method/Architecture, Eq. 10]:
                                         q = W_in LN1(x) (W_in stacks the per-head I_g), heads of q mixed, and
@@ -187,11 +190,16 @@ int srm_decode_step(srm_model* m, srm_state* s, const int32_t* d_tok_in,
                     const srm_sampling* sampling, int32_t step, int32_t* d_tok_out,
                     float* d_logits_out, void* d_ws, size_t ws_bytes, void* stream);
 
-/* Generation loop: `steps` decode steps, each consuming the previously selected token
+/* Generation loop [Recurrent Throughput and Concurrency; the paper moved its loop inside the compiled graph
+ * to escape a per-call driver delay]: `steps` decode steps, each consuming the previously selected token
  * (the one left by srm_prefill or the previous step). Step j (0-based) writes its selection
  * to d_out[b * out_stride + j] and uses Philox step first_step + j. No host synchronisation
  * between steps. Fails with SRM_ERR_CTX_OVERFLOW before enqueuing anything if
- * pos + steps > n_ctx. */
+ * pos + steps > n_ctx. For batches small enough to be bound by the host's kernel-launch rate one step is
+ * captured once as a CUDA graph (on a stream the model owns; position, Philox step and store column live
+ * in device-side counters of the state header that a one-thread kernel advances) and replayed `steps`
+ * times on `stream`; the graph is kept and reused while state, workspace, sampling and output buffer stay
+ * the same. Results are identical to the launch-by-launch loop. */
 int srm_generate(srm_model* m, srm_state* s, int32_t steps, int32_t first_step,
                  const srm_sampling* sampling, int32_t* d_out, int64_t out_stride,
                  void* d_ws, size_t ws_bytes, void* stream);

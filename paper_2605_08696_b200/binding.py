@@ -18,6 +18,8 @@ EPI_BIAS_GELU, EPI_BIAS_RESIDUAL, EPI_PLAIN = 0, 1, 2
 DTYPE_FP32, DTYPE_BF16 = 0, 1
 FLAG_SIMT_GEMM = 1
 FLAG_HEAD_PROJ = 2
+FLAG_NO_GRAPH = 4
+FLAG_GRAPH = 8
 
 # enum srm_tensor
 T_E, T_LN1_G, T_LN1_B, T_ALPHA, T_BETA, T_LAMBDA, T_LN2_G, T_LN2_B, T_W1, T_B1, T_W2, T_B2, \
@@ -309,8 +311,10 @@ class SRM:
                  out: torch.Tensor | None = None) -> torch.Tensor:
         if out is None:
             out = torch.empty(state.B, steps, dtype=torch.int32, device=self.device)
+        assert out.dtype == torch.int32 and out.stride(1) == 1 and out.shape[1] >= steps     # rows may be strided
         s = sampling.c()
-        _check(_lib().srm_generate(self.handle, state.handle, steps, first_step, C.byref(s), _ptr(out), out.stride(0),
+        _check(_lib().srm_generate(self.handle, state.handle, steps, first_step, C.byref(s),
+                                   C.c_void_p(out.data_ptr()), out.stride(0),
                                    _ptr(ws), ws.numel(), _stream()), "srm_generate")
         return out
 

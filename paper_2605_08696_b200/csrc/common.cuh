@@ -25,6 +25,13 @@ __device__ __forceinline__ void raise_status(uint32_t* status, uint32_t bit) {
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// Device-side step counters (words 1..3 of the state header; word 0 is the status word). When a decode
+// step is replayed from a CUDA graph its kernel arguments are frozen, so the values that change from step
+// to step are read from here instead, and a one-thread kernel advances them at the end of every step.
+constexpr int kCtrPos = 1;     // absolute position of the token being consumed
+constexpr int kCtrStep = 2;    // Philox step of the selection
+constexpr int kCtrCol = 3;     // column of the token store the selection writes
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);

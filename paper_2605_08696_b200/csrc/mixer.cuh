@@ -23,6 +23,7 @@ struct MixerParams {
   int d, h, n_ctx, t, vocab;
   float eps;
   uint32_t* status;
+  const int32_t* ctr;    // device-side step counters, or nullptr: then `t` above is the position
 };
 
 constexpr int kMixerWarps = 4;
@@ -82,6 +83,7 @@ __global__ void __launch_bounds__(kMixerWarps * 32) mixer_step_kernel(const Mixe
   const int d = p.d;
   const int dh = d / p.h;
   const int h_row = p.h >> 1;
+  const int t = p.ctr != nullptr ? p.ctr[kCtrPos] : p.t;
 
   float4 v[NV];
   if (p.tok != nullptr) {
@@ -116,7 +118,7 @@ __global__ void __launch_bounds__(kMixerWarps * 32) mixer_step_kernel(const Mixe
   float mean, rstd;
   row_stats<NV>(v, lane, d, p.eps, mean, rstd);
 
-  const float* beta_t = p.beta + (int64_t)p.t * d;
+  const float* beta_t = p.beta + (int64_t)t * d;
   float* xr = p.x + row * d;
 #pragma unroll
   for (int i = 0; i < NV; ++i) {
@@ -124,7 +126,7 @@ __global__ void __launch_bounds__(kMixerWarps * 32) mixer_step_kernel(const Mixe
     if (c < d) {
       const float4 z = norm4(v[i], mean, rstd, ldg4(p.ln1_g + c), ldg4(p.ln1_b + c));
       const int g = c / dh;
-      const float al = __ldg(p.alpha + (int64_t)g * p.n_ctx + p.t);
+      const float al = __ldg(p.alpha + (int64_t)g * p.n_ctx + t);
       const float lm = __ldg(p.lam + g);
       const float4 bt = ldg4(beta_t + c);
       float4 y, sn;

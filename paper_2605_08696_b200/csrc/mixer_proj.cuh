@@ -21,6 +21,7 @@ struct MixProjParams {
   int d, h, n_ctx;
   int t;                 // decode: position
   int n;                 // prefill: prompt length
+  const int32_t* ctr;    // decode: device-side step counters, or nullptr: then `t` is the position
 };
 
 constexpr int kMixProjThreads = 256;
@@ -57,8 +58,9 @@ __global__ void __launch_bounds__(kMixProjThreads) mixer_proj_step_kernel(const 
   const int64_t r = vec / vpr;
   const int c = (int)(vec % vpr) * 4;
   const int g = c / (p.d / p.h);
-  const float al = __ldg(p.alpha + (int64_t)g * p.n_ctx + p.t), lm = __ldg(p.lam + g);
-  const float4 bt = ldg4(p.beta + (int64_t)p.t * p.d + c);
+  const int t = p.ctr != nullptr ? p.ctr[kCtrPos] : p.t;
+  const float al = __ldg(p.alpha + (int64_t)g * p.n_ctx + t), lm = __ldg(p.lam + g);
+  const float4 bt = ldg4(p.beta + (int64_t)t * p.d + c);
   const float4 q = ld4(p.q + r * p.d + c);
   ST* Sp = reinterpret_cast<ST*>(p.S) + r * p.d + c;
   const float4 s = ld4(Sp);

@@ -58,9 +58,10 @@ __global__ void __launch_bounds__(kStreamMaxWarps * 32, 1) mixer_stream_kernel(c
   uint8_t* slots = sm + mixer_stream_param_bytes(d);
   uint64_t* bars = reinterpret_cast<uint64_t*>(slots + (size_t)W * 2 * slot_bytes);
 
-  // ---- parameters of this layer and position: constant data, fetched ahead of the dependency wait ----
-  {
-    const float* beta_t = p.beta + (int64_t)p.t * d;
+  // ---- parameters of this layer and position: constant data, fetched ahead of the dependency wait
+  //      (unless the position comes from the device-side counter, which the previous step advanced) ----
+  auto stage_params = [&](int t) {
+    const float* beta_t = p.beta + (int64_t)t * d;
     for (int i = threadIdx.x * 4; i < d; i += blockDim.x * 4) {
       st4(prm + i, ldg4(p.ln1_g + i));
       st4(prm + d + i, ldg4(p.ln1_b + i));
@@ -69,14 +70,19 @@ __global__ void __launch_bounds__(kStreamMaxWarps * 32, 1) mixer_stream_kernel(c
       st4(prm + 4 * d + i, ldg4(p.ln2_b + i));
     }
     if (threadIdx.x < p.h) {
-      heads[threadIdx.x] = __ldg(p.alpha + (int64_t)threadIdx.x * p.n_ctx + p.t);
+      heads[threadIdx.x] = __ldg(p.alpha + (int64_t)threadIdx.x * p.n_ctx + t);
       heads[8 + threadIdx.x] = __ldg(p.lam + threadIdx.x);
     }
-    if (threadIdx.x < 2 * W) tc::mbar_init(&bars[threadIdx.x], 1);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
+  };
+  if (p.ctr == nullptr) stage_params(p.t);
+  if (threadIdx.x < 2 * W) tc::mbar_init(&bars[threadIdx.x], 1);
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   __syncthreads();
   pdl_wait();
+  if (p.ctr != nullptr) {
+    stage_params(p.ctr[kCtrPos]);
+    __syncthreads();
+  }
 
   // ---- row schedule: CTA c owns rows c, c + G, c + 2G, ...; its i-th row goes to warp i % W ----
   const int64_t G = gridDim.x;

@@ -18,12 +18,13 @@ struct SelectOut {
   int64_t store_stride;
   int64_t store_col;
   int64_t row_div;      // output row r reads logits row r / row_div (replicas of one prompt share a row); >= 1
+  const int32_t* ctr;   // device-side step counters (store column, Philox step), or nullptr: host values apply
 };
 
 __device__ __forceinline__ void write_token(const SelectOut& o, int64_t row, int tok) {
   o.last_tok[row] = tok;
   if (o.tok_out != nullptr) o.tok_out[row] = tok;
-  if (o.store != nullptr) o.store[row * o.store_stride + o.store_col] = tok;
+  if (o.store != nullptr) o.store[row * o.store_stride + (o.ctr != nullptr ? (int64_t)o.ctr[kCtrCol] : o.store_col)] = tok;
 }
 
 // ---- greedy -------------------------------------------------------------------------------
@@ -252,7 +253,7 @@ select_topk_kernel(const float* __restrict__ logits, int64_t R, int V, int k, fl
       cdf[i] = c;
     }
     const uint64_t sidx = sample_base + (uint64_t)row;
-    const uint32_t r = philox4x32_10_word0((uint32_t)sidx, (uint32_t)step, 0u, 0u, (uint32_t)seed,
+    const uint32_t r = philox4x32_10_word0((uint32_t)sidx, (uint32_t)(out.ctr != nullptr ? out.ctr[kCtrStep] : step), 0u, 0u, (uint32_t)seed,
                                            (uint32_t)(seed >> 32));
     const float u = (float)(r >> 8) * (1.0f / 16777216.0f);
     const float target = u * c;
@@ -376,7 +377,7 @@ select_topk_stream_kernel(const float* __restrict__ logits, int64_t R, int V, in
       cdf[i] = acc;
     }
     const uint64_t sidx = sample_base + (uint64_t)row;
-    const uint32_t r = philox4x32_10_word0((uint32_t)sidx, (uint32_t)step, 0u, 0u, (uint32_t)seed,
+    const uint32_t r = philox4x32_10_word0((uint32_t)sidx, (uint32_t)(out.ctr != nullptr ? out.ctr[kCtrStep] : step), 0u, 0u, (uint32_t)seed,
                                            (uint32_t)(seed >> 32));
     const float u = (float)(r >> 8) * (1.0f / 16777216.0f);
     const float target = u * acc;
@@ -398,6 +399,18 @@ broadcast_rows_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, in
   if (i >= np * replicas * vec_per_row) return;
   const int64_t row = i / vec_per_row, v = i % vec_per_row;
   dst[i] = __ldg(src + (row / replicas) * vec_per_row + v);
+}
+
+// Step counters in the state header: set before a replayed generation loop, advanced after every step.
+__global__ void set_counters_kernel(int32_t* hdr, int pos, int step, int col) {
+  pdl_trigger();
+  pdl_wait();
+  hdr[kCtrPos] = pos; hdr[kCtrStep] = step; hdr[kCtrCol] = col;
+}
+__global__ void advance_counters_kernel(int32_t* hdr) {
+  pdl_trigger();
+  pdl_wait();
+  hdr[kCtrPos] += 1; hdr[kCtrStep] += 1; hdr[kCtrCol] += 1;
 }
 
 }  // namespace srm

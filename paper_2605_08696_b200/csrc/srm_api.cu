@@ -160,6 +160,20 @@ struct srm_model {
   bool tc_ready = false;                 // smem attribute set for the tensor-core kernels
   int tc_clusters = 0;                   // CTA pairs of the tensor-core kernel that are resident at once
   std::vector<TmapCacheEntry> tmaps;     // weight and activation descriptors, built on first use
+  // One decode step captured as a CUDA graph for srm_generate (launch-bound batches): the stream it is
+  // captured on, the instantiated graph, and what it was captured for.
+  cudaStream_t cap_stream = nullptr;
+  cudaGraphExec_t step_exec = nullptr;
+  uint64_t step_launches = 0;            // kernels in the captured step
+  struct StepKey {
+    const srm_state* s = nullptr; const void* ws = nullptr; size_t ws_bytes = 0; const int32_t* out = nullptr;
+    int64_t out_stride = 0; srm_sampling samp = {};
+    bool operator==(const StepKey& o) const {
+      return s == o.s && ws == o.ws && ws_bytes == o.ws_bytes && out == o.out && out_stride == o.out_stride &&
+             samp.mode == o.samp.mode && samp.top_k == o.samp.top_k && samp.temperature == o.samp.temperature &&
+             samp.seed == o.samp.seed && samp.sample_idx_base == o.samp.sample_idx_base;
+    }
+  } step_key;
   bool profiling = false;                // bracket every launch with CUDA events on its stream
   std::vector<ProfRecord> prof;          // open records, folded into the totals by srm_profile_read
   std::vector<cudaEvent_t> event_pool;
@@ -340,7 +354,7 @@ int launch_mixer_nv(const MixerParams& p, int num_sms, cudaStream_t st) {
 }
 
 int launch_mixer(const srm_model& m, int layer, int t, int64_t R, const int32_t* tok, float* x, void* S, void* a,
-                 uint32_t* status, cudaStream_t st) {
+                 uint32_t* status, cudaStream_t st, const int32_t* ctr = nullptr) {
   if (R <= 0) return SRM_OK;
   LaunchScope scope(m, SRM_KERNEL_MIXER, st);
   MixerParams p;
@@ -349,7 +363,7 @@ int launch_mixer(const srm_model& m, int layer, int t, int64_t R, const int32_t*
   p.ln2_g = m.fptr(layer, SRM_T_LN2_G); p.ln2_b = m.fptr(layer, SRM_T_LN2_B);
   p.alpha = m.fptr(layer, SRM_T_ALPHA); p.beta = m.fptr(layer, SRM_T_BETA); p.lam = m.fptr(layer, SRM_T_LAMBDA);
   p.R = R; p.d = m.cfg.d_model; p.h = m.cfg.n_heads; p.n_ctx = m.cfg.n_ctx; p.t = t; p.vocab = m.cfg.vocab;
-  p.eps = m.cfg.ln_eps; p.status = status;
+  p.eps = m.cfg.ln_eps; p.status = status; p.ctr = ctr;
   const bool wb = m.cfg.dtype == SRM_DTYPE_BF16, sb = m.cfg.state_dtype == SRM_DTYPE_BF16;
   if (wb && sb) return launch_mixer_nv<bf16, bf16>(p, m.num_sms, st);
   if (wb) return launch_mixer_nv<bf16, float>(p, m.num_sms, st);
@@ -561,7 +575,8 @@ int launch_mix_proj_t(bool prefill, const MixProjParams& p, int64_t vecs, cudaSt
 }
 
 int launch_mixer_block_proj(srm_model& m, int layer, int t, int64_t rows, int64_t samples, int n, const int32_t* tok,
-                            float* x, void* S, void* a, float* q, uint32_t* status, cudaStream_t st) {
+                            float* x, void* S, void* a, float* q, uint32_t* status, cudaStream_t st,
+                            const int32_t* ctr = nullptr) {
   if (rows <= 0) return SRM_OK;
   const srm_config& c = m.cfg;
   const int d = c.d_model;
@@ -584,6 +599,7 @@ int launch_mixer_block_proj(srm_model& m, int layer, int t, int64_t rows, int64_
     p.q = q; p.S = S; p.y = a;
     p.alpha = m.fptr(layer, SRM_T_ALPHA); p.beta = m.fptr(layer, SRM_T_BETA); p.lam = m.fptr(layer, SRM_T_LAMBDA);
     p.R = prefill ? samples : rows; p.d = d; p.h = c.n_heads; p.n_ctx = c.n_ctx; p.t = prefill ? 0 : t; p.n = n;
+    p.ctr = prefill ? nullptr : ctr;
     const int64_t vecs = p.R * (d / 4);
     if (wb && sb) rc = launch_mix_proj_t<bf16, bf16>(prefill, p, vecs, st);
     else if (wb) rc = launch_mix_proj_t<bf16, float>(prefill, p, vecs, st);
@@ -597,7 +613,8 @@ int launch_mixer_block_proj(srm_model& m, int layer, int t, int64_t rows, int64_
 
 // One decode step for rows [b0, b0 + R) of the state.
 int decode_chunk(srm_model& m, srm_state& s, int64_t b0, int64_t R, const int32_t* tok_in, const srm_sampling& samp,
-                 int step, const SelectOut& out_all, float* logits_out, const DecodeWs& w, cudaStream_t st) {
+                 int step, const SelectOut& out_all, float* logits_out, const DecodeWs& w, cudaStream_t st,
+                 const int32_t* ctr) {
   const srm_config& c = m.cfg;
   const int d = c.d_model;
   const int64_t F = m.F();
@@ -606,8 +623,8 @@ int decode_chunk(srm_model& m, srm_state& s, int64_t b0, int64_t R, const int32_
   for (int l = 0; l < c.n_layers; ++l) {
     uint8_t* Sl = static_cast<uint8_t*>(s.layer_ptr(l)) + (size_t)b0 * d * m.state_bytes();
     if (m.head_proj()) {
-      if ((rc = launch_mixer_block_proj(m, l, t, R, R, 1, l == 0 ? tok_in + b0 : nullptr, w.x, Sl, w.a, w.q, s.status, st))) return rc;
-    } else if ((rc = launch_mixer(m, l, t, R, l == 0 ? tok_in + b0 : nullptr, w.x, Sl, w.a, s.status, st))) return rc;
+      if ((rc = launch_mixer_block_proj(m, l, t, R, R, 1, l == 0 ? tok_in + b0 : nullptr, w.x, Sl, w.a, w.q, s.status, st, ctr))) return rc;
+    } else if ((rc = launch_mixer(m, l, t, R, l == 0 ? tok_in + b0 : nullptr, w.x, Sl, w.a, s.status, st, ctr))) return rc;
     if ((rc = launch_gemm(m, kEpiBiasGelu, R, F, d, w.a, m.ptr(l, SRM_T_W1), m.fptr(l, SRM_T_B1), w.H, s.status, st))) return rc;
     if ((rc = launch_gemm(m, kEpiBiasResidual, R, d, F, w.H, m.ptr(l, SRM_T_W2), m.fptr(l, SRM_T_B2), w.x, s.status, st))) return rc;
   }
@@ -622,9 +639,10 @@ int decode_chunk(srm_model& m, srm_state& s, int64_t b0, int64_t R, const int32_
   return launch_select(m, R, lg, samp, samp.sample_idx_base + (uint64_t)b0, step, o, s.status, st);
 }
 
+// `ctr` non-null: position, Philox step and store column come from the device-side counters (graph replay).
 int decode_step_impl(srm_model* m, srm_state* s, const int32_t* d_tok_in, const srm_sampling* samp, int step,
                      int32_t* d_tok_out, int32_t* d_store, int64_t store_stride, int64_t store_col,
-                     float* d_logits_out, void* d_ws, size_t ws_bytes, cudaStream_t st) {
+                     float* d_logits_out, void* d_ws, size_t ws_bytes, cudaStream_t st, const int32_t* ctr = nullptr) {
   if (m == nullptr || s == nullptr || s->m != m || d_ws == nullptr) return SRM_ERR_INVALID_ARG;
   int rc = check_sampling(*m, samp);
   if (rc) return rc;
@@ -634,10 +652,10 @@ int decode_step_impl(srm_model* m, srm_state* s, const int32_t* d_tok_in, const 
   if (rows < 1) return SRM_ERR_BUFFER_TOO_SMALL;
   const DecodeWs w = carve_decode(*m, d_ws, rows);
   const int32_t* tok_in = d_tok_in != nullptr ? d_tok_in : s->last_tok;
-  SelectOut out{s->last_tok, d_tok_out, d_store, store_stride, store_col, 1};
+  SelectOut out{s->last_tok, d_tok_out, d_store, store_stride, store_col, 1, ctr};
   for (int64_t b0 = 0; b0 < s->B; b0 += rows) {
     const int64_t R = (s->B - b0 < rows) ? s->B - b0 : rows;
-    if ((rc = decode_chunk(*m, *s, b0, R, tok_in, *samp, step, out, d_logits_out, w, st))) return rc;
+    if ((rc = decode_chunk(*m, *s, b0, R, tok_in, *samp, step, out, d_logits_out, w, st, ctr))) return rc;
   }
   s->pos += 1;
   return SRM_OK;
@@ -710,6 +728,8 @@ int srm_create(const srm_config* cfg, const void* d_weights, size_t nbytes, srm_
 
 int srm_destroy(srm_model* m) {
   if (m != nullptr) {
+    if (m->step_exec != nullptr) cudaGraphExecDestroy(m->step_exec);
+    if (m->cap_stream != nullptr) cudaStreamDestroy(m->cap_stream);
     for (auto& r : m->prof) { cudaEventDestroy(r.start); cudaEventDestroy(r.stop); }
     for (auto& e : m->event_pool) cudaEventDestroy(e);
   }
@@ -770,6 +790,11 @@ int srm_state_create(srm_model* m, int64_t B, void* d_state, size_t nbytes, void
 }
 
 int srm_state_destroy(srm_state* s) {
+  if (s != nullptr && s->m != nullptr && s->m->step_key.s == s && s->m->step_exec != nullptr) {
+    cudaGraphExecDestroy(s->m->step_exec);        // the captured step refers to this state's buffers
+    s->m->step_exec = nullptr;
+    s->m->step_key = srm_model::StepKey();
+  }
   delete s;
   return SRM_OK;
 }
@@ -904,13 +929,81 @@ int srm_decode_step(srm_model* m, srm_state* s, const int32_t* d_tok_in, const s
                           static_cast<cudaStream_t>(stream));
 }
 
+}  // extern "C"
+
+namespace {
+
+// Whether srm_generate replays a captured step: worth it when the step is bound by the host's launch rate
+// (about 50 kernels of a few microseconds each), i.e. for small batches.
+bool use_step_graph(const srm_model& m, const srm_state& s, int steps) {
+  if (m.profiling || (m.cfg.flags & SRM_FLAG_NO_GRAPH) || steps < 4) return false;
+  if (m.cfg.flags & SRM_FLAG_GRAPH) return true;
+  return s.B * (int64_t)m.cfg.d_model <= (int64_t)1 << 21;
+}
+
+// Captures one decode step (all its kernels, driven by the device-side counters, plus the kernel that
+// advances them) on the model's own stream and instantiates it; reuses the previous graph when nothing it
+// was captured for has changed. Nothing is executed here.
+int prepare_step_graph(srm_model* m, srm_state* s, const srm_sampling* samp, int32_t* d_out, int64_t out_stride,
+                       void* d_ws, size_t ws_bytes) {
+  srm_model::StepKey key;
+  key.s = s; key.ws = d_ws; key.ws_bytes = ws_bytes; key.out = d_out; key.out_stride = out_stride; key.samp = *samp;
+  if (m->step_exec != nullptr && m->step_key == key) return SRM_OK;
+  if (m->step_exec != nullptr) { cudaGraphExecDestroy(m->step_exec); m->step_exec = nullptr; }
+  if (m->cap_stream == nullptr) SRM_CUDA(cudaStreamCreateWithFlags(&m->cap_stream, cudaStreamNonBlocking));
+  int32_t* hdr = reinterpret_cast<int32_t*>(s->status);
+  const int64_t pos0 = s->pos;
+  SRM_CUDA(cudaStreamBeginCapture(m->cap_stream, cudaStreamCaptureModeRelaxed));
+  int rc = decode_step_impl(m, s, nullptr, samp, 0, nullptr, d_out, out_stride, 0, nullptr, d_ws, ws_bytes,
+                            m->cap_stream, hdr);
+  cudaError_t e = cudaSuccess;
+  if (rc == SRM_OK) {
+    ++g_kernel_launches;
+    e = launch_kernel(advance_counters_kernel, dim3(1), dim3(1), 0, m->cap_stream, hdr);
+  }
+  cudaGraph_t graph = nullptr;
+  const cudaError_t e2 = cudaStreamEndCapture(m->cap_stream, &graph);
+  s->pos = pos0;                                       // the captured step has not run
+  if (rc != SRM_OK) { if (graph) cudaGraphDestroy(graph); return rc; }
+  if (e != cudaSuccess || e2 != cudaSuccess || graph == nullptr) {
+    if (graph) cudaGraphDestroy(graph);
+    g_last_cuda_error = (int)(e != cudaSuccess ? e : e2);
+    return SRM_ERR_CUDA;
+  }
+  e = cudaGraphInstantiate(&m->step_exec, graph, 0);
+  cudaGraphDestroy(graph);
+  if (e != cudaSuccess) { m->step_exec = nullptr; g_last_cuda_error = (int)e; return SRM_ERR_CUDA; }
+  m->step_key = key;
+  return SRM_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
 int srm_generate(srm_model* m, srm_state* s, int32_t steps, int32_t first_step, const srm_sampling* samp,
                  int32_t* d_out, int64_t out_stride, void* d_ws, size_t ws_bytes, void* stream) {
-  if (m == nullptr || s == nullptr || steps < 0 || (d_out != nullptr && out_stride < steps)) return SRM_ERR_INVALID_ARG;
+  if (m == nullptr || s == nullptr || s->m != m || steps < 0 || (d_out != nullptr && out_stride < steps)) return SRM_ERR_INVALID_ARG;
   if (s->pos + steps > m->cfg.n_ctx) return SRM_ERR_CTX_OVERFLOW;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (samp != nullptr && d_ws != nullptr && use_step_graph(*m, *s, steps)) {
+    const uint64_t launches0 = g_kernel_launches;
+    int rc = prepare_step_graph(m, s, samp, d_out, out_stride, d_ws, ws_bytes);
+    if (rc) return rc;
+    const uint64_t per_step = g_kernel_launches - launches0;      // 0 when the graph was reused
+    if (per_step) m->step_launches = per_step;
+    g_kernel_launches = launches0;
+    SRM_CUDA(launch_kernel(set_counters_kernel, dim3(1), dim3(1), 0, st, reinterpret_cast<int32_t*>(s->status),
+                           (int)s->pos, (int)first_step, 0));
+    ++g_kernel_launches;
+    for (int j = 0; j < steps; ++j) SRM_CUDA(cudaGraphLaunch(m->step_exec, st));
+    g_kernel_launches += (uint64_t)steps * m->step_launches;
+    s->pos += steps;
+    return SRM_OK;
+  }
   for (int j = 0; j < steps; ++j) {
     int rc = decode_step_impl(m, s, nullptr, samp, first_step + j, nullptr, d_out, out_stride, j, nullptr, d_ws,
-                              ws_bytes, static_cast<cudaStream_t>(stream));
+                              ws_bytes, st);
     if (rc) return rc;
   }
   return SRM_OK;
