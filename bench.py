@@ -198,7 +198,7 @@ def cpu_baseline(shape, W, workload, w, seconds_target=12.0):
         tok = O.select_greedy(lg)
         steps += 1
         dt = time.perf_counter() - t0
-        if dt > seconds_target or steps >= 64:
+        if dt > seconds_target or steps >= 512:
             break
     return {"value": sample * steps / dt, "unit": UNIT, "cores": _blas_threads(), "kind": "oracle",
             "sample": f"{sample} samples x {steps} decode steps of the same model (numpy fp64 oracle, {dt:.1f} s)"}
