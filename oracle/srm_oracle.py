@@ -21,6 +21,9 @@ Parity status of each function (what pins it, see tests/test_oracle_*.py):
   layer_norm, gelu_erf     pinned: moments / identities / tabulated erf values
   philox4x32_10            pinned: cuRAND's host Philox4_32_10 generator, bijectivity
   select_greedy, select_topk  pinned: brute-force sort, frequency test
+  select_topp              pinned: brute force over all subsets (smallest set of most probable tokens
+                           with mass >= p), p = 1 == plain inverse-CDF sampling (numpy searchsorted),
+                           p -> 0 == greedy, frequency test against the renormalised nucleus
   token_mixer_parallel / _recurrent with head projections (Eq. 10)
                            pinned: brute-force Eq. 10 in the paper's d x n orientation with explicit
                            per-head I_g, identity projections == no projections, parallel == recurrent
@@ -213,6 +216,48 @@ def select_topk(logits: np.ndarray, k: int, temperature: float, seed: int,
     return (out, detail) if return_detail else out
 
 
+def nucleus(row: np.ndarray, p: float, temperature: float):
+    """(ids of the nucleus in (logit desc, id asc) order, their weights): with probabilities
+    softmax(row / T), the shortest prefix of that order whose probability mass reaches p
+    (Holtzman et al., 'The curious case of neural text degeneration', ICLR 2020: the smallest
+    set of most probable tokens with total probability >= p). Weights are exp((l - max) / T)."""
+    row = row.astype(np.float64)
+    order = topk_order(row, row.shape[0])
+    w = np.exp((row[order] - row[order[0]]) / temperature)
+    c = np.cumsum(w)
+    m = int(np.searchsorted(c, p * c[-1], side="left"))     # first prefix with mass >= p
+    m = min(m, len(order) - 1)
+    return order[: m + 1], w[: m + 1]
+
+
+def select_topp(logits: np.ndarray, p: float, temperature: float, seed: int,
+                sample_idx: np.ndarray, step: int, return_detail: bool = False):
+    """Temperature + nucleus (top-p) sampling, the sampler of the paper's GRPO rollouts
+    (Training details: top-p 0.9, temperature 0.7). Tokens outside the nucleus get probability
+    zero; the token is drawn from what is left by inverse CDF over the vocabulary in id order:
+    c_v = sum of the nucleus weights with id <= v, u = philox_uniform(...), the token is the
+    first nucleus id v with c_v > u * c_last (the last nucleus id if none)."""
+    B = logits.shape[0]
+    out = np.empty(B, dtype=np.int32)
+    detail = []
+    for b in range(B):
+        ids, w = nucleus(logits[b], p, temperature)
+        by_id = np.argsort(ids, kind="stable")
+        ids, w = ids[by_id], w[by_id]
+        c = np.cumsum(w)
+        u = philox_uniform(seed, int(sample_idx[b]), step)
+        thr = u * c[-1]
+        pick = len(ids) - 1
+        for i in range(len(ids)):
+            if c[i] > thr:
+                pick = i
+                break
+        out[b] = ids[pick]
+        if return_detail:
+            detail.append(dict(ids=ids, cdf=c, thr=thr, pick=pick, u=u))
+    return (out, detail) if return_detail else out
+
+
 # --------------------------------------------------------------------------------------
 # Head projections (Method / Architecture, Eq. 10): Y = P_out (concat_g [(I_g X) M_g + beta_g])
 # --------------------------------------------------------------------------------------
@@ -341,5 +386,8 @@ class SRMOracle:
     def select(logits, sampling, sample_idx, step):
         if sampling.get("mode", "greedy") == "greedy":
             return select_greedy(logits)
+        if sampling["mode"] == "topp":
+            return select_topp(logits, sampling["top_p"], sampling["temperature"],
+                               sampling["seed"], sample_idx, step)
         return select_topk(logits, sampling["top_k"], sampling["temperature"],
                            sampling["seed"], sample_idx, step)

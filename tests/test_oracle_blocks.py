@@ -144,3 +144,77 @@ def test_topk_sampling_frequencies_match_softmax():
     # distinct steps give a different stream for the same sample
     t2 = O.select_topk(lg[:200], k, T, seed=5, sample_idx=np.arange(200), step=1)
     assert np.any(t2 != toks[:200])
+
+
+# ---- nucleus (top-p) sampling ------------------------------------------------------------------
+
+def _probs(row, T):
+    w = np.array([math.exp((v - max(row)) / T) for v in row])
+    return w / w.sum()
+
+
+def test_nucleus_is_the_smallest_set_of_most_probable_tokens_with_mass_p_bruteforce():
+    """All 2^V subsets of a small vocabulary: among the sets whose mass reaches p the nucleus has the fewest
+    tokens, and among those of that size the largest mass (it takes the most probable tokens)."""
+    import itertools
+    rng = np.random.default_rng(11)
+    V, T = 10, 0.7
+    for trial in range(6):
+        row = rng.normal(size=V) * 1.5
+        pr = _probs(row, T)
+        for p in (0.3, 0.6, 0.9, 0.99):
+            ids, w = O.nucleus(row, p, T)
+            best = None
+            for r in range(1, V + 1):
+                sets = [s for s in itertools.combinations(range(V), r) if sum(pr[list(s)]) >= p - 1e-15]
+                if sets:
+                    best = max(sets, key=lambda s: sum(pr[list(s)]))
+                    break
+            assert sorted(ids.tolist()) == sorted(best)
+            # the weights are the unnormalised probabilities of exactly those tokens, most probable first
+            assert np.allclose(w / w.sum(), pr[ids] / pr[ids].sum(), rtol=1e-12)
+            assert np.all(np.diff(row[ids]) <= 0)
+
+
+def test_nucleus_ties_and_limits():
+    row = np.array([1.0, 3.0, 3.0, 3.0, 0.0, 3.0])
+    # four equal maxima of probability ~0.23 each: p = 0.5 needs three of them, the lowest ids
+    ids, _ = O.nucleus(row, 0.5, 1.0)
+    assert ids.tolist() == [1, 2, 3]
+    assert O.nucleus(row, 1e-9, 1.0)[0].tolist() == [1]               # p -> 0: the argmax alone
+    assert sorted(O.nucleus(row, 1.0, 1.0)[0].tolist()) == list(range(6))    # p = 1: everything
+    # a mass reached exactly keeps the prefix that reaches it, no more (probabilities 1/2, 1/4, 1/8, 1/8)
+    dyadic = np.log(np.array([0.5, 0.25, 0.125, 0.125]))
+    assert O.nucleus(dyadic, 0.75, 1.0)[0].tolist() == [0, 1]
+
+
+def test_topp_with_p_one_is_plain_inverse_cdf_sampling_and_with_small_p_greedy():
+    rng = np.random.default_rng(12)
+    B, V, T, seed = 40, 97, 0.7, 9
+    lg = rng.normal(size=(B, V)) * 2
+    toks = O.select_topp(lg, 1.0, T, seed, np.arange(B), step=3)
+    for b in range(B):
+        w = np.exp((lg[b] - lg[b].max()) / T)
+        c = np.cumsum(w)
+        u = O.philox_uniform(seed, b, 3)
+        assert toks[b] == min(int(np.searchsorted(c, u * c[-1], side="right")), V - 1)
+    assert np.array_equal(O.select_topp(lg, 1e-12, T, seed, np.arange(B), step=3), O.select_greedy(lg))
+
+
+def test_topp_sampling_frequencies_match_the_renormalised_nucleus():
+    V, p, T = 64, 0.9, 0.7
+    rng = np.random.default_rng(13)
+    row = rng.normal(size=V) * 2
+    N = 20000
+    lg = np.broadcast_to(row, (N, V))
+    toks = O.select_topp(lg, p, T, seed=6, sample_idx=np.arange(N), step=0)
+    ids, w = O.nucleus(row, p, T)
+    pr = w / w.sum()
+    assert 1 < len(ids) < V
+    freq = np.array([(toks == i).mean() for i in ids])
+    sigma = np.sqrt(pr * (1 - pr) / N)
+    assert np.all(np.abs(freq - pr) < 4.5 * sigma + 1e-4)
+    assert set(np.unique(toks)) <= set(ids.tolist())
+    # the mass outside the nucleus is below 1 - p, and dropping the least probable member breaks the bound
+    full = _probs(row, T)
+    assert full[ids].sum() >= p > full[ids[:-1]].sum()
