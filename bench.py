@@ -248,6 +248,8 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device(dev))
 
     w = I.WORKLOADS[args.workload]
+    if args.top_p is not None:         # nucleus sampling instead of the workload's selection rule
+        w = dict(w, sampling="topp", top_p=args.top_p, temperature=args.temperature or 0.7)
     shape = I.CONFIGS[w["model"]]
     if args.head_proj:
         import dataclasses
@@ -259,9 +261,11 @@ def run_ours(args):
     W = I.make_weights(shape)
     model = P.SRM(shape, W, device=dev, state_dtype=args.state_dtype,
                   flags={"auto": 0, "on": P.FLAG_GRAPH, "off": P.FLAG_NO_GRAPH}[args.graph])
-    samp = P.Sampling("greedy") if w["sampling"] == "greedy" else \
-        P.Sampling("topk", w["top_k"], w["temperature"], seed=shape.seed,
-                   sample_idx_base=rank_plan(rank, world, B)["sample_idx_base"])
+    sidx0 = rank_plan(rank, world, B)["sample_idx_base"]
+    samp = {"greedy": lambda: P.Sampling("greedy"),
+            "topk": lambda: P.Sampling("topk", w["top_k"], w["temperature"], seed=shape.seed, sample_idx_base=sidx0),
+            "topp": lambda: P.Sampling("topp", temperature=w["temperature"], seed=shape.seed, sample_idx_base=sidx0,
+                                       top_p=w["top_p"])}[w["sampling"]]()
     prompts = torch.from_numpy(I.make_prompts(args.workload, batch=B)).to(dev)
     chunk = min(B, args.chunk)
     st = model.new_state(B)
@@ -495,6 +499,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--head-proj", action="store_true",
                     help="token mixer with head projections (Eq. 10): adds W_in, W_out [d, d] per layer")
+    ap.add_argument("--top-p", type=float, default=None,
+                    help="select tokens by nucleus sampling with this p (temperature 0.7 unless --temperature)")
+    ap.add_argument("--temperature", type=float, default=None)
     ap.add_argument("--graph", default="auto", choices=["auto", "on", "off"],
                     help="srm_generate replays a captured step: auto = only for launch-bound (small) batches")
     ap.add_argument("--no-prompt-dedup", action="store_true",

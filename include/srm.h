@@ -58,7 +58,7 @@ enum srm_status_bits {
 };
 
 enum { SRM_DTYPE_FP32 = 0, SRM_DTYPE_BF16 = 1 };
-enum { SRM_SELECT_GREEDY = 0, SRM_SELECT_TOPK = 1 };
+enum { SRM_SELECT_GREEDY = 0, SRM_SELECT_TOPK = 1, SRM_SELECT_TOPP = 2 };
 enum {
   SRM_FLAG_NO_GRAPH = 4,             /* srm_generate never replays a captured step                     */
   SRM_FLAG_GRAPH = 8,                /* srm_generate always replays a captured step (default: only for
@@ -89,12 +89,18 @@ typedef struct {
 /* Token selection. Greedy: smallest id among the maxima. Top-k: keep the top_k largest logits
  * ordered by (logit desc, id asc), weights exp((l - l_max)/temperature), inverse-CDF draw with
  * u = (r >> 8) * 2^-24 where r is the first word of Philox4x32-10 with key (seed lo, seed hi)
- * and counter (sample_idx_base + b, step, 0, 0); 1 <= top_k <= 256. */
+ * and counter (sample_idx_base + b, step, 0, 0); 1 <= top_k <= 256.
+ * Top-p (nucleus sampling, the sampler of the paper's GRPO rollouts [Training details: top-p 0.9,
+ * temperature 0.7]): probabilities softmax(l / temperature); the nucleus is the shortest prefix of the
+ * (logit desc, id asc) order whose probability reaches top_p; the token is drawn from the nucleus by
+ * inverse CDF over ids in ascending order with the same u. Masses are summed as 64-bit fixed-point
+ * integers (weight of the most probable token = 2^32), so the result does not depend on scheduling;
+ * 0 < top_p <= 1. */
 typedef struct {
   int32_t  mode;             /* SRM_SELECT_*                                               */
   int32_t  top_k;
   float    temperature;
-  int32_t  reserved;
+  float    top_p;            /* SRM_SELECT_TOPP only                                       */
   uint64_t seed;
   uint64_t sample_idx_base;  /* Philox sample index of row 0 of the state                  */
 } srm_sampling;

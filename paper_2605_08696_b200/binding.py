@@ -46,19 +46,20 @@ class _Config(C.Structure):
 
 class _Sampling(C.Structure):
     _fields_ = [("mode", C.c_int32), ("top_k", C.c_int32), ("temperature", C.c_float),
-                ("reserved", C.c_int32), ("seed", C.c_uint64), ("sample_idx_base", C.c_uint64)]
+                ("top_p", C.c_float), ("seed", C.c_uint64), ("sample_idx_base", C.c_uint64)]
 
 
 @dataclass
 class Sampling:
-    mode: str = "greedy"          # "greedy" or "topk"
+    mode: str = "greedy"          # "greedy", "topk" or "topp"
     top_k: int = 50
     temperature: float = 1.0
     seed: int = 0
     sample_idx_base: int = 0
+    top_p: float = 1.0
 
     def c(self) -> _Sampling:
-        return _Sampling(0 if self.mode == "greedy" else 1, self.top_k, self.temperature, 0,
+        return _Sampling({"greedy": 0, "topk": 1, "topp": 2}[self.mode], self.top_k, self.temperature, self.top_p,
                          self.seed & 0xFFFFFFFFFFFFFFFF, self.sample_idx_base)
 
 

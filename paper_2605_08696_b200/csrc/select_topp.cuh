@@ -1,0 +1,289 @@
+// Temperature + nucleus (top-p) sampling over the vocabulary (Holtzman et al., ICLR 2020; the sampler of
+// the paper's GRPO rollouts: Training details, top-p 0.9 at temperature 0.7).
+//
+// Definition (one row of logits l_v): probabilities softmax(l / T); the nucleus is the shortest prefix of
+// the order (logit descending, id ascending) whose probability mass reaches p; the token is drawn from the
+// nucleus by inverse CDF over ids in ascending order with u = Philox4x32-10(seed; sample, step).
+//
+// A nucleus can hold most of the vocabulary (flat distributions), so nothing here sorts the row.
+//   * Weights are fixed-point integers q_v = round(2^32 exp((l_v - max) / T)) and every mass is an exact
+//     64-bit integer sum: sums do not depend on the order of addition, so neither the nucleus nor the drawn
+//     token depends on thread scheduling, and thresholds are compared exactly.
+//   * The key of the last nucleus member (keys: order-preserving uint32 image of the float) is found by
+//     four-way search on the key range: each pass sums mass and count of the range's four parts (pivots
+//     evenly spaced in logit value while the range is wide, in key space afterwards, which bounds the passes),
+//     keeps the part in which the cumulative mass from the top crosses p Z, and stops when that part holds
+//     at most kToppCap tokens (they are then ranked exactly, ties by id) or a single key (all ties).
+//   * The draw scans the row in id order: every thread owns a contiguous chunk, two block-wide prefix sums
+//     (ties before the chunk, nucleus mass before the chunk) locate the thread that holds the token.
+// One block per row; the row is staged in shared memory when it fits (V <= kToppSmemFloats), else re-read
+// from global memory (L2) on every pass.
+#pragma once
+
+#include "common.cuh"
+#include "select.cuh"
+
+namespace srm {
+
+constexpr int kToppThreads = 512;
+constexpr int kToppWarps = kToppThreads / 32;
+constexpr int kToppCap = 512;                    // tokens ranked exactly in the last stage (one per thread)
+constexpr int kToppMaxPasses = 28;               // 6 passes with value pivots, then 4-way search on at most 2^32 keys
+constexpr int kToppSmemFloats = 48 * 1024;       // rows up to 192 KB are staged in shared memory
+constexpr float kToppFixedOne = 4294967296.0f;   // 2^32: weight of the most probable token
+
+struct ToppScratch {
+  unsigned long long red[kToppWarps][8];         // block reductions: 4 masses + 4 counts
+  unsigned long long scan[kToppWarps];           // block prefix sums
+  unsigned long long bcast[8];
+  uint32_t ckey[kToppCap], skey[kToppCap];
+  int32_t cid[kToppCap], sid[kToppCap];
+  unsigned long long cq[kToppCap], sq[kToppCap];
+  int n_cand, pos, first;
+  float fmax_w[kToppWarps];
+};
+
+__device__ __forceinline__ unsigned long long topp_weight(float l, float m, float s) {
+  const float x = (l - m) * s;                   // <= 0; s = log2(e) / T
+  return (x > -40.f) ? __float2ull_rn(exp2f(x) * kToppFixedOne) : 0ull;     // NaN compares false: weight 0
+}
+// NaN sorts below everything
+__device__ __forceinline__ uint32_t topp_key(float l) { return (l == l) ? order_key(l) : 0u; }
+
+__device__ __forceinline__ unsigned long long warp_sum_u64(unsigned long long v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// exclusive prefix sum of one value per thread over the block; `total` receives the block sum
+__device__ __forceinline__ unsigned long long block_exclusive_scan(unsigned long long v, ToppScratch* sc,
+                                                                   unsigned long long* total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  unsigned long long incl = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const unsigned long long t = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += t;
+  }
+  __syncthreads();                               // previous users of sc->scan are done
+  if (lane == 31) sc->scan[warp] = incl;
+  __syncthreads();
+  unsigned long long base = 0, tot = 0;
+#pragma unroll
+  for (int w = 0; w < kToppWarps; ++w) {
+    const unsigned long long s = sc->scan[w];
+    if (w < warp) base += s;
+    tot += s;
+  }
+  *total = tot;
+  return base + incl - v;
+}
+
+template <bool ROW_IN_SMEM>
+__global__ void __launch_bounds__(kToppThreads)
+select_topp_kernel(const float* __restrict__ logits, int64_t R, int V, float top_p, float inv_temp, uint64_t seed,
+                   uint64_t sample_base, int step, SelectOut out, uint32_t* status) {
+  pdl_trigger();
+  pdl_wait();
+  extern __shared__ __align__(16) uint8_t topp_smem[];
+  ToppScratch* sc = reinterpret_cast<ToppScratch*>(topp_smem);
+  float* srow = reinterpret_cast<float*>(topp_smem + ((sizeof(ToppScratch) + 15) & ~size_t(15)));
+  const int64_t row = blockIdx.x;
+  if (row >= R) return;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const float* grow = logits + (row / out.row_div) * (int64_t)V;
+
+  // ---- pass 0: stage the row, maximum (NaN ignored, flagged) ----
+  float mx = -INFINITY;
+  bool bad = false;
+  for (int i = tid; i < V; i += kToppThreads) {
+    const float l = grow[i];
+    if (ROW_IN_SMEM) srow[i] = l;
+    bad |= !(fabsf(l) <= 3.0e38f);               // NaN or infinity
+    if (l > mx) mx = l;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  if (lane == 0) sc->fmax_w[warp] = mx;
+  if (bad) raise_status(status, kStatusNonFinite);
+  __syncthreads();
+  mx = sc->fmax_w[0];
+#pragma unroll
+  for (int w = 1; w < kToppWarps; ++w) mx = fmaxf(mx, sc->fmax_w[w]);
+  const float* rowp = ROW_IN_SMEM ? srow : grow;
+  if (!(mx > -INFINITY) || !(mx < INFINITY)) {   // no finite maximum: nothing to sample from
+    if (tid == 0) write_token(out, row, 0);
+    return;
+  }
+
+  const float s = inv_temp * 1.4426950408889634f;
+  // search range [lo, hi) in key space; `above` = mass of the keys >= hi
+  uint64_t lo = topp_key(mx - 34.0f / s), hi = (uint64_t)topp_key(mx) + 1;
+  unsigned long long above = 0, target = 0, in_mass = 0;
+  long long in_cnt = 0;
+  for (int pass = 0; pass < kToppMaxPasses; ++pass) {
+    // three pivots lo < p1 <= p2 <= p3 < hi (as keys)
+    uint32_t pv[3];
+    const uint64_t width = hi - lo;
+    bool by_value = pass < 6 && width > (1u << 12);
+    if (by_value) {
+      const float vlo = key_value((uint32_t)lo), vhi = key_value((uint32_t)(hi - 1));
+      const float st = (vhi - vlo) * 0.25f;
+#pragma unroll
+      for (int j = 0; j < 3; ++j) pv[j] = topp_key(vlo + st * (float)(j + 1));
+      by_value = (pv[0] > lo) && (pv[0] <= pv[1]) && (pv[1] <= pv[2]) && (pv[2] < hi - 1) && (vhi - vlo < INFINITY);
+    }
+    if (!by_value) {
+      const uint64_t w4 = (width + 3) / 4;
+#pragma unroll
+      for (int j = 0; j < 3; ++j) {
+        const uint64_t pj = lo + w4 * (uint64_t)(j + 1);
+        pv[j] = (uint32_t)(pj < hi ? pj : hi - 1);
+      }
+    }
+    unsigned long long m0 = 0, m1 = 0, m2 = 0, m3 = 0;
+    unsigned int c0 = 0, c1 = 0, c2 = 0, c3 = 0;
+    for (int i = tid; i < V; i += kToppThreads) {
+      const float l = rowp[i];
+      const uint32_t k = topp_key(l);
+      if (k >= lo && k < hi) {
+        const unsigned long long q = topp_weight(l, mx, s);
+        const int b = (k >= pv[0]) + (k >= pv[1]) + (k >= pv[2]);
+        m0 += (b == 0) ? q : 0ull; m1 += (b == 1) ? q : 0ull; m2 += (b == 2) ? q : 0ull; m3 += (b == 3) ? q : 0ull;
+        c0 += (b == 0); c1 += (b == 1); c2 += (b == 2); c3 += (b == 3);
+      }
+    }
+    m0 = warp_sum_u64(m0); m1 = warp_sum_u64(m1); m2 = warp_sum_u64(m2); m3 = warp_sum_u64(m3);
+    c0 = __reduce_add_sync(0xffffffffu, c0); c1 = __reduce_add_sync(0xffffffffu, c1);
+    c2 = __reduce_add_sync(0xffffffffu, c2); c3 = __reduce_add_sync(0xffffffffu, c3);
+    __syncthreads();
+    if (lane == 0) {
+      sc->red[warp][0] = m0; sc->red[warp][1] = m1; sc->red[warp][2] = m2; sc->red[warp][3] = m3;
+      sc->red[warp][4] = c0; sc->red[warp][5] = c1; sc->red[warp][6] = c2; sc->red[warp][7] = c3;
+    }
+    __syncthreads();
+    unsigned long long mass[4] = {0, 0, 0, 0}, cnt[4] = {0, 0, 0, 0};
+#pragma unroll
+    for (int w = 0; w < kToppWarps; ++w) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) { mass[j] += sc->red[w][j]; cnt[j] += sc->red[w][4 + j]; }
+    }
+    if (pass == 0) {
+      // the first range holds every token of non-zero weight: Z, and the mass the nucleus must reach
+      const unsigned long long Z = mass[0] + mass[1] + mass[2] + mass[3];
+      const double t = ceil((double)top_p * (double)Z);
+      target = t < 1.0 ? 1ull : (t > (double)Z ? Z : (unsigned long long)t);
+    }
+    // from the top: the part in which the cumulative mass reaches the target
+    int chosen = 0;
+    unsigned long long acc = above;
+#pragma unroll
+    for (int b = 3; b >= 0; --b) {
+      if (acc + mass[b] >= target) { chosen = b; break; }
+      acc += mass[b];
+    }
+    above = acc;
+    const uint64_t nlo = chosen == 0 ? lo : pv[chosen - 1], nhi = chosen == 3 ? hi : pv[chosen];
+    lo = nlo; hi = nhi;
+    in_mass = mass[chosen];
+    in_cnt = (long long)cnt[chosen];
+    if (in_cnt <= kToppCap || hi - lo <= 1) break;
+  }
+
+  // ---- the last nucleus member: its key, how many tokens of that key are in, the nucleus mass ----
+  uint32_t kstar;
+  long long n_ties_in;
+  unsigned long long nucleus_mass;
+  if (in_cnt <= kToppCap) {
+    if (tid == 0) { sc->n_cand = 0; sc->pos = kToppCap; sc->first = kToppCap; }
+    __syncthreads();
+    for (int i = tid; i < V; i += kToppThreads) {
+      const float l = rowp[i];
+      const uint32_t k = topp_key(l);
+      if (k >= lo && k < hi) {
+        const int slot = atomicAdd(&sc->n_cand, 1);
+        if (slot < kToppCap) { sc->ckey[slot] = k; sc->cid[slot] = i; sc->cq[slot] = topp_weight(l, mx, s); }
+      }
+    }
+    __syncthreads();
+    const int n = sc->n_cand < kToppCap ? sc->n_cand : kToppCap;
+    if (tid < n) {                               // rank by (key descending, id ascending)
+      const uint32_t kt = sc->ckey[tid];
+      const int it = sc->cid[tid];
+      int rank = 0;
+      for (int j = 0; j < n; ++j) rank += (sc->ckey[j] > kt) || (sc->ckey[j] == kt && sc->cid[j] < it);
+      sc->skey[rank] = kt; sc->sid[rank] = it; sc->sq[rank] = sc->cq[tid];
+    }
+    __syncthreads();
+    unsigned long long tot;
+    const unsigned long long mine = tid < n ? sc->sq[tid] : 0ull;
+    const unsigned long long before = block_exclusive_scan(mine, sc, &tot);
+    if (tid < n && above + before + mine >= target) atomicMin(&sc->pos, tid);
+    __syncthreads();
+    const int pos = sc->pos < n ? sc->pos : n - 1;     // (n >= 1: the chosen part holds the boundary token)
+    kstar = sc->skey[pos];
+    if (tid <= pos && sc->skey[tid] == kstar) atomicMin(&sc->first, tid);
+    if (tid == pos) sc->bcast[0] = above + before + mine;
+    __syncthreads();
+    n_ties_in = pos - sc->first + 1;
+    nucleus_mass = sc->bcast[0];
+  } else {
+    // a single key with more than kToppCap tokens: all ties, taken in id order
+    kstar = (uint32_t)lo;
+    const unsigned long long qt = in_mass / (unsigned long long)in_cnt;       // they all carry the same weight
+    long long c = qt > 0 ? (long long)((target - above + qt - 1) / qt) : in_cnt;
+    n_ties_in = c < 1 ? 1 : (c > in_cnt ? in_cnt : c);
+    nucleus_mass = above + (unsigned long long)n_ties_in * qt;
+  }
+
+  // ---- the draw: first id whose cumulative nucleus mass exceeds floor(u * nucleus mass) ----
+  const uint64_t sidx = sample_base + (uint64_t)row;
+  const uint32_t r = philox4x32_10_word0((uint32_t)sidx, (uint32_t)(out.ctr != nullptr ? out.ctr[kCtrStep] : step), 0u, 0u,
+                                         (uint32_t)seed, (uint32_t)(seed >> 32));
+  const double u = (double)(r >> 8) * (1.0 / 16777216.0);
+  const unsigned long long thr = (unsigned long long)(u * (double)nucleus_mass);
+  const int chunk = ((V + kToppThreads - 1) / kToppThreads) | 1;             // odd: conflict-free in shared memory
+  const int i0 = tid * chunk < V ? tid * chunk : V, i1 = i0 + chunk < V ? i0 + chunk : V;
+  unsigned long long my_ties = 0;
+  for (int i = i0; i < i1; ++i) my_ties += topp_key(rowp[i]) == kstar;
+  unsigned long long tot;
+  const unsigned long long ties_before = block_exclusive_scan(my_ties, sc, &tot);
+  unsigned long long my_mass = 0;
+  {
+    long long t = (long long)ties_before;
+    for (int i = i0; i < i1; ++i) {
+      const float l = rowp[i];
+      const uint32_t k = topp_key(l);
+      const bool in = k > kstar || (k == kstar && t++ < n_ties_in);
+      if (in) my_mass += topp_weight(l, mx, s);
+    }
+  }
+  if (tid == 0) sc->pos = -1;
+  const unsigned long long mass_before = block_exclusive_scan(my_mass, sc, &tot);      // (barriers inside)
+  if (thr >= mass_before && thr < mass_before + my_mass) {
+    unsigned long long c = mass_before;
+    long long t = (long long)ties_before;
+    int pick = -1;
+    for (int i = i0; i < i1; ++i) {
+      const float l = rowp[i];
+      const uint32_t k = topp_key(l);
+      const bool in = k > kstar || (k == kstar && t++ < n_ties_in);
+      if (in) {
+        c += topp_weight(l, mx, s);
+        if (c > thr) { pick = i; break; }
+      }
+    }
+    if (pick >= 0) {
+      write_token(out, row, pick);
+      sc->pos = pick;
+    }
+  }
+  __syncthreads();
+  if (tid == 0 && sc->pos < 0) {                  // cannot happen while the sums above are consistent
+    raise_status(status, kStatusNonFinite);
+    write_token(out, row, 0);
+  }
+}
+
+}  // namespace srm

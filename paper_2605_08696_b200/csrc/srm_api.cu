@@ -22,6 +22,7 @@
 #include "mixer_proj.cuh"
 #include "prefill.cuh"
 #include "select.cuh"
+#include "select_topp.cuh"
 
 using namespace srm;
 
@@ -171,6 +172,7 @@ struct srm_model {
     bool operator==(const StepKey& o) const {
       return s == o.s && ws == o.ws && ws_bytes == o.ws_bytes && out == o.out && out_stride == o.out_stride &&
              samp.mode == o.samp.mode && samp.top_k == o.samp.top_k && samp.temperature == o.samp.temperature &&
+             samp.top_p == o.samp.top_p &&
              samp.seed == o.samp.seed && samp.sample_idx_base == o.samp.sample_idx_base;
     }
   } step_key;
@@ -480,6 +482,9 @@ int launch_gemm(srm_model& m, int epi, int64_t M, int64_t N, int64_t K, const vo
 int check_sampling(const srm_model& m, const srm_sampling* s) {
   if (s == nullptr) return SRM_ERR_INVALID_ARG;
   if (s->mode == SRM_SELECT_GREEDY) return SRM_OK;
+  if (s->mode == SRM_SELECT_TOPP) {
+    return (s->top_p > 0.f && s->top_p <= 1.f && s->temperature > 0.f) ? SRM_OK : SRM_ERR_INVALID_ARG;
+  }
   if (s->mode != SRM_SELECT_TOPK) return SRM_ERR_INVALID_ARG;
   if (s->top_k < 1 || s->top_k > kTopKMax || s->top_k > m.cfg.vocab || !(s->temperature > 0.f)) return SRM_ERR_INVALID_ARG;
   return SRM_OK;
@@ -492,6 +497,23 @@ int launch_select(const srm_model& m, int64_t R, const float* logits, const srm_
   const int V = m.cfg.vocab;
   if (s.mode == SRM_SELECT_GREEDY) {
     SRM_CUDA(launch_kernel(select_greedy_kernel, dim3((unsigned)R), dim3(kSelThreads), 0, st, logits, R, V, out, status));
+  } else if (s.mode == SRM_SELECT_TOPP) {
+    const float inv_t = 1.0f / s.temperature;
+    const size_t scratch = (sizeof(ToppScratch) + 15) & ~size_t(15);
+    if (V <= kToppSmemFloats) {
+      const size_t smem = scratch + (size_t)V * 4;
+      static bool attr_set = false;
+      if (!attr_set) {
+        SRM_CUDA(cudaFuncSetAttribute(select_topp_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      (int)(scratch + (size_t)kToppSmemFloats * 4)));
+        attr_set = true;
+      }
+      SRM_CUDA(launch_kernel(select_topp_kernel<true>, dim3((unsigned)R), dim3(kToppThreads), smem, st, logits, R, V,
+                             s.top_p, inv_t, s.seed, sample_base, step, out, status));
+    } else {
+      SRM_CUDA(launch_kernel(select_topp_kernel<false>, dim3((unsigned)R), dim3(kToppThreads), scratch, st, logits, R, V,
+                             s.top_p, inv_t, s.seed, sample_base, step, out, status));
+    }
   } else {
     const float inv_t = 1.0f / s.temperature;
     // threshold start: the normal quantile that leaves about 2.5 k of the V logits above it

@@ -28,3 +28,24 @@ def custom_shape(**kw):
     base = dict(n_layers=2, d_model=64, vocab=256, n_ctx=32, dtype="fp32", seed=0)
     base.update(kw)
     return I.SRMShape(**base)
+
+
+def topp_is_strict(row, p, T, det, tol=2e-6):
+    """True when neither decision of nucleus sampling is within rounding (fp32 exp, 2^-32 weight grid, against
+    fp64) of flipping the drawn token. The nucleus closes where the descending cumulative mass reaches p Z: if
+    that is within tol, a token at the edge may flip in or out, which moves u * mass by at most that token's
+    weight. The draw compares u * mass with the CDF edges of the drawn token."""
+    from oracle import srm_oracle as O
+    order = O.topk_order(row.astype(np.float64), row.shape[0])
+    w = np.exp((row[order].astype(np.float64) - row[order[0]]) / T)
+    c = np.cumsum(w)
+    m = len(det["ids"]) - 1
+    g1 = (c[m] - p * c[-1]) / c[-1] if m < len(c) - 1 else np.inf        # (the whole vocabulary cannot grow)
+    if m > 0 and p < 1.0:                            # (p = 1 keeps everything, whatever the last weights are)
+        g1 = min(g1, (p * c[-1] - c[m - 1]) / c[-1])
+    edge = 0.0 if g1 > tol else max(w[m], w[min(m + 1, len(w) - 1)]) / c[m]
+    cdf, thr, k = det["cdf"], det["thr"], det["pick"]
+    g2 = (cdf[k] - thr) / cdf[-1]
+    if k > 0:
+        g2 = min(g2, (thr - cdf[k - 1]) / cdf[-1])
+    return g2 > tol + 2 * edge

@@ -4,7 +4,7 @@ import pytest
 import torch
 
 import srm_inputs as I
-from helpers import custom_shape, rel_err_rows
+from helpers import custom_shape, rel_err_rows, topp_is_strict
 
 pytestmark = pytest.mark.gpu
 
@@ -227,6 +227,68 @@ def test_topk_sampling_matches_oracle(V, k):
             assert np.min(np.abs(c - thr)) < 1e-6 * c[-1], (r, got[r], want[r])
             exempt += 1
     assert exempt <= 1
+
+
+@pytest.mark.parametrize("V,p", [(256, 0.9), (8000, 0.9), (32000, 0.9), (32000, 0.3), (32000, 1.0), (1024, 1e-6),
+                                 (50000, 0.9), (50000, 0.999)])
+def test_topp_sampling_matches_oracle(V, p):
+    from oracle import srm_oracle as O
+    import paper_2605_08696_b200 as P
+    shape = custom_shape(vocab=V)
+    m, _ = _model(shape)
+    rng = np.random.default_rng(V + int(p * 1000))
+    R, T, seed, step, base = 40, 0.7, 0x0123456789abcdef, 5, 2000
+    lg = (rng.normal(size=(R, V)) * rng.choice([0.3, 1.0, 3.0], size=(R, 1))).astype(np.float32)
+    lg[0] = np.round(lg[0], 0)                       # heavy ties, also across the edge of the nucleus
+    lg[1, :] = 0.25                                  # all equal: the nucleus is the first ceil(p V) ids
+    lg[2] = np.round(lg[2], 1)
+    lg[3, : V // 2] = 1.5                            # a tie group far larger than the exact last stage holds
+    tok = torch.full((R,), -7, dtype=torch.int32, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    samp = P.Sampling("topp", temperature=T, seed=seed, sample_idx_base=base, top_p=p)
+    m.k_select(_t(lg), samp, step, tok, status=status)
+    got = tok.cpu().numpy()
+    assert status.item() == 0
+    want, det = O.select_topp(lg, np.float32(p), T, seed, base + np.arange(R), step, return_detail=True)
+    strict = 0
+    for r in range(R):
+        if topp_is_strict(lg[r], float(np.float32(p)), T, det[r]):
+            assert got[r] == want[r], (r, got[r], want[r])
+            strict += 1
+        else:
+            # a decision within rounding of flipping: the token must still come from the nucleus (one more
+            # token allowed at its edge)
+            sup, _ = O.nucleus(lg[r], min(1.0, float(np.float32(p)) + 1e-5), T)
+            assert got[r] in sup
+    assert strict >= R // 2          # (50000 similar tokens: a CDF step is 2e-5 wide, a fifth of the draws land within tol of an edge)
+
+
+def test_topp_sampling_is_reproducible_and_keyed_by_sample_and_step():
+    import paper_2605_08696_b200 as P
+    shape = custom_shape(vocab=8000)
+    m, _ = _model(shape)
+    lg = _t(np.tile(np.random.default_rng(0).normal(size=(1, 8000)).astype(np.float32), (64, 1)))
+    outs = []
+    for base, step in [(0, 0), (0, 1), (64, 0), (0, 0)]:
+        tok = torch.zeros(64, dtype=torch.int32, device=DEV)
+        m.k_select(lg, P.Sampling("topp", temperature=0.7, seed=5, sample_idx_base=base, top_p=0.9), step, tok)
+        outs.append(tok.cpu().numpy())
+    assert np.array_equal(outs[0], outs[3])
+    assert not np.array_equal(outs[0], outs[1]) and not np.array_equal(outs[0], outs[2])
+    assert len(np.unique(outs[0])) > 20
+
+
+def test_topp_rejects_bad_parameters():
+    import paper_2605_08696_b200 as P
+    m, _ = _model(custom_shape(vocab=256))
+    lg = torch.zeros(4, 256, device=DEV)
+    tok = torch.zeros(4, dtype=torch.int32, device=DEV)
+    for bad in (dict(top_p=0.0), dict(top_p=1.5), dict(top_p=0.9, temperature=0.0)):
+        kw = dict(temperature=0.7, top_p=0.9)
+        kw.update(bad)
+        with pytest.raises(P.SRMError) as e:
+            m.k_select(lg, P.Sampling("topp", **kw), 0, tok)
+        assert e.value.code == -1
 
 
 def test_topk_sampling_stream_is_keyed_by_sample_and_step():

@@ -93,6 +93,37 @@ def _teacher_forced(shape, W, model, prompts, gen, sampling=None, sample_idx=Non
     return dict(worst=worst, mismatches=mism, checked=checked, exempt=exempt, tokens=toks_o)
 
 
+def test_tiny_config_nucleus_sampling_follows_the_oracle_sampler_step_by_step():
+    """Free-running generation with top-p 0.9 at temperature 0.7 (the paper's rollout sampler) on the tiny
+    fp32 model: at every step the oracle's nucleus sampler, run on the logits the device produced, with the
+    same Philox key, sample index and step, draws the device's token (decisions within rounding of flipping
+    excepted); replicas of one prompt draw different continuations."""
+    import paper_2605_08696_b200 as P
+    from oracle import srm_oracle as O
+    from helpers import topp_is_strict
+    shape, W, model = _build("tiny")
+    prompts = np.repeat(I.make_prompts("tiny")[:2], 8, axis=0)           # 2 prompts x 8 replicas
+    B, n = prompts.shape
+    p, T, seed, base = 0.9, 0.7, 99, 500
+    samp = P.Sampling("topp", temperature=T, seed=seed, sample_idx_base=base, top_p=p)
+    st = model.new_state(B)
+    ws = model.new_workspace(B, n, prefill_samples=B)
+    tok, lg = model.prefill(st, torch.from_numpy(prompts).to(DEV), samp, ws, want_logits=True)
+    checked, seqs = 0, [tok.cpu().numpy().copy()]
+    for k in range(20):
+        lg_np, tok_np = lg.cpu().numpy(), tok.cpu().numpy()
+        want, det = O.select_topp(lg_np, np.float32(p), T, seed, base + np.arange(B), k, return_detail=True)
+        for b in range(B):
+            if topp_is_strict(lg_np[b], float(np.float32(p)), T, det[b]):
+                assert tok_np[b] == want[b], (k, b)
+                checked += 1
+        tok, lg = model.decode_step(st, None, samp, k + 1, ws, want_logits=True)
+        seqs.append(tok.cpu().numpy().copy())
+    assert checked > 0.9 * 20 * B
+    seqs = np.stack(seqs, 1)
+    assert len({tuple(r) for r in seqs[:8]}) > 4 and st.status() == 0
+
+
 def test_tiny_config_full_parity_fp32():
     """Config 'tiny': 4 prompts x 8 tokens, greedy 24 tokens, fp32, tolerance 1e-4; every token
     with margin > 1e-2 bit-exact; also free-running generation equals the oracle's tokens."""
@@ -192,7 +223,7 @@ def test_fused_greedy_head_equals_logits_then_selection_on_device():
     assert st_a.status() == 0 and st_b.status() == 0
 
 
-@pytest.mark.parametrize("mode", ["greedy", "topk"])
+@pytest.mark.parametrize("mode", ["greedy", "topk", "topp"])
 def test_replicated_prefill_equals_prefill_of_the_replicated_prompts(mode):
     """srm_prefill_replicated (each distinct prompt run once, cache copied to its replicas, one selection per
     replica) leaves, bit for bit, what srm_prefill on the replicated token matrix leaves: cache, first tokens,
@@ -203,7 +234,8 @@ def test_replicated_prefill_equals_prefill_of_the_replicated_prompts(mode):
     B = n_prompts * replicas
     base = torch.from_numpy(I.uniform_prompts(n_prompts, n, shape.vocab, seed=31)).to(DEV)
     full = base.repeat_interleave(replicas, dim=0).contiguous()
-    samp = P.Sampling("greedy") if mode == "greedy" else P.Sampling("topk", 50, 0.8, seed=77, sample_idx_base=1000)
+    samp = {"greedy": P.Sampling("greedy"), "topk": P.Sampling("topk", 50, 0.8, seed=77, sample_idx_base=1000),
+            "topp": P.Sampling("topp", temperature=0.7, seed=77, sample_idx_base=1000, top_p=0.9)}[mode]
     ws = model.new_workspace(B, n, prefill_samples=B + 8)
     st_a, st_b, st_c = model.new_state(B), model.new_state(B), model.new_state(B)
     first_a = model.prefill(st_a, full, samp, ws)
@@ -213,7 +245,7 @@ def test_replicated_prefill_equals_prefill_of_the_replicated_prompts(mode):
     assert torch.equal(first_a, first_b) and torch.equal(first_a, first_c)
     assert torch.equal(st_a.cache(), st_b.cache()) and torch.equal(st_a.cache(), st_c.cache())
     assert lg_b.shape == (n_prompts, shape.vocab)
-    if mode == "topk":
+    if mode != "greedy":
         assert len(set(first_a[:replicas].tolist())) > 1                     # replicas of one prompt draw differently
     else:
         assert len(set(first_a[:replicas].tolist())) == 1
@@ -224,7 +256,7 @@ def test_replicated_prefill_equals_prefill_of_the_replicated_prompts(mode):
     assert st_a.status() == 0 and st_b.status() == 0 and st_c.status() == 0 and st_b.pos == n + 3
 
 
-@pytest.mark.parametrize("mode", ["greedy", "topk"])
+@pytest.mark.parametrize("mode", ["greedy", "topk", "topp"])
 def test_generate_by_graph_replay_equals_launch_by_launch(mode):
     """srm_generate replaying one captured step (position, Philox step and store column in device-side
     counters) emits exactly the tokens and leaves exactly the cache of the launch-by-launch loop; a second call
@@ -236,7 +268,8 @@ def test_generate_by_graph_replay_equals_launch_by_launch(mode):
     m_graph = P.SRM(shape, W, device=DEV, flags=P.FLAG_GRAPH)
     B, n = 48, 32
     prompts = torch.from_numpy(I.uniform_prompts(B, n, shape.vocab, seed=41)).to(DEV)
-    samp = P.Sampling("greedy") if mode == "greedy" else P.Sampling("topk", 50, 0.8, seed=5, sample_idx_base=7)
+    samp = {"greedy": P.Sampling("greedy"), "topk": P.Sampling("topk", 50, 0.8, seed=5, sample_idx_base=7),
+            "topp": P.Sampling("topp", temperature=0.7, seed=5, sample_idx_base=7, top_p=0.9)}[mode]
     outs = []
     for model in (m_loop, m_graph):
         st = model.new_state(B)
