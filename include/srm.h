@@ -94,7 +94,7 @@ typedef struct {
  * temperature 0.7]): probabilities softmax(l / temperature); the nucleus is the shortest prefix of the
  * (logit desc, id asc) order whose probability reaches top_p; the token is drawn from the nucleus by
  * inverse CDF over ids in ascending order with the same u. Masses are summed as 64-bit fixed-point
- * integers (weight of the most probable token = 2^32), so the result does not depend on scheduling;
+ * integers (weight of the most probable token = 2^31), so the result does not depend on scheduling;
  * 0 < top_p <= 1. */
 typedef struct {
   int32_t  mode;             /* SRM_SELECT_*                                               */

@@ -6,18 +6,18 @@
 // nucleus by inverse CDF over ids in ascending order with u = Philox4x32-10(seed; sample, step).
 //
 // A nucleus can hold most of the vocabulary (flat distributions), so nothing here sorts the row.
-//   * Weights are fixed-point integers q_v = round(2^32 exp((l_v - max) / T)) and every mass is an exact
+//   * Weights are fixed-point integers q_v = round(2^31 exp((l_v - max) / T)) and every mass is an exact
 //     64-bit integer sum: sums do not depend on the order of addition, so neither the nucleus nor the drawn
 //     token depends on thread scheduling, and thresholds are compared exactly.
 //   * The key of the last nucleus member (keys: order-preserving uint32 image of the float) is found by
 //     four-way search on the key range: each pass sums mass and count of the range's four parts (pivots
 //     evenly spaced in logit value while the range is wide, in key space afterwards, which bounds the passes),
 //     keeps the part in which the cumulative mass from the top crosses p Z, and stops when that part holds
-//     at most kToppCap tokens (they are then ranked exactly, ties by id) or a single key (all ties).
+//     at most kToppExact tokens (they are then ranked exactly, ties by id) or a single key (all ties).
 //   * The draw scans the row in id order: every thread owns a contiguous chunk, two block-wide prefix sums
 //     (ties before the chunk, nucleus mass before the chunk) locate the thread that holds the token.
-// One block per row; the row is staged in shared memory when it fits (V <= kToppSmemFloats), else re-read
-// from global memory (L2) on every pass.
+// One block per row; the row's keys are staged in shared memory when they fit (V <= kToppSmemFloats), else
+// the row is re-read from global memory (L2) on every pass.
 #pragma once
 
 #include "common.cuh"
@@ -25,27 +25,35 @@
 
 namespace srm {
 
-constexpr int kToppThreads = 512;
+constexpr int kToppThreads = 1024;
 constexpr int kToppWarps = kToppThreads / 32;
-constexpr int kToppCap = 512;                    // tokens ranked exactly in the last stage (one per thread)
+constexpr int kToppCap = 1024;                   // capacity of the exact last stage (one token per thread)
+constexpr int kToppExact = 256;                  // the search stops when the part that holds the edge has this few tokens
+                                                 // (ranking n candidates costs n^2 comparisons)
 constexpr int kToppMaxPasses = 28;               // 6 passes with value pivots, then 4-way search on at most 2^32 keys
-constexpr int kToppSmemFloats = 48 * 1024;       // rows up to 192 KB are staged in shared memory
-constexpr float kToppFixedOne = 4294967296.0f;   // 2^32: weight of the most probable token
+constexpr int kToppSmemFloats = 44 * 1024;       // rows up to 176 KB are staged in shared memory
+constexpr float kToppFixedOne = 2147483648.0f;   // 2^31: weight of the most probable token (weights fit 32 bits)
 
 struct ToppScratch {
   unsigned long long red[kToppWarps][8];         // block reductions: 4 masses + 4 counts
   unsigned long long scan[kToppWarps];           // block prefix sums
+  unsigned long long scan_total;
   unsigned long long bcast[8];
   uint32_t ckey[kToppCap], skey[kToppCap];
   int32_t cid[kToppCap], sid[kToppCap];
   unsigned long long cq[kToppCap], sq[kToppCap];
   int n_cand, pos, first;
-  float fmax_w[kToppWarps];
+  float fmax_w[kToppWarps], fmin_w[kToppWarps];
 };
 
+// round(2^31 exp((l - m) / T)) = round(2^(31 + (l - m) s)), s = log2(e) / T: one fused multiply-add, the
+// hardware exp2 (relative error 2^-22, well inside the tolerance of the comparison with the oracle), one
+// conversion. Arguments below -1 give less than one half and round to zero; NaN converts to zero.
 __device__ __forceinline__ unsigned long long topp_weight(float l, float m, float s) {
-  const float x = (l - m) * s;                   // <= 0; s = log2(e) / T
-  return (x > -40.f) ? __float2ull_rn(exp2f(x) * kToppFixedOne) : 0ull;     // NaN compares false: weight 0
+  const float x = fmaf(l - m, s, 31.0f);
+  float e;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(x));
+  return (unsigned long long)__float2uint_rn(e);
 }
 // NaN sorts below everything
 __device__ __forceinline__ uint32_t topp_key(float l) { return (l == l) ? order_key(l) : 0u; }
@@ -69,15 +77,20 @@ __device__ __forceinline__ unsigned long long block_exclusive_scan(unsigned long
   __syncthreads();                               // previous users of sc->scan are done
   if (lane == 31) sc->scan[warp] = incl;
   __syncthreads();
-  unsigned long long base = 0, tot = 0;
+  if (warp == 0) {                               // exclusive scan of the warp totals (lane = warp index)
+    const unsigned long long t = lane < kToppWarps ? sc->scan[lane] : 0ull;
+    unsigned long long ti = t;
 #pragma unroll
-  for (int w = 0; w < kToppWarps; ++w) {
-    const unsigned long long s = sc->scan[w];
-    if (w < warp) base += s;
-    tot += s;
+    for (int o = 1; o < 32; o <<= 1) {
+      const unsigned long long u = __shfl_up_sync(0xffffffffu, ti, o);
+      if (lane >= o) ti += u;
+    }
+    if (lane < kToppWarps) sc->scan[lane] = ti - t;
+    if (lane == 31) sc->scan_total = ti;
   }
-  *total = tot;
-  return base + incl - v;
+  __syncthreads();
+  *total = sc->scan_total;
+  return sc->scan[warp] + incl - v;
 }
 
 template <bool ROW_IN_SMEM>
@@ -88,30 +101,43 @@ select_topp_kernel(const float* __restrict__ logits, int64_t R, int V, float top
   pdl_wait();
   extern __shared__ __align__(16) uint8_t topp_smem[];
   ToppScratch* sc = reinterpret_cast<ToppScratch*>(topp_smem);
-  float* srow = reinterpret_cast<float*>(topp_smem + ((sizeof(ToppScratch) + 15) & ~size_t(15)));
+  uint32_t* skeys = reinterpret_cast<uint32_t*>(topp_smem + ((sizeof(ToppScratch) + 15) & ~size_t(15)));
   const int64_t row = blockIdx.x;
   if (row >= R) return;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const float* grow = logits + (row / out.row_div) * (int64_t)V;
 
   // ---- pass 0: stage the row, maximum (NaN ignored, flagged) ----
-  float mx = -INFINITY;
+  float mx = -INFINITY, mn = INFINITY;
   bool bad = false;
   for (int i = tid; i < V; i += kToppThreads) {
     const float l = grow[i];
-    if (ROW_IN_SMEM) srow[i] = l;
+    if (ROW_IN_SMEM) skeys[i] = topp_key(l);
     bad |= !(fabsf(l) <= 3.0e38f);               // NaN or infinity
     if (l > mx) mx = l;
+    if (l < mn) mn = l;
   }
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-  if (lane == 0) sc->fmax_w[warp] = mx;
+  for (int o = 16; o > 0; o >>= 1) {
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+  }
+  if (lane == 0) { sc->fmax_w[warp] = mx; sc->fmin_w[warp] = mn; }
   if (bad) raise_status(status, kStatusNonFinite);
   __syncthreads();
-  mx = sc->fmax_w[0];
+  if (warp == 0) {
+    mx = lane < kToppWarps ? sc->fmax_w[lane] : -INFINITY;
+    mn = lane < kToppWarps ? sc->fmin_w[lane] : INFINITY;
 #pragma unroll
-  for (int w = 1; w < kToppWarps; ++w) mx = fmaxf(mx, sc->fmax_w[w]);
-  const float* rowp = ROW_IN_SMEM ? srow : grow;
+    for (int o = 16; o > 0; o >>= 1) {
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+      mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+    }
+    if (lane == 0) { sc->fmax_w[0] = mx; sc->fmin_w[0] = mn; }
+  }
+  __syncthreads();
+  mx = sc->fmax_w[0]; mn = sc->fmin_w[0];
+  auto key_at = [&](int i) -> uint32_t { return ROW_IN_SMEM ? skeys[i] : topp_key(grow[i]); };
   if (!(mx > -INFINITY) || !(mx < INFINITY)) {   // no finite maximum: nothing to sample from
     if (tid == 0) write_token(out, row, 0);
     return;
@@ -119,7 +145,8 @@ select_topp_kernel(const float* __restrict__ logits, int64_t R, int V, float top
 
   const float s = inv_temp * 1.4426950408889634f;
   // search range [lo, hi) in key space; `above` = mass of the keys >= hi
-  uint64_t lo = topp_key(mx - 34.0f / s), hi = (uint64_t)topp_key(mx) + 1;
+  // (tokens more than 33 / s below the maximum have weight zero; nothing lies below the row's minimum)
+  uint64_t lo = topp_key(fmaxf(mx - 33.0f / s, mn)), hi = (uint64_t)topp_key(mx) + 1;
   unsigned long long above = 0, target = 0, in_mass = 0;
   long long in_cnt = 0;
   for (int pass = 0; pass < kToppMaxPasses; ++pass) {
@@ -142,14 +169,15 @@ select_topp_kernel(const float* __restrict__ logits, int64_t R, int V, float top
         pv[j] = (uint32_t)(pj < hi ? pj : hi - 1);
       }
     }
+    const uint32_t p1 = pv[0], p2 = pv[1], p3 = pv[2];
     unsigned long long m0 = 0, m1 = 0, m2 = 0, m3 = 0;
     unsigned int c0 = 0, c1 = 0, c2 = 0, c3 = 0;
+    const uint32_t lo32 = (uint32_t)lo, hi32 = (uint32_t)(hi - 1);           // inclusive upper end
     for (int i = tid; i < V; i += kToppThreads) {
-      const float l = rowp[i];
-      const uint32_t k = topp_key(l);
-      if (k >= lo && k < hi) {
-        const unsigned long long q = topp_weight(l, mx, s);
-        const int b = (k >= pv[0]) + (k >= pv[1]) + (k >= pv[2]);
+      const uint32_t k = key_at(i);
+      if (k >= lo32 && k <= hi32) {
+        const unsigned long long q = topp_weight(key_value(k), mx, s);
+        const int b = (k >= p1) + (k >= p2) + (k >= p3);
         m0 += (b == 0) ? q : 0ull; m1 += (b == 1) ? q : 0ull; m2 += (b == 2) ? q : 0ull; m3 += (b == 3) ? q : 0ull;
         c0 += (b == 0); c1 += (b == 1); c2 += (b == 2); c3 += (b == 3);
       }
@@ -163,12 +191,17 @@ select_topp_kernel(const float* __restrict__ logits, int64_t R, int V, float top
       sc->red[warp][4] = c0; sc->red[warp][5] = c1; sc->red[warp][6] = c2; sc->red[warp][7] = c3;
     }
     __syncthreads();
-    unsigned long long mass[4] = {0, 0, 0, 0}, cnt[4] = {0, 0, 0, 0};
+    if (warp == 0) {                             // one warp folds the per-warp partials (lane = warp index)
 #pragma unroll
-    for (int w = 0; w < kToppWarps; ++w) {
-#pragma unroll
-      for (int j = 0; j < 4; ++j) { mass[j] += sc->red[w][j]; cnt[j] += sc->red[w][4 + j]; }
+      for (int j = 0; j < 8; ++j) {
+        const unsigned long long t = warp_sum_u64(lane < kToppWarps ? sc->red[lane][j] : 0ull);
+        if (lane == 0) sc->bcast[j] = t;
+      }
     }
+    __syncthreads();
+    unsigned long long mass[4], cnt[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) { mass[j] = sc->bcast[j]; cnt[j] = sc->bcast[4 + j]; }
     if (pass == 0) {
       // the first range holds every token of non-zero weight: Z, and the mass the nucleus must reach
       const unsigned long long Z = mass[0] + mass[1] + mass[2] + mass[3];
@@ -188,7 +221,7 @@ select_topp_kernel(const float* __restrict__ logits, int64_t R, int V, float top
     lo = nlo; hi = nhi;
     in_mass = mass[chosen];
     in_cnt = (long long)cnt[chosen];
-    if (in_cnt <= kToppCap || hi - lo <= 1) break;
+    if (in_cnt <= kToppExact || hi - lo <= 1) break;
   }
 
   // ---- the last nucleus member: its key, how many tokens of that key are in, the nucleus mass ----
@@ -199,11 +232,10 @@ select_topp_kernel(const float* __restrict__ logits, int64_t R, int V, float top
     if (tid == 0) { sc->n_cand = 0; sc->pos = kToppCap; sc->first = kToppCap; }
     __syncthreads();
     for (int i = tid; i < V; i += kToppThreads) {
-      const float l = rowp[i];
-      const uint32_t k = topp_key(l);
+      const uint32_t k = key_at(i);
       if (k >= lo && k < hi) {
         const int slot = atomicAdd(&sc->n_cand, 1);
-        if (slot < kToppCap) { sc->ckey[slot] = k; sc->cid[slot] = i; sc->cq[slot] = topp_weight(l, mx, s); }
+        if (slot < kToppCap) { sc->ckey[slot] = k; sc->cid[slot] = i; sc->cq[slot] = topp_weight(key_value(k), mx, s); }
       }
     }
     __syncthreads();
@@ -246,17 +278,16 @@ select_topp_kernel(const float* __restrict__ logits, int64_t R, int V, float top
   const int chunk = ((V + kToppThreads - 1) / kToppThreads) | 1;             // odd: conflict-free in shared memory
   const int i0 = tid * chunk < V ? tid * chunk : V, i1 = i0 + chunk < V ? i0 + chunk : V;
   unsigned long long my_ties = 0;
-  for (int i = i0; i < i1; ++i) my_ties += topp_key(rowp[i]) == kstar;
+  for (int i = i0; i < i1; ++i) my_ties += key_at(i) == kstar;
   unsigned long long tot;
   const unsigned long long ties_before = block_exclusive_scan(my_ties, sc, &tot);
   unsigned long long my_mass = 0;
   {
     long long t = (long long)ties_before;
     for (int i = i0; i < i1; ++i) {
-      const float l = rowp[i];
-      const uint32_t k = topp_key(l);
+      const uint32_t k = key_at(i);
       const bool in = k > kstar || (k == kstar && t++ < n_ties_in);
-      if (in) my_mass += topp_weight(l, mx, s);
+      if (in) my_mass += topp_weight(key_value(k), mx, s);
     }
   }
   if (tid == 0) sc->pos = -1;
@@ -266,11 +297,10 @@ select_topp_kernel(const float* __restrict__ logits, int64_t R, int V, float top
     long long t = (long long)ties_before;
     int pick = -1;
     for (int i = i0; i < i1; ++i) {
-      const float l = rowp[i];
-      const uint32_t k = topp_key(l);
+      const uint32_t k = key_at(i);
       const bool in = k > kstar || (k == kstar && t++ < n_ties_in);
       if (in) {
-        c += topp_weight(l, mx, s);
+        c += topp_weight(key_value(k), mx, s);
         if (c > thr) { pick = i; break; }
       }
     }

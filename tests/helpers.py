@@ -31,7 +31,7 @@ def custom_shape(**kw):
 
 
 def topp_is_strict(row, p, T, det, tol=2e-6):
-    """True when neither decision of nucleus sampling is within rounding (fp32 exp, 2^-32 weight grid, against
+    """True when neither decision of nucleus sampling is within rounding (fp32 exp, 2^-31 weight grid, against
     fp64) of flipping the drawn token. The nucleus closes where the descending cumulative mass reaches p Z: if
     that is within tol, a token at the edge may flip in or out, which moves u * mass by at most that token's
     weight. The draw compares u * mass with the CDF edges of the drawn token."""
