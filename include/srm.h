@@ -177,6 +177,19 @@ int srm_prefill(srm_model* m, srm_state* s, const int32_t* d_tokens, int32_t n,
                 const srm_sampling* sampling, int32_t* d_first_tok, float* d_logits_last,
                 void* d_ws, size_t ws_bytes, void* stream);
 
+/* Prefill of prompts of different lengths (a serving batch). d_tokens int32[B, n_max] holds the prompts
+ * left-aligned, sample b uses its first d_lengths[b] tokens (1 <= length <= n_max; the rest of the row must
+ * still hold valid token ids, they are not used). Each sample's cache is the one its own length leaves
+ * [Eq. 1, Eq. 3 on its own positions], its first generated token comes from the logits of its last prompt
+ * position, and from here on the state keeps ONE POSITION PER SAMPLE on the device: srm_decode_step,
+ * srm_generate and the other step calls read alpha_t, beta_t at each sample's own t and advance it, so
+ * sample b behaves exactly as if it had been prefilled and decoded alone. srm_state_pos then reports the
+ * position of the longest sample (the one that reaches n_ctx first) and srm_state_set_pos is refused.
+ * Lengths outside [1, n_max] are clamped and reported through srm_status (SRM_STATUS_TOKEN_RANGE). */
+int srm_prefill_ragged(srm_model* m, srm_state* s, const int32_t* d_tokens, int32_t n_max,
+                       const int32_t* d_lengths, const srm_sampling* sampling, int32_t* d_first_tok,
+                       float* d_logits_last, void* d_ws, size_t ws_bytes, void* stream);
+
 /* Prefill for replicated prompts [Inference Compute Scaling: many samples per question, as in the
  * GRPO rollouts]: d_tokens holds n_prompts DISTINCT prompts [n_prompts, n]; the state has
  * B = n_prompts * replicas samples and sample p * replicas + j is replica j of prompt p. Every prompt runs

@@ -83,6 +83,7 @@ SYMBOLS = {
     "srm_state_last_token_ptr": (_P, [_P]),
     "srm_status": (C.c_int, [_P, _P, C.POINTER(C.c_uint32)]),
     "srm_prefill": (C.c_int, [_P, _P, _P, _I32, C.POINTER(_Sampling), _P, _P, _P, _SZ, _P]),
+    "srm_prefill_ragged": (C.c_int, [_P, _P, _P, _I32, _P, C.POINTER(_Sampling), _P, _P, _P, _SZ, _P]),
     "srm_prefill_replicated": (C.c_int, [_P, _P, _P, _I32, _I32, _I32, C.POINTER(_Sampling), _P, _P, _P, _SZ, _P]),
     "srm_decode_step": (C.c_int, [_P, _P, _P, C.POINTER(_Sampling), _I32, _P, _P, _P, _SZ, _P]),
     "srm_generate": (C.c_int, [_P, _P, _I32, _I32, C.POINTER(_Sampling), _P, _I64, _P, _SZ, _P]),
@@ -283,6 +284,19 @@ class SRM:
         s = sampling.c()
         _check(_lib().srm_prefill(self.handle, state.handle, _ptr(tokens), n, C.byref(s), _ptr(first), _ptr(logits),
                                   _ptr(ws), ws.numel(), _stream()), "srm_prefill")
+        return (first, logits) if want_logits else first
+
+    def prefill_ragged(self, state: SRMState, tokens: torch.Tensor, lengths: torch.Tensor, sampling: Sampling,
+                       ws: torch.Tensor, want_logits: bool = False):
+        """tokens [B, n_max] left-aligned prompts, lengths int32 [B]; afterwards every sample has its own position."""
+        B, n = tokens.shape
+        assert B == state.B and tokens.dtype == torch.int32 and lengths.dtype == torch.int32 and lengths.numel() == B
+        first = torch.empty(B, dtype=torch.int32, device=self.device)
+        logits = torch.empty(B, self.cfg.vocab, dtype=torch.float32, device=self.device) if want_logits else None
+        s = sampling.c()
+        _check(_lib().srm_prefill_ragged(self.handle, state.handle, _ptr(tokens), n, _ptr(lengths), C.byref(s),
+                                         _ptr(first), _ptr(logits), _ptr(ws), ws.numel(), _stream()),
+               "srm_prefill_ragged")
         return (first, logits) if want_logits else first
 
     def prefill_replicated(self, state: SRMState, tokens: torch.Tensor, replicas: int, sampling: Sampling,

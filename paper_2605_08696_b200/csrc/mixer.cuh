@@ -24,6 +24,7 @@ struct MixerParams {
   float eps;
   uint32_t* status;
   const int32_t* ctr;    // device-side step counters, or nullptr: then `t` above is the position
+  const int32_t* pos;    // [R] per-row positions (samples of different lengths), or nullptr: one position for all rows
 };
 
 constexpr int kMixerWarps = 4;
@@ -83,7 +84,7 @@ __global__ void __launch_bounds__(kMixerWarps * 32) mixer_step_kernel(const Mixe
   const int d = p.d;
   const int dh = d / p.h;
   const int h_row = p.h >> 1;
-  const int t = p.ctr != nullptr ? p.ctr[kCtrPos] : p.t;
+  const int t = p.pos != nullptr ? min(max(p.pos[row], 0), p.n_ctx - 1) : (p.ctr != nullptr ? p.ctr[kCtrPos] : p.t);
 
   float4 v[NV];
   if (p.tok != nullptr) {
@@ -154,17 +155,19 @@ __global__ void __launch_bounds__(kMixerWarps * 32) mixer_step_kernel(const Mixe
   }
 }
 
-// out[r, :] = LN(x[r * src_stride + src_offset, :]) in the activation type.
+// out[r, :] = LN(x[r * src_stride + src_offset, :]) in the activation type; with row_len the offset of row r
+// is row_len[r] - 1 (the last position of a sample of that length).
 template <int NV, typename WT>
 __global__ void __launch_bounds__(kMixerWarps * 32)
 norm_rows_kernel(const float* __restrict__ x, int64_t R, int64_t src_stride, int64_t src_offset,
                  const float* __restrict__ g, const float* __restrict__ b, float eps, int d,
-                 WT* __restrict__ out) {
+                 WT* __restrict__ out, const int32_t* __restrict__ row_len) {
   pdl_trigger();
   pdl_wait();
   const int lane = threadIdx.x & 31;
   const int64_t row = (int64_t)blockIdx.x * kMixerWarps + (threadIdx.x >> 5);
   if (row >= R) return;
+  if (row_len != nullptr) src_offset = min(max((int64_t)row_len[row], (int64_t)1), src_stride) - 1;
   const float* xr = x + (row * src_stride + src_offset) * d;
   float4 v[NV];
 #pragma unroll

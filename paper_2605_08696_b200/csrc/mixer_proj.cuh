@@ -22,6 +22,8 @@ struct MixProjParams {
   int t;                 // decode: position
   int n;                 // prefill: prompt length
   const int32_t* ctr;    // decode: device-side step counters, or nullptr: then `t` is the position
+  const int32_t* pos;    // decode: [R] per-row positions, or nullptr; prefill: [R] prompt lengths (<= n), or nullptr
+  uint32_t* status;      // device status word (a prompt length outside [1, n] is clamped and flagged)
 };
 
 constexpr int kMixProjThreads = 256;
@@ -58,7 +60,7 @@ __global__ void __launch_bounds__(kMixProjThreads) mixer_proj_step_kernel(const 
   const int64_t r = vec / vpr;
   const int c = (int)(vec % vpr) * 4;
   const int g = c / (p.d / p.h);
-  const int t = p.ctr != nullptr ? p.ctr[kCtrPos] : p.t;
+  const int t = p.pos != nullptr ? min(max(p.pos[r], 0), p.n_ctx - 1) : (p.ctr != nullptr ? p.ctr[kCtrPos] : p.t);
   const float al = __ldg(p.alpha + (int64_t)g * p.n_ctx + t), lm = __ldg(p.lam + g);
   const float4 bt = ldg4(p.beta + (int64_t)t * p.d + c);
   const float4 q = ld4(p.q + r * p.d + c);
@@ -104,8 +106,10 @@ __global__ void __launch_bounds__(kMixProjThreads) mixer_proj_prefill_kernel(con
   for (int k = 1; k < T; ++k) lp[k] = lp[k - 1] * lm;
   const float* al = p.alpha + (int64_t)g * p.n_ctx;
   float4 carry = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int j0 = 0; j0 < p.n; j0 += T) {
-    const int rows = min(T, p.n - j0);
+  const int nb = p.pos != nullptr ? min(max(p.pos[b], 1), p.n) : p.n;      // this sample's length; rows stay n apart
+  if (p.pos != nullptr && c == 0 && p.pos[b] != nb) raise_status(p.status, kStatusTokenRange);
+  for (int j0 = 0; j0 < nb; j0 += T) {
+    const int rows = min(T, nb - j0);
     float4 u[T];
     float a[T];
 #pragma unroll
@@ -140,6 +144,8 @@ __global__ void __launch_bounds__(kMixProjThreads) mixer_proj_prefill_kernel(con
       }
     }
   }
+  for (int j = nb; j < p.n; ++j)          // positions beyond the sample's length: defined values for the GEMM that follows
+    st4(reinterpret_cast<WT*>(p.y) + (b * p.n + j) * p.d + c, make_float4(0.f, 0.f, 0.f, 0.f));
   st4(reinterpret_cast<ST*>(p.S) + b * p.d + c, carry);
 }
 

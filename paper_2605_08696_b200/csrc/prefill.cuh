@@ -34,6 +34,7 @@ struct PrefillParams {
   int n, d, h, n_ctx, vocab;
   float eps;
   uint32_t* status;
+  const int32_t* len;    // [Bp] prompt lengths (1 .. n; rows of a sample stay n apart), or nullptr: all prompts have n tokens
 };
 
 template <typename WT, typename ST>
@@ -47,9 +48,17 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_mixer_kernel(const Pr
   __shared__ float mu[T], rs[T];                      // LN1 statistics of the tile's rows
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int d = p.d, n = p.n, h = p.h, dh = d / h, h_row = h >> 1;
+  const int d = p.d, stride = p.n, h = p.h, dh = d / h, h_row = h >> 1;
   const int64_t b = blockIdx.x;
   if (b >= p.Bp) return;
+  int n = stride;                                      // positions of this sample
+  if (p.len != nullptr) {
+    n = p.len[b];
+    if (n < 1 || n > stride) {
+      if (tid == 0) raise_status(p.status, kStatusTokenRange);
+      n = n < 1 ? 1 : stride;
+    }
+  }
 
   for (int i = tid; i < h * (T + 1); i += kPrefillThreads) {
     const int g = i / (T + 1), k = i % (T + 1);
@@ -61,7 +70,7 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_mixer_kernel(const Pr
 
   for (int j0 = 0; j0 < n; j0 += T) {
     const int rows = min(T, n - j0);
-    const int64_t row0 = b * n + j0;
+    const int64_t row0 = b * stride + j0;
     __syncthreads();     // previous tile fully written back before xs / Mt are overwritten
     // ---- load the tile (embedding rows for the first layer) ----
     if (p.tok != nullptr) {
@@ -169,6 +178,11 @@ __global__ void __launch_bounds__(kPrefillThreads) prefill_mixer_kernel(const Pr
         st4(ao + c, norm4(v, mean, rstd, ldg4(p.ln2_g + c), ldg4(p.ln2_b + c)));
       }
     }
+  }
+  // positions beyond the sample's length: defined values for the GEMMs that follow (their results are not used)
+  for (int64_t i = (int64_t)tid * 4; i < (int64_t)(stride - n) * d; i += kPrefillThreads * 4) {
+    st4(p.x + (b * stride + n) * d + i, make_float4(0.f, 0.f, 0.f, 0.f));
+    st4(reinterpret_cast<WT*>(p.a) + (b * stride + n) * d + i, make_float4(0.f, 0.f, 0.f, 0.f));
   }
   ST* So = reinterpret_cast<ST*>(p.S) + b * d;
 #pragma unroll

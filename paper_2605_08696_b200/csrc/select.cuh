@@ -19,12 +19,14 @@ struct SelectOut {
   int64_t store_col;
   int64_t row_div;      // output row r reads logits row r / row_div (replicas of one prompt share a row); >= 1
   const int32_t* ctr;   // device-side step counters (store column, Philox step), or nullptr: host values apply
+  int32_t* pos;         // [R] per-row positions, advanced by one with every selection, or nullptr
 };
 
 __device__ __forceinline__ void write_token(const SelectOut& o, int64_t row, int tok) {
   o.last_tok[row] = tok;
   if (o.tok_out != nullptr) o.tok_out[row] = tok;
   if (o.store != nullptr) o.store[row * o.store_stride + (o.ctr != nullptr ? (int64_t)o.ctr[kCtrCol] : o.store_col)] = tok;
+  if (o.pos != nullptr) o.pos[row] += 1;
 }
 
 // ---- greedy -------------------------------------------------------------------------------

@@ -215,8 +215,10 @@ struct srm_state {
   size_t nbytes;
   uint32_t* status;       // device status word (header)
   int32_t* last_tok;      // [B]
+  int32_t* pos_dev;       // [B] per-sample positions, used after srm_prefill_ragged
   uint8_t* S;             // [L, B, d] in state dtype
-  int64_t pos;
+  int64_t pos;            // position of the next token (ragged: of the longest sample)
+  bool ragged = false;    // samples have their own positions (pos_dev)
 
   void* layer_ptr(int l) const { return S + (size_t)l * B * m->cfg.d_model * m->state_bytes(); }
 };
@@ -245,7 +247,7 @@ constexpr size_t kStateHeader = 256;
 
 size_t state_bytes_for(const srm_config& c, int64_t B) {
   const size_t sb = c.state_dtype == SRM_DTYPE_BF16 ? 2 : 4;
-  return kStateHeader + align_up((size_t)B * 4, 256) + (size_t)c.n_layers * B * c.d_model * sb;
+  return kStateHeader + 2 * align_up((size_t)B * 4, 256) + (size_t)c.n_layers * B * c.d_model * sb;
 }
 
 // ---- workspace carving ----------------------------------------------------------------------
@@ -338,7 +340,9 @@ template <typename WT, typename ST>
 int launch_mixer_nv(const MixerParams& p, int num_sms, cudaStream_t st) {
   const int nv = (p.d + 127) / 128;
   // whole 128-channel vectors per lane, each inside one head: the streaming kernel
-  const bool fast = p.d % 128 == 0 && (p.d / p.h) % 128 == 0 && p.h <= 8 && mixer_stream_warps(p.d, (int)sizeof(ST)) >= 1;
+  // (one position for all rows: the streaming kernel stages that position's parameters once per CTA)
+  const bool fast = p.pos == nullptr && p.d % 128 == 0 && (p.d / p.h) % 128 == 0 && p.h <= 8 &&
+                    mixer_stream_warps(p.d, (int)sizeof(ST)) >= 1;
   if (fast && nv == 4) return launch_mixer_stream<4, WT, ST>(p, num_sms, st);
   if (fast && nv == 8) return launch_mixer_stream<8, WT, ST>(p, num_sms, st);
   if (fast && nv == 12) return launch_mixer_stream<12, WT, ST>(p, num_sms, st);
@@ -356,7 +360,7 @@ int launch_mixer_nv(const MixerParams& p, int num_sms, cudaStream_t st) {
 }
 
 int launch_mixer(const srm_model& m, int layer, int t, int64_t R, const int32_t* tok, float* x, void* S, void* a,
-                 uint32_t* status, cudaStream_t st, const int32_t* ctr = nullptr) {
+                 uint32_t* status, cudaStream_t st, const int32_t* ctr = nullptr, const int32_t* pos = nullptr) {
   if (R <= 0) return SRM_OK;
   LaunchScope scope(m, SRM_KERNEL_MIXER, st);
   MixerParams p;
@@ -365,7 +369,7 @@ int launch_mixer(const srm_model& m, int layer, int t, int64_t R, const int32_t*
   p.ln2_g = m.fptr(layer, SRM_T_LN2_G); p.ln2_b = m.fptr(layer, SRM_T_LN2_B);
   p.alpha = m.fptr(layer, SRM_T_ALPHA); p.beta = m.fptr(layer, SRM_T_BETA); p.lam = m.fptr(layer, SRM_T_LAMBDA);
   p.R = R; p.d = m.cfg.d_model; p.h = m.cfg.n_heads; p.n_ctx = m.cfg.n_ctx; p.t = t; p.vocab = m.cfg.vocab;
-  p.eps = m.cfg.ln_eps; p.status = status; p.ctr = ctr;
+  p.eps = m.cfg.ln_eps; p.status = status; p.ctr = ctr; p.pos = pos;
   const bool wb = m.cfg.dtype == SRM_DTYPE_BF16, sb = m.cfg.state_dtype == SRM_DTYPE_BF16;
   if (wb && sb) return launch_mixer_nv<bf16, bf16>(p, m.num_sms, st);
   if (wb) return launch_mixer_nv<bf16, float>(p, m.num_sms, st);
@@ -375,18 +379,18 @@ int launch_mixer(const srm_model& m, int layer, int t, int64_t R, const int32_t*
 
 template <typename WT>
 int launch_norm_t(const float* x, int64_t R, int64_t stride, int64_t offset, const float* g, const float* b, float eps,
-                  int d, void* out, cudaStream_t st) {
+                  int d, void* out, cudaStream_t st, const int32_t* row_len = nullptr) {
   const int nv = (d + 127) / 128;
   const unsigned grid = (unsigned)((R + kMixerWarps - 1) / kMixerWarps);
   const dim3 blk(kMixerWarps * 32);
   WT* o = reinterpret_cast<WT*>(out);
-  if (nv <= 1) SRM_CUDA(launch_kernel(norm_rows_kernel<1, WT>, dim3(grid), dim3(blk), 0, st, x, R, stride, offset, g, b, eps, d, o));
-  else if (nv <= 2) SRM_CUDA(launch_kernel(norm_rows_kernel<2, WT>, dim3(grid), dim3(blk), 0, st, x, R, stride, offset, g, b, eps, d, o));
-  else if (nv <= 4) SRM_CUDA(launch_kernel(norm_rows_kernel<4, WT>, dim3(grid), dim3(blk), 0, st, x, R, stride, offset, g, b, eps, d, o));
-  else if (nv <= 6) SRM_CUDA(launch_kernel(norm_rows_kernel<6, WT>, dim3(grid), dim3(blk), 0, st, x, R, stride, offset, g, b, eps, d, o));
-  else if (nv <= 8) SRM_CUDA(launch_kernel(norm_rows_kernel<8, WT>, dim3(grid), dim3(blk), 0, st, x, R, stride, offset, g, b, eps, d, o));
-  else if (nv <= 12) SRM_CUDA(launch_kernel(norm_rows_kernel<12, WT>, dim3(grid), dim3(blk), 0, st, x, R, stride, offset, g, b, eps, d, o));
-  else SRM_CUDA(launch_kernel(norm_rows_kernel<16, WT>, dim3(grid), dim3(blk), 0, st, x, R, stride, offset, g, b, eps, d, o));
+  if (nv <= 1) SRM_CUDA(launch_kernel(norm_rows_kernel<1, WT>, dim3(grid), dim3(blk), 0, st, x, R, stride, offset, g, b, eps, d, o, row_len));
+  else if (nv <= 2) SRM_CUDA(launch_kernel(norm_rows_kernel<2, WT>, dim3(grid), dim3(blk), 0, st, x, R, stride, offset, g, b, eps, d, o, row_len));
+  else if (nv <= 4) SRM_CUDA(launch_kernel(norm_rows_kernel<4, WT>, dim3(grid), dim3(blk), 0, st, x, R, stride, offset, g, b, eps, d, o, row_len));
+  else if (nv <= 6) SRM_CUDA(launch_kernel(norm_rows_kernel<6, WT>, dim3(grid), dim3(blk), 0, st, x, R, stride, offset, g, b, eps, d, o, row_len));
+  else if (nv <= 8) SRM_CUDA(launch_kernel(norm_rows_kernel<8, WT>, dim3(grid), dim3(blk), 0, st, x, R, stride, offset, g, b, eps, d, o, row_len));
+  else if (nv <= 12) SRM_CUDA(launch_kernel(norm_rows_kernel<12, WT>, dim3(grid), dim3(blk), 0, st, x, R, stride, offset, g, b, eps, d, o, row_len));
+  else SRM_CUDA(launch_kernel(norm_rows_kernel<16, WT>, dim3(grid), dim3(blk), 0, st, x, R, stride, offset, g, b, eps, d, o, row_len));
   SRM_CUDA(cudaGetLastError());
   return SRM_OK;
 }
@@ -401,13 +405,13 @@ int launch_norm(const srm_model& m, const float* x, int64_t R, int64_t stride, i
 }
 
 int launch_final_norm(const srm_model& m, const float* x, int64_t R, int64_t stride, int64_t offset, void* out,
-                      cudaStream_t st) {
+                      cudaStream_t st, const int32_t* row_len = nullptr) {
   if (R <= 0) return SRM_OK;
   LaunchScope scope(m, SRM_KERNEL_NORM, st);
   const float* g = m.fptr(-1, SRM_T_LNF_G);
   const float* b = m.fptr(-1, SRM_T_LNF_B);
-  if (m.cfg.dtype == SRM_DTYPE_BF16) return launch_norm_t<bf16>(x, R, stride, offset, g, b, m.cfg.ln_eps, m.cfg.d_model, out, st);
-  return launch_norm_t<float>(x, R, stride, offset, g, b, m.cfg.ln_eps, m.cfg.d_model, out, st);
+  if (m.cfg.dtype == SRM_DTYPE_BF16) return launch_norm_t<bf16>(x, R, stride, offset, g, b, m.cfg.ln_eps, m.cfg.d_model, out, st, row_len);
+  return launch_norm_t<float>(x, R, stride, offset, g, b, m.cfg.ln_eps, m.cfg.d_model, out, st, row_len);
 }
 
 template <typename T>
@@ -560,7 +564,7 @@ int launch_lm_head_greedy(srm_model& m, int64_t R, const void* a, void* part, co
 }
 
 int launch_prefill_mixer(const srm_model& m, int layer, int64_t Bp, int n, const int32_t* tok, float* x, void* S,
-                         void* a, uint32_t* status, cudaStream_t st) {
+                         void* a, uint32_t* status, cudaStream_t st, const int32_t* len = nullptr) {
   if (Bp <= 0) return SRM_OK;
   LaunchScope scope(m, SRM_KERNEL_PREFILL_MIXER, st);
   PrefillParams p;
@@ -569,7 +573,7 @@ int launch_prefill_mixer(const srm_model& m, int layer, int64_t Bp, int n, const
   p.ln2_g = m.fptr(layer, SRM_T_LN2_G); p.ln2_b = m.fptr(layer, SRM_T_LN2_B);
   p.alpha = m.fptr(layer, SRM_T_ALPHA); p.beta = m.fptr(layer, SRM_T_BETA); p.lam = m.fptr(layer, SRM_T_LAMBDA);
   p.Bp = Bp; p.n = n; p.d = m.cfg.d_model; p.h = m.cfg.n_heads; p.n_ctx = m.cfg.n_ctx; p.vocab = m.cfg.vocab;
-  p.eps = m.cfg.ln_eps; p.status = status;
+  p.eps = m.cfg.ln_eps; p.status = status; p.len = len;
   const size_t smem = (size_t)kPrefillTile * m.cfg.d_model * 4;
   const bool wb = m.cfg.dtype == SRM_DTYPE_BF16, sb = m.cfg.state_dtype == SRM_DTYPE_BF16;
   auto go = [&](auto kernel) -> int {
@@ -598,7 +602,7 @@ int launch_mix_proj_t(bool prefill, const MixProjParams& p, int64_t vecs, cudaSt
 
 int launch_mixer_block_proj(srm_model& m, int layer, int t, int64_t rows, int64_t samples, int n, const int32_t* tok,
                             float* x, void* S, void* a, float* q, uint32_t* status, cudaStream_t st,
-                            const int32_t* ctr = nullptr) {
+                            const int32_t* ctr = nullptr, const int32_t* pos = nullptr) {
   if (rows <= 0) return SRM_OK;
   const srm_config& c = m.cfg;
   const int d = c.d_model;
@@ -622,6 +626,8 @@ int launch_mixer_block_proj(srm_model& m, int layer, int t, int64_t rows, int64_
     p.alpha = m.fptr(layer, SRM_T_ALPHA); p.beta = m.fptr(layer, SRM_T_BETA); p.lam = m.fptr(layer, SRM_T_LAMBDA);
     p.R = prefill ? samples : rows; p.d = d; p.h = c.n_heads; p.n_ctx = c.n_ctx; p.t = prefill ? 0 : t; p.n = n;
     p.ctr = prefill ? nullptr : ctr;
+    p.pos = pos;                                   // decode: per-row positions; prefill: prompt lengths
+    p.status = status;
     const int64_t vecs = p.R * (d / 4);
     if (wb && sb) rc = launch_mix_proj_t<bf16, bf16>(prefill, p, vecs, st);
     else if (wb) rc = launch_mix_proj_t<bf16, float>(prefill, p, vecs, st);
@@ -640,13 +646,14 @@ int decode_chunk(srm_model& m, srm_state& s, int64_t b0, int64_t R, const int32_
   const srm_config& c = m.cfg;
   const int d = c.d_model;
   const int64_t F = m.F();
-  const int t = (int)s.pos;
+  const int t = (int)(s.pos < c.n_ctx ? s.pos : c.n_ctx - 1);
+  const int32_t* pos = s.ragged ? s.pos_dev + b0 : nullptr;       // samples of different lengths: a position per row
   int rc;
   for (int l = 0; l < c.n_layers; ++l) {
     uint8_t* Sl = static_cast<uint8_t*>(s.layer_ptr(l)) + (size_t)b0 * d * m.state_bytes();
     if (m.head_proj()) {
-      if ((rc = launch_mixer_block_proj(m, l, t, R, R, 1, l == 0 ? tok_in + b0 : nullptr, w.x, Sl, w.a, w.q, s.status, st, ctr))) return rc;
-    } else if ((rc = launch_mixer(m, l, t, R, l == 0 ? tok_in + b0 : nullptr, w.x, Sl, w.a, s.status, st, ctr))) return rc;
+      if ((rc = launch_mixer_block_proj(m, l, t, R, R, 1, l == 0 ? tok_in + b0 : nullptr, w.x, Sl, w.a, w.q, s.status, st, ctr, pos))) return rc;
+    } else if ((rc = launch_mixer(m, l, t, R, l == 0 ? tok_in + b0 : nullptr, w.x, Sl, w.a, s.status, st, ctr, pos))) return rc;
     if ((rc = launch_gemm(m, kEpiBiasGelu, R, F, d, w.a, m.ptr(l, SRM_T_W1), m.fptr(l, SRM_T_B1), w.H, s.status, st))) return rc;
     if ((rc = launch_gemm(m, kEpiBiasResidual, R, d, F, w.H, m.ptr(l, SRM_T_W2), m.fptr(l, SRM_T_B2), w.x, s.status, st))) return rc;
   }
@@ -655,6 +662,7 @@ int decode_chunk(srm_model& m, srm_state& s, int64_t b0, int64_t R, const int32_
   o.last_tok += b0;
   if (o.tok_out) o.tok_out += b0;
   if (o.store) o.store += b0 * o.store_stride;
+  if (o.pos) o.pos += b0;
   if (can_fuse_greedy(m, samp, logits_out)) return launch_lm_head_greedy(m, R, w.a, w.logits, o, s.status, st);
   float* lg = logits_out != nullptr ? logits_out + b0 * c.vocab : w.logits;
   if ((rc = launch_gemm(m, kEpiPlain, R, c.vocab, d, w.a, m.ptr(-1, SRM_T_W_LM), nullptr, lg, s.status, st))) return rc;
@@ -674,7 +682,7 @@ int decode_step_impl(srm_model* m, srm_state* s, const int32_t* d_tok_in, const 
   if (rows < 1) return SRM_ERR_BUFFER_TOO_SMALL;
   const DecodeWs w = carve_decode(*m, d_ws, rows);
   const int32_t* tok_in = d_tok_in != nullptr ? d_tok_in : s->last_tok;
-  SelectOut out{s->last_tok, d_tok_out, d_store, store_stride, store_col, 1, ctr};
+  SelectOut out{s->last_tok, d_tok_out, d_store, store_stride, store_col, 1, ctr, s->ragged ? s->pos_dev : nullptr};
   for (int64_t b0 = 0; b0 < s->B; b0 += rows) {
     const int64_t R = (s->B - b0 < rows) ? s->B - b0 : rows;
     if ((rc = decode_chunk(*m, *s, b0, R, tok_in, *samp, step, out, d_logits_out, w, st, ctr))) return rc;
@@ -803,7 +811,8 @@ int srm_state_create(srm_model* m, int64_t B, void* d_state, size_t nbytes, void
   s->m = m; s->B = B; s->base = static_cast<uint8_t*>(d_state); s->nbytes = state_bytes_for(m->cfg, B);
   s->status = reinterpret_cast<uint32_t*>(s->base);
   s->last_tok = reinterpret_cast<int32_t*>(s->base + kStateHeader);
-  s->S = s->base + kStateHeader + align_up((size_t)B * 4, 256);
+  s->pos_dev = reinterpret_cast<int32_t*>(s->base + kStateHeader + align_up((size_t)B * 4, 256));
+  s->S = s->base + kStateHeader + 2 * align_up((size_t)B * 4, 256);
   s->pos = 0;
   int rc = srm_state_reset(s, stream);
   if (rc != SRM_OK) { delete s; return rc; }
@@ -825,6 +834,7 @@ int srm_state_reset(srm_state* s, void* stream) {
   if (s == nullptr) return SRM_ERR_INVALID_ARG;
   SRM_CUDA(cudaMemsetAsync(s->base, 0, s->nbytes, static_cast<cudaStream_t>(stream)));
   s->pos = 0;
+  s->ragged = false;
   return SRM_OK;
 }
 
@@ -832,6 +842,7 @@ int64_t srm_state_pos(const srm_state* s) { return s ? s->pos : -1; }
 
 int srm_state_set_pos(srm_state* s, int64_t pos) {
   if (s == nullptr || pos < 0 || pos > s->m->cfg.n_ctx) return SRM_ERR_INVALID_ARG;
+  if (s->ragged) return SRM_ERR_INVALID_ARG;            // the positions live on the device, one per sample
   s->pos = pos;
   return SRM_OK;
 }
@@ -864,7 +875,7 @@ namespace {
 // selects its own first token from the prompt's last-position logits.
 int prefill_impl(srm_model* m, srm_state* s, const int32_t* d_tokens, int64_t P, int32_t n, int64_t replicas,
                  const srm_sampling* samp, int32_t* d_first_tok, float* d_logits_last, void* d_ws, size_t ws_bytes,
-                 cudaStream_t st) {
+                 cudaStream_t st, const int32_t* d_len = nullptr) {
   const srm_config& c = m->cfg;
   const int d = c.d_model;
   const int64_t F = m->F();
@@ -885,8 +896,10 @@ int prefill_impl(srm_model* m, srm_state* s, const int32_t* d_tokens, int64_t P,
       uint8_t* Sl = replicas > 1 ? stage + (size_t)l * np * row_bytes
                                  : static_cast<uint8_t*>(s->layer_ptr(l)) + (size_t)b0 * row_bytes;
       if (m->head_proj()) {
-        if ((rc = launch_mixer_block_proj(*m, l, -1, rows, np, n, l == 0 ? d_tokens + p0 * n : nullptr, w.x, Sl, w.a, w.q, s->status, st))) return rc;
-      } else if ((rc = launch_prefill_mixer(*m, l, np, n, l == 0 ? d_tokens + p0 * n : nullptr, w.x, Sl, w.a, s->status, st))) return rc;
+        if ((rc = launch_mixer_block_proj(*m, l, -1, rows, np, n, l == 0 ? d_tokens + p0 * n : nullptr, w.x, Sl, w.a, w.q, s->status, st,
+                                          nullptr, d_len ? d_len + p0 : nullptr))) return rc;
+      } else if ((rc = launch_prefill_mixer(*m, l, np, n, l == 0 ? d_tokens + p0 * n : nullptr, w.x, Sl, w.a, s->status, st,
+                                            d_len ? d_len + p0 : nullptr))) return rc;
       if ((rc = launch_gemm(*m, kEpiBiasGelu, rows, F, d, w.a, m->ptr(l, SRM_T_W1), m->fptr(l, SRM_T_B1), w.H, s->status, st))) return rc;
       if ((rc = launch_gemm(*m, kEpiBiasResidual, rows, d, F, w.H, m->ptr(l, SRM_T_W2), m->fptr(l, SRM_T_B2), w.x, s->status, st))) return rc;
       if (replicas > 1) {
@@ -898,7 +911,7 @@ int prefill_impl(srm_model* m, srm_state* s, const int32_t* d_tokens, int64_t P,
       }
     }
     // LM head on the last prompt position only; selection per state row
-    if ((rc = launch_final_norm(*m, w.x, np, n, n - 1, w.a_last, st))) return rc;
+    if ((rc = launch_final_norm(*m, w.x, np, n, n - 1, w.a_last, st, d_len ? d_len + p0 : nullptr))) return rc;
     SelectOut o{s->last_tok + b0, d_first_tok ? d_first_tok + b0 : nullptr, nullptr, 0, 0, replicas};
     if (replicas == 1 && can_fuse_greedy(*m, *samp, d_logits_last)) {
       if ((rc = launch_lm_head_greedy(*m, np, w.a_last, w.logits, o, s->status, st))) return rc;
@@ -909,6 +922,11 @@ int prefill_impl(srm_model* m, srm_state* s, const int32_t* d_tokens, int64_t P,
     if ((rc = launch_select(*m, nb, lg, *samp, samp->sample_idx_base + (uint64_t)b0, 0, o, s->status, st))) return rc;
   }
   s->pos = n;
+  if (d_len != nullptr) {
+    // from here on every sample has its own position: its prompt length (srm_prefill_ragged checked replicas == 1)
+    SRM_CUDA(cudaMemcpyAsync(s->pos_dev, d_len, (size_t)s->B * 4, cudaMemcpyDeviceToDevice, st));
+    s->ragged = true;
+  }
   return SRM_OK;
 }
 
@@ -933,6 +951,17 @@ int srm_prefill(srm_model* m, srm_state* s, const int32_t* d_tokens, int32_t n, 
   if (rc) return rc;
   return prefill_impl(m, s, d_tokens, s->B, n, 1, samp, d_first_tok, d_logits_last, d_ws, ws_bytes,
                       static_cast<cudaStream_t>(stream));
+}
+
+int srm_prefill_ragged(srm_model* m, srm_state* s, const int32_t* d_tokens, int32_t n_max, const int32_t* d_lengths,
+                       const srm_sampling* samp, int32_t* d_first_tok, float* d_logits_last, void* d_ws, size_t ws_bytes,
+                       void* stream) {
+  int rc = prefill_check(m, s, d_tokens, n_max, samp, d_first_tok, d_logits_last, d_ws);
+  if (rc) return rc;
+  if (d_lengths == nullptr) return SRM_ERR_INVALID_ARG;
+  if (!aligned(d_lengths, 4)) return SRM_ERR_ALIGNMENT;
+  return prefill_impl(m, s, d_tokens, s->B, n_max, 1, samp, d_first_tok, d_logits_last, d_ws, ws_bytes,
+                      static_cast<cudaStream_t>(stream), d_lengths);
 }
 
 int srm_prefill_replicated(srm_model* m, srm_state* s, const int32_t* d_tokens, int32_t n_prompts, int32_t n,

@@ -1,0 +1,141 @@
+"""Prompts of different lengths in one batch (srm_prefill_ragged, then the ordinary step calls with one
+position per sample kept on the device): every sample must behave as if it had been prefilled and decoded
+alone. Checked against the oracle run sample by sample (each with its own length and positions), and against
+the device's own single-sample runs."""
+import numpy as np
+import pytest
+import torch
+
+import srm_inputs as I
+from helpers import oracle_for, rel_err_rows, top2_margin
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+TOL = {"fp32": 1e-4, "bf16": 3e-2}
+
+
+def _ragged_batch(shape, lengths, seed):
+    n_max = max(lengths)
+    toks = I.uniform_prompts(len(lengths), n_max, shape.vocab, seed=seed)
+    for b, n in enumerate(lengths):
+        toks[b, n:] = (7 * b + 3) % shape.vocab           # padding: valid ids that must not matter
+    return toks
+
+
+@pytest.mark.parametrize("name,lengths,gen", [
+    ("tiny", [8, 3, 5, 1, 8, 6], 12),                     # fp32, d 64: 1e-4
+    ("small", [40, 17, 33, 9, 40, 1, 25], 6),             # bf16, d 512, several position tiles and a ragged last tile
+])
+def test_ragged_batch_matches_the_oracle_run_sample_by_sample(name, lengths, gen):
+    import paper_2605_08696_b200 as P
+    shape = I.CONFIGS[name]
+    W = I.make_weights(shape)
+    model = P.SRM(shape, W, device=DEV)
+    orc = oracle_for(shape, W)
+    B, n_max = len(lengths), max(lengths)
+    toks = _ragged_batch(shape, lengths, seed=17)
+    st = model.new_state(B)
+    ws = model.new_workspace(B, n_max, prefill_samples=B)
+    g = P.Sampling("greedy")
+    lens_dev = torch.tensor(lengths, dtype=torch.int32, device=DEV)
+    tok, lg = model.prefill_ragged(st, torch.from_numpy(toks).to(DEV), lens_dev, g, ws, want_logits=True)
+    assert st.pos == n_max
+    # the oracle, one sample at a time, fed the device's tokens (teacher forcing)
+    states = []
+    worst, checked = 0.0, 0
+    lg_np, tok_np = lg.cpu().numpy(), tok.cpu().numpy()
+    for b, n in enumerate(lengths):
+        lo, so = orc.forward_parallel(toks[b:b + 1, :n])
+        worst = max(worst, rel_err_rows(lg_np[b], lo[0, n - 1]))
+        if top2_margin(lo[0, n - 1]) > 1e-2 + 2 * np.max(np.abs(lg_np[b] - lo[0, n - 1])):
+            assert tok_np[b] == int(np.argmax(lo[0, n - 1]))
+            checked += 1
+        states.append(so)
+    for k in range(gen):
+        tok_in = tok_np.copy()
+        tok, lg = model.decode_step(st, None, g, k + 1, ws, want_logits=True)
+        lg_np, tok_np = lg.cpu().numpy(), tok.cpu().numpy()
+        for b, n in enumerate(lengths):
+            lo, states[b] = orc.decode_step(states[b], tok_in[b:b + 1], n + k)      # this sample's own position
+            worst = max(worst, rel_err_rows(lg_np[b], lo[0]))
+            if top2_margin(lo[0]) > 1e-2 + 2 * np.max(np.abs(lg_np[b] - lo[0])):
+                assert tok_np[b] == int(np.argmax(lo[0]))
+                checked += 1
+    assert worst < TOL[shape.dtype], worst
+    assert checked > 0.5 * B * (gen + 1)
+    cache = st.cache().cpu().numpy()
+    for b in range(B):
+        assert rel_err_rows(cache[:, b], states[b][:, 0]) < TOL[shape.dtype]
+    assert st.pos == n_max + gen and st.status() == 0
+
+
+@pytest.mark.parametrize("sampling", ["greedy", "topk"])
+def test_ragged_batch_equals_single_sample_runs_on_the_device(sampling):
+    """Same kernels, same arithmetic: sample b of the ragged batch and a batch of one holding only that prompt
+    (same Philox sample index) give the same tokens and the same cache, bit for bit; the uniform API on that
+    prompt agrees to rounding (it may take the streaming mixer kernel, whose LayerNorm sums run in another
+    order)."""
+    import paper_2605_08696_b200 as P
+    shape = I.CONFIGS["small"]
+    W = I.make_weights(shape)
+    model = P.SRM(shape, W, device=DEV)
+    lengths = [31, 8, 19, 31, 2]
+    B, n_max, gen = len(lengths), max(lengths), 8
+    toks = _ragged_batch(shape, lengths, seed=23)
+    mk = (lambda base: P.Sampling("greedy")) if sampling == "greedy" else \
+        (lambda base: P.Sampling("topk", 50, 0.8, seed=9, sample_idx_base=base))
+    st = model.new_state(B)
+    ws = model.new_workspace(B, n_max, prefill_samples=B)
+    lens_dev = torch.tensor(lengths, dtype=torch.int32, device=DEV)
+    first = model.prefill_ragged(st, torch.from_numpy(toks).to(DEV), lens_dev, mk(100), ws).clone()
+    rest = model.generate(st, gen, 1, mk(100), ws)               # the generation loop (graph or launches) works on it too
+    got = torch.cat([first[:, None], rest], 1).cpu().numpy()
+    cache = st.cache()
+    for b, n in enumerate(lengths):
+        s1 = model.new_state(1)
+        w1 = model.new_workspace(1, n, prefill_samples=1)
+        t1 = torch.from_numpy(toks[b:b + 1, :n].copy()).to(DEV)
+        f1 = model.prefill_ragged(s1, t1, lens_dev[b:b + 1].clone(), mk(100 + b), w1).clone()
+        r1 = model.generate(s1, gen, 1, mk(100 + b), w1)
+        alone = torch.cat([f1[:, None], r1], 1).cpu().numpy()[0]
+        assert np.array_equal(got[b], alone), (b, got[b], alone)
+        assert torch.equal(cache[:, b], s1.cache()[:, 0])
+        assert s1.pos == n + gen
+        # the uniform API on the same prompt: same first-token logits up to rounding
+        s2 = model.new_state(1)
+        _, lg_u = model.prefill(s2, t1, mk(100 + b), w1, want_logits=True)
+        s3 = model.new_state(1)
+        _, lg_r = model.prefill_ragged(s3, t1, lens_dev[b:b + 1].clone(), mk(100 + b), w1, want_logits=True)
+        assert rel_err_rows(lg_r.cpu().numpy(), lg_u.cpu().numpy()) < 1e-3
+    assert st.pos == n_max + gen and st.status() == 0
+
+
+def test_ragged_with_head_projections_and_argument_checks():
+    import dataclasses
+    import paper_2605_08696_b200 as P
+    shape = dataclasses.replace(I.CONFIGS["small"], head_proj=True)
+    W = I.make_weights(shape)
+    model = P.SRM(shape, W, device=DEV)
+    orc = oracle_for(shape, W)
+    lengths = [12, 5, 9]
+    B, n_max = 3, 12
+    toks = _ragged_batch(shape, lengths, seed=29)
+    st = model.new_state(B)
+    ws = model.new_workspace(B, n_max, prefill_samples=B)
+    g = P.Sampling("greedy")
+    lens_dev = torch.tensor(lengths, dtype=torch.int32, device=DEV)
+    tok, lg = model.prefill_ragged(st, torch.from_numpy(toks).to(DEV), lens_dev, g, ws, want_logits=True)
+    tok2, lg2 = model.decode_step(st, None, g, 1, ws, want_logits=True)
+    for b, n in enumerate(lengths):
+        lo, so = orc.forward_parallel(toks[b:b + 1, :n])
+        assert rel_err_rows(lg.cpu().numpy()[b], lo[0, n - 1]) < 3e-2
+        lo2, _ = orc.decode_step(so, tok.cpu().numpy()[b:b + 1], n)
+        assert rel_err_rows(lg2.cpu().numpy()[b], lo2[0]) < 3e-2
+    # positions live on the device now
+    with pytest.raises(P.SRMError):
+        st.pos = 3
+    # a length outside [1, n_max] is clamped and reported
+    st_bad = model.new_state(B)
+    bad = torch.tensor([12, 0, 40], dtype=torch.int32, device=DEV)
+    model.prefill_ragged(st_bad, torch.from_numpy(toks).to(DEV), bad, g, ws)
+    assert st_bad.status() & 1
