@@ -282,13 +282,22 @@ def run_ours(args):
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sync_all()
     prefill_ms = None
+    lengths = None
+    if args.ragged:                          # a serving mix: prompt lengths uniform on [n/2, n], one position per sample
+        import numpy as np
+        rng = np.random.Generator(np.random.Philox(key=shape.seed + 77))
+        lengths = torch.from_numpy(rng.integers(n // 2, n + 1, size=B).astype(np.int32)).to(dev)
+        if args.no_prefill:
+            raise SystemExit("--ragged needs the prefill (it sets the per-sample positions)")
     if args.no_prefill:                      # profiling aid: decode cost does not depend on the cache contents
         st.pos = n
     else:
         replicated = w["prompts"] == "replicated" and B % w["n_prompts"] == 0 and not args.no_prompt_dedup
 
         def do_prefill():
-            if replicated:                   # each distinct prompt runs once, its cache is copied to its replicas
+            if lengths is not None:
+                model.prefill_ragged(st, prompts, lengths, samp, ws)
+            elif replicated:                   # each distinct prompt runs once, its cache is copied to its replicas
                 reps = B // w["n_prompts"]
                 model.prefill_replicated(st, prompts[::reps].contiguous(), reps, samp, ws)
             else:
@@ -303,6 +312,15 @@ def run_ours(args):
         torch.cuda.synchronize()
         prefill_ms = e0.elapsed_time(e1)
 
+    def rewind():
+        """Back to the end of the prompt when the context is exhausted (timing only: alpha/beta indices stay in
+        range). Per-sample positions live on the device, so a ragged state is prefilled again instead."""
+        if lengths is not None:
+            st.reset()
+            do_prefill()
+        else:
+            st.pos = n
+
     step_no = [1]
     store = torch.empty(B, shape.n_ctx - n, dtype=torch.int32, device=dev)       # generated-token store
 
@@ -313,7 +331,7 @@ def run_ours(args):
         while k > 0:
             room = shape.n_ctx - st.pos
             if room == 0:
-                st.pos = n
+                rewind()
                 continue
             c = min(k, room)
             model.generate(st, c, step_no[0], samp, ws, out=store)
@@ -340,6 +358,8 @@ def run_ours(args):
     value = whole_job_value(world, B, args.steps, t_ms_max)
 
     # ---- per-kernel durations, CUDA events on the launching stream, same workload ----
+    if lengths is not None and shape.n_ctx - st.pos < args.steps:
+        rewind()
     model.profile_reset()
     model.profile(True)
     run_steps(args.steps)
@@ -366,18 +386,20 @@ def run_ours(args):
     kernels["select"]["gbs"] = round(args.steps * B * V * 4 / (prof["select"][1] / 1e3) / 1e9, 1)
 
     # ---- end to end through the host-buffer call: H2D tokens in, D2H tokens out, every step ----
+    if lengths is not None and shape.n_ctx - st.pos < args.steps + 2:
+        rewind()
     h_in = st.last_token().cpu().pin_memory()
     h_out = torch.empty_like(h_in).pin_memory()
     for _ in range(2):
         if st.pos >= shape.n_ctx:
-            st.pos = n
+            rewind()
         model.decode_step_host(st, h_in, samp, step_no[0], h_out, ws); step_no[0] += 1
         torch.cuda.synchronize(); h_in.copy_(h_out)
     sync_all()
     e0.record()
     for _ in range(args.steps):
         if st.pos >= shape.n_ctx:
-            st.pos = n
+            rewind()
         model.decode_step_host(st, h_in, samp, step_no[0], h_out, ws); step_no[0] += 1
         torch.cuda.current_stream().synchronize()      # the next step's input is this step's output
         h_in.copy_(h_out)
@@ -401,7 +423,7 @@ def run_ours(args):
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if shape.dtype == "bf16" else "f32",
             "data": "synthetic",
             "config": _config_dict(args, shape, w, B, extra={
-                "state_dtype": args.state_dtype, "chunk_rows": chunk, "graph": args.graph,
+                "state_dtype": args.state_dtype, "chunk_rows": chunk, "graph": args.graph, "ragged_prompts": bool(args.ragged),
                 "l2": f"inputs larger than L2: per-step working set (cache {L * B * d * sbytes / 1e6:.0f} MB + weights "
                       f"{model.blob.numel() / 1e6:.0f} MB + logits {chunk * V * 4 / 1e6:.0f} MB) vs 126 MB L2; no flush"}),
             "gpu_launches": int(launches),
@@ -499,6 +521,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--head-proj", action="store_true",
                     help="token mixer with head projections (Eq. 10): adds W_in, W_out [d, d] per layer")
+    ap.add_argument("--ragged", action="store_true",
+                    help="prompt lengths uniform on [n/2, n] (srm_prefill_ragged; one position per sample in the decode steps)")
     ap.add_argument("--top-p", type=float, default=None,
                     help="select tokens by nucleus sampling with this p (temperature 0.7 unless --temperature)")
     ap.add_argument("--temperature", type=float, default=None)

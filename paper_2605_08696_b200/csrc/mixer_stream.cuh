@@ -12,6 +12,9 @@
 //     works on the current one, so with W warps 2W rows (up to 192 KB) are in flight per SM;
 //   - reads a row from shared memory into registers once, and writes x, the cache and the bf16 activation
 //     straight to global memory with 128-bit stores, 512 contiguous bytes per warp instruction.
+// With one position per row (MixerParams::pos, samples of different lengths) beta_t and alpha_t cannot be
+// staged per CTA: each lane fetches its pieces of the row's beta_t (an L2 hit: the table is a few MB) and the
+// head scalars with read-only loads, issued before the row's bulk copy is waited for.
 // Requires d % 128 == 0 and a head width that is a multiple of 128 (every 128-channel vector lies in one
 // head); other shapes take mixer_step_kernel. Every wait is bounded (status bit, then a clean exit).
 #pragma once
@@ -113,6 +116,7 @@ __global__ void __launch_bounds__(kStreamMaxWarps * 32, 1) mixer_stream_kernel(c
   if (lane == 0) { issue(0); issue(1); }
 
   const int c0 = lane * 4;
+  const bool per_row = p.pos != nullptr;
   const int h_row = p.h >> 1;
   const int vph = (d / p.h) >> 7;           // 128-channel vectors per head
   const float inv_d = 1.0f / (float)d;
@@ -121,6 +125,10 @@ __global__ void __launch_bounds__(kStreamMaxWarps * 32, 1) mixer_stream_kernel(c
     const int64_t r = first + (int64_t)j * stride;
     if (r >= p.R) break;
     uint8_t* slot = slots + ((size_t)warp * 2 + (j & 1)) * slot_bytes;
+    // per-row position: its beta row and the head scalars come straight from global memory
+    const int t_r = per_row ? min(max(p.pos[r], 0), p.n_ctx - 1) : 0;
+    const float* beta_r = p.beta + (int64_t)t_r * d + c0;
+    const float* alpha_r = p.alpha + t_r;
     if (!tc::mbar_wait(&bars[warp * 2 + (j & 1)], (uint32_t)(j >> 1) & 1u, p.status)) { ok = false; break; }
 
     float4 v[NV];
@@ -141,10 +149,11 @@ __global__ void __launch_bounds__(kStreamMaxWarps * 32, 1) mixer_stream_kernel(c
     ST* Sg = reinterpret_cast<ST*>(p.S) + r * d + c0;
     float* xg = p.x + r * d + c0;
     int g = 0, left = vph;
-    float al = heads[0], lm = heads[8];
+    float al = per_row ? __ldg(alpha_r) : heads[0], lm = heads[8];
 #pragma unroll
     for (int i = 0; i < NV; ++i) {
-      const float4 gg = ld4(prm + c0 + i * 128), bb = ld4(prm + d + c0 + i * 128), bt = ld4(prm + 2 * d + c0 + i * 128);
+      const float4 gg = ld4(prm + c0 + i * 128), bb = ld4(prm + d + c0 + i * 128);
+      const float4 bt = per_row ? ldg4(beta_r + i * 128) : ld4(prm + 2 * d + c0 + i * 128);
       const float4 s = ld4(Ss + i * 128);
       float4 z;
       z.x = fmaf(fmaf(v[i].x, rstd, nmr), gg.x, bb.x); z.y = fmaf(fmaf(v[i].y, rstd, nmr), gg.y, bb.y);
@@ -164,7 +173,7 @@ __global__ void __launch_bounds__(kStreamMaxWarps * 32, 1) mixer_stream_kernel(c
       st4(xg + i * 128, v[i]);
       if (--left == 0 && i + 1 < NV) {                   // next vector starts the next head
         ++g; left = vph;
-        al = heads[g]; lm = heads[8 + g];
+        al = per_row ? __ldg(alpha_r + (int64_t)g * p.n_ctx) : heads[g]; lm = heads[8 + g];
       }
     }
     // the slot has been read: order these generic-proxy reads before the next bulk copy into it

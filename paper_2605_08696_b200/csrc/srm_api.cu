@@ -340,9 +340,7 @@ template <typename WT, typename ST>
 int launch_mixer_nv(const MixerParams& p, int num_sms, cudaStream_t st) {
   const int nv = (p.d + 127) / 128;
   // whole 128-channel vectors per lane, each inside one head: the streaming kernel
-  // (one position for all rows: the streaming kernel stages that position's parameters once per CTA)
-  const bool fast = p.pos == nullptr && p.d % 128 == 0 && (p.d / p.h) % 128 == 0 && p.h <= 8 &&
-                    mixer_stream_warps(p.d, (int)sizeof(ST)) >= 1;
+  const bool fast = p.d % 128 == 0 && (p.d / p.h) % 128 == 0 && p.h <= 8 && mixer_stream_warps(p.d, (int)sizeof(ST)) >= 1;
   if (fast && nv == 4) return launch_mixer_stream<4, WT, ST>(p, num_sms, st);
   if (fast && nv == 8) return launch_mixer_stream<8, WT, ST>(p, num_sms, st);
   if (fast && nv == 12) return launch_mixer_stream<12, WT, ST>(p, num_sms, st);
