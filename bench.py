@@ -260,7 +260,8 @@ def run_ours(args):
 
     W = I.make_weights(shape)
     model = P.SRM(shape, W, device=dev, state_dtype=args.state_dtype,
-                  flags={"auto": 0, "on": P.FLAG_GRAPH, "off": P.FLAG_NO_GRAPH}[args.graph])
+                  flags={"auto": 0, "on": P.FLAG_GRAPH, "off": P.FLAG_NO_GRAPH}[args.graph] |
+                  (P.FLAG_NO_SPLITK if args.no_splitk else 0))
     sidx0 = rank_plan(rank, world, B)["sample_idx_base"]
     samp = {"greedy": lambda: P.Sampling("greedy"),
             "topk": lambda: P.Sampling("topk", w["top_k"], w["temperature"], seed=shape.seed, sample_idx_base=sidx0),
@@ -521,6 +522,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--head-proj", action="store_true",
                     help="token mixer with head projections (Eq. 10): adds W_in, W_out [d, d] per layer")
+    ap.add_argument("--no-splitk", action="store_true",
+                    help="down projection with whole output tiles per CTA pair (no sharing of K between pairs)")
     ap.add_argument("--ragged", action="store_true",
                     help="prompt lengths uniform on [n/2, n] (srm_prefill_ragged; one position per sample in the decode steps)")
     ap.add_argument("--top-p", type=float, default=None,

@@ -64,6 +64,8 @@ enum {
   SRM_FLAG_GRAPH = 8,                /* srm_generate always replays a captured step (default: only for
                                         batches small enough to be bound by the host's launch rate)     */
   SRM_FLAG_SIMT_GEMM = 1,            /* debug: run the bf16 GEMMs on the plain SIMT kernel  */
+  SRM_FLAG_NO_SPLITK = 16,           /* the down projection of a decode step always gives whole output tiles to a CTA
+                                        pair (see srm_k_gemm_splitk); for comparison and measurement */
   SRM_FLAG_HEAD_PROJ = 2             /* token mixer with head projections [Method/Architecture, Eq. 10]:
                                         q = W_in LN1(x) (W_in stacks the per-head I_g), heads of q mixed, and
                                         x += W_out (concatenated heads); the cache holds projected values.
@@ -278,6 +280,26 @@ int srm_k_final_norm(srm_model* m, int64_t R, const float* d_x, void* d_a, void*
 int srm_k_gemm(srm_model* m, int32_t epilogue, int64_t M, int64_t N, int64_t K, const void* d_A,
                const void* d_W, const float* d_bias, void* d_out, uint32_t* d_status,
                void* stream);
+/* Epilogue 1 of srm_k_gemm (out_f32[M, N] += A W^T + bias, bf16 tensor-core path) with the K dimension shared out
+ * between CTA pairs: the (256 x 256 tile, 64-wide k-block) sequence is cut into one contiguous range per pair, so
+ * that no pair idles when the tile count is not a multiple of the pair count [the down projection of the
+ * feed-forward: x += H W2^T + b2]. A tile is cut at most once; its two partial products are added in a fixed
+ * order (upper k-range first), so the result is reproducible; it differs from srm_k_gemm's in the last bits.
+ * This is what srm_decode_step and srm_generate run for the down projection when it is the faster kernel (a long
+ * K and a partly empty last round: 192 tiles of 96 k-blocks on 74 pairs, the rollout model; with 64 or 128
+ * tiles of 64 k-blocks the extra epilogues cost more than the shorter ranges save, and the unsplit kernel stays). d_order: scratch of srm_k_gemm_splitk_order_bytes(M, N) bytes, 256-byte aligned,
+ * cleared by the call. SRM_ERR_UNSUPPORTED when the shape does not call for a split (the tiles fill whole
+ * rounds, or there are fewer than half as many tiles as pairs): use srm_k_gemm then. */
+size_t srm_k_gemm_splitk_order_bytes(int64_t M, int64_t N);
+int srm_k_gemm_splitk(srm_model* m, int64_t M, int64_t N, int64_t K, const void* d_A, const void* d_W,
+                      const float* d_bias, float* d_out, void* d_order, size_t order_bytes,
+                      uint32_t* d_status, void* stream);
+/* The work list of CTA pair `pair` of `pairs` in srm_k_gemm_splitk: up to max_pieces entries of four int64
+ * {tile row, tile column, first k-block, end k-block} written to the HOST array `pieces`. Returns the number
+ * of pieces of that pair, or a negative SRM_ERR_* (SRM_ERR_UNSUPPORTED: no split for this shape). Pure host
+ * arithmetic: needs no device. */
+int64_t srm_k_gemm_splitk_plan(int64_t M, int64_t N, int64_t K, int32_t pairs, int32_t pair,
+                               int64_t* pieces, int64_t max_pieces);
 /* LM head with greedy selection fused into the GEMM epilogue (bf16 models only): d_tok[r] =
  * argmax_v (a[r, :] . W_lm[v, :]), lowest id among equal maxima - the token srm_k_gemm (epilogue 2)
  * followed by greedy srm_k_select gives, without writing the R x V logits. d_a [R, d] in the

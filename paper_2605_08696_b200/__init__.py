@@ -5,4 +5,4 @@ torch device buffers and streams into the calls, nothing else. All arithmetic of
 in the CUDA kernels under csrc/.
 """
 from .binding import (SRM, SRMState, Sampling, SRMError, load_library, lib_path,  # noqa: F401
-                      EPI_BIAS_GELU, EPI_BIAS_RESIDUAL, EPI_PLAIN, FLAG_NO_GRAPH, FLAG_GRAPH)
+                      EPI_BIAS_GELU, EPI_BIAS_RESIDUAL, EPI_PLAIN, FLAG_NO_GRAPH, FLAG_GRAPH, FLAG_NO_SPLITK)

@@ -20,6 +20,7 @@ FLAG_SIMT_GEMM = 1
 FLAG_HEAD_PROJ = 2
 FLAG_NO_GRAPH = 4
 FLAG_GRAPH = 8
+FLAG_NO_SPLITK = 16
 
 # enum srm_tensor
 T_E, T_LN1_G, T_LN1_B, T_ALPHA, T_BETA, T_LAMBDA, T_LN2_G, T_LN2_B, T_W1, T_B1, T_W2, T_B2, \
@@ -92,6 +93,9 @@ SYMBOLS = {
     "srm_k_mixer_step": (C.c_int, [_P, _I32, _I32, _I64, _P, _P, _P, _P, _P, _P]),
     "srm_k_final_norm": (C.c_int, [_P, _I64, _P, _P, _P]),
     "srm_k_gemm": (C.c_int, [_P, _I32, _I64, _I64, _I64, _P, _P, _P, _P, _P, _P]),
+    "srm_k_gemm_splitk_order_bytes": (_SZ, [_I64, _I64]),
+    "srm_k_gemm_splitk": (C.c_int, [_P, _I64, _I64, _I64, _P, _P, _P, _P, _P, _SZ, _P, _P]),
+    "srm_k_gemm_splitk_plan": (_I64, [_I64, _I64, _I64, _I32, _I32, C.POINTER(_I64), _I64]),
     "srm_k_lm_head_greedy": (C.c_int, [_P, _I64, _P, _P, _SZ, _P, _P, _P]),
     "srm_k_select": (C.c_int, [_P, _I64, _P, C.POINTER(_Sampling), _I32, _P, _P, _P]),
     "srm_k_prefill_mixer": (C.c_int, [_P, _I32, _I64, _I32, _P, _P, _P, _P, _P, _P]),
@@ -388,6 +392,15 @@ class SRM:
         N = W.shape[0]
         _check(_lib().srm_k_gemm(self.handle, epilogue, M, N, K, _ptr(A), _ptr(W), _ptr(bias), _ptr(out),
                                  _ptr(status), _stream()), "srm_k_gemm")
+
+    def k_gemm_splitk(self, A, W, bias, out, order=None, status=None):
+        """out += A W^T + bias with K shared out between CTA pairs (raises SRMError -2 when the shape needs no split)."""
+        M, K = A.shape
+        N = W.shape[0]
+        if order is None:
+            order = torch.empty(_lib().srm_k_gemm_splitk_order_bytes(M, N), dtype=torch.uint8, device=A.device)
+        _check(_lib().srm_k_gemm_splitk(self.handle, M, N, K, _ptr(A), _ptr(W), _ptr(bias), _ptr(out), _ptr(order),
+                                        order.numel() * order.element_size(), _ptr(status), _stream()), "srm_k_gemm_splitk")
 
     def k_lm_head_greedy(self, a, part, tok, status=None):
         _check(_lib().srm_k_lm_head_greedy(self.handle, a.shape[0], _ptr(a), _ptr(part), part.numel() * part.element_size(),

@@ -17,6 +17,7 @@
 #include "common.cuh"
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
+#include "gemm_tc_splitk.cuh"
 #include "mixer.cuh"
 #include "mixer_stream.cuh"
 #include "mixer_proj.cuh"
@@ -251,13 +252,27 @@ size_t state_bytes_for(const srm_config& c, int64_t B) {
 }
 
 // ---- workspace carving ----------------------------------------------------------------------
-struct DecodeWs { float* x; void* a; void* H; float* logits; float* q; int64_t rows; };     // q: head projections only
+struct DecodeWs {
+  float* x; void* a; void* H; float* logits;
+  float* q;               // head projections only
+  int32_t* order;         // split-K down projection: one word per (tile of x, CTA of the pair, epilogue warp)
+  size_t order_bytes;
+  int64_t rows;
+};
 struct PrefillWs { float* x; void* a; void* H; void* a_last; float* logits; float* q; int64_t samples; };
 
+// The down projection of a decode step may be split along K between CTA pairs (gemm_tc_splitk.cuh).
+bool splitk_enabled(const srm_config& c) {
+  return c.dtype == SRM_DTYPE_BF16 && !(c.flags & (SRM_FLAG_SIMT_GEMM | SRM_FLAG_NO_SPLITK));
+}
+size_t splitk_order_bytes(int64_t M, int64_t N) {
+  return align_up(tc::split_order_words(((M + tc::BM - 1) / tc::BM) * ((N + tc::BN - 1) / tc::BN)) * 4, 256);
+}
 size_t decode_ws_bytes(const srm_model& m, int64_t rows) {
   const size_t d = m.cfg.d_model, F = m.F(), V = m.cfg.vocab, ab = m.act_bytes();
   return align_up(rows * d * 4, 256) + align_up(rows * d * ab, 256) + align_up(rows * F * ab, 256) +
-         align_up(rows * V * 4, 256) + (m.head_proj() ? align_up(rows * d * 4, 256) : 0);
+         align_up(rows * V * 4, 256) + (m.head_proj() ? align_up(rows * d * 4, 256) : 0) +
+         (splitk_enabled(m.cfg) ? splitk_order_bytes(rows, m.cfg.d_model) : 0);
 }
 size_t prefill_ws_bytes(const srm_model& m, int64_t samples, int n) {
   const size_t d = m.cfg.d_model, F = m.F(), V = m.cfg.vocab, ab = m.act_bytes(), rows = (size_t)samples * n;
@@ -287,6 +302,9 @@ DecodeWs carve_decode(const srm_model& m, void* ws, int64_t rows) {
   w.H = p; p += align_up(rows * F * ab, 256);
   w.logits = reinterpret_cast<float*>(p); p += align_up(rows * (size_t)m.cfg.vocab * 4, 256);
   w.q = m.head_proj() ? reinterpret_cast<float*>(p) : nullptr;
+  if (m.head_proj()) p += align_up(rows * d * 4, 256);
+  w.order_bytes = splitk_enabled(m.cfg) ? splitk_order_bytes(rows, m.cfg.d_model) : 0;
+  w.order = w.order_bytes ? reinterpret_cast<int32_t*>(p) : nullptr;
   return w;
 }
 PrefillWs carve_prefill(const srm_model& m, void* ws, int64_t samples, int n) {
@@ -431,6 +449,7 @@ int ensure_tc_ready(srm_model& m) {
   SRM_CUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<kEpiBiasResidual>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes));
   SRM_CUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<kEpiPlain>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes));
   SRM_CUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<kEpiArgmax>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes));
+  SRM_CUDA(cudaFuncSetAttribute(tc::gemm_tc_splitk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes));
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2 * (m.num_sms / 2));
   cfg.blockDim = dim3(tc::kThreads);
@@ -479,6 +498,32 @@ int launch_gemm(srm_model& m, int epi, int64_t M, int64_t N, int64_t K, const vo
   if (m.cfg.dtype == SRM_DTYPE_FP32) return launch_gemm_simt<float>(epi, M, N, K, A, W, bias, out, st);
   if (m.cfg.flags & SRM_FLAG_SIMT_GEMM) return launch_gemm_simt<bf16>(epi, M, N, K, A, W, bias, out, st);
   return launch_gemm_tc(m, epi, M, N, K, A, W, bias, out, status, st);
+}
+
+// out[M, N] += A[M, K] W[N, K]^T + bias with K shared out between CTA pairs. `order`: zeroed words (split_order_words).
+// Returns SRM_ERR_UNSUPPORTED when the shape does not call for it (whole tiles per pair lose nothing, or too
+// few tiles): the caller then takes the unsplit kernel.
+int launch_gemm_splitk(srm_model& m, int64_t M, int64_t N, int64_t K, const void* A, const void* W, const float* bias,
+                       float* out, int32_t* order, uint32_t* status, cudaStream_t st, bool only_if_faster = false) {
+  if (M <= 0) return SRM_OK;
+  int rc = ensure_tc_ready(m);
+  if (rc != SRM_OK) return rc;
+  tc::SplitPlan P;
+  const int64_t tiles = ((M + tc::BM - 1) / tc::BM) * ((N + tc::BN - 1) / tc::BN);
+  if (K % tc::BK || !tc::split_plan(tiles, (int)(K / tc::BK), m.tc_clusters, &P)) return SRM_ERR_UNSUPPORTED;
+  if (only_if_faster && tc::split_saved_kb(P) < tc::kSplitWorthKb) return SRM_ERR_UNSUPPORTED;
+  LaunchScope scope(m, SRM_KERNEL_GEMM_DOWN, st);
+  CUtensorMap ta, tb, td;
+  if ((rc = m.tmap(A, M, K, tc::kRowsPerCta, 2, &ta)) != SRM_OK) return rc;
+  if ((rc = m.tmap(W, N, K, tc::kRowsPerCta, 2, &tb)) != SRM_OK) return rc;
+  if ((rc = m.tmap(out, M, N, tc::kOutBoxRows, 4, &td)) != SRM_OK) return rc;
+  const uint8_t* wb = static_cast<const uint8_t*>(W);
+  const int w_static = wb >= m.w && wb < m.w + m.layout.total;
+  tc::SplitArgs g{M, N, K, bias, status, order, w_static};
+  SRM_CUDA(launch_kernel(tc::gemm_tc_splitk_kernel, dim3(2u * (unsigned)P.pairs), dim3(tc::kThreads), tc::kSmemBytes, st,
+                         ta, tb, td, g, P));
+  SRM_CUDA(cudaGetLastError());
+  return SRM_OK;
 }
 
 int check_sampling(const srm_model& m, const srm_sampling* s) {
@@ -647,13 +692,18 @@ int decode_chunk(srm_model& m, srm_state& s, int64_t b0, int64_t R, const int32_
   const int t = (int)(s.pos < c.n_ctx ? s.pos : c.n_ctx - 1);
   const int32_t* pos = s.ragged ? s.pos_dev + b0 : nullptr;       // samples of different lengths: a position per row
   int rc;
+  if (w.order != nullptr) SRM_CUDA(cudaMemsetAsync(w.order, 0, w.order_bytes, st));
   for (int l = 0; l < c.n_layers; ++l) {
     uint8_t* Sl = static_cast<uint8_t*>(s.layer_ptr(l)) + (size_t)b0 * d * m.state_bytes();
     if (m.head_proj()) {
       if ((rc = launch_mixer_block_proj(m, l, t, R, R, 1, l == 0 ? tok_in + b0 : nullptr, w.x, Sl, w.a, w.q, s.status, st, ctr, pos))) return rc;
     } else if ((rc = launch_mixer(m, l, t, R, l == 0 ? tok_in + b0 : nullptr, w.x, Sl, w.a, s.status, st, ctr, pos))) return rc;
     if ((rc = launch_gemm(m, kEpiBiasGelu, R, F, d, w.a, m.ptr(l, SRM_T_W1), m.fptr(l, SRM_T_B1), w.H, s.status, st))) return rc;
-    if ((rc = launch_gemm(m, kEpiBiasResidual, R, d, F, w.H, m.ptr(l, SRM_T_W2), m.fptr(l, SRM_T_B2), w.x, s.status, st))) return rc;
+    rc = w.order != nullptr ? launch_gemm_splitk(m, R, d, F, w.H, m.ptr(l, SRM_T_W2), m.fptr(l, SRM_T_B2), w.x, w.order, s.status, st, true)
+                            : SRM_ERR_UNSUPPORTED;
+    if (rc == SRM_ERR_UNSUPPORTED)
+      rc = launch_gemm(m, kEpiBiasResidual, R, d, F, w.H, m.ptr(l, SRM_T_W2), m.fptr(l, SRM_T_B2), w.x, s.status, st);
+    if (rc) return rc;
   }
   if ((rc = launch_final_norm(m, w.x, R, 1, 0, w.a, st))) return rc;
   SelectOut o = out_all;
@@ -1144,6 +1194,50 @@ int srm_k_gemm(srm_model* m, int32_t epilogue, int64_t M, int64_t N, int64_t K, 
   if (K % 64 || N % 8) return SRM_ERR_UNSUPPORTED;
   if (!aligned(d_A, 16) || !aligned(d_W, 16) || !aligned(d_out, 16) || !aligned(d_bias, 16)) return SRM_ERR_ALIGNMENT;
   return launch_gemm(*m, epilogue, M, N, K, d_A, d_W, d_bias, d_out, d_status, static_cast<cudaStream_t>(stream));
+}
+
+size_t srm_k_gemm_splitk_order_bytes(int64_t M, int64_t N) {
+  if (M < 1 || N < 1) return 0;
+  return splitk_order_bytes(M, N);
+}
+
+int srm_k_gemm_splitk(srm_model* m, int64_t M, int64_t N, int64_t K, const void* d_A, const void* d_W,
+                      const float* d_bias, float* d_out, void* d_order, size_t order_bytes, uint32_t* d_status,
+                      void* stream) {
+  if (m == nullptr || M < 0 || N < 1 || K < 1) return SRM_ERR_INVALID_ARG;
+  if (M == 0) return SRM_OK;
+  if (d_A == nullptr || d_W == nullptr || d_out == nullptr || d_order == nullptr) return SRM_ERR_INVALID_ARG;
+  if (m->cfg.dtype != SRM_DTYPE_BF16 || (m->cfg.flags & SRM_FLAG_SIMT_GEMM) || K % 64 || N % 8) return SRM_ERR_UNSUPPORTED;
+  if (!aligned(d_A, 16) || !aligned(d_W, 16) || !aligned(d_out, 16) || !aligned(d_bias, 16) || !aligned(d_order, 256)) return SRM_ERR_ALIGNMENT;
+  const size_t need = splitk_order_bytes(M, N);
+  if (order_bytes < need) return SRM_ERR_BUFFER_TOO_SMALL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int rc = ensure_tc_ready(*m);
+  if (rc != SRM_OK) return rc;
+  tc::SplitPlan P;
+  if (!tc::split_plan(((M + tc::BM - 1) / tc::BM) * ((N + tc::BN - 1) / tc::BN), (int)(K / 64), m->tc_clusters, &P)) return SRM_ERR_UNSUPPORTED;
+  SRM_CUDA(cudaMemsetAsync(d_order, 0, need, st));
+  return launch_gemm_splitk(*m, M, N, K, d_A, d_W, d_bias, d_out, static_cast<int32_t*>(d_order), d_status, st);
+}
+
+int64_t srm_k_gemm_splitk_plan(int64_t M, int64_t N, int64_t K, int32_t pairs, int32_t pair, int64_t* pieces, int64_t max_pieces) {
+  if (M < 1 || N < 1 || K < 64 || K % 64 || pairs < 1 || pair < 0 || pair >= pairs || max_pieces < 0) return SRM_ERR_INVALID_ARG;
+  if (max_pieces > 0 && pieces == nullptr) return SRM_ERR_INVALID_ARG;
+  tc::SplitPlan P;
+  const int64_t m_tiles = (M + tc::BM - 1) / tc::BM;
+  if (!tc::split_plan(m_tiles * ((N + tc::BN - 1) / tc::BN), (int)(K / 64), pairs, &P)) return SRM_ERR_UNSUPPORTED;
+  tc::SplitCursor cur;
+  cur.init(P, pair);
+  tc::SplitPiece pc;
+  int64_t n = 0;
+  while (cur.next(P, &pc)) {
+    if (n < max_pieces) {
+      int64_t* o = pieces + 4 * n;
+      o[0] = pc.tile % m_tiles; o[1] = pc.tile / m_tiles; o[2] = pc.kb0; o[3] = pc.kb1;
+    }
+    ++n;
+  }
+  return n;
 }
 
 int srm_k_lm_head_greedy(srm_model* m, int64_t R, const void* d_a, void* d_part, size_t part_bytes, int32_t* d_tok,

@@ -132,6 +132,50 @@ def test_tensor_core_gemm_equals_simt_gemm_on_device():
         assert rel_err_rows(a, b) < (8e-3 if epi == 0 else 1e-5)
 
 
+# ---- down projection with K shared out between CTA pairs -----------------------------------------
+
+@pytest.mark.parametrize("M,N,K", [(4096, 1024, 4096), (8192, 1024, 4096), (4096, 1536, 6144), (3000, 1024, 4096),
+                                   (2100, 1304, 4096)])
+def test_split_k_residual_gemm_matches_fp64_and_the_unsplit_kernel(M, N, K):
+    import paper_2605_08696_b200 as P
+    shape = custom_shape(d_model=64, dtype="bf16")
+    m, _ = _model(shape)
+    rng = np.random.default_rng(M + N + K)
+    A = _t(rng.normal(size=(M, K)), torch.bfloat16)
+    W = _t(rng.normal(size=(N, K)) * 0.05, torch.bfloat16)
+    bias = _t(rng.normal(size=N))
+    x0 = rng.normal(size=(M, N)).astype(np.float32)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    nb = P.load_library().srm_k_gemm_splitk_order_bytes(M, N)
+    order = torch.full((nb // 4,), 0x33333333, dtype=torch.int32, device=DEV)      # the call must clear it
+    outs = []
+    for _ in range(2):
+        x = _t(x0)
+        m.k_gemm_splitk(A, W, bias, x, order=order, status=status)
+        outs.append(x)
+    x_ref = _t(x0)
+    m.k_gemm(1, A, W, bias, x_ref, status=status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    assert (order.cpu().numpy() == 0).all()                   # every cut tile was completed and its word put back
+    assert torch.equal(outs[0].view(torch.int32), outs[1].view(torch.int32))       # reproducible bit for bit
+    A64, W64 = A.float().cpu().numpy().astype(np.float64), W.float().cpu().numpy().astype(np.float64)
+    want = x0.astype(np.float64) + A64 @ W64.T + bias.cpu().numpy().astype(np.float64)
+    assert rel_err_rows(outs[0].cpu().numpy(), want) < 2e-5
+    assert rel_err_rows(outs[0].cpu().numpy(), x_ref.cpu().numpy()) < 1e-5       # same products, other order of additions
+
+
+def test_split_k_is_refused_where_whole_tiles_lose_nothing():
+    import paper_2605_08696_b200 as P
+    m, _ = _model(custom_shape(d_model=64, dtype="bf16"))
+    A = torch.zeros(256, 256, dtype=torch.bfloat16, device=DEV)
+    W = torch.zeros(1024, 256, dtype=torch.bfloat16, device=DEV)
+    x = torch.ones(256, 1024, device=DEV)
+    with pytest.raises(P.SRMError) as e:
+        m.k_gemm_splitk(A, W, None, x)
+    assert e.value.code == -2 and bool((x == 1).all())
+
+
 @pytest.mark.parametrize("M,N,K", [(4, 256, 64), (70, 130 * 8, 256), (129, 64, 128)])
 @pytest.mark.parametrize("epi", [0, 1, 2])
 def test_fp32_simt_gemm_matches_fp64_matmul(M, N, K, epi):

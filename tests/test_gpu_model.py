@@ -124,6 +124,32 @@ def test_tiny_config_nucleus_sampling_follows_the_oracle_sampler_step_by_step():
     assert len({tuple(r) for r in seqs[:8]}) > 4 and st.status() == 0
 
 
+def test_decode_with_and_without_split_k_down_projection_agree():
+    """The decode step shares the K dimension of the down projection out between CTA pairs where that is the
+    faster kernel (the rollout model at 8192 rows: 192 tiles of 96 k-blocks for 74 pairs).
+    Same products, another order of fp32 additions in x; through 16 bf16 layers a last-bit difference in x now
+    and then flips the bf16 rounding of an activation, so the two runs differ by what bf16 inputs allow (the
+    kernel-level test shows 1e-5 for one projection): both stay inside the bf16 tolerance of each other."""
+    import paper_2605_08696_b200 as P
+    shape = I.CONFIGS["rl"]
+    W = I.make_weights(shape)
+    B, n = 8192, 4
+    prompts = torch.from_numpy(I.uniform_prompts(B, n, shape.vocab, seed=3)).to(DEV)
+    res = []
+    for flags in (0, P.FLAG_NO_SPLITK):
+        model = P.SRM(shape, W, device=DEV, flags=flags)
+        st = model.new_state(B)
+        ws = model.new_workspace(B, n, prefill_samples=B)
+        tok = model.prefill(st, prompts, P.Sampling("greedy"), ws)
+        for k in range(2):
+            tok, lg = model.decode_step(st, tok, P.Sampling("greedy"), k + 1, ws, want_logits=True)
+        res.append((lg[:64].cpu().numpy(), st.cache()[:, :64].cpu().numpy(), st.status()))
+    assert res[0][2] == 0 and res[1][2] == 0
+    assert not np.array_equal(res[0][0], res[1][0])          # (the split kernel did run: other order of additions)
+    assert rel_err_rows(res[0][0], res[1][0]) < 2e-2
+    assert rel_err_rows(res[0][1], res[1][1]) < 2e-2
+
+
 def test_tiny_config_full_parity_fp32():
     """Config 'tiny': 4 prompts x 8 tokens, greedy 24 tokens, fp32, tolerance 1e-4; every token
     with margin > 1e-2 bit-exact; also free-running generation equals the oracle's tokens."""
