@@ -692,15 +692,23 @@ int decode_chunk(srm_model& m, srm_state& s, int64_t b0, int64_t R, const int32_
   const int t = (int)(s.pos < c.n_ctx ? s.pos : c.n_ctx - 1);
   const int32_t* pos = s.ragged ? s.pos_dev + b0 : nullptr;       // samples of different lengths: a position per row
   int rc;
-  if (w.order != nullptr) SRM_CUDA(cudaMemsetAsync(w.order, 0, w.order_bytes, st));
+  // the down projection shares K out between CTA pairs where that is the faster kernel for R rows
+  bool split = false;
+  if (w.order != nullptr && F % tc::BK == 0) {
+    if ((rc = ensure_tc_ready(m))) return rc;
+    tc::SplitPlan P;
+    const int64_t tiles = ((R + tc::BM - 1) / tc::BM) * ((d + tc::BN - 1) / tc::BN);
+    split = tc::split_plan(tiles, (int)(F / tc::BK), m.tc_clusters, &P) && tc::split_saved_kb(P) >= tc::kSplitWorthKb;
+  }
+  if (split) SRM_CUDA(cudaMemsetAsync(w.order, 0, w.order_bytes, st));
   for (int l = 0; l < c.n_layers; ++l) {
     uint8_t* Sl = static_cast<uint8_t*>(s.layer_ptr(l)) + (size_t)b0 * d * m.state_bytes();
     if (m.head_proj()) {
       if ((rc = launch_mixer_block_proj(m, l, t, R, R, 1, l == 0 ? tok_in + b0 : nullptr, w.x, Sl, w.a, w.q, s.status, st, ctr, pos))) return rc;
     } else if ((rc = launch_mixer(m, l, t, R, l == 0 ? tok_in + b0 : nullptr, w.x, Sl, w.a, s.status, st, ctr, pos))) return rc;
     if ((rc = launch_gemm(m, kEpiBiasGelu, R, F, d, w.a, m.ptr(l, SRM_T_W1), m.fptr(l, SRM_T_B1), w.H, s.status, st))) return rc;
-    rc = w.order != nullptr ? launch_gemm_splitk(m, R, d, F, w.H, m.ptr(l, SRM_T_W2), m.fptr(l, SRM_T_B2), w.x, w.order, s.status, st, true)
-                            : SRM_ERR_UNSUPPORTED;
+    rc = split ? launch_gemm_splitk(m, R, d, F, w.H, m.ptr(l, SRM_T_W2), m.fptr(l, SRM_T_B2), w.x, w.order, s.status, st, true)
+               : SRM_ERR_UNSUPPORTED;
     if (rc == SRM_ERR_UNSUPPORTED)
       rc = launch_gemm(m, kEpiBiasResidual, R, d, F, w.H, m.ptr(l, SRM_T_W2), m.fptr(l, SRM_T_B2), w.x, s.status, st);
     if (rc) return rc;
