@@ -516,7 +516,7 @@ def main():
     ap.add_argument("--workload", default="mid", choices=["tiny", "small", "mid", "rl"])
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch per GPU")
     ap.add_argument("--chunk", type=int, default=8192, help="samples per decode pass (workspace size)")
-    ap.add_argument("--prefill-rows", type=int, default=262144, help="prompt rows per prefill pass")
+    ap.add_argument("--prefill-rows", type=int, default=524288, help="prompt rows per prefill pass")
     ap.add_argument("--state-dtype", default="fp32", choices=["fp32", "bf16"])
     ap.add_argument("--ref-samples", type=int, default=32)
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -22,6 +22,7 @@
 #include "mixer_stream.cuh"
 #include "mixer_proj.cuh"
 #include "prefill.cuh"
+#include "prefill_scan.cuh"
 #include "select.cuh"
 #include "select_topp.cuh"
 
@@ -606,6 +607,34 @@ int launch_lm_head_greedy(srm_model& m, int64_t R, const void* a, void* part, co
   return SRM_OK;
 }
 
+// From this many prompts per pass the scan kernel (one warp per prompt) is the faster prefill mixer.
+constexpr int64_t kPrefillScanMinSamples = 384;
+
+template <int NV, typename WT, typename ST>
+int launch_prefill_scan(const PrefillParams& p, int num_sms, cudaStream_t st) {
+  const int warps = prefill_scan_warps(p.d, p.Bp, num_sms);
+  const size_t smem = prefill_scan_smem(p.d, warps);
+  static bool attr_set = false;               // per instantiation
+  if (!attr_set) {
+    SRM_CUDA(cudaFuncSetAttribute(prefill_scan_kernel<NV, WT, ST>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScanSmemBudget));
+    attr_set = true;
+  }
+  const unsigned grid = (unsigned)(p.Bp < num_sms ? p.Bp : num_sms);
+  SRM_CUDA(launch_kernel(prefill_scan_kernel<NV, WT, ST>, dim3(grid), dim3(warps * 32), smem, st, p));
+  SRM_CUDA(cudaGetLastError());
+  return SRM_OK;
+}
+
+template <typename WT, typename ST>
+int launch_prefill_scan_nv(const PrefillParams& p, int num_sms, cudaStream_t st) {
+  switch (p.d / 128) {
+    case 4: return launch_prefill_scan<4, WT, ST>(p, num_sms, st);
+    case 8: return launch_prefill_scan<8, WT, ST>(p, num_sms, st);
+    case 12: return launch_prefill_scan<12, WT, ST>(p, num_sms, st);
+    default: return launch_prefill_scan<16, WT, ST>(p, num_sms, st);
+  }
+}
+
 int launch_prefill_mixer(const srm_model& m, int layer, int64_t Bp, int n, const int32_t* tok, float* x, void* S,
                          void* a, uint32_t* status, cudaStream_t st, const int32_t* len = nullptr) {
   if (Bp <= 0) return SRM_OK;
@@ -619,6 +648,14 @@ int launch_prefill_mixer(const srm_model& m, int layer, int64_t Bp, int n, const
   p.eps = m.cfg.ln_eps; p.status = status; p.len = len;
   const size_t smem = (size_t)kPrefillTile * m.cfg.d_model * 4;
   const bool wb = m.cfg.dtype == SRM_DTYPE_BF16, sb = m.cfg.state_dtype == SRM_DTYPE_BF16;
+  const int nv = p.d / 128;
+  const bool scan_shape = p.d % 128 == 0 && (p.d / p.h) % 128 == 0 && p.h <= 8 && (nv == 4 || nv == 8 || nv == 12 || nv == 16);
+  if (scan_shape && Bp >= kPrefillScanMinSamples) {        // many prompts: one warp walks each prompt's positions
+    if (wb && sb) return launch_prefill_scan_nv<bf16, bf16>(p, m.num_sms, st);
+    if (wb) return launch_prefill_scan_nv<bf16, float>(p, m.num_sms, st);
+    if (sb) return launch_prefill_scan_nv<float, bf16>(p, m.num_sms, st);
+    return launch_prefill_scan_nv<float, float>(p, m.num_sms, st);
+  }
   auto go = [&](auto kernel) -> int {
     SRM_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     SRM_CUDA(launch_kernel(kernel, dim3((unsigned)Bp), dim3(kPrefillThreads), smem, st, p));

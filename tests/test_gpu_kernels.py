@@ -352,6 +352,39 @@ def test_topk_sampling_stream_is_keyed_by_sample_and_step():
 
 # ---- sequence-parallel token mixing (Eq. 1, Eq. 3) -----------------------------------------------
 
+@pytest.mark.parametrize("d,dtype,n,Bp", [(512, "bf16", 37, 400), (1024, "bf16", 50, 1200), (1536, "bf16", 9, 500),
+                                          (1024, "fp32", 12, 390)])
+@pytest.mark.parametrize("embed", [False, True])
+def test_prefill_scan_kernel_matches_oracle_parallel_form(d, dtype, n, Bp, embed):
+    """Many prompts per pass take the scan kernel (one warp per prompt, the cache in registers, the matrix M applied
+    through its recurrence): same oracle, the explicit n x n matrices of Eq. 1 / Eq. 3. A third of the prompts
+    is checked (they are independent; the checked ones are spread over the grid)."""
+    from oracle import srm_oracle as O
+    shape = custom_shape(n_layers=1, d_model=d, vocab=512, n_ctx=max(n, 40), dtype=dtype, seed=9)
+    m, W = _model(shape)
+    lw = {k: np.asarray(v, np.float64) for k, v in W["layers"][0].items()}
+    rng = np.random.default_rng(n + Bp)
+    tok = rng.integers(0, shape.vocab, size=(Bp, n)).astype(np.int32)
+    x0 = W["E"][tok].astype(np.float64) if embed else rng.normal(size=(Bp, n, d)).astype(np.float32).astype(np.float64)
+    x = _t(np.zeros((Bp * n, d)) if embed else x0.reshape(Bp * n, d))
+    S = torch.full((Bp, d), float("nan"), device=DEV)
+    a = torch.zeros(Bp * n, d, dtype=m.act_dtype, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    m.k_prefill_mixer(0, Bp, n, x, S, a, tok=_t(tok.reshape(-1), torch.int32) if embed else None, status=status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    xg, Sg, ag = x.cpu().numpy(), S.cpu().numpy(), a.float().cpu().numpy()
+    assert np.isfinite(Sg).all()
+    for b in list(range(0, Bp, 3)) + [Bp - 1]:
+        z = O.layer_norm(x0[b], lw["ln1_g"], lw["ln1_b"], shape.ln_eps)
+        y, Sn = O.mixer_parallel(z, lw["alpha"], lw["beta"], lw["lam"], shape.n_heads)
+        x1 = x0[b] + y
+        a1 = O.layer_norm(x1, lw["ln2_g"], lw["ln2_b"], shape.ln_eps)
+        assert rel_err_rows(xg[b * n:(b + 1) * n], x1) < 2e-5
+        assert rel_err_rows(Sg[b], Sn) < 2e-5
+        assert rel_err_rows(ag[b * n:(b + 1) * n], a1) < (2e-5 if dtype == "fp32" else 6e-3)
+
+
 @pytest.mark.parametrize("d,dtype,n", [(64, "fp32", 8), (64, "fp32", 32), (64, "fp32", 37), (512, "bf16", 128),
                                        (1024, "bf16", 50), (1536, "bf16", 33)])
 @pytest.mark.parametrize("embed", [False, True])

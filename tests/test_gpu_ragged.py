@@ -139,3 +139,31 @@ def test_ragged_with_head_projections_and_argument_checks():
     bad = torch.tensor([12, 0, 40], dtype=torch.int32, device=DEV)
     model.prefill_ragged(st_bad, torch.from_numpy(toks).to(DEV), bad, g, ws)
     assert st_bad.status() & 1
+
+
+def test_ragged_prefill_through_the_scan_kernel_matches_the_tile_kernel():
+    """With many prompts per pass the prefill mixer is the scan kernel, with few the tile kernel (explicit diagonal
+    blocks of M): the same ragged prompts through both (one pass of 512 prompts, and passes of 64) leave the same
+    cache and first tokens up to what bf16 activations allow (each kernel is checked against the oracle elsewhere)."""
+    import paper_2605_08696_b200 as P
+    shape = I.CONFIGS["small"]
+    W = I.make_weights(shape)
+    model = P.SRM(shape, W, device=DEV)
+    B, n_max = 512, 24
+    rng = np.random.default_rng(5)
+    lengths = rng.integers(1, n_max + 1, size=B).astype(np.int32)
+    lengths[:3] = (n_max, 1, 2)
+    toks = _ragged_batch(shape, [int(v) for v in lengths], seed=31)
+    lens_dev = torch.from_numpy(lengths).to(DEV)
+    g = P.Sampling("greedy")
+    res = []
+    for samples in (B, 64):
+        st = model.new_state(B)
+        ws = model.new_workspace(B, n_max, prefill_samples=samples)
+        tok, lg = model.prefill_ragged(st, torch.from_numpy(toks).to(DEV), lens_dev, g, ws, want_logits=True)
+        res.append((tok.cpu().numpy(), lg.cpu().numpy(), st.cache().cpu().numpy()))
+        assert st.status() == 0
+    # (eight bf16 layers: a last-bit difference in x now and then flips the bf16 rounding of an activation)
+    assert rel_err_rows(res[0][1], res[1][1]) < 2e-2
+    assert rel_err_rows(res[0][2], res[1][2]) < 2e-2
+    assert (res[0][0] == res[1][0]).mean() > 0.9
