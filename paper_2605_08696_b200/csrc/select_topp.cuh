@@ -9,11 +9,14 @@
 //   * Weights are fixed-point integers q_v = round(2^31 exp((l_v - max) / T)) and every mass is an exact
 //     64-bit integer sum: sums do not depend on the order of addition, so neither the nucleus nor the drawn
 //     token depends on thread scheduling, and thresholds are compared exactly.
-//   * The key of the last nucleus member (keys: order-preserving uint32 image of the float) is found by
-//     four-way search on the key range: each pass sums mass and count of the range's four parts (pivots
-//     evenly spaced in logit value while the range is wide, in key space afterwards, which bounds the passes),
-//     keeps the part in which the cumulative mass from the top crosses p Z, and stops when that part holds
-//     at most kToppExact tokens (they are then ranked exactly, ties by id) or a single key (all ties).
+//   * The last nucleus member is located with one histogram pass: mass and count of 2048 buckets evenly
+//     spaced in logit value between the smallest logit of non-zero weight and the maximum (shared-memory
+//     atomics; with that many buckets neighbouring tokens rarely meet), a block-wide suffix sum over the
+//     buckets finds the one in which the cumulative mass from the top crosses p Z, and its few dozen tokens
+//     are ranked exactly (ties by id). Only when more tokens share that bucket than the exact stage holds
+//     (heavy ties) a four-way search on the bucket's key range follows: each pass sums mass and count of the
+//     range's four parts (pivots evenly spaced in logit value while the range is wide, in key space
+//     afterwards, which bounds the passes) until at most kToppExact tokens or a single key (all ties) remain.
 //   * The draw scans the row in id order: every thread owns a contiguous chunk, two block-wide prefix sums
 //     (ties before the chunk, nucleus mass before the chunk) locate the thread that holds the token.
 // One block per row; the row's keys are staged in shared memory when they fit (V <= kToppSmemFloats), else
@@ -31,7 +34,8 @@ constexpr int kToppCap = 1024;                   // capacity of the exact last s
 constexpr int kToppExact = 256;                  // the search stops when the part that holds the edge has this few tokens
                                                  // (ranking n candidates costs n^2 comparisons)
 constexpr int kToppMaxPasses = 28;               // 6 passes with value pivots, then 4-way search on at most 2^32 keys
-constexpr int kToppSmemFloats = 44 * 1024;       // rows up to 176 KB are staged in shared memory
+constexpr int kToppSmemFloats = 40 * 1024;       // rows up to 160 KB are staged in shared memory
+constexpr int kToppBuckets = 2048;               // histogram buckets (two per thread in the suffix sum)
 constexpr float kToppFixedOne = 2147483648.0f;   // 2^31: weight of the most probable token (weights fit 32 bits)
 
 struct ToppScratch {
@@ -42,7 +46,8 @@ struct ToppScratch {
   uint32_t ckey[kToppCap], skey[kToppCap];
   int32_t cid[kToppCap], sid[kToppCap];
   unsigned long long cq[kToppCap], sq[kToppCap];
-  int n_cand, pos, first;
+  int n_cand, pos, first, bstar, n_ties;
+  unsigned int kmin, kmax;
   float fmax_w[kToppWarps], fmin_w[kToppWarps];
 };
 
@@ -55,6 +60,11 @@ __device__ __forceinline__ unsigned long long topp_weight(float l, float m, floa
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(x));
   return (unsigned long long)__float2uint_rn(e);
 }
+struct ToppHist {
+  unsigned long long mass[kToppBuckets];
+  unsigned int cnt[kToppBuckets];
+};
+
 // NaN sorts below everything
 __device__ __forceinline__ uint32_t topp_key(float l) { return (l == l) ? order_key(l) : 0u; }
 
@@ -101,7 +111,8 @@ select_topp_kernel(const float* __restrict__ logits, int64_t R, int V, float top
   pdl_wait();
   extern __shared__ __align__(16) uint8_t topp_smem[];
   ToppScratch* sc = reinterpret_cast<ToppScratch*>(topp_smem);
-  uint32_t* skeys = reinterpret_cast<uint32_t*>(topp_smem + ((sizeof(ToppScratch) + 15) & ~size_t(15)));
+  ToppHist* hist = reinterpret_cast<ToppHist*>(topp_smem + ((sizeof(ToppScratch) + 15) & ~size_t(15)));
+  uint32_t* skeys = reinterpret_cast<uint32_t*>(topp_smem + ((sizeof(ToppScratch) + 15) & ~size_t(15)) + sizeof(ToppHist));
   const int64_t row = blockIdx.x;
   if (row >= R) return;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -146,10 +157,65 @@ select_topp_kernel(const float* __restrict__ logits, int64_t R, int V, float top
   const float s = inv_temp * 1.4426950408889634f;
   // search range [lo, hi) in key space; `above` = mass of the keys >= hi
   // (tokens more than 33 / s below the maximum have weight zero; nothing lies below the row's minimum)
-  uint64_t lo = topp_key(fmaxf(mx - 33.0f / s, mn)), hi = (uint64_t)topp_key(mx) + 1;
+  const float lo_v = fmaxf(mx - 33.0f / s, mn);
+  uint64_t lo = topp_key(lo_v), hi = (uint64_t)topp_key(mx) + 1;
   unsigned long long above = 0, target = 0, in_mass = 0;
   long long in_cnt = 0;
-  for (int pass = 0; pass < kToppMaxPasses; ++pass) {
+
+  // ---- histogram over logit value: the bucket in which the cumulative mass from the top reaches p Z ----
+  const float b_scale = mx > lo_v ? (float)kToppBuckets / (mx - lo_v) : 0.f;
+  auto bucket_of = [&](float l) -> int {         // monotone in l; -1 for weight-zero tokens and NaN
+    if (!(l >= lo_v)) return -1;
+    const int b = (int)((l - lo_v) * b_scale);
+    return b < kToppBuckets ? b : kToppBuckets - 1;
+  };
+  for (int i = tid; i < kToppBuckets; i += kToppThreads) { hist->mass[i] = 0ull; hist->cnt[i] = 0u; }
+  if (tid == 0) { sc->bstar = kToppBuckets - 1; sc->bcast[1] = 0ull; }      // (always overwritten: Z >= the maximum's weight)
+  __syncthreads();
+  for (int i = tid; i < V; i += kToppThreads) {
+    const float l = key_value(key_at(i));
+    const int b = bucket_of(l);
+    if (b >= 0) {
+      atomicAdd(&hist->mass[b], topp_weight(l, mx, s));
+      atomicAdd(&hist->cnt[b], 1u);
+    }
+  }
+  __syncthreads();
+  {
+    // thread t owns buckets B-1-2t (upper) and B-2-2t: an exclusive scan over threads is a suffix sum over buckets
+    const int bu = kToppBuckets - 1 - 2 * tid, bl = bu - 1;
+    const unsigned long long mu = bu >= 0 ? hist->mass[bu] : 0ull, ml = bl >= 0 ? hist->mass[bl] : 0ull;
+    unsigned long long Z;
+    const unsigned long long before = block_exclusive_scan(mu + ml, sc, &Z);
+    // Z: every token of non-zero weight; the mass the nucleus must reach
+    const double t = ceil((double)top_p * (double)Z);
+    target = t < 1.0 ? 1ull : (t > (double)Z ? Z : (unsigned long long)t);
+    if (before < target && target <= before + mu) { sc->bstar = bu; sc->bcast[1] = before; }
+    else if (before + mu < target && target <= before + mu + ml) { sc->bstar = bl; sc->bcast[1] = before + mu; }
+    __syncthreads();
+  }
+  const int bstar = sc->bstar;
+  above = sc->bcast[1];
+  in_cnt = (long long)hist->cnt[bstar];
+  in_mass = hist->mass[bstar];
+  bool by_keys = false;                        // candidates are selected by key range (after the search) or by bucket
+  if (in_cnt > kToppCap) {
+    // heavy ties: more tokens in the edge bucket than the exact stage holds. Its key range (bucket_of is
+    // monotone, so every key between two of its keys belongs to it), then the four-way search on that range.
+    if (tid == 0) { sc->kmin = 0xffffffffu; sc->kmax = 0u; }
+    __syncthreads();
+    unsigned int kmn = 0xffffffffu, kmx = 0u;
+    for (int i = tid; i < V; i += kToppThreads) {
+      const uint32_t k = key_at(i);
+      if (bucket_of(key_value(k)) == bstar) { kmn = k < kmn ? k : kmn; kmx = k > kmx ? k : kmx; }
+    }
+    kmn = __reduce_min_sync(0xffffffffu, kmn); kmx = __reduce_max_sync(0xffffffffu, kmx);
+    if (lane == 0) { atomicMin(&sc->kmin, kmn); atomicMax(&sc->kmax, kmx); }
+    __syncthreads();
+    lo = sc->kmin; hi = (uint64_t)sc->kmax + 1;
+    by_keys = true;
+  }
+  for (int pass = 0; by_keys && hi - lo > 1 && pass < kToppMaxPasses; ++pass) {
     // three pivots lo < p1 <= p2 <= p3 < hi (as keys)
     uint32_t pv[3];
     const uint64_t width = hi - lo;
@@ -202,12 +268,6 @@ select_topp_kernel(const float* __restrict__ logits, int64_t R, int V, float top
     unsigned long long mass[4], cnt[4];
 #pragma unroll
     for (int j = 0; j < 4; ++j) { mass[j] = sc->bcast[j]; cnt[j] = sc->bcast[4 + j]; }
-    if (pass == 0) {
-      // the first range holds every token of non-zero weight: Z, and the mass the nucleus must reach
-      const unsigned long long Z = mass[0] + mass[1] + mass[2] + mass[3];
-      const double t = ceil((double)top_p * (double)Z);
-      target = t < 1.0 ? 1ull : (t > (double)Z ? Z : (unsigned long long)t);
-    }
     // from the top: the part in which the cumulative mass reaches the target
     int chosen = 0;
     unsigned long long acc = above;
@@ -226,14 +286,14 @@ select_topp_kernel(const float* __restrict__ logits, int64_t R, int V, float top
 
   // ---- the last nucleus member: its key, how many tokens of that key are in, the nucleus mass ----
   uint32_t kstar;
-  long long n_ties_in;
+  long long n_ties_in, n_ties_all;             // tokens of the edge key that are in the nucleus / that exist
   unsigned long long nucleus_mass;
   if (in_cnt <= kToppCap) {
-    if (tid == 0) { sc->n_cand = 0; sc->pos = kToppCap; sc->first = kToppCap; }
+    if (tid == 0) { sc->n_cand = 0; sc->pos = kToppCap; sc->first = kToppCap; sc->n_ties = 0; }
     __syncthreads();
     for (int i = tid; i < V; i += kToppThreads) {
       const uint32_t k = key_at(i);
-      if (k >= lo && k < hi) {
+      if (by_keys ? (k >= lo && k < hi) : (bucket_of(key_value(k)) == bstar)) {
         const int slot = atomicAdd(&sc->n_cand, 1);
         if (slot < kToppCap) { sc->ckey[slot] = k; sc->cid[slot] = i; sc->cq[slot] = topp_weight(key_value(k), mx, s); }
       }
@@ -256,9 +316,11 @@ select_topp_kernel(const float* __restrict__ logits, int64_t R, int V, float top
     const int pos = sc->pos < n ? sc->pos : n - 1;     // (n >= 1: the chosen part holds the boundary token)
     kstar = sc->skey[pos];
     if (tid <= pos && sc->skey[tid] == kstar) atomicMin(&sc->first, tid);
+    if (tid < n && sc->skey[tid] == kstar) atomicAdd(&sc->n_ties, 1);
     if (tid == pos) sc->bcast[0] = above + before + mine;
     __syncthreads();
     n_ties_in = pos - sc->first + 1;
+    n_ties_all = sc->n_ties;
     nucleus_mass = sc->bcast[0];
   } else {
     // a single key with more than kToppCap tokens: all ties, taken in id order
@@ -266,6 +328,7 @@ select_topp_kernel(const float* __restrict__ logits, int64_t R, int V, float top
     const unsigned long long qt = in_mass / (unsigned long long)in_cnt;       // they all carry the same weight
     long long c = qt > 0 ? (long long)((target - above + qt - 1) / qt) : in_cnt;
     n_ties_in = c < 1 ? 1 : (c > in_cnt ? in_cnt : c);
+    n_ties_all = in_cnt;
     nucleus_mass = above + (unsigned long long)n_ties_in * qt;
   }
 
@@ -277,16 +340,21 @@ select_topp_kernel(const float* __restrict__ logits, int64_t R, int V, float top
   const unsigned long long thr = (unsigned long long)(u * (double)nucleus_mass);
   const int chunk = ((V + kToppThreads - 1) / kToppThreads) | 1;             // odd: conflict-free in shared memory
   const int i0 = tid * chunk < V ? tid * chunk : V, i1 = i0 + chunk < V ? i0 + chunk : V;
-  unsigned long long my_ties = 0;
-  for (int i = i0; i < i1; ++i) my_ties += key_at(i) == kstar;
-  unsigned long long tot;
-  const unsigned long long ties_before = block_exclusive_scan(my_ties, sc, &tot);
+  // Membership: key above the edge key, or the edge key itself and among its first n_ties_in ids. When all
+  // tokens of the edge key are in (the usual case) the count of ties before a chunk is not needed.
+  const bool all_ties = n_ties_in >= n_ties_all;
+  unsigned long long tot, ties_before = 0;
+  if (!all_ties) {
+    unsigned long long my_ties = 0;
+    for (int i = i0; i < i1; ++i) my_ties += key_at(i) == kstar;
+    ties_before = block_exclusive_scan(my_ties, sc, &tot);
+  }
   unsigned long long my_mass = 0;
   {
     long long t = (long long)ties_before;
     for (int i = i0; i < i1; ++i) {
       const uint32_t k = key_at(i);
-      const bool in = k > kstar || (k == kstar && t++ < n_ties_in);
+      const bool in = k > kstar || (k == kstar && (all_ties || t++ < n_ties_in));
       if (in) my_mass += topp_weight(key_value(k), mx, s);
     }
   }
@@ -298,7 +366,7 @@ select_topp_kernel(const float* __restrict__ logits, int64_t R, int V, float top
     int pick = -1;
     for (int i = i0; i < i1; ++i) {
       const uint32_t k = key_at(i);
-      const bool in = k > kstar || (k == kstar && t++ < n_ties_in);
+      const bool in = k > kstar || (k == kstar && (all_ties || t++ < n_ties_in));
       if (in) {
         c += topp_weight(key_value(k), mx, s);
         if (c > thr) { pick = i; break; }

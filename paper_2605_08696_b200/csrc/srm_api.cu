@@ -547,7 +547,7 @@ int launch_select(const srm_model& m, int64_t R, const float* logits, const srm_
     SRM_CUDA(launch_kernel(select_greedy_kernel, dim3((unsigned)R), dim3(kSelThreads), 0, st, logits, R, V, out, status));
   } else if (s.mode == SRM_SELECT_TOPP) {
     const float inv_t = 1.0f / s.temperature;
-    const size_t scratch = (sizeof(ToppScratch) + 15) & ~size_t(15);
+    const size_t scratch = ((sizeof(ToppScratch) + 15) & ~size_t(15)) + sizeof(ToppHist);
     if (V <= kToppSmemFloats) {
       const size_t smem = scratch + (size_t)V * 4;
       static bool attr_set = false;
@@ -559,6 +559,11 @@ int launch_select(const srm_model& m, int64_t R, const float* logits, const srm_
       SRM_CUDA(launch_kernel(select_topp_kernel<true>, dim3((unsigned)R), dim3(kToppThreads), smem, st, logits, R, V,
                              s.top_p, inv_t, s.seed, sample_base, step, out, status));
     } else {
+      static bool attr_set_g = false;           // the scratch alone exceeds the default dynamic shared-memory limit
+      if (!attr_set_g) {
+        SRM_CUDA(cudaFuncSetAttribute(select_topp_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)scratch));
+        attr_set_g = true;
+      }
       SRM_CUDA(launch_kernel(select_topp_kernel<false>, dim3((unsigned)R), dim3(kToppThreads), scratch, st, logits, R, V,
                              s.top_p, inv_t, s.seed, sample_base, step, out, status));
     }
