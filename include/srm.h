@@ -161,6 +161,12 @@ int srm_state_reset(srm_state* s, void* stream);
 /* Position bookkeeping (host side): number of tokens consumed so far. */
 int64_t srm_state_pos(const srm_state* s);
 int srm_state_set_pos(srm_state* s, int64_t pos);
+/* For a state whose buffer was copied from a state left by srm_prefill_ragged (checkpoint / resume): declares
+ * that the per-sample position vector inside the buffer is valid and that the longest sample stands at
+ * max_pos (what srm_state_pos reported for the source state). From then on the state behaves as the source. */
+int srm_state_adopt_positions(srm_state* s, int64_t max_pos);
+/* 1 when the state keeps one position per sample (after srm_prefill_ragged or srm_state_adopt_positions). */
+int srm_state_is_ragged(const srm_state* s);
 /* Device address of the cache slab of one layer, [B, d] in state_dtype (for checkpointing
  * and tests), and of the last-token vector int32[B]. */
 void* srm_state_layer_ptr(const srm_state* s, int32_t layer);

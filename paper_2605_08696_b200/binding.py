@@ -80,6 +80,8 @@ SYMBOLS = {
     "srm_state_reset": (C.c_int, [_P, _P]),
     "srm_state_pos": (_I64, [_P]),
     "srm_state_set_pos": (C.c_int, [_P, _I64]),
+    "srm_state_adopt_positions": (C.c_int, [_P, _I64]),
+    "srm_state_is_ragged": (C.c_int, [_P]),
     "srm_state_layer_ptr": (_P, [_P, _I32]),
     "srm_state_last_token_ptr": (_P, [_P]),
     "srm_status": (C.c_int, [_P, _P, C.POINTER(C.c_uint32)]),
@@ -183,6 +185,14 @@ class SRMState:
 
     def reset(self):
         _check(_lib().srm_state_reset(self.handle, _stream()), "srm_state_reset")
+
+    @property
+    def ragged(self) -> bool:
+        return bool(_lib().srm_state_is_ragged(self.handle))
+
+    def adopt_positions(self, max_pos: int):
+        """After copying the buffer of a ragged state into this one: its per-sample positions are valid."""
+        _check(_lib().srm_state_adopt_positions(self.handle, max_pos), "srm_state_adopt_positions")
 
     def status(self) -> int:
         """Synchronises, returns and clears the device status word."""

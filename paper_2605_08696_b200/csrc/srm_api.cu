@@ -945,6 +945,15 @@ int srm_state_set_pos(srm_state* s, int64_t pos) {
   return SRM_OK;
 }
 
+int srm_state_adopt_positions(srm_state* s, int64_t max_pos) {
+  if (s == nullptr || max_pos < 1 || max_pos > s->m->cfg.n_ctx) return SRM_ERR_INVALID_ARG;
+  s->pos = max_pos;
+  s->ragged = true;
+  return SRM_OK;
+}
+
+int srm_state_is_ragged(const srm_state* s) { return s != nullptr && s->ragged ? 1 : 0; }
+
 void* srm_state_layer_ptr(const srm_state* s, int32_t layer) {
   if (s == nullptr || layer < 0 || layer >= s->m->cfg.n_layers) return nullptr;
   return s->layer_ptr(layer);

@@ -167,3 +167,30 @@ def test_ragged_prefill_through_the_scan_kernel_matches_the_tile_kernel():
     assert rel_err_rows(res[0][1], res[1][1]) < 2e-2
     assert rel_err_rows(res[0][2], res[1][2]) < 2e-2
     assert (res[0][0] == res[1][0]).mean() > 0.9
+
+
+def test_resume_of_a_ragged_state_from_a_copied_buffer():
+    """generate(2k) == generate(k), copy the state buffer into a fresh state, adopt its positions, generate(k)."""
+    import paper_2605_08696_b200 as P
+    shape = I.CONFIGS["small"]
+    model = P.SRM(shape, I.make_weights(shape), device=DEV)
+    lengths = [20, 3, 11, 20]
+    B, n_max, k = 4, 20, 5
+    toks = torch.from_numpy(_ragged_batch(shape, lengths, seed=37)).to(DEV)
+    lens_dev = torch.tensor(lengths, dtype=torch.int32, device=DEV)
+    g = P.Sampling("topk", 50, 0.8, seed=3, sample_idx_base=40)
+    ws = model.new_workspace(B, n_max, prefill_samples=B)
+    a = model.new_state(B)
+    model.prefill_ragged(a, toks, lens_dev, g, ws)
+    full = model.generate(a, 2 * k, 1, g, ws).clone()
+    b = model.new_state(B)
+    model.prefill_ragged(b, toks, lens_dev, g, ws)
+    first = model.generate(b, k, 1, g, ws).clone()
+    c = model.new_state(B)
+    assert not c.ragged and b.ragged
+    c.buf.copy_(b.buf)
+    c.adopt_positions(b.pos)
+    assert c.ragged and c.pos == n_max + k
+    rest = model.generate(c, k, k + 1, g, ws)
+    assert torch.equal(full, torch.cat([first, rest], 1))
+    assert torch.equal(a.cache(), c.cache()) and a.status() == 0 and c.status() == 0
