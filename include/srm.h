@@ -142,7 +142,9 @@ size_t srm_state_bytes(const srm_config* cfg, int64_t B);
 /* Workspace bytes so that decode processes `B_chunk` samples per pass and prefill handles
  * prompts of up to `n_prefill_max` tokens in one pass of at least one sample. Calls accept any
  * workspace at least this large for B_chunk = 1 and split the batch into as many passes as
- * the given workspace requires. */
+ * the given workspace requires. Decode never uses more than 12288 rows of it in one pass: a larger
+ * batch runs as equal passes of at most 10240 rows (whole 256-row tiles), which keeps a layer's
+ * activations in L2 between its kernels; results do not depend on the split. */
 size_t srm_workspace_bytes(const srm_config* cfg, int64_t B_chunk, int32_t n_prefill_max);
 
 /* ---- handles ------------------------------------------------------------------------------ */

@@ -767,6 +767,22 @@ int decode_chunk(srm_model& m, srm_state& s, int64_t b0, int64_t R, const int32_
   return launch_select(m, R, lg, samp, samp.sample_idx_base + (uint64_t)b0, step, o, s.status, st);
 }
 
+// Rows per decode pass for a batch of B rows when the workspace holds up to `fit` rows. Up to kOnePassRows the
+// batch runs as one pass. Beyond that it is cut into the fewest equal passes of at most kMaxPassRows rows, each a
+// whole number of 256-row tiles: a larger pass pushes the activations of a layer (H, x, a: 14 KB per row for
+// d = 1024) out of L2 between the GEMMs, a smaller one leaves rounds of tiles partly empty. Measured at 32768
+// rows, d = 1024: 4096 / 5888 / 8192 / 9472 / 16384 / 32768 rows per pass take 11.95 / 11.75 / 11.35 / 11.24 /
+// 11.49 / 11.68 ms per step; at 16384 rows, d = 1536: 4608 / 9472 / 16384 rows take 17.67 / 16.84 / 17.33 ms.
+constexpr int64_t kOnePassRows = 12288, kMaxPassRows = 10240;
+int64_t choose_pass_rows(int64_t B, int64_t fit) {
+  if (fit < B && fit < kMaxPassRows) return fit;              // the workspace decides
+  if (B <= kOnePassRows && fit >= B) return B;
+  const int64_t passes = (B + kMaxPassRows - 1) / kMaxPassRows;
+  int64_t rows = (B + passes - 1) / passes;
+  rows = (rows + tc::BM - 1) / tc::BM * tc::BM;
+  return rows < fit ? rows : fit;
+}
+
 // `ctr` non-null: position, Philox step and store column come from the device-side counters (graph replay).
 int decode_step_impl(srm_model* m, srm_state* s, const int32_t* d_tok_in, const srm_sampling* samp, int step,
                      int32_t* d_tok_out, int32_t* d_store, int64_t store_stride, int64_t store_col,
@@ -776,8 +792,9 @@ int decode_step_impl(srm_model* m, srm_state* s, const int32_t* d_tok_in, const 
   if (rc) return rc;
   if (!aligned(d_ws, 256) || !aligned(d_tok_in, 4) || !aligned(d_tok_out, 4) || !aligned(d_logits_out, 16)) return SRM_ERR_ALIGNMENT;
   if (s->pos >= m->cfg.n_ctx) return SRM_ERR_CTX_OVERFLOW;
-  const int64_t rows = fit_rows(ws_bytes, s->B, decode_need, *m, 0);
-  if (rows < 1) return SRM_ERR_BUFFER_TOO_SMALL;
+  const int64_t fit = fit_rows(ws_bytes, s->B, decode_need, *m, 0);
+  if (fit < 1) return SRM_ERR_BUFFER_TOO_SMALL;
+  const int64_t rows = choose_pass_rows(s->B, fit);
   const DecodeWs w = carve_decode(*m, d_ws, rows);
   const int32_t* tok_in = d_tok_in != nullptr ? d_tok_in : s->last_tok;
   SelectOut out{s->last_tok, d_tok_out, d_store, store_stride, store_col, 1, ctr, s->ragged ? s->pos_dev : nullptr};
