@@ -27,6 +27,13 @@ Parity status of each function (what pins it, see tests/test_oracle_*.py):
   token_mixer_parallel / _recurrent with head projections (Eq. 10)
                            pinned: brute-force Eq. 10 in the paper's d x n orientation with explicit
                            per-head I_g, identity projections == no projections, parallel == recurrent
+  combined_parallel / combined_recurrent_step (linearly combined heads, Architecture)
+                           pinned: scalar-loop definition, weights (1, 0) / (0, 1) == the mixed-head
+                           mixer, closed form for constant inputs, parallel == recurrent, cache size 2 d
+  kernel_parallel / kernel_recurrent_step (non-unitary kernels, Eq. 11)
+                           pinned: scalar-loop evaluation of Eq. 11 on the padded d+k rows, k = 1 == a
+                           column-repeat head, shift structure (a one-hot channel spreads to the k
+                           channels below it), parallel == recurrent, cache size k d
   SRMOracle (full model logits)  PARITY UNPINNED beyond self-consistency (parallel ==
                            recurrent, causality): the paper prints no activations and
                            its architecture figure is missing, so the block structure
@@ -282,6 +289,97 @@ def token_mixer_recurrent(z: np.ndarray, S: np.ndarray, t: int, lw: dict, n_head
     q = z @ lw["W_in"].T
     yh, S_new = mixer_recurrent_step(q, S, t, lw["alpha"], lw["beta"], lw["lam"], n_heads)
     return yh @ lw["W_out"].T, S_new
+
+
+# --------------------------------------------------------------------------------------
+# Linearly combined heads (Architecture: every head holds one row-repeat and one column-repeat
+# matrix and its output is a linear combination of the two products; twice the cache).
+# Reading: the combination weights are two scalars per head, w[g] = (w_row, w_col); the per-position
+# bias beta is added once.
+# --------------------------------------------------------------------------------------
+
+def combined_parallel(Z, alpha_r, alpha_c, beta, lam_r, lam_c, w, n_heads: int):
+    """Z[n, d] -> Y[n, d] and the two hand-off caches S_r[d], S_c[d] for position n.
+    Head g, channel slice c:  Y_c^T = w[g,0] Z_c^T M_row(alpha_r[g], lam_r[g])
+                                    + w[g,1] Z_c^T M_col(alpha_c[g], lam_c[g]) + beta_c^T."""
+    n, d = Z.shape
+    dh = d // n_heads
+    dt = Z.dtype.type
+    Y = np.empty_like(Z)
+    S_r = np.zeros(d, dtype=Z.dtype)
+    S_c = np.zeros(d, dtype=Z.dtype)
+    for g in range(n_heads):
+        c = slice(g * dh, (g + 1) * dh)
+        Mr = mixing_matrix("row", alpha_r[g], lam_r[g], n, dtype=dt)
+        Mc = mixing_matrix("col", alpha_c[g], lam_c[g], n, dtype=dt)
+        X = Z[:, c].T
+        Y[:, c] = (dt(w[g][0]) * (X @ Mr) + dt(w[g][1]) * (X @ Mc)).T + beta[:n, c]
+        for m in range(n):
+            S_r[c] += dt(lam_r[g]) ** (n - m) * dt(alpha_r[g][m]) * Z[m, c]
+            S_c[c] += dt(lam_c[g]) ** (n - m) * Z[m, c]
+    return Y, S_r, S_c
+
+
+def combined_recurrent_step(z, S_r, S_c, t: int, alpha_r, alpha_c, beta, lam_r, lam_c, w, n_heads: int):
+    """Recurrent form of combined_parallel at position t (batched over leading dimensions):
+      y    = w_row (alpha_r[t] z + S_r) + w_col alpha_c[t] (z + S_c) + beta_t      (Eq. 2 and Eq. 3, combined)
+      S_r' = lam_r (S_r + alpha_r[t] z) ;  S_c' = lam_c (S_c + z)."""
+    d = z.shape[-1]
+    dh = d // n_heads
+    dt = z.dtype.type
+    y = np.empty_like(z)
+    Sr_new, Sc_new = np.empty_like(S_r), np.empty_like(S_c)
+    for g in range(n_heads):
+        c = slice(g * dh, (g + 1) * dh)
+        ar, ac = dt(alpha_r[g][t]), dt(alpha_c[g][t])
+        u = ar * z[..., c]
+        v = z[..., c] + S_c[..., c]
+        y[..., c] = dt(w[g][0]) * (u + S_r[..., c]) + dt(w[g][1]) * (ac * v) + beta[t, c]
+        Sr_new[..., c] = dt(lam_r[g]) * (S_r[..., c] + u)
+        Sc_new[..., c] = dt(lam_c[g]) * v
+    return y, Sr_new, Sc_new
+
+
+# --------------------------------------------------------------------------------------
+# Non-unitary kernels (Architecture, Eq. 11): Y = sum_{i<k} X_(i:d+i, :) W_i + beta with k column-repeat
+# matrices W_i and X zero-padded to d + k rows, stride 1.
+# Readings: the sum runs over the k filters i = 0..k-1 (the printed upper limit k would index a filter
+# that W in R^{k x n x n} does not have); the zero rows follow the d hidden channels, so that output
+# channel c mixes hidden channels c..c+k-1 and channels past d-1 contribute nothing; one set of k filters
+# serves the whole hidden dimension (the equation has no head index).
+# --------------------------------------------------------------------------------------
+
+def kernel_parallel(Z, alpha, beta, lam, k: int):
+    """Z[n, d] -> Y[n, d] by Eq. 11 as written, and the hand-off cache P[k, d] for position n:
+    P[i] = sum_{m<n} lam[i]^(n-m) z_m (the sum term of Eq. 3 for filter i over the unpadded channels).
+    alpha[k, >=n], lam[k], beta[>=n, d]."""
+    n, d = Z.shape
+    dt = Z.dtype.type
+    Xpad = np.zeros((d + k, n), dtype=Z.dtype)
+    Xpad[:d] = Z.T
+    Yt = np.zeros((d, n), dtype=Z.dtype)
+    for i in range(k):
+        Yt += Xpad[i:d + i, :] @ mixing_matrix("col", alpha[i], lam[i], n, dtype=dt)
+    P = np.zeros((k, d), dtype=Z.dtype)
+    for i in range(k):
+        for m in range(n):
+            P[i] += dt(lam[i]) ** (n - m) * Z[m]
+    return Yt.T + beta[:n], P
+
+
+def kernel_recurrent_step(z, P, t: int, alpha, beta, lam, k: int):
+    """Recurrent form of kernel_parallel at position t. z[..., d], P[k, ..., d].
+      v_i = z + P_i ;  y[c] = sum_i alpha[i][t] v_i[c + i] (terms with c + i >= d are the zero padding) + beta_t[c]
+      P_i' = lam[i] v_i."""
+    d = z.shape[-1]
+    dt = z.dtype.type
+    y = np.zeros_like(z)
+    P_new = np.empty_like(P)
+    for i in range(k):
+        v = z + P[i]
+        y[..., :d - i] += dt(alpha[i][t]) * v[..., i:]
+        P_new[i] = dt(lam[i]) * v
+    return y + beta[t], P_new
 
 
 # --------------------------------------------------------------------------------------
