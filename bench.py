@@ -507,6 +507,48 @@ def run_sweep(args):
     print(json.dumps(line), flush=True)
 
 
+def run_variants(args):
+    """Device time of the recurrent step of the two further mixer variants (linearly combined heads; kernels of
+    size k, Eq. 11) on 65536 rows of d = 1024, against the bytes the step has to move. One JSON line."""
+    import torch
+    import paper_2605_08696_b200 as P
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    peaks, peak_src = measured_peaks()
+    R, d, h, n_ctx = 65536, 1024, 4, 16
+    gen = torch.Generator(device=dev).manual_seed(0)
+    rnd = lambda *s: torch.randn(*s, device=dev, generator=gen)
+    uni = lambda *s: torch.rand(*s, device=dev, generator=gen)
+
+    def timed(f, n=20):
+        for _ in range(3):
+            f()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(n):
+            f()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / n
+
+    z, y, beta = rnd(R, d), torch.empty(R, d, device=dev), rnd(n_ctx, d)
+    S_r, S_c = rnd(R, d), rnd(R, d)
+    a, lam, w = uni(h, n_ctx), uni(h) * 0.5, uni(h, 2)
+    out = []
+    ms = timed(lambda: P.k_mixer_combined_step(3, z, S_r, S_c, a, a, beta, lam, lam, w, y))
+    out.append({"kernel": "combined_step_kernel", "rows": R, "d": d, "us": round(ms * 1e3, 1),
+                "gbs": round(R * d * 24 / ms / 1e6, 1)})
+    for k in (4, 8):
+        Pk, al, lk = rnd(k, R, d), uni(k, n_ctx), uni(k) * 0.5
+        ms = timed(lambda: P.k_mixer_kernel_step(3, z, Pk, al, beta, lk, y))
+        out.append({"kernel": "kernel_mix_step_kernel", "k": k, "rows": R, "d": d, "us": round(ms * 1e3, 1),
+                    "gbs": round(R * d * 4 * (2 * k + 2) / ms / 1e6, 1)})
+    for o in out:
+        o["frac_of_hbm_peak"] = round(o["gbs"] / peaks["hbm_gbs"], 3)
+    print(json.dumps({"variants": out, "peak": f"{peak_src}: {peaks['hbm_gbs']} GB/s", "inputs": "larger than L2"}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -537,11 +579,15 @@ def main():
                     help="skip the prefill (cache stays zero, pos = prompt length): keeps profiler captures short")
     ap.add_argument("--sweep", action="store_true")
     ap.add_argument("--sweep-max", type=int, default=0)
+    ap.add_argument("--variants", action="store_true",
+                    help="time the stand-alone steps of the combined-head and kernel-size-k mixers")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
     elif args.sweep:
         run_sweep(args)
+    elif args.variants:
+        run_variants(args)
     else:
         run_ours(args)
 

@@ -277,6 +277,27 @@ int srm_decode_step_static(srm_model* m, srm_state* s, const int32_t* d_tok_in,
  * d_x float[R, d] in/out, d_S [R, d] in state_dtype in/out, d_a [R, d] out. */
 int srm_k_mixer_step(srm_model* m, int32_t layer, int32_t t, int64_t R, const int32_t* d_tok,
                      float* d_x, void* d_S, void* d_a, uint32_t* d_status, void* stream);
+/* Recurrent step of a layer with LINEARLY COMBINED heads [Architecture: every head holds one row-repeat and
+ * one column-repeat matrix, the two products are combined linearly; twice the cache] on R rows of normed
+ * inputs at position t, fp32, no model handle (all arrays are the caller's device memory, 16-byte aligned):
+ *   y     = w[g][0] (alpha_row[g][t] z + S_row) + w[g][1] alpha_col[g][t] (z + S_col) + beta[t]   [Eq. 2, Eq. 3]
+ *   S_row <- lam_row[g] (S_row + alpha_row[g][t] z);   S_col <- lam_col[g] (S_col + z)
+ * for head g = channel / (d / n_heads). d_z, d_y float[R, d]; d_S_row, d_S_col float[R, d] in/out;
+ * d_alpha_row, d_alpha_col float[n_heads, n_ctx]; d_beta float[n_ctx, d]; d_lam_row, d_lam_col float[n_heads];
+ * d_w float[n_heads, 2]. d / n_heads must be a multiple of 4 (SRM_ERR_UNSUPPORTED); t >= n_ctx is
+ * SRM_ERR_CTX_OVERFLOW. Asynchronous on `stream`. */
+int srm_k_mixer_combined_step(int64_t R, int32_t d, int32_t n_heads, int32_t t, int32_t n_ctx, const float* d_z,
+                              float* d_S_row, float* d_S_col, const float* d_alpha_row, const float* d_alpha_col,
+                              const float* d_beta, const float* d_lam_row, const float* d_lam_col, const float* d_w,
+                              float* d_y, void* stream);
+/* Recurrent step of a layer with a NON-UNITARY KERNEL of size k [Eq. 11: k column-repeat filters, filter i
+ * applied to the hidden channels shifted by i, X zero-padded past its last channel, stride 1], fp32:
+ *   v_i = z + P_i;   y[c] = sum_{i < k, c + i < d} alpha[i][t] v_i[c + i] + beta[t][c];   P_i <- lam[i] v_i
+ * d_z, d_y float[R, d]; d_P float[k, R, d] in/out (the sum term of Eq. 3 per filter: k times the cache);
+ * d_alpha float[k, n_ctx]; d_beta float[n_ctx, d]; d_lam float[k]. Needs d % 4 == 0, k <= 16, k <= d and
+ * k * d * 4 bytes of shared memory within 200 KB, else SRM_ERR_UNSUPPORTED. Asynchronous on `stream`. */
+int srm_k_mixer_kernel_step(int64_t R, int32_t d, int32_t k, int32_t t, int32_t n_ctx, const float* d_z, float* d_P,
+                            const float* d_alpha, const float* d_beta, const float* d_lam, float* d_y, void* stream);
 /* out = LN_f(x) in the activation type: d_x float[R, d] -> d_a [R, d]. */
 int srm_k_final_norm(srm_model* m, int64_t R, const float* d_x, void* d_a, void* stream);
 /* Dense projection D[M, N] = A[M, K] * W[N, K]^T with one of three epilogues:

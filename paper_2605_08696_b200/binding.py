@@ -98,6 +98,8 @@ SYMBOLS = {
     "srm_k_gemm_splitk_order_bytes": (_SZ, [_I64, _I64]),
     "srm_k_gemm_splitk": (C.c_int, [_P, _I64, _I64, _I64, _P, _P, _P, _P, _P, _SZ, _P, _P]),
     "srm_k_gemm_splitk_plan": (_I64, [_I64, _I64, _I64, _I32, _I32, C.POINTER(_I64), _I64]),
+    "srm_k_mixer_combined_step": (C.c_int, [_I64, _I32, _I32, _I32, _I32] + [_P] * 11),
+    "srm_k_mixer_kernel_step": (C.c_int, [_I64, _I32, _I32, _I32, _I32] + [_P] * 7),
     "srm_k_lm_head_greedy": (C.c_int, [_P, _I64, _P, _P, _SZ, _P, _P, _P]),
     "srm_k_select": (C.c_int, [_P, _I64, _P, C.POINTER(_Sampling), _I32, _P, _P, _P]),
     "srm_k_prefill_mixer": (C.c_int, [_P, _I32, _I64, _I32, _P, _P, _P, _P, _P, _P]),
@@ -155,6 +157,25 @@ def _stream():
 
 def _shape_get(shape, key):
     return shape[key] if isinstance(shape, dict) else getattr(shape, key)
+
+
+def k_mixer_combined_step(t, z, S_row, S_col, alpha_row, alpha_col, beta, lam_row, lam_col, w, y):
+    """Recurrent step of a layer with linearly combined heads (srm_k_mixer_combined_step): fp32 CUDA tensors,
+    z, y, S_row, S_col [R, d]; alpha_* [h, n_ctx]; beta [n_ctx, d]; lam_* [h]; w [h, 2]. Updates S_row, S_col, y."""
+    R, d = z.shape
+    h, n_ctx = alpha_row.shape
+    _check(_lib().srm_k_mixer_combined_step(R, d, h, t, n_ctx, _ptr(z), _ptr(S_row), _ptr(S_col), _ptr(alpha_row),
+                                            _ptr(alpha_col), _ptr(beta), _ptr(lam_row), _ptr(lam_col), _ptr(w), _ptr(y),
+                                            _stream()), "srm_k_mixer_combined_step")
+
+
+def k_mixer_kernel_step(t, z, P, alpha, beta, lam, y):
+    """Recurrent step of a layer with a kernel of size k (Eq. 11; srm_k_mixer_kernel_step): fp32 CUDA tensors,
+    z, y [R, d]; P [k, R, d]; alpha [k, n_ctx]; beta [n_ctx, d]; lam [k]. Updates P and y."""
+    R, d = z.shape
+    k, n_ctx = alpha.shape
+    _check(_lib().srm_k_mixer_kernel_step(R, d, k, t, n_ctx, _ptr(z), _ptr(P), _ptr(alpha), _ptr(beta), _ptr(lam), _ptr(y),
+                                          _stream()), "srm_k_mixer_kernel_step")
 
 
 class SRMState:

@@ -21,6 +21,7 @@
 #include "mixer.cuh"
 #include "mixer_stream.cuh"
 #include "mixer_proj.cuh"
+#include "mixer_variants.cuh"
 #include "prefill.cuh"
 #include "prefill_scan.cuh"
 #include "select.cuh"
@@ -1251,6 +1252,62 @@ int srm_k_mixer_step(srm_model* m, int32_t layer, int32_t t, int64_t R, const in
   if (t >= m->cfg.n_ctx) return SRM_ERR_CTX_OVERFLOW;
   if (!aligned(d_x, 16) || !aligned(d_S, 16) || !aligned(d_a, 16)) return SRM_ERR_ALIGNMENT;
   return launch_mixer(*m, layer, t, R, d_tok, d_x, d_S, d_a, d_status, static_cast<cudaStream_t>(stream));
+}
+
+namespace {
+int device_sm_count(int* sms) {
+  int dev = 0;
+  SRM_CUDA(cudaGetDevice(&dev));
+  SRM_CUDA(cudaDeviceGetAttribute(sms, cudaDevAttrMultiProcessorCount, dev));
+  return SRM_OK;
+}
+}  // namespace
+
+int srm_k_mixer_combined_step(int64_t R, int32_t d, int32_t n_heads, int32_t t, int32_t n_ctx, const float* d_z,
+                              float* d_S_row, float* d_S_col, const float* d_alpha_row, const float* d_alpha_col,
+                              const float* d_beta, const float* d_lam_row, const float* d_lam_col, const float* d_w,
+                              float* d_y, void* stream) {
+  if (R < 0 || d < 4 || n_heads < 1 || n_ctx < 1 || t < 0) return SRM_ERR_INVALID_ARG;
+  if (t >= n_ctx) return SRM_ERR_CTX_OVERFLOW;
+  if (d % n_heads || (d / n_heads) % 4) return SRM_ERR_UNSUPPORTED;
+  if (R == 0) return SRM_OK;
+  if (!d_z || !d_S_row || !d_S_col || !d_alpha_row || !d_alpha_col || !d_beta || !d_lam_row || !d_lam_col || !d_w || !d_y)
+    return SRM_ERR_INVALID_ARG;
+  if (!aligned(d_z, 16) || !aligned(d_S_row, 16) || !aligned(d_S_col, 16) || !aligned(d_beta, 16) || !aligned(d_y, 16))
+    return SRM_ERR_ALIGNMENT;
+  int sms = 0, rc = device_sm_count(&sms);
+  if (rc != SRM_OK) return rc;
+  CombinedParams p{R, d, n_heads, t, n_ctx, d_z, d_S_row, d_S_col, d_alpha_row, d_alpha_col, d_beta, d_lam_row, d_lam_col, d_w, d_y};
+  const int64_t blocks = (R * (d / 4) + kVariantThreads - 1) / kVariantThreads, cap = (int64_t)sms * 8;
+  ++g_kernel_launches;
+  SRM_CUDA(launch_kernel(combined_step_kernel, dim3((unsigned)(blocks < cap ? blocks : cap)), dim3(kVariantThreads), 0,
+                         static_cast<cudaStream_t>(stream), p));
+  return SRM_OK;
+}
+
+int srm_k_mixer_kernel_step(int64_t R, int32_t d, int32_t k, int32_t t, int32_t n_ctx, const float* d_z, float* d_P,
+                            const float* d_alpha, const float* d_beta, const float* d_lam, float* d_y, void* stream) {
+  if (R < 0 || d < 4 || k < 1 || n_ctx < 1 || t < 0) return SRM_ERR_INVALID_ARG;
+  if (t >= n_ctx) return SRM_ERR_CTX_OVERFLOW;
+  if (d % 4 || k > kKernelMixMaxK || k > d || kernel_mix_smem(d, k) > 200 * 1024) return SRM_ERR_UNSUPPORTED;
+  if (R == 0) return SRM_OK;
+  if (!d_z || !d_P || !d_alpha || !d_beta || !d_lam || !d_y) return SRM_ERR_INVALID_ARG;
+  if (!aligned(d_z, 16) || !aligned(d_P, 16) || !aligned(d_y, 16)) return SRM_ERR_ALIGNMENT;
+  int sms = 0, rc = device_sm_count(&sms);
+  if (rc != SRM_OK) return rc;
+  static std::once_flag once;
+  static cudaError_t attr_err = cudaSuccess;
+  std::call_once(once, [] {
+    attr_err = cudaFuncSetAttribute(kernel_mix_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+  });
+  SRM_CUDA(attr_err);
+  KernelMixParams p{R, d, k, t, n_ctx, d_z, d_P, d_alpha, d_beta, d_lam, d_y};
+  const size_t smem = kernel_mix_smem(d, k);
+  const int64_t per_sm = (int64_t)(200 * 1024 / smem) < 8 ? (int64_t)(200 * 1024 / smem) : 8, cap = (int64_t)sms * per_sm;
+  ++g_kernel_launches;
+  SRM_CUDA(launch_kernel(kernel_mix_step_kernel, dim3((unsigned)(R < cap ? R : cap)), dim3(kVariantThreads), smem,
+                         static_cast<cudaStream_t>(stream), p));
+  return SRM_OK;
 }
 
 int srm_k_final_norm(srm_model* m, int64_t R, const float* d_x, void* d_a, void* stream) {
