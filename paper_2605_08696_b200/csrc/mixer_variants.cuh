@@ -80,16 +80,25 @@ __global__ void __launch_bounds__(kVariantThreads) kernel_mix_step_kernel(const 
   __syncthreads();
   pdl_wait();
   const float* bt = p.beta + (int64_t)p.t * d;
+  const int64_t plane = p.R * (int64_t)d;
   for (int64_t row = blockIdx.x; row < p.R; row += gridDim.x) {
     for (int e = threadIdx.x * 4; e < d; e += kVariantThreads * 4) {
       const float4 z = ld4(p.z + row * d + e);
-      for (int i = 0; i < k; ++i) {
-        float* Pi = p.P + ((int64_t)i * p.R + row) * d + e;
-        const float4 s = ld4(Pi);
-        const float4 v = make_float4(z.x + s.x, z.y + s.y, z.z + s.z, z.w + s.w);
-        st4(vs + (size_t)i * d + e, v);
-        const float l = l_s[i];
-        st4(Pi, make_float4(l * v.x, l * v.y, l * v.z, l * v.w));
+      float* P0 = p.P + row * d + e;
+      for (int i0 = 0; i0 < k; i0 += 4) {          // four filters' loads in flight before the first store
+        float4 s[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+          if (i0 + u < k) s[u] = ld4(P0 + (int64_t)(i0 + u) * plane);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          if (i0 + u < k) {
+            const float4 v = make_float4(z.x + s[u].x, z.y + s[u].y, z.z + s[u].z, z.w + s[u].w);
+            st4(vs + (size_t)(i0 + u) * d + e, v);
+            const float l = l_s[i0 + u];
+            st4(P0 + (int64_t)(i0 + u) * plane, make_float4(l * v.x, l * v.y, l * v.z, l * v.w));
+          }
+        }
       }
     }
     __syncthreads();

@@ -1303,7 +1303,10 @@ int srm_k_mixer_kernel_step(int64_t R, int32_t d, int32_t k, int32_t t, int32_t 
   SRM_CUDA(attr_err);
   KernelMixParams p{R, d, k, t, n_ctx, d_z, d_P, d_alpha, d_beta, d_lam, d_y};
   const size_t smem = kernel_mix_smem(d, k);
-  const int64_t per_sm = (int64_t)(200 * 1024 / smem) < 8 ? (int64_t)(200 * 1024 / smem) : 8, cap = (int64_t)sms * per_sm;
+  // one wave of resident blocks: a second, partly filled wave would run at a fraction of the bandwidth
+  int per_sm = 0;
+  SRM_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel_mix_step_kernel, kVariantThreads, smem));
+  const int64_t cap = (int64_t)sms * (per_sm < 1 ? 1 : per_sm);
   ++g_kernel_launches;
   SRM_CUDA(launch_kernel(kernel_mix_step_kernel, dim3((unsigned)(R < cap ? R : cap)), dim3(kVariantThreads), smem,
                          static_cast<cudaStream_t>(stream), p));
