@@ -1278,6 +1278,8 @@ int srm_k_mixer_combined_step(int64_t R, int32_t d, int32_t n_heads, int32_t t, 
   int sms = 0, rc = device_sm_count(&sms);
   if (rc != SRM_OK) return rc;
   CombinedParams p{R, d, n_heads, t, n_ctx, d_z, d_S_row, d_S_col, d_alpha_row, d_alpha_col, d_beta, d_lam_row, d_lam_col, d_w, d_y};
+  // 8 blocks per SM, of which 5 are resident: measured 256 us per 65536 x 1024 against 273 us with exactly one
+  // resident wave (each thread then walks more elements with three loads in flight)
   const int64_t blocks = (R * (d / 4) + kVariantThreads - 1) / kVariantThreads, cap = (int64_t)sms * 8;
   ++g_kernel_launches;
   SRM_CUDA(launch_kernel(combined_step_kernel, dim3((unsigned)(blocks < cap ? blocks : cap)), dim3(kVariantThreads), 0,
