@@ -146,6 +146,9 @@ size_t srm_state_bytes(const srm_config* cfg, int64_t B);
  * batch runs as equal passes of at most 10240 rows (whole 256-row tiles), which keeps a layer's
  * activations in L2 between its kernels; results do not depend on the split. */
 size_t srm_workspace_bytes(const srm_config* cfg, int64_t B_chunk, int32_t n_prefill_max);
+/* Rows per decode pass that a batch of B samples is processed in when the workspace has room for
+ * `ws_rows` rows (the rule stated above; host only, no device work). 0 if B < 1 or ws_rows < 1. */
+int64_t srm_decode_pass_rows(int64_t B, int64_t ws_rows);
 
 /* ---- handles ------------------------------------------------------------------------------ */
 

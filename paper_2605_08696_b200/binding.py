@@ -107,6 +107,7 @@ SYMBOLS = {
     "srm_profile_read": (C.c_int, [_P, _I32, C.POINTER(C.c_uint64), C.POINTER(C.c_double)]),
     "srm_profile_reset": (C.c_int, [_P]),
     "srm_kernel_launches": (C.c_uint64, []),
+    "srm_decode_pass_rows": (_I64, [_I64, _I64]),
     "srm_strerror": (C.c_char_p, [C.c_int]),
     "srm_last_cuda_error": (C.c_int, []),
     "srm_version": (C.c_char_p, []),

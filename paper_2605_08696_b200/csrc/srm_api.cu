@@ -916,6 +916,8 @@ int srm_profile_reset(srm_model* m) {
 
 uint64_t srm_kernel_launches(void) { return g_kernel_launches; }
 
+int64_t srm_decode_pass_rows(int64_t B, int64_t ws_rows) { return B < 1 || ws_rows < 1 ? 0 : choose_pass_rows(B, ws_rows); }
+
 int srm_state_create(srm_model* m, int64_t B, void* d_state, size_t nbytes, void* stream, srm_state** out) {
   if (out == nullptr) return SRM_ERR_INVALID_ARG;
   *out = nullptr;

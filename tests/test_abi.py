@@ -86,3 +86,24 @@ def test_null_and_alignment_errors_without_device_work():
     assert lib.srm_decode_step(None, None, None, None, 0, None, None, None, 0, None) == -1
     assert lib.srm_strerror(-5) == b"position would exceed n_ctx"
     assert lib.srm_state_pos(None) == -1
+
+
+def test_decode_pass_rows_rule():
+    """Small batches run as one pass, large ones as equal passes of whole 256-row tiles of at most 10240 rows,
+    and a small workspace decides by itself. Every pass size is positive and the passes cover the batch."""
+    lib = P.load_library()
+    f = lib.srm_decode_pass_rows
+    assert f(0, 100) == 0 and f(100, 0) == 0
+    assert f(1, 1 << 20) == 1 and f(4096, 1 << 20) == 4096 and f(12288, 1 << 20) == 12288
+    assert f(16384, 1 << 20) == 8192 and f(32768, 1 << 20) == 8192 and f(37888, 1 << 20) == 9472
+    assert f(20000, 1 << 20) == 10240                      # two passes: 10240 + 9760
+    assert f(12289, 1 << 20) == 6400                       # two passes of 25 tiles
+    assert f(4096, 1000) == 1000 and f(100000, 8192) == 8192 and f(100000, 300) == 300
+    assert f(8192, 8192) == 8192 and f(8192, 8191) == 8191
+    assert f(1 << 21, 49152) == 10240
+    for B in (1, 255, 6145, 12288, 12289, 16385, 99999, 1 << 21):
+        for fit in (1, 255, 4096, 10239, 10240, 16384, 1 << 22):
+            r = f(B, fit)
+            assert 1 <= r <= min(B, fit), (B, fit, r)
+            if B > 12288 and fit >= 10240:
+                assert r % 256 == 0 and r <= 10240
