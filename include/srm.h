@@ -301,6 +301,18 @@ int srm_k_mixer_combined_step(int64_t R, int32_t d, int32_t n_heads, int32_t t, 
  * k * d * 4 bytes of shared memory within 200 KB, else SRM_ERR_UNSUPPORTED. Asynchronous on `stream`. */
 int srm_k_mixer_kernel_step(int64_t R, int32_t d, int32_t k, int32_t t, int32_t n_ctx, const float* d_z, float* d_P,
                             const float* d_alpha, const float* d_beta, const float* d_lam, float* d_y, void* stream);
+/* The same two variants over whole sequences (the prefill form, evaluated through the recurrence): d_Z, d_Y
+ * float[Bp, n, d] hold positions t0 .. t0 + n - 1 of Bp samples; the caches (d_S_row, d_S_col float[Bp, d];
+ * d_P float[k, Bp, d]) enter as the sum terms for position t0 (zeros for a fresh prompt) and leave as those for
+ * position t0 + n. Equal to the product with the explicit n x n matrices [Eq. 1, Eq. 3, Eq. 11] up to rounding
+ * order. Parameters as in the step calls; t0 + n > n_ctx is SRM_ERR_CTX_OVERFLOW; the kernel-size-k call needs
+ * 2 k d * 4 bytes of shared memory within 200 KB (SRM_ERR_UNSUPPORTED). */
+int srm_k_mixer_combined_scan(int64_t Bp, int32_t n, int32_t t0, int32_t d, int32_t n_heads, int32_t n_ctx, const float* d_Z,
+                              float* d_S_row, float* d_S_col, const float* d_alpha_row, const float* d_alpha_col,
+                              const float* d_beta, const float* d_lam_row, const float* d_lam_col, const float* d_w,
+                              float* d_Y, void* stream);
+int srm_k_mixer_kernel_scan(int64_t Bp, int32_t n, int32_t t0, int32_t d, int32_t k, int32_t n_ctx, const float* d_Z, float* d_P,
+                            const float* d_alpha, const float* d_beta, const float* d_lam, float* d_Y, void* stream);
 /* out = LN_f(x) in the activation type: d_x float[R, d] -> d_a [R, d]. */
 int srm_k_final_norm(srm_model* m, int64_t R, const float* d_x, void* d_a, void* stream);
 /* Dense projection D[M, N] = A[M, K] * W[N, K]^T with one of three epilogues:

@@ -5,5 +5,5 @@ torch device buffers and streams into the calls, nothing else. All arithmetic of
 in the CUDA kernels under csrc/.
 """
 from .binding import (SRM, SRMState, Sampling, SRMError, load_library, lib_path,  # noqa: F401
-                      k_mixer_combined_step, k_mixer_kernel_step,
+                      k_mixer_combined_step, k_mixer_kernel_step, k_mixer_combined_scan, k_mixer_kernel_scan,
                       EPI_BIAS_GELU, EPI_BIAS_RESIDUAL, EPI_PLAIN, FLAG_NO_GRAPH, FLAG_GRAPH, FLAG_NO_SPLITK)

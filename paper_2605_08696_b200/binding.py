@@ -100,6 +100,8 @@ SYMBOLS = {
     "srm_k_gemm_splitk_plan": (_I64, [_I64, _I64, _I64, _I32, _I32, C.POINTER(_I64), _I64]),
     "srm_k_mixer_combined_step": (C.c_int, [_I64, _I32, _I32, _I32, _I32] + [_P] * 11),
     "srm_k_mixer_kernel_step": (C.c_int, [_I64, _I32, _I32, _I32, _I32] + [_P] * 7),
+    "srm_k_mixer_combined_scan": (C.c_int, [_I64, _I32, _I32, _I32, _I32, _I32] + [_P] * 11),
+    "srm_k_mixer_kernel_scan": (C.c_int, [_I64, _I32, _I32, _I32, _I32, _I32] + [_P] * 7),
     "srm_k_lm_head_greedy": (C.c_int, [_P, _I64, _P, _P, _SZ, _P, _P, _P]),
     "srm_k_select": (C.c_int, [_P, _I64, _P, C.POINTER(_Sampling), _I32, _P, _P, _P]),
     "srm_k_prefill_mixer": (C.c_int, [_P, _I32, _I64, _I32, _P, _P, _P, _P, _P, _P]),
@@ -177,6 +179,23 @@ def k_mixer_kernel_step(t, z, P, alpha, beta, lam, y):
     k, n_ctx = alpha.shape
     _check(_lib().srm_k_mixer_kernel_step(R, d, k, t, n_ctx, _ptr(z), _ptr(P), _ptr(alpha), _ptr(beta), _ptr(lam), _ptr(y),
                                           _stream()), "srm_k_mixer_kernel_step")
+
+
+def k_mixer_combined_scan(t0, Z, S_row, S_col, alpha_row, alpha_col, beta, lam_row, lam_col, w, Y):
+    """Positions t0 .. t0+n-1 of a layer with linearly combined heads (srm_k_mixer_combined_scan): Z, Y [Bp, n, d]."""
+    Bp, n, d = Z.shape
+    h, n_ctx = alpha_row.shape
+    _check(_lib().srm_k_mixer_combined_scan(Bp, n, t0, d, h, n_ctx, _ptr(Z), _ptr(S_row), _ptr(S_col), _ptr(alpha_row),
+                                            _ptr(alpha_col), _ptr(beta), _ptr(lam_row), _ptr(lam_col), _ptr(w), _ptr(Y),
+                                            _stream()), "srm_k_mixer_combined_scan")
+
+
+def k_mixer_kernel_scan(t0, Z, P, alpha, beta, lam, Y):
+    """Positions t0 .. t0+n-1 of a layer with a kernel of size k (srm_k_mixer_kernel_scan): Z, Y [Bp, n, d], P [k, Bp, d]."""
+    Bp, n, d = Z.shape
+    k, n_ctx = alpha.shape
+    _check(_lib().srm_k_mixer_kernel_scan(Bp, n, t0, d, k, n_ctx, _ptr(Z), _ptr(P), _ptr(alpha), _ptr(beta), _ptr(lam),
+                                          _ptr(Y), _stream()), "srm_k_mixer_kernel_scan")
 
 
 class SRMState:

@@ -112,4 +112,142 @@ __global__ void __launch_bounds__(kVariantThreads) kernel_mix_step_kernel(const 
   }
 }
 
+// ---- the same two variants over whole sequences (the prefill form, through the recurrence) -----------------
+// Z[Bp, n, d] holds n consecutive positions t0 .. t0 + n - 1 of Bp samples; the caches enter as the sum terms
+// for position t0 (zeros for a fresh prompt) and leave as the sum terms for position t0 + n. The result equals
+// the product with the explicit n x n matrices of Eq. 1 / Eq. 3 (and Eq. 11) up to rounding order.
+
+struct CombinedScanParams {
+  int64_t Bp;
+  int n, t0, d, h, n_ctx;
+  const float* Z;                 // [Bp, n, d]
+  float *S_row, *S_col;           // [Bp, d] in/out
+  const float *alpha_row, *alpha_col, *beta, *lam_row, *lam_col, *w;
+  float* Y;                       // [Bp, n, d]
+};
+
+// One thread owns four channels of one sample and walks the positions with both sum terms in registers; the
+// inputs of four positions are in flight at a time (they do not depend on the recurrence). 8 d bytes per position.
+__global__ void __launch_bounds__(kVariantThreads) combined_scan_kernel(const CombinedScanParams p) {
+  pdl_trigger();
+  pdl_wait();
+  const int q = p.d >> 2, dh = p.d / p.h;
+  const int64_t n4 = p.Bp * q;
+  for (int64_t idx = (int64_t)blockIdx.x * kVariantThreads + threadIdx.x; idx < n4; idx += (int64_t)gridDim.x * kVariantThreads) {
+    const int64_t b = idx / q;
+    const int c = (int)(idx - b * q) << 2;
+    const int g = c / dh;
+    const float lr = __ldg(p.lam_row + g), lc = __ldg(p.lam_col + g);
+    const float wr = __ldg(p.w + 2 * g), wc0 = __ldg(p.w + 2 * g + 1);
+    const float* ar_g = p.alpha_row + (int64_t)g * p.n_ctx + p.t0;
+    const float* ac_g = p.alpha_col + (int64_t)g * p.n_ctx + p.t0;
+    const float* bt = p.beta + (int64_t)p.t0 * p.d + c;
+    const float* zp = p.Z + b * p.n * (int64_t)p.d + c;
+    float* yp = p.Y + b * p.n * (int64_t)p.d + c;
+    float4 sr = ld4(p.S_row + b * p.d + c), sc = ld4(p.S_col + b * p.d + c);
+    for (int j0 = 0; j0 < p.n; j0 += 4) {
+      float4 z[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (j0 + u < p.n) z[u] = ld4(zp + (int64_t)(j0 + u) * p.d);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int j = j0 + u;
+        if (j < p.n) {
+          const float ar = __ldg(ar_g + j), wc = wc0 * __ldg(ac_g + j);
+          const float4 b4 = ldg4(bt + (int64_t)j * p.d);
+          const float4 uu = make_float4(ar * z[u].x, ar * z[u].y, ar * z[u].z, ar * z[u].w);
+          const float4 v = make_float4(z[u].x + sc.x, z[u].y + sc.y, z[u].z + sc.z, z[u].w + sc.w);
+          float4 y;
+          y.x = fmaf(wr, uu.x + sr.x, fmaf(wc, v.x, b4.x)); y.y = fmaf(wr, uu.y + sr.y, fmaf(wc, v.y, b4.y));
+          y.z = fmaf(wr, uu.z + sr.z, fmaf(wc, v.z, b4.z)); y.w = fmaf(wr, uu.w + sr.w, fmaf(wc, v.w, b4.w));
+          st4(yp + (int64_t)j * p.d, y);
+          sr = make_float4(lr * (sr.x + uu.x), lr * (sr.y + uu.y), lr * (sr.z + uu.z), lr * (sr.w + uu.w));
+          sc = make_float4(lc * v.x, lc * v.y, lc * v.z, lc * v.w);
+        }
+      }
+    }
+    st4(p.S_row + b * p.d + c, sr);
+    st4(p.S_col + b * p.d + c, sc);
+  }
+}
+
+struct KernelScanParams {
+  int64_t Bp;
+  int n, t0, d, k, n_ctx;
+  const float* Z;        // [Bp, n, d]
+  float* P;              // [k, Bp, d] in/out
+  const float *alpha, *beta, *lam;
+  float* Y;              // [Bp, n, d]
+};
+inline size_t kernel_scan_smem(int d, int k) { return 2 * (size_t)k * d * 4 + kKernelMixMaxK * 4; }
+
+// One CTA owns a sample: the k sum terms live in shared memory for the whole sequence (each element touched by
+// one thread only), the k vectors z + P_i of the current position in a second slab that the shifted reads of
+// Eq. 11 take after a barrier. The next position's input is loaded before the barrier. 8 d bytes per position.
+__global__ void __launch_bounds__(kVariantThreads) kernel_scan_kernel(const KernelScanParams p) {
+  pdl_trigger();
+  extern __shared__ __align__(16) float ks[];            // P [k][d] | v [k][d] | lam_i
+  const int d = p.d, k = p.k;
+  float* Ps = ks;
+  float* vs = ks + (size_t)k * d;
+  float* l_s = vs + (size_t)k * d;
+  if (threadIdx.x < k) l_s[threadIdx.x] = __ldg(p.lam + threadIdx.x);
+  pdl_wait();
+  const int64_t plane = p.Bp * (int64_t)d;
+  constexpr int kMaxVec = 4;                              // float4 per thread held ahead: d <= 4096 prefetched
+  for (int64_t b = blockIdx.x; b < p.Bp; b += gridDim.x) {
+    __syncthreads();                                      // previous sample's slabs are no longer read
+    for (int e = threadIdx.x * 4; e < d; e += kVariantThreads * 4)
+      for (int i = 0; i < k; ++i) st4(Ps + (size_t)i * d + e, ld4(p.P + (int64_t)i * plane + b * d + e));
+    const float* zb = p.Z + b * p.n * (int64_t)d;
+    float* yb = p.Y + b * p.n * (int64_t)d;
+    float4 zn[kMaxVec];
+#pragma unroll
+    for (int m = 0; m < kMaxVec; ++m) {
+      const int e = (threadIdx.x + m * kVariantThreads) * 4;
+      if (e < d) zn[m] = ld4(zb + e);
+    }
+    for (int j = 0; j < p.n; ++j) {
+      int m = 0;
+      for (int e = threadIdx.x * 4; e < d; e += kVariantThreads * 4, ++m) {
+        float4 z;
+        if (m < kMaxVec) {
+#pragma unroll
+          for (int mm = 0; mm < kMaxVec; ++mm) if (mm == m) z = zn[mm];
+        } else {
+          z = ld4(zb + (int64_t)j * d + e);
+        }
+        for (int i = 0; i < k; ++i) {
+          float* Pi = Ps + (size_t)i * d + e;
+          const float4 s = ld4(Pi);
+          const float4 v = make_float4(z.x + s.x, z.y + s.y, z.z + s.z, z.w + s.w);
+          st4(vs + (size_t)i * d + e, v);
+          const float l = l_s[i];
+          st4(Pi, make_float4(l * v.x, l * v.y, l * v.z, l * v.w));
+        }
+      }
+      if (j + 1 < p.n) {
+#pragma unroll
+        for (int mm = 0; mm < kMaxVec; ++mm) {
+          const int e = (threadIdx.x + mm * kVariantThreads) * 4;
+          if (e < d) zn[mm] = ld4(zb + (int64_t)(j + 1) * d + e);
+        }
+      }
+      __syncthreads();
+      const float* bt = p.beta + (int64_t)(p.t0 + j) * d;
+      const float* al = p.alpha + p.t0 + j;
+      for (int c = threadIdx.x; c < d; c += kVariantThreads) {
+        float acc = __ldg(bt + c);
+        const int kk = d - c < k ? d - c : k;
+        for (int i = 0; i < kk; ++i) acc = fmaf(__ldg(al + (int64_t)i * p.n_ctx), vs[(size_t)i * d + c + i], acc);
+        yb[(int64_t)j * d + c] = acc;
+      }
+      __syncthreads();
+    }
+    for (int e = threadIdx.x * 4; e < d; e += kVariantThreads * 4)
+      for (int i = 0; i < k; ++i) st4(p.P + (int64_t)i * plane + b * d + e, ld4(Ps + (size_t)i * d + e));
+  }
+}
+
 }  // namespace srm

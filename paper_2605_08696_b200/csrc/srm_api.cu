@@ -1317,6 +1317,55 @@ int srm_k_mixer_kernel_step(int64_t R, int32_t d, int32_t k, int32_t t, int32_t 
   return SRM_OK;
 }
 
+int srm_k_mixer_combined_scan(int64_t Bp, int32_t n, int32_t t0, int32_t d, int32_t n_heads, int32_t n_ctx, const float* d_Z,
+                              float* d_S_row, float* d_S_col, const float* d_alpha_row, const float* d_alpha_col,
+                              const float* d_beta, const float* d_lam_row, const float* d_lam_col, const float* d_w,
+                              float* d_Y, void* stream) {
+  if (Bp < 0 || n < 1 || d < 4 || n_heads < 1 || n_ctx < 1 || t0 < 0) return SRM_ERR_INVALID_ARG;
+  if ((int64_t)t0 + n > n_ctx) return SRM_ERR_CTX_OVERFLOW;
+  if (d % n_heads || (d / n_heads) % 4) return SRM_ERR_UNSUPPORTED;
+  if (Bp == 0) return SRM_OK;
+  if (!d_Z || !d_S_row || !d_S_col || !d_alpha_row || !d_alpha_col || !d_beta || !d_lam_row || !d_lam_col || !d_w || !d_Y)
+    return SRM_ERR_INVALID_ARG;
+  if (!aligned(d_Z, 16) || !aligned(d_S_row, 16) || !aligned(d_S_col, 16) || !aligned(d_beta, 16) || !aligned(d_Y, 16))
+    return SRM_ERR_ALIGNMENT;
+  int sms = 0, rc = device_sm_count(&sms);
+  if (rc != SRM_OK) return rc;
+  CombinedScanParams p{Bp, n, t0, d, n_heads, n_ctx, d_Z, d_S_row, d_S_col, d_alpha_row, d_alpha_col, d_beta, d_lam_row, d_lam_col, d_w, d_Y};
+  const int64_t blocks = (Bp * (d / 4) + kVariantThreads - 1) / kVariantThreads, cap = (int64_t)sms * 8;
+  ++g_kernel_launches;
+  SRM_CUDA(launch_kernel(combined_scan_kernel, dim3((unsigned)(blocks < cap ? blocks : cap)), dim3(kVariantThreads), 0,
+                         static_cast<cudaStream_t>(stream), p));
+  return SRM_OK;
+}
+
+int srm_k_mixer_kernel_scan(int64_t Bp, int32_t n, int32_t t0, int32_t d, int32_t k, int32_t n_ctx, const float* d_Z, float* d_P,
+                            const float* d_alpha, const float* d_beta, const float* d_lam, float* d_Y, void* stream) {
+  if (Bp < 0 || n < 1 || d < 4 || k < 1 || n_ctx < 1 || t0 < 0) return SRM_ERR_INVALID_ARG;
+  if ((int64_t)t0 + n > n_ctx) return SRM_ERR_CTX_OVERFLOW;
+  if (d % 4 || k > kKernelMixMaxK || k > d || kernel_scan_smem(d, k) > 200 * 1024) return SRM_ERR_UNSUPPORTED;
+  if (Bp == 0) return SRM_OK;
+  if (!d_Z || !d_P || !d_alpha || !d_beta || !d_lam || !d_Y) return SRM_ERR_INVALID_ARG;
+  if (!aligned(d_Z, 16) || !aligned(d_P, 16) || !aligned(d_Y, 16)) return SRM_ERR_ALIGNMENT;
+  int sms = 0, rc = device_sm_count(&sms);
+  if (rc != SRM_OK) return rc;
+  static std::once_flag once;
+  static cudaError_t attr_err = cudaSuccess;
+  std::call_once(once, [] {
+    attr_err = cudaFuncSetAttribute(kernel_scan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+  });
+  SRM_CUDA(attr_err);
+  KernelScanParams p{Bp, n, t0, d, k, n_ctx, d_Z, d_P, d_alpha, d_beta, d_lam, d_Y};
+  const size_t smem = kernel_scan_smem(d, k);
+  int per_sm = 0;
+  SRM_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel_scan_kernel, kVariantThreads, smem));
+  const int64_t cap = (int64_t)sms * (per_sm < 1 ? 1 : per_sm);
+  ++g_kernel_launches;
+  SRM_CUDA(launch_kernel(kernel_scan_kernel, dim3((unsigned)(Bp < cap ? Bp : cap)), dim3(kVariantThreads), smem,
+                         static_cast<cudaStream_t>(stream), p));
+  return SRM_OK;
+}
+
 int srm_k_final_norm(srm_model* m, int64_t R, const float* d_x, void* d_a, void* stream) {
   if (m == nullptr || R < 0) return SRM_ERR_INVALID_ARG;
   if (R == 0) return SRM_OK;
