@@ -544,6 +544,20 @@ def run_variants(args):
         ms = timed(lambda: P.k_mixer_kernel_step(3, z, Pk, al, beta, lk, y))
         out.append({"kernel": "kernel_mix_step_kernel", "k": k, "rows": R, "d": d, "us": round(ms * 1e3, 1),
                     "gbs": round(R * d * 4 * (2 * k + 2) / ms / 1e6, 1)})
+    del S_r, S_c
+    # the sequence form: 1024 prompts of 256 positions (8 bytes per element: input read, output written)
+    Bp, n = 1024, 256
+    Z, Y = rnd(Bp, n, d), torch.empty(Bp, n, d, device=dev)
+    an, betan = uni(h, n), rnd(n, d)
+    S_r, S_c = torch.zeros(Bp, d, device=dev), torch.zeros(Bp, d, device=dev)
+    ms = timed(lambda: P.k_mixer_combined_scan(0, Z, S_r, S_c, an, an, betan, lam, lam, w, Y), n=10)
+    out.append({"kernel": "combined_scan_kernel", "prompts": Bp, "n": n, "d": d, "us": round(ms * 1e3, 1),
+                "gbs": round(Bp * n * d * 8 / ms / 1e6, 1)})
+    for k in (4, 8):
+        Pk, al, lk = torch.zeros(k, Bp, d, device=dev), uni(k, n), uni(k) * 0.5
+        ms = timed(lambda: P.k_mixer_kernel_scan(0, Z, Pk, al, betan, lk, Y), n=10)
+        out.append({"kernel": "kernel_scan_kernel", "k": k, "prompts": Bp, "n": n, "d": d, "us": round(ms * 1e3, 1),
+                    "gbs": round(Bp * n * d * 8 / ms / 1e6, 1)})
     for o in out:
         o["frac_of_hbm_peak"] = round(o["gbs"] / peaks["hbm_gbs"], 3)
     print(json.dumps({"variants": out, "peak": f"{peak_src}: {peaks['hbm_gbs']} GB/s", "inputs": "larger than L2"}), flush=True)
