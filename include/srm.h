@@ -306,7 +306,7 @@ int srm_k_mixer_kernel_step(int64_t R, int32_t d, int32_t k, int32_t t, int32_t 
  * d_P float[k, Bp, d]) enter as the sum terms for position t0 (zeros for a fresh prompt) and leave as those for
  * position t0 + n. Equal to the product with the explicit n x n matrices [Eq. 1, Eq. 3, Eq. 11] up to rounding
  * order. Parameters as in the step calls; t0 + n > n_ctx is SRM_ERR_CTX_OVERFLOW; the kernel-size-k call needs
- * 2 k d * 4 bytes of shared memory within 200 KB (SRM_ERR_UNSUPPORTED). */
+ * (2 k + 8) d * 4 bytes of shared memory within 200 KB (SRM_ERR_UNSUPPORTED). */
 int srm_k_mixer_combined_scan(int64_t Bp, int32_t n, int32_t t0, int32_t d, int32_t n_heads, int32_t n_ctx, const float* d_Z,
                               float* d_S_row, float* d_S_col, const float* d_alpha_row, const float* d_alpha_col,
                               const float* d_beta, const float* d_lam_row, const float* d_lam_col, const float* d_w,

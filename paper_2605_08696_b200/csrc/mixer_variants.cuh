@@ -180,44 +180,59 @@ struct KernelScanParams {
   const float *alpha, *beta, *lam;
   float* Y;              // [Bp, n, d]
 };
-inline size_t kernel_scan_smem(int d, int k) { return 2 * (size_t)k * d * 4 + kKernelMixMaxK * 4; }
+constexpr int kScanRing = 4;               // positions of input and beta rows in flight per CTA
+inline size_t kernel_scan_smem(int d, int k) { return (2 * (size_t)k + 2 * kScanRing) * d * 4 + 2 * kKernelMixMaxK * 4; }
+
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 // One CTA owns a sample: the k sum terms live in shared memory for the whole sequence (each element touched by
 // one thread only), the k vectors z + P_i of the current position in a second slab that the shifted reads of
-// Eq. 11 take after a barrier. The next position's input is loaded before the barrier. 8 d bytes per position.
+// Eq. 11 take after a barrier. The input row and the beta row of the next kScanRing - 1 positions are on their
+// way into a shared-memory ring (16-byte asynchronous copies, each thread waiting for its own), so that neither
+// latency sits in the chain from one position to the next. 8 d bytes per position.
 __global__ void __launch_bounds__(kVariantThreads) kernel_scan_kernel(const KernelScanParams p) {
   pdl_trigger();
-  extern __shared__ __align__(16) float ks[];            // P [k][d] | v [k][d] | lam_i
+  extern __shared__ __align__(16) float ks[];            // P [k][d] | v [k][d] | z ring | beta ring | lam_i | alpha_i[t]
   const int d = p.d, k = p.k;
   float* Ps = ks;
   float* vs = ks + (size_t)k * d;
-  float* l_s = vs + (size_t)k * d;
+  float* zr = vs + (size_t)k * d;
+  float* br = zr + (size_t)kScanRing * d;
+  float* l_s = br + (size_t)kScanRing * d;
+  float* a_s = l_s + kKernelMixMaxK;
   if (threadIdx.x < k) l_s[threadIdx.x] = __ldg(p.lam + threadIdx.x);
   pdl_wait();
   const int64_t plane = p.Bp * (int64_t)d;
-  constexpr int kMaxVec = 4;                              // float4 per thread held ahead: d <= 4096 prefetched
   for (int64_t b = blockIdx.x; b < p.Bp; b += gridDim.x) {
-    __syncthreads();                                      // previous sample's slabs are no longer read
-    for (int e = threadIdx.x * 4; e < d; e += kVariantThreads * 4)
-      for (int i = 0; i < k; ++i) st4(Ps + (size_t)i * d + e, ld4(p.P + (int64_t)i * plane + b * d + e));
+    __syncthreads();                                      // previous sample's slabs and rings are no longer read
     const float* zb = p.Z + b * p.n * (int64_t)d;
     float* yb = p.Y + b * p.n * (int64_t)d;
-    float4 zn[kMaxVec];
-#pragma unroll
-    for (int m = 0; m < kMaxVec; ++m) {
-      const int e = (threadIdx.x + m * kVariantThreads) * 4;
-      if (e < d) zn[m] = ld4(zb + e);
-    }
-    for (int j = 0; j < p.n; ++j) {
-      int m = 0;
-      for (int e = threadIdx.x * 4; e < d; e += kVariantThreads * 4, ++m) {
-        float4 z;
-        if (m < kMaxVec) {
-#pragma unroll
-          for (int mm = 0; mm < kMaxVec; ++mm) if (mm == m) z = zn[mm];
-        } else {
-          z = ld4(zb + (int64_t)j * d + e);
+    const float* bb = p.beta + (int64_t)p.t0 * d;
+    auto issue = [&](int jj) {                            // one group per position, empty past the end
+      if (jj < p.n) {
+        const int slot = jj % kScanRing;
+        for (int e = threadIdx.x * 4; e < d; e += kVariantThreads * 4) {
+          cp_async16(zr + (size_t)slot * d + e, zb + (int64_t)jj * d + e);
+          cp_async16(br + (size_t)slot * d + e, bb + (int64_t)jj * d + e);
         }
+      }
+      cp_async_commit();
+    };
+#pragma unroll
+    for (int jj = 0; jj < kScanRing - 1; ++jj) issue(jj);
+    for (int e = threadIdx.x * 4; e < d; e += kVariantThreads * 4)
+      for (int i = 0; i < k; ++i) st4(Ps + (size_t)i * d + e, ld4(p.P + (int64_t)i * plane + b * d + e));
+    for (int j = 0; j < p.n; ++j) {
+      issue(j + kScanRing - 1);                           // into the slot whose beta row was read one position ago
+      cp_async_wait<kScanRing - 1>();                     // this thread's copies of position j have landed
+      const int slot = j % kScanRing;
+      if (threadIdx.x < k) a_s[threadIdx.x] = __ldg(p.alpha + (int64_t)threadIdx.x * p.n_ctx + p.t0 + j);
+      for (int e = threadIdx.x * 4; e < d; e += kVariantThreads * 4) {
+        const float4 z = ld4(zr + (size_t)slot * d + e);
         for (int i = 0; i < k; ++i) {
           float* Pi = Ps + (size_t)i * d + e;
           const float4 s = ld4(Pi);
@@ -227,24 +242,18 @@ __global__ void __launch_bounds__(kVariantThreads) kernel_scan_kernel(const Kern
           st4(Pi, make_float4(l * v.x, l * v.y, l * v.z, l * v.w));
         }
       }
-      if (j + 1 < p.n) {
-#pragma unroll
-        for (int mm = 0; mm < kMaxVec; ++mm) {
-          const int e = (threadIdx.x + mm * kVariantThreads) * 4;
-          if (e < d) zn[mm] = ld4(zb + (int64_t)(j + 1) * d + e);
-        }
-      }
-      __syncthreads();
-      const float* bt = p.beta + (int64_t)(p.t0 + j) * d;
-      const float* al = p.alpha + p.t0 + j;
+      __syncthreads();                                    // v, alpha and everybody's beta copies of position j are visible
+      const float* bt = br + (size_t)slot * d;
+#pragma unroll 4
       for (int c = threadIdx.x; c < d; c += kVariantThreads) {
-        float acc = __ldg(bt + c);
+        float acc = bt[c];
         const int kk = d - c < k ? d - c : k;
-        for (int i = 0; i < kk; ++i) acc = fmaf(__ldg(al + (int64_t)i * p.n_ctx), vs[(size_t)i * d + c + i], acc);
+        for (int i = 0; i < kk; ++i) acc = fmaf(a_s[i], vs[(size_t)i * d + c + i], acc);
         yb[(int64_t)j * d + c] = acc;
       }
       __syncthreads();
     }
+    cp_async_wait<0>();
     for (int e = threadIdx.x * 4; e < d; e += kVariantThreads * 4)
       for (int i = 0; i < k; ++i) st4(p.P + (int64_t)i * plane + b * d + e, ld4(Ps + (size_t)i * d + e));
   }

@@ -1346,7 +1346,7 @@ int srm_k_mixer_kernel_scan(int64_t Bp, int32_t n, int32_t t0, int32_t d, int32_
   if (d % 4 || k > kKernelMixMaxK || k > d || kernel_scan_smem(d, k) > 200 * 1024) return SRM_ERR_UNSUPPORTED;
   if (Bp == 0) return SRM_OK;
   if (!d_Z || !d_P || !d_alpha || !d_beta || !d_lam || !d_Y) return SRM_ERR_INVALID_ARG;
-  if (!aligned(d_Z, 16) || !aligned(d_P, 16) || !aligned(d_Y, 16)) return SRM_ERR_ALIGNMENT;
+  if (!aligned(d_Z, 16) || !aligned(d_P, 16) || !aligned(d_Y, 16) || !aligned(d_beta, 16)) return SRM_ERR_ALIGNMENT;
   int sms = 0, rc = device_sm_count(&sms);
   if (rc != SRM_OK) return rc;
   static std::once_flag once;
