@@ -126,10 +126,20 @@ struct CombinedScanParams {
   float* Y;                       // [Bp, n, d]
 };
 
-// One thread owns four channels of one sample and walks the positions with both sum terms in registers; the
-// inputs of four positions are in flight at a time (they do not depend on the recurrence). 8 d bytes per position.
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+constexpr int kCombinedRing = 8;           // positions of input in flight per thread
+// One thread owns four channels of one sample and walks the positions with both sum terms in registers; its
+// inputs of the next seven positions are on their way into a private ring in shared memory (16-byte asynchronous
+// copies; they do not depend on the recurrence). 8 d bytes per position.
 __global__ void __launch_bounds__(kVariantThreads) combined_scan_kernel(const CombinedScanParams p) {
   pdl_trigger();
+  __shared__ __align__(16) float rings[kVariantThreads * kCombinedRing * 4];
+  float* ring = rings + threadIdx.x * 4;          // this thread's slots, kVariantThreads * 4 floats apart (no bank conflicts)
   pdl_wait();
   const int q = p.d >> 2, dh = p.d / p.h;
   const int64_t n4 = p.Bp * q;
@@ -145,28 +155,28 @@ __global__ void __launch_bounds__(kVariantThreads) combined_scan_kernel(const Co
     const float* zp = p.Z + b * p.n * (int64_t)p.d + c;
     float* yp = p.Y + b * p.n * (int64_t)p.d + c;
     float4 sr = ld4(p.S_row + b * p.d + c), sc = ld4(p.S_col + b * p.d + c);
-    for (int j0 = 0; j0 < p.n; j0 += 4) {
-      float4 z[4];
+    auto issue = [&](int jj) {                 // one group per position, empty past the end
+      if (jj < p.n) cp_async16(ring + (jj % kCombinedRing) * (kVariantThreads * 4), zp + (int64_t)jj * p.d);
+      cp_async_commit();
+    };
 #pragma unroll
-      for (int u = 0; u < 4; ++u)
-        if (j0 + u < p.n) z[u] = ld4(zp + (int64_t)(j0 + u) * p.d);
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int j = j0 + u;
-        if (j < p.n) {
-          const float ar = __ldg(ar_g + j), wc = wc0 * __ldg(ac_g + j);
-          const float4 b4 = ldg4(bt + (int64_t)j * p.d);
-          const float4 uu = make_float4(ar * z[u].x, ar * z[u].y, ar * z[u].z, ar * z[u].w);
-          const float4 v = make_float4(z[u].x + sc.x, z[u].y + sc.y, z[u].z + sc.z, z[u].w + sc.w);
-          float4 y;
-          y.x = fmaf(wr, uu.x + sr.x, fmaf(wc, v.x, b4.x)); y.y = fmaf(wr, uu.y + sr.y, fmaf(wc, v.y, b4.y));
-          y.z = fmaf(wr, uu.z + sr.z, fmaf(wc, v.z, b4.z)); y.w = fmaf(wr, uu.w + sr.w, fmaf(wc, v.w, b4.w));
-          st4(yp + (int64_t)j * p.d, y);
-          sr = make_float4(lr * (sr.x + uu.x), lr * (sr.y + uu.y), lr * (sr.z + uu.z), lr * (sr.w + uu.w));
-          sc = make_float4(lc * v.x, lc * v.y, lc * v.z, lc * v.w);
-        }
-      }
+    for (int jj = 0; jj < kCombinedRing - 1; ++jj) issue(jj);
+    for (int j = 0; j < p.n; ++j) {
+      issue(j + kCombinedRing - 1);            // into the slot read one position ago
+      cp_async_wait<kCombinedRing - 1>();
+      const float4 z = ld4(ring + (j % kCombinedRing) * (kVariantThreads * 4));
+      const float ar = __ldg(ar_g + j), wc = wc0 * __ldg(ac_g + j);
+      const float4 b4 = ldg4(bt + (int64_t)j * p.d);
+      const float4 uu = make_float4(ar * z.x, ar * z.y, ar * z.z, ar * z.w);
+      const float4 v = make_float4(z.x + sc.x, z.y + sc.y, z.z + sc.z, z.w + sc.w);
+      float4 y;
+      y.x = fmaf(wr, uu.x + sr.x, fmaf(wc, v.x, b4.x)); y.y = fmaf(wr, uu.y + sr.y, fmaf(wc, v.y, b4.y));
+      y.z = fmaf(wr, uu.z + sr.z, fmaf(wc, v.z, b4.z)); y.w = fmaf(wr, uu.w + sr.w, fmaf(wc, v.w, b4.w));
+      st4(yp + (int64_t)j * p.d, y);
+      sr = make_float4(lr * (sr.x + uu.x), lr * (sr.y + uu.y), lr * (sr.z + uu.z), lr * (sr.w + uu.w));
+      sc = make_float4(lc * v.x, lc * v.y, lc * v.z, lc * v.w);
     }
+    cp_async_wait<0>();
     st4(p.S_row + b * p.d + c, sr);
     st4(p.S_col + b * p.d + c, sc);
   }
@@ -182,12 +192,6 @@ struct KernelScanParams {
 };
 constexpr int kScanRing = 4;               // positions of input and beta rows in flight per CTA
 inline size_t kernel_scan_smem(int d, int k) { return (2 * (size_t)k + 2 * kScanRing) * d * 4 + 2 * kKernelMixMaxK * 4; }
-
-__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 // One CTA owns a sample: the k sum terms live in shared memory for the whole sequence (each element touched by
 // one thread only), the k vectors z + P_i of the current position in a second slab that the shifted reads of
