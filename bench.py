@@ -384,7 +384,8 @@ def run_ours(args):
     if shape.head_proj:
         kernels["gemm_proj"]["tflops"] = round(args.steps * L * B * 4 * d * d / (prof["gemm_proj"][1] / 1e3) / 1e12, 1)
     kernels["mixer"]["gbs"] = round(mixer_bytes / (prof["mixer"][1] / 1e3) / 1e9, 1)
-    kernels["select"]["gbs"] = round(args.steps * B * V * 4 / (prof["select"][1] / 1e3) / 1e9, 1)
+    if samp.mode != "greedy":            # greedy selection is fused into the LM head: no logits in HBM, nothing to rate
+        kernels["select"]["gbs"] = round(args.steps * B * V * 4 / (prof["select"][1] / 1e3) / 1e9, 1)
 
     # ---- end to end through the host-buffer call: H2D tokens in, D2H tokens out, every step ----
     if lengths is not None and shape.n_ctx - st.pos < args.steps + 2:
