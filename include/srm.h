@@ -6,9 +6,9 @@
  *     token-mixer cache update [Method/Architecture, Eq. 2 (row-repeat heads) and Eq. 3
  *     (column-repeat heads), "mixed" heads], then the channel-mixing feed-forward, then
  *     the LM head and token selection [Recurrent Throughput and Concurrency];
- *   - the sequence-parallel form over a prompt, which yields the same cache
- *     [Method/Architecture, Eq. 1 and Eq. 3; "either recurrent or sequence parallel
- *     operations without any change to the underlying cache structure"].
+ *   - the sequence-parallel form over a prompt, which yields the same cache: the two forms
+ *     share parameters and cache layout, so a model can switch between them at any position
+ *     [Method/Architecture, Eq. 1 and Eq. 3].
  *
  * Conventions
  *   - Every pointer named d_* is a DEVICE pointer, 16-byte aligned unless stated; h_* is a
@@ -19,8 +19,8 @@
  *   - `stream` is a cudaStream_t passed as void*. All device work is enqueued on it and the
  *     calls return without synchronising, except where stated.
  *   - All functions return 0 (SRM_OK) or a negative srm_error. No exceptions, no global
- *     mutable state besides the last CUDA error code. Handles are not thread-safe; distinct
- *     handles may be used from distinct threads.
+ *     mutable state besides the last CUDA error code and the launch counter (atomic). Handles
+ *     are not thread-safe; distinct handles may be used from distinct threads.
  *   - Matrices are row-major [out, in]. Positions are absolute, 0-based; all samples of a
  *     state share one position counter.
  *   - The CUDA device current at srm_create is the one the handles belong to.
@@ -76,7 +76,7 @@ enum {
 typedef struct {
   int32_t n_layers;      /* L >= 1                                                        */
   int32_t d_model;       /* d, multiple of 64, <= 2048                                    */
-  int32_t n_heads;       /* h, even, d % (4h) == 0                                        */
+  int32_t n_heads;       /* h, even, 2 <= h <= 8, d % (4h) == 0                           */
   int32_t ffn_mult;      /* F = ffn_mult * d                                              */
   int32_t vocab;         /* V, multiple of 8                                              */
   int32_t n_ctx;         /* positions for which alpha/beta exist                          */
@@ -137,7 +137,8 @@ size_t srm_weights_bytes(const srm_config* cfg);
 int srm_weight_slot(const srm_config* cfg, int32_t layer, int32_t tensor,
                     size_t* offset, size_t* nbytes, int32_t* elem_bytes);
 /* Bytes of the state buffer for B samples: a 256-byte header (status word, counters), the
- * last selected token int32[B], then the cache [L, B, d] in state_dtype. */
+ * last selected token int32[B], the per-sample position int32[B] (used after srm_prefill_ragged),
+ * each rounded up to 256 bytes, then the cache [L, B, d] in state_dtype. */
 size_t srm_state_bytes(const srm_config* cfg, int64_t B);
 /* Workspace bytes so that decode processes `B_chunk` samples per pass and prefill handles
  * prompts of up to `n_prefill_max` tokens in one pass of at least one sample. Calls accept any
@@ -198,7 +199,8 @@ int srm_prefill(srm_model* m, srm_state* s, const int32_t* d_tokens, int32_t n,
  * srm_generate and the other step calls read alpha_t, beta_t at each sample's own t and advance it, so
  * sample b behaves exactly as if it had been prefilled and decoded alone. srm_state_pos then reports the
  * position of the longest sample (the one that reaches n_ctx first) and srm_state_set_pos is refused.
- * Lengths outside [1, n_max] are clamped and reported through srm_status (SRM_STATUS_TOKEN_RANGE). */
+ * Lengths outside [1, n_max] are clamped to that range (the prefill and the positions kept for the decode
+ * steps use the clamped value) and reported through srm_status (SRM_STATUS_TOKEN_RANGE). */
 int srm_prefill_ragged(srm_model* m, srm_state* s, const int32_t* d_tokens, int32_t n_max,
                        const int32_t* d_lengths, const srm_sampling* sampling, int32_t* d_first_tok,
                        float* d_logits_last, void* d_ws, size_t ws_bytes, void* stream);

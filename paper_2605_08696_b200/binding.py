@@ -21,6 +21,9 @@ FLAG_HEAD_PROJ = 2
 FLAG_NO_GRAPH = 4
 FLAG_GRAPH = 8
 FLAG_NO_SPLITK = 16
+# enum srm_error
+ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_BUFFER_TOO_SMALL, ERR_CTX_OVERFLOW, ERR_CUDA, \
+    ERR_DEVICE_STATUS, ERR_STATIC_SCRATCH = -1, -2, -3, -4, -5, -6, -7, -8
 
 # enum srm_tensor
 T_E, T_LN1_G, T_LN1_B, T_ALPHA, T_BETA, T_LAMBDA, T_LN2_G, T_LN2_B, T_W1, T_B1, T_W2, T_B2, \

@@ -404,6 +404,16 @@ broadcast_rows_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, in
   dst[i] = __ldg(src + (row / replicas) * vec_per_row + v);
 }
 
+// Per-sample positions after a prefill of prompts of different lengths: the lengths as the prefill used them
+// (clamped to [1, n_max]), so that the decode steps continue from the same positions.
+__global__ void __launch_bounds__(256)
+clamp_lengths_kernel(const int32_t* __restrict__ len, int32_t* __restrict__ pos, int64_t B, int lo, int hi) {
+  pdl_trigger();
+  pdl_wait();
+  const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  if (i < B) pos[i] = min(max(len[i], lo), hi);
+}
+
 // Step counters in the state header: set before a replayed generation loop, advanced after every step.
 __global__ void set_counters_kernel(int32_t* hdr, int pos, int step, int col) {
   pdl_trigger();

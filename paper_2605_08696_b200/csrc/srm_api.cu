@@ -6,6 +6,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <atomic>
 #include <cmath>
 #include <cstdio>
 #include <cstring>
@@ -146,9 +147,24 @@ int make_tmap(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, in
   return SRM_OK;
 }
 
+// cudaFuncAttributeMaxDynamicSharedMemorySize is a per-device setting: remember which (kernel, device) pairs have
+// it, so that a model on a second device of the process gets it too. Safe from several host threads.
+int ensure_dynamic_smem(const void* func, int bytes) {
+  static std::mutex mu;
+  static std::vector<std::pair<const void*, int>> done;      // (kernel, device ordinal)
+  int dev = -1;
+  SRM_CUDA(cudaGetDevice(&dev));
+  std::lock_guard<std::mutex> lock(mu);
+  for (const auto& e : done)
+    if (e.first == func && e.second == dev) return SRM_OK;
+  SRM_CUDA(cudaFuncSetAttribute(func, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+  done.emplace_back(func, dev);
+  return SRM_OK;
+}
+
 struct TmapCacheEntry { const void* base; int64_t rows, cols; int box_rows, elem_bytes; CUtensorMap map; };
 
-unsigned long long g_kernel_launches = 0;     // kernels launched by this library since load
+std::atomic<unsigned long long> g_kernel_launches{0};     // kernels launched by this library since load (all threads)
 
 struct ProfRecord { cudaEvent_t start, stop; int cls; };
 
@@ -172,8 +188,9 @@ struct srm_model {
   struct StepKey {
     const srm_state* s = nullptr; const void* ws = nullptr; size_t ws_bytes = 0; const int32_t* out = nullptr;
     int64_t out_stride = 0; srm_sampling samp = {};
+    bool ragged = false;                 // per-sample positions: the captured kernels then take the position vector
     bool operator==(const StepKey& o) const {
-      return s == o.s && ws == o.ws && ws_bytes == o.ws_bytes && out == o.out && out_stride == o.out_stride &&
+      return ragged == o.ragged && s == o.s && ws == o.ws && ws_bytes == o.ws_bytes && out == o.out && out_stride == o.out_stride &&
              samp.mode == o.samp.mode && samp.top_k == o.samp.top_k && samp.temperature == o.samp.temperature &&
              samp.top_p == o.samp.top_p &&
              samp.seed == o.samp.seed && samp.sample_idx_base == o.samp.sample_idx_base;
@@ -345,12 +362,8 @@ template <int NV, typename WT, typename ST>
 int launch_mixer_stream(const MixerParams& p, int num_sms, cudaStream_t st) {
   const int warps = mixer_stream_warps(p.d, (int)sizeof(ST));
   const size_t smem = mixer_stream_smem(p.d, (int)sizeof(ST), warps);
-  static bool attr_set = false;               // per instantiation
-  if (!attr_set) {
-    SRM_CUDA(cudaFuncSetAttribute(mixer_stream_kernel<NV, WT, ST>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                  kStreamSmemBudget));
-    attr_set = true;
-  }
+  int rc = ensure_dynamic_smem(reinterpret_cast<const void*>(mixer_stream_kernel<NV, WT, ST>), kStreamSmemBudget);
+  if (rc != SRM_OK) return rc;
   const unsigned grid = (unsigned)(p.R < num_sms ? p.R : num_sms);
   SRM_CUDA(launch_kernel(mixer_stream_kernel<NV, WT, ST>, dim3(grid), dim3(warps * 32), smem, st, p));
   return SRM_OK;
@@ -551,20 +564,15 @@ int launch_select(const srm_model& m, int64_t R, const float* logits, const srm_
     const size_t scratch = ((sizeof(ToppScratch) + 15) & ~size_t(15)) + sizeof(ToppHist);
     if (V <= kToppSmemFloats) {
       const size_t smem = scratch + (size_t)V * 4;
-      static bool attr_set = false;
-      if (!attr_set) {
-        SRM_CUDA(cudaFuncSetAttribute(select_topp_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      (int)(scratch + (size_t)kToppSmemFloats * 4)));
-        attr_set = true;
-      }
+      int rc = ensure_dynamic_smem(reinterpret_cast<const void*>(select_topp_kernel<true>),
+                                   (int)(scratch + (size_t)kToppSmemFloats * 4));
+      if (rc != SRM_OK) return rc;
       SRM_CUDA(launch_kernel(select_topp_kernel<true>, dim3((unsigned)R), dim3(kToppThreads), smem, st, logits, R, V,
                              s.top_p, inv_t, s.seed, sample_base, step, out, status));
     } else {
-      static bool attr_set_g = false;           // the scratch alone exceeds the default dynamic shared-memory limit
-      if (!attr_set_g) {
-        SRM_CUDA(cudaFuncSetAttribute(select_topp_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)scratch));
-        attr_set_g = true;
-      }
+      // the scratch alone exceeds the default dynamic shared-memory limit
+      int rc = ensure_dynamic_smem(reinterpret_cast<const void*>(select_topp_kernel<false>), (int)scratch);
+      if (rc != SRM_OK) return rc;
       SRM_CUDA(launch_kernel(select_topp_kernel<false>, dim3((unsigned)R), dim3(kToppThreads), scratch, st, logits, R, V,
                              s.top_p, inv_t, s.seed, sample_base, step, out, status));
     }
@@ -620,11 +628,8 @@ template <int NV, typename WT, typename ST>
 int launch_prefill_scan(const PrefillParams& p, int num_sms, cudaStream_t st) {
   const int warps = prefill_scan_warps(p.d, p.Bp, num_sms);
   const size_t smem = prefill_scan_smem(p.d, warps);
-  static bool attr_set = false;               // per instantiation
-  if (!attr_set) {
-    SRM_CUDA(cudaFuncSetAttribute(prefill_scan_kernel<NV, WT, ST>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScanSmemBudget));
-    attr_set = true;
-  }
+  int rc = ensure_dynamic_smem(reinterpret_cast<const void*>(prefill_scan_kernel<NV, WT, ST>), kScanSmemBudget);
+  if (rc != SRM_OK) return rc;
   const unsigned grid = (unsigned)(p.Bp < num_sms ? p.Bp : num_sms);
   SRM_CUDA(launch_kernel(prefill_scan_kernel<NV, WT, ST>, dim3(grid), dim3(warps * 32), smem, st, p));
   SRM_CUDA(cudaGetLastError());
@@ -663,7 +668,7 @@ int launch_prefill_mixer(const srm_model& m, int layer, int64_t Bp, int n, const
     return launch_prefill_scan_nv<float, float>(p, m.num_sms, st);
   }
   auto go = [&](auto kernel) -> int {
-    SRM_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    SRM_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));   // smem depends on d: set per launch
     SRM_CUDA(launch_kernel(kernel, dim3((unsigned)Bp), dim3(kPrefillThreads), smem, st, p));
     SRM_CUDA(cudaGetLastError());
     return SRM_OK;
@@ -1051,7 +1056,9 @@ int prefill_impl(srm_model* m, srm_state* s, const int32_t* d_tokens, int64_t P,
   s->pos = n;
   if (d_len != nullptr) {
     // from here on every sample has its own position: its prompt length (srm_prefill_ragged checked replicas == 1)
-    SRM_CUDA(cudaMemcpyAsync(s->pos_dev, d_len, (size_t)s->B * 4, cudaMemcpyDeviceToDevice, st));
+    ++g_kernel_launches;
+    SRM_CUDA(launch_kernel(clamp_lengths_kernel, dim3((unsigned)((s->B + 255) / 256)), dim3(256), 0, st, d_len, s->pos_dev,
+                           s->B, 1, (int)n));
     s->ragged = true;
   }
   return SRM_OK;
@@ -1126,6 +1133,7 @@ int prepare_step_graph(srm_model* m, srm_state* s, const srm_sampling* samp, int
                        void* d_ws, size_t ws_bytes) {
   srm_model::StepKey key;
   key.s = s; key.ws = d_ws; key.ws_bytes = ws_bytes; key.out = d_out; key.out_stride = out_stride; key.samp = *samp;
+  key.ragged = s->ragged;
   if (m->step_exec != nullptr && m->step_key == key) return SRM_OK;
   if (m->step_exec != nullptr) { cudaGraphExecDestroy(m->step_exec); m->step_exec = nullptr; }
   if (m->cap_stream == nullptr) SRM_CUDA(cudaStreamCreateWithFlags(&m->cap_stream, cudaStreamNonBlocking));
@@ -1299,12 +1307,7 @@ int srm_k_mixer_kernel_step(int64_t R, int32_t d, int32_t k, int32_t t, int32_t 
   if (!aligned(d_z, 16) || !aligned(d_P, 16) || !aligned(d_y, 16)) return SRM_ERR_ALIGNMENT;
   int sms = 0, rc = device_sm_count(&sms);
   if (rc != SRM_OK) return rc;
-  static std::once_flag once;
-  static cudaError_t attr_err = cudaSuccess;
-  std::call_once(once, [] {
-    attr_err = cudaFuncSetAttribute(kernel_mix_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-  });
-  SRM_CUDA(attr_err);
+  if ((rc = ensure_dynamic_smem(reinterpret_cast<const void*>(kernel_mix_step_kernel), 200 * 1024)) != SRM_OK) return rc;
   KernelMixParams p{R, d, k, t, n_ctx, d_z, d_P, d_alpha, d_beta, d_lam, d_y};
   const size_t smem = kernel_mix_smem(d, k);
   // one wave of resident blocks: a second, partly filled wave would run at a fraction of the bandwidth
@@ -1349,12 +1352,7 @@ int srm_k_mixer_kernel_scan(int64_t Bp, int32_t n, int32_t t0, int32_t d, int32_
   if (!aligned(d_Z, 16) || !aligned(d_P, 16) || !aligned(d_Y, 16) || !aligned(d_beta, 16)) return SRM_ERR_ALIGNMENT;
   int sms = 0, rc = device_sm_count(&sms);
   if (rc != SRM_OK) return rc;
-  static std::once_flag once;
-  static cudaError_t attr_err = cudaSuccess;
-  std::call_once(once, [] {
-    attr_err = cudaFuncSetAttribute(kernel_scan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-  });
-  SRM_CUDA(attr_err);
+  if ((rc = ensure_dynamic_smem(reinterpret_cast<const void*>(kernel_scan_kernel), 200 * 1024)) != SRM_OK) return rc;
   KernelScanParams p{Bp, n, t0, d, k, n_ctx, d_Z, d_P, d_alpha, d_beta, d_lam, d_Y};
   const size_t smem = kernel_scan_smem(d, k);
   int per_sm = 0;

@@ -1,7 +1,16 @@
 """Shared test helpers: model construction for both sides, error metric."""
+import functools
+
 import numpy as np
 
 import srm_inputs as I
+
+
+@functools.lru_cache(maxsize=2)
+def weights_for(name: str):
+    """Seeded weights of a benchmark configuration (drawing the larger ones takes most of a minute: shared
+    between the tests of one session; treat as read-only)."""
+    return I.make_weights(I.CONFIGS[name])
 
 
 def oracle_for(shape, W, dtype=np.float64):

@@ -10,7 +10,7 @@ import pytest
 import torch
 
 import srm_inputs as I
-from helpers import oracle_for, rel_err_rows, top2_margin
+from helpers import oracle_for, rel_err_rows, top2_margin, weights_for
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -23,7 +23,7 @@ def _run(name, steps, rows, chunk):
     w = I.WORKLOADS[name]
     shape = I.CONFIGS[w["model"]]
     B, n = w["batch"], w["prompt_len"]
-    W = I.make_weights(shape)
+    W = weights_for(w["model"])
     model = P.SRM(shape, W, device=DEV)
     topk = w["sampling"] == "topk"
     samp = P.Sampling("topk", w["top_k"], w["temperature"], seed=shape.seed) if topk else P.Sampling("greedy")

@@ -194,3 +194,42 @@ def test_resume_of_a_ragged_state_from_a_copied_buffer():
     rest = model.generate(c, k, k + 1, g, ws)
     assert torch.equal(full, torch.cat([first, rest], 1))
     assert torch.equal(a.cache(), c.cache()) and a.status() == 0 and c.status() == 0
+
+
+def test_captured_step_is_not_reused_across_a_change_of_position_mode():
+    """srm_generate keeps the captured step for as long as state, workspace, sampling and output buffer stay
+    the same. Whether the samples share one position or keep their own is part of what was captured (the
+    kernels take the position vector or not), so a state that is reset and prefilled the other way on the SAME
+    buffers must get a new capture: both orders give exactly the tokens and cache of the launch-by-launch loop."""
+    import paper_2605_08696_b200 as P
+    shape = I.CONFIGS["small"]
+    W = I.make_weights(shape)
+    lengths = [24, 9, 17, 24, 3, 12]
+    B, n = len(lengths), max(lengths)
+    toks = torch.from_numpy(_ragged_batch(shape, lengths, seed=23)).to(DEV)
+    lens = torch.tensor(lengths, dtype=torch.int32, device=DEV)
+    g = P.Sampling("greedy")
+    for order in (("plain", "ragged", "plain"), ("ragged", "plain")):
+        res = {}
+        for flags in (P.FLAG_NO_GRAPH, P.FLAG_GRAPH):
+            model = P.SRM(shape, W, device=DEV, flags=flags)
+            st = model.new_state(B)
+            ws = model.new_workspace(B, n, prefill_samples=B)
+            out = torch.full((B, 6), -1, dtype=torch.int32, device=DEV)
+            got = []
+            for mode in order:
+                st.reset()
+                if mode == "plain":
+                    first = model.prefill(st, toks, g, ws)
+                else:
+                    first = model.prefill_ragged(st, toks, lens, g, ws)
+                model.generate(st, 6, 1, g, ws, out=out)
+                got.append((first.clone(), out.clone(), st.cache().clone()))
+                assert st.ragged == (mode == "ragged")
+            assert st.status() == 0
+            res[flags] = got
+        for a_, b_ in zip(res[P.FLAG_NO_GRAPH], res[P.FLAG_GRAPH]):
+            for x_, y_ in zip(a_, b_):
+                assert torch.equal(x_, y_)
+        # the two modes really differ (shorter samples stand at other positions)
+        assert not torch.equal(res[P.FLAG_GRAPH][0][1], res[P.FLAG_GRAPH][1][1])
