@@ -14,6 +14,7 @@ from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import statistics
 import subprocess
@@ -28,9 +29,34 @@ if ROOT not in sys.path:
 METRIC, UNIT = "generated_tokens_per_s", "tokens/s"
 L2_BYTES = 126e6
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# DRAM traffic of the dominant kernel per launch (bytes), from the ncu capture summarised in
-# profiles/; None until a capture exists for the benchmarked shape.
-GEMM_DRAM_TRAFFIC_PER_STEP = {"mid": 1.303e9}      # cold-cache (ncu flushes between passes), mid model at batch 4096
+MIN_TIMED_S = 1.0          # a K-step block is repeated until this much device time has been timed
+
+
+def gemm_sources_sha():
+    """Short hash of the tensor-core GEMM sources: a DRAM-traffic figure taken under ncu holds only for the
+    kernel it was taken on."""
+    import hashlib
+    h = hashlib.sha256()
+    for f in ("gemm_tc.cuh", "gemm_tc_splitk.cuh"):
+        with open(os.path.join(ROOT, "paper_2605_08696_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:12]
+
+
+def dram_traffic_per_step(workload: str, batch: int):
+    """DRAM bytes (read + write) of the GEMM launches of one decode step, from the ncu summaries under profiles/:
+    a line `dram_traffic_per_step: workload=<w> batch=<B> bytes=<x> gemm_sources=<sha>`. None when no capture
+    exists for this workload and batch, or when the GEMM sources have changed since it was taken."""
+    import glob
+    import re
+    pat = re.compile(r"dram_traffic_per_step:\s*workload=(\w+)\s+batch=(\d+)\s+bytes=([0-9.eE+]+)\s+gemm_sources=(\w+)")
+    sha = gemm_sources_sha()
+    for path in sorted(glob.glob(os.path.join(ROOT, "profiles", "*.md"))):
+        with open(path) as f:
+            for m in pat.finditer(f.read()):
+                if m.group(1) == workload and int(m.group(2)) == batch and m.group(4) == sha:
+                    return float(m.group(3))
+    return None
 
 
 def measured_peaks():
@@ -43,61 +69,125 @@ def measured_peaks():
 
 
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+    """Samples SM clock, power and clock-event (throttle) reasons of one GPU every ~10 ms while the timed
+    regions run: NVML queries from a thread of this process (read-only), or an `nvidia-smi` loop when NVML
+    cannot be loaded. Only samples that fall inside a marked region are summarised."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
+    PERIOD_S = 0.010
 
-    def __init__(self, index: int):
-        self.index, self.rows, self.proc = index, [], None
-        self.t0 = self.t1 = None
+    def __init__(self, index: int, uuid: str | None = None):
+        self.index, self.uuid = index, uuid
+        self.rows = []            # (monotonic time, sm MHz, max MHz, watts, set of reasons)
+        self.regions = []         # [t0, t1] of the marked regions
+        self.proc = self.thread = self.nvml = None
+        self.stop = threading.Event()
+        self.source = None
 
+    # -- regions --
     def mark_start(self):
-        self.t0 = time.monotonic()
+        self.regions.append([time.monotonic(), None])
 
     def mark_stop(self):
-        self.t1 = time.monotonic()
+        self.regions[-1][1] = time.monotonic()
+
+    # -- NVML --
+    def _nvml_open(self):
+        import pynvml
+        pynvml.nvmlInit()
+        h = None
+        if self.uuid:
+            for u in (self.uuid, "GPU-" + self.uuid):
+                try:
+                    h = pynvml.nvmlDeviceGetHandleByUUID(u if isinstance(u, bytes) else u.encode())
+                    break
+                except Exception:
+                    h = None
+        if h is None:
+            h = pynvml.nvmlDeviceGetHandleByIndex(self.index)
+        self.nvml, self.h = pynvml, h
+        self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
+        n = pynvml
+        self.bits = [(getattr(n, "nvmlClocksEventReasonSwPowerCap", 0x4), "sw_power_cap"),
+                     (getattr(n, "nvmlClocksThrottleReasonHwSlowdown", 0x8), "hw_slowdown"),
+                     (getattr(n, "nvmlClocksEventReasonSwThermalSlowdown", 0x20), "sw_thermal_slowdown"),
+                     (getattr(n, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40), "hw_thermal_slowdown")]
+
+    def _nvml_loop(self):
+        n, h = self.nvml, self.h
+        get_reasons = getattr(n, "nvmlDeviceGetCurrentClocksEventReasons", None) or n.nvmlDeviceGetCurrentClocksThrottleReasons
+        while not self.stop.is_set():
+            try:
+                mhz = float(n.nvmlDeviceGetClockInfo(h, n.NVML_CLOCK_SM))
+                mask = int(get_reasons(h))
+                watts = n.nvmlDeviceGetPowerUsage(h) / 1000.0
+                self.rows.append((time.monotonic(), mhz, self.max_mhz, watts,
+                                  {name for bit, name in self.bits if mask & bit}))
+            except Exception:
+                pass
+            time.sleep(self.PERIOD_S)
+
+    # -- nvidia-smi fallback --
+    def _smi_loop(self):
+        for line in self.proc.stdout:
+            r = [c.strip() for c in line.split(",")]
+            if len(r) < 8:
+                continue
+            try:
+                mhz, mx, watts = float(r[0]), float(r[1]), float(r[2])
+            except ValueError:
+                continue
+            reasons = {name for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[4:8])
+                       if v.lower().startswith("active")}
+            self.rows.append((time.monotonic(), mhz, mx, watts, reasons))
 
     def __enter__(self):
         try:
-            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
-                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-            self.thread = threading.Thread(target=self._read, daemon=True)
+            self._nvml_open()
+            self.thread = threading.Thread(target=self._nvml_loop, daemon=True)
+            self.source = "nvml, 10 ms"
+        except Exception:
+            self.nvml = None
+            try:
+                self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                              "--format=csv,noheader,nounits", "-lms", "20"],
+                                             stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                self.thread = threading.Thread(target=self._smi_loop, daemon=True)
+                self.source = "nvidia-smi, 20 ms"
+            except OSError:
+                self.proc = self.thread = None
+        if self.thread is not None:
             self.thread.start()
-        except OSError:
-            self.proc = None
         return self
 
-    def _read(self):
-        for line in self.proc.stdout:
-            self.rows.append((time.monotonic(), [c.strip() for c in line.split(",")]))
-
     def __exit__(self, *a):
+        self.stop.set()
         if self.proc is not None:
             self.proc.terminate()
             try:
                 self.proc.wait(timeout=2)
             except subprocess.TimeoutExpired:
                 self.proc.kill()
-
-    def summary(self):
-        sm, mx, reasons = [], [], set()
-        # a sample printed at time ts describes the ~100 ms before it
-        inside = [r for ts, r in self.rows if self.t0 is None or (self.t0 + 0.05 <= ts <= (self.t1 or ts) + 0.1)]
-        for r in inside:
-            if len(r) < 8:
-                continue
+        if self.thread is not None:
+            self.thread.join(timeout=2)
+        if self.nvml is not None:
             try:
-                sm.append(float(r[0])); mx.append(float(r[1]))
-            except ValueError:
-                continue
-            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[4:8]):
-                if v.lower().startswith("active"):
-                    reasons.add(name)
-        if not sm:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
-        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm)}
+                self.nvml.nvmlShutdown()
+            except Exception:
+                pass
+
+    def summary(self, regions=None):
+        """Median SM clock, maximum clock, reasons seen and sample count over the marked regions (or the given
+        [t0, t1] pairs)."""
+        regions = self.regions if regions is None else regions
+        inside = [r for r in self.rows if any(t0 <= r[0] <= (t1 if t1 is not None else r[0]) for t0, t1 in regions)]
+        if not inside:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "source": self.source}
+        reasons = set().union(*[r[4] for r in inside])
+        return {"sm_mhz": statistics.median(r[1] for r in inside), "sm_max_mhz": max(r[2] for r in inside),
+                "sm_mhz_min": min(r[1] for r in inside), "power_w": round(statistics.median(r[3] for r in inside), 1),
+                "reasons": sorted(reasons), "samples": len(inside), "source": self.source}
 
 
 def step_flops(shape):
@@ -240,8 +330,10 @@ def run_ours(args):
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world != args.gpus:
+        raise SystemExit(f"--gpus {args.gpus} but the launcher started {world} rank(s)")
     if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+        raise SystemExit(f"rank {rank}: bench.py needs a CUDA device (there is no CPU fallback)")
     torch.cuda.set_device(local)
     dev = f"cuda:{local}"
     if world > 1:
@@ -339,53 +431,76 @@ def run_ours(args):
             step_no[0] += c
             k -= c
 
-    with ClockSampler(local) as clk:         # nvidia-smi starts up during the warm-up steps
+    def timed_blocks(run_block, clk):
+        """Times run_block (EXACTLY K steps) between a barrier + synchronize on both sides, MAX over ranks, and
+        repeats the block until MIN_TIMED_S of device time has been timed: a single 20-step block lasts tens of
+        milliseconds, which measures the clock transient after the prefill, not the kernels. Every rank
+        computes the same number of blocks from the first block's MAX-over-ranks time."""
+        times, n_target = [], None
+        while n_target is None or len(times) < n_target:
+            sync_all()
+            clk.mark_start()
+            e0.record()
+            run_block()
+            e1.record()
+            torch.cuda.synchronize()
+            clk.mark_stop()
+            times.append(max_over_ranks(e0.elapsed_time(e1), world, dev))
+            if n_target is None:
+                n_target = max(1, min(args.max_blocks, math.ceil(args.min_time * 1e3 / max(times[0], 1e-3))))
+        return times
+
+    try:
+        uuid = str(torch.cuda.get_device_properties(local).uuid)
+    except Exception:
+        uuid = None
+    with ClockSampler(local, uuid) as clk:
         run_steps(max(args.warmup, 3))
-        # ---- timed region: exactly K steps ----
+        # ---- timed region: blocks of exactly K steps ----
         sync_all()
         launches0 = model.kernel_launches()
-        clk.mark_start()
-        e0.record()
-        run_steps(args.steps)
-        e1.record()
+        run_steps(args.steps)                # one more untimed block, to count the launches of K steps
         torch.cuda.synchronize()
-        clk.mark_stop()
-        time.sleep(0.15)                     # let the sample that covers the end of the region arrive
-    t_ms = e0.elapsed_time(e1)
-    launches = model.kernel_launches() - launches0
-    if world > 1:
-        dist.barrier()
-    t_ms_max = max_over_ranks(t_ms, world, dev)
+        launches = model.kernel_launches() - launches0
+        block_ms = timed_blocks(lambda: run_steps(args.steps), clk)
+        timed_regions = list(clk.regions)
+    t_ms_max = statistics.median(block_ms)
     value = whole_job_value(world, B, args.steps, t_ms_max)
 
     # ---- per-kernel durations, CUDA events on the launching stream, same workload ----
     if lengths is not None and shape.n_ctx - st.pos < args.steps:
         rewind()
-    model.profile_reset()
+    prof_steps = args.steps * max(1, min(len(block_ms), 256 // max(args.steps, 1)))   # long enough to sit at the
+    model.profile_reset()                                                              # same clocks, bounded events
     model.profile(True)
-    run_steps(args.steps)
+    run_steps(prof_steps)
     torch.cuda.synchronize()
     model.profile(False)
     prof = model.profile_read()
     d, L, V, F = shape.d_model, shape.n_layers, shape.vocab, shape.d_ffn
     gemm_ms = sum(prof[k][1] for k in ("gemm_up", "gemm_down", "gemm_lm", "gemm_proj"))
     gemm_launches = sum(prof[k][0] for k in ("gemm_up", "gemm_down", "gemm_lm", "gemm_proj"))
-    gemm_flops = args.steps * B * step_flops(shape)
+    gemm_flops = prof_steps * B * step_flops(shape)
     achieved_tf = gemm_flops / (gemm_ms / 1e3) / 1e12 if gemm_ms > 0 else 0.0
     prof_total = sum(v[1] for v in prof.values())
     peak_tf = peaks["bf16_tflops_sustained"]
     t_roof, bound, t_tc, t_hbm = step_roofline_s(shape, B, sbytes, peaks)
-    mixer_bytes = args.steps * L * B * d * (4 + 4 + 2 * sbytes + 2)       # x r/w, cache r/w, bf16 activation
+    mixer_bytes = prof_steps * L * B * d * (4 + 4 + 2 * sbytes + 2)       # x r/w, cache r/w, bf16 activation
+    mixer_cache_bytes = prof_steps * L * B * d * 2 * sbytes                # the part that must cross HBM: cache read + write
     kernels = {k: {"launches": v[0], "ms_total": round(v[1], 3), "share": round(v[1] / prof_total, 4) if prof_total else 0}
                for k, v in prof.items() if v[0]}
-    kernels["gemm_up"]["tflops"] = round(args.steps * L * B * 2 * d * F / (prof["gemm_up"][1] / 1e3) / 1e12, 1)
-    kernels["gemm_down"]["tflops"] = round(args.steps * L * B * 2 * d * F / (prof["gemm_down"][1] / 1e3) / 1e12, 1)
-    kernels["gemm_lm"]["tflops"] = round(args.steps * B * 2 * d * V / (prof["gemm_lm"][1] / 1e3) / 1e12, 1)
+    kernels["gemm_up"]["tflops"] = round(prof_steps * L * B * 2 * d * F / (prof["gemm_up"][1] / 1e3) / 1e12, 1)
+    kernels["gemm_down"]["tflops"] = round(prof_steps * L * B * 2 * d * F / (prof["gemm_down"][1] / 1e3) / 1e12, 1)
+    kernels["gemm_lm"]["tflops"] = round(prof_steps * B * 2 * d * V / (prof["gemm_lm"][1] / 1e3) / 1e12, 1)
     if shape.head_proj:
-        kernels["gemm_proj"]["tflops"] = round(args.steps * L * B * 4 * d * d / (prof["gemm_proj"][1] / 1e3) / 1e12, 1)
-    kernels["mixer"]["gbs"] = round(mixer_bytes / (prof["mixer"][1] / 1e3) / 1e9, 1)
+        kernels["gemm_proj"]["tflops"] = round(prof_steps * L * B * 4 * d * d / (prof["gemm_proj"][1] / 1e3) / 1e12, 1)
+    kernels["mixer"]["gbs"] = round(mixer_bytes / (prof["mixer"][1] / 1e3) / 1e9, 1)          # all bytes it moves (x and a: L2)
+    kernels["mixer"]["cache_gbs"] = round(mixer_cache_bytes / (prof["mixer"][1] / 1e3) / 1e9, 1)   # algorithmic: the cache
+    kernels["mixer"]["cache_frac_of_hbm_peak"] = round(kernels["mixer"]["cache_gbs"] / peaks["hbm_gbs"], 3)
+    for k_ in kernels.values():
+        k_["us_per_launch"] = round(k_["ms_total"] * 1e3 / k_["launches"], 2)
     if samp.mode != "greedy":            # greedy selection is fused into the LM head: no logits in HBM, nothing to rate
-        kernels["select"]["gbs"] = round(args.steps * B * V * 4 / (prof["select"][1] / 1e3) / 1e9, 1)
+        kernels["select"]["gbs"] = round(prof_steps * B * V * 4 / (prof["select"][1] / 1e3) / 1e9, 1)
 
     # ---- end to end through the host-buffer call: H2D tokens in, D2H tokens out, every step ----
     if lengths is not None and shape.n_ctx - st.pos < args.steps + 2:
@@ -397,19 +512,19 @@ def run_ours(args):
             rewind()
         model.decode_step_host(st, h_in, samp, step_no[0], h_out, ws); step_no[0] += 1
         torch.cuda.synchronize(); h_in.copy_(h_out)
-    sync_all()
-    e0.record()
-    for _ in range(args.steps):
-        if st.pos >= shape.n_ctx:
-            rewind()
-        model.decode_step_host(st, h_in, samp, step_no[0], h_out, ws); step_no[0] += 1
-        torch.cuda.current_stream().synchronize()      # the next step's input is this step's output
-        h_in.copy_(h_out)
-    e1.record()
-    torch.cuda.synchronize()
-    if world > 1:
-        dist.barrier()
-    e2e_value = whole_job_value(world, B, args.steps, max_over_ranks(e0.elapsed_time(e1), world, dev))
+
+    def e2e_block():
+        for _ in range(args.steps):
+            if st.pos >= shape.n_ctx:
+                rewind()
+            model.decode_step_host(st, h_in, samp, step_no[0], h_out, ws); step_no[0] += 1
+            torch.cuda.current_stream().synchronize()      # the next step's input is this step's output
+            h_in.copy_(h_out)
+
+    with ClockSampler(local, uuid) as clk2:
+        e2e_ms = timed_blocks(e2e_block, clk2)
+        e2e_clocks = clk2.summary()
+    e2e_value = whole_job_value(world, B, args.steps, statistics.median(e2e_ms))
     status = st.status()
 
     if rank == 0:
@@ -417,11 +532,18 @@ def run_ours(args):
         per_sample = L * d * sbytes + 4 * w["gen"] + 4
         fixed = model.blob.numel() + ws.numel()
         max_conc = int((total_b * 0.97 - fixed) // per_sample)
-        clocks = clk.summary()
+        clocks = clk.summary(timed_regions)
         cpu = cpu_baseline(shape, W, args.workload, w) if world == 1 and not args.no_cpu_baseline else None
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": t_ms_max / args.steps, "higher_is_better": True,
+            "blocks": {"n": len(block_ms), "steps_per_block": args.steps, "timed_s": round(sum(block_ms) / 1e3, 3),
+                       "ms_per_step_median": round(t_ms_max / args.steps, 5),
+                       "ms_per_step_min": round(min(block_ms) / args.steps, 5),
+                       "ms_per_step_max": round(max(block_ms) / args.steps, 5),
+                       "ms_per_step_first": round(block_ms[0] / args.steps, 5),
+                       "note": "value and ms_per_step are the median block; every block is K steps between a "
+                               "barrier + synchronize on both sides, MAX over ranks"},
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if shape.dtype == "bf16" else "f32",
             "data": "synthetic",
             "config": _config_dict(args, shape, w, B, extra={
@@ -430,13 +552,17 @@ def run_ours(args):
                       f"{model.blob.numel() / 1e6:.0f} MB + logits {chunk * V * 4 / 1e6:.0f} MB) vs 126 MB L2; no flush"}),
             "gpu_launches": int(launches),
             "clocks": clocks,
-            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": B * 4, "d2h_bytes_per_step": B * 4},
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": B * 4, "d2h_bytes_per_step": B * 4,
+                    "ms_per_step": round(statistics.median(e2e_ms) / args.steps, 5), "blocks": len(e2e_ms),
+                    "clocks": e2e_clocks},
             "roofline": {"bound": "tensor", "kernel": "gemm_tc_kernel (feed-forward up/down + LM head)",
                          "achieved": round(achieved_tf, 1), "peak": peak_tf, "unit": "TFLOP/s",
                          "frac": round(achieved_tf / peak_tf, 4), "peak_source": f"bf16_tflops_sustained, {peak_src}",
                          "frac_of_burst_peak": round(achieved_tf / peaks["bf16_tflops"], 4),
-                         "launches": int(gemm_launches),
-                         "traffic": GEMM_DRAM_TRAFFIC_PER_STEP.get(args.workload) if B == 4096 else None,
+                         "launches": int(gemm_launches), "steps_profiled": prof_steps,
+                         "traffic": dram_traffic_per_step(args.workload, B) if not shape.head_proj else None,
+                         "traffic_note": "DRAM bytes of the GEMM launches of one step (ncu, cold cache; see profiles/); "
+                                         "null when no capture exists for this workload, batch and GEMM source",
                          "flops_per_step": B * step_flops(shape)},
             "step_roofline": {"bound": bound, "t_roof_ms": round(t_roof * 1e3, 4), "t_tensor_ms": round(t_tc * 1e3, 4),
                               "t_hbm_ms": round(t_hbm * 1e3, 4), "frac": round(t_roof * 1e3 / (t_ms_max / args.steps), 4),
@@ -482,27 +608,45 @@ def run_sweep(args):
     if args.sweep_max:
         batches = [b for b in batches if b <= args.sweep_max]
     curve = []
-    for B in batches:
-        st = model.new_state(B)
-        prompts = torch.from_numpy(I.uniform_prompts(min(B, 65536), w["prompt_len"], shape.vocab, shape.seed)).to(dev)
-        if B > prompts.shape[0]:
-            prompts = prompts.repeat((B + prompts.shape[0] - 1) // prompts.shape[0], 1)[:B].contiguous()
-        model.prefill(st, prompts, g, ws)
-        steps = 8 if B >= 262144 else 24
-        store = torch.empty(B, steps, dtype=torch.int32, device=dev)
-        model.generate(st, 4, 1, g, ws, out=store)
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        e0.record()
-        model.generate(st, steps, 5, g, ws, out=store)
-        e1.record()
-        torch.cuda.synchronize()
-        ms = e0.elapsed_time(e1) / steps
-        curve.append({"batch": B, "ms_per_step": round(ms, 4), "tokens_per_s": round(B / (ms / 1e3), 1),
-                      "state_bytes_per_sample": L * d * sbytes, "status": st.status()})
-        print(json.dumps(curve[-1]), file=sys.stderr, flush=True)
-        del st, prompts, store
-        torch.cuda.empty_cache()
+    try:
+        uuid = str(torch.cuda.get_device_properties(0).uuid)
+    except Exception:
+        uuid = None
+    with ClockSampler(0, uuid) as clk:
+        for B in batches:
+            st = model.new_state(B)
+            prompts = torch.from_numpy(I.uniform_prompts(min(B, 65536), w["prompt_len"], shape.vocab, shape.seed)).to(dev)
+            if B > prompts.shape[0]:
+                prompts = prompts.repeat((B + prompts.shape[0] - 1) // prompts.shape[0], 1)[:B].contiguous()
+            model.prefill(st, prompts, g, ws)
+            steps = 8 if B >= 262144 else 24
+            store = torch.empty(B, steps, dtype=torch.int32, device=dev)
+            model.generate(st, 4, 1, g, ws, out=store)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            # blocks of `steps` steps until MIN_TIMED_S has been timed (the context has room for 896 steps)
+            blocks, n_target, region0 = [], None, len(clk.regions)
+            while n_target is None or len(blocks) < n_target:
+                if st.pos + steps > shape.n_ctx:
+                    st.pos = w["prompt_len"]             # timing only: alpha/beta indices stay in range
+                torch.cuda.synchronize()
+                clk.mark_start()
+                e0.record()
+                model.generate(st, steps, 5, g, ws, out=store)
+                e1.record()
+                torch.cuda.synchronize()
+                clk.mark_stop()
+                blocks.append(e0.elapsed_time(e1))
+                if n_target is None:
+                    n_target = max(1, min(args.max_blocks, math.ceil(args.min_time * 1e3 / blocks[0])))
+            ms = statistics.median(blocks) / steps
+            curve.append({"batch": B, "ms_per_step": round(ms, 4), "tokens_per_s": round(B / (ms / 1e3), 1),
+                          "blocks": len(blocks), "steps_per_block": steps,
+                          "ms_per_step_min": round(min(blocks) / steps, 4), "ms_per_step_max": round(max(blocks) / steps, 4),
+                          "state_bytes_per_sample": L * d * sbytes, "status": st.status(),
+                          "clocks": clk.summary(clk.regions[region0:])})
+            print(json.dumps(curve[-1]), file=sys.stderr, flush=True)
+            del st, prompts, store
+            torch.cuda.empty_cache()
     line = {"metric": METRIC, "unit": UNIT, "n_gpus": 1, "sweep": curve, "max_concurrent_samples": max_conc,
             "state_dtype": args.state_dtype, "config": {"workload": "sweep: mid SRM, 128-token uniform prompts"}}
     print(json.dumps(line), flush=True)
@@ -564,6 +708,18 @@ def run_variants(args):
     print(json.dumps({"variants": out, "peak": f"{peak_src}: {peaks['hbm_gbs']} GB/s", "inputs": "larger than L2"}), flush=True)
 
 
+def self_launch(n: int, argv) -> int:
+    """`python bench.py --gpus N` without a launcher: start N local ranks (one process per GPU) of this same
+    command through torch.distributed.run on the loopback address and return its exit code."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
+    return subprocess.call(cmd)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -592,6 +748,9 @@ def main():
                     help="rl workload: prefill all 16384 rows instead of the 16 distinct prompts")
     ap.add_argument("--no-prefill", action="store_true",
                     help="skip the prefill (cache stays zero, pos = prompt length): keeps profiler captures short")
+    ap.add_argument("--min-time", type=float, default=MIN_TIMED_S,
+                    help="the K-step block is repeated until this many seconds of device time have been timed")
+    ap.add_argument("--max-blocks", type=int, default=400)
     ap.add_argument("--sweep", action="store_true")
     ap.add_argument("--sweep-max", type=int, default=0)
     ap.add_argument("--variants", action="store_true",
@@ -599,6 +758,8 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(self_launch(args.gpus, sys.argv[1:]))
     elif args.sweep:
         run_sweep(args)
     elif args.variants:

@@ -66,6 +66,9 @@ enum {
   SRM_FLAG_SIMT_GEMM = 1,            /* debug: run the bf16 GEMMs on the plain SIMT kernel  */
   SRM_FLAG_NO_SPLITK = 16,           /* the down projection of a decode step always gives whole output tiles to a CTA
                                         pair (see srm_k_gemm_splitk); for comparison and measurement */
+  SRM_FLAG_NO_FUSED_TOPK = 32,       /* top-k selection always from fp32 logits written to the workspace (default: the
+                                        candidates are collected inside the LM-head epilogue and no logits are written
+                                        when the caller does not ask for them); for comparison and measurement */
   SRM_FLAG_HEAD_PROJ = 2             /* token mixer with head projections [Method/Architecture, Eq. 10]:
                                         q = W_in LN1(x) (W_in stacks the per-head I_g), heads of q mixed, and
                                         x += W_out (concatenated heads); the cache holds projected values.
@@ -137,8 +140,9 @@ size_t srm_weights_bytes(const srm_config* cfg);
 int srm_weight_slot(const srm_config* cfg, int32_t layer, int32_t tensor,
                     size_t* offset, size_t* nbytes, int32_t* elem_bytes);
 /* Bytes of the state buffer for B samples: a 256-byte header (status word, counters), the
- * last selected token int32[B], the per-sample position int32[B] (used after srm_prefill_ragged),
- * each rounded up to 256 bytes, then the cache [L, B, d] in state_dtype. */
+ * last selected token int32[B], the per-sample position int32[B] (used after srm_prefill_ragged), the
+ * per-sample candidate threshold float[B] of the fused top-k selection, each rounded up to 256 bytes, then the
+ * cache [L, B, d] in state_dtype. */
 size_t srm_state_bytes(const srm_config* cfg, int64_t B);
 /* Workspace bytes so that decode processes `B_chunk` samples per pass and prefill handles
  * prompts of up to `n_prefill_max` tokens in one pass of at least one sample. Calls accept any
@@ -177,6 +181,18 @@ int srm_state_is_ragged(const srm_state* s);
  * and tests), and of the last-token vector int32[B]. */
 void* srm_state_layer_ptr(const srm_state* s, int32_t layer);
 int32_t* srm_state_last_token_ptr(const srm_state* s);
+/* Fused top-k selection [Recurrent Throughput and Concurrency: choosing the next tokens from the logits is the
+ * step the paper measures as its large-batch bottleneck]. With SRM_SELECT_TOPK, top_k <= 160, V >= 2048, the
+ * tensor-core path and no logits requested, srm_decode_step / srm_generate collect, inside the LM-head epilogue,
+ * every logit of a row at or above that row's threshold and select among those: no logits reach HBM. The set is
+ * exact whenever it holds at least top_k logits. The threshold of a sample is carried from one selection to its
+ * next (float[B] in the state buffer; all-zero bits = none yet) and aims at about max(192, 3 top_k) candidates. A
+ * row with no threshold, fewer than top_k candidates or more than 1024 is handed back: its logits alone are
+ * recomputed into the workspace and it goes through the same kernels as the logits path, so ids are identical to
+ * that path in every case. The two calls below expose the threshold vector (device pointer, for tests and
+ * checkpoints) and the number of rows handed back since the state was last reset (synchronises `stream`). */
+float* srm_state_topk_threshold_ptr(const srm_state* s);
+int srm_state_topk_handed_back(srm_state* s, void* stream, uint64_t* rows);
 /* Synchronises `stream`, copies the device status word to *flags and clears it.
  * Returns SRM_ERR_DEVICE_STATUS when any bit was set. */
 int srm_status(srm_state* s, void* stream, uint32_t* flags);

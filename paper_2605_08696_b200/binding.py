@@ -21,6 +21,7 @@ FLAG_HEAD_PROJ = 2
 FLAG_NO_GRAPH = 4
 FLAG_GRAPH = 8
 FLAG_NO_SPLITK = 16
+FLAG_NO_FUSED_TOPK = 32
 # enum srm_error
 ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_BUFFER_TOO_SMALL, ERR_CTX_OVERFLOW, ERR_CUDA, \
     ERR_DEVICE_STATUS, ERR_STATIC_SCRATCH = -1, -2, -3, -4, -5, -6, -7, -8
@@ -87,6 +88,8 @@ SYMBOLS = {
     "srm_state_is_ragged": (C.c_int, [_P]),
     "srm_state_layer_ptr": (_P, [_P, _I32]),
     "srm_state_last_token_ptr": (_P, [_P]),
+    "srm_state_topk_threshold_ptr": (_P, [_P]),
+    "srm_state_topk_handed_back": (C.c_int, [_P, _P, C.POINTER(C.c_uint64)]),
     "srm_status": (C.c_int, [_P, _P, C.POINTER(C.c_uint32)]),
     "srm_prefill": (C.c_int, [_P, _P, _P, _I32, C.POINTER(_Sampling), _P, _P, _P, _SZ, _P]),
     "srm_prefill_ragged": (C.c_int, [_P, _P, _P, _I32, _P, C.POINTER(_Sampling), _P, _P, _P, _SZ, _P]),
@@ -259,6 +262,17 @@ class SRMState:
     def cache(self) -> torch.Tensor:
         """[L, B, d] copy of the whole cache in fp32."""
         return torch.stack([self.layer(l).float() for l in range(self.model.cfg.n_layers)])
+
+    def topk_thresholds(self) -> torch.Tensor:
+        """View of the per-sample candidate thresholds of the fused top-k selection, float32 [B] (0 bits: none)."""
+        off = _lib().srm_state_topk_threshold_ptr(self.handle) - self.buf.data_ptr()
+        return self.buf[off: off + 4 * self.B].view(torch.float32)
+
+    def topk_handed_back(self) -> int:
+        """Rows the fused top-k selection handed back to the logits path since the last reset (synchronises)."""
+        n = C.c_uint64(0)
+        _check(_lib().srm_state_topk_handed_back(self.handle, _stream(), C.byref(n)), "srm_state_topk_handed_back")
+        return n.value
 
     def last_token(self) -> torch.Tensor:
         off = _lib().srm_state_last_token_ptr(self.handle) - self.buf.data_ptr()

@@ -31,6 +31,7 @@ __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.lau
 constexpr int kCtrPos = 1;     // absolute position of the token being consumed
 constexpr int kCtrStep = 2;    // Philox step of the selection
 constexpr int kCtrCol = 3;     // column of the token store the selection writes
+constexpr int kCtrHandedBack = 4;   // rows the fused top-k selection handed back to the logits path, since the last reset
 
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll

@@ -11,7 +11,9 @@ enum GemmEpilogue {
   kEpiBiasGelu = 0,       // out = gelu(D + bias) in the activation type
   kEpiBiasResidual = 1,   // out += D + bias (fp32)
   kEpiPlain = 2,          // out = D (fp32)
-  kEpiArgmax = 3          // tensor-core kernel only: per-row (max, lowest column) of every 64-column slice of D
+  kEpiArgmax = 3,         // tensor-core kernel only: per-row (max, lowest column) of every 64-column slice of D
+  kEpiCollect = 4         // tensor-core kernel only: per row, every element of D at or above the row's threshold is
+                          // appended to the row's candidate list (top-k selection without writing D)
 };
 
 constexpr int kSimtBM = 64, kSimtBN = 64, kSimtBK = 16;

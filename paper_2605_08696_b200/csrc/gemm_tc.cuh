@@ -230,7 +230,22 @@ struct GemmArgs {
                        // results uint2 [argmax_slots(N)][M] = (bits of the slice maximum, its column)
   uint32_t* status;
   int w_static;        // W is constant data (model weights): its first tiles may be fetched before pdl_wait()
+  // kEpiCollect: out = candidate lists, unsigned long long [M][cap]; an element v of row r in column c with
+  // v >= thr[r] takes the next free place of row r (cnt[r], counted atomically; places beyond cap are dropped but
+  // counted) as ((~order_key(v)) << 32 | c): ascending order of these words is (value descending, column ascending).
+  const float* thr;    // [M] per-row thresholds; a NaN or all-zero word means "none": nothing is collected
+  uint32_t* cnt;       // [M] zero on entry
+  int cap;
+  // Only the first *m_limit rows (a device word written by an earlier kernel of the stream) are computed; nullptr:
+  // all M rows. The first weight tiles are then not fetched ahead of the dependency wait.
+  const uint32_t* m_limit;
 };
+
+// order-preserving map float -> uint32 (larger float, larger key)
+__device__ __forceinline__ uint32_t order_key_bits(float f) {
+  const uint32_t u = __float_as_uint(f);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
 
 // kEpiArgmax: one partial result per row and per 64-column slice of the (256-column padded) output.
 __host__ __device__ inline int64_t argmax_slots(int64_t N) { return (N + BN - 1) / BN * (BN / 64); }
@@ -319,6 +334,33 @@ __device__ __forceinline__ void argmax_chunk16(const uint32_t (&r)[16], int col,
   }
 }
 
+// Top-k candidates among 16 consecutive logits r[0..15] of columns col .. col+15 of this lane's row: everything
+// at or above the row's threshold goes to the row's list. The chunk maximum decides in eight instructions
+// whether the lane has anything to do (about one chunk in ten has, with some 200 candidates per row of 32000).
+// A NaN never qualifies (it is reported through `bad`).
+__device__ __forceinline__ void collect_chunk16(const uint32_t (&r)[16], int col, const GemmArgs& g, int64_t row, float thr,
+                                                bool& bad) {
+  float f[16];
+#pragma unroll
+  for (int j = 0; j < 16; ++j) f[j] = __uint_as_float(r[j]);
+  const float m = max3_nan(max3_nan(max3_nan(f[0], f[1], f[2]), max3_nan(f[3], f[4], f[5]), max3_nan(f[6], f[7], f[8])),
+                           max3_nan(max3_nan(f[9], f[10], f[11]), max3_nan(f[12], f[13], f[14]), f[15]), -INFINITY);
+  if (m >= thr || m != m) {
+    unsigned long long* list = reinterpret_cast<unsigned long long*>(g.out) + row * (int64_t)g.cap;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      if (col + j < g.N) {
+        bad |= !(f[j] == f[j]);
+        if (f[j] >= thr) {
+          const uint32_t slot = atomicAdd(g.cnt + row, 1u);
+          if (slot < (uint32_t)g.cap)
+            list[slot] = ((unsigned long long)(~order_key_bits(f[j])) << 32) | (uint32_t)(col + j);
+        }
+      }
+    }
+  }
+}
+
 // The 64 accumulator columns [col0, col0 + 64) of this warp's 32 rows: TMEM -> registers -> bias /
 // activation -> one (bf16) or two (fp32) boxes of 128 bytes per row, or the fused greedy selection.
 // The columns come in four chunks of 16; the load of chunk i+1 is in flight while chunk i is processed
@@ -332,6 +374,11 @@ __device__ __forceinline__ void epilogue_columns(const GemmArgs& g, const CUtens
   float bv = -INFINITY;                  // kEpiArgmax: running maximum and its column
   int bi = 0x7fffffff;
   bool bad = false;
+  float thr = INFINITY;                  // kEpiCollect: this row's threshold
+  if (EPI == kEpiCollect && row0 + lane < g.M) {
+    thr = __ldg(g.thr + row0 + lane);
+    if (!(thr == thr) || __float_as_uint(thr) == 0u) thr = INFINITY;
+  }
   tmem_ld16(taddr, ra);
   tmem_ld_wait();
 #pragma unroll
@@ -342,6 +389,8 @@ __device__ __forceinline__ void epilogue_columns(const GemmArgs& g, const CUtens
     const int col = col0 + 16 * c;
     if (EPI == kEpiArgmax) {
       if (col < g.N) argmax_chunk16(cur, col, g.N, bv, bi, bad);
+    } else if (EPI == kEpiCollect) {
+      if (col < g.N && row0 + lane < g.M) collect_chunk16(cur, col, g, row0 + lane, thr, bad);
     } else if (EPI == kEpiBiasGelu) {
 #pragma unroll
       for (int j = 0; j < 16; j += 4) {
@@ -373,6 +422,7 @@ __device__ __forceinline__ void epilogue_columns(const GemmArgs& g, const CUtens
     }
     if (c + 1 < kChunks) tmem_ld_wait();
   }
+  if (EPI == kEpiCollect && bad) raise_status(g.status, kStatusNonFinite);
   if (EPI == kEpiArgmax) {
     if (bad) raise_status(g.status, kStatusNonFinite);
     const int64_t slot = col0 / kColsPerEpiWarp;
@@ -416,9 +466,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const uint32_t tmem_base = *tmem_slot;
   // Barriers, tensor memory and the cluster handshake are set up; from here on global memory is touched.
   // The producer thread orders itself (it may fetch weights, which no kernel writes, ahead of the wait).
-  if (threadIdx.x != 0) pdl_wait();
+  if (threadIdx.x != 0 || g.m_limit != nullptr) pdl_wait();
+  int64_t M_rows = g.M;
+  if (g.m_limit != nullptr) {              // a row count left on the device by an earlier kernel
+    const int64_t lim = (int64_t)*reinterpret_cast<const volatile uint32_t*>(g.m_limit);
+    M_rows = lim < M_rows ? lim : M_rows;
+  }
 
-  const int64_t m_tiles = (g.M + BM - 1) / BM, n_tiles = (g.N + BN - 1) / BN;
+  const int64_t m_tiles = (M_rows + BM - 1) / BM, n_tiles = (g.N + BN - 1) / BN;
   const int64_t tiles = m_tiles * n_tiles;
   const int k_blocks = static_cast<int>(g.K / BK);
 
@@ -510,7 +565,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int col0 = static_cast<int>(n0) + cgrp * kColsPerEpiWarp;
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) +
                              static_cast<uint32_t>(acc * BN + cgrp * kColsPerEpiWarp);
-      if (row0 < g.M && (col0 < g.N || EPI == kEpiArgmax)) epilogue_columns<EPI>(g, &tmD, buf, lane, taddr, row0, col0);
+      if (row0 < M_rows && (col0 < g.N || EPI == kEpiArgmax)) epilogue_columns<EPI>(g, &tmD, buf, lane, taddr, row0, col0);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(mapa(smem_u32(&tempty[acc]), 0));

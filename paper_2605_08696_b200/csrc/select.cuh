@@ -20,7 +20,26 @@ struct SelectOut {
   int64_t row_div;      // output row r reads logits row r / row_div (replicas of one prompt share a row); >= 1
   const int32_t* ctr;   // device-side step counters (store column, Philox step), or nullptr: host values apply
   int32_t* pos;         // [R] per-row positions, advanced by one with every selection, or nullptr
+  // Compacted launch (the rows that the fused top-k path hands back): block i serves output row row_map[i] and
+  // reads logits row i; only the first *n_rows blocks have work. nullptr: block i serves row i.
+  const int32_t* row_map;
+  const uint32_t* n_rows;
+  float* thr_out;       // [R] or nullptr: top-k only, the candidate threshold to use for this row's next selection
 };
+
+// Output row and logits row of block `i`; false when the block has nothing to do.
+__device__ __forceinline__ bool select_rows(const SelectOut& o, int64_t i, int64_t R, int64_t* row, int64_t* lrow) {
+  if (o.row_map != nullptr) {
+    if (i >= (int64_t)*o.n_rows || i >= R) return false;
+    *row = o.row_map[i];
+    *lrow = i;
+    return true;
+  }
+  if (i >= R) return false;
+  *row = i;
+  *lrow = i / o.row_div;
+  return true;
+}
 
 __device__ __forceinline__ void write_token(const SelectOut& o, int64_t row, int tok) {
   o.last_tok[row] = tok;
@@ -132,6 +151,82 @@ __device__ __forceinline__ float key_value(uint32_t k) {
   return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
 }
 
+// ---- candidate threshold carried from one selection of a row to its next (fused top-k) ----------
+// The LM head with fused top-k keeps, per row, every logit at or above a threshold; the selection is exact when
+// that set holds at least k logits. The threshold for the NEXT step of the same sample is taken from this
+// step's sorted candidates so that about topk_target(k) logits are expected above it: the logits of consecutive
+// positions of one sample have nearly the same scale. With fewer candidates than the target the upper tail is
+// continued below the lowest one as an exponential in the value. 0 (all bits zero) stands for "no threshold".
+__host__ __device__ inline int topk_target(int k) { return 3 * k > 192 ? 3 * k : 192; }
+constexpr int kFusedTopkCap = 1024;      // places per row in the candidate lists
+constexpr int kFusedTopkMaxK = 160;      // 3 k must stay well below the capacity
+
+__device__ __forceinline__ float cand_value(unsigned long long w) { return key_value(~(uint32_t)(w >> 32)); }
+
+__device__ inline float next_threshold(const unsigned long long* sorted, int c, int k) {
+  const int T = topk_target(k);
+  float t;
+  if (c >= T) {
+    t = cand_value(sorted[T - 1]);
+  } else {
+    // slope of log(rank) against value between rank i (the k-th, or a quarter of the way in when k is small) and
+    // the lowest candidate; with too few candidates below rank i, between the first and the k-th instead
+    const int i = k > (c + 3) / 4 ? k : (c + 3) / 4;
+    const float v1 = cand_value(sorted[0]), vk = cand_value(sorted[k - 1]), vi = cand_value(sorted[i - 1]),
+                vn = cand_value(sorted[c - 1]);
+    float s = 0.f;
+    if (c >= i + (i / 4 > 2 ? i / 4 : 2)) s = (vi - vn) / logf((float)c / (float)i);
+    else if (k >= 2) s = (v1 - vk) / logf((float)k);
+    t = vn - s * logf((float)T / (float)c);
+    if (!(s > 0.f)) t = 0.f;
+  }
+  if (!(fabsf(t) < INFINITY)) return 0.f;        // NaN, infinities: none
+  return t == 0.f ? -0.0f : t;                   // a threshold of zero keeps a bit set
+}
+
+// Thread 0 of a block: inverse-CDF draw over the k first of `sorted` (logit desc, id asc) and the row's outputs.
+__device__ inline void draw_topk(const unsigned long long* sorted, int c, int k, float inv_temp, uint64_t seed,
+                                 uint64_t sidx, int step, const SelectOut& out, int64_t row, float* cdf) {
+  const float l0 = cand_value(sorted[0]);
+  float acc = 0.f;
+  for (int i = 0; i < k; ++i) {
+    acc += expf((cand_value(sorted[i]) - l0) * inv_temp);
+    cdf[i] = acc;
+  }
+  const uint32_t r = philox4x32_10_word0((uint32_t)sidx, (uint32_t)(out.ctr != nullptr ? out.ctr[kCtrStep] : step), 0u, 0u,
+                                         (uint32_t)seed, (uint32_t)(seed >> 32));
+  const float u = (float)(r >> 8) * (1.0f / 16777216.0f);
+  const float target = u * acc;
+  int pick = k - 1;
+  for (int i = 0; i < k; ++i) {
+    if (cdf[i] > target) { pick = i; break; }
+  }
+  if (out.thr_out != nullptr) out.thr_out[row] = next_threshold(sorted, c, k);
+  write_token(out, row, (int)(uint32_t)(sorted[pick] & 0xffffffffull));
+}
+
+// Sorts cand[0 .. c) of a block's shared memory ascending, i.e. by (logit desc, id asc); c <= the array's
+// power-of-two capacity. All threads of the block call it.
+__device__ inline void sort_candidates(unsigned long long* cand, int c, int tid, int nthreads) {
+  int P = 2;
+  while (P < c) P <<= 1;
+  for (int i = c + tid; i < P; i += nthreads) cand[i] = ~0ull;
+  __syncthreads();
+  for (int size = 2; size <= P; size <<= 1) {
+    for (int stride = size >> 1; stride > 0; stride >>= 1) {
+      for (int i = tid; i < P; i += nthreads) {
+        const int j = i ^ stride;
+        if (j > i) {
+          const unsigned long long a = cand[i], b = cand[j];
+          const bool up = (i & size) == 0;
+          if ((a > b) == up) { cand[i] = b; cand[j] = a; }
+        }
+      }
+      __syncthreads();
+    }
+  }
+}
+
 // ---- top-k + temperature + inverse-CDF draw ------------------------------------------------
 // 1. radix-select (4 passes of 8 bits) the key of the k-th largest logit;
 // 2. collect everything above it, plus the lowest ids among the ties at it;
@@ -144,17 +239,17 @@ select_topk_kernel(const float* __restrict__ logits, int64_t R, int V, int k, fl
                    uint64_t sample_base, int step, SelectOut out, uint32_t* status, int only_marked) {
   pdl_trigger();
   pdl_wait();
+  int64_t row, lrow;
+  if (!select_rows(out, blockIdx.x, R, &row, &lrow)) return;
   // second stage of the streaming kernel below: only the rows it marked (-1) are processed here
-  if (only_marked && out.last_tok[blockIdx.x < R ? blockIdx.x : 0] != -1) return;
+  if (only_marked && out.last_tok[row] != -1) return;
   extern __shared__ float srow[];
   __shared__ uint32_t hist[256];
   __shared__ unsigned long long cand[kTopKMax];
   __shared__ uint32_t sh_prefix, sh_need, sh_ties, sh_count, sh_running;
   __shared__ uint32_t warp_cnt[kSelThreads / 32];
 
-  const int64_t row = blockIdx.x;
-  if (row >= R) return;
-  const float* lr = logits + (row / out.row_div) * (int64_t)V;
+  const float* lr = logits + lrow * (int64_t)V;
   const int tid = threadIdx.x;
   bool bad = false;
   if (ROW_IN_SMEM) {
@@ -264,6 +359,7 @@ select_topk_kernel(const float* __restrict__ logits, int64_t R, int V, int k, fl
     for (int i = 0; i < k; ++i) {
       if (cdf[i] > target) { pick = i; break; }
     }
+    if (out.thr_out != nullptr) out.thr_out[row] = 0.f;     // no candidate set to take a threshold from
     write_token(out, row, (int)(uint32_t)(cand[pick] & 0xffffffffull));
   }
 }
@@ -293,9 +389,9 @@ select_topk_stream_kernel(const float* __restrict__ logits, int64_t R, int V, in
   __shared__ uint32_t sh_count;
   __shared__ float cdf[kTopKMax];
 
-  const int64_t row = blockIdx.x;
-  if (row >= R) return;
-  const float* lr = logits + (row / out.row_div) * (int64_t)V;
+  int64_t row, lrow;
+  if (!select_rows(out, blockIdx.x, R, &row, &lrow)) return;
+  const float* lr = logits + lrow * (int64_t)V;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
   // ---- pass 1: moments ----
@@ -353,43 +449,52 @@ select_topk_stream_kernel(const float* __restrict__ logits, int64_t R, int V, in
     return;
   }
 
-  // ---- sort the c candidates ascending by (~key, id) = (logit desc, id asc) ----
-  int P = 2;
-  while (P < (int)c) P <<= 1;
-  for (int i = (int)c + tid; i < P; i += kSelThreads) cand[i] = ~0ull;
+  sort_candidates(cand, (int)c, tid, kSelThreads);
+  if (tid == 0) draw_topk(cand, (int)c, k, inv_temp, seed, sample_base + (uint64_t)row, step, out, row, cdf);
+}
+
+// ---- top-k fused into the LM head: second stage ------------------------------------------------------
+// The LM head (kEpiCollect epilogue) has left, per row, the logits at or above the row's threshold as sortable
+// words in lists[row][0 .. cnt[row]). A row whose list holds at least k and at most `cap` of them is settled
+// here exactly as the streaming kernel settles it (any set {x >= t} with at least k members contains the k
+// largest logits and every tie at the k-th place): sort, softmax weights, Philox draw. A row without a
+// threshold yet, with fewer than k candidates, or with more than fit is handed back: its activation row is
+// copied to the next free row of a_fb and its index to fb_rows (n_fb counts them), and the caller recomputes
+// the logits of just those rows and runs the streaming kernel on them (SelectOut::row_map).
+__global__ void __launch_bounds__(kSelThreads)
+topk_merge_kernel(const unsigned long long* __restrict__ lists, const uint32_t* __restrict__ cnt, const float* __restrict__ thr,
+                  int cap, int64_t R, int k, float inv_temp, uint64_t seed, uint64_t sample_base, int step, SelectOut out,
+                  const uint4* __restrict__ a, uint4* __restrict__ a_fb, int row_vecs, int32_t* __restrict__ fb_rows,
+                  uint32_t* __restrict__ n_fb, uint32_t* __restrict__ handed_back) {
+  pdl_trigger();
+  pdl_wait();
+  __shared__ unsigned long long cand[kFusedTopkCap];
+  __shared__ float cdf[kTopKMax];
+  __shared__ uint32_t sh_idx;
+  const int64_t row = blockIdx.x;
+  if (row >= R) return;
+  const int tid = threadIdx.x;
+  const uint32_t c = cnt[row];
+  const float t = thr[row];
+  const bool have_thr = (t == t) && __float_as_uint(t) != 0u;
+  if (!have_thr || c < (uint32_t)k || c > (uint32_t)cap) {          // block-uniform
+    if (tid == 0) {
+      const uint32_t idx = atomicAdd(n_fb, 1u);
+      fb_rows[idx] = (int32_t)row;
+      sh_idx = idx;
+      if (handed_back != nullptr) atomicAdd(handed_back, 1u);
+    }
+    __syncthreads();
+    const uint4* src = a + row * (int64_t)row_vecs;
+    uint4* dst = a_fb + (int64_t)sh_idx * row_vecs;
+    for (int i = tid; i < row_vecs; i += kSelThreads) dst[i] = src[i];
+    return;
+  }
+  const unsigned long long* lr = lists + row * (int64_t)cap;
+  for (int i = tid; i < (int)c; i += kSelThreads) cand[i] = lr[i];
   __syncthreads();
-  for (int size = 2; size <= P; size <<= 1) {
-    for (int stride = size >> 1; stride > 0; stride >>= 1) {
-      for (int i = tid; i < P; i += kSelThreads) {
-        const int j = i ^ stride;
-        if (j > i) {
-          const unsigned long long a = cand[i], b = cand[j];
-          const bool up = (i & size) == 0;
-          if ((a > b) == up) { cand[i] = b; cand[j] = a; }
-        }
-      }
-      __syncthreads();
-    }
-  }
-  if (tid == 0) {
-    const float l0 = key_value(~(uint32_t)(cand[0] >> 32));
-    float acc = 0.f;
-    for (int i = 0; i < k; ++i) {
-      const float li = key_value(~(uint32_t)(cand[i] >> 32));
-      acc += expf((li - l0) * inv_temp);
-      cdf[i] = acc;
-    }
-    const uint64_t sidx = sample_base + (uint64_t)row;
-    const uint32_t r = philox4x32_10_word0((uint32_t)sidx, (uint32_t)(out.ctr != nullptr ? out.ctr[kCtrStep] : step), 0u, 0u, (uint32_t)seed,
-                                           (uint32_t)(seed >> 32));
-    const float u = (float)(r >> 8) * (1.0f / 16777216.0f);
-    const float target = u * acc;
-    int pick = k - 1;
-    for (int i = 0; i < k; ++i) {
-      if (cdf[i] > target) { pick = i; break; }
-    }
-    write_token(out, row, (int)(uint32_t)(cand[pick] & 0xffffffffull));
-  }
+  sort_candidates(cand, (int)c, tid, kSelThreads);
+  if (tid == 0) draw_topk(cand, (int)c, k, inv_temp, seed, sample_base + (uint64_t)row, step, out, row, cdf);
 }
 
 // Cache rows of `replicas` consecutive samples = the row of their prompt:

@@ -236,6 +236,7 @@ struct srm_state {
   uint32_t* status;       // device status word (header)
   int32_t* last_tok;      // [B]
   int32_t* pos_dev;       // [B] per-sample positions, used after srm_prefill_ragged
+  float* thr;             // [B] candidate threshold of each sample's next top-k selection (0: none yet)
   uint8_t* S;             // [L, B, d] in state dtype
   int64_t pos;            // position of the next token (ragged: of the longest sample)
   bool ragged = false;    // samples have their own positions (pos_dev)
@@ -267,7 +268,7 @@ constexpr size_t kStateHeader = 256;
 
 size_t state_bytes_for(const srm_config& c, int64_t B) {
   const size_t sb = c.state_dtype == SRM_DTYPE_BF16 ? 2 : 4;
-  return kStateHeader + 2 * align_up((size_t)B * 4, 256) + (size_t)c.n_layers * B * c.d_model * sb;
+  return kStateHeader + 3 * align_up((size_t)B * 4, 256) + (size_t)c.n_layers * B * c.d_model * sb;
 }
 
 // ---- workspace carving ----------------------------------------------------------------------
@@ -464,6 +465,7 @@ int ensure_tc_ready(srm_model& m) {
   SRM_CUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<kEpiBiasResidual>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes));
   SRM_CUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<kEpiPlain>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes));
   SRM_CUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<kEpiArgmax>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes));
+  SRM_CUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<kEpiCollect>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes));
   SRM_CUDA(cudaFuncSetAttribute(tc::gemm_tc_splitk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes));
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2 * (m.num_sms / 2));
@@ -541,6 +543,17 @@ int launch_gemm_splitk(srm_model& m, int64_t M, int64_t N, int64_t K, const void
   return SRM_OK;
 }
 
+float topk_z0(int top_k, int V) {
+  // threshold start of the streaming kernel: the normal quantile that leaves about 2.5 k (at least 96: the set also
+  // yields the row's next candidate threshold, which wants a tail to measure) of the V logits above it
+  // (rational approximation 26.2.23 of Abramowitz & Stegun; only a starting point, the kernel adapts)
+  double pr = (2.5 * top_k > 96.0 ? 2.5 * top_k : 96.0) / (double)V;
+  if (pr > 0.45) pr = 0.45;
+  const double tt = std::sqrt(-2.0 * std::log(pr));
+  return (float)(tt - (2.515517 + 0.802853 * tt + 0.010328 * tt * tt) /
+                          (1.0 + 1.432788 * tt + 0.189269 * tt * tt + 0.001308 * tt * tt * tt));
+}
+
 int check_sampling(const srm_model& m, const srm_sampling* s) {
   if (s == nullptr) return SRM_ERR_INVALID_ARG;
   if (s->mode == SRM_SELECT_GREEDY) return SRM_OK;
@@ -578,13 +591,7 @@ int launch_select(const srm_model& m, int64_t R, const float* logits, const srm_
     }
   } else {
     const float inv_t = 1.0f / s.temperature;
-    // threshold start: the normal quantile that leaves about 2.5 k of the V logits above it
-    // (rational approximation 26.2.23 of Abramowitz & Stegun; only a starting point, the kernel adapts)
-    double pr = 2.5 * s.top_k / (double)V;
-    if (pr > 0.45) pr = 0.45;
-    const double tt = std::sqrt(-2.0 * std::log(pr));
-    const float z0 = (float)(tt - (2.515517 + 0.802853 * tt + 0.010328 * tt * tt) /
-                                      (1.0 + 1.432788 * tt + 0.189269 * tt * tt + 0.001308 * tt * tt * tt));
+    const float z0 = topk_z0(s.top_k, V);
     SRM_CUDA(launch_kernel(select_topk_stream_kernel, dim3((unsigned)R), dim3(kSelThreads), 0, st, logits, R, V, s.top_k,
                            inv_t, z0, s.seed, sample_base, step, out, status));
     // rows the streaming kernel could not settle (marked -1): the radix selection, reading the row from
@@ -617,6 +624,80 @@ int launch_lm_head_greedy(srm_model& m, int64_t R, const void* a, void* part, co
   const unsigned grid = (unsigned)((R + kArgmaxRows - 1) / kArgmaxRows);
   SRM_CUDA(launch_kernel(argmax_reduce_kernel, dim3(grid), dim3(kArgmaxRows * kArgmaxLanes), 0, st, reinterpret_cast<const uint2*>(part), R,
                                                                    tc::argmax_slots(V), V, out));
+  SRM_CUDA(cudaGetLastError());
+  return SRM_OK;
+}
+
+// True when top-k selection can be fused into the LM-head GEMM (candidates collected in the epilogue, no logits
+// written): tensor-core path, no logits requested, k small enough for three times k candidates to sit well
+// inside a list, and a workspace whose logits and hidden-layer areas are large enough for the lists and for the
+// rows handed back (V >= 2048, F >= 2 d).
+bool can_fuse_topk(const srm_model& m, const srm_sampling& s, const float* logits_out) {
+  return s.mode == SRM_SELECT_TOPK && logits_out == nullptr && m.cfg.dtype == SRM_DTYPE_BF16 &&
+         !(m.cfg.flags & (SRM_FLAG_SIMT_GEMM | SRM_FLAG_NO_FUSED_TOPK)) && s.top_k <= kFusedTopkMaxK &&
+         (size_t)m.cfg.vocab * 4 >= (size_t)kFusedTopkCap * 8 && m.cfg.ffn_mult >= 2;
+}
+
+// LM head with top-k / temperature / Philox selection and no logits in HBM. `lists` (the logits area of the
+// workspace) receives the per-row candidate lists; `scratch` (the hidden-layer area, free after the last down
+// projection) holds the activation rows handed back, their indices and the counters. Rows the merge kernel
+// cannot settle (no threshold yet, too few or too many candidates) get their logits from a second LM-head
+// launch over just those rows, written over the (then dead) lists, and the streaming selection.
+int launch_lm_head_topk(srm_model& m, int64_t R, const void* a, void* lists, void* scratch, const float* thr,
+                        const srm_sampling& s, uint64_t sample_base, int step, const SelectOut& out, uint32_t* status,
+                        uint32_t* handed_back, cudaStream_t st) {
+  if (R <= 0) return SRM_OK;
+  const int V = m.cfg.vocab, d = m.cfg.d_model;
+  const size_t row_bytes = (size_t)d * 2;
+  uint8_t* p = static_cast<uint8_t*>(scratch);
+  void* a_fb = p; p += align_up((size_t)R * row_bytes, 256);
+  int32_t* fb_rows = reinterpret_cast<int32_t*>(p); p += align_up((size_t)R * 4, 256);
+  uint32_t* cnt = reinterpret_cast<uint32_t*>(p); p += align_up((size_t)R * 4, 256);
+  uint32_t* n_fb = reinterpret_cast<uint32_t*>(p);
+  SRM_CUDA(cudaMemsetAsync(cnt, 0, align_up((size_t)R * 4, 256) + 256, st));       // counters and n_fb
+  int rc = ensure_tc_ready(m);
+  if (rc != SRM_OK) return rc;
+  const float inv_t = 1.0f / s.temperature;
+  CUtensorMap ta, tb;
+  {
+    LaunchScope scope(m, SRM_KERNEL_GEMM_LM, st);
+    if ((rc = m.tmap(a, R, d, tc::kRowsPerCta, 2, &ta)) != SRM_OK) return rc;
+    if ((rc = m.tmap(m.ptr(-1, SRM_T_W_LM), V, d, tc::kRowsPerCta, 2, &tb)) != SRM_OK) return rc;
+    tc::GemmArgs g{R, V, d, nullptr, lists, status, 1, thr, cnt, kFusedTopkCap, nullptr};
+    const int64_t tiles = ((R + tc::BM - 1) / tc::BM) * ((V + tc::BN - 1) / tc::BN);
+    const unsigned grid = 2u * (unsigned)(tiles < m.tc_clusters ? tiles : m.tc_clusters);
+    SRM_CUDA(launch_kernel(tc::gemm_tc_kernel<kEpiCollect>, dim3(grid), dim3(tc::kThreads), tc::kSmemBytes, st, ta, tb, ta, g));
+  }
+  {
+    LaunchScope scope(m, SRM_KERNEL_SELECT, st);
+    SRM_CUDA(launch_kernel(topk_merge_kernel, dim3((unsigned)R), dim3(kSelThreads), 0, st,
+                           reinterpret_cast<const unsigned long long*>(lists), cnt, thr, kFusedTopkCap, R, s.top_k, inv_t, s.seed,
+                           sample_base, step, out, reinterpret_cast<const uint4*>(a), reinterpret_cast<uint4*>(a_fb),
+                           (int)(row_bytes / 16), fb_rows, n_fb, handed_back));
+  }
+  {
+    // the rows handed back: logits of the first *n_fb rows of a_fb only (no tile when there is none)
+    LaunchScope scope(m, SRM_KERNEL_GEMM_LM, st);
+    CUtensorMap tf, td;
+    if ((rc = m.tmap(a_fb, R, d, tc::kRowsPerCta, 2, &tf)) != SRM_OK) return rc;
+    if ((rc = m.tmap(lists, R, V, tc::kOutBoxRows, 4, &td)) != SRM_OK) return rc;
+    tc::GemmArgs g{R, V, d, nullptr, lists, status, 0, nullptr, nullptr, 0, n_fb};
+    const int64_t tiles = ((R + tc::BM - 1) / tc::BM) * ((V + tc::BN - 1) / tc::BN);
+    const unsigned grid = 2u * (unsigned)(tiles < m.tc_clusters ? tiles : m.tc_clusters);
+    SRM_CUDA(launch_kernel(tc::gemm_tc_kernel<kEpiPlain>, dim3(grid), dim3(tc::kThreads), tc::kSmemBytes, st, tf, tb, td, g));
+  }
+  {
+    LaunchScope scope(m, SRM_KERNEL_SELECT, st);
+    SelectOut o = out;
+    o.row_map = fb_rows;
+    o.n_rows = n_fb;
+    const float* lg = reinterpret_cast<const float*>(lists);
+    SRM_CUDA(launch_kernel(select_topk_stream_kernel, dim3((unsigned)R), dim3(kSelThreads), 0, st, lg, R, V, s.top_k, inv_t,
+                           topk_z0(s.top_k, V), s.seed, sample_base, step, o, status));
+    SRM_CUDA(launch_kernel(select_topk_kernel<false>, dim3((unsigned)R), dim3(kSelThreads), 0, st, lg, R, V, s.top_k, inv_t,
+                           s.seed, sample_base, step, o, status, 1));
+    ++g_kernel_launches;
+  }
   SRM_CUDA(cudaGetLastError());
   return SRM_OK;
 }
@@ -767,7 +848,11 @@ int decode_chunk(srm_model& m, srm_state& s, int64_t b0, int64_t R, const int32_
   if (o.tok_out) o.tok_out += b0;
   if (o.store) o.store += b0 * o.store_stride;
   if (o.pos) o.pos += b0;
+  if (o.thr_out) o.thr_out += b0;
   if (can_fuse_greedy(m, samp, logits_out)) return launch_lm_head_greedy(m, R, w.a, w.logits, o, s.status, st);
+  if (can_fuse_topk(m, samp, logits_out))
+    return launch_lm_head_topk(m, R, w.a, w.logits, w.H, s.thr + b0, samp, samp.sample_idx_base + (uint64_t)b0, step, o,
+                               s.status, s.status + kCtrHandedBack, st);
   float* lg = logits_out != nullptr ? logits_out + b0 * c.vocab : w.logits;
   if ((rc = launch_gemm(m, kEpiPlain, R, c.vocab, d, w.a, m.ptr(-1, SRM_T_W_LM), nullptr, lg, s.status, st))) return rc;
   return launch_select(m, R, lg, samp, samp.sample_idx_base + (uint64_t)b0, step, o, s.status, st);
@@ -803,7 +888,8 @@ int decode_step_impl(srm_model* m, srm_state* s, const int32_t* d_tok_in, const 
   const int64_t rows = choose_pass_rows(s->B, fit);
   const DecodeWs w = carve_decode(*m, d_ws, rows);
   const int32_t* tok_in = d_tok_in != nullptr ? d_tok_in : s->last_tok;
-  SelectOut out{s->last_tok, d_tok_out, d_store, store_stride, store_col, 1, ctr, s->ragged ? s->pos_dev : nullptr};
+  SelectOut out{s->last_tok, d_tok_out, d_store, store_stride, store_col, 1, ctr, s->ragged ? s->pos_dev : nullptr,
+                nullptr, nullptr, samp->mode == SRM_SELECT_TOPK ? s->thr : nullptr};
   for (int64_t b0 = 0; b0 < s->B; b0 += rows) {
     const int64_t R = (s->B - b0 < rows) ? s->B - b0 : rows;
     if ((rc = decode_chunk(*m, *s, b0, R, tok_in, *samp, step, out, d_logits_out, w, st, ctr))) return rc;
@@ -935,7 +1021,8 @@ int srm_state_create(srm_model* m, int64_t B, void* d_state, size_t nbytes, void
   s->status = reinterpret_cast<uint32_t*>(s->base);
   s->last_tok = reinterpret_cast<int32_t*>(s->base + kStateHeader);
   s->pos_dev = reinterpret_cast<int32_t*>(s->base + kStateHeader + align_up((size_t)B * 4, 256));
-  s->S = s->base + kStateHeader + 2 * align_up((size_t)B * 4, 256);
+  s->thr = reinterpret_cast<float*>(s->base + kStateHeader + 2 * align_up((size_t)B * 4, 256));
+  s->S = s->base + kStateHeader + 3 * align_up((size_t)B * 4, 256);
   s->pos = 0;
   int rc = srm_state_reset(s, stream);
   if (rc != SRM_OK) { delete s; return rc; }
@@ -985,6 +1072,18 @@ void* srm_state_layer_ptr(const srm_state* s, int32_t layer) {
 }
 
 int32_t* srm_state_last_token_ptr(const srm_state* s) { return s ? s->last_tok : nullptr; }
+
+float* srm_state_topk_threshold_ptr(const srm_state* s) { return s ? s->thr : nullptr; }
+
+int srm_state_topk_handed_back(srm_state* s, void* stream, uint64_t* rows) {
+  if (s == nullptr || rows == nullptr) return SRM_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint32_t v = 0;
+  SRM_CUDA(cudaMemcpyAsync(&v, s->status + kCtrHandedBack, 4, cudaMemcpyDeviceToHost, st));
+  SRM_CUDA(cudaStreamSynchronize(st));
+  *rows = v;
+  return SRM_OK;
+}
 
 int srm_status(srm_state* s, void* stream, uint32_t* flags) {
   if (s == nullptr) return SRM_ERR_INVALID_ARG;
@@ -1044,7 +1143,8 @@ int prefill_impl(srm_model* m, srm_state* s, const int32_t* d_tokens, int64_t P,
     }
     // LM head on the last prompt position only; selection per state row
     if ((rc = launch_final_norm(*m, w.x, np, n, n - 1, w.a_last, st, d_len ? d_len + p0 : nullptr))) return rc;
-    SelectOut o{s->last_tok + b0, d_first_tok ? d_first_tok + b0 : nullptr, nullptr, 0, 0, replicas};
+    SelectOut o{s->last_tok + b0, d_first_tok ? d_first_tok + b0 : nullptr, nullptr, 0, 0, replicas, nullptr, nullptr,
+                nullptr, nullptr, samp->mode == SRM_SELECT_TOPK ? s->thr + b0 : nullptr};
     if (replicas == 1 && can_fuse_greedy(*m, *samp, d_logits_last)) {
       if ((rc = launch_lm_head_greedy(*m, np, w.a_last, w.logits, o, s->status, st))) return rc;
       continue;

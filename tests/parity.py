@@ -26,9 +26,11 @@ from helpers import oracle_for, rel_err_rows, top2_margin
 DEV = "cuda:0"
 TOL = {"fp32": 1e-4, "bf16": 3e-2}       # max relative error per row (logits, cache)
 MARGIN = 1e-2                            # tokens must agree where the oracle's top-2 gap exceeds this
-# Fixed bounds on the absolute logit error of a row (max over the vocabulary), per configuration: about twice
-# what was measured over the full horizons (fp32: 2e-6; bf16: grows with depth and width of the model).
-EPS_ABS = {"tiny": 2e-5, "small": 1.2e-2, "mid": 3.0e-2, "rl": 4.0e-2}
+# Fixed bounds on the absolute logit error of a row (max over the vocabulary), per configuration: about one and a
+# half times what was measured over the full horizons (tiny fp32 3e-7; bf16 grows with depth and width: small
+# 0.0083, mid 0.0169, rl 0.0258; with the cache stored in bf16 its rounding adds to it: small 0.0147 after 9 steps).
+EPS_ABS = {"tiny": 2e-5, "small": 1.3e-2, "mid": 2.6e-2, "rl": 4.0e-2,
+           "small/bf16-cache": 2.2e-2, "mid/bf16-cache": 4.0e-2}
 
 
 def report(name, stats):
@@ -37,13 +39,15 @@ def report(name, stats):
     if not path:
         return
     keep = {k: (float(v) if isinstance(v, (np.floating, float)) else int(v) if isinstance(v, (np.integer, int)) else v)
-            for k, v in stats.items() if k != "tokens"}
+            for k, v in stats.items() if k not in ("tokens", "worst_by_step")}
+    wb = stats.get("worst_by_step") or []
+    keep["worst_at_steps"] = {str(i): round(float(max(wb[:i + 1])), 5) for i in (0, 15, 63, 127, 255, 511, len(wb) - 1) if i < len(wb)}
     with open(path, "a") as f:
         f.write(json.dumps({"run": name, **keep}) + "\n")
 
 
 def teacher_forced(name, shape, W, model, prompts, gen, sampling=None, sample_idx=None, check_state=True,
-                   run_to_ctx_end=False):
+                   run_to_ctx_end=False, state_tol=None, logit_tol=None):
     """Prefill + `gen` selections. The oracle free-runs; the device consumes the ORACLE's tokens (teacher
     forcing), so one early disagreement cannot cascade. Logits are compared at every step, the cache at the
     end. With run_to_ctx_end the last position of the context is consumed as well and the call after it
@@ -64,13 +68,15 @@ def teacher_forced(name, shape, W, model, prompts, gen, sampling=None, sample_id
     st = model.new_state(B)
     ws = model.new_workspace(B, n, prefill_samples=B)
     tol = TOL[shape.dtype]
+    ltol = tol if logit_tol is None else logit_tol
     first, lg = model.prefill(st, torch.from_numpy(prompts).to(DEV), samp, ws, want_logits=True)
     s = dict(rows=0, thin=0, guarded=0, strict=0, strict_mismatches=0, plain_mismatches=0, worst=0.0, eps_max=0.0,
-             in_situ_checked=0, in_situ_edge=0, stable=0, stable_mismatches=0)
+             in_situ_checked=0, in_situ_edge=0, stable=0, stable_mismatches=0, worst_by_step=[])
     tok_g = first.cpu().numpy()
     for k in range(gen):
         lg_np = lg.cpu().numpy()
-        s["worst"] = max(s["worst"], rel_err_rows(lg_np, logits_o[k]))
+        s["worst_by_step"].append(rel_err_rows(lg_np, logits_o[k]))
+        s["worst"] = max(s["worst"], s["worst_by_step"][-1])
         eps_row = np.max(np.abs(lg_np - logits_o[k]), axis=-1)
         s["eps_max"] = max(s["eps_max"], float(eps_row.max()))
         s["rows"] += B
@@ -117,7 +123,7 @@ def teacher_forced(name, shape, W, model, prompts, gen, sampling=None, sample_id
         # the oracle's final state corresponds to the same consumed tokens
         cache = st.cache().cpu().numpy()
         s["cache_err"] = rel_err_rows(cache, state_o)
-        assert s["cache_err"] < tol, f"cache rel err {s['cache_err']}"
+        assert s["cache_err"] < (tol if state_tol is None else state_tol), f"cache rel err {s['cache_err']}"
     if run_to_ctx_end:
         assert st.pos == shape.n_ctx - 1
         tok_in = torch.from_numpy(toks_o[:, gen - 1].copy()).to(DEV)
@@ -131,7 +137,7 @@ def teacher_forced(name, shape, W, model, prompts, gen, sampling=None, sample_id
         except P.SRMError as e:
             assert e.code == P.ERR_CTX_OVERFLOW, e
         assert st.pos == shape.n_ctx
-    assert s["worst"] < tol, f"logits rel err {s['worst']}"
+    assert s["worst"] < ltol, f"logits rel err {s['worst']}"
     assert s["eps_max"] <= EPS_ABS[name], (name, s["eps_max"])
     assert s["strict_mismatches"] == 0 and s["stable_mismatches"] == 0, s
     s["tokens"] = toks_o

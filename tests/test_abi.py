@@ -59,7 +59,8 @@ def test_size_queries_and_layout():
     assert lib.srm_weights_bytes(C.byref(cb)) < total
     # state: one d-vector per layer per sample (+ header and last-token vector)
     s1, s2 = lib.srm_state_bytes(C.byref(c), 1000), lib.srm_state_bytes(C.byref(c), 2000)
-    assert s2 - s1 == 1000 * (2 * 64 * 4) + 2 * 4096        # cache rows + last-token and position vectors (4000 -> 4096, 8000 -> 8192 each)
+    # cache rows + last-token, position and top-k threshold vectors (4000 -> 4096, 8000 -> 8192 bytes each)
+    assert s2 - s1 == 1000 * (2 * 64 * 4) + 3 * 4096
     assert lib.srm_workspace_bytes(C.byref(c), 8, 0) < lib.srm_workspace_bytes(C.byref(c), 16, 0)
 
 

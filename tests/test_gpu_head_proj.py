@@ -32,8 +32,9 @@ def test_bf16_with_head_projections_parity_subset(state_dtype):
     shape = I.SRMShape(n_layers=4, d_model=512, vocab=8000, n_ctx=128, dtype="bf16", seed=21, head_proj=True)
     W, model = _build(shape, state_dtype=state_dtype)
     prompts = I.uniform_prompts(12, 50, shape.vocab, seed=8)      # 50 positions: six full tiles and a ragged one
-    r = teacher_forced("small", shape, W, model, prompts, 6)      # (error bound of the small configuration)
-    assert_greedy_coverage(r, 0.05)
+    # (error bound of the small configuration; 72 decisions: a handful of guarded ones is a large share)
+    r = teacher_forced("small" if state_dtype == "fp32" else "small/bf16-cache", shape, W, model, prompts, 6)
+    assert_greedy_coverage(r, 0.12)
 
 
 def test_head_projection_prefill_equals_decode_on_device_and_chunking():

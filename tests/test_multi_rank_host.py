@@ -54,3 +54,26 @@ def test_single_rank_is_the_identity():
     assert bench.max_over_ranks(12.5, 1) == 12.5
     assert bench.rank_plan(0, 1, 7) == {"sample_idx_base": 0, "first_sample": 0, "last_sample": 6, "total_samples": 7}
     assert bench.whole_job_value(1, 100, 3, 1.0) == 300000.0
+
+
+def test_bench_starts_its_own_ranks_when_no_launcher_did():
+    """`python bench.py --gpus 2` with WORLD_SIZE unset starts two local ranks itself. On a box without a GPU
+    both ranks must stop with the no-CUDA message (there is no CPU fallback) and the command must fail, rather
+    than one rank running silently as a 1-GPU job."""
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    env["CUDA_VISIBLE_DEVICES"] = ""
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--steps", "1", "--warmup", "0"],
+                         capture_output=True, text=True, timeout=300, env=env)
+    assert res.returncode != 0
+    text = res.stdout + res.stderr
+    assert "rank 0: bench.py needs a CUDA device" in text and "rank 1: bench.py needs a CUDA device" in text
+    assert '"n_gpus"' not in res.stdout                    # no result line was printed
+
+
+def test_a_rank_count_that_contradicts_the_flag_is_refused():
+    import subprocess
+    env = dict(os.environ, WORLD_SIZE="1", RANK="0", LOCAL_RANK="0", CUDA_VISIBLE_DEVICES="")
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--steps", "1"],
+                         capture_output=True, text=True, timeout=300, env=env)
+    assert res.returncode != 0 and "--gpus 2 but the launcher started 1 rank" in res.stderr
