@@ -363,7 +363,7 @@ def run_ours(args):
     chunk = min(B, args.chunk)
     st = model.new_state(B)
     ws = model.new_workspace(chunk, n, prefill_samples=max(1, min(B, args.prefill_rows // n)))
-    sbytes = 2 if args.state_dtype == "bf16" else 4
+    sbytes = 4 if args.state_dtype == "fp32" else 2
 
     def sync_all():
         torch.cuda.synchronize()
@@ -595,7 +595,7 @@ def run_sweep(args):
     W = I.make_weights(shape)
     model = P.SRM(shape, W, device=dev, state_dtype=args.state_dtype)
     g = P.Sampling("greedy")
-    sbytes = 2 if args.state_dtype == "bf16" else 4
+    sbytes = 4 if args.state_dtype == "fp32" else 2
     L, d = shape.n_layers, shape.d_model
     chunk = args.chunk
     ws = model.new_workspace(chunk, w["prompt_len"], prefill_samples=max(1, args.prefill_rows // w["prompt_len"]))
@@ -730,7 +730,7 @@ def main():
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch per GPU")
     ap.add_argument("--chunk", type=int, default=8192, help="samples per decode pass (workspace size)")
     ap.add_argument("--prefill-rows", type=int, default=524288, help="prompt rows per prefill pass")
-    ap.add_argument("--state-dtype", default="fp32", choices=["fp32", "bf16"])
+    ap.add_argument("--state-dtype", default="fp32", choices=["fp32", "fp16", "bf16"])
     ap.add_argument("--ref-samples", type=int, default=32)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--head-proj", action="store_true",

@@ -57,7 +57,7 @@ enum srm_status_bits {
   SRM_STATUS_NONFINITE = 4u          /* the sampler met a non-finite logit                 */
 };
 
-enum { SRM_DTYPE_FP32 = 0, SRM_DTYPE_BF16 = 1 };
+enum { SRM_DTYPE_FP32 = 0, SRM_DTYPE_BF16 = 1, SRM_DTYPE_FP16 = 2 /* cache storage only */ };
 enum { SRM_SELECT_GREEDY = 0, SRM_SELECT_TOPK = 1, SRM_SELECT_TOPP = 2 };
 enum {
   SRM_FLAG_NO_GRAPH = 4,             /* srm_generate never replays a captured step                     */
@@ -86,7 +86,12 @@ typedef struct {
   int32_t dtype;         /* SRM_DTYPE_FP32: fp32 weights, plain fp32 FMA everywhere;
                             SRM_DTYPE_BF16: bf16 matrices and GEMM inputs, fp32 accumulate,
                             fp32 residual stream, norms and mixer arithmetic              */
-  int32_t state_dtype;   /* storage type of the cache: SRM_DTYPE_FP32 or SRM_DTYPE_BF16    */
+  int32_t state_dtype;   /* storage type of the cache [Method/Architecture: the cache may be kept in half
+                            precision]: SRM_DTYPE_FP32; SRM_DTYPE_FP16 (half the bytes per sample; values are
+                            clamped to +-65504 when stored); SRM_DTYPE_BF16 (half the bytes; 8 significant bits:
+                            in a decay-free head the rounding errors add up as a random walk, about 2^-9 sqrt(t)
+                            of the cache after t steps, which leaves the bf16 logit tolerance after a few hundred
+                            positions; for short contexts only)                           */
   float   ln_eps;        /* LayerNorm epsilon                                             */
   int32_t flags;         /* SRM_FLAG_* (0 in production)                                  */
 } srm_config;

@@ -391,9 +391,15 @@ class SRMOracle:
     of numpy arrays with those names works); all arithmetic runs in `dtype`."""
 
     def __init__(self, n_layers, d_model, vocab, n_ctx, W, n_heads=4, ln_eps=1e-5,
-                 dtype=np.float64):
+                 dtype=np.float64, mixer="mixed", kernel_size=1):
+        """mixer: "mixed" (Eq. 2 / Eq. 3 heads side by side; cache [L, B, d]), "combined" (every head holds a
+        row-repeat and a column-repeat matrix, outputs linearly combined; cache [L, 2, B, d]) or "kernel"
+        (Eq. 11 with kernel_size filters; cache [L, k, B, d]). Head projections go with "mixed" only."""
         self.L, self.d, self.V, self.n_ctx, self.h = n_layers, d_model, vocab, n_ctx, n_heads
         self.eps, self.dt = ln_eps, dtype
+        assert mixer in ("mixed", "combined", "kernel")
+        self.mixer, self.k = mixer, kernel_size
+        self.C = {"mixed": 1, "combined": 2, "kernel": kernel_size}[mixer]     # d-vectors of cache per layer and sample
         cv = lambda a: np.asarray(a, dtype=dtype)
         self.E, self.W_lm = cv(W["E"]), cv(W["W_lm"])
         self.lnf_g, self.lnf_b = cv(W["lnf_g"]), cv(W["lnf_b"])
@@ -408,15 +414,23 @@ class SRMOracle:
         B, n = tokens.shape
         assert n <= self.n_ctx
         x = self.E[tokens]                                   # [B, n, d]; no positional embedding
-        state = np.zeros((self.L, B, self.d), dtype=self.dt)
+        state = self.init_state(B)
         xs = []
         for l, lw in enumerate(self.layers):
             z = layer_norm(x, lw["ln1_g"], lw["ln1_b"], self.eps)
             y = np.empty_like(z)
-            Ms = [mixing_matrix(kind, lw["alpha"][g], lw["lam"][g], n, dtype=self.dt)
-                  for g, kind in enumerate(head_kinds(self.h))]
-            for b in range(B):
-                y[b], state[l, b] = token_mixer_parallel(z[b], lw, self.h, Ms)
+            if self.mixer == "combined":
+                for b in range(B):
+                    y[b], state[l, 0, b], state[l, 1, b] = combined_parallel(
+                        z[b], lw["alpha"], lw["alpha_col"], lw["beta"], lw["lam"], lw["lam_col"], lw["w_comb"], self.h)
+            elif self.mixer == "kernel":
+                for b in range(B):
+                    y[b], state[l, :, b] = kernel_parallel(z[b], lw["alpha"], lw["beta"], lw["lam"], self.k)
+            else:
+                Ms = [mixing_matrix(kind, lw["alpha"][g], lw["lam"][g], n, dtype=self.dt)
+                      for g, kind in enumerate(head_kinds(self.h))]
+                for b in range(B):
+                    y[b], state[l, b] = token_mixer_parallel(z[b], lw, self.h, Ms)
             x = x + y
             a = layer_norm(x, lw["ln2_g"], lw["ln2_b"], self.eps)
             x = x + feed_forward(a, lw["W1"], lw["b1"], lw["W2"], lw["b2"])
@@ -427,7 +441,9 @@ class SRMOracle:
 
     # -- recurrent form ----------------------------------------------------------------
     def init_state(self, B: int) -> np.ndarray:
-        return np.zeros((self.L, B, self.d), dtype=self.dt)
+        if self.mixer == "mixed":
+            return np.zeros((self.L, B, self.d), dtype=self.dt)
+        return np.zeros((self.L, self.C, B, self.d), dtype=self.dt)
 
     def decode_step(self, state: np.ndarray, tok: np.ndarray, pos: int, keep_x: bool = False):
         """Consume tok[B] at absolute position `pos`: returns logits[B, V] (predicting
@@ -438,7 +454,14 @@ class SRMOracle:
         xs = []
         for l, lw in enumerate(self.layers):
             z = layer_norm(x, lw["ln1_g"], lw["ln1_b"], self.eps)
-            y, new_state[l] = token_mixer_recurrent(z, state[l], pos, lw, self.h)
+            if self.mixer == "combined":
+                y, new_state[l, 0], new_state[l, 1] = combined_recurrent_step(
+                    z, state[l, 0], state[l, 1], pos, lw["alpha"], lw["alpha_col"], lw["beta"], lw["lam"], lw["lam_col"],
+                    lw["w_comb"], self.h)
+            elif self.mixer == "kernel":
+                y, new_state[l] = kernel_recurrent_step(z, state[l], pos, lw["alpha"], lw["beta"], lw["lam"], self.k)
+            else:
+                y, new_state[l] = token_mixer_recurrent(z, state[l], pos, lw, self.h)
             x = x + y
             a = layer_norm(x, lw["ln2_g"], lw["ln2_b"], self.eps)
             x = x + feed_forward(a, lw["W1"], lw["b1"], lw["W2"], lw["b2"])

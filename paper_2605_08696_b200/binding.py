@@ -15,7 +15,7 @@ import torch
 from . import build as _build
 
 EPI_BIAS_GELU, EPI_BIAS_RESIDUAL, EPI_PLAIN = 0, 1, 2
-DTYPE_FP32, DTYPE_BF16 = 0, 1
+DTYPE_FP32, DTYPE_BF16, DTYPE_FP16 = 0, 1, 2
 FLAG_SIMT_GEMM = 1
 FLAG_HEAD_PROJ = 2
 FLAG_NO_GRAPH = 4
@@ -254,8 +254,8 @@ class SRMState:
         m = self.model
         ptr = _lib().srm_state_layer_ptr(self.handle, l)
         off = ptr - self.buf.data_ptr()
-        es = 2 if m.cfg.state_dtype == DTYPE_BF16 else 4
-        dt = torch.bfloat16 if es == 2 else torch.float32
+        es = 4 if m.cfg.state_dtype == DTYPE_FP32 else 2
+        dt = {DTYPE_FP32: torch.float32, DTYPE_BF16: torch.bfloat16, DTYPE_FP16: torch.float16}[m.cfg.state_dtype]
         n = self.B * m.cfg.d_model
         return self.buf[off: off + n * es].view(dt).view(self.B, m.cfg.d_model)
 
@@ -290,7 +290,7 @@ class SRM:
         self.cfg = _Config(_shape_get(shape, "n_layers"), _shape_get(shape, "d_model"), _shape_get(shape, "n_heads"),
                            _shape_get(shape, "ffn_mult"), _shape_get(shape, "vocab"), _shape_get(shape, "n_ctx"),
                            DTYPE_BF16 if dt == "bf16" else DTYPE_FP32,
-                           DTYPE_BF16 if state_dtype == "bf16" else DTYPE_FP32,
+                           {"fp32": DTYPE_FP32, "bf16": DTYPE_BF16, "fp16": DTYPE_FP16}[state_dtype],
                            _shape_get(shape, "ln_eps"), flags)
         self.device = torch.device(device)
         self.act_dtype = torch.bfloat16 if dt == "bf16" else torch.float32

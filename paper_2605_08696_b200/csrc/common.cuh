@@ -2,12 +2,14 @@
 #pragma once
 
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
 namespace srm {
 
 typedef __nv_bfloat16 bf16;
+typedef __half fp16;                 // cache storage only: values are clamped to the finite fp16 range when stored
 
 constexpr uint32_t kStatusTokenRange = 1u;
 constexpr uint32_t kStatusWaitTimeout = 2u;
@@ -57,6 +59,20 @@ __device__ __forceinline__ void st4(bf16* p, float4 v) {
   u.y = *reinterpret_cast<uint32_t*>(&b);
   *reinterpret_cast<uint2*>(p) = u;
 }
+__device__ __forceinline__ float4 ld4(const fp16* p) {
+  uint2 u = *reinterpret_cast<const uint2*>(p);
+  const float2 fa = __half22float2(*reinterpret_cast<__half2*>(&u.x)), fb = __half22float2(*reinterpret_cast<__half2*>(&u.y));
+  return make_float4(fa.x, fa.y, fb.x, fb.y);
+}
+__device__ __forceinline__ float clamp_fp16(float v) { return fminf(fmaxf(v, -65504.0f), 65504.0f); }
+__device__ __forceinline__ void st4(fp16* p, float4 v) {
+  __half2 a = __floats2half2_rn(clamp_fp16(v.x), clamp_fp16(v.y));
+  __half2 b = __floats2half2_rn(clamp_fp16(v.z), clamp_fp16(v.w));
+  uint2 u;
+  u.x = *reinterpret_cast<uint32_t*>(&a);
+  u.y = *reinterpret_cast<uint32_t*>(&b);
+  *reinterpret_cast<uint2*>(p) = u;
+}
 // read-only (parameter) variants
 __device__ __forceinline__ float4 ldg4(const float* p) { return __ldg(reinterpret_cast<const float4*>(p)); }
 __device__ __forceinline__ float4 ldg4(const bf16* p) {
@@ -69,9 +85,11 @@ __device__ __forceinline__ float4 ldg4(const bf16* p) {
 
 __device__ __forceinline__ float to_float(float v) { return v; }
 __device__ __forceinline__ float to_float(bf16 v) { return __bfloat162float(v); }
+__device__ __forceinline__ float to_float(fp16 v) { return __half2float(v); }
 template <typename T> __device__ __forceinline__ T from_float(float v);
 template <> __device__ __forceinline__ float from_float<float>(float v) { return v; }
 template <> __device__ __forceinline__ bf16 from_float<bf16>(float v) { return __float2bfloat16_rn(v); }
+template <> __device__ __forceinline__ fp16 from_float<fp16>(float v) { return __float2half_rn(clamp_fp16(v)); }
 
 // exact (erf) GELU in fp32
 __device__ __forceinline__ float gelu_erf(float v) {

@@ -62,7 +62,7 @@ bool config_ok(const srm_config* c) {
   if (c->n_heads < 2 || c->n_heads > kPrefillMaxHeads || c->n_heads % 2 || c->d_model % (4 * c->n_heads)) return false;
   if (c->ffn_mult < 1 || c->vocab < 8 || c->vocab % 8 || c->n_ctx < 1) return false;
   if (c->dtype != SRM_DTYPE_FP32 && c->dtype != SRM_DTYPE_BF16) return false;
-  if (c->state_dtype != SRM_DTYPE_FP32 && c->state_dtype != SRM_DTYPE_BF16) return false;
+  if (c->state_dtype != SRM_DTYPE_FP32 && c->state_dtype != SRM_DTYPE_BF16 && c->state_dtype != SRM_DTYPE_FP16) return false;
   if (!(c->ln_eps > 0.f)) return false;
   return true;
 }
@@ -208,7 +208,7 @@ struct srm_model {
   }
   const float* fptr(int layer, int t) const { return reinterpret_cast<const float*>(ptr(layer, t)); }
   int act_bytes() const { return cfg.dtype == SRM_DTYPE_BF16 ? 2 : 4; }
-  int state_bytes() const { return cfg.state_dtype == SRM_DTYPE_BF16 ? 2 : 4; }
+  int state_bytes() const { return cfg.state_dtype == SRM_DTYPE_FP32 ? 4 : 2; }
   int64_t F() const { return (int64_t)cfg.ffn_mult * cfg.d_model; }
 
   // Copies the descriptor out: the cache may reallocate or be cleared by a later insertion.
@@ -267,7 +267,7 @@ struct LaunchScope {
 constexpr size_t kStateHeader = 256;
 
 size_t state_bytes_for(const srm_config& c, int64_t B) {
-  const size_t sb = c.state_dtype == SRM_DTYPE_BF16 ? 2 : 4;
+  const size_t sb = c.state_dtype == SRM_DTYPE_FP32 ? 4 : 2;
   return kStateHeader + 3 * align_up((size_t)B * 4, 256) + (size_t)c.n_layers * B * c.d_model * sb;
 }
 
@@ -359,6 +359,17 @@ cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_
   return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
 
+// Calls f(WT{}, ST{}) with the weight / activation type and the cache storage type of the configuration.
+template <typename F>
+int dispatch_types(const srm_config& c, F&& f) {
+  const bool wb = c.dtype == SRM_DTYPE_BF16;
+  switch (c.state_dtype) {
+    case SRM_DTYPE_BF16: return wb ? f(bf16{}, bf16{}) : f(float{}, bf16{});
+    case SRM_DTYPE_FP16: return wb ? f(bf16{}, fp16{}) : f(float{}, fp16{});
+    default: return wb ? f(bf16{}, float{}) : f(float{}, float{});
+  }
+}
+
 template <int NV, typename WT, typename ST>
 int launch_mixer_stream(const MixerParams& p, int num_sms, cudaStream_t st) {
   const int warps = mixer_stream_warps(p.d, (int)sizeof(ST));
@@ -402,11 +413,7 @@ int launch_mixer(const srm_model& m, int layer, int t, int64_t R, const int32_t*
   p.alpha = m.fptr(layer, SRM_T_ALPHA); p.beta = m.fptr(layer, SRM_T_BETA); p.lam = m.fptr(layer, SRM_T_LAMBDA);
   p.R = R; p.d = m.cfg.d_model; p.h = m.cfg.n_heads; p.n_ctx = m.cfg.n_ctx; p.t = t; p.vocab = m.cfg.vocab;
   p.eps = m.cfg.ln_eps; p.status = status; p.ctr = ctr; p.pos = pos;
-  const bool wb = m.cfg.dtype == SRM_DTYPE_BF16, sb = m.cfg.state_dtype == SRM_DTYPE_BF16;
-  if (wb && sb) return launch_mixer_nv<bf16, bf16>(p, m.num_sms, st);
-  if (wb) return launch_mixer_nv<bf16, float>(p, m.num_sms, st);
-  if (sb) return launch_mixer_nv<float, bf16>(p, m.num_sms, st);
-  return launch_mixer_nv<float, float>(p, m.num_sms, st);
+  return dispatch_types(m.cfg, [&](auto w, auto c) { return launch_mixer_nv<decltype(w), decltype(c)>(p, m.num_sms, st); });
 }
 
 template <typename WT>
@@ -739,14 +746,10 @@ int launch_prefill_mixer(const srm_model& m, int layer, int64_t Bp, int n, const
   p.Bp = Bp; p.n = n; p.d = m.cfg.d_model; p.h = m.cfg.n_heads; p.n_ctx = m.cfg.n_ctx; p.vocab = m.cfg.vocab;
   p.eps = m.cfg.ln_eps; p.status = status; p.len = len;
   const size_t smem = (size_t)kPrefillTile * m.cfg.d_model * 4;
-  const bool wb = m.cfg.dtype == SRM_DTYPE_BF16, sb = m.cfg.state_dtype == SRM_DTYPE_BF16;
   const int nv = p.d / 128;
   const bool scan_shape = p.d % 128 == 0 && (p.d / p.h) % 128 == 0 && p.h <= 8 && (nv == 4 || nv == 8 || nv == 12 || nv == 16);
   if (scan_shape && Bp >= kPrefillScanMinSamples) {        // many prompts: one warp walks each prompt's positions
-    if (wb && sb) return launch_prefill_scan_nv<bf16, bf16>(p, m.num_sms, st);
-    if (wb) return launch_prefill_scan_nv<bf16, float>(p, m.num_sms, st);
-    if (sb) return launch_prefill_scan_nv<float, bf16>(p, m.num_sms, st);
-    return launch_prefill_scan_nv<float, float>(p, m.num_sms, st);
+    return dispatch_types(m.cfg, [&](auto w, auto c) { return launch_prefill_scan_nv<decltype(w), decltype(c)>(p, m.num_sms, st); });
   }
   auto go = [&](auto kernel) -> int {
     SRM_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));   // smem depends on d: set per launch
@@ -754,10 +757,7 @@ int launch_prefill_mixer(const srm_model& m, int layer, int64_t Bp, int n, const
     SRM_CUDA(cudaGetLastError());
     return SRM_OK;
   };
-  if (wb && sb) return go(prefill_mixer_kernel<bf16, bf16>);
-  if (wb) return go(prefill_mixer_kernel<bf16, float>);
-  if (sb) return go(prefill_mixer_kernel<float, bf16>);
-  return go(prefill_mixer_kernel<float, float>);
+  return dispatch_types(m.cfg, [&](auto w, auto c) { return go(prefill_mixer_kernel<decltype(w), decltype(c)>); });
 }
 
 // Token-mixing block with head projections (Eq. 10) on `rows` rows of the residual stream:
@@ -779,7 +779,7 @@ int launch_mixer_block_proj(srm_model& m, int layer, int t, int64_t rows, int64_
   const srm_config& c = m.cfg;
   const int d = c.d_model;
   const bool prefill = t < 0;
-  const bool wb = c.dtype == SRM_DTYPE_BF16, sb = c.state_dtype == SRM_DTYPE_BF16;
+  const bool wb = c.dtype == SRM_DTYPE_BF16;
   int rc;
   if (tok != nullptr) {
     LaunchScope scope(m, prefill ? SRM_KERNEL_PREFILL_MIXER : SRM_KERNEL_MIXER, st);
@@ -801,10 +801,7 @@ int launch_mixer_block_proj(srm_model& m, int layer, int t, int64_t rows, int64_
     p.pos = pos;                                   // decode: per-row positions; prefill: prompt lengths
     p.status = status;
     const int64_t vecs = p.R * (d / 4);
-    if (wb && sb) rc = launch_mix_proj_t<bf16, bf16>(prefill, p, vecs, st);
-    else if (wb) rc = launch_mix_proj_t<bf16, float>(prefill, p, vecs, st);
-    else if (sb) rc = launch_mix_proj_t<float, bf16>(prefill, p, vecs, st);
-    else rc = launch_mix_proj_t<float, float>(prefill, p, vecs, st);
+    rc = dispatch_types(c, [&](auto w, auto cs) { return launch_mix_proj_t<decltype(w), decltype(cs)>(prefill, p, vecs, st); });
     if (rc) return rc;
   }
   if ((rc = launch_gemm(m, kEpiBiasResidual, rows, d, d, a, m.ptr(layer, SRM_T_W_OUT), nullptr, x, status, st, SRM_KERNEL_GEMM_PROJ))) return rc;

@@ -30,6 +30,9 @@ class SRMShape:
     seed: int = 0
     ln_eps: float = 1e-5
     head_proj: bool = False    # per-head input projections I_h (stacked: W_in[d,d]) and output projection W_out[d,d]
+    mixer: str = "mixed"       # "mixed" (half row-repeat, half column-repeat heads), "combined" (every head holds both
+                               # matrices, outputs linearly combined, twice the cache) or "kernel" (kernel_size filters)
+    kernel_size: int = 1       # number of column-repeat filters of the "kernel" mixer (Eq. 11)
 
     @property
     def d_ffn(self) -> int:
@@ -107,6 +110,19 @@ def make_weights(shape: SRMShape, *, std: float = 0.02, alpha_std: float | None 
             "ln2_g": (1.0 + nrm(d)).astype(np.float32), "ln2_b": nrm(d),
             "W1": mat(F, d), "b1": nrm(F), "W2": mat(d, F), "b2": nrm(d),
         })
+        lw = W["layers"][-1]
+        if shape.mixer == "combined":      # second set of repeated weights and decays, and the combination weights
+            lam_c = rng.uniform(lam_lo, 1.0, size=h).astype(np.float32)
+            lam_c[-1] = 1.0
+            lw["alpha_col"] = nrm(h, n, sd=a_std)
+            lw["lam_col"] = lam_c
+            lw["w_comb"] = (0.5 + 0.5 * rng.random(size=(h, 2))).astype(np.float32)
+        elif shape.mixer == "kernel":      # k filters instead of h heads
+            k = shape.kernel_size
+            lam_k = rng.uniform(lam_lo, 1.0, size=k).astype(np.float32)
+            lam_k[0] = 1.0
+            lw["alpha"] = nrm(k, n, sd=a_std)
+            lw["lam"] = lam_k
         if shape.head_proj:        # drawn last, so the tensors above do not depend on the switch within a layer
             W["layers"][-1]["W_in"] = mat(d, d)
             W["layers"][-1]["W_out"] = mat(d, d)

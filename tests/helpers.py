@@ -16,7 +16,8 @@ def weights_for(name: str):
 def oracle_for(shape, W, dtype=np.float64):
     from oracle import srm_oracle as O
     return O.SRMOracle(shape.n_layers, shape.d_model, shape.vocab, shape.n_ctx, W,
-                       n_heads=shape.n_heads, ln_eps=shape.ln_eps, dtype=dtype)
+                       n_heads=shape.n_heads, ln_eps=shape.ln_eps, dtype=dtype,
+                       mixer=shape.mixer, kernel_size=shape.kernel_size)
 
 
 def rel_err_rows(got, want) -> float:

@@ -107,3 +107,75 @@ def test_input_generators():
     assert np.array_equal(W1["E"], W2["E"])
     for lw in W1["layers"]:
         assert lw["lam"][0] == 1.0 and np.all(lw["lam"] > 0.9) and np.all(lw["lam"] <= 1.0)
+
+
+# ---- the model built from the further mixer variants (linearly combined heads; kernels of size k, Eq. 11) ----
+
+def _variant(mixer, k=1, alpha_std=0.4):
+    import dataclasses
+    shape = dataclasses.replace(I.CONFIGS["tiny"], mixer=mixer, kernel_size=k)
+    W = I.make_weights(shape, alpha_std=alpha_std)
+    return shape, W, O.SRMOracle(shape.n_layers, shape.d_model, shape.vocab, shape.n_ctx, W, n_heads=shape.n_heads,
+                                 ln_eps=shape.ln_eps, mixer=mixer, kernel_size=k)
+
+
+@pytest.mark.parametrize("mixer,k", [("combined", 1), ("kernel", 4), ("kernel", 8), ("kernel", 1)])
+def test_variant_model_parallel_equals_recurrent_and_is_causal(mixer, k):
+    """The model-level facts the mathematics fixes hold for the variant models too: the explicit n x n matrices
+    (the definition) and the recurrence give the same logits and the same cache to 1e-9 in fp64; a later token
+    cannot change an earlier output."""
+    shape, W, orc = _variant(mixer, k)
+    toks = I.uniform_prompts(3, 20, shape.vocab, seed=14)
+    lp, sp = orc.forward_parallel(toks)
+    lr, sr = orc.prefill_recurrent(toks)
+    C = {"combined": 2, "kernel": k}[mixer]
+    assert sp.shape == (shape.n_layers, C, 3, shape.d_model) and sr.shape == sp.shape
+    assert np.max(np.abs(lp - lr)) < 1e-9 and np.max(np.abs(sp - sr)) < 1e-9
+    alt = toks.copy()
+    alt[:, 9] = (alt[:, 9] + 1) % shape.vocab
+    out, _ = orc.forward_parallel(alt)
+    assert np.array_equal(out[:, :9], lp[:, :9]) and np.max(np.abs(out[:, 9] - lp[:, 9])) > 0
+
+
+def test_combined_model_with_one_matrix_switched_off_per_head_is_the_mixed_model():
+    """Combination weights (1, 0) on the first half of the heads and (0, 1) on the second half leave exactly the
+    mixed-head model (row-repeat heads first, column-repeat heads second) with the matching parameters."""
+    shape, W, orc = _variant("combined")
+    h = shape.n_heads
+    Wm = {k: v for k, v in W.items() if k != "layers"}
+    Wm["layers"] = []
+    for lw in W["layers"]:
+        lw["w_comb"] = np.array([[1.0, 0.0]] * (h // 2) + [[0.0, 1.0]] * (h // 2), dtype=np.float32)
+        m = {k: v for k, v in lw.items() if k not in ("alpha_col", "lam_col", "w_comb")}
+        m["alpha"] = np.concatenate([lw["alpha"][:h // 2], lw["alpha_col"][h // 2:]])
+        m["lam"] = np.concatenate([lw["lam"][:h // 2], lw["lam_col"][h // 2:]])
+        Wm["layers"].append(m)
+    orc_c = O.SRMOracle(shape.n_layers, shape.d_model, shape.vocab, shape.n_ctx, W, mixer="combined")
+    orc_m = O.SRMOracle(shape.n_layers, shape.d_model, shape.vocab, shape.n_ctx, Wm)
+    toks = I.uniform_prompts(2, 12, shape.vocab, seed=15)
+    lc, sc = orc_c.forward_parallel(toks)
+    lm, sm = orc_m.forward_parallel(toks)
+    assert np.max(np.abs(lc - lm)) < 1e-12
+    dh = shape.d_model // h
+    half = (h // 2) * dh
+    assert np.max(np.abs(sc[:, 0, :, :half] - sm[:, :, :half])) < 1e-12       # row-repeat sum terms of the first heads
+    assert np.max(np.abs(sc[:, 1, :, half:] - sm[:, :, half:])) < 1e-12       # column-repeat sum terms of the others
+
+
+def test_kernel_model_of_size_one_is_a_model_of_column_repeat_heads():
+    """k = 1: Eq. 11 is a single column-repeat matrix over all channels, i.e. the mixed-head recurrence with every
+    head column-repeat and the same alpha, lambda: checked through Eq. 3's closed form on the first layer."""
+    shape, W, orc = _variant("kernel", 1)
+    toks = I.uniform_prompts(2, 10, shape.vocab, seed=16)
+    _, _, xs = orc.forward_parallel(toks, keep_x=True)
+    lw = orc.layers[0]
+    x0 = orc.E[toks]
+    z = O.layer_norm(x0, lw["ln1_g"], lw["ln1_b"], shape.ln_eps)
+    n = toks.shape[1]
+    y = np.zeros_like(z)
+    for j in range(n):                              # Eq. 3: y_j = alpha_j sum_{i <= j} lambda^(j - i) z_i + beta_j
+        acc = sum(lw["lam"][0] ** (j - i) * z[:, i] for i in range(j + 1))
+        y[:, j] = lw["alpha"][0][j] * acc + lw["beta"][j]
+    x1 = x0 + y
+    x1 = x1 + O.feed_forward(O.layer_norm(x1, lw["ln2_g"], lw["ln2_b"], shape.ln_eps), lw["W1"], lw["b1"], lw["W2"], lw["b2"])
+    assert np.max(np.abs(xs[0] - x1)) < 1e-10
