@@ -75,7 +75,22 @@ enum {
                                         Adds W_in, W_out [d, d] per layer to the blob and 4 L d^2 flop per token */
 };
 
-/* Model description. Heads g < n_heads/2 are row-repeat, the rest column-repeat. */
+/* Token mixer of the model [Method/Architecture].
+ *   SRM_MIXER_MIXED     mixed heads: heads g < n_heads/2 row-repeat [Eq. 2], the rest column-repeat [Eq. 3], outputs
+ *                       concatenated; the cache is d values per sample and layer (the default, and the hot path);
+ *   SRM_MIXER_COMBINED  linearly combined heads: every head holds one row-repeat and one column-repeat matrix and
+ *                       outputs w[g][0] * (row-repeat product) + w[g][1] * (column-repeat product) + beta; the cache
+ *                       is both sum terms, 2 d values ("double the cache");
+ *   SRM_MIXER_KERNEL    non-unitary kernels [Eq. 11]: kernel_size column-repeat filters over the whole hidden
+ *                       dimension, filter i reading the channels shifted by i (zero past the last channel); the
+ *                       cache is one sum term per filter, kernel_size * d values; alpha is [kernel_size, n_ctx] and
+ *                       lambda [kernel_size] (n_heads is not used by the mixing).
+ * The two further mixers run through fused step kernels of their own (warp per row); their sequence form is
+ * evaluated through the recurrence, one launch per position over all prompts of a pass. They take the cache in
+ * fp32 or fp16, d_model <= 1024, no head projections and no per-sample positions (srm_prefill_ragged). */
+enum { SRM_MIXER_MIXED = 0, SRM_MIXER_COMBINED = 1, SRM_MIXER_KERNEL = 2 };
+
+/* Model description. */
 typedef struct {
   int32_t n_layers;      /* L >= 1                                                        */
   int32_t d_model;       /* d, multiple of 64, <= 2048                                    */
@@ -94,6 +109,8 @@ typedef struct {
                             positions; for short contexts only)                           */
   float   ln_eps;        /* LayerNorm epsilon                                             */
   int32_t flags;         /* SRM_FLAG_* (0 in production)                                  */
+  int32_t mixer;         /* SRM_MIXER_*                                                   */
+  int32_t kernel_size;   /* SRM_MIXER_KERNEL: number of filters k, 1 <= k <= 16; else ignored */
 } srm_config;
 
 /* Token selection. Greedy: smallest id among the maxima. Top-k: keep the top_k largest logits
@@ -135,6 +152,10 @@ enum srm_tensor {
   SRM_T_W_IN,         /* [d, d]    per layer, only with SRM_FLAG_HEAD_PROJ: rows g*d_h.. are I_g; placed
                                    after B2 in the layer's part of the blob                          */
   SRM_T_W_OUT,        /* [d, d]    per layer, only with SRM_FLAG_HEAD_PROJ: P_out                   */
+  SRM_T_ALPHA_COL,    /* [h, n_ctx] SRM_MIXER_COMBINED only: weights of the column-repeat matrices (SRM_T_ALPHA then
+                                   holds those of the row-repeat matrices); placed after the tensors above        */
+  SRM_T_LAMBDA_COL,   /* [h]       SRM_MIXER_COMBINED only: decays of the column-repeat matrices                  */
+  SRM_T_W_COMB,       /* [h, 2]    SRM_MIXER_COMBINED only: combination weights (row-repeat, column-repeat)       */
   SRM_T_COUNT
 };
 
@@ -147,8 +168,10 @@ int srm_weight_slot(const srm_config* cfg, int32_t layer, int32_t tensor,
 /* Bytes of the state buffer for B samples: a 256-byte header (status word, counters), the
  * last selected token int32[B], the per-sample position int32[B] (used after srm_prefill_ragged), the
  * per-sample candidate threshold float[B] of the fused top-k selection, each rounded up to 256 bytes, then the
- * cache [L, B, d] in state_dtype. */
+ * cache [L, C, B, d] in state_dtype, C = srm_cache_planes(cfg). */
 size_t srm_state_bytes(const srm_config* cfg, int64_t B);
+/* d-vectors of cache per sample and layer: 1 (mixed heads), 2 (combined heads), kernel_size (kernels). 0: bad config. */
+int32_t srm_cache_planes(const srm_config* cfg);
 /* Workspace bytes so that decode processes `B_chunk` samples per pass and prefill handles
  * prompts of up to `n_prefill_max` tokens in one pass of at least one sample. Calls accept any
  * workspace at least this large for B_chunk = 1 and split the batch into as many passes as
@@ -182,7 +205,7 @@ int srm_state_set_pos(srm_state* s, int64_t pos);
 int srm_state_adopt_positions(srm_state* s, int64_t max_pos);
 /* 1 when the state keeps one position per sample (after srm_prefill_ragged or srm_state_adopt_positions). */
 int srm_state_is_ragged(const srm_state* s);
-/* Device address of the cache slab of one layer, [B, d] in state_dtype (for checkpointing
+/* Device address of the cache slab of one layer, [C, B, d] in state_dtype (for checkpointing
  * and tests), and of the last-token vector int32[B]. */
 void* srm_state_layer_ptr(const srm_state* s, int32_t layer);
 int32_t* srm_state_last_token_ptr(const srm_state* s);
@@ -300,7 +323,7 @@ int srm_decode_step_static(srm_model* m, srm_state* s, const int32_t* d_tok_in,
 /* Fused token-mixer step of one layer on R rows at position t [Eq. 2, Eq. 3]:
  *   x <- (d_tok != NULL ? E[tok] : x);  z = LN1(x);  y, S' = mixer(z, S, t);  x <- x + y;
  *   a = LN2(x) in the activation type of cfg.dtype.
- * d_x float[R, d] in/out, d_S [R, d] in state_dtype in/out, d_a [R, d] out. */
+ * d_x float[R, d] in/out, d_S [R, d] in state_dtype in/out ([C, R, d] for the further mixers), d_a [R, d] out. */
 int srm_k_mixer_step(srm_model* m, int32_t layer, int32_t t, int64_t R, const int32_t* d_tok,
                      float* d_x, void* d_S, void* d_a, uint32_t* d_status, void* stream);
 /* Recurrent step of a layer with LINEARLY COMBINED heads [Architecture: every head holds one row-repeat and

@@ -28,7 +28,8 @@ ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_BUFFER_TOO_SMALL, ERR_CTX_O
 
 # enum srm_tensor
 T_E, T_LN1_G, T_LN1_B, T_ALPHA, T_BETA, T_LAMBDA, T_LN2_G, T_LN2_B, T_W1, T_B1, T_W2, T_B2, \
-    T_LNF_G, T_LNF_B, T_W_LM, T_W_IN, T_W_OUT = range(17)
+    T_LNF_G, T_LNF_B, T_W_LM, T_W_IN, T_W_OUT, T_ALPHA_COL, T_LAMBDA_COL, T_W_COMB = range(20)
+MIXER_MIXED, MIXER_COMBINED, MIXER_KERNEL = 0, 1, 2
 _LAYER_TENSORS = {"ln1_g": T_LN1_G, "ln1_b": T_LN1_B, "alpha": T_ALPHA, "beta": T_BETA, "lam": T_LAMBDA,
                   "ln2_g": T_LN2_G, "ln2_b": T_LN2_B, "W1": T_W1, "b1": T_B1, "W2": T_W2, "b2": T_B2}
 _GLOBAL_TENSORS = {"E": T_E, "lnf_g": T_LNF_G, "lnf_b": T_LNF_B, "W_lm": T_W_LM}
@@ -46,7 +47,7 @@ class _Config(C.Structure):
     _fields_ = [("n_layers", C.c_int32), ("d_model", C.c_int32), ("n_heads", C.c_int32),
                 ("ffn_mult", C.c_int32), ("vocab", C.c_int32), ("n_ctx", C.c_int32),
                 ("dtype", C.c_int32), ("state_dtype", C.c_int32), ("ln_eps", C.c_float),
-                ("flags", C.c_int32)]
+                ("flags", C.c_int32), ("mixer", C.c_int32), ("kernel_size", C.c_int32)]
 
 
 class _Sampling(C.Structure):
@@ -76,6 +77,7 @@ SYMBOLS = {
     "srm_weights_bytes": (_SZ, [C.POINTER(_Config)]),
     "srm_weight_slot": (C.c_int, [C.POINTER(_Config), _I32, _I32, C.POINTER(_SZ), C.POINTER(_SZ), C.POINTER(_I32)]),
     "srm_state_bytes": (_SZ, [C.POINTER(_Config), _I64]),
+    "srm_cache_planes": (_I32, [C.POINTER(_Config)]),
     "srm_workspace_bytes": (_SZ, [C.POINTER(_Config), _I64, _I32]),
     "srm_create": (C.c_int, [C.POINTER(_Config), _P, _SZ, C.POINTER(_P)]),
     "srm_destroy": (C.c_int, [_P]),
@@ -164,6 +166,10 @@ def _stream():
     return C.c_void_p(torch.cuda.current_stream().cuda_stream)
 
 
+def _shape_opt(shape, key, default):
+    return shape.get(key, default) if isinstance(shape, dict) else getattr(shape, key, default)
+
+
 def _shape_get(shape, key):
     return shape[key] if isinstance(shape, dict) else getattr(shape, key)
 
@@ -250,17 +256,21 @@ class SRMState:
         return f.value
 
     def layer(self, l: int) -> torch.Tensor:
-        """View of the cache slab of one layer, [B, d] in the state dtype."""
+        """View of the cache slab of one layer in the state dtype: [B, d], or [C, B, d] for the mixers that keep
+        C > 1 d-vectors per sample and layer."""
         m = self.model
         ptr = _lib().srm_state_layer_ptr(self.handle, l)
         off = ptr - self.buf.data_ptr()
         es = 4 if m.cfg.state_dtype == DTYPE_FP32 else 2
         dt = {DTYPE_FP32: torch.float32, DTYPE_BF16: torch.bfloat16, DTYPE_FP16: torch.float16}[m.cfg.state_dtype]
-        n = self.B * m.cfg.d_model
-        return self.buf[off: off + n * es].view(dt).view(self.B, m.cfg.d_model)
+        n = m.planes * self.B * m.cfg.d_model
+        v = self.buf[off: off + n * es].view(dt)
+        if m.cfg.mixer == MIXER_MIXED:
+            return v.view(self.B, m.cfg.d_model)
+        return v.view(m.planes, self.B, m.cfg.d_model)
 
     def cache(self) -> torch.Tensor:
-        """[L, B, d] copy of the whole cache in fp32."""
+        """[L, B, d] (or [L, C, B, d]) copy of the whole cache in fp32."""
         return torch.stack([self.layer(l).float() for l in range(self.model.cfg.n_layers)])
 
     def topk_thresholds(self) -> torch.Tensor:
@@ -291,7 +301,10 @@ class SRM:
                            _shape_get(shape, "ffn_mult"), _shape_get(shape, "vocab"), _shape_get(shape, "n_ctx"),
                            DTYPE_BF16 if dt == "bf16" else DTYPE_FP32,
                            {"fp32": DTYPE_FP32, "bf16": DTYPE_BF16, "fp16": DTYPE_FP16}[state_dtype],
-                           _shape_get(shape, "ln_eps"), flags)
+                           _shape_get(shape, "ln_eps"), flags,
+                           {"mixed": MIXER_MIXED, "combined": MIXER_COMBINED, "kernel": MIXER_KERNEL}[_shape_opt(shape, "mixer", "mixed")],
+                           _shape_opt(shape, "kernel_size", 1))
+        self.planes = lib.srm_cache_planes(C.byref(self.cfg))
         self.device = torch.device(device)
         self.act_dtype = torch.bfloat16 if dt == "bf16" else torch.float32
         nbytes = lib.srm_weights_bytes(C.byref(self.cfg))
@@ -319,6 +332,10 @@ class SRM:
             if flags & FLAG_HEAD_PROJ:
                 put(l, T_W_IN, lw["W_in"])
                 put(l, T_W_OUT, lw["W_out"])
+            if self.cfg.mixer == MIXER_COMBINED:
+                put(l, T_ALPHA_COL, lw["alpha_col"])
+                put(l, T_LAMBDA_COL, lw["lam_col"])
+                put(l, T_W_COMB, lw["w_comb"])
         with torch.cuda.device(self.device):
             self.blob = host.to(self.device)
             self.handle = C.c_void_p()

@@ -23,6 +23,7 @@
 #include "mixer_stream.cuh"
 #include "mixer_proj.cuh"
 #include "mixer_variants.cuh"
+#include "mixer_model_variants.cuh"
 #include "prefill.cuh"
 #include "prefill_scan.cuh"
 #include "select.cuh"
@@ -64,16 +65,29 @@ bool config_ok(const srm_config* c) {
   if (c->dtype != SRM_DTYPE_FP32 && c->dtype != SRM_DTYPE_BF16) return false;
   if (c->state_dtype != SRM_DTYPE_FP32 && c->state_dtype != SRM_DTYPE_BF16 && c->state_dtype != SRM_DTYPE_FP16) return false;
   if (!(c->ln_eps > 0.f)) return false;
+  if (c->mixer != SRM_MIXER_MIXED && c->mixer != SRM_MIXER_COMBINED && c->mixer != SRM_MIXER_KERNEL) return false;
+  if (c->mixer != SRM_MIXER_MIXED) {
+    // the further mixers: no head projections, cache in fp32 or fp16, rows of at most 1024 channels
+    if ((c->flags & SRM_FLAG_HEAD_PROJ) || c->state_dtype == SRM_DTYPE_BF16 || c->d_model > 1024) return false;
+    if (c->mixer == SRM_MIXER_KERNEL && (c->kernel_size < 1 || c->kernel_size > 16 || c->kernel_size > c->d_model)) return false;
+  }
   return true;
 }
 
+// d-vectors of cache per sample and layer: 1 (mixed heads), 2 (combined heads: both sum terms), k (kernel of size k)
+int cache_planes(const srm_config& c) {
+  return c.mixer == SRM_MIXER_COMBINED ? 2 : c.mixer == SRM_MIXER_KERNEL ? c.kernel_size : 1;
+}
+
 size_t tensor_elems(const srm_config& c, int t) {
-  const size_t d = c.d_model, F = (size_t)c.ffn_mult * d, V = c.vocab, n = c.n_ctx, h = c.n_heads;
+  const size_t d = c.d_model, F = (size_t)c.ffn_mult * d, V = c.vocab, n = c.n_ctx;
+  const size_t h = c.mixer == SRM_MIXER_KERNEL ? (size_t)c.kernel_size : (size_t)c.n_heads;   // filters take the heads' place
   switch (t) {
     case SRM_T_E: case SRM_T_W_LM: return V * d;
-    case SRM_T_ALPHA: return h * n;
+    case SRM_T_ALPHA: case SRM_T_ALPHA_COL: return h * n;
     case SRM_T_BETA: return n * d;
-    case SRM_T_LAMBDA: return h;
+    case SRM_T_LAMBDA: case SRM_T_LAMBDA_COL: return h;
+    case SRM_T_W_COMB: return 2 * h;
     case SRM_T_W1: case SRM_T_W2: return F * d;
     case SRM_T_W_IN: case SRM_T_W_OUT: return d * d;
     case SRM_T_B1: return F;
@@ -105,6 +119,8 @@ Layout make_layout(const srm_config& c) {
       L.layer[(size_t)l * SRM_T_COUNT + SRM_T_W_IN] = place(SRM_T_W_IN);
       L.layer[(size_t)l * SRM_T_COUNT + SRM_T_W_OUT] = place(SRM_T_W_OUT);
     }
+    if (c.mixer == SRM_MIXER_COMBINED)
+      for (int t = SRM_T_ALPHA_COL; t <= SRM_T_W_COMB; ++t) L.layer[(size_t)l * SRM_T_COUNT + t] = place(t);
   }
   L.global[SRM_T_LNF_G] = place(SRM_T_LNF_G);
   L.global[SRM_T_LNF_B] = place(SRM_T_LNF_B);
@@ -241,7 +257,10 @@ struct srm_state {
   int64_t pos;            // position of the next token (ragged: of the longest sample)
   bool ragged = false;    // samples have their own positions (pos_dev)
 
-  void* layer_ptr(int l) const { return S + (size_t)l * B * m->cfg.d_model * m->state_bytes(); }
+  // Layer l: planes() consecutive slabs [B, d] (plane_elems() elements apart)
+  int planes() const { return cache_planes(m->cfg); }
+  int64_t plane_elems() const { return B * (int64_t)m->cfg.d_model; }
+  void* layer_ptr(int l) const { return S + (size_t)l * planes() * B * m->cfg.d_model * m->state_bytes(); }
 };
 
 namespace {
@@ -268,7 +287,7 @@ constexpr size_t kStateHeader = 256;
 
 size_t state_bytes_for(const srm_config& c, int64_t B) {
   const size_t sb = c.state_dtype == SRM_DTYPE_FP32 ? 4 : 2;
-  return kStateHeader + 3 * align_up((size_t)B * 4, 256) + (size_t)c.n_layers * B * c.d_model * sb;
+  return kStateHeader + 3 * align_up((size_t)B * 4, 256) + (size_t)c.n_layers * cache_planes(c) * B * c.d_model * sb;
 }
 
 // ---- workspace carving ----------------------------------------------------------------------
@@ -414,6 +433,49 @@ int launch_mixer(const srm_model& m, int layer, int t, int64_t R, const int32_t*
   p.R = R; p.d = m.cfg.d_model; p.h = m.cfg.n_heads; p.n_ctx = m.cfg.n_ctx; p.t = t; p.vocab = m.cfg.vocab;
   p.eps = m.cfg.ln_eps; p.status = status; p.ctr = ctr; p.pos = pos;
   return dispatch_types(m.cfg, [&](auto w, auto c) { return launch_mixer_nv<decltype(w), decltype(c)>(p, m.num_sms, st); });
+}
+
+// Fused step of the combined-head / kernel-size-k mixers on R rows at position t (mixer_model_variants.cuh).
+// S: plane 0 of the rows' cache, planes `plane` elements apart; x, a rows x_stride elements apart.
+template <typename WT, typename ST>
+int launch_mixer_variant_t(const VariantParams& p, bool kernel_mix, cudaStream_t st) {
+  const unsigned grid = (unsigned)((p.R + kMixerWarps - 1) / kMixerWarps);
+  const dim3 blk(kMixerWarps * 32);
+  const int nv = (p.d + 127) / 128;
+#define SRM_VARIANT_LAUNCH(NV)                                                                                          \
+  do {                                                                                                                  \
+    if (kernel_mix) SRM_CUDA(launch_kernel(mixer_variant_step_kernel<NV, WT, ST, true>, dim3(grid), dim3(blk), 0, st, p)); \
+    else SRM_CUDA(launch_kernel(mixer_variant_step_kernel<NV, WT, ST, false>, dim3(grid), dim3(blk), 0, st, p));           \
+  } while (0)
+  if (nv <= 1) SRM_VARIANT_LAUNCH(1);
+  else if (nv <= 4) SRM_VARIANT_LAUNCH(4);
+  else SRM_VARIANT_LAUNCH(8);
+#undef SRM_VARIANT_LAUNCH
+  return SRM_OK;
+}
+
+int launch_mixer_variant(const srm_model& m, int layer, int t, int64_t R, const int32_t* tok, int64_t tok_stride, float* x,
+                         void* a, int64_t x_stride, void* S, int64_t plane, uint32_t* status, cudaStream_t st,
+                         const int32_t* ctr = nullptr, int cls = SRM_KERNEL_MIXER) {
+  if (R <= 0) return SRM_OK;
+  LaunchScope scope(m, cls, st);
+  const srm_config& c = m.cfg;
+  VariantParams p;
+  p.x = x; p.tok = tok; p.E = m.ptr(-1, SRM_T_E); p.S = S; p.a = a;
+  p.ln1_g = m.fptr(layer, SRM_T_LN1_G); p.ln1_b = m.fptr(layer, SRM_T_LN1_B);
+  p.ln2_g = m.fptr(layer, SRM_T_LN2_G); p.ln2_b = m.fptr(layer, SRM_T_LN2_B);
+  p.alpha = m.fptr(layer, SRM_T_ALPHA); p.beta = m.fptr(layer, SRM_T_BETA); p.lam = m.fptr(layer, SRM_T_LAMBDA);
+  const bool comb = c.mixer == SRM_MIXER_COMBINED;
+  p.alpha_col = comb ? m.fptr(layer, SRM_T_ALPHA_COL) : nullptr;
+  p.lam_col = comb ? m.fptr(layer, SRM_T_LAMBDA_COL) : nullptr;
+  p.w_comb = comb ? m.fptr(layer, SRM_T_W_COMB) : nullptr;
+  p.R = R; p.x_stride = x_stride; p.tok_stride = tok_stride; p.plane = plane;
+  p.d = c.d_model; p.h = c.n_heads; p.k = c.kernel_size; p.n_ctx = c.n_ctx; p.t = t; p.vocab = c.vocab;
+  p.eps = c.ln_eps; p.status = status; p.ctr = ctr;
+  const bool wb = c.dtype == SRM_DTYPE_BF16, half_cache = c.state_dtype == SRM_DTYPE_FP16;
+  const bool km = c.mixer == SRM_MIXER_KERNEL;
+  if (wb) return half_cache ? launch_mixer_variant_t<bf16, fp16>(p, km, st) : launch_mixer_variant_t<bf16, float>(p, km, st);
+  return half_cache ? launch_mixer_variant_t<float, fp16>(p, km, st) : launch_mixer_variant_t<float, float>(p, km, st);
 }
 
 template <typename WT>
@@ -829,7 +891,10 @@ int decode_chunk(srm_model& m, srm_state& s, int64_t b0, int64_t R, const int32_
   if (split) SRM_CUDA(cudaMemsetAsync(w.order, 0, w.order_bytes, st));
   for (int l = 0; l < c.n_layers; ++l) {
     uint8_t* Sl = static_cast<uint8_t*>(s.layer_ptr(l)) + (size_t)b0 * d * m.state_bytes();
-    if (m.head_proj()) {
+    if (c.mixer != SRM_MIXER_MIXED) {
+      if ((rc = launch_mixer_variant(m, l, t, R, l == 0 ? tok_in + b0 : nullptr, 1, w.x, w.a, d, Sl, s.plane_elems(), s.status,
+                                     st, ctr))) return rc;
+    } else if (m.head_proj()) {
       if ((rc = launch_mixer_block_proj(m, l, t, R, R, 1, l == 0 ? tok_in + b0 : nullptr, w.x, Sl, w.a, w.q, s.status, st, ctr, pos))) return rc;
     } else if ((rc = launch_mixer(m, l, t, R, l == 0 ? tok_in + b0 : nullptr, w.x, Sl, w.a, s.status, st, ctr, pos))) return rc;
     if ((rc = launch_gemm(m, kEpiBiasGelu, R, F, d, w.a, m.ptr(l, SRM_T_W1), m.fptr(l, SRM_T_B1), w.H, s.status, st))) return rc;
@@ -1070,6 +1135,8 @@ void* srm_state_layer_ptr(const srm_state* s, int32_t layer) {
 
 int32_t* srm_state_last_token_ptr(const srm_state* s) { return s ? s->last_tok : nullptr; }
 
+int32_t srm_cache_planes(const srm_config* cfg) { return config_ok(cfg) ? cache_planes(*cfg) : 0; }
+
 float* srm_state_topk_threshold_ptr(const srm_state* s) { return s ? s->thr : nullptr; }
 
 int srm_state_topk_handed_back(srm_state* s, void* stream, uint64_t* rows) {
@@ -1108,7 +1175,8 @@ int prefill_impl(srm_model* m, srm_state* s, const int32_t* d_tokens, int64_t P,
   const int d = c.d_model;
   const int64_t F = m->F();
   const size_t row_bytes = (size_t)d * m->state_bytes();
-  const size_t stage_per_prompt = replicas > 1 ? align_up((size_t)c.n_layers * row_bytes, 256) : 0;
+  const int planes = cache_planes(c);
+  const size_t stage_per_prompt = replicas > 1 ? align_up((size_t)c.n_layers * planes * row_bytes, 256) : 0;
   // largest number of prompts per pass whose workspace and staging both fit
   int64_t Bp = fit_rows(ws_bytes, P, prefill_need, *m, n);
   while (Bp >= 1 && prefill_ws_bytes(*m, Bp, n) + (size_t)Bp * stage_per_prompt > ws_bytes) --Bp;
@@ -1121,21 +1189,32 @@ int prefill_impl(srm_model* m, srm_state* s, const int32_t* d_tokens, int64_t P,
     const int64_t rows = np * n;
     const int64_t b0 = p0 * replicas, nb = np * replicas;          // state rows of this pass
     for (int l = 0; l < c.n_layers; ++l) {
-      uint8_t* Sl = replicas > 1 ? stage + (size_t)l * np * row_bytes
+      uint8_t* Sl = replicas > 1 ? stage + (size_t)l * planes * np * row_bytes
                                  : static_cast<uint8_t*>(s->layer_ptr(l)) + (size_t)b0 * row_bytes;
-      if (m->head_proj()) {
+      if (c.mixer != SRM_MIXER_MIXED) {
+        // the sequence form of these mixers through their recurrence: one launch per position over all prompts of the
+        // pass, the (zeroed) cache updated in place; rows of one prompt are n apart in x and a
+        const int64_t plane = replicas > 1 ? np * (int64_t)d : s->plane_elems();
+        for (int pl = 0; pl < planes; ++pl)          // the recurrence starts from an empty cache
+          SRM_CUDA(cudaMemsetAsync(Sl + (size_t)pl * plane * m->state_bytes(), 0, (size_t)np * row_bytes, st));
+        for (int t = 0; t < n; ++t)
+          if ((rc = launch_mixer_variant(*m, l, t, np, l == 0 ? d_tokens + p0 * n + t : nullptr, n, w.x + (size_t)t * d,
+                                         static_cast<uint8_t*>(w.a) + (size_t)t * d * m->act_bytes(), (int64_t)n * d, Sl, plane,
+                                         s->status, st, nullptr, SRM_KERNEL_PREFILL_MIXER))) return rc;
+      } else if (m->head_proj()) {
         if ((rc = launch_mixer_block_proj(*m, l, -1, rows, np, n, l == 0 ? d_tokens + p0 * n : nullptr, w.x, Sl, w.a, w.q, s->status, st,
                                           nullptr, d_len ? d_len + p0 : nullptr))) return rc;
       } else if ((rc = launch_prefill_mixer(*m, l, np, n, l == 0 ? d_tokens + p0 * n : nullptr, w.x, Sl, w.a, s->status, st,
                                             d_len ? d_len + p0 : nullptr))) return rc;
       if ((rc = launch_gemm(*m, kEpiBiasGelu, rows, F, d, w.a, m->ptr(l, SRM_T_W1), m->fptr(l, SRM_T_B1), w.H, s->status, st))) return rc;
       if ((rc = launch_gemm(*m, kEpiBiasResidual, rows, d, F, w.H, m->ptr(l, SRM_T_W2), m->fptr(l, SRM_T_B2), w.x, s->status, st))) return rc;
-      if (replicas > 1) {
+      for (int pl = 0; replicas > 1 && pl < planes; ++pl) {
         LaunchScope scope(*m, SRM_KERNEL_PREFILL_MIXER, st);
         const int64_t vpr = (int64_t)row_bytes / 16, total = nb * vpr;
-        uint8_t* dst = static_cast<uint8_t*>(s->layer_ptr(l)) + (size_t)b0 * row_bytes;
+        const uint8_t* src = Sl + (size_t)pl * np * row_bytes;
+        uint8_t* dst = static_cast<uint8_t*>(s->layer_ptr(l)) + ((size_t)pl * s->B + (size_t)b0) * row_bytes;
         SRM_CUDA(launch_kernel(broadcast_rows_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, st,
-                               reinterpret_cast<const uint4*>(Sl), reinterpret_cast<uint4*>(dst), np, replicas, vpr));
+                               reinterpret_cast<const uint4*>(src), reinterpret_cast<uint4*>(dst), np, replicas, vpr));
       }
     }
     // LM head on the last prompt position only; selection per state row
@@ -1191,6 +1270,7 @@ int srm_prefill_ragged(srm_model* m, srm_state* s, const int32_t* d_tokens, int3
   if (rc) return rc;
   if (d_lengths == nullptr) return SRM_ERR_INVALID_ARG;
   if (!aligned(d_lengths, 4)) return SRM_ERR_ALIGNMENT;
+  if (m->cfg.mixer != SRM_MIXER_MIXED) return SRM_ERR_UNSUPPORTED;      // one position per sample: mixed heads only
   return prefill_impl(m, s, d_tokens, s->B, n_max, 1, samp, d_first_tok, d_logits_last, d_ws, ws_bytes,
                       static_cast<cudaStream_t>(stream), d_lengths);
 }
@@ -1358,6 +1438,9 @@ int srm_k_mixer_step(srm_model* m, int32_t layer, int32_t t, int64_t R, const in
   if (layer < 0 || layer >= m->cfg.n_layers || t < 0) return SRM_ERR_INVALID_ARG;
   if (t >= m->cfg.n_ctx) return SRM_ERR_CTX_OVERFLOW;
   if (!aligned(d_x, 16) || !aligned(d_S, 16) || !aligned(d_a, 16)) return SRM_ERR_ALIGNMENT;
+  if (m->cfg.mixer != SRM_MIXER_MIXED)      // d_S: the planes [C][R, d] of these R rows
+    return launch_mixer_variant(*m, layer, t, R, d_tok, 1, d_x, d_a, m->cfg.d_model, d_S, R * (int64_t)m->cfg.d_model, d_status,
+                                static_cast<cudaStream_t>(stream));
   return launch_mixer(*m, layer, t, R, d_tok, d_x, d_S, d_a, d_status, static_cast<cudaStream_t>(stream));
 }
 
@@ -1556,6 +1639,7 @@ int srm_k_prefill_mixer(srm_model* m, int32_t layer, int64_t Bp, int32_t n, cons
   if (layer < 0 || layer >= m->cfg.n_layers) return SRM_ERR_INVALID_ARG;
   if (n > m->cfg.n_ctx) return SRM_ERR_CTX_OVERFLOW;
   if (!aligned(d_x, 16) || !aligned(d_S, 16) || !aligned(d_a, 16)) return SRM_ERR_ALIGNMENT;
+  if (m->cfg.mixer != SRM_MIXER_MIXED) return SRM_ERR_UNSUPPORTED;
   return launch_prefill_mixer(*m, layer, Bp, n, d_tok, d_x, d_S, d_a, d_status, static_cast<cudaStream_t>(stream));
 }
 

@@ -30,7 +30,7 @@ def test_every_declared_symbol_is_exported_and_bound():
 
 def _cfg(**kw):
     base = dict(n_layers=2, d_model=64, n_heads=4, ffn_mult=4, vocab=256, n_ctx=32, dtype=0, state_dtype=0,
-                ln_eps=1e-5, flags=0)
+                ln_eps=1e-5, flags=0, mixer=0, kernel_size=1)
     base.update(kw)
     return Bd._Config(*[base[k] for k, _ in Bd._Config._fields_])
 
