@@ -260,7 +260,8 @@ def _blas_threads():
 
 
 def _config_dict(args, shape, w, B, extra=None):
-    c = {"workload": f"{args.workload}{' + head projections' if shape.head_proj else ''}: SRM L{shape.n_layers} d{shape.d_model} F{shape.d_ffn} V{shape.vocab} "
+    mix = {"mixed": "", "combined": " + combined heads", "kernel": f" + kernels of size {shape.kernel_size}"}[shape.mixer]
+    c = {"workload": f"{args.workload}{' + head projections' if shape.head_proj else ''}{mix}: SRM L{shape.n_layers} d{shape.d_model} F{shape.d_ffn} V{shape.vocab} "
                      f"n_ctx{shape.n_ctx} {shape.dtype}, batch {B}, prompts {w['prompt_len']} tokens ({w['prompts']}), "
                      f"{w['sampling']} selection",
          "batch_per_gpu": B, "prompt_len": w["prompt_len"], "selection": w["sampling"],
@@ -343,9 +344,12 @@ def run_ours(args):
     if args.top_p is not None:         # nucleus sampling instead of the workload's selection rule
         w = dict(w, sampling="topp", top_p=args.top_p, temperature=args.temperature or 0.7)
     shape = I.CONFIGS[w["model"]]
+    import dataclasses
     if args.head_proj:
-        import dataclasses
         shape = dataclasses.replace(shape, head_proj=True)
+    if args.mixer != "mixed":
+        shape = dataclasses.replace(shape, mixer=args.mixer, kernel_size=args.kernel_size if args.mixer == "kernel" else 1)
+    planes = {"mixed": 1, "combined": 2, "kernel": args.kernel_size}[args.mixer]     # d-vectors of cache per sample and layer
     B = args.batch or w["batch"] or 4096
     n = w["prompt_len"]
     peaks, peak_src = measured_peaks()
@@ -484,9 +488,9 @@ def run_ours(args):
     achieved_tf = gemm_flops / (gemm_ms / 1e3) / 1e12 if gemm_ms > 0 else 0.0
     prof_total = sum(v[1] for v in prof.values())
     peak_tf = peaks["bf16_tflops_sustained"]
-    t_roof, bound, t_tc, t_hbm = step_roofline_s(shape, B, sbytes, peaks)
-    mixer_bytes = prof_steps * L * B * d * (4 + 4 + 2 * sbytes + 2)       # x r/w, cache r/w, bf16 activation
-    mixer_cache_bytes = prof_steps * L * B * d * 2 * sbytes                # the part that must cross HBM: cache read + write
+    t_roof, bound, t_tc, t_hbm = step_roofline_s(shape, B, sbytes * planes, peaks)
+    mixer_bytes = prof_steps * L * B * d * (4 + 4 + 2 * sbytes * planes + 2)       # x r/w, cache r/w, bf16 activation
+    mixer_cache_bytes = prof_steps * L * B * d * 2 * sbytes * planes                # the part that must cross HBM: cache read + write
     kernels = {k: {"launches": v[0], "ms_total": round(v[1], 3), "share": round(v[1] / prof_total, 4) if prof_total else 0}
                for k, v in prof.items() if v[0]}
     kernels["gemm_up"]["tflops"] = round(prof_steps * L * B * 2 * d * F / (prof["gemm_up"][1] / 1e3) / 1e12, 1)
@@ -529,7 +533,7 @@ def run_ours(args):
 
     if rank == 0:
         free_b, total_b = torch.cuda.mem_get_info()
-        per_sample = L * d * sbytes + 4 * w["gen"] + 4
+        per_sample = L * planes * d * sbytes + 4 * w["gen"] + 4
         fixed = model.blob.numel() + ws.numel()
         max_conc = int((total_b * 0.97 - fixed) // per_sample)
         clocks = clk.summary(timed_regions)
@@ -571,7 +575,7 @@ def run_ours(args):
             "prefill": None if prefill_ms is None else
             {"ms": round(prefill_ms, 2), "prompt_tokens_per_s": round(B * n / (prefill_ms / 1e3), 1),
              "distinct_prompts": w.get("n_prompts") if (w["prompts"] == "replicated" and not args.no_prompt_dedup) else B},
-            "state_bytes_per_sample": L * d * sbytes,
+            "state_bytes_per_sample": L * planes * d * sbytes,
             "max_concurrent_samples": max_conc,
             "device_status": status,
             "cpu_baseline": cpu,
@@ -735,6 +739,10 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--head-proj", action="store_true",
                     help="token mixer with head projections (Eq. 10): adds W_in, W_out [d, d] per layer")
+    ap.add_argument("--mixer", default="mixed", choices=["mixed", "combined", "kernel"],
+                    help="token mixer of the model: mixed heads (the hot path), linearly combined heads (twice the cache) "
+                         "or kernels of size --kernel-size (Eq. 11; that many times the cache)")
+    ap.add_argument("--kernel-size", type=int, default=4)
     ap.add_argument("--no-splitk", action="store_true",
                     help="down projection with whole output tiles per CTA pair (no sharing of K between pairs)")
     ap.add_argument("--ragged", action="store_true",
