@@ -69,6 +69,10 @@ enum {
   SRM_FLAG_NO_FUSED_TOPK = 32,       /* top-k selection always from fp32 logits written to the workspace (default: the
                                         candidates are collected inside the LM-head epilogue and no logits are written
                                         when the caller does not ask for them); for comparison and measurement */
+  SRM_FLAG_NO_SMALL_BATCH = 64,      /* batches of at most 64 samples also run one kernel per operation (default: such a
+                                        batch, on a bf16 mixed-head model of at most 1024 channels, runs its whole
+                                        decode step in ONE cooperative kernel that streams the weights with all SMs;
+                                        results agree with the other path to rounding, not bit for bit) */
   SRM_FLAG_HEAD_PROJ = 2             /* token mixer with head projections [Method/Architecture, Eq. 10]:
                                         q = W_in LN1(x) (W_in stacks the per-head I_g), heads of q mixed, and
                                         x += W_out (concatenated heads); the cache holds projected values.
@@ -419,6 +423,7 @@ enum srm_kernel_class {
   SRM_KERNEL_SELECT,             /* token selection                                            */
   SRM_KERNEL_PREFILL_MIXER,      /* sequence-parallel token mixing                             */
   SRM_KERNEL_GEMM_PROJ,          /* head projections W_in, W_out (SRM_FLAG_HEAD_PROJ)          */
+  SRM_KERNEL_STEP_SMALL,         /* the single-kernel decode step of a small batch             */
   SRM_KERNEL_CLASS_COUNT
 };
 /* While enabled, every kernel launch of this model is bracketed by two CUDA events recorded on the

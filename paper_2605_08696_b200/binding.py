@@ -22,6 +22,7 @@ FLAG_NO_GRAPH = 4
 FLAG_GRAPH = 8
 FLAG_NO_SPLITK = 16
 FLAG_NO_FUSED_TOPK = 32
+FLAG_NO_SMALL_BATCH = 64
 # enum srm_error
 ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_BUFFER_TOO_SMALL, ERR_CTX_OVERFLOW, ERR_CUDA, \
     ERR_DEVICE_STATUS, ERR_STATIC_SCRATCH = -1, -2, -3, -4, -5, -6, -7, -8
@@ -443,7 +444,8 @@ class SRM:
         return (tok_out, logits) if want_logits else tok_out
 
     # ---- measurement ----
-    KERNEL_CLASSES = ("mixer", "gemm_up", "gemm_down", "gemm_lm", "norm", "select", "prefill_mixer", "gemm_proj")
+    KERNEL_CLASSES = ("mixer", "gemm_up", "gemm_down", "gemm_lm", "norm", "select", "prefill_mixer", "gemm_proj",
+                      "step_small")
 
     def profile(self, on: bool):
         _check(_lib().srm_profile_enable(self.handle, int(on)), "srm_profile_enable")

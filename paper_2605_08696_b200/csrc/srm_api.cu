@@ -28,6 +28,7 @@
 #include "prefill_scan.cuh"
 #include "select.cuh"
 #include "select_topp.cuh"
+#include "step_small.cuh"
 
 using namespace srm;
 
@@ -291,8 +292,15 @@ size_t state_bytes_for(const srm_config& c, int64_t B) {
 }
 
 // ---- workspace carving ----------------------------------------------------------------------
+// Scratch of the small-batch step kernel (step_small.cuh): partial sums of the down projection
+// [8][64, d] fp32, the per-CTA results of the LM-head slabs [256][64] and the grid-barrier word.
+size_t small_scratch_bytes(const srm_config& c) {
+  return align_up((size_t)8 * sb::kMaxRows * c.d_model * 4, 256) + align_up((size_t)256 * sb::kMaxRows * 8, 256) + 256;
+}
+
 struct DecodeWs {
   float* x; void* a; void* H; float* logits;
+  uint8_t* small;         // small_scratch_bytes
   float* q;               // head projections only
   int32_t* order;         // split-K down projection: one word per (tile of x, CTA of the pair, epilogue warp)
   size_t order_bytes;
@@ -311,7 +319,7 @@ size_t decode_ws_bytes(const srm_model& m, int64_t rows) {
   const size_t d = m.cfg.d_model, F = m.F(), V = m.cfg.vocab, ab = m.act_bytes();
   return align_up(rows * d * 4, 256) + align_up(rows * d * ab, 256) + align_up(rows * F * ab, 256) +
          align_up(rows * V * 4, 256) + (m.head_proj() ? align_up(rows * d * 4, 256) : 0) +
-         (splitk_enabled(m.cfg) ? splitk_order_bytes(rows, m.cfg.d_model) : 0);
+         (splitk_enabled(m.cfg) ? splitk_order_bytes(rows, m.cfg.d_model) : 0) + small_scratch_bytes(m.cfg);
 }
 size_t prefill_ws_bytes(const srm_model& m, int64_t samples, int n) {
   const size_t d = m.cfg.d_model, F = m.F(), V = m.cfg.vocab, ab = m.act_bytes(), rows = (size_t)samples * n;
@@ -344,6 +352,8 @@ DecodeWs carve_decode(const srm_model& m, void* ws, int64_t rows) {
   if (m.head_proj()) p += align_up(rows * d * 4, 256);
   w.order_bytes = splitk_enabled(m.cfg) ? splitk_order_bytes(rows, m.cfg.d_model) : 0;
   w.order = w.order_bytes ? reinterpret_cast<int32_t*>(p) : nullptr;
+  p += w.order_bytes;
+  w.small = p;
   return w;
 }
 PrefillWs carve_prefill(const srm_model& m, void* ws, int64_t samples, int n) {
@@ -920,6 +930,96 @@ int decode_chunk(srm_model& m, srm_state& s, int64_t b0, int64_t R, const int32_
   return launch_select(m, R, lg, samp, samp.sample_idx_base + (uint64_t)b0, step, o, s.status, st);
 }
 
+// ---- small batches: the whole step in one cooperative kernel (step_small.cuh) ----------------------
+struct SmallPlan { sb::Params p; int grid; size_t smem; };
+
+// Whether a batch of B samples takes the single-kernel step, and its slab plan. Mixed heads, bf16 weights, at most
+// 64 samples and 1024 channels; everything else takes the kernel-per-operation path.
+bool small_step_plan(const srm_model& m, const srm_state& s, SmallPlan* P) {
+  const srm_config& c = m.cfg;
+  if (c.dtype != SRM_DTYPE_BF16 || (c.flags & (SRM_FLAG_SIMT_GEMM | SRM_FLAG_NO_SMALL_BATCH | SRM_FLAG_HEAD_PROJ))) return false;
+  if (c.mixer != SRM_MIXER_MIXED || s.ragged || s.B > sb::kMaxRows || c.d_model > 1024 || m.num_sms < 16 || m.num_sms > 256) return false;
+  const int d = c.d_model, F = (int)m.F(), V = c.vocab, G = m.num_sms;
+  if (F % 16 || d % 64) return false;
+  sb::Params& p = P->p;
+  p.up_cols = ((F + G - 1) / G + 7) / 8 * 8;
+  p.up_ctas = (F + p.up_cols - 1) / p.up_cols;
+  p.dn_cols = 64;
+  p.dn_nslabs = d / 64;
+  int ks = G / p.dn_nslabs;
+  ks = ks > 8 ? 8 : ks;
+  if (ks < 1) return false;
+  p.dn_klen = ((F + ks - 1) / ks + 15) / 16 * 16;
+  p.dn_kslabs = (F + p.dn_klen - 1) / p.dn_klen;
+  p.lm_cols = ((V + G - 1) / G + sb::kLmChunkCols - 1) / sb::kLmChunkCols * sb::kLmChunkCols;
+  p.lm_ctas = (V + p.lm_cols - 1) / p.lm_cols;
+  P->grid = G;
+  P->smem = 128 + (size_t)sb::act_region_bytes(d, p.dn_klen) + (size_t)sb::weight_region_bytes(d, p.up_cols, p.dn_cols, p.dn_klen);
+  return P->smem <= (size_t)sb::kSmemBytes;
+}
+
+template <typename ST>
+int launch_step_small_t(const SmallPlan& P, cudaStream_t st) {
+  int rc = ensure_dynamic_smem(reinterpret_cast<const void*>(sb::step_small_kernel<ST>), sb::kSmemBytes);
+  if (rc != SRM_OK) return rc;
+  int per_sm = 0;
+  SRM_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, sb::step_small_kernel<ST>, sb::kThreads, P.smem));
+  if (per_sm < 1) return SRM_ERR_UNSUPPORTED;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)P.grid);
+  cfg.blockDim = dim3(sb::kThreads);
+  cfg.dynamicSmemBytes = P.smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeCooperative;           // all CTAs resident at once: the kernel has grid-wide barriers
+  attr.val.cooperative = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  SRM_CUDA(cudaLaunchKernelEx(&cfg, sb::step_small_kernel<ST>, P.p));
+  return SRM_OK;
+}
+
+// One decode step of all B <= 64 samples of the state. SRM_ERR_UNSUPPORTED: take the ordinary path.
+int decode_step_small(srm_model& m, srm_state& s, SmallPlan& P, const int32_t* tok_in, const srm_sampling& samp, int step,
+                      const SelectOut& out, float* logits_out, const DecodeWs& w, cudaStream_t st, const int32_t* ctr) {
+  const srm_config& c = m.cfg;
+  sb::Params& p = P.p;
+  p.B = (int)s.B; p.d = c.d_model; p.F = (int)m.F(); p.V = c.vocab; p.h = c.n_heads; p.n_ctx = c.n_ctx; p.L = c.n_layers;
+  p.t = (int)(s.pos < c.n_ctx ? s.pos : c.n_ctx - 1);
+  p.eps = c.ln_eps;
+  p.tok_in = tok_in;
+  p.E = reinterpret_cast<const bf16*>(m.ptr(-1, SRM_T_E));
+  p.W_lm = reinterpret_cast<const bf16*>(m.ptr(-1, SRM_T_W_LM));
+  p.lnf_g = m.fptr(-1, SRM_T_LNF_G); p.lnf_b = m.fptr(-1, SRM_T_LNF_B);
+  p.layer0 = sb::LayerW{m.fptr(0, SRM_T_LN1_G), m.fptr(0, SRM_T_LN1_B), m.fptr(0, SRM_T_LN2_G), m.fptr(0, SRM_T_LN2_B),
+                        m.fptr(0, SRM_T_ALPHA), m.fptr(0, SRM_T_BETA), m.fptr(0, SRM_T_LAMBDA), m.fptr(0, SRM_T_B1),
+                        m.fptr(0, SRM_T_B2), reinterpret_cast<const bf16*>(m.ptr(0, SRM_T_W1)),
+                        reinterpret_cast<const bf16*>(m.ptr(0, SRM_T_W2))};
+  p.layer_bytes = c.n_layers > 1 ? (int64_t)(m.layout.layer[SRM_T_COUNT + SRM_T_LN1_G].off - m.layout.layer[SRM_T_LN1_G].off) : 0;
+  p.S = s.layer_ptr(0);
+  p.layer_stride = (int64_t)s.B * c.d_model * m.state_bytes();
+  p.x = w.x; p.a = reinterpret_cast<bf16*>(w.a); p.H = reinterpret_cast<bf16*>(w.H);
+  uint8_t* q = w.small;
+  p.part = reinterpret_cast<float*>(q); q += align_up((size_t)8 * sb::kMaxRows * c.d_model * 4, 256);
+  p.best = reinterpret_cast<unsigned long long*>(q); q += align_up((size_t)256 * sb::kMaxRows * 8, 256);
+  p.bar = reinterpret_cast<uint32_t*>(q);
+  p.status = s.status;
+  p.ctr = ctr;
+  p.greedy = samp.mode == SRM_SELECT_GREEDY ? 1 : 0;
+  p.logits = logits_out != nullptr ? logits_out : (p.greedy ? nullptr : w.logits);
+  p.out = out;
+  SRM_CUDA(cudaMemsetAsync(p.bar, 0, 256, st));
+  int rc;
+  {
+    LaunchScope scope(m, SRM_KERNEL_STEP_SMALL, st);
+    if (c.state_dtype == SRM_DTYPE_FP16) rc = launch_step_small_t<fp16>(P, st);
+    else if (c.state_dtype == SRM_DTYPE_BF16) rc = launch_step_small_t<bf16>(P, st);
+    else rc = launch_step_small_t<float>(P, st);
+  }
+  if (rc != SRM_OK || p.greedy) return rc;
+  return launch_select(m, s.B, p.logits, samp, samp.sample_idx_base, step, out, s.status, st);
+}
+
 // Rows per decode pass for a batch of B rows when the workspace holds up to `fit` rows. Up to kOnePassRows the
 // batch runs as one pass. Beyond that it is cut into the fewest equal passes of at most kMaxPassRows rows, each a
 // whole number of 256-row tiles: a larger pass pushes the activations of a layer (H, x, a: 14 KB per row for
@@ -952,6 +1052,14 @@ int decode_step_impl(srm_model* m, srm_state* s, const int32_t* d_tok_in, const 
   const int32_t* tok_in = d_tok_in != nullptr ? d_tok_in : s->last_tok;
   SelectOut out{s->last_tok, d_tok_out, d_store, store_stride, store_col, 1, ctr, s->ragged ? s->pos_dev : nullptr,
                 nullptr, nullptr, samp->mode == SRM_SELECT_TOPK ? s->thr : nullptr};
+  SmallPlan small;
+  if (rows >= s->B && small_step_plan(*m, *s, &small)) {
+    rc = decode_step_small(*m, *s, small, tok_in, *samp, step, out, d_logits_out, w, st, ctr);
+    if (rc != SRM_ERR_UNSUPPORTED) {
+      if (rc == SRM_OK) s->pos += 1;
+      return rc;
+    }
+  }
   for (int64_t b0 = 0; b0 < s->B; b0 += rows) {
     const int64_t R = (s->B - b0 < rows) ? s->B - b0 : rows;
     if ((rc = decode_chunk(*m, *s, b0, R, tok_in, *samp, step, out, d_logits_out, w, st, ctr))) return rc;

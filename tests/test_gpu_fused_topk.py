@@ -15,7 +15,8 @@ DEV = "cuda:0"
 
 def _pair(shape, W):
     import paper_2605_08696_b200 as P
-    return P.SRM(shape, W, device=DEV), P.SRM(shape, W, device=DEV, flags=P.FLAG_NO_FUSED_TOPK)
+    return (P.SRM(shape, W, device=DEV, flags=P.FLAG_NO_SMALL_BATCH),
+            P.SRM(shape, W, device=DEV, flags=P.FLAG_NO_FUSED_TOPK | P.FLAG_NO_SMALL_BATCH))
 
 
 @pytest.mark.parametrize("B,k,T", [(300, 50, 0.8), (70, 1, 1.0), (257, 160, 0.7), (33, 7, 1.3)])

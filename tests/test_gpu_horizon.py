@@ -19,6 +19,7 @@ def _model(name, **kw):
     import paper_2605_08696_b200 as P
     shape = I.CONFIGS[name]
     W = weights_for(name)
+    kw["flags"] = kw.get("flags", 0) | P.FLAG_NO_SMALL_BATCH      # the kernels of the large-batch path, on a few samples
     return shape, W, P.SRM(shape, W, device=DEV, **kw)
 
 

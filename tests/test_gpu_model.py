@@ -16,6 +16,7 @@ def _build(name, **kw):
     import paper_2605_08696_b200 as P
     shape = I.CONFIGS[name]
     W = weights_for(name)
+    kw["flags"] = kw.get("flags", 0) | P.FLAG_NO_SMALL_BATCH      # these tests are about the kernel-per-operation path
     return shape, W, P.SRM(shape, W, device=DEV, **kw)
 
 
