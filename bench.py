@@ -482,8 +482,10 @@ def run_ours(args):
     model.profile(False)
     prof = model.profile_read()
     d, L, V, F = shape.d_model, shape.n_layers, shape.vocab, shape.d_ffn
-    gemm_ms = sum(prof[k][1] for k in ("gemm_up", "gemm_down", "gemm_lm", "gemm_proj"))
-    gemm_launches = sum(prof[k][0] for k in ("gemm_up", "gemm_down", "gemm_lm", "gemm_proj"))
+    single_kernel = prof["step_small"][0] > 0          # small batch: the whole step is one kernel (dense work included)
+    gemm_classes = ("step_small",) if single_kernel else ("gemm_up", "gemm_down", "gemm_lm", "gemm_proj")
+    gemm_ms = sum(prof[k][1] for k in gemm_classes)
+    gemm_launches = sum(prof[k][0] for k in gemm_classes)
     gemm_flops = prof_steps * B * step_flops(shape)
     achieved_tf = gemm_flops / (gemm_ms / 1e3) / 1e12 if gemm_ms > 0 else 0.0
     prof_total = sum(v[1] for v in prof.values())
@@ -493,17 +495,21 @@ def run_ours(args):
     mixer_cache_bytes = prof_steps * L * B * d * 2 * sbytes * planes                # the part that must cross HBM: cache read + write
     kernels = {k: {"launches": v[0], "ms_total": round(v[1], 3), "share": round(v[1] / prof_total, 4) if prof_total else 0}
                for k, v in prof.items() if v[0]}
-    kernels["gemm_up"]["tflops"] = round(prof_steps * L * B * 2 * d * F / (prof["gemm_up"][1] / 1e3) / 1e12, 1)
-    kernels["gemm_down"]["tflops"] = round(prof_steps * L * B * 2 * d * F / (prof["gemm_down"][1] / 1e3) / 1e12, 1)
-    kernels["gemm_lm"]["tflops"] = round(prof_steps * B * 2 * d * V / (prof["gemm_lm"][1] / 1e3) / 1e12, 1)
-    if shape.head_proj:
-        kernels["gemm_proj"]["tflops"] = round(prof_steps * L * B * 4 * d * d / (prof["gemm_proj"][1] / 1e3) / 1e12, 1)
-    kernels["mixer"]["gbs"] = round(mixer_bytes / (prof["mixer"][1] / 1e3) / 1e9, 1)          # all bytes it moves (x and a: L2)
-    kernels["mixer"]["cache_gbs"] = round(mixer_cache_bytes / (prof["mixer"][1] / 1e3) / 1e9, 1)   # algorithmic: the cache
-    kernels["mixer"]["cache_frac_of_hbm_peak"] = round(kernels["mixer"]["cache_gbs"] / peaks["hbm_gbs"], 3)
+    if not single_kernel:
+        kernels["gemm_up"]["tflops"] = round(prof_steps * L * B * 2 * d * F / (prof["gemm_up"][1] / 1e3) / 1e12, 1)
+        kernels["gemm_down"]["tflops"] = round(prof_steps * L * B * 2 * d * F / (prof["gemm_down"][1] / 1e3) / 1e12, 1)
+        kernels["gemm_lm"]["tflops"] = round(prof_steps * B * 2 * d * V / (prof["gemm_lm"][1] / 1e3) / 1e12, 1)
+        if shape.head_proj:
+            kernels["gemm_proj"]["tflops"] = round(prof_steps * L * B * 4 * d * d / (prof["gemm_proj"][1] / 1e3) / 1e12, 1)
+        kernels["mixer"]["gbs"] = round(mixer_bytes / (prof["mixer"][1] / 1e3) / 1e9, 1)          # all bytes it moves (x and a: L2)
+        kernels["mixer"]["cache_gbs"] = round(mixer_cache_bytes / (prof["mixer"][1] / 1e3) / 1e9, 1)   # algorithmic: the cache
+        kernels["mixer"]["cache_frac_of_hbm_peak"] = round(kernels["mixer"]["cache_gbs"] / peaks["hbm_gbs"], 3)
+    else:                                # bound by reading the weights once per step
+        kernels["step_small"]["weight_gbs"] = round(prof_steps * step_flops(shape) / (prof["step_small"][1] / 1e3) / 1e9, 1)
+        kernels["step_small"]["frac_of_hbm_peak"] = round(kernels["step_small"]["weight_gbs"] / peaks["hbm_gbs"], 3)
     for k_ in kernels.values():
         k_["us_per_launch"] = round(k_["ms_total"] * 1e3 / k_["launches"], 2)
-    if samp.mode != "greedy":            # greedy selection is fused into the LM head: no logits in HBM, nothing to rate
+    if samp.mode != "greedy" and "select" in kernels:   # greedy selection is fused into the LM head: nothing to rate
         kernels["select"]["gbs"] = round(prof_steps * B * V * 4 / (prof["select"][1] / 1e3) / 1e9, 1)
 
     # ---- end to end through the host-buffer call: H2D tokens in, D2H tokens out, every step ----
@@ -531,6 +537,24 @@ def run_ours(args):
     e2e_value = whole_job_value(world, B, args.steps, statistics.median(e2e_ms))
     status = st.status()
 
+    if single_kernel:
+        # the step is one weight-streaming kernel: algorithmic bytes = the bf16 weights once + the cache read and written
+        step_bytes = step_flops(shape) + B * 2 * L * d * sbytes
+        gbs = prof_steps * step_bytes / (gemm_ms / 1e3) / 1e9 if gemm_ms > 0 else 0.0
+        roofline = {"bound": "hbm", "kernel": "step_small_kernel (the whole decode step of a batch of at most 64 samples)",
+                    "achieved": round(gbs, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": round(gbs / peaks["hbm_gbs"], 4),
+                    "peak_source": f"hbm_gbs, {peak_src}", "launches": int(gemm_launches), "steps_profiled": prof_steps,
+                    "traffic": None, "bytes_per_step": step_bytes}
+    else:
+        roofline = {"bound": "tensor", "kernel": "gemm_tc_kernel (feed-forward up/down + LM head)",
+                    "achieved": round(achieved_tf, 1), "peak": peak_tf, "unit": "TFLOP/s",
+                    "frac": round(achieved_tf / peak_tf, 4), "peak_source": f"bf16_tflops_sustained, {peak_src}",
+                    "frac_of_burst_peak": round(achieved_tf / peaks["bf16_tflops"], 4),
+                    "launches": int(gemm_launches), "steps_profiled": prof_steps,
+                    "traffic": dram_traffic_per_step(args.workload, B) if not (shape.head_proj or planes > 1) else None,
+                    "traffic_note": "DRAM bytes of the GEMM launches of one step (ncu, cold cache; see profiles/); "
+                                    "null when no capture exists for this workload, batch and GEMM source",
+                    "flops_per_step": B * step_flops(shape)}
     if rank == 0:
         free_b, total_b = torch.cuda.mem_get_info()
         per_sample = L * planes * d * sbytes + 4 * w["gen"] + 4
@@ -559,15 +583,7 @@ def run_ours(args):
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": B * 4, "d2h_bytes_per_step": B * 4,
                     "ms_per_step": round(statistics.median(e2e_ms) / args.steps, 5), "blocks": len(e2e_ms),
                     "clocks": e2e_clocks},
-            "roofline": {"bound": "tensor", "kernel": "gemm_tc_kernel (feed-forward up/down + LM head)",
-                         "achieved": round(achieved_tf, 1), "peak": peak_tf, "unit": "TFLOP/s",
-                         "frac": round(achieved_tf / peak_tf, 4), "peak_source": f"bf16_tflops_sustained, {peak_src}",
-                         "frac_of_burst_peak": round(achieved_tf / peaks["bf16_tflops"], 4),
-                         "launches": int(gemm_launches), "steps_profiled": prof_steps,
-                         "traffic": dram_traffic_per_step(args.workload, B) if not shape.head_proj else None,
-                         "traffic_note": "DRAM bytes of the GEMM launches of one step (ncu, cold cache; see profiles/); "
-                                         "null when no capture exists for this workload, batch and GEMM source",
-                         "flops_per_step": B * step_flops(shape)},
+            "roofline": roofline,
             "step_roofline": {"bound": bound, "t_roof_ms": round(t_roof * 1e3, 4), "t_tensor_ms": round(t_tc * 1e3, 4),
                               "t_hbm_ms": round(t_hbm * 1e3, 4), "frac": round(t_roof * 1e3 / (t_ms_max / args.steps), 4),
                               "peaks": f"{peak_src}: {peak_tf} TFLOP/s sustained bf16, {peaks['hbm_gbs']} GB/s HBM"},

@@ -940,16 +940,16 @@ bool small_step_plan(const srm_model& m, const srm_state& s, SmallPlan* P) {
   if (c.dtype != SRM_DTYPE_BF16 || (c.flags & (SRM_FLAG_SIMT_GEMM | SRM_FLAG_NO_SMALL_BATCH | SRM_FLAG_HEAD_PROJ))) return false;
   if (c.mixer != SRM_MIXER_MIXED || s.ragged || s.B > sb::kMaxRows || c.d_model > 1024 || m.num_sms < 16 || m.num_sms > 256) return false;
   const int d = c.d_model, F = (int)m.F(), V = c.vocab, G = m.num_sms;
-  if (F % 16 || d % 64) return false;
+  if (F % 32 || d % 64) return false;
   sb::Params& p = P->p;
-  p.up_cols = ((F + G - 1) / G + 7) / 8 * 8;
+  p.up_cols = ((F + G - 1) / G + 15) / 16 * 16;
   p.up_ctas = (F + p.up_cols - 1) / p.up_cols;
   p.dn_cols = 64;
   p.dn_nslabs = d / 64;
   int ks = G / p.dn_nslabs;
   ks = ks > 8 ? 8 : ks;
   if (ks < 1) return false;
-  p.dn_klen = ((F + ks - 1) / ks + 15) / 16 * 16;
+  p.dn_klen = ((F + ks - 1) / ks + 31) / 32 * 32;
   p.dn_kslabs = (F + p.dn_klen - 1) / p.dn_klen;
   p.lm_cols = ((V + G - 1) / G + sb::kLmChunkCols - 1) / sb::kLmChunkCols * sb::kLmChunkCols;
   p.lm_ctas = (V + p.lm_cols - 1) / p.lm_cols;

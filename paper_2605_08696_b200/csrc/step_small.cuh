@@ -123,26 +123,36 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], 
                : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
 }
 
-// One 16 x 8 output tile over K (a multiple of 16): rows m0.. of A (row-major, lda bytes per row) times rows
-// n0.. of W (row-major [n][k], ldw bytes per row), both in shared memory. Fragment layout of the result: lane l
-// holds c[0], c[1] = (row m0 + l / 4, columns n0 + 2 (l % 4), + 1) and c[2], c[3] = the same columns of row + 8.
-__device__ __forceinline__ void tile_16x8(float (&c)[4], const uint8_t* A, int lda, int m0, const uint8_t* W, int ldw,
-                                          int n0, int K, int lane) {
-  c[0] = c[1] = c[2] = c[3] = 0.f;
+// One 16 x 16 output tile over K (a multiple of 32): rows m0.. of A (row-major, lda bytes per row) times rows
+// n0 .. n0 + 15 of W (row-major [n][k], ldw bytes per row), both in shared memory. c0 holds columns n0 .. n0 + 7, c1
+// columns n0 + 8 .. n0 + 15; fragment layout: lane l holds c[0], c[1] = (row m0 + l / 4, columns 2 (l % 4), + 1 of its
+// eight) and c[2], c[3] = the same columns of row + 8. Even and odd k-steps accumulate separately (four independent
+// chains of dependent mma instructions instead of one: with a few rows the tile is latency-bound) and are added at
+// the end.
+__device__ __forceinline__ void tile_16x16(float (&c0)[4], float (&c1)[4], const uint8_t* A, int lda, int m0, const uint8_t* W,
+                                           int ldw, int n0, int K, int lane) {
+  float e0[4] = {0.f, 0.f, 0.f, 0.f}, e1[4] = {0.f, 0.f, 0.f, 0.f}, o0[4] = {0.f, 0.f, 0.f, 0.f}, o1[4] = {0.f, 0.f, 0.f, 0.f};
   // A: matrices (rows 0-7, k 0-7), (rows 8-15, k 0-7), (rows 0-7, k 8-15), (rows 8-15, k 8-15): lane l points at
-  // row (l % 16), k offset 8 (l / 16). B: (n 0-7, k 0-7), (n 0-7, k 8-15): lane l % 16 points at row (l % 8), k
-  // offset 8 ((l / 8) % 2).
+  // row (l % 16), k offset 8 (l / 16). W: (n 0-7, k 0-7), (n 0-7, k 8-15), (n 8-15, k 0-7), (n 8-15, k 8-15): lane l
+  // points at row (l % 8) + 8 (l / 16), k offset 8 ((l / 8) % 2).
   const uint32_t a_addr = tc::smem_u32(A + (size_t)(m0 + (lane & 15)) * lda + (lane >> 4) * 16);
-  const uint32_t b_addr = tc::smem_u32(W + (size_t)(n0 + (lane & 7)) * ldw + ((lane >> 3) & 1) * 16);
-#pragma unroll 4
-  for (int k = 0; k < K; k += 16) {
-    uint32_t a[4], b[2];
+  const uint32_t b_addr = tc::smem_u32(W + (size_t)(n0 + (lane & 7) + ((lane >> 4) << 3)) * ldw + ((lane >> 3) & 1) * 16);
+#pragma unroll 2
+  for (int k = 0; k < K; k += 32) {
+    uint32_t a[4], b[4], a2[4], b2[4];
     ldsm_x4(a, a_addr + k * 2);
-    ldsm_x2(b, b_addr + k * 2);
-    mma_bf16(c, a, b);
+    ldsm_x4(b, b_addr + k * 2);
+    ldsm_x4(a2, a_addr + k * 2 + 32);
+    ldsm_x4(b2, b_addr + k * 2 + 32);
+    const uint32_t bl[2] = {b[0], b[1]}, bh[2] = {b[2], b[3]}, bl2[2] = {b2[0], b2[1]}, bh2[2] = {b2[2], b2[3]};
+    mma_bf16(e0, a, bl);
+    mma_bf16(e1, a, bh);
+    mma_bf16(o0, a2, bl2);
+    mma_bf16(o1, a2, bh2);
   }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) { c0[i] = e0[i] + o0[i]; c1[i] = e1[i] + o1[i]; }
 }
-
 
 // ---- shared-memory staging --------------------------------------------------------------------
 // `rows` rows of `row_bytes` bytes (a multiple of 16), `src_stride` bytes apart in global memory, to rows
@@ -164,91 +174,93 @@ __device__ __forceinline__ bool wait_stage(uint64_t* bar, uint32_t parity, uint3
   return tc::mbar_wait(bar, parity, status);
 }
 
-// ---- row phase: one warp per sample row ---------------------------------------------------------
+// ---- row phase: one CTA per sample row -------------------------------------------------------------
+// Sum over the CTA of one value per thread (all threads call it; `red` holds one float per warp).
+__device__ __forceinline__ float cta_sum(float v, float* red) {
+  v = warp_sum(v);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+  __syncthreads();
+  float t = 0.f;
+#pragma unroll
+  for (int w = 0; w < kWarps; ++w) t += red[w];
+  __syncthreads();                         // red may be written again
+  return t;
+}
+
 // x_in = E[tok] (layer 0) or x + b2 of the previous layer + the partial sums of its down projection in slab order.
-// layer < L: the fused mixer step of mixer_step_kernel (LN1, Eq. 2 / Eq. 3 update of the cache, residual, LN2),
-// leaving x and the activation a. layer == L: a = LN_f(x_in) (x is not needed any more).
+// layer < L: the fused mixer step (LN1, Eq. 2 / Eq. 3 update of the cache, residual, LN2), leaving x and the
+// activation a. layer == L: a = LN_f(x_in). Thread i owns channels 4 i .. 4 i + 3 (d <= 1024): every global load
+// of the row is issued before the first reduction, so the phase costs a few memory latencies, not one per vector.
 template <typename ST>
-__device__ __forceinline__ void row_phase(const Params& p, int layer, int64_t row, int lane, int t) {
-  constexpr int NV = 8;                    // d <= 1024
-  const int d = p.d;
-  float4 v[NV];
+__device__ __forceinline__ void row_phase(const Params& p, int layer, int64_t row, int t, float* red) {
+  const int d = p.d, c = threadIdx.x * 4;
+  const bool on = c < d;
+  const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+  float4 v = zero;
   if (layer == 0) {
     int tk = p.tok_in[row];
     if (tk < 0 || tk >= p.V) {
-      if (lane == 0) raise_status(p.status, kStatusTokenRange);
+      if (threadIdx.x == 0) raise_status(p.status, kStatusTokenRange);
       tk = tk < 0 ? 0 : p.V - 1;
     }
-    const bf16* e = p.E + (int64_t)tk * d;
+    if (on) v = ldg4(p.E + (int64_t)tk * d + c);
+  } else if (on) {
+    // written by other CTAs in this kernel: not through L1
+    float4 q[8];
 #pragma unroll
-    for (int i = 0; i < NV; ++i) {
-      const int c = (i * 32 + lane) * 4;
-      if (c < d) v[i] = ldg4(e + c);
-    }
-  } else {
-    const float* xr = p.x + row * d;
-    const float* b2 = layer_w(p, layer - 1).b2;
+    for (int ks = 0; ks < 8; ++ks)
+      q[ks] = ks < p.dn_kslabs ? __ldcg(reinterpret_cast<const float4*>(p.part + ((int64_t)ks * p.B + row) * d + c)) : zero;
+    v = __ldcg(reinterpret_cast<const float4*>(p.x + row * d + c));
+    const float4 bb = ldg4(layer_w(p, layer - 1).b2 + c);
+    v = make_float4(v.x + bb.x, v.y + bb.y, v.z + bb.z, v.w + bb.w);
 #pragma unroll
-    for (int i = 0; i < NV; ++i) {
-      const int c = (i * 32 + lane) * 4;
-      if (c < d) {
-        float4 acc = __ldcg(reinterpret_cast<const float4*>(xr + c));      // written by other CTAs in this kernel: not through L1
-        const float4 bb = ldg4(b2 + c);
-        acc = make_float4(acc.x + bb.x, acc.y + bb.y, acc.z + bb.z, acc.w + bb.w);
-        for (int ks = 0; ks < p.dn_kslabs; ++ks) {
-          const float4 q = __ldcg(reinterpret_cast<const float4*>(p.part + ((int64_t)ks * p.B + row) * d + c));
-          acc = make_float4(acc.x + q.x, acc.y + q.y, acc.z + q.z, acc.w + q.w);
-        }
-        v[i] = acc;
-      }
+    for (int ks = 0; ks < 8; ++ks) v = make_float4(v.x + q[ks].x, v.y + q[ks].y, v.z + q[ks].z, v.w + q[ks].w);
+  }
+  const bool last = layer == p.L;
+  const LayerW w = layer_w(p, last ? 0 : layer);
+  // parameters and the cache row: independent of the statistics, so their loads overlap the reductions
+  float4 g1 = zero, b1 = zero, g2 = zero, b2n = zero, bt = zero, s = zero;
+  float al = 0.f, lm = 0.f;
+  int g = 0;
+  ST* Sr = nullptr;
+  if (on) {
+    if (last) {
+      g2 = ldg4(p.lnf_g + c); b2n = ldg4(p.lnf_b + c);
+    } else {
+      g = c / (d / p.h);
+      g1 = ldg4(w.ln1_g + c); b1 = ldg4(w.ln1_b + c); g2 = ldg4(w.ln2_g + c); b2n = ldg4(w.ln2_b + c);
+      bt = ldg4(w.beta + (int64_t)t * d + c);
+      al = __ldg(w.alpha + (int64_t)g * p.n_ctx + t); lm = __ldg(w.lam + g);
+      Sr = reinterpret_cast<ST*>(static_cast<uint8_t*>(p.S) + (int64_t)layer * p.layer_stride) + row * d + c;
+      s = ld4(Sr);
     }
   }
-  float mean, rstd;
-  row_stats<NV>(v, lane, d, p.eps, mean, rstd);
-  bf16* ar = p.a + row * d;
-  if (layer == p.L) {
-#pragma unroll
-    for (int i = 0; i < NV; ++i) {
-      const int c = (i * 32 + lane) * 4;
-      if (c < d) st4(ar + c, norm4(v[i], mean, rstd, ldg4(p.lnf_g + c), ldg4(p.lnf_b + c)));
-    }
-    return;
-  }
-  const LayerW w = layer_w(p, layer);
-  const int dh = d / p.h, h_row = p.h >> 1;
-  const float* beta_t = w.beta + (int64_t)t * d;
-  ST* Sr = reinterpret_cast<ST*>(static_cast<uint8_t*>(p.S) + (int64_t)layer * p.layer_stride) + row * d;
-  float* xo = p.x + row * d;
-#pragma unroll
-  for (int i = 0; i < NV; ++i) {
-    const int c = (i * 32 + lane) * 4;
-    if (c < d) {
-      const float4 s = ld4(Sr + c);
-      const float4 z = norm4(v[i], mean, rstd, ldg4(w.ln1_g + c), ldg4(w.ln1_b + c));
-      const int g = c / dh;
-      const float al = __ldg(w.alpha + (int64_t)g * p.n_ctx + t), lm = __ldg(w.lam + g);
-      const float4 bt = ldg4(beta_t + c);
+  const float inv_d = 1.0f / (float)d;
+  if (!last) {
+    const float mean = cta_sum((v.x + v.y) + (v.z + v.w), red) * inv_d;
+    const float4 cd = on ? make_float4(v.x - mean, v.y - mean, v.z - mean, v.w - mean) : zero;
+    const float rstd = rsqrtf(cta_sum((cd.x * cd.x + cd.y * cd.y) + (cd.z * cd.z + cd.w * cd.w), red) * inv_d + p.eps);
+    if (on) {
+      const float4 z = norm4(v, mean, rstd, g1, b1);
       float4 y, sn;
-      if (g < h_row) {            // row-repeat head, Eq. 2
+      if (g < (p.h >> 1)) {       // row-repeat head, Eq. 2: y = a z + b + S ; S' = l (S + a z)
         const float4 u = make_float4(al * z.x, al * z.y, al * z.z, al * z.w);
         y = make_float4(u.x + bt.x + s.x, u.y + bt.y + s.y, u.z + bt.z + s.z, u.w + bt.w + s.w);
         sn = make_float4(lm * (s.x + u.x), lm * (s.y + u.y), lm * (s.z + u.z), lm * (s.w + u.w));
-      } else {                    // column-repeat head, Eq. 3
+      } else {                    // column-repeat head, Eq. 3: y = a (z + S) + b ; S' = l (z + S)
         const float4 q = make_float4(z.x + s.x, z.y + s.y, z.z + s.z, z.w + s.w);
         y = make_float4(al * q.x + bt.x, al * q.y + bt.y, al * q.z + bt.z, al * q.w + bt.w);
         sn = make_float4(lm * q.x, lm * q.y, lm * q.z, lm * q.w);
       }
-      st4(Sr + c, sn);
-      v[i] = make_float4(v[i].x + y.x, v[i].y + y.y, v[i].z + y.z, v[i].w + y.w);
-      st4(xo + c, v[i]);
+      st4(Sr, sn);
+      v = make_float4(v.x + y.x, v.y + y.y, v.z + y.z, v.w + y.w);
+      st4(p.x + row * d + c, v);
     }
   }
-  row_stats<NV>(v, lane, d, p.eps, mean, rstd);
-#pragma unroll
-  for (int i = 0; i < NV; ++i) {
-    const int c = (i * 32 + lane) * 4;
-    if (c < d) st4(ar + c, norm4(v[i], mean, rstd, ldg4(w.ln2_g + c), ldg4(w.ln2_b + c)));
-  }
+  const float mean = cta_sum((v.x + v.y) + (v.z + v.w), red) * inv_d;
+  const float4 cd = on ? make_float4(v.x - mean, v.y - mean, v.z - mean, v.w - mean) : zero;
+  const float rstd = rsqrtf(cta_sum((cd.x * cd.x + cd.y * cd.y) + (cd.z * cd.z + cd.w * cd.w), red) * inv_d + p.eps);
+  if (on) st4(p.a + row * d + c, norm4(v, mean, rstd, g2, b2n));
 }
 
 // Shared memory: 128 bytes of mbarriers | activation rows (kMaxRows padded rows) | weight rows.
@@ -258,7 +270,7 @@ __host__ __device__ inline int act_region_bytes(int d, int klen) {
 }
 __host__ __device__ inline int weight_region_bytes(int d, int up_cols, int dn_cols, int klen) {
   int b = up_cols * (2 * d + kPadBytes);
-  const int dn = dn_cols * (2 * klen + kPadBytes), lm = 2 * kLmChunkCols * (2 * d + kPadBytes);
+  const int dn = dn_cols * (2 * klen + kPadBytes), lm = 2 * kLmChunkCols * (2 * d + kPadBytes) + 4096;   // + partial sums
   b = b > dn ? b : dn;
   return b > lm ? b : lm;
 }
@@ -272,6 +284,7 @@ __global__ void __launch_bounds__(kThreads, 1) step_small_kernel(const Params p)
   extern __shared__ __align__(128) uint8_t sm[];
   uint64_t* barA = reinterpret_cast<uint64_t*>(sm);
   uint64_t* barW = barA + 1;                             // two stages
+  float* red32 = reinterpret_cast<float*>(sm + 96);     // one float per warp for the row-phase reductions
   uint8_t* sA = sm + 128;
   uint8_t* sW = sA + act_region_bytes(p.d, p.dn_klen);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -321,7 +334,7 @@ __global__ void __launch_bounds__(kThreads, 1) step_small_kernel(const Params p)
   stage_up(0);
   for (int l = 0; l < p.L; ++l) {
     // ---- token mixer: one warp per row ----
-    for (int64_t r = cta + (int64_t)warp * G; r < B; r += (int64_t)kWarps * G) row_phase<ST>(p, l, r, lane, t);
+    for (int64_t r = cta; r < B; r += G) row_phase<ST>(p, l, r, t, red32);
     gb.sync();
 
     // ---- up projection: H[:, slab] = gelu(a W1[slab]^T + b1) ----
@@ -332,19 +345,27 @@ __global__ void __launch_bounds__(kThreads, 1) step_small_kernel(const Params p)
       parA ^= 1u; parW0 ^= 1u;
       if (!ok) gb.dead = true;
       const float* b1 = layer_w(p, l).b1;
-      const int tiles = m_tiles * (up_n >> 3);
+      const int n16 = (up_n + 15) >> 4, tiles = m_tiles * n16;
       for (int tile = warp; ok && tile < tiles; tile += kWarps) {
         const int mt = tile % m_tiles, nt = tile / m_tiles;
-        float c[4];
-        tile_16x8(c, sA, ld_d, mt * 16, sW, ld_d, nt * 8, d, lane);
-        const int col = up_n0 + nt * 8 + 2 * (lane & 3), r0 = mt * 16 + (lane >> 2);
-        const float2 bb = __ldg(reinterpret_cast<const float2*>(b1 + col));
-        if (r0 < B)
-          *reinterpret_cast<__nv_bfloat162*>(p.H + (int64_t)r0 * F + col) =
-              __floats2bfloat162_rn(tc::gelu_fast(c[0] + bb.x), tc::gelu_fast(c[1] + bb.y));
-        if (r0 + 8 < B)
-          *reinterpret_cast<__nv_bfloat162*>(p.H + (int64_t)(r0 + 8) * F + col) =
-              __floats2bfloat162_rn(tc::gelu_fast(c[2] + bb.x), tc::gelu_fast(c[3] + bb.y));
+        float c0[4], c1[4];
+        tile_16x16(c0, c1, sA, ld_d, mt * 16, sW, ld_d, nt * 16, d, lane);
+        const int r0 = mt * 16 + (lane >> 2);
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf) {
+          const float (&c)[4] = hf ? c1 : c0;
+          const int cl = nt * 16 + hf * 8 + 2 * (lane & 3);          // column inside the slab
+          if (cl < up_n) {
+            const int col = up_n0 + cl;
+            const float2 bb = __ldg(reinterpret_cast<const float2*>(b1 + col));
+            if (r0 < B)
+              *reinterpret_cast<__nv_bfloat162*>(p.H + (int64_t)r0 * F + col) =
+                  __floats2bfloat162_rn(tc::gelu_fast(c[0] + bb.x), tc::gelu_fast(c[1] + bb.y));
+            if (r0 + 8 < B)
+              *reinterpret_cast<__nv_bfloat162*>(p.H + (int64_t)(r0 + 8) * F + col) =
+                  __floats2bfloat162_rn(tc::gelu_fast(c[2] + bb.x), tc::gelu_fast(c[3] + bb.y));
+          }
+        }
       }
     }
     __syncthreads();                       // the weight rows have been read: the region may be refilled
@@ -359,14 +380,20 @@ __global__ void __launch_bounds__(kThreads, 1) step_small_kernel(const Params p)
       parA ^= 1u; parW0 ^= 1u;
       if (!ok) gb.dead = true;
       float* out = p.part + (int64_t)dn_ks * B * d;
-      const int tiles = m_tiles * (p.dn_cols >> 3);
+      const int tiles = m_tiles * (p.dn_cols >> 4);
       for (int tile = warp; ok && tile < tiles; tile += kWarps) {
         const int mt = tile % m_tiles, nt = tile / m_tiles;
-        float c[4];
-        tile_16x8(c, sA, ld_k, mt * 16, sW, ld_k, nt * 8, dn_k, lane);
-        const int col = dn_ns * p.dn_cols + nt * 8 + 2 * (lane & 3), r0 = mt * 16 + (lane >> 2);
-        if (r0 < B) *reinterpret_cast<float2*>(out + (int64_t)r0 * d + col) = make_float2(c[0], c[1]);
-        if (r0 + 8 < B) *reinterpret_cast<float2*>(out + (int64_t)(r0 + 8) * d + col) = make_float2(c[2], c[3]);
+        float c0[4], c1[4];
+        tile_16x16(c0, c1, sA, ld_k, mt * 16, sW, ld_k, nt * 16, dn_k, lane);
+        const int col = dn_ns * p.dn_cols + nt * 16 + 2 * (lane & 3), r0 = mt * 16 + (lane >> 2);
+        if (r0 < B) {
+          *reinterpret_cast<float2*>(out + (int64_t)r0 * d + col) = make_float2(c0[0], c0[1]);
+          *reinterpret_cast<float2*>(out + (int64_t)r0 * d + col + 8) = make_float2(c1[0], c1[1]);
+        }
+        if (r0 + 8 < B) {
+          *reinterpret_cast<float2*>(out + (int64_t)(r0 + 8) * d + col) = make_float2(c0[2], c0[3]);
+          *reinterpret_cast<float2*>(out + (int64_t)(r0 + 8) * d + col + 8) = make_float2(c1[2], c1[3]);
+        }
       }
     }
     __syncthreads();
@@ -376,7 +403,7 @@ __global__ void __launch_bounds__(kThreads, 1) step_small_kernel(const Params p)
   }
 
   // ---- final norm ----
-  for (int64_t r = cta + (int64_t)warp * G; r < B; r += (int64_t)kWarps * G) row_phase<ST>(p, p.L, r, lane, t);
+  for (int64_t r = cta; r < B; r += G) row_phase<ST>(p, p.L, r, t, red32);
   gb.sync();
 
   // ---- LM head over this CTA's vocabulary slab, chunk by chunk through two stages ----
@@ -384,7 +411,11 @@ __global__ void __launch_bounds__(kThreads, 1) step_small_kernel(const Params p)
     if (warp == 0) stage_rows(sA, p.a, B, 2 * d, 2 * (int64_t)d, barA, lane);
     bool ok = wait_stage(barA, parA, p.status, gb.dead);
     parA ^= 1u;
-    const int mt = warp & 3, nt = warp >> 2;                   // one 16 x 8 tile of every chunk per warp
+    // Every chunk is one 16-column tile per 16 rows. Warp w takes row tile w % 4 and half w / 4 of K; the upper
+    // halves' partial sums go through shared memory to the lower warps, which own the results.
+    const int mt = warp & 3, kh = warp >> 2;
+    const int k_half = d >> 1;
+    float* xch = reinterpret_cast<float*>(sW + 2 * lm_stage);   // [4 row tiles][32 lanes][8] partial sums
     float bv0 = -INFINITY, bv1 = -INFINITY;
     int bi0 = 0x7fffffff, bi1 = 0x7fffffff;
     bool bad = false;
@@ -393,26 +424,54 @@ __global__ void __launch_bounds__(kThreads, 1) step_small_kernel(const Params p)
       ok = wait_stage(&barW[s], s ? parW1 : parW0, p.status, gb.dead || !ok) && ok;
       if (s) parW1 ^= 1u; else parW0 ^= 1u;
       const int rows = lm_n - ch * kLmChunkCols < kLmChunkCols ? lm_n - ch * kLmChunkCols : kLmChunkCols;
-      if (ok && mt < m_tiles && nt * 8 < rows) {
-        float c[4];
-        tile_16x8(c, sA, ld_d, mt * 16, sW + s * lm_stage, ld_d, nt * 8, d, lane);
-        const int col = lm_n0 + ch * kLmChunkCols + nt * 8 + 2 * (lane & 3), r0 = mt * 16 + (lane >> 2);
-        if (p.logits != nullptr) {
-          if (r0 < B) *reinterpret_cast<float2*>(p.logits + (int64_t)r0 * p.V + col) = make_float2(c[0], c[1]);
-          if (r0 + 8 < B) *reinterpret_cast<float2*>(p.logits + (int64_t)(r0 + 8) * p.V + col) = make_float2(c[2], c[3]);
+      float c0[4], c1[4];
+      const bool work = ok && mt < m_tiles;
+      if (work) {
+        tile_16x16(c0, c1, sA + kh * k_half * 2, ld_d, mt * 16, sW + s * lm_stage + kh * k_half * 2, ld_d, 0, k_half, lane);
+        if (kh == 1) {
+          float4* o = reinterpret_cast<float4*>(xch + (mt * 32 + lane) * 8);
+          o[0] = make_float4(c0[0], c0[1], c0[2], c0[3]);
+          o[1] = make_float4(c1[0], c1[1], c1[2], c1[3]);
         }
-        bad |= !(c[0] == c[0]) | !(c[1] == c[1]) | !(c[2] == c[2]) | !(c[3] == c[3]);
-        if (c[0] > bv0) { bv0 = c[0]; bi0 = col; }              // ascending columns: the lowest among equals is kept
-        if (c[1] > bv0) { bv0 = c[1]; bi0 = col + 1; }
-        if (c[2] > bv1) { bv1 = c[2]; bi1 = col; }
-        if (c[3] > bv1) { bv1 = c[3]; bi1 = col + 1; }
       }
-      __syncthreads();                                           // stage s has been read by every warp
+      __syncthreads();                                           // partial sums are visible; stage s has been read
       stage_lm(ch + 2);
+      if (work && kh == 0) {
+        const float4* o = reinterpret_cast<const float4*>(xch + (mt * 32 + lane) * 8);
+        const float4 q0 = o[0], q1 = o[1];
+        c0[0] += q0.x; c0[1] += q0.y; c0[2] += q0.z; c0[3] += q0.w;
+        c1[0] += q1.x; c1[1] += q1.y; c1[2] += q1.z; c1[3] += q1.w;
+        const int col = lm_n0 + ch * kLmChunkCols + 2 * (lane & 3), r0 = mt * 16 + (lane >> 2);
+        const bool second = rows > 8;                            // V is a multiple of 8: a last chunk may hold 8 columns
+        if (p.logits != nullptr) {
+          if (r0 < B) {
+            *reinterpret_cast<float2*>(p.logits + (int64_t)r0 * p.V + col) = make_float2(c0[0], c0[1]);
+            if (second) *reinterpret_cast<float2*>(p.logits + (int64_t)r0 * p.V + col + 8) = make_float2(c1[0], c1[1]);
+          }
+          if (r0 + 8 < B) {
+            *reinterpret_cast<float2*>(p.logits + (int64_t)(r0 + 8) * p.V + col) = make_float2(c0[2], c0[3]);
+            if (second) *reinterpret_cast<float2*>(p.logits + (int64_t)(r0 + 8) * p.V + col + 8) = make_float2(c1[2], c1[3]);
+          }
+        }
+        // (rows past B of a partly filled tile hold whatever the shared memory held: not looked at)
+        if (r0 < B) bad |= !(c0[0] == c0[0]) | !(c0[1] == c0[1]) | (second & (!(c1[0] == c1[0]) | !(c1[1] == c1[1])));
+        if (r0 + 8 < B) bad |= !(c0[2] == c0[2]) | !(c0[3] == c0[3]) | (second & (!(c1[2] == c1[2]) | !(c1[3] == c1[3])));
+        if (c0[0] > bv0) { bv0 = c0[0]; bi0 = col; }            // ascending columns: the lowest among equals is kept
+        if (c0[1] > bv0) { bv0 = c0[1]; bi0 = col + 1; }
+        if (c0[2] > bv1) { bv1 = c0[2]; bi1 = col; }
+        if (c0[3] > bv1) { bv1 = c0[3]; bi1 = col + 1; }
+        if (second) {
+          if (c1[0] > bv0) { bv0 = c1[0]; bi0 = col + 8; }
+          if (c1[1] > bv0) { bv0 = c1[1]; bi0 = col + 9; }
+          if (c1[2] > bv1) { bv1 = c1[2]; bi1 = col + 8; }
+          if (c1[3] > bv1) { bv1 = c1[3]; bi1 = col + 9; }
+        }
+      }
+      __syncthreads();                                           // the partial sums have been taken
     }
     if (!ok) gb.dead = true;
     if (p.greedy) {
-      // per row: over the four lanes of a quad, then over the two warps that share the row tile
+      // per row: over the four lanes of a quad (their columns interleave, so the packed (value, lowest column) decides)
       unsigned long long k0 = bi0 == 0x7fffffff ? 0ull : pack_best(bv0, bi0), k1 = bi1 == 0x7fffffff ? 0ull : pack_best(bv1, bi1);
 #pragma unroll
       for (int o = 1; o <= 2; o <<= 1) {
@@ -420,13 +479,9 @@ __global__ void __launch_bounds__(kThreads, 1) step_small_kernel(const Params p)
         k0 = q0 > k0 ? q0 : k0; k1 = q1 > k1 ? q1 : k1;
       }
       unsigned long long* red = reinterpret_cast<unsigned long long*>(sW);      // the weight stages are free now
-      if ((lane & 3) == 0) { red[warp * 16 + (lane >> 2)] = k0; red[warp * 16 + 8 + (lane >> 2)] = k1; }
+      if (kh == 0 && (lane & 3) == 0) { red[mt * 16 + (lane >> 2)] = k0; red[mt * 16 + 8 + (lane >> 2)] = k1; }
       __syncthreads();
-      if (threadIdx.x < kMaxRows) {
-        const int row = threadIdx.x, m = row >> 4, rr = row & 15;
-        const unsigned long long a0 = red[m * 16 + rr], a1 = red[(m + 4) * 16 + rr];
-        if (row < B) p.best[(int64_t)cta * B + row] = a0 > a1 ? a0 : a1;
-      }
+      if (threadIdx.x < B) p.best[(int64_t)cta * B + threadIdx.x] = red[threadIdx.x];
       if (bad) raise_status(p.status, kStatusNonFinite);
     }
   }

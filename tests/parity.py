@@ -117,7 +117,8 @@ def teacher_forced(name, shape, W, model, prompts, gen, sampling=None, sample_id
             tok_in = torch.from_numpy(toks_o[:, k].copy()).to(DEV)
             tok_dev, lg = model.decode_step(st, tok_in, samp, k + 1, ws, want_logits=True)
             tok_g = tok_dev.cpu().numpy()
-    assert st.status() == 0
+    flags = st.status()
+    assert flags == 0, f"device status flags {flags}"
     assert st.pos == n + gen - 1
     if check_state:
         # the oracle's final state corresponds to the same consumed tokens
