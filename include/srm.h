@@ -73,8 +73,6 @@ enum {
                                         batch, on a bf16 mixed-head model of at most 1024 channels, runs its whole
                                         decode step in ONE cooperative kernel that streams the weights with all SMs;
                                         results agree with the other path to rounding, not bit for bit) */
-  SRM_FLAG_MIXER_ROWS = 128,         /* the fused token-mixer step runs as one CTA per row (per-channel parameters in
-                                        registers for all rows of a CTA) instead of one warp per row */
   SRM_FLAG_HEAD_PROJ = 2             /* token mixer with head projections [Method/Architecture, Eq. 10]:
                                         q = W_in LN1(x) (W_in stacks the per-head I_g), heads of q mixed, and
                                         x += W_out (concatenated heads); the cache holds projected values.

@@ -21,7 +21,6 @@
 #include "gemm_tc_splitk.cuh"
 #include "mixer.cuh"
 #include "mixer_stream.cuh"
-#include "mixer_rows.cuh"
 #include "mixer_proj.cuh"
 #include "mixer_variants.cuh"
 #include "mixer_model_variants.cuh"
@@ -432,18 +431,6 @@ int launch_mixer_nv(const MixerParams& p, int num_sms, cudaStream_t st) {
   return SRM_OK;
 }
 
-// One CTA per row (mixer_rows.cuh): as many CTAs as stay resident at once walk the rows.
-template <typename WT, typename ST>
-int launch_mixer_rows(const MixerParams& p, int num_sms, cudaStream_t st) {
-  const int threads = ((p.d / 4) + 31) / 32 * 32;
-  int per_sm = 0;
-  SRM_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, mixer_rows_kernel<WT, ST>, threads, 0));
-  if (per_sm < 1) return SRM_ERR_UNSUPPORTED;
-  const int64_t cap = (int64_t)num_sms * per_sm;
-  SRM_CUDA(launch_kernel(mixer_rows_kernel<WT, ST>, dim3((unsigned)(p.R < cap ? p.R : cap)), dim3(threads), 0, st, p));
-  return SRM_OK;
-}
-
 int launch_mixer(const srm_model& m, int layer, int t, int64_t R, const int32_t* tok, float* x, void* S, void* a,
                  uint32_t* status, cudaStream_t st, const int32_t* ctr = nullptr, const int32_t* pos = nullptr) {
   if (R <= 0) return SRM_OK;
@@ -455,8 +442,6 @@ int launch_mixer(const srm_model& m, int layer, int t, int64_t R, const int32_t*
   p.alpha = m.fptr(layer, SRM_T_ALPHA); p.beta = m.fptr(layer, SRM_T_BETA); p.lam = m.fptr(layer, SRM_T_LAMBDA);
   p.R = R; p.d = m.cfg.d_model; p.h = m.cfg.n_heads; p.n_ctx = m.cfg.n_ctx; p.t = t; p.vocab = m.cfg.vocab;
   p.eps = m.cfg.ln_eps; p.status = status; p.ctr = ctr; p.pos = pos;
-  if (m.cfg.flags & SRM_FLAG_MIXER_ROWS)
-    return dispatch_types(m.cfg, [&](auto w, auto c) { return launch_mixer_rows<decltype(w), decltype(c)>(p, m.num_sms, st); });
   return dispatch_types(m.cfg, [&](auto w, auto c) { return launch_mixer_nv<decltype(w), decltype(c)>(p, m.num_sms, st); });
 }
 

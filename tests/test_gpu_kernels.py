@@ -27,14 +27,10 @@ def _t(a, dtype=torch.float32):
                                                  (1536, "bf16", "fp32"), (1024, "bf16", "bf16"), (2048, "fp32", "fp32"),
                                                  (192, "fp32", "bf16"), (1024, "bf16", "fp16"), (192, "fp32", "fp16")])
 @pytest.mark.parametrize("embed", [False, True])
-@pytest.mark.parametrize("cta_per_row", [False, True])
-def test_mixer_step_matches_oracle(d, dtype, state_dtype, embed, cta_per_row):
-    """Both distributions of the fused mixer step: one warp per row (streaming or general kernel, by shape) and one
-    CTA per row."""
+def test_mixer_step_matches_oracle(d, dtype, state_dtype, embed):
     from oracle import srm_oracle as O
-    import paper_2605_08696_b200 as P
     shape = custom_shape(n_layers=2, d_model=d, vocab=512, n_ctx=40, dtype=dtype, seed=7)
-    m, W = _model(shape, state_dtype=state_dtype, flags=P.FLAG_MIXER_ROWS if cta_per_row else 0)
+    m, W = _model(shape, state_dtype=state_dtype)
     rng = np.random.default_rng(d)
     R, layer, t = 37, 1, 17                       # ragged row count (not a multiple of the 4 rows per block)
     lw = {k: np.asarray(v, np.float64) for k, v in W["layers"][layer].items()}
