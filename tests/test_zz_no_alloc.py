@@ -22,7 +22,7 @@ TOL = {"fp32": 1e-4, "bf16": 3e-2}     # the tolerances of the model-level parit
 BF16_SHAPE = I.SRMShape(n_layers=2, d_model=256, vocab=1000, n_ctx=32, dtype="bf16", seed=7)
 
 
-@pytest.mark.parametrize("shape,B", [(I.CONFIGS["tiny"], 4), (BF16_SHAPE, 300)])
+@pytest.mark.parametrize("shape,B", [(I.CONFIGS["tiny"], 4), (BF16_SHAPE, 300), (BF16_SHAPE, 40)])     # 40: the single-kernel step
 def test_static_scratch_step_matches_workspace_step_twice_in_a_row(shape, B):
     import paper_2605_08696_b200 as P
     from helpers import oracle_for
