@@ -357,7 +357,7 @@ def run_ours(args):
     W = I.make_weights(shape)
     model = P.SRM(shape, W, device=dev, state_dtype=args.state_dtype,
                   flags={"auto": 0, "on": P.FLAG_GRAPH, "off": P.FLAG_NO_GRAPH}[args.graph] |
-                  (P.FLAG_NO_SPLITK if args.no_splitk else 0))
+                  (P.FLAG_NO_SPLITK if args.no_splitk else 0) | (P.FLAG_NO_TAIL_SPLIT if args.no_tail_split else 0))
     sidx0 = rank_plan(rank, world, B)["sample_idx_base"]
     samp = {"greedy": lambda: P.Sampling("greedy"),
             "topk": lambda: P.Sampling("topk", w["top_k"], w["temperature"], seed=shape.seed, sample_idx_base=sidx0),
@@ -759,6 +759,8 @@ def main():
                     help="token mixer of the model: mixed heads (the hot path), linearly combined heads (twice the cache) "
                          "or kernels of size --kernel-size (Eq. 11; that many times the cache)")
     ap.add_argument("--kernel-size", type=int, default=4)
+    ap.add_argument("--no-tail-split", action="store_true",
+                    help="tensor-core projections keep the tiles of a partly filled last round whole (256 x 256)")
     ap.add_argument("--no-splitk", action="store_true",
                     help="down projection with whole output tiles per CTA pair (no sharing of K between pairs)")
     ap.add_argument("--ragged", action="store_true",

@@ -73,6 +73,9 @@ enum {
                                         batch, on a bf16 mixed-head model of at most 1024 channels, runs its whole
                                         decode step in ONE cooperative kernel that streams the weights with all SMs;
                                         results agree with the other path to rounding, not bit for bit) */
+  SRM_FLAG_NO_TAIL_SPLIT = 128,      /* tensor-core projections process every 256 x 256 tile whole (default: the tiles of a
+                                        last, partly filled round run as two 256 x 128 pieces each, which keeps nearly all
+                                        CTA pairs busy to the end); for comparison and measurement */
   SRM_FLAG_HEAD_PROJ = 2             /* token mixer with head projections [Method/Architecture, Eq. 10]:
                                         q = W_in LN1(x) (W_in stacks the per-head I_g), heads of q mixed, and
                                         x += W_out (concatenated heads); the cache holds projected values.

@@ -23,6 +23,7 @@ FLAG_GRAPH = 8
 FLAG_NO_SPLITK = 16
 FLAG_NO_FUSED_TOPK = 32
 FLAG_NO_SMALL_BATCH = 64
+FLAG_NO_TAIL_SPLIT = 128
 # enum srm_error
 ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_BUFFER_TOO_SMALL, ERR_CTX_OVERFLOW, ERR_CUDA, \
     ERR_DEVICE_STATUS, ERR_STATIC_SCRATCH = -1, -2, -3, -4, -5, -6, -7, -8

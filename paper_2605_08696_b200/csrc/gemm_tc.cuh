@@ -12,7 +12,8 @@
 // Pairing halves the W bytes each SM pulls from L2 per flop compared with a 128 x 256 tile per
 // SM, which is what bounded the single-CTA version of this kernel.
 //
-// The kernel is persistent: grid = 2 * min(tiles, resident clusters), tiles taken round-robin.
+// The kernel is persistent: grid = 2 * min(pieces, resident clusters), pieces taken round-robin; a piece is a
+// whole tile or, for the tiles of a partly filled last round, one of its two 256 x 128 halves (GemmArgs::tail_tiles).
 // Warp roles per CTA: warp 0 = TMA producer, warp 1 = MMA issuer (leader only) and TMEM owner,
 // warps 2..17 = epilogue (warp w reads TMEM lanes 32*(w%4) .. +31, one accumulator row per thread;
 // the four warps that share a lane quarter split the tile's columns; four warps per scheduler hide
@@ -220,8 +221,11 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
   return d;
 }
 // Instruction descriptor: fp32 accumulate, bf16 A and B, both K-major, N = BN, M = BM (pair).
-constexpr uint32_t kInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(BN >> 3) << 17) |
-                                (uint32_t(BM >> 4) << 24);
+__host__ __device__ constexpr uint32_t instr_desc(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(n >> 3) << 17) | (uint32_t(BM >> 4) << 24);
+}
+constexpr uint32_t kInstrDesc = instr_desc(BN);
+constexpr int kHalfN = BN / 2;                   // width of the pieces the last tiles may be cut into
 
 struct GemmArgs {
   int64_t M, N, K;
@@ -239,7 +243,20 @@ struct GemmArgs {
   // Only the first *m_limit rows (a device word written by an earlier kernel of the stream) are computed; nullptr:
   // all M rows. The first weight tiles are then not fetched ahead of the dependency wait.
   const uint32_t* m_limit;
+  // The last `tail_tiles` tiles (in tile order) are processed as two pieces of 128 columns each, so that a last,
+  // partly filled round of tiles keeps (nearly) all CTA pairs busy: a half piece moves three quarters of a tile's
+  // operand bytes for half its flops, and 2 r half pieces on 74 pairs end earlier than r tiles on r pairs.
+  int tail_tiles;
 };
+
+// Piece q of a launch: the tile it belongs to, its first column inside the tile and its width.
+struct Piece { int64_t tile; int noff, nw; };
+__device__ __forceinline__ Piece piece_of(int64_t q, int64_t tiles, int tail) {
+  const int64_t whole = tiles - tail;
+  if (q < whole) return Piece{q, 0, BN};
+  const int64_t j = q - whole;
+  return Piece{whole + (j >> 1), (int)(j & 1) * kHalfN, kHalfN};
+}
 
 // order-preserving map float -> uint32 (larger float, larger key)
 __device__ __forceinline__ uint32_t order_key_bits(float f) {
@@ -434,7 +451,7 @@ __device__ __forceinline__ void epilogue_columns(const GemmArgs& g, const CUtens
 template <int EPI>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-               const __grid_constant__ CUtensorMap tmD, const GemmArgs g) {
+               const __grid_constant__ CUtensorMap tmD, const __grid_constant__ CUtensorMap tmB64, const GemmArgs g) {
   pdl_trigger();
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -475,6 +492,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
   const int64_t m_tiles = (M_rows + BM - 1) / BM, n_tiles = (g.N + BN - 1) / BN;
   const int64_t tiles = m_tiles * n_tiles;
+  const int tail = g.m_limit != nullptr ? 0 : g.tail_tiles;
+  const int64_t pieces = tiles + tail;                 // a tail tile counts as two pieces
   const int k_blocks = static_cast<int>(g.K / BK);
 
   if (warp == 0) {
@@ -488,15 +507,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       // While the predecessor kernel drains: start the first tile's W loads (the ring is empty, so
       // the first kStages stages need no wait), then order against the predecessor and add the A loads.
       int pre = 0;
-      if (cluster_id < tiles) {
-        const int m0 = static_cast<int>(cluster_id % m_tiles) * BM + static_cast<int>(rank) * kRowsPerCta;
-        const int n0 = static_cast<int>(cluster_id / m_tiles) * BN + static_cast<int>(rank) * kRowsPerCta;
+      if (cluster_id < pieces) {
+        const Piece pc = piece_of(cluster_id, tiles, tail);
+        const int w_rows = pc.nw >> 1;                                       // W rows each CTA of the pair loads
+        const CUtensorMap* mapB = pc.nw == BN ? &tmB : &tmB64;
+        const uint32_t stage_bytes = kAStageBytes + (uint32_t)w_rows * BK * 2;
+        const int m0 = static_cast<int>(pc.tile % m_tiles) * BM + static_cast<int>(rank) * kRowsPerCta;
+        const int n0 = static_cast<int>(pc.tile / m_tiles) * BN + pc.noff + static_cast<int>(rank) * w_rows;
         pre = k_blocks < kStages ? k_blocks : kStages;
         if (!g.w_static) pdl_wait();
         for (int kb = 0; kb < pre; ++kb) {
           const uint32_t full_leader = mapa(smem_u32(&full[kb]), 0);
-          mbar_expect_tx_cluster(full_leader, kStageBytes);
-          tma_load_2d(sB + kb * kBStageBytes, &tmB, full_leader, kb * BK, n0);
+          mbar_expect_tx_cluster(full_leader, stage_bytes);
+          tma_load_2d(sB + kb * kBStageBytes, mapB, full_leader, kb * BK, n0);
         }
         if (g.w_static) pdl_wait();
         for (int kb = 0; kb < pre; ++kb)
@@ -506,15 +529,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       } else {
         pdl_wait();
       }
-      for (int64_t tile = cluster_id; ok && tile < tiles; tile += n_clusters) {
-        const int m0 = static_cast<int>(tile % m_tiles) * BM + static_cast<int>(rank) * kRowsPerCta;
-        const int n0 = static_cast<int>(tile / m_tiles) * BN + static_cast<int>(rank) * kRowsPerCta;
-        for (int kb = (tile == cluster_id ? pre : 0); kb < k_blocks; ++kb) {
+      for (int64_t q = cluster_id; ok && q < pieces; q += n_clusters) {
+        const Piece pc = piece_of(q, tiles, tail);
+        const int w_rows = pc.nw >> 1;
+        const CUtensorMap* mapB = pc.nw == BN ? &tmB : &tmB64;
+        const uint32_t stage_bytes = kAStageBytes + (uint32_t)w_rows * BK * 2;
+        const int m0 = static_cast<int>(pc.tile % m_tiles) * BM + static_cast<int>(rank) * kRowsPerCta;
+        const int n0 = static_cast<int>(pc.tile / m_tiles) * BN + pc.noff + static_cast<int>(rank) * w_rows;
+        for (int kb = (q == cluster_id ? pre : 0); kb < k_blocks; ++kb) {
           if (!mbar_wait(&empty[stage], phase ^ 1u, g.status)) { ok = false; break; }
           const uint32_t full_leader = mapa(smem_u32(&full[stage]), 0);
-          mbar_expect_tx_cluster(full_leader, kStageBytes);
+          mbar_expect_tx_cluster(full_leader, stage_bytes);
           tma_load_2d(sA + stage * kAStageBytes, &tmA, full_leader, kb * BK, m0);
-          tma_load_2d(sB + stage * kBStageBytes, &tmB, full_leader, kb * BK, n0);
+          tma_load_2d(sB + stage * kBStageBytes, mapB, full_leader, kb * BK, n0);
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
       }
@@ -530,7 +557,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       int stage = 0, acc = 0;
       uint32_t phase = 0, acc_phase = 0;
       bool ok = true;
-      for (int64_t tile = cluster_id; ok && tile < tiles; tile += n_clusters) {
+      for (int64_t q = cluster_id; ok && q < pieces; q += n_clusters) {
+        const uint32_t idesc = instr_desc(piece_of(q, tiles, tail).nw);
         if (!mbar_wait(&tempty[acc], acc_phase ^ 1u, g.status)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN);
@@ -541,7 +569,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           const uint64_t db = make_smem_desc(smem_u32(sB + stage * kBStageBytes));
 #pragma unroll
           for (int k = 0; k < BK / 16; ++k)
-            umma_bf16(d_tmem, da + 2u * k, db + 2u * k, kInstrDesc, (kb | k) != 0 ? 1u : 0u);
+            umma_bf16(d_tmem, da + 2u * k, db + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
           umma_commit_pair(&empty[stage]);
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
@@ -557,15 +585,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmD)) : "memory");
     int acc = 0;
     uint32_t acc_phase = 0;
-    for (int64_t tile = cluster_id; tile < tiles; tile += n_clusters) {
-      const int64_t m0 = (tile % m_tiles) * BM + rank * kRowsPerCta, n0 = (tile / m_tiles) * BN;
+    for (int64_t q = cluster_id; q < pieces; q += n_clusters) {
+      const Piece pc = piece_of(q, tiles, tail);
+      const int64_t m0 = (pc.tile % m_tiles) * BM + rank * kRowsPerCta, n0 = (pc.tile / m_tiles) * BN + pc.noff;
       if (!mbar_wait(&tfull[acc], acc_phase, g.status)) break;
       tc_fence_after();
       const int row0 = static_cast<int>(m0) + quad * 32;
       const int col0 = static_cast<int>(n0) + cgrp * kColsPerEpiWarp;
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) +
                              static_cast<uint32_t>(acc * BN + cgrp * kColsPerEpiWarp);
-      if (row0 < M_rows && (col0 < g.N || EPI == kEpiArgmax)) epilogue_columns<EPI>(g, &tmD, buf, lane, taddr, row0, col0);
+      // (a half piece fills the first 128 accumulator columns: the warps of the other two column groups only arrive)
+      if (cgrp * kColsPerEpiWarp < pc.nw && row0 < M_rows && (col0 < g.N || EPI == kEpiArgmax))
+        epilogue_columns<EPI>(g, &tmD, buf, lane, taddr, row0, col0);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(mapa(smem_u32(&tempty[acc]), 0));

@@ -563,24 +563,37 @@ int ensure_tc_ready(srm_model& m) {
   return SRM_OK;
 }
 
+// How many of the last tiles of a launch run as two half-width pieces (gemm_tc.cuh): the r tiles of a last, partly
+// filled round when their 2 r halves still fit in one round (they then end after three quarters of a tile's time
+// with nearly every pair busy); none with SRM_FLAG_NO_TAIL_SPLIT.
+int gemm_tail_tiles(const srm_model& m, int64_t tiles) {
+  if (m.cfg.flags & SRM_FLAG_NO_TAIL_SPLIT) return 0;
+  const int64_t r = tiles % m.tc_clusters;
+  return (r > 0 && 2 * r <= m.tc_clusters) ? (int)r : 0;
+}
+
 int launch_gemm_tc(srm_model& m, int epi, int64_t M, int64_t N, int64_t K, const void* A, const void* W,
                    const float* bias, void* out, uint32_t* status, cudaStream_t st) {
   int rc = ensure_tc_ready(m);
   if (rc != SRM_OK) return rc;
-  CUtensorMap ta, tb, td;
+  CUtensorMap ta, tb, td, tb64;
   if ((rc = m.tmap(A, M, K, tc::kRowsPerCta, 2, &ta)) != SRM_OK) return rc;
   if ((rc = m.tmap(W, N, K, tc::kRowsPerCta, 2, &tb)) != SRM_OK) return rc;
+  if ((rc = m.tmap(W, N, K, tc::kHalfN / 2, 2, &tb64)) != SRM_OK) return rc;      // W rows of a half-width piece
   if (epi == kEpiArgmax) td = ta;       // no output matrix: the descriptor is not used
   else if ((rc = m.tmap(out, M, N, tc::kOutBoxRows, epi == kEpiBiasGelu ? 2 : 4, &td)) != SRM_OK) return rc;
   const uint8_t* wb = static_cast<const uint8_t*>(W);
   const int w_static = wb >= m.w && wb < m.w + m.layout.total;      // inside the weight blob
-  tc::GemmArgs g{M, N, K, bias, out, status, w_static};
   const int64_t tiles = ((M + tc::BM - 1) / tc::BM) * ((N + tc::BN - 1) / tc::BN);
-  const unsigned grid = 2u * (unsigned)(tiles < m.tc_clusters ? tiles : m.tc_clusters);
-  if (epi == kEpiBiasGelu) SRM_CUDA(launch_kernel(tc::gemm_tc_kernel<kEpiBiasGelu>, dim3(grid), dim3(tc::kThreads), tc::kSmemBytes, st, ta, tb, td, g));
-  else if (epi == kEpiBiasResidual) SRM_CUDA(launch_kernel(tc::gemm_tc_kernel<kEpiBiasResidual>, dim3(grid), dim3(tc::kThreads), tc::kSmemBytes, st, ta, tb, td, g));
-  else if (epi == kEpiArgmax) SRM_CUDA(launch_kernel(tc::gemm_tc_kernel<kEpiArgmax>, dim3(grid), dim3(tc::kThreads), tc::kSmemBytes, st, ta, tb, td, g));
-  else SRM_CUDA(launch_kernel(tc::gemm_tc_kernel<kEpiPlain>, dim3(grid), dim3(tc::kThreads), tc::kSmemBytes, st, ta, tb, td, g));
+  const int tail = gemm_tail_tiles(m, tiles);
+  tc::GemmArgs g{M, N, K, bias, out, status, w_static};
+  g.tail_tiles = tail;
+  const int64_t pieces = tiles + tail;
+  const unsigned grid = 2u * (unsigned)(pieces < m.tc_clusters ? pieces : m.tc_clusters);
+  if (epi == kEpiBiasGelu) SRM_CUDA(launch_kernel(tc::gemm_tc_kernel<kEpiBiasGelu>, dim3(grid), dim3(tc::kThreads), tc::kSmemBytes, st, ta, tb, td, tb64, g));
+  else if (epi == kEpiBiasResidual) SRM_CUDA(launch_kernel(tc::gemm_tc_kernel<kEpiBiasResidual>, dim3(grid), dim3(tc::kThreads), tc::kSmemBytes, st, ta, tb, td, tb64, g));
+  else if (epi == kEpiArgmax) SRM_CUDA(launch_kernel(tc::gemm_tc_kernel<kEpiArgmax>, dim3(grid), dim3(tc::kThreads), tc::kSmemBytes, st, ta, tb, td, tb64, g));
+  else SRM_CUDA(launch_kernel(tc::gemm_tc_kernel<kEpiPlain>, dim3(grid), dim3(tc::kThreads), tc::kSmemBytes, st, ta, tb, td, tb64, g));
   SRM_CUDA(cudaGetLastError());
   return SRM_OK;
 }
@@ -742,10 +755,13 @@ int launch_lm_head_topk(srm_model& m, int64_t R, const void* a, void* lists, voi
     LaunchScope scope(m, SRM_KERNEL_GEMM_LM, st);
     if ((rc = m.tmap(a, R, d, tc::kRowsPerCta, 2, &ta)) != SRM_OK) return rc;
     if ((rc = m.tmap(m.ptr(-1, SRM_T_W_LM), V, d, tc::kRowsPerCta, 2, &tb)) != SRM_OK) return rc;
-    tc::GemmArgs g{R, V, d, nullptr, lists, status, 1, thr, cnt, kFusedTopkCap, nullptr};
+    CUtensorMap tb64;
+    if ((rc = m.tmap(m.ptr(-1, SRM_T_W_LM), V, d, tc::kHalfN / 2, 2, &tb64)) != SRM_OK) return rc;
     const int64_t tiles = ((R + tc::BM - 1) / tc::BM) * ((V + tc::BN - 1) / tc::BN);
-    const unsigned grid = 2u * (unsigned)(tiles < m.tc_clusters ? tiles : m.tc_clusters);
-    SRM_CUDA(launch_kernel(tc::gemm_tc_kernel<kEpiCollect>, dim3(grid), dim3(tc::kThreads), tc::kSmemBytes, st, ta, tb, ta, g));
+    tc::GemmArgs g{R, V, d, nullptr, lists, status, 1, thr, cnt, kFusedTopkCap, nullptr, gemm_tail_tiles(m, tiles)};
+    const int64_t pieces = tiles + g.tail_tiles;
+    const unsigned grid = 2u * (unsigned)(pieces < m.tc_clusters ? pieces : m.tc_clusters);
+    SRM_CUDA(launch_kernel(tc::gemm_tc_kernel<kEpiCollect>, dim3(grid), dim3(tc::kThreads), tc::kSmemBytes, st, ta, tb, ta, tb64, g));
   }
   {
     LaunchScope scope(m, SRM_KERNEL_SELECT, st);
@@ -760,10 +776,10 @@ int launch_lm_head_topk(srm_model& m, int64_t R, const void* a, void* lists, voi
     CUtensorMap tf, td;
     if ((rc = m.tmap(a_fb, R, d, tc::kRowsPerCta, 2, &tf)) != SRM_OK) return rc;
     if ((rc = m.tmap(lists, R, V, tc::kOutBoxRows, 4, &td)) != SRM_OK) return rc;
-    tc::GemmArgs g{R, V, d, nullptr, lists, status, 0, nullptr, nullptr, 0, n_fb};
+    tc::GemmArgs g{R, V, d, nullptr, lists, status, 0, nullptr, nullptr, 0, n_fb, 0};
     const int64_t tiles = ((R + tc::BM - 1) / tc::BM) * ((V + tc::BN - 1) / tc::BN);
     const unsigned grid = 2u * (unsigned)(tiles < m.tc_clusters ? tiles : m.tc_clusters);
-    SRM_CUDA(launch_kernel(tc::gemm_tc_kernel<kEpiPlain>, dim3(grid), dim3(tc::kThreads), tc::kSmemBytes, st, tf, tb, td, g));
+    SRM_CUDA(launch_kernel(tc::gemm_tc_kernel<kEpiPlain>, dim3(grid), dim3(tc::kThreads), tc::kSmemBytes, st, tf, tb, td, tb, g));
   }
   {
     LaunchScope scope(m, SRM_KERNEL_SELECT, st);

@@ -110,7 +110,8 @@ def _gemm_case(m, M, N, K, epi, act, seed=0):
 
 
 @pytest.mark.parametrize("M,N,K", [(128, 256, 64), (256, 512, 128), (1, 256, 64), (300, 1000, 192),
-                                   (77, 8000, 512), (520, 264, 1024), (4096, 1024, 4096)])
+                                   (77, 8000, 512), (520, 264, 1024), (4096, 1024, 4096), (4096, 4096, 1024),
+                                   (2048, 1024, 512)])
 @pytest.mark.parametrize("epi", [0, 1, 2])
 def test_tensor_core_gemm_matches_fp64_matmul(M, N, K, epi):
     shape = custom_shape(d_model=64, dtype="bf16")
@@ -151,6 +152,24 @@ def test_epilogue_gelu_alone_against_the_erf_form():
     assert np.all(np.abs(got - want) <= bound), float(np.max(np.abs(got - want) - bound))
     want_bf16 = torch.from_numpy(want.astype(np.float32)).to(torch.bfloat16).float().numpy().astype(np.float64)
     assert np.mean(got == want_bf16) > 0.55
+
+
+@pytest.mark.parametrize("M,N,K", [(4096, 4096, 1024),      # 256 tiles on 74 pairs: the last 34 run as 68 half-width pieces
+                                   (2048, 1024, 512),       # 32 tiles: all of them as 64 half-width pieces
+                                   (300, 1000, 192),        # ragged N: the second half of the last tile is mostly padding
+                                   (77, 8000, 512), (4096, 1024, 4096)])      # (the last: 64 tiles, no split)
+def test_half_width_tail_pieces_change_no_bit(M, N, K):
+    """The tiles of a partly filled last round run as two 256 x 128 pieces each. Every output element is still one
+    sum over K in the same order, so all epilogues must give exactly the bits of whole tiles, and the fused greedy
+    selection the same tokens."""
+    import paper_2605_08696_b200 as P
+    shape = custom_shape(d_model=64, dtype="bf16")
+    m_split, _ = _model(shape)
+    m_whole, _ = _model(shape, flags=P.FLAG_NO_TAIL_SPLIT)
+    for epi in (0, 1, 2):
+        a, _ = _gemm_case(m_split, M, N, K, epi, torch.bfloat16, seed=5)
+        b, _ = _gemm_case(m_whole, M, N, K, epi, torch.bfloat16, seed=5)
+        assert np.array_equal(a, b), epi
 
 
 def test_tensor_core_gemm_equals_simt_gemm_on_device():
