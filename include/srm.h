@@ -416,6 +416,12 @@ int srm_k_select(srm_model* m, int64_t R, const float* d_logits, const srm_sampl
 int srm_k_prefill_mixer(srm_model* m, int32_t layer, int64_t Bp, int32_t n, const int32_t* d_tok,
                         float* d_x, void* d_S, void* d_a, uint32_t* d_status, void* stream);
 
+/* Failure-detection check without a fault: launches one thread that waits, with the bounded wait all pipelines of
+ * this library use, on a barrier that nothing completes. After limit_cycles (1 .. 2^31 SM clock cycles) the wait
+ * gives up, SRM_STATUS_WAIT_TIMEOUT is raised in *d_status, *d_gave_up (may be NULL) is set to 1 and the kernel ends;
+ * the context stays usable. Asynchronous on `stream`. */
+int srm_k_wait_probe(uint32_t* d_status, int64_t limit_cycles, int32_t* d_gave_up, void* stream);
+
 /* ---- measurement -------------------------------------------------------------------------- */
 enum srm_kernel_class {
   SRM_KERNEL_MIXER = 0,          /* fused recurrent token-mixer step                           */

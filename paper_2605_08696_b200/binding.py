@@ -115,6 +115,7 @@ SYMBOLS = {
     "srm_k_lm_head_greedy": (C.c_int, [_P, _I64, _P, _P, _SZ, _P, _P, _P]),
     "srm_k_select": (C.c_int, [_P, _I64, _P, C.POINTER(_Sampling), _I32, _P, _P, _P]),
     "srm_k_prefill_mixer": (C.c_int, [_P, _I32, _I64, _I32, _P, _P, _P, _P, _P, _P]),
+    "srm_k_wait_probe": (C.c_int, [_P, _I64, _P, _P]),
     "srm_profile_enable": (C.c_int, [_P, C.c_int]),
     "srm_profile_read": (C.c_int, [_P, _I32, C.POINTER(C.c_uint64), C.POINTER(C.c_double)]),
     "srm_profile_reset": (C.c_int, [_P]),
@@ -174,6 +175,11 @@ def _shape_opt(shape, key, default):
 
 def _shape_get(shape, key):
     return shape[key] if isinstance(shape, dict) else getattr(shape, key)
+
+
+def k_wait_probe(status: torch.Tensor, limit_cycles: int, gave_up: torch.Tensor | None = None):
+    """A bounded wait on a barrier that nothing completes: must give up after limit_cycles and raise the status bit."""
+    _check(_lib().srm_k_wait_probe(_ptr(status), limit_cycles, _ptr(gave_up), _stream()), "srm_k_wait_probe")
 
 
 def k_mixer_combined_step(t, z, S_row, S_col, alpha_row, alpha_col, beta, lam_row, lam_col, w, y):

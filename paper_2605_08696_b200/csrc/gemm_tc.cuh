@@ -82,18 +82,33 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait. Returns false (after raising the status bit) when the phase never completes.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint32_t* status) {
+// Bounded wait. Returns false (after raising the status bit) when the phase has not completed within `limit` clock
+// cycles (the pipelines use kWaitLimitCycles: far longer than any kernel of this library runs).
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint32_t* status,
+                                          long long limit = kWaitLimitCycles) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (;;) {
 #pragma unroll 1
     for (int i = 0; i < 256; ++i)
       if (mbar_try_wait(bar, parity)) return true;
-    if (clock64() - t0 > kWaitLimitCycles) {
+    if (clock64() - t0 > limit) {
       raise_status(status, kStatusWaitTimeout);
       return false;
     }
+  }
+}
+
+// One thread waits, with the bounded wait every pipeline of this library uses, on an mbarrier phase that nothing
+// ever completes: the wait must give up after `limit` cycles, raise kStatusWaitTimeout and let the kernel end.
+// (The host-visible check that a stuck pipeline cannot hang the GPU.)
+__global__ void wait_probe_kernel(uint32_t* status, long long limit, int* gave_up) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    const bool ok = mbar_wait(&bar, 0u, status, limit);
+    if (gave_up != nullptr) *gave_up = ok ? 0 : 1;
   }
 }
 __device__ __forceinline__ uint32_t cluster_ctarank() {

@@ -462,3 +462,25 @@ def test_prefill_mixer_matches_oracle_parallel_form(d, dtype, n, embed):
         assert rel_err_rows(x[b * n:(b + 1) * n].cpu().numpy(), x1) < 2e-5
         assert rel_err_rows(S[b].cpu().numpy(), Sn) < 2e-5
         assert rel_err_rows(a[b * n:(b + 1) * n].float().cpu().numpy(), a1) < (2e-5 if dtype == "fp32" else 6e-3)
+
+
+def test_a_bounded_wait_that_nothing_completes_gives_up_and_reports():
+    """Failure detection without a fault: a wait on a barrier that nothing completes (the bounded wait of every
+    pipeline of the library, here with a limit of about a millisecond) gives up, raises the wait-time-out bit of the
+    status word and lets the kernel end; the context stays usable (a projection runs and is correct afterwards)."""
+    import time
+    import paper_2605_08696_b200 as P
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    gave_up = torch.full((1,), -1, dtype=torch.int32, device=DEV)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    P.k_wait_probe(status, 2_000_000, gave_up)                  # ~1 ms of SM clocks
+    torch.cuda.synchronize()
+    assert time.perf_counter() - t0 < 1.0
+    assert int(status.item()) == 2 and int(gave_up.item()) == 1  # SRM_STATUS_WAIT_TIMEOUT
+    with pytest.raises(P.SRMError):
+        P.k_wait_probe(status, 0)
+    shape = custom_shape(d_model=64, dtype="bf16")
+    m, _ = _model(shape)
+    got, want = _gemm_case(m, 300, 520, 256, 2, torch.bfloat16, seed=1)
+    assert rel_err_rows(got, want) < 2e-5
