@@ -129,23 +129,35 @@ __global__ void __launch_bounds__(kMixerWarps * 32) mixer_variant_step_kernel(co
   } else {
     // kernels of size k:  v_i = z + P_i ;  y[c] = beta_t[c] + sum_i alpha_i[t] v_i[c + i] (zero past channel d - 1) ;
     //                     P_i <- lam_i v_i
-    float4 z[NV], f[NV];
+    // y starts as x + beta_t (the residual is folded in, so the row itself need not stay in registers); the cache
+    // row of the NEXT filter is loaded before this filter's shuffles, so its latency overlaps them.
+    float4 z[NV], f[NV], nx[NV];
 #pragma unroll
     for (int i = 0; i < NV; ++i) {
       const int c = (i * 32 + lane) * 4;
       z[i] = c < d ? norm4(v[i], mean, rstd, ldg4(p.ln1_g + c), ldg4(p.ln1_b + c)) : zero;
-      y[i] = c < d ? ldg4(beta_t + c) : zero;
+      if (c < d) {
+        const float4 bt = ldg4(beta_t + c);
+        y[i] = make_float4(v[i].x + bt.x, v[i].y + bt.y, v[i].z + bt.z, v[i].w + bt.w);
+      } else {
+        y[i] = zero;
+      }
+      f[i] = c < d ? ld4(S0 + c) : zero;                       // filter 0's cache row
     }
     for (int fi = 0; fi < p.k; ++fi) {
       const float al = __ldg(p.alpha + (int64_t)fi * p.n_ctx + t), lm = __ldg(p.lam + fi);
       ST* Pf = S0 + (int64_t)fi * p.plane;
+      const bool more = fi + 1 < p.k;
 #pragma unroll
       for (int i = 0; i < NV; ++i) {
         const int c = (i * 32 + lane) * 4;
-        f[i] = zero;
+        nx[i] = (more && c < d) ? ld4(Pf + p.plane + c) : zero;
+      }
+#pragma unroll
+      for (int i = 0; i < NV; ++i) {
+        const int c = (i * 32 + lane) * 4;
         if (c < d) {
-          const float4 s = ld4(Pf + c);
-          const float4 w = make_float4(z[i].x + s.x, z[i].y + s.y, z[i].z + s.z, z[i].w + s.w);
+          const float4 w = make_float4(z[i].x + f[i].x, z[i].y + f[i].y, z[i].z + f[i].z, z[i].w + f[i].w);
           st4(Pf + c, make_float4(lm * w.x, lm * w.y, lm * w.z, lm * w.w));
           f[i] = make_float4(al * w.x, al * w.y, al * w.z, al * w.w);
         }
@@ -155,7 +167,11 @@ __global__ void __launch_bounds__(kMixerWarps * 32) mixer_variant_step_kernel(co
         const float4 sh = shifted4<NV>(f, i, fi, lane);
         y[i] = make_float4(y[i].x + sh.x, y[i].y + sh.y, y[i].z + sh.z, y[i].w + sh.w);
       }
+#pragma unroll
+      for (int i = 0; i < NV; ++i) f[i] = nx[i];
     }
+#pragma unroll
+    for (int i = 0; i < NV; ++i) v[i] = y[i];                  // x + y
   }
 
   float* xr = p.x + row * p.x_stride;
@@ -163,7 +179,7 @@ __global__ void __launch_bounds__(kMixerWarps * 32) mixer_variant_step_kernel(co
   for (int i = 0; i < NV; ++i) {
     const int c = (i * 32 + lane) * 4;
     if (c < d) {
-      v[i] = make_float4(v[i].x + y[i].x, v[i].y + y[i].y, v[i].z + y[i].z, v[i].w + y[i].w);
+      if (!KERNEL_MIX) v[i] = make_float4(v[i].x + y[i].x, v[i].y + y[i].y, v[i].z + y[i].z, v[i].w + y[i].w);
       st4(xr + c, v[i]);
     }
   }
