@@ -311,13 +311,14 @@ int srm_decode_step_host(srm_model* m, srm_state* s, const int32_t* h_tok_in,
  * Same arguments and results as srm_decode_step, minus the workspace. Differences:
  *   - the whole batch must fit in one pass: if srm_workspace_bytes(cfg, B, 0) exceeds
  *     SRM_STATIC_SCRATCH_BYTES the call enqueues nothing and returns SRM_ERR_STATIC_SCRATCH
- *     (e.g. the mid model, 142 KB per row, takes up to 236 rows; the tiny model about 14 000);
+ *     (e.g. the mid model, 142 KB per row next to 2.2 MB of fixed scratch, takes up to about 220 rows; the tiny
+ *     model about 13 000);
  *   - the device that is current must be the model's device (else SRM_ERR_INVALID_ARG);
  *   - the first call on each device looks up the array's device address (cudaGetSymbolAddress).
  *     Make that first call outside of any stream capture; later calls only enqueue kernels;
  *   - no cudaMalloc, cudaFree or other allocating routine is called, on any call;
  *   - every call on a device shares the one array. It keeps whatever the previous call left
- *     there; the step overwrites every byte it later reads, so nothing has to be cleared. Two
+ *     there; the step overwrites (or clears, on the stream) every byte it later reads, so the caller has nothing to clear. Two
  *     calls whose GPU work can overlap (different streams, or different host threads without
  *     ordering) race on the array and produce garbage: serialise them on one stream. */
 #define SRM_STATIC_SCRATCH_BYTES (32u << 20)

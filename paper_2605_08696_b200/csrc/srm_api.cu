@@ -463,8 +463,10 @@ int srm_decode_step_static(srm_model* m, srm_state* s, const int32_t* d_tok_in, 
   void* ws = nullptr;
   int rc = static_scratch_address(m->device, &ws);
   if (rc != SRM_OK) return rc;
-  // Nothing in the workspace has to start at zero: the first mixer launch writes x and a, the up
-  // projection writes H, the LM head writes the logits, each before anything reads them.
+  // The caller has nothing to clear: the first mixer launch writes x and a, the up projection writes H, the LM head
+  // writes the logits, each before anything reads them, and the few words that must start at zero (order words of a
+  // split down projection, candidate counters of the fused top-k selection, the grid-barrier word of the small-batch
+  // kernel) are cleared by the step itself with memsets on the stream.
   return decode_step_impl(m, s, d_tok_in, samp, step, d_tok_out, nullptr, 0, 0, d_logits_out, ws,
                           (size_t)SRM_STATIC_SCRATCH_BYTES, static_cast<cudaStream_t>(stream));
 }

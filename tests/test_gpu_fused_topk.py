@@ -117,3 +117,27 @@ def test_k_above_the_fused_limit_takes_the_logits_path():
     for step in (1, 2, 3):
         assert torch.equal(fused.decode_step(st_f, None, samp, step, ws), plain.decode_step(st_p, None, samp, step, ws))
     assert st_f.topk_handed_back() == 0
+
+
+def test_fused_topk_on_the_rollout_model_equals_the_logits_path_over_many_steps():
+    """The rl model (L24 d1536 V32000), replicas of two prompts, 96 free-running sampled steps: thresholds carried
+    from step to step on nearly flat logits; every id equal to the logits path, and after the prefill's thresholds
+    only a few rows per thousand decisions are handed back."""
+    import paper_2605_08696_b200 as P
+    shape = I.CONFIGS["rl"]
+    fused, plain = _pair(shape, weights_for("rl"))
+    reps, n, gen = 12, 200, 96
+    base = torch.from_numpy(I.make_prompts("rl", batch=32)[::2][:2].copy()).to(DEV)      # two distinct prompts
+    B = 2 * reps
+    samp = P.Sampling("topk", 50, 0.8, seed=shape.seed, sample_idx_base=4096)
+    outs = []
+    for model in (fused, plain):
+        st = model.new_state(B)
+        ws = model.new_workspace(B, n, prefill_samples=4)
+        first = model.prefill_replicated(st, base, reps, samp, ws)
+        rest = model.generate(st, gen, 1, samp, ws)
+        outs.append((first.clone(), rest.clone(), st.topk_handed_back()))
+        assert st.status() == 0
+    assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
+    assert outs[1][2] == 0 and outs[0][2] <= 0.01 * B * gen, outs[0][2]
+    assert len({tuple(r.tolist()) for r in outs[0][1][:reps]}) == reps                    # replicas of one prompt diverge
