@@ -470,21 +470,26 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   pdl_trigger();
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  // The selecting epilogues stage nothing in shared memory: their 64 KB of output boxes become two more operand
+  // stages (seven k-blocks in flight per SM instead of five).
+  constexpr bool kNoBoxes = EPI == kEpiArgmax || EPI == kEpiCollect;
+  constexpr int NS = kNoBoxes ? kStages + 2 : kStages;
+  static_assert(NS * kStageBytes + (kNoBoxes ? 0 : kEpiWarps * kOutBoxBytes) + kBarrierBytes + 1024 <= kSmemBytes, "shared memory");
   uint8_t* sA = smem;
-  uint8_t* sB = smem + kStages * kAStageBytes;
-  uint64_t* full = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes + kEpiWarps * kOutBoxBytes);   // used in the leader CTA
-  uint64_t* empty = full + kStages;      // per CTA: stage may be refilled
-  uint64_t* tfull = empty + kStages;     // per CTA [2]: accumulator ready for the epilogue
+  uint8_t* sB = smem + NS * kAStageBytes;
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + NS * kStageBytes + (kNoBoxes ? 0 : kEpiWarps * kOutBoxBytes));   // used in the leader CTA
+  uint64_t* empty = full + NS;           // per CTA: stage may be refilled
+  uint64_t* tfull = empty + NS;     // per CTA [2]: accumulator ready for the epilogue
   uint64_t* tempty = tfull + 2;          // leader [2]: accumulator drained by both CTAs' epilogues
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty + 2);
-  uint8_t* boxes = smem + kStages * kStageBytes;      // 1024-byte aligned, one staging buffer per epilogue warp
+  uint8_t* boxes = smem + NS * kStageBytes;           // 1024-byte aligned, one staging buffer per epilogue warp (not with kNoBoxes)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();           // 0 = leader of the pair
   const int64_t cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 2); mbar_init(&empty[s], 1); }
+    for (int s = 0; s < NS; ++s) { mbar_init(&full[s], 2); mbar_init(&empty[s], 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(&tfull[a], 1); mbar_init(&tempty[a], 2 * kEpiWarps); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -520,7 +525,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       uint32_t phase = 0;
       bool ok = true;
       // While the predecessor kernel drains: start the first tile's W loads (the ring is empty, so
-      // the first kStages stages need no wait), then order against the predecessor and add the A loads.
+      // the first NS stages need no wait), then order against the predecessor and add the A loads.
       int pre = 0;
       if (cluster_id < pieces) {
         const Piece pc = piece_of(cluster_id, tiles, tail);
@@ -529,7 +534,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const uint32_t stage_bytes = kAStageBytes + (uint32_t)w_rows * BK * 2;
         const int m0 = static_cast<int>(pc.tile % m_tiles) * BM + static_cast<int>(rank) * kRowsPerCta;
         const int n0 = static_cast<int>(pc.tile / m_tiles) * BN + pc.noff + static_cast<int>(rank) * w_rows;
-        pre = k_blocks < kStages ? k_blocks : kStages;
+        pre = k_blocks < NS ? k_blocks : NS;
         if (!g.w_static) pdl_wait();
         for (int kb = 0; kb < pre; ++kb) {
           const uint32_t full_leader = mapa(smem_u32(&full[kb]), 0);
@@ -540,7 +545,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         for (int kb = 0; kb < pre; ++kb)
           tma_load_2d(sA + kb * kAStageBytes, &tmA, mapa(smem_u32(&full[kb]), 0), kb * BK, m0);
         stage = pre;
-        if (stage == kStages) { stage = 0; phase ^= 1u; }
+        if (stage == NS) { stage = 0; phase ^= 1u; }
       } else {
         pdl_wait();
       }
@@ -557,7 +562,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           mbar_expect_tx_cluster(full_leader, stage_bytes);
           tma_load_2d(sA + stage * kAStageBytes, &tmA, full_leader, kb * BK, m0);
           tma_load_2d(sB + stage * kBStageBytes, mapB, full_leader, kb * BK, n0);
-          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+          if (++stage == NS) { stage = 0; phase ^= 1u; }
         }
       }
       if (!ok) {
@@ -586,7 +591,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           for (int k = 0; k < BK / 16; ++k)
             umma_bf16(d_tmem, da + 2u * k, db + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
           umma_commit_pair(&empty[stage]);
-          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+          if (++stage == NS) { stage = 0; phase ^= 1u; }
         }
         if (ok) umma_commit_pair(&tfull[acc]);
         if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
