@@ -77,3 +77,18 @@ def test_a_rank_count_that_contradicts_the_flag_is_refused():
     res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--steps", "1"],
                          capture_output=True, text=True, timeout=300, env=env)
     assert res.returncode != 0 and "--gpus 2 but the launcher started 1 rank" in res.stderr
+
+
+def test_traffic_figure_is_read_from_the_profile_summaries_and_dropped_when_the_kernel_changed(tmp_path, monkeypatch):
+    """bench.py takes the DRAM traffic of the dominant kernel from a line in profiles/*.md that names workload, batch
+    and the hash of the GEMM sources it was captured on; no line, another batch or another hash give None."""
+    import bench
+    (tmp_path / "profiles").mkdir()
+    (tmp_path / "profiles" / "x.md").write_text(
+        "text\n    dram_traffic_per_step: workload=mid batch=4096 bytes=1.25e9 gemm_sources=abc123\nmore\n")
+    monkeypatch.setattr(bench, "ROOT", str(tmp_path))
+    monkeypatch.setattr(bench, "gemm_sources_sha", lambda: "abc123")
+    assert bench.dram_traffic_per_step("mid", 4096) == 1.25e9
+    assert bench.dram_traffic_per_step("mid", 8192) is None and bench.dram_traffic_per_step("rl", 4096) is None
+    monkeypatch.setattr(bench, "gemm_sources_sha", lambda: "fff000")
+    assert bench.dram_traffic_per_step("mid", 4096) is None
