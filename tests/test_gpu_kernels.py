@@ -55,6 +55,33 @@ def test_mixer_step_matches_oracle(d, dtype, state_dtype, embed):
     assert rel_err_rows(a.float().cpu().numpy(), a1) < (1e-5 if dtype == "fp32" else 6e-3)
 
 
+@pytest.mark.parametrize("offset", [0.0, 4.0, 50.0, -300.0])
+def test_streaming_mixer_statistics_with_a_large_row_mean(offset):
+    """LayerNorm statistics of rows whose mean is far from zero (0, 4, 50 and -300 standard deviations): the two-pass
+    statistics (mean, then centred squares) keep the fp32 tolerance up to what the fp32 representation of such a
+    row allows (its values carry an absolute rounding of |offset| * 2^-24)."""
+    from oracle import srm_oracle as O
+    shape = custom_shape(n_layers=1, d_model=1024, vocab=512, n_ctx=40, dtype="bf16", seed=3)
+    m, W = _model(shape)
+    rng = np.random.default_rng(17)
+    R, t = 300, 9
+    lw = {k: np.asarray(v, np.float64) for k, v in W["layers"][0].items()}
+    x0 = (rng.normal(size=(R, 1024)) + offset).astype(np.float32)
+    S0 = rng.normal(size=(R, 1024)).astype(np.float32)
+    x, S = _t(x0), _t(S0)
+    a = torch.zeros(R, 1024, dtype=torch.bfloat16, device=DEV)
+    m.k_mixer_step(0, t, x, S, a)
+    torch.cuda.synchronize()
+    z = O.layer_norm(x0.astype(np.float64), lw["ln1_g"], lw["ln1_b"], shape.ln_eps)
+    y, S1 = O.mixer_recurrent_step(z, S0.astype(np.float64), t, lw["alpha"], lw["beta"], lw["lam"], shape.n_heads)
+    x1 = x0.astype(np.float64) + y
+    a1 = O.layer_norm(x1, lw["ln2_g"], lw["ln2_b"], shape.ln_eps)
+    tol = 1e-5 * max(1.0, abs(offset) / 50.0)
+    assert rel_err_rows(S.cpu().numpy(), S1) < tol
+    assert rel_err_rows(x.cpu().numpy(), x1) < 1e-5
+    assert rel_err_rows(a.float().cpu().numpy(), a1) < 6e-3          # bf16 output
+
+
 def test_mixer_step_zero_rows_and_token_clamp():
     shape = custom_shape(d_model=64, vocab=256)
     m, W = _model(shape)
