@@ -184,7 +184,9 @@ int32_t srm_cache_planes(const srm_config* cfg);
  * workspace at least this large for B_chunk = 1 and split the batch into as many passes as
  * the given workspace requires. Decode never uses more than 12288 rows of it in one pass: a larger
  * batch runs as equal passes of at most 10240 rows (whole 256-row tiles), which keeps a layer's
- * activations in L2 between its kernels; results do not depend on the split. */
+ * activations in L2 between its kernels; results do not depend on the split (one exception: a batch of at most 64
+ * samples whose workspace holds it in one pass takes the single-kernel step, see SRM_FLAG_NO_SMALL_BATCH, whose
+ * sums run in another order than those of the kernel-per-operation path). */
 size_t srm_workspace_bytes(const srm_config* cfg, int64_t B_chunk, int32_t n_prefill_max);
 /* Rows per decode pass that a batch of B samples is processed in when the workspace has room for
  * `ws_rows` rows (the rule stated above; host only, no device work). 0 if B < 1 or ws_rows < 1. */
