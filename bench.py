@@ -37,7 +37,7 @@ def gemm_sources_sha():
     kernel it was taken on."""
     import hashlib
     h = hashlib.sha256()
-    for f in ("gemm_tc.cuh", "gemm_tc_splitk.cuh"):
+    for f in ("gemm_tc.cuh", "gemm_tc_splitk.cuh", "ffn_fused.cuh", "ffn_plan.h"):
         with open(os.path.join(ROOT, "paper_2605_08696_b200", "csrc", f), "rb") as fh:
             h.update(fh.read())
     return h.hexdigest()[:12]
@@ -357,7 +357,8 @@ def run_ours(args):
     W = I.make_weights(shape)
     model = P.SRM(shape, W, device=dev, state_dtype=args.state_dtype,
                   flags={"auto": 0, "on": P.FLAG_GRAPH, "off": P.FLAG_NO_GRAPH}[args.graph] |
-                  (P.FLAG_NO_SPLITK if args.no_splitk else 0) | (P.FLAG_NO_TAIL_SPLIT if args.no_tail_split else 0))
+                  (P.FLAG_NO_SPLITK if args.no_splitk else 0) | (P.FLAG_NO_TAIL_SPLIT if args.no_tail_split else 0) |
+                  (P.FLAG_NO_FUSED_FFN if args.no_fused_ffn else 0))
     sidx0 = rank_plan(rank, world, B)["sample_idx_base"]
     samp = {"greedy": lambda: P.Sampling("greedy"),
             "topk": lambda: P.Sampling("topk", w["top_k"], w["temperature"], seed=shape.seed, sample_idx_base=sidx0),
@@ -483,7 +484,7 @@ def run_ours(args):
     prof = model.profile_read()
     d, L, V, F = shape.d_model, shape.n_layers, shape.vocab, shape.d_ffn
     single_kernel = prof["step_small"][0] > 0          # small batch: the whole step is one kernel (dense work included)
-    gemm_classes = ("step_small",) if single_kernel else ("gemm_up", "gemm_down", "gemm_lm", "gemm_proj")
+    gemm_classes = ("step_small",) if single_kernel else ("ffn", "gemm_up", "gemm_down", "gemm_lm", "gemm_proj")
     gemm_ms = sum(prof[k][1] for k in gemm_classes)
     gemm_launches = sum(prof[k][0] for k in gemm_classes)
     gemm_flops = prof_steps * B * step_flops(shape)
@@ -496,8 +497,11 @@ def run_ours(args):
     kernels = {k: {"launches": v[0], "ms_total": round(v[1], 3), "share": round(v[1] / prof_total, 4) if prof_total else 0}
                for k, v in prof.items() if v[0]}
     if not single_kernel:
-        kernels["gemm_up"]["tflops"] = round(prof_steps * L * B * 2 * d * F / (prof["gemm_up"][1] / 1e3) / 1e12, 1)
-        kernels["gemm_down"]["tflops"] = round(prof_steps * L * B * 2 * d * F / (prof["gemm_down"][1] / 1e3) / 1e12, 1)
+        if "ffn" in kernels:             # up and down projection of a layer in one kernel
+            kernels["ffn"]["tflops"] = round(prof_steps * L * B * 4 * d * F / (prof["ffn"][1] / 1e3) / 1e12, 1)
+        if "gemm_up" in kernels:
+            kernels["gemm_up"]["tflops"] = round(prof_steps * L * B * 2 * d * F / (prof["gemm_up"][1] / 1e3) / 1e12, 1)
+            kernels["gemm_down"]["tflops"] = round(prof_steps * L * B * 2 * d * F / (prof["gemm_down"][1] / 1e3) / 1e12, 1)
         kernels["gemm_lm"]["tflops"] = round(prof_steps * B * 2 * d * V / (prof["gemm_lm"][1] / 1e3) / 1e12, 1)
         if shape.head_proj:
             kernels["gemm_proj"]["tflops"] = round(prof_steps * L * B * 4 * d * d / (prof["gemm_proj"][1] / 1e3) / 1e12, 1)
@@ -546,7 +550,7 @@ def run_ours(args):
                     "peak_source": f"hbm_gbs, {peak_src}", "launches": int(gemm_launches), "steps_profiled": prof_steps,
                     "traffic": None, "bytes_per_step": step_bytes}
     else:
-        roofline = {"bound": "tensor", "kernel": "gemm_tc_kernel (feed-forward up/down + LM head)",
+        roofline = {"bound": "tensor", "kernel": "ffn_fused_kernel + gemm_tc_kernel (feed-forward up/down + LM head)" if prof["ffn"][0] else "gemm_tc_kernel (feed-forward up/down + LM head)",
                     "achieved": round(achieved_tf, 1), "peak": peak_tf, "unit": "TFLOP/s",
                     "frac": round(achieved_tf / peak_tf, 4), "peak_source": f"bf16_tflops_sustained, {peak_src}",
                     "frac_of_burst_peak": round(achieved_tf / peaks["bf16_tflops"], 4),
@@ -759,6 +763,8 @@ def main():
                     help="token mixer of the model: mixed heads (the hot path), linearly combined heads (twice the cache) "
                          "or kernels of size --kernel-size (Eq. 11; that many times the cache)")
     ap.add_argument("--kernel-size", type=int, default=4)
+    ap.add_argument("--no-fused-ffn", action="store_true",
+                    help="feed-forward block as two launches (up projection, down projection) instead of one kernel")
     ap.add_argument("--no-tail-split", action="store_true",
                     help="tensor-core projections keep the tiles of a partly filled last round whole (256 x 256)")
     ap.add_argument("--no-splitk", action="store_true",

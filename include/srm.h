@@ -76,6 +76,11 @@ enum {
   SRM_FLAG_NO_TAIL_SPLIT = 128,      /* tensor-core projections process every 256 x 256 tile whole (default: the tiles of a
                                         last, partly filled round run as two 256 x 128 pieces each, which keeps nearly all
                                         CTA pairs busy to the end); for comparison and measurement */
+  SRM_FLAG_NO_FUSED_FFN = 256,       /* the feed-forward block of a decode step always runs as two launches, up projection
+                                        then down projection (default, bf16 models whose d is a multiple of 256, passes
+                                        of at most 16384 rows with at least one and a half 256 x 256 tiles per CTA pair:
+                                        ONE kernel computes the tiles of both projections, see srm_k_ffn; same results
+                                        bit for bit); for comparison and measurement */
   SRM_FLAG_HEAD_PROJ = 2             /* token mixer with head projections [Method/Architecture, Eq. 10]:
                                         q = W_in LN1(x) (W_in stacks the per-head I_g), heads of q mixed, and
                                         x += W_out (concatenated heads); the cache holds projected values.
@@ -400,6 +405,30 @@ int srm_k_gemm_splitk(srm_model* m, int64_t M, int64_t N, int64_t K, const void*
  * arithmetic: needs no device. */
 int64_t srm_k_gemm_splitk_plan(int64_t M, int64_t N, int64_t K, int32_t pairs, int32_t pair,
                                int64_t* pieces, int64_t max_pieces);
+/* The feed-forward block of layer `layer` on M rows as one kernel [Method/Architecture: the channel-mixing
+ * feed-forward that follows the token mixer]: H = gelu(a W1^T + b1), x += H W2^T + b2. d_a [M, d] bf16 in, d_H [M, F]
+ * bf16 out (scratch of the block), d_x [M, d] fp32 in/out. The 256 x 256 tiles of BOTH projections are dealt to the
+ * CTA pairs by a host-made plan (srm_k_ffn_plan); a down tile reads H column tile after column tile along its K
+ * dimension and waits, per column tile, for a counter the epilogue warps of that up tile raise, so pairs with a down
+ * tile start it while other pairs still compute up tiles of the same rows, and no pair idles through the down
+ * projection. Results equal srm_k_gemm (epilogue 0) followed by srm_k_gemm (epilogue 1) bit for bit. d_ready: scratch
+ * of srm_k_ffn_ready_bytes(M, F) bytes, 256-byte aligned, cleared by the call. The CTA pairs of the launch wait for
+ * one another: do not run it concurrently with other work on the same device (it then may time out: status bit
+ * SRM_STATUS_WAIT_TIMEOUT, result invalid). SRM_ERR_UNSUPPORTED: not a bf16 tensor-core model, d or F not a multiple of
+ * 256, more than 16384 rows or more than 2048 tiles. This is what srm_decode_step and srm_generate run per layer
+ * for passes with at least one and a half tiles per CTA pair (mid model: from 1536 rows), unless
+ * SRM_FLAG_NO_FUSED_FFN is set. */
+size_t srm_k_ffn_ready_bytes(int64_t M, int64_t F);
+int srm_k_ffn(srm_model* m, int32_t layer, int64_t M, const void* d_a, void* d_H, float* d_x, void* d_ready,
+              size_t ready_bytes, uint32_t* d_status, void* stream);
+/* The work lists of srm_k_ffn for M rows of a model of width d and hidden width F on `pairs` CTA pairs, written to
+ * HOST arrays: off[pairs + 1] (pair c owns items off[c] .. off[c + 1] - 1, in this order) and up to max_items items
+ * of three int32 {0 = up tile / 1 = down tile, row block, column tile}. Returns the number of items (every tile of
+ * both projections exactly once), or a negative SRM_ERR_*. *makespan / *ideal (may be NULL): the plan's length and
+ * the even-share lower bound under the cost model of the planner, in k-block times. Pure host arithmetic: needs no
+ * device. */
+int64_t srm_k_ffn_plan(int64_t M, int32_t d, int32_t F, int32_t pairs, int32_t* off, int32_t* items, int64_t max_items,
+                       double* makespan, double* ideal);
 /* LM head with greedy selection fused into the GEMM epilogue (bf16 models only): d_tok[r] =
  * argmax_v (a[r, :] . W_lm[v, :]), lowest id among equal maxima - the token srm_k_gemm (epilogue 2)
  * followed by greedy srm_k_select gives, without writing the R x V logits. d_a [R, d] in the
@@ -436,6 +465,7 @@ enum srm_kernel_class {
   SRM_KERNEL_PREFILL_MIXER,      /* sequence-parallel token mixing                             */
   SRM_KERNEL_GEMM_PROJ,          /* head projections W_in, W_out (SRM_FLAG_HEAD_PROJ)          */
   SRM_KERNEL_STEP_SMALL,         /* the single-kernel decode step of a small batch             */
+  SRM_KERNEL_FFN,                /* feed-forward block as one kernel (up and down projection)  */
   SRM_KERNEL_CLASS_COUNT
 };
 /* While enabled, every kernel launch of this model is bracketed by two CUDA events recorded on the

@@ -24,6 +24,7 @@ FLAG_NO_SPLITK = 16
 FLAG_NO_FUSED_TOPK = 32
 FLAG_NO_SMALL_BATCH = 64
 FLAG_NO_TAIL_SPLIT = 128
+FLAG_NO_FUSED_FFN = 256
 # enum srm_error
 ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_BUFFER_TOO_SMALL, ERR_CTX_OVERFLOW, ERR_CUDA, \
     ERR_DEVICE_STATUS, ERR_STATIC_SCRATCH = -1, -2, -3, -4, -5, -6, -7, -8
@@ -108,6 +109,10 @@ SYMBOLS = {
     "srm_k_gemm_splitk_order_bytes": (_SZ, [_I64, _I64]),
     "srm_k_gemm_splitk": (C.c_int, [_P, _I64, _I64, _I64, _P, _P, _P, _P, _P, _SZ, _P, _P]),
     "srm_k_gemm_splitk_plan": (_I64, [_I64, _I64, _I64, _I32, _I32, C.POINTER(_I64), _I64]),
+    "srm_k_ffn_ready_bytes": (_SZ, [_I64, _I64]),
+    "srm_k_ffn": (C.c_int, [_P, _I32, _I64, _P, _P, _P, _P, _SZ, _P, _P]),
+    "srm_k_ffn_plan": (_I64, [_I64, _I32, _I32, _I32, C.POINTER(_I32), C.POINTER(_I32), _I64, C.POINTER(C.c_double),
+                              C.POINTER(C.c_double)]),
     "srm_k_mixer_combined_step": (C.c_int, [_I64, _I32, _I32, _I32, _I32] + [_P] * 11),
     "srm_k_mixer_kernel_step": (C.c_int, [_I64, _I32, _I32, _I32, _I32] + [_P] * 7),
     "srm_k_mixer_combined_scan": (C.c_int, [_I64, _I32, _I32, _I32, _I32, _I32] + [_P] * 11),
@@ -175,6 +180,20 @@ def _shape_opt(shape, key, default):
 
 def _shape_get(shape, key):
     return shape[key] if isinstance(shape, dict) else getattr(shape, key)
+
+
+def k_ffn_plan(M: int, d: int, F: int, pairs: int):
+    """Work lists of the fused feed-forward kernel (host arithmetic only): returns (lists, makespan, ideal) where
+    lists[c] is pair c's sequence of (down, row_block, column_tile)."""
+    off = (_I32 * (pairs + 1))()
+    n = _lib().srm_k_ffn_plan(M, d, F, pairs, off, None, 0, None, None)
+    if n < 0:
+        raise SRMError(int(n), "srm_k_ffn_plan")
+    items = (_I32 * (3 * n))()
+    mk, ideal = C.c_double(), C.c_double()
+    _check(min(0, _lib().srm_k_ffn_plan(M, d, F, pairs, off, items, n, C.byref(mk), C.byref(ideal))), "srm_k_ffn_plan")
+    lists = [[(items[3 * i], items[3 * i + 1], items[3 * i + 2]) for i in range(off[c], off[c + 1])] for c in range(pairs)]
+    return lists, mk.value, ideal.value
 
 
 def k_wait_probe(status: torch.Tensor, limit_cycles: int, gave_up: torch.Tensor | None = None):
@@ -452,7 +471,7 @@ class SRM:
 
     # ---- measurement ----
     KERNEL_CLASSES = ("mixer", "gemm_up", "gemm_down", "gemm_lm", "norm", "select", "prefill_mixer", "gemm_proj",
-                      "step_small")
+                      "step_small", "ffn")
 
     def profile(self, on: bool):
         _check(_lib().srm_profile_enable(self.handle, int(on)), "srm_profile_enable")
@@ -495,6 +514,14 @@ class SRM:
             order = torch.empty(_lib().srm_k_gemm_splitk_order_bytes(M, N), dtype=torch.uint8, device=A.device)
         _check(_lib().srm_k_gemm_splitk(self.handle, M, N, K, _ptr(A), _ptr(W), _ptr(bias), _ptr(out), _ptr(order),
                                         order.numel() * order.element_size(), _ptr(status), _stream()), "srm_k_gemm_splitk")
+
+    def k_ffn(self, layer, a, H, x, ready=None, status=None):
+        """The feed-forward block of one layer as one kernel: H = gelu(a W1^T + b1), x += H W2^T + b2."""
+        M = a.shape[0]
+        if ready is None:
+            ready = torch.empty(_lib().srm_k_ffn_ready_bytes(M, H.shape[1]), dtype=torch.uint8, device=a.device)
+        _check(_lib().srm_k_ffn(self.handle, layer, M, _ptr(a), _ptr(H), _ptr(x), _ptr(ready),
+                                ready.numel() * ready.element_size(), _ptr(status), _stream()), "srm_k_ffn")
 
     def k_lm_head_greedy(self, a, part, tok, status=None):
         _check(_lib().srm_k_lm_head_greedy(self.handle, a.shape[0], _ptr(a), _ptr(part), part.numel() * part.element_size(),

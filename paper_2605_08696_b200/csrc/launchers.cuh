@@ -183,6 +183,7 @@ int ensure_tc_ready(srm_model& m) {
   SRM_CUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<kEpiArgmax>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes));
   SRM_CUDA(cudaFuncSetAttribute(tc::gemm_tc_kernel<kEpiCollect>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes));
   SRM_CUDA(cudaFuncSetAttribute(tc::gemm_tc_splitk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes));
+  SRM_CUDA(cudaFuncSetAttribute(tc::ffn_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes));
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(2 * (m.num_sms / 2));
   cfg.blockDim = dim3(tc::kThreads);
@@ -268,6 +269,66 @@ int launch_gemm_splitk(srm_model& m, int64_t M, int64_t N, int64_t K, const void
   tc::SplitArgs g{M, N, K, bias, status, order, w_static};
   SRM_CUDA(launch_kernel(tc::gemm_tc_splitk_kernel, dim3(2u * (unsigned)P.pairs), dim3(tc::kThreads), tc::kSmemBytes, st,
                          ta, tb, td, g, P));
+  SRM_CUDA(cudaGetLastError());
+  return SRM_OK;
+}
+
+// ---- the feed-forward block as one kernel (ffn_fused.cuh) --------------------------------------
+tc::FfnShape ffn_shape(int64_t M, int d, int64_t F) {
+  return tc::FfnShape{(int)((M + tc::BM - 1) / tc::BM), (int)(F / tc::BN), d / tc::BK, d / tc::BN, (int)(F / tc::BK)};
+}
+size_t ffn_ready_bytes(int64_t M, int64_t F) { return align_up((size_t)((M + tc::BM - 1) / tc::BM) * (size_t)(F / tc::BN) * 4, 256); }
+
+// Whether M rows of this model can take the fused kernel (shape limits of the plan and of whole 256-wide tiles).
+bool ffn_fused_shape_ok(const srm_model& m, int64_t M) {
+  const srm_config& c = m.cfg;
+  if (c.dtype != SRM_DTYPE_BF16 || (c.flags & SRM_FLAG_SIMT_GEMM)) return false;
+  const int64_t F = m.F();
+  if (c.d_model % tc::BN || F % tc::BN || M < 1 || M > (int64_t)tc::kFfnMaxRb * tc::BM) return false;
+  return tc::ffn_shape_ok(ffn_shape(M, c.d_model, F), 2);
+}
+
+// Whether the decode step takes it for a pass of M rows: from one and a half tiles per CTA pair. With fewer the chain
+// up tile -> epilogue -> counter -> down tile is longer than two launches that overlap through programmatic dependent
+// launch. Measured on the mid model (74 pairs, 20 tiles per 256 rows), one kernel against two launches, ms per step:
+// 512 rows 0.73 / 0.64, 1024: 0.76 / 0.71, 1536: 0.80 / 0.81, 2048: 0.89 / 0.93, 3072: 1.14 / 1.24, 4096: 1.47 / 1.51.
+bool ffn_fused_worthwhile(const srm_model& m, int64_t M) {
+  const tc::FfnShape s = ffn_shape(M, m.cfg.d_model, m.F());
+  return m.tc_clusters >= 2 && 2 * (int64_t)s.Rb * (s.Cu + s.Cd) >= 3 * (int64_t)m.tc_clusters;
+}
+
+// `ready`: ffn_ready_bytes(M, F) bytes of zeroed words. SRM_ERR_UNSUPPORTED: take the two launches.
+int launch_ffn_fused(srm_model& m, int layer, int64_t M, const void* a, void* H, float* x, int32_t* ready, uint32_t* status,
+                     cudaStream_t st) {
+  if (M <= 0) return SRM_OK;
+  if (!ffn_fused_shape_ok(m, M)) return SRM_ERR_UNSUPPORTED;
+  int rc = ensure_tc_ready(m);
+  if (rc != SRM_OK) return rc;
+  const int d = m.cfg.d_model;
+  const int64_t F = m.F();
+  const tc::FfnShape shape = ffn_shape(M, d, F);
+  if (m.tc_clusters < 2 || !tc::ffn_shape_ok(shape, m.tc_clusters)) return SRM_ERR_UNSUPPORTED;
+  const tc::FfnPlan* plan = nullptr;
+  for (const auto& e : m.ffn_plans)
+    if (e.first == shape.Rb) plan = &e.second;
+  if (plan == nullptr) {
+    m.ffn_plans.emplace_back(shape.Rb, tc::FfnPlan{});
+    if (!tc::ffn_make_plan(shape, m.tc_clusters, &m.ffn_plans.back().second)) { m.ffn_plans.pop_back(); return SRM_ERR_UNSUPPORTED; }
+    plan = &m.ffn_plans.back().second;
+  }
+  LaunchScope scope(m, SRM_KERNEL_FFN, st);
+  CUtensorMap ta, tw1, ths, th, tw2, tx;
+  const void* W1 = m.ptr(layer, SRM_T_W1);
+  const void* W2 = m.ptr(layer, SRM_T_W2);
+  if ((rc = m.tmap(a, M, d, tc::kRowsPerCta, 2, &ta)) != SRM_OK) return rc;
+  if ((rc = m.tmap(W1, F, d, tc::kRowsPerCta, 2, &tw1)) != SRM_OK) return rc;
+  if ((rc = m.tmap(H, M, F, tc::kOutBoxRows, 2, &ths)) != SRM_OK) return rc;
+  if ((rc = m.tmap(H, M, F, tc::kRowsPerCta, 2, &th)) != SRM_OK) return rc;
+  if ((rc = m.tmap(W2, d, F, tc::kRowsPerCta, 2, &tw2)) != SRM_OK) return rc;
+  if ((rc = m.tmap(x, M, d, tc::kOutBoxRows, 4, &tx)) != SRM_OK) return rc;
+  tc::FfnArgs g{M, d, (int)F, m.fptr(layer, SRM_T_B1), m.fptr(layer, SRM_T_B2), status, ready, 1};
+  SRM_CUDA(launch_kernel(tc::ffn_fused_kernel, dim3(2u * (unsigned)m.tc_clusters), dim3(tc::kThreads), tc::kSmemBytes, st,
+                         ta, tw1, ths, th, tw2, tx, g, *plan));
   SRM_CUDA(cudaGetLastError());
   return SRM_OK;
 }
@@ -551,7 +612,17 @@ int decode_chunk(srm_model& m, srm_state& s, int64_t b0, int64_t R, const int32_
     const int64_t tiles = ((R + tc::BM - 1) / tc::BM) * ((d + tc::BN - 1) / tc::BN);
     split = tc::split_plan(tiles, (int)(F / tc::BK), m.tc_clusters, &P) && tc::split_saved_kb(P) >= tc::kSplitWorthKb;
   }
-  if (split) SRM_CUDA(cudaMemsetAsync(w.order, 0, w.order_bytes, st));
+  // the feed-forward block as one kernel: its per-layer counters sit in the logits area, which nothing uses before
+  // the LM head
+  const size_t ready_layer = ffn_ready_bytes(R, F);
+  bool fused_ffn = !(c.flags & SRM_FLAG_NO_FUSED_FFN) && ffn_fused_shape_ok(m, R) &&
+                   ready_layer * c.n_layers <= align_up((size_t)w.rows * c.vocab * 4, 256);
+  if (fused_ffn) {
+    if ((rc = ensure_tc_ready(m))) return rc;
+    fused_ffn = ffn_fused_worthwhile(m, R);
+  }
+  if (fused_ffn) SRM_CUDA(cudaMemsetAsync(w.logits, 0, ready_layer * c.n_layers, st));
+  else if (split) SRM_CUDA(cudaMemsetAsync(w.order, 0, w.order_bytes, st));
   for (int l = 0; l < c.n_layers; ++l) {
     uint8_t* Sl = static_cast<uint8_t*>(s.layer_ptr(l)) + (size_t)b0 * d * m.state_bytes();
     if (c.mixer != SRM_MIXER_MIXED) {
@@ -560,6 +631,14 @@ int decode_chunk(srm_model& m, srm_state& s, int64_t b0, int64_t R, const int32_
     } else if (m.head_proj()) {
       if ((rc = launch_mixer_block_proj(m, l, t, R, R, 1, l == 0 ? tok_in + b0 : nullptr, w.x, Sl, w.a, w.q, s.status, st, ctr, pos))) return rc;
     } else if ((rc = launch_mixer(m, l, t, R, l == 0 ? tok_in + b0 : nullptr, w.x, Sl, w.a, s.status, st, ctr, pos))) return rc;
+    if (fused_ffn) {
+      int32_t* ready = reinterpret_cast<int32_t*>(reinterpret_cast<uint8_t*>(w.logits) + (size_t)l * ready_layer);
+      rc = launch_ffn_fused(m, l, R, w.a, w.H, w.x, ready, s.status, st);
+      if (rc == SRM_OK) continue;
+      if (rc != SRM_ERR_UNSUPPORTED) return rc;
+      fused_ffn = false;                                   // (no plan for this shape: decided at the first layer)
+      if (split) SRM_CUDA(cudaMemsetAsync(w.order, 0, w.order_bytes, st));
+    }
     if ((rc = launch_gemm(m, kEpiBiasGelu, R, F, d, w.a, m.ptr(l, SRM_T_W1), m.fptr(l, SRM_T_B1), w.H, s.status, st))) return rc;
     rc = split ? launch_gemm_splitk(m, R, d, F, w.H, m.ptr(l, SRM_T_W2), m.fptr(l, SRM_T_B2), w.x, w.order, s.status, st, true)
                : SRM_ERR_UNSUPPORTED;

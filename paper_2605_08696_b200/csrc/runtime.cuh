@@ -20,6 +20,7 @@
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
 #include "gemm_tc_splitk.cuh"
+#include "ffn_fused.cuh"
 #include "mixer.cuh"
 #include "mixer_stream.cuh"
 #include "mixer_proj.cuh"
@@ -198,6 +199,7 @@ struct srm_model {
   bool tc_ready = false;                 // smem attribute set for the tensor-core kernels
   int tc_clusters = 0;                   // CTA pairs of the tensor-core kernel that are resident at once
   std::vector<TmapCacheEntry> tmaps;     // weight and activation descriptors, built on first use
+  std::vector<std::pair<int, tc::FfnPlan>> ffn_plans;   // work lists of the fused feed-forward kernel, by row blocks
   // One decode step captured as a CUDA graph for srm_generate (launch-bound batches): the stream it is
   // captured on, the instantiated graph, and what it was captured for.
   cudaStream_t cap_stream = nullptr;

@@ -649,6 +649,49 @@ int64_t srm_k_gemm_splitk_plan(int64_t M, int64_t N, int64_t K, int32_t pairs, i
   return n;
 }
 
+size_t srm_k_ffn_ready_bytes(int64_t M, int64_t F) {
+  if (M < 1 || F < tc::BN) return 0;
+  return ffn_ready_bytes(M, F);
+}
+
+int srm_k_ffn(srm_model* m, int32_t layer, int64_t M, const void* d_a, void* d_H, float* d_x, void* d_ready,
+              size_t ready_bytes, uint32_t* d_status, void* stream) {
+  if (m == nullptr || M < 0 || layer < 0 || layer >= m->cfg.n_layers) return SRM_ERR_INVALID_ARG;
+  if (M == 0) return SRM_OK;
+  if (d_a == nullptr || d_H == nullptr || d_x == nullptr || d_ready == nullptr) return SRM_ERR_INVALID_ARG;
+  if (!ffn_fused_shape_ok(*m, M)) return SRM_ERR_UNSUPPORTED;
+  if (!aligned(d_a, 16) || !aligned(d_H, 16) || !aligned(d_x, 16) || !aligned(d_ready, 256)) return SRM_ERR_ALIGNMENT;
+  const size_t need = ffn_ready_bytes(M, m->F());
+  if (ready_bytes < need) return SRM_ERR_BUFFER_TOO_SMALL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  SRM_CUDA(cudaMemsetAsync(d_ready, 0, need, st));
+  return launch_ffn_fused(*m, layer, M, d_a, d_H, d_x, static_cast<int32_t*>(d_ready), d_status, st);
+}
+
+int64_t srm_k_ffn_plan(int64_t M, int32_t d, int32_t F, int32_t pairs, int32_t* off, int32_t* items, int64_t max_items,
+                       double* makespan, double* ideal) {
+  if (M < 1 || d < tc::BN || F < tc::BN || pairs < 1 || max_items < 0 || off == nullptr) return SRM_ERR_INVALID_ARG;
+  if (max_items > 0 && items == nullptr) return SRM_ERR_INVALID_ARG;
+  if (d % tc::BN || F % tc::BN || M > (int64_t)tc::kFfnMaxRb * tc::BM) return SRM_ERR_UNSUPPORTED;
+  const tc::FfnShape shape = ffn_shape(M, d, F);
+  if (!tc::ffn_shape_ok(shape, pairs)) return SRM_ERR_UNSUPPORTED;
+  tc::FfnPlan* plan = new (std::nothrow) tc::FfnPlan();
+  if (plan == nullptr) return SRM_ERR_INVALID_ARG;
+  if (!tc::ffn_make_plan(shape, pairs, plan)) { delete plan; return SRM_ERR_UNSUPPORTED; }
+  for (int p = 0; p <= pairs; ++p) off[p] = plan->off[p];
+  const int64_t n = plan->off[pairs];
+  for (int64_t i = 0; i < n && i < max_items; ++i) {
+    const uint16_t it = plan->item[i];
+    items[3 * i] = tc::ffn_item_down(it) ? 1 : 0;
+    items[3 * i + 1] = tc::ffn_item_rb(it);
+    items[3 * i + 2] = tc::ffn_item_cb(it);
+  }
+  if (makespan != nullptr) *makespan = tc::ffn_simulate(shape, *plan);
+  if (ideal != nullptr) *ideal = tc::ffn_ideal(shape, pairs);
+  delete plan;
+  return n;
+}
+
 int srm_k_lm_head_greedy(srm_model* m, int64_t R, const void* d_a, void* d_part, size_t part_bytes, int32_t* d_tok,
                          uint32_t* d_status, void* stream) {
   if (m == nullptr || R < 0) return SRM_ERR_INVALID_ARG;

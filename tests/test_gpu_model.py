@@ -63,7 +63,8 @@ def test_decode_with_and_without_split_k_down_projection_agree():
     B, n = 8192, 4
     prompts = torch.from_numpy(I.uniform_prompts(B, n, shape.vocab, seed=3)).to(DEV)
     res = []
-    for flags in (0, P.FLAG_NO_SPLITK):
+    # (with the feed-forward block as two launches: the single-kernel block never splits K)
+    for flags in (P.FLAG_NO_FUSED_FFN, P.FLAG_NO_FUSED_FFN | P.FLAG_NO_SPLITK):
         model = P.SRM(shape, W, device=DEV, flags=flags)
         st = model.new_state(B)
         ws = model.new_workspace(B, n, prefill_samples=B)
