@@ -117,3 +117,33 @@ def test_decode_steps_with_and_without_the_fused_block_are_equal(B, d, head_proj
     assert torch.equal(lg_a, lg_b)
     assert torch.equal(tok_a, tok_b)
     assert torch.equal(S_a, S_b)
+
+
+def test_captured_step_with_the_fused_block_equals_launch_by_launch():
+    """srm_generate replaying a captured step whose feed-forward blocks are the single kernel (the work lists are
+    part of the captured launch parameters, the counters are cleared by a captured memset) against the
+    launch-by-launch loop: same tokens, same cache, also when the captured graph is replayed by a second call."""
+    import paper_2605_08696_b200 as P
+    shape = custom_shape(n_layers=3, d_model=512, vocab=2048, n_ctx=40, dtype="bf16", seed=8)
+    W = I.make_weights(shape, alpha_std=0.5, beta_std=0.5)
+    B, n = 3100, 4
+    prompts = torch.from_numpy(np.random.default_rng(3).integers(0, shape.vocab, size=(B, n)).astype(np.int32)).to(DEV)
+    samp = P.Sampling("topk", 20, 0.9, seed=4, sample_idx_base=11)
+    outs = []
+    for flags in (P.FLAG_NO_GRAPH, P.FLAG_GRAPH):
+        m = P.SRM(shape, W, device=DEV, flags=flags)
+        st = m.new_state(B)
+        ws = m.new_workspace(B, n, prefill_samples=B)
+        first = m.prefill(st, prompts, samp, ws)
+        m.profile(True)
+        m.profile_reset()
+        a = m.generate(st, 6, 1, samp, ws)
+        prof = m.profile_read()
+        m.profile(False)
+        b = m.generate(st, 5, 7, samp, ws, out=a[:, :5].clone())
+        assert st.status() == 0 and st.pos == n + 11
+        outs.append((first.clone(), a.clone(), b.clone(), st.cache().clone()))
+        if flags == P.FLAG_NO_GRAPH:
+            assert prof["ffn"][0] == 6 * shape.n_layers        # (launches inside a replayed graph are not bracketed)
+    for x_, y_ in zip(outs[0], outs[1]):
+        assert torch.equal(x_, y_)
