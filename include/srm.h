@@ -423,8 +423,8 @@ int srm_k_ffn(srm_model* m, int32_t layer, int64_t M, const void* d_a, void* d_H
               size_t ready_bytes, uint32_t* d_status, void* stream);
 /* The work lists of srm_k_ffn for M rows of a model of width d and hidden width F on `pairs` CTA pairs, written to
  * HOST arrays: off[pairs + 1] (pair c owns items off[c] .. off[c + 1] - 1, in this order) and up to max_items items
- * of three int32 {0 = up tile / 1 = down tile, row block, column tile}. Returns the number of items (every tile of
- * both projections exactly once), or a negative SRM_ERR_*. *makespan / *ideal (may be NULL): the plan's length and
+ * of three int32 {0 = up tile / 1 = down tile / 2, 3 = first, second 256 x 128 half of an up tile, row block, column
+ * tile}. Returns the number of items (every tile of both projections exactly once, some up tiles as two halves), or a negative SRM_ERR_*. *makespan / *ideal (may be NULL): the plan's length and
  * the even-share lower bound under the cost model of the planner, in k-block times. Pure host arithmetic: needs no
  * device. */
 int64_t srm_k_ffn_plan(int64_t M, int32_t d, int32_t F, int32_t pairs, int32_t* off, int32_t* items, int64_t max_items,

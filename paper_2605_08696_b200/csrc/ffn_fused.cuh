@@ -65,6 +65,7 @@ __device__ __forceinline__ bool ready_wait(const int32_t* p, int32_t want, uint3
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 ffn_fused_kernel(const __grid_constant__ CUtensorMap tmA,     // a   [M, d] bf16, load boxes of 128 rows
                  const __grid_constant__ CUtensorMap tmW1,    // W1  [F, d]
+                 const __grid_constant__ CUtensorMap tmW1h,   // W1, load boxes of 64 rows (half-width pieces)
                  const __grid_constant__ CUtensorMap tmHs,    // H   [M, F] bf16, store boxes of 32 rows
                  const __grid_constant__ CUtensorMap tmH,     // H, load boxes of 128 rows
                  const __grid_constant__ CUtensorMap tmW2,    // W2  [d, F]
@@ -120,26 +121,29 @@ ffn_fused_kernel(const __grid_constant__ CUtensorMap tmA,     // a   [M, d] bf16
       int pre = 0;
       if (i0 < i1 && g.w_static) {
         const uint16_t it = plan.item[i0];
-        const bool down = ffn_item_down(it);
+        const bool down = ffn_item_down(it), half = ffn_item_half(it);
         const int kbs = down ? kb_dn : kb_up;
-        const int n_row = ffn_item_cb(it) * BN + (int)rank * kRowsPerCta;
+        const int w_rows = half ? kHalfN / 2 : kRowsPerCta;               // W rows each CTA of the pair loads
+        const int n_row = ffn_item_cb(it) * BN + ffn_item_noff(it) + (int)rank * w_rows;
         pre = kbs < kStages ? kbs : kStages;
         for (int i = 0; i < pre; ++i) {
           const uint32_t full_leader = mapa(smem_u32(&full[i]), 0);
-          mbar_expect_tx_cluster(full_leader, kStageBytes);
-          tma_load_2d(sB + i * kBStageBytes, down ? &tmW2 : &tmW1, full_leader, i * BK, n_row);
+          mbar_expect_tx_cluster(full_leader, kAStageBytes + (uint32_t)w_rows * BK * 2);
+          tma_load_2d(sB + i * kBStageBytes, down ? &tmW2 : (half ? &tmW1h : &tmW1), full_leader, i * BK, n_row);
         }
       }
       pdl_wait();
       for (int i = i0; ok && i < i1; ++i) {
         const uint16_t it = plan.item[i];
-        const bool down = ffn_item_down(it);
+        const bool down = ffn_item_down(it), half = ffn_item_half(it);
         const int rb = ffn_item_rb(it);
         const int kbs = down ? kb_dn : kb_up;
+        const int w_rows = half ? kHalfN / 2 : kRowsPerCta;
+        const uint32_t stage_bytes = kAStageBytes + (uint32_t)w_rows * BK * 2;
         const CUtensorMap* mapA = down ? &tmH : &tmA;
-        const CUtensorMap* mapB = down ? &tmW2 : &tmW1;
+        const CUtensorMap* mapB = down ? &tmW2 : (half ? &tmW1h : &tmW1);
         const int m_row = rb * BM + (int)rank * kRowsPerCta;
-        const int n_row = ffn_item_cb(it) * BN + (int)rank * kRowsPerCta;
+        const int n_row = ffn_item_cb(it) * BN + ffn_item_noff(it) + (int)rank * w_rows;
         const int32_t* rdy = g.ready + (int64_t)rb * Cu;
         for (int kb = 0; kb < kbs; ++kb) {
           const uint32_t full_leader = mapa(smem_u32(&full[stage]), 0);
@@ -147,7 +151,7 @@ ffn_fused_kernel(const __grid_constant__ CUtensorMap tmA,     // a   [M, d] bf16
             --pre;
           } else {
             if (!mbar_wait(&empty[stage], phase ^ 1u, g.status)) { ok = false; break; }
-            mbar_expect_tx_cluster(full_leader, kStageBytes);
+            mbar_expect_tx_cluster(full_leader, stage_bytes);
             tma_load_2d(sB + stage * kBStageBytes, mapB, full_leader, kb * BK, n_row);
           }
           if (down && (kb % kFfnKbPerHTile) == 0) {
@@ -172,6 +176,7 @@ ffn_fused_kernel(const __grid_constant__ CUtensorMap tmA,     // a   [M, d] bf16
       bool ok = true;
       for (int i = i0; ok && i < i1; ++i) {
         const int kbs = ffn_item_down(plan.item[i]) ? kb_dn : kb_up;
+        const uint32_t idesc = ffn_item_half(plan.item[i]) ? instr_desc(kHalfN) : kInstrDesc;
         if (!mbar_wait(&tempty[acc], acc_phase ^ 1u, g.status)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN);
@@ -182,7 +187,7 @@ ffn_fused_kernel(const __grid_constant__ CUtensorMap tmA,     // a   [M, d] bf16
           const uint64_t db = make_smem_desc(smem_u32(sB + stage * kBStageBytes));
 #pragma unroll
           for (int k = 0; k < BK / 16; ++k)
-            umma_bf16(d_tmem, da + 2u * k, db + 2u * k, kInstrDesc, (kb | k) != 0 ? 1u : 0u);
+            umma_bf16(d_tmem, da + 2u * k, db + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
           umma_commit_pair(&empty[stage]);
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
@@ -208,10 +213,12 @@ ffn_fused_kernel(const __grid_constant__ CUtensorMap tmA,     // a   [M, d] bf16
       if (!mbar_wait(&tfull[acc], acc_phase, g.status)) break;
       tc_fence_after();
       const int row0 = rb * BM + (int)rank * kRowsPerCta + quad * 32;
-      const int col0 = cb * BN + cgrp * kColsPerEpiWarp;
+      const int col0 = cb * BN + ffn_item_noff(it) + cgrp * kColsPerEpiWarp;
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) +
                              static_cast<uint32_t>(acc * BN + cgrp * kColsPerEpiWarp);
-      if (row0 < g.M) {
+      // (a half piece fills the first 128 accumulator columns: the warps of the other two column groups only arrive)
+      const bool mine = !ffn_item_half(it) || cgrp * kColsPerEpiWarp < kHalfN;
+      if (row0 < g.M && mine) {
         if (down) {
           const GemmArgs ga{g.M, g.d, g.F, g.b2, nullptr, g.status, 0};
           epilogue_columns<kEpiBiasResidual>(ga, &tmX, buf, lane, taddr, row0, col0);
@@ -224,9 +231,10 @@ ffn_fused_kernel(const __grid_constant__ CUtensorMap tmA,     // a   [M, d] bf16
       __syncwarp();
       if (lane == 0) {
         mbar_arrive_cluster(mapa(smem_u32(&tempty[acc]), 0));
-        if (!down) {
+        if (!down && mine) {
           // this warp's part of the H tile is in global memory: count it in (the next accumulator is a tile's
-          // main loop away, so the wait for the store costs nothing)
+          // main loop away, so the wait for the store costs nothing); the two halves of a tile computed in halves
+          // count 16 warps each
           bulk_wait_all();
           fence_async_global();
           red_release_add(g.ready + (int64_t)rb * Cu + cb, 1);

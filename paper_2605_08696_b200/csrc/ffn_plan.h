@@ -37,7 +37,9 @@ constexpr int kFfnMaxRb = 64;          // row blocks of 256 rows
 constexpr int kFfnMaxCu = 32;          // column tiles of H (F <= 8192)
 constexpr int kFfnKbPerHTile = 4;      // k-blocks (64) of the down projection per column tile (256) of H
 
-// Item: bit 15 = down projection, bits 5..10 = row block, bits 0..4 = column tile.
+// Item: bit 15 = down projection, bits 5..10 = row block, bits 0..4 = column tile; up projection only: bit 14 = one
+// 256 x 128 half of the tile (the tiles of a last, partly filled round of up tiles run as two halves on two pairs,
+// which ends earlier than whole tiles on half as many pairs), bit 13 = its second half (columns 128..255).
 struct FfnPlan {
   uint16_t n_pairs;
   uint16_t off[kFfnMaxPairs + 1];      // pair c owns item[off[c]] .. item[off[c + 1] - 1], in order
@@ -47,6 +49,10 @@ SRM_HD inline uint16_t ffn_item(bool down, int rb, int cb) { return (uint16_t)((
 SRM_HD inline bool ffn_item_down(uint16_t it) { return (it & 0x8000) != 0; }
 SRM_HD inline int ffn_item_rb(uint16_t it) { return (it >> 5) & 63; }
 SRM_HD inline int ffn_item_cb(uint16_t it) { return it & 31; }
+SRM_HD inline bool ffn_item_half(uint16_t it) { return (it & 0x4000) != 0; }
+SRM_HD inline int ffn_item_noff(uint16_t it) { return (it & 0x2000) ? 128 : 0; }     // first column inside the tile
+constexpr uint16_t kFfnHalf = 0x4000, kFfnSecond = 0x2000;
+constexpr double kFfnHalfCost = 0.75;  // a half piece moves three quarters of a tile's operand bytes for half its flops
 
 struct FfnShape {
   int Rb;        // row blocks
@@ -66,7 +72,7 @@ struct FfnCost {
 
 inline bool ffn_shape_ok(const FfnShape& s, int pairs) {
   return s.Rb >= 1 && s.Rb <= kFfnMaxRb && s.Cu >= 1 && s.Cu <= kFfnMaxCu && s.Cd >= 1 && s.Cd <= 8 && s.ku >= 1 &&
-         s.kd == kFfnKbPerHTile * s.Cu && pairs >= 1 && pairs <= kFfnMaxPairs && s.Rb * (s.Cu + s.Cd) <= kFfnMaxItems;
+         s.kd == kFfnKbPerHTile * s.Cu && pairs >= 1 && pairs <= kFfnMaxPairs && s.Rb * (s.Cu + s.Cd) + kFfnMaxPairs / 2 <= kFfnMaxItems;
 }
 
 // Forward run of a plan under the cost model. Returns the time the last pair ends, or -1 when the lists block one
@@ -75,14 +81,16 @@ inline double ffn_simulate(const FfnShape& s, const FfnPlan& P, const FfnCost& c
   const int n = P.n_pairs;
   std::vector<double> ready((size_t)s.Rb * s.Cu, -1.0);      // time H tile (rb, hc) becomes visible; -1: not known yet
   std::vector<int> seen_up((size_t)s.Rb * s.Cu, 0), seen_dn((size_t)s.Rb * s.Cd, 0);
+  std::vector<double> pend((size_t)s.Rb * s.Cu, 0.0);        // end of the first half of a tile computed in halves
   std::vector<int> pos(n, 0);
   std::vector<double> t(n, 0.0);
-  int left = 0;
+  int left = 0, halves = 0;
   for (int p = 0; p < n; ++p) {
     if (P.off[p + 1] < P.off[p] || P.off[p + 1] > kFfnMaxItems) return -1.0;
     left += P.off[p + 1] - P.off[p];
+    for (int i = P.off[p]; i < P.off[p + 1]; ++i) halves += ffn_item_half(P.item[i]) ? 1 : 0;
   }
-  if (left != s.Rb * (s.Cu + s.Cd)) return -1.0;
+  if (halves % 2 || left - halves / 2 != s.Rb * (s.Cu + s.Cd)) return -1.0;
   bool progress = true;
   while (left > 0 && progress) {
     progress = false;
@@ -92,9 +100,15 @@ inline double ffn_simulate(const FfnShape& s, const FfnPlan& P, const FfnCost& c
         const int rb = ffn_item_rb(it), cb = ffn_item_cb(it);
         if (rb >= s.Rb) return -1.0;
         if (!ffn_item_down(it)) {
-          if (cb >= s.Cu || seen_up[(size_t)rb * s.Cu + cb]++) return -1.0;
-          t[p] += s.ku * c.up_kb + c.up_tile;
-          ready[(size_t)rb * s.Cu + cb] = t[p] + c.ready_lag;
+          // seen_up: bit 0 = columns 0..127 computed, bit 1 = columns 128..255
+          if (cb >= s.Cu) return -1.0;
+          int& seen = seen_up[(size_t)rb * s.Cu + cb];
+          const int bits = ffn_item_half(it) ? (ffn_item_noff(it) ? 2 : 1) : 3;
+          if (seen & bits) return -1.0;
+          seen |= bits;
+          t[p] += (ffn_item_half(it) ? kFfnHalfCost : 1.0) * s.ku * c.up_kb + c.up_tile;
+          if (seen == 3) ready[(size_t)rb * s.Cu + cb] = std::max(pend[(size_t)rb * s.Cu + cb], t[p]) + c.ready_lag;
+          else pend[(size_t)rb * s.Cu + cb] = t[p];
         } else {
           if (cb >= s.Cd) return -1.0;
           bool known = true;
@@ -123,7 +137,8 @@ inline double ffn_ideal(const FfnShape& s, int pairs, const FfnCost& c = FfnCost
   return std::max(((double)s.Rb * s.Cu * up + (double)s.Rb * s.Cd * dn) / pairs, up + kFfnKbPerHTile * c.dn_kb + dn - 0.0 * c.ready_lag);
 }
 
-inline bool ffn_make_plan(const FfnShape& s, int pairs, FfnPlan* out, const FfnCost& c = FfnCost()) {
+// The plan in which the last `n_half` up tiles placed (the first of the forward lists) go out as halves.
+inline bool ffn_make_plan_halves(const FfnShape& s, int pairs, int n_half, FfnPlan* out, const FfnCost& c) {
   if (!ffn_shape_ok(s, pairs)) return false;
   const double up_cost = s.ku * c.up_kb + c.up_tile, dn_cost = s.kd * c.dn_kb + c.dn_tile;
   const double h_tile = kFfnKbPerHTile * c.dn_kb;             // time a down tile spends on one column tile of H
@@ -138,10 +153,21 @@ inline bool ffn_make_plan(const FfnShape& s, int pairs, FfnPlan* out, const FfnC
   int next_dn_rb = s.Rb - 1;                                  // down tiles go from the last row block to the first
   int open = 0;                                               // row blocks with a down tile placed and up tiles left
   int left = s.Rb * (s.Cu + s.Cd);
+  int ups_left = s.Rb * s.Cu, dns_left = s.Rb * s.Cd;
+  int pending_half = -1;                                      // the second half of a tile whose first half has been placed
+  double pending_rel = 0.0;
+  const double half_cost = kFfnHalfCost * s.ku * c.up_kb + c.up_tile;
   while (left > 0) {
     int p = 0;
     for (int q = 1; q < pairs; ++q) if (free_at[q] < free_at[p]) p = q;
     const double t = free_at[p];
+    if (pending_half >= 0) {                                  // (goes to the next pair that is free, whatever else is released)
+      rev[p].push_back((uint16_t)pending_half);
+      free_at[p] = std::max(t, pending_rel) + half_cost;
+      pending_half = -1;
+      --left;
+      continue;
+    }
     // (a) a down tile: of a row block already begun, or of the next one while the H budget allows
     while (next_dn_rb >= 0 && dn_placed[next_dn_rb] == s.Cd) --next_dn_rb;
     const bool dn_ok = next_dn_rb >= 0 && (dn_placed[next_dn_rb] > 0 || open < open_max);
@@ -153,6 +179,7 @@ inline bool ffn_make_plan(const FfnShape& s, int pairs, FfnPlan* out, const FfnC
       ++dn_placed[rb];
       free_at[p] = t + dn_cost;
       --left;
+      --dns_left;
       continue;
     }
     // (b) a released up tile: the highest row block first, within it the highest column tile (placed backwards)
@@ -167,9 +194,21 @@ inline bool ffn_make_plan(const FfnShape& s, int pairs, FfnPlan* out, const FfnC
     }
     if (best_rb >= 0) {
       const int rb = best_rb, hc = s.Cu - 1 - up_placed[rb];
-      rev[p].push_back(ffn_item(false, rb, hc));
+      // the last up tiles (in reversed time: the first of the forward lists), when they no longer fill a round of
+      // whole tiles, go out as halves to twice as many pairs
+      const bool halves = dns_left == 0 && ups_left <= n_half;
+      if (halves) {
+        rev[p].push_back((uint16_t)(ffn_item(false, rb, hc) | kFfnHalf | kFfnSecond));
+        pending_half = ffn_item(false, rb, hc) | kFfnHalf;
+        pending_rel = t;
+        ++left;                                               // one tile, two items
+        free_at[p] = t + half_cost;
+      } else {
+        rev[p].push_back(ffn_item(false, rb, hc));
+        free_at[p] = t + up_cost;
+      }
       if (++up_placed[rb] == s.Cu) --open;
-      free_at[p] = t + up_cost;
+      --ups_left;
       --left;
       continue;
     }
@@ -188,6 +227,25 @@ inline bool ffn_make_plan(const FfnShape& s, int pairs, FfnPlan* out, const FfnC
   }
   for (int p = pairs; p <= kFfnMaxPairs; ++p) out->off[p] = (uint16_t)o;
   return ffn_simulate(s, *out, c) >= 0.0;
+}
+
+// The plan of the decode step: as few up tiles in halves as reach (within half a k-block time) the shortest plan any
+// number of halves up to pairs / 2 gives. A half moves three quarters of a tile's operand bytes for half its flops,
+// and the step runs at the power cap: halves that do not shorten the plan only cost clock.
+inline bool ffn_make_plan(const FfnShape& s, int pairs, FfnPlan* out, const FfnCost& c = FfnCost()) {
+  if (!ffn_shape_ok(s, pairs)) return false;
+  const int h_max = std::min(pairs / 2, s.Rb * s.Cu);
+  std::vector<double> len(h_max + 1, -1.0);
+  double best = -1.0;
+  for (int h = 0; h <= h_max; ++h) {
+    if (!ffn_make_plan_halves(s, pairs, h, out, c)) continue;
+    len[h] = ffn_simulate(s, *out, c);
+    if (len[h] >= 0.0 && (best < 0.0 || len[h] < best)) best = len[h];
+  }
+  if (best < 0.0) return false;
+  for (int h = 0; h <= h_max; ++h)
+    if (len[h] >= 0.0 && len[h] <= best + 0.5) return ffn_make_plan_halves(s, pairs, h, out, c);
+  return false;
 }
 
 }  // namespace tc

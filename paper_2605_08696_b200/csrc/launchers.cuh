@@ -317,18 +317,19 @@ int launch_ffn_fused(srm_model& m, int layer, int64_t M, const void* a, void* H,
     plan = &m.ffn_plans.back().second;
   }
   LaunchScope scope(m, SRM_KERNEL_FFN, st);
-  CUtensorMap ta, tw1, ths, th, tw2, tx;
+  CUtensorMap ta, tw1, tw1h, ths, th, tw2, tx;
   const void* W1 = m.ptr(layer, SRM_T_W1);
   const void* W2 = m.ptr(layer, SRM_T_W2);
   if ((rc = m.tmap(a, M, d, tc::kRowsPerCta, 2, &ta)) != SRM_OK) return rc;
   if ((rc = m.tmap(W1, F, d, tc::kRowsPerCta, 2, &tw1)) != SRM_OK) return rc;
+  if ((rc = m.tmap(W1, F, d, tc::kHalfN / 2, 2, &tw1h)) != SRM_OK) return rc;        // W1 rows of a half-width piece
   if ((rc = m.tmap(H, M, F, tc::kOutBoxRows, 2, &ths)) != SRM_OK) return rc;
   if ((rc = m.tmap(H, M, F, tc::kRowsPerCta, 2, &th)) != SRM_OK) return rc;
   if ((rc = m.tmap(W2, d, F, tc::kRowsPerCta, 2, &tw2)) != SRM_OK) return rc;
   if ((rc = m.tmap(x, M, d, tc::kOutBoxRows, 4, &tx)) != SRM_OK) return rc;
   tc::FfnArgs g{M, d, (int)F, m.fptr(layer, SRM_T_B1), m.fptr(layer, SRM_T_B2), status, ready, 1};
   SRM_CUDA(launch_kernel(tc::ffn_fused_kernel, dim3(2u * (unsigned)m.tc_clusters), dim3(tc::kThreads), tc::kSmemBytes, st,
-                         ta, tw1, ths, th, tw2, tx, g, *plan));
+                         ta, tw1, tw1h, ths, th, tw2, tx, g, *plan));
   SRM_CUDA(cudaGetLastError());
   return SRM_OK;
 }

@@ -682,7 +682,7 @@ int64_t srm_k_ffn_plan(int64_t M, int32_t d, int32_t F, int32_t pairs, int32_t* 
   const int64_t n = plan->off[pairs];
   for (int64_t i = 0; i < n && i < max_items; ++i) {
     const uint16_t it = plan->item[i];
-    items[3 * i] = tc::ffn_item_down(it) ? 1 : 0;
+    items[3 * i] = tc::ffn_item_down(it) ? 1 : tc::ffn_item_half(it) ? (tc::ffn_item_noff(it) ? 3 : 2) : 0;
     items[3 * i + 1] = tc::ffn_item_rb(it);
     items[3 * i + 2] = tc::ffn_item_cb(it);
   }

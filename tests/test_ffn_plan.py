@@ -1,5 +1,6 @@
 """Work lists of the fused feed-forward kernel (srm_k_ffn_plan: pure host arithmetic; the lists travel to the kernel
-as a launch parameter). Every tile of both projections exactly once; the lists cannot block one another (a down tile
+as a launch parameter). Every tile of both projections exactly once (an up tile possibly as its two 256 x 128 halves:
+item kinds 0 = up tile, 1 = down tile, 2 / 3 = first / second half of an up tile); the lists cannot block one another (a down tile
 waits for the up tiles of its row block, which other pairs hold further down their own lists); under the planner's
 cost model the plan ends close to the even share of all work and never later than two launches in whole rounds."""
 import pytest
@@ -24,7 +25,7 @@ SHAPES = [
 def _run_lists(lists, Rb, Cu, Cd):
     """Executes the lists with the STRICTEST reading of the dependency (a down tile cannot finish before every up
     tile of its row block has): returns the number of sweeps, or None when the lists block one another."""
-    up_done = [[False] * Cu for _ in range(Rb)]
+    up_done = [[0] * Cu for _ in range(Rb)]          # bit 0: columns 0..127 done, bit 1: columns 128..255
     pos = [0] * len(lists)
     left = sum(len(l) for l in lists)
     sweeps = 0
@@ -32,11 +33,11 @@ def _run_lists(lists, Rb, Cu, Cd):
         progress = False
         for c, l in enumerate(lists):
             while pos[c] < len(l):
-                down, rb, cb = l[pos[c]]
-                if down and not all(up_done[rb]):
+                kind, rb, cb = l[pos[c]]
+                if kind == 1 and not all(v == 3 for v in up_done[rb]):
                     break
-                if not down:
-                    up_done[rb][cb] = True
+                if kind != 1:
+                    up_done[rb][cb] |= {0: 3, 2: 1, 3: 2}[kind]
                 pos[c] += 1
                 left -= 1
                 progress = True
@@ -51,9 +52,12 @@ def test_plan_holds_every_tile_once_and_cannot_block(M, d, F, pairs):
     lists, makespan, ideal = P.k_ffn_plan(M, d, F, pairs)
     Rb, Cu, Cd = -(-M // 256), F // 256, d // 256
     assert len(lists) == pairs
-    ups = [(rb, cb) for l in lists for (down, rb, cb) in l if not down]
-    downs = [(rb, cb) for l in lists for (down, rb, cb) in l if down]
-    assert sorted(ups) == [(rb, cb) for rb in range(Rb) for cb in range(Cu)]
+    ups = [(rb, cb) for l in lists for (kind, rb, cb) in l if kind == 0]
+    first = [(rb, cb) for l in lists for (kind, rb, cb) in l if kind == 2]
+    second = [(rb, cb) for l in lists for (kind, rb, cb) in l if kind == 3]
+    downs = [(rb, cb) for l in lists for (kind, rb, cb) in l if kind == 1]
+    assert sorted(first) == sorted(second) and len(set(first)) == len(first) and 2 * len(first) <= pairs
+    assert sorted(ups + first) == [(rb, cb) for rb in range(Rb) for cb in range(Cu)]
     assert sorted(downs) == [(rb, cb) for rb in range(Rb) for cb in range(Cd)]
     assert _run_lists(lists, Rb, Cu, Cd) is not None
     assert makespan > 0 and ideal > 0
@@ -79,10 +83,20 @@ def test_within_a_row_block_up_tiles_come_in_column_order():
     lists, _, _ = P.k_ffn_plan(4096, 1024, 4096, 74)
     for l in lists:
         last = {}
-        for down, rb, cb in l:
-            if not down:
+        for kind, rb, cb in l:
+            if kind != 1:
                 assert last.get(rb, -1) < cb
                 last[rb] = cb
+
+
+def test_last_round_of_up_tiles_goes_out_as_halves():
+    """Mid model, 4096 rows on 74 pairs: 64 pairs take three up tiles and a down tile, ten pairs up tiles only; the
+    four tiles left over would give four pairs a fourth up tile: they go out as eight halves instead."""
+    lists, makespan, ideal = P.k_ffn_plan(4096, 1024, 4096, 74)
+    halves = [(c, it) for c, l in enumerate(lists) for it in l if it[0] in (2, 3)]
+    assert len(halves) == 8 and len({c for c, _ in halves}) == 8
+    assert all(l.index(it) == 0 for c, it in halves for l in [lists[c]])        # the first item of their pairs
+    assert makespan < 1.13 * ideal
 
 
 def test_unsupported_shapes_are_refused():
