@@ -81,6 +81,11 @@ enum {
                                         of at most 16384 rows with at least one and a half 256 x 256 tiles per CTA pair:
                                         ONE kernel computes the tiles of both projections, see srm_k_ffn; same results
                                         bit for bit); for comparison and measurement */
+  SRM_FLAG_NO_KSLICE = 512,          /* the down projection of a small decode pass always adds whole tiles into x (default,
+                                        where its tiles fill less than half of the CTA pairs, bf16 mixed-head models: the
+                                        K dimension is cut into up to 8 ranges, one CTA pair each, and the next layer's
+                                        mixer adds the partial products in a fixed order; results then differ in the
+                                        last bits from those of a pass large enough not to be cut); for comparison */
   SRM_FLAG_HEAD_PROJ = 2             /* token mixer with head projections [Method/Architecture, Eq. 10]:
                                         q = W_in LN1(x) (W_in stacks the per-head I_g), heads of q mixed, and
                                         x += W_out (concatenated heads); the cache holds projected values.
@@ -189,10 +194,16 @@ int32_t srm_cache_planes(const srm_config* cfg);
  * workspace at least this large for B_chunk = 1 and split the batch into as many passes as
  * the given workspace requires. Decode never uses more than 12288 rows of it in one pass: a larger
  * batch runs as equal passes of at most 10240 rows (whole 256-row tiles), which keeps a layer's
- * activations in L2 between its kernels; results do not depend on the split (one exception: a batch of at most 64
- * samples whose workspace holds it in one pass takes the single-kernel step, see SRM_FLAG_NO_SMALL_BATCH, whose
- * sums run in another order than those of the kernel-per-operation path). */
+ * activations in L2 between its kernels; results do not depend on the split, with two exceptions in the last bits:
+ * a batch of at most 64 samples whose workspace holds it in one pass takes the single-kernel step (see
+ * SRM_FLAG_NO_SMALL_BATCH), whose sums run in another order than those of the kernel-per-operation path; and a pass
+ * small enough for its down projection to be cut along K (see SRM_FLAG_NO_KSLICE) adds that projection's partial
+ * products in another order than a large pass, whatever batch it is part of. */
 size_t srm_workspace_bytes(const srm_config* cfg, int64_t B_chunk, int32_t n_prefill_max);
+/* Workspace bytes with which srm_prefill (and its variants) processes `samples` prompts of up to n tokens in one
+ * pass [Eq. 1, Eq. 3: the sequence-parallel form over all positions of a pass]. A workspace for both calls is the
+ * larger of this and srm_workspace_bytes(cfg, B_chunk, 0). 0: bad arguments. */
+size_t srm_prefill_workspace_bytes(const srm_config* cfg, int64_t samples, int32_t n);
 /* Rows per decode pass that a batch of B samples is processed in when the workspace has room for
  * `ws_rows` rows (the rule stated above; host only, no device work). 0 if B < 1 or ws_rows < 1. */
 int64_t srm_decode_pass_rows(int64_t B, int64_t ws_rows);
@@ -318,7 +329,7 @@ int srm_decode_step_host(srm_model* m, srm_state* s, const int32_t* h_tok_in,
  * Same arguments and results as srm_decode_step, minus the workspace. Differences:
  *   - the whole batch must fit in one pass: if srm_workspace_bytes(cfg, B, 0) exceeds
  *     SRM_STATIC_SCRATCH_BYTES the call enqueues nothing and returns SRM_ERR_STATIC_SCRATCH
- *     (e.g. the mid model, 142 KB per row next to 2.2 MB of fixed scratch, takes up to about 220 rows; the tiny
+ *     (e.g. the mid model, 142 KB per row next to 10.6 MB of fixed scratch, takes up to about 160 rows; the tiny
  *     model about 13 000);
  *   - the device that is current must be the model's device (else SRM_ERR_INVALID_ARG);
  *   - the first call on each device looks up the array's device address (cudaGetSymbolAddress).

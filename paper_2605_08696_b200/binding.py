@@ -25,6 +25,7 @@ FLAG_NO_FUSED_TOPK = 32
 FLAG_NO_SMALL_BATCH = 64
 FLAG_NO_TAIL_SPLIT = 128
 FLAG_NO_FUSED_FFN = 256
+FLAG_NO_KSLICE = 512
 # enum srm_error
 ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_BUFFER_TOO_SMALL, ERR_CTX_OVERFLOW, ERR_CUDA, \
     ERR_DEVICE_STATUS, ERR_STATIC_SCRATCH = -1, -2, -3, -4, -5, -6, -7, -8
@@ -82,6 +83,7 @@ SYMBOLS = {
     "srm_state_bytes": (_SZ, [C.POINTER(_Config), _I64]),
     "srm_cache_planes": (_I32, [C.POINTER(_Config)]),
     "srm_workspace_bytes": (_SZ, [C.POINTER(_Config), _I64, _I32]),
+    "srm_prefill_workspace_bytes": (_SZ, [C.POINTER(_Config), _I64, _I32]),
     "srm_create": (C.c_int, [C.POINTER(_Config), _P, _SZ, C.POINTER(_P)]),
     "srm_destroy": (C.c_int, [_P]),
     "srm_state_create": (C.c_int, [_P, _I64, _P, _SZ, _P, C.POINTER(_P)]),
@@ -387,7 +389,8 @@ class SRM:
         return _lib().srm_workspace_bytes(C.byref(self.cfg), B_chunk, n_prefill)
 
     def new_workspace(self, B_chunk: int, n_prefill: int = 0, prefill_samples: int = 1) -> torch.Tensor:
-        nb = max(self.workspace_bytes(B_chunk, 0), prefill_samples * self.workspace_bytes(1, n_prefill) if n_prefill else 0)
+        nb = max(self.workspace_bytes(B_chunk, 0),
+                 _lib().srm_prefill_workspace_bytes(C.byref(self.cfg), prefill_samples, n_prefill) if n_prefill else 0)
         return torch.empty(nb, dtype=torch.uint8, device=self.device)
 
     # ---- hot path ----

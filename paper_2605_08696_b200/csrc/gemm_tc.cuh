@@ -262,6 +262,13 @@ struct GemmArgs {
   // partly filled round of tiles keeps (nearly) all CTA pairs busy: a half piece moves three quarters of a tile's
   // operand bytes for half its flops, and 2 r half pieces on 74 pairs end earlier than r tiles on r pairs.
   int tail_tiles;
+  // kEpiPlain only. k_slices > 1: the K dimension of every tile is cut into k_slices equal ranges of k-blocks, a
+  // piece is (tile, range), and range s writes its partial product to rows [s * plane_rows, s * plane_rows + M) of
+  // the output (plane_rows a multiple of 256, >= M): with a few tiles and a long K (the down projection of a small
+  // batch: 4 tiles of 64 k-blocks for 74 pairs) all pairs work on it, and the consumer adds the planes in a fixed
+  // order. No half-width pieces then.
+  int k_slices;
+  int64_t plane_rows;
 };
 
 // Piece q of a launch: the tile it belongs to, its first column inside the tile and its width.
@@ -512,9 +519,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
   const int64_t m_tiles = (M_rows + BM - 1) / BM, n_tiles = (g.N + BN - 1) / BN;
   const int64_t tiles = m_tiles * n_tiles;
-  const int tail = g.m_limit != nullptr ? 0 : g.tail_tiles;
-  const int64_t pieces = tiles + tail;                 // a tail tile counts as two pieces
-  const int k_blocks = static_cast<int>(g.K / BK);
+  const int ks = (EPI == kEpiPlain && g.k_slices > 1 && g.m_limit == nullptr) ? g.k_slices : 1;   // ranges of K per tile
+  const int tail = (g.m_limit != nullptr || ks > 1) ? 0 : g.tail_tiles;
+  const int64_t pieces = (tiles + tail) * ks;          // a tail tile counts as two pieces
+  const int k_all = static_cast<int>(g.K / BK);
+  const int k_blocks = (k_all + ks - 1) / ks;          // k-blocks per piece (the last range of a tile may be shorter)
 
   if (warp == 0) {
     // ---------------- TMA producer (both CTAs) ----------------
@@ -528,40 +537,44 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       // the first NS stages need no wait), then order against the predecessor and add the A loads.
       int pre = 0;
       if (cluster_id < pieces) {
-        const Piece pc = piece_of(cluster_id, tiles, tail);
+        const Piece pc = piece_of(cluster_id / ks, tiles, tail);
+        const int kb0 = static_cast<int>(cluster_id % ks) * k_blocks;          // first k-block of this piece's range
+        const int kbn = k_all - kb0 < k_blocks ? k_all - kb0 : k_blocks;
         const int w_rows = pc.nw >> 1;                                       // W rows each CTA of the pair loads
         const CUtensorMap* mapB = pc.nw == BN ? &tmB : &tmB64;
         const uint32_t stage_bytes = kAStageBytes + (uint32_t)w_rows * BK * 2;
         const int m0 = static_cast<int>(pc.tile % m_tiles) * BM + static_cast<int>(rank) * kRowsPerCta;
         const int n0 = static_cast<int>(pc.tile / m_tiles) * BN + pc.noff + static_cast<int>(rank) * w_rows;
-        pre = k_blocks < NS ? k_blocks : NS;
+        pre = kbn < NS ? (kbn > 0 ? kbn : 0) : NS;
         if (!g.w_static) pdl_wait();
         for (int kb = 0; kb < pre; ++kb) {
           const uint32_t full_leader = mapa(smem_u32(&full[kb]), 0);
           mbar_expect_tx_cluster(full_leader, stage_bytes);
-          tma_load_2d(sB + kb * kBStageBytes, mapB, full_leader, kb * BK, n0);
+          tma_load_2d(sB + kb * kBStageBytes, mapB, full_leader, (kb0 + kb) * BK, n0);
         }
         if (g.w_static) pdl_wait();
         for (int kb = 0; kb < pre; ++kb)
-          tma_load_2d(sA + kb * kAStageBytes, &tmA, mapa(smem_u32(&full[kb]), 0), kb * BK, m0);
+          tma_load_2d(sA + kb * kAStageBytes, &tmA, mapa(smem_u32(&full[kb]), 0), (kb0 + kb) * BK, m0);
         stage = pre;
         if (stage == NS) { stage = 0; phase ^= 1u; }
       } else {
         pdl_wait();
       }
       for (int64_t q = cluster_id; ok && q < pieces; q += n_clusters) {
-        const Piece pc = piece_of(q, tiles, tail);
+        const Piece pc = piece_of(q / ks, tiles, tail);
+        const int kb0 = static_cast<int>(q % ks) * k_blocks;
+        const int kbn = k_all - kb0 < k_blocks ? k_all - kb0 : k_blocks;
         const int w_rows = pc.nw >> 1;
         const CUtensorMap* mapB = pc.nw == BN ? &tmB : &tmB64;
         const uint32_t stage_bytes = kAStageBytes + (uint32_t)w_rows * BK * 2;
         const int m0 = static_cast<int>(pc.tile % m_tiles) * BM + static_cast<int>(rank) * kRowsPerCta;
         const int n0 = static_cast<int>(pc.tile / m_tiles) * BN + pc.noff + static_cast<int>(rank) * w_rows;
-        for (int kb = (q == cluster_id ? pre : 0); kb < k_blocks; ++kb) {
+        for (int kb = (q == cluster_id ? pre : 0); kb < kbn; ++kb) {
           if (!mbar_wait(&empty[stage], phase ^ 1u, g.status)) { ok = false; break; }
           const uint32_t full_leader = mapa(smem_u32(&full[stage]), 0);
           mbar_expect_tx_cluster(full_leader, stage_bytes);
-          tma_load_2d(sA + stage * kAStageBytes, &tmA, full_leader, kb * BK, m0);
-          tma_load_2d(sB + stage * kBStageBytes, mapB, full_leader, kb * BK, n0);
+          tma_load_2d(sA + stage * kAStageBytes, &tmA, full_leader, (kb0 + kb) * BK, m0);
+          tma_load_2d(sB + stage * kBStageBytes, mapB, full_leader, (kb0 + kb) * BK, n0);
           if (++stage == NS) { stage = 0; phase ^= 1u; }
         }
       }
@@ -578,11 +591,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       uint32_t phase = 0, acc_phase = 0;
       bool ok = true;
       for (int64_t q = cluster_id; ok && q < pieces; q += n_clusters) {
-        const uint32_t idesc = instr_desc(piece_of(q, tiles, tail).nw);
+        const uint32_t idesc = instr_desc(piece_of(q / ks, tiles, tail).nw);
+        const int kb0 = static_cast<int>(q % ks) * k_blocks;
+        const int kbn = k_all - kb0 < k_blocks ? k_all - kb0 : k_blocks;
         if (!mbar_wait(&tempty[acc], acc_phase ^ 1u, g.status)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN);
-        for (int kb = 0; kb < k_blocks; ++kb) {
+        for (int kb = 0; kb < kbn; ++kb) {
           if (!mbar_wait(&full[stage], phase, g.status)) { ok = false; break; }
           tc_fence_after();
           const uint64_t da = make_smem_desc(smem_u32(sA + stage * kAStageBytes));
@@ -606,17 +621,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     int acc = 0;
     uint32_t acc_phase = 0;
     for (int64_t q = cluster_id; q < pieces; q += n_clusters) {
-      const Piece pc = piece_of(q, tiles, tail);
+      const Piece pc = piece_of(q / ks, tiles, tail);
       const int64_t m0 = (pc.tile % m_tiles) * BM + rank * kRowsPerCta, n0 = (pc.tile / m_tiles) * BN + pc.noff;
       if (!mbar_wait(&tfull[acc], acc_phase, g.status)) break;
       tc_fence_after();
       const int row0 = static_cast<int>(m0) + quad * 32;
+      const int plane0 = static_cast<int>((q % ks) * g.plane_rows);      // first output row of this piece's range of K
       const int col0 = static_cast<int>(n0) + cgrp * kColsPerEpiWarp;
       const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) +
                              static_cast<uint32_t>(acc * BN + cgrp * kColsPerEpiWarp);
       // (a half piece fills the first 128 accumulator columns: the warps of the other two column groups only arrive)
       if (cgrp * kColsPerEpiWarp < pc.nw && row0 < M_rows && (col0 < g.N || EPI == kEpiArgmax))
-        epilogue_columns<EPI>(g, &tmD, buf, lane, taddr, row0, col0);
+        epilogue_columns<EPI>(g, &tmD, buf, lane, taddr, ks > 1 ? plane0 + row0 : row0, col0);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(mapa(smem_u32(&tempty[acc]), 0));

@@ -68,11 +68,21 @@ int launch_mixer_nv(const MixerParams& p, int num_sms, cudaStream_t st) {
   return SRM_OK;
 }
 
+// Whether the token-mixer step of this model runs on mixer_stream_kernel (whole 128-channel vectors per head).
+bool mixer_stream_shape(const srm_config& c, int state_elem) {
+  const int d = c.d_model, nv = d / 128;
+  return c.mixer == SRM_MIXER_MIXED && !(c.flags & SRM_FLAG_HEAD_PROJ) && d % 128 == 0 && (d / c.n_heads) % 128 == 0 &&
+         c.n_heads <= 8 && (nv == 4 || nv == 8 || nv == 12 || nv == 16) && mixer_stream_warps(d, state_elem) >= 1;
+}
+
+// ps: partial products of the previous layer's down projection still to be added into x (mixer_stream_kernel only).
 int launch_mixer(const srm_model& m, int layer, int t, int64_t R, const int32_t* tok, float* x, void* S, void* a,
-                 uint32_t* status, cudaStream_t st, const int32_t* ctr = nullptr, const int32_t* pos = nullptr) {
+                 uint32_t* status, cudaStream_t st, const int32_t* ctr = nullptr, const int32_t* pos = nullptr,
+                 const PartialSum& ps = PartialSum()) {
   if (R <= 0) return SRM_OK;
   LaunchScope scope(m, SRM_KERNEL_MIXER, st);
   MixerParams p;
+  p.part = ps.part; p.n_part = ps.n_part; p.part_plane = ps.plane; p.part_bias = ps.bias;
   p.x = x; p.tok = tok; p.E = m.ptr(-1, SRM_T_E); p.S = S; p.a = a;
   p.ln1_g = m.fptr(layer, SRM_T_LN1_G); p.ln1_b = m.fptr(layer, SRM_T_LN1_B);
   p.ln2_g = m.fptr(layer, SRM_T_LN2_G); p.ln2_b = m.fptr(layer, SRM_T_LN2_B);
@@ -127,18 +137,18 @@ int launch_mixer_variant(const srm_model& m, int layer, int t, int64_t R, const 
 
 template <typename WT>
 int launch_norm_t(const float* x, int64_t R, int64_t stride, int64_t offset, const float* g, const float* b, float eps,
-                  int d, void* out, cudaStream_t st, const int32_t* row_len = nullptr) {
+                  int d, void* out, cudaStream_t st, const int32_t* row_len = nullptr, const PartialSum& ps = PartialSum()) {
   const int nv = (d + 127) / 128;
   const unsigned grid = (unsigned)((R + kMixerWarps - 1) / kMixerWarps);
   const dim3 blk(kMixerWarps * 32);
   WT* o = reinterpret_cast<WT*>(out);
-  if (nv <= 1) SRM_CUDA(launch_kernel(norm_rows_kernel<1, WT>, dim3(grid), dim3(blk), 0, st, x, R, stride, offset, g, b, eps, d, o, row_len));
-  else if (nv <= 2) SRM_CUDA(launch_kernel(norm_rows_kernel<2, WT>, dim3(grid), dim3(blk), 0, st, x, R, stride, offset, g, b, eps, d, o, row_len));
-  else if (nv <= 4) SRM_CUDA(launch_kernel(norm_rows_kernel<4, WT>, dim3(grid), dim3(blk), 0, st, x, R, stride, offset, g, b, eps, d, o, row_len));
-  else if (nv <= 6) SRM_CUDA(launch_kernel(norm_rows_kernel<6, WT>, dim3(grid), dim3(blk), 0, st, x, R, stride, offset, g, b, eps, d, o, row_len));
-  else if (nv <= 8) SRM_CUDA(launch_kernel(norm_rows_kernel<8, WT>, dim3(grid), dim3(blk), 0, st, x, R, stride, offset, g, b, eps, d, o, row_len));
-  else if (nv <= 12) SRM_CUDA(launch_kernel(norm_rows_kernel<12, WT>, dim3(grid), dim3(blk), 0, st, x, R, stride, offset, g, b, eps, d, o, row_len));
-  else SRM_CUDA(launch_kernel(norm_rows_kernel<16, WT>, dim3(grid), dim3(blk), 0, st, x, R, stride, offset, g, b, eps, d, o, row_len));
+  if (nv <= 1) SRM_CUDA(launch_kernel(norm_rows_kernel<1, WT>, dim3(grid), dim3(blk), 0, st, x, R, stride, offset, g, b, eps, d, o, row_len, ps));
+  else if (nv <= 2) SRM_CUDA(launch_kernel(norm_rows_kernel<2, WT>, dim3(grid), dim3(blk), 0, st, x, R, stride, offset, g, b, eps, d, o, row_len, ps));
+  else if (nv <= 4) SRM_CUDA(launch_kernel(norm_rows_kernel<4, WT>, dim3(grid), dim3(blk), 0, st, x, R, stride, offset, g, b, eps, d, o, row_len, ps));
+  else if (nv <= 6) SRM_CUDA(launch_kernel(norm_rows_kernel<6, WT>, dim3(grid), dim3(blk), 0, st, x, R, stride, offset, g, b, eps, d, o, row_len, ps));
+  else if (nv <= 8) SRM_CUDA(launch_kernel(norm_rows_kernel<8, WT>, dim3(grid), dim3(blk), 0, st, x, R, stride, offset, g, b, eps, d, o, row_len, ps));
+  else if (nv <= 12) SRM_CUDA(launch_kernel(norm_rows_kernel<12, WT>, dim3(grid), dim3(blk), 0, st, x, R, stride, offset, g, b, eps, d, o, row_len, ps));
+  else SRM_CUDA(launch_kernel(norm_rows_kernel<16, WT>, dim3(grid), dim3(blk), 0, st, x, R, stride, offset, g, b, eps, d, o, row_len, ps));
   SRM_CUDA(cudaGetLastError());
   return SRM_OK;
 }
@@ -153,13 +163,13 @@ int launch_norm(const srm_model& m, const float* x, int64_t R, int64_t stride, i
 }
 
 int launch_final_norm(const srm_model& m, const float* x, int64_t R, int64_t stride, int64_t offset, void* out,
-                      cudaStream_t st, const int32_t* row_len = nullptr) {
+                      cudaStream_t st, const int32_t* row_len = nullptr, const PartialSum& ps = PartialSum()) {
   if (R <= 0) return SRM_OK;
   LaunchScope scope(m, SRM_KERNEL_NORM, st);
   const float* g = m.fptr(-1, SRM_T_LNF_G);
   const float* b = m.fptr(-1, SRM_T_LNF_B);
-  if (m.cfg.dtype == SRM_DTYPE_BF16) return launch_norm_t<bf16>(x, R, stride, offset, g, b, m.cfg.ln_eps, m.cfg.d_model, out, st, row_len);
-  return launch_norm_t<float>(x, R, stride, offset, g, b, m.cfg.ln_eps, m.cfg.d_model, out, st, row_len);
+  if (m.cfg.dtype == SRM_DTYPE_BF16) return launch_norm_t<bf16>(x, R, stride, offset, g, b, m.cfg.ln_eps, m.cfg.d_model, out, st, row_len, ps);
+  return launch_norm_t<float>(x, R, stride, offset, g, b, m.cfg.ln_eps, m.cfg.d_model, out, st, row_len, ps);
 }
 
 template <typename T>
@@ -210,8 +220,10 @@ int gemm_tail_tiles(const srm_model& m, int64_t tiles) {
   return (r > 0 && 2 * r <= m.tc_clusters) ? (int)r : 0;
 }
 
+// k_slices > 1 (epilogue kEpiPlain only; K / 64 a multiple of k_slices): out is k_slices planes of plane_rows x N
+// partial products (GemmArgs::k_slices).
 int launch_gemm_tc(srm_model& m, int epi, int64_t M, int64_t N, int64_t K, const void* A, const void* W,
-                   const float* bias, void* out, uint32_t* status, cudaStream_t st) {
+                   const float* bias, void* out, uint32_t* status, cudaStream_t st, int k_slices = 1, int64_t plane_rows = 0) {
   int rc = ensure_tc_ready(m);
   if (rc != SRM_OK) return rc;
   CUtensorMap ta, tb, td, tb64;
@@ -219,14 +231,16 @@ int launch_gemm_tc(srm_model& m, int epi, int64_t M, int64_t N, int64_t K, const
   if ((rc = m.tmap(W, N, K, tc::kRowsPerCta, 2, &tb)) != SRM_OK) return rc;
   if ((rc = m.tmap(W, N, K, tc::kHalfN / 2, 2, &tb64)) != SRM_OK) return rc;      // W rows of a half-width piece
   if (epi == kEpiArgmax) td = ta;       // no output matrix: the descriptor is not used
-  else if ((rc = m.tmap(out, M, N, tc::kOutBoxRows, epi == kEpiBiasGelu ? 2 : 4, &td)) != SRM_OK) return rc;
+  else if ((rc = m.tmap(out, k_slices > 1 ? k_slices * plane_rows : M, N, tc::kOutBoxRows, epi == kEpiBiasGelu ? 2 : 4, &td)) != SRM_OK) return rc;
   const uint8_t* wb = static_cast<const uint8_t*>(W);
   const int w_static = wb >= m.w && wb < m.w + m.layout.total;      // inside the weight blob
   const int64_t tiles = ((M + tc::BM - 1) / tc::BM) * ((N + tc::BN - 1) / tc::BN);
-  const int tail = gemm_tail_tiles(m, tiles);
+  const int tail = k_slices > 1 ? 0 : gemm_tail_tiles(m, tiles);
   tc::GemmArgs g{M, N, K, bias, out, status, w_static};
   g.tail_tiles = tail;
-  const int64_t pieces = tiles + tail;
+  g.k_slices = k_slices > 1 ? k_slices : 1;
+  g.plane_rows = plane_rows;
+  const int64_t pieces = (tiles + tail) * g.k_slices;
   const unsigned grid = 2u * (unsigned)(pieces < m.tc_clusters ? pieces : m.tc_clusters);
   if (epi == kEpiBiasGelu) SRM_CUDA(launch_kernel(tc::gemm_tc_kernel<kEpiBiasGelu>, dim3(grid), dim3(tc::kThreads), tc::kSmemBytes, st, ta, tb, td, tb64, g));
   else if (epi == kEpiBiasResidual) SRM_CUDA(launch_kernel(tc::gemm_tc_kernel<kEpiBiasResidual>, dim3(grid), dim3(tc::kThreads), tc::kSmemBytes, st, ta, tb, td, tb64, g));
@@ -332,6 +346,17 @@ int launch_ffn_fused(srm_model& m, int layer, int64_t M, const void* a, void* H,
                          ta, tw1, tw1h, ths, th, tw2, tx, g, *plan));
   SRM_CUDA(cudaGetLastError());
   return SRM_OK;
+}
+
+// Ranges the K dimension of a small down projection is cut into (GemmArgs::k_slices): the largest power of two up
+// to kMaxKSlices that divides the k-blocks, leaves at least four k-blocks per range and keeps tiles x ranges within the CTA
+// pairs; 1 (no cut) when the tiles alone fill half the pairs. Depends on the tile count, so rows of passes of very
+// different sizes see sums in another order (last bits); equal-sized passes and all smaller ones agree bit for bit.
+int down_k_slices(int64_t tiles, int k_blocks, int pairs) {
+  if (tiles < 1 || 2 * tiles > pairs) return 1;
+  int ks = 1;
+  while (ks < kMaxKSlices && k_blocks % (2 * ks) == 0 && k_blocks / (2 * ks) >= 4 && tiles * 2 * ks <= pairs) ks *= 2;
+  return ks;
 }
 
 float topk_z0(int top_k, int V) {
@@ -624,6 +649,18 @@ int decode_chunk(srm_model& m, srm_state& s, int64_t b0, int64_t R, const int32_
   }
   if (fused_ffn) SRM_CUDA(cudaMemsetAsync(w.logits, 0, ready_layer * c.n_layers, st));
   else if (split) SRM_CUDA(cudaMemsetAsync(w.order, 0, w.order_bytes, st));
+  // A small pass (the down projection has less than half as many tiles as there are CTA pairs): its K dimension is
+  // cut into ranges so that all pairs work on it; the partial products go to planes of their own in the workspace
+  // and the next consumer of x (the next layer's mixer, the final norm) adds them in a fixed order.
+  PartialSum ps_none, ps;
+  int k_slices = 1;
+  const int64_t plane_rows = (R + tc::BM - 1) / tc::BM * tc::BM;
+  if (!fused_ffn && !split && w.part != nullptr) {
+    if ((rc = ensure_tc_ready(m))) return rc;
+    k_slices = down_k_slices(plane_rows / tc::BM * ((d + tc::BN - 1) / tc::BN), (int)(F / tc::BK), m.tc_clusters);
+    while (k_slices > 1 && (size_t)k_slices * plane_rows * d * 4 > w.part_bytes) k_slices /= 2;
+  }
+  if (k_slices > 1) ps = PartialSum{w.part, k_slices, plane_rows * (int64_t)d, nullptr};
   for (int l = 0; l < c.n_layers; ++l) {
     uint8_t* Sl = static_cast<uint8_t*>(s.layer_ptr(l)) + (size_t)b0 * d * m.state_bytes();
     if (c.mixer != SRM_MIXER_MIXED) {
@@ -631,7 +668,11 @@ int decode_chunk(srm_model& m, srm_state& s, int64_t b0, int64_t R, const int32_
                                      st, ctr))) return rc;
     } else if (m.head_proj()) {
       if ((rc = launch_mixer_block_proj(m, l, t, R, R, 1, l == 0 ? tok_in + b0 : nullptr, w.x, Sl, w.a, w.q, s.status, st, ctr, pos))) return rc;
-    } else if ((rc = launch_mixer(m, l, t, R, l == 0 ? tok_in + b0 : nullptr, w.x, Sl, w.a, s.status, st, ctr, pos))) return rc;
+    } else {
+      PartialSum pl = l > 0 ? ps : ps_none;                // what layer l - 1's down projection left in planes
+      if (l > 0) pl.bias = m.fptr(l - 1, SRM_T_B2);
+      if ((rc = launch_mixer(m, l, t, R, l == 0 ? tok_in + b0 : nullptr, w.x, Sl, w.a, s.status, st, ctr, pos, pl))) return rc;
+    }
     if (fused_ffn) {
       int32_t* ready = reinterpret_cast<int32_t*>(reinterpret_cast<uint8_t*>(w.logits) + (size_t)l * ready_layer);
       rc = launch_ffn_fused(m, l, R, w.a, w.H, w.x, ready, s.status, st);
@@ -643,11 +684,18 @@ int decode_chunk(srm_model& m, srm_state& s, int64_t b0, int64_t R, const int32_
     if ((rc = launch_gemm(m, kEpiBiasGelu, R, F, d, w.a, m.ptr(l, SRM_T_W1), m.fptr(l, SRM_T_B1), w.H, s.status, st))) return rc;
     rc = split ? launch_gemm_splitk(m, R, d, F, w.H, m.ptr(l, SRM_T_W2), m.fptr(l, SRM_T_B2), w.x, w.order, s.status, st, true)
                : SRM_ERR_UNSUPPORTED;
-    if (rc == SRM_ERR_UNSUPPORTED)
-      rc = launch_gemm(m, kEpiBiasResidual, R, d, F, w.H, m.ptr(l, SRM_T_W2), m.fptr(l, SRM_T_B2), w.x, s.status, st);
+    if (rc == SRM_ERR_UNSUPPORTED) {
+      if (k_slices > 1) {
+        LaunchScope scope(m, SRM_KERNEL_GEMM_DOWN, st);
+        rc = launch_gemm_tc(m, kEpiPlain, R, d, F, w.H, m.ptr(l, SRM_T_W2), nullptr, w.part, s.status, st, k_slices, plane_rows);
+      } else {
+        rc = launch_gemm(m, kEpiBiasResidual, R, d, F, w.H, m.ptr(l, SRM_T_W2), m.fptr(l, SRM_T_B2), w.x, s.status, st);
+      }
+    }
     if (rc) return rc;
   }
-  if ((rc = launch_final_norm(m, w.x, R, 1, 0, w.a, st))) return rc;
+  if (k_slices > 1) ps.bias = m.fptr(c.n_layers - 1, SRM_T_B2);
+  if ((rc = launch_final_norm(m, w.x, R, 1, 0, w.a, st, nullptr, k_slices > 1 ? ps : ps_none))) return rc;
   SelectOut o = out_all;
   o.last_tok += b0;
   if (o.tok_out) o.tok_out += b0;

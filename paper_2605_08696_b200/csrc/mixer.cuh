@@ -25,6 +25,22 @@ struct MixerParams {
   uint32_t* status;
   const int32_t* ctr;    // device-side step counters, or nullptr: then `t` above is the position
   const int32_t* pos;    // [R] per-row positions (samples of different lengths), or nullptr: one position for all rows
+  // mixer_stream_kernel only: partial products of the previous layer's down projection that have not been added into
+  // x yet (the projection ran with its K dimension cut into n_part ranges, see GemmArgs::k_slices). The row this
+  // kernel works on is x[r] + part_bias + part[0][r] + ... + part[n_part - 1][r], added in this order.
+  const float* part = nullptr;        // [n_part] planes of part_plane elements, row r of a plane at r * d
+  int n_part = 0;
+  int64_t part_plane = 0;
+  const float* part_bias = nullptr;   // [d]
+};
+
+// What a consumer adds to a row of the residual stream whose last down projection left partial products (see
+// MixerParams::part); nullptr: nothing.
+struct PartialSum {
+  const float* part = nullptr;
+  int n_part = 0;
+  int64_t plane = 0;
+  const float* bias = nullptr;
 };
 
 constexpr int kMixerWarps = 4;
@@ -161,7 +177,7 @@ template <int NV, typename WT>
 __global__ void __launch_bounds__(kMixerWarps * 32)
 norm_rows_kernel(const float* __restrict__ x, int64_t R, int64_t src_stride, int64_t src_offset,
                  const float* __restrict__ g, const float* __restrict__ b, float eps, int d,
-                 WT* __restrict__ out, const int32_t* __restrict__ row_len) {
+                 WT* __restrict__ out, const int32_t* __restrict__ row_len, const PartialSum ps) {
   pdl_trigger();
   pdl_wait();
   const int lane = threadIdx.x & 31;
@@ -174,6 +190,27 @@ norm_rows_kernel(const float* __restrict__ x, int64_t R, int64_t src_stride, int
   for (int i = 0; i < NV; ++i) {
     const int c = (i * 32 + lane) * 4;
     if (c < d) v[i] = ld4(xr + c);
+  }
+  if (ps.part != nullptr) {              // x + bias + plane 0 + plane 1 + ... (row r of every plane)
+#pragma unroll
+    for (int i = 0; i < NV; ++i) {
+      const int c = (i * 32 + lane) * 4;
+      if (c < d) {
+        const float4 bb = ldg4(ps.bias + c);
+        v[i] = make_float4(v[i].x + bb.x, v[i].y + bb.y, v[i].z + bb.z, v[i].w + bb.w);
+      }
+    }
+    for (int s = 0; s < ps.n_part; ++s) {
+      const float* pr = ps.part + (int64_t)s * ps.plane + row * d;
+#pragma unroll
+      for (int i = 0; i < NV; ++i) {
+        const int c = (i * 32 + lane) * 4;
+        if (c < d) {
+          const float4 q = ld4(pr + c);
+          v[i] = make_float4(v[i].x + q.x, v[i].y + q.y, v[i].z + q.z, v[i].w + q.w);
+        }
+      }
+    }
   }
   float mean, rstd;
   row_stats<NV>(v, lane, d, eps, mean, rstd);

@@ -141,6 +141,21 @@ __global__ void __launch_bounds__(kStreamMaxWarps * 32, 1) mixer_stream_kernel(c
 #pragma unroll
       for (int i = 0; i < NV; ++i) v[i] = ld4(xs + i * 128);
     }
+    if (p.part != nullptr) {              // x + bias + plane 0 + plane 1 + ... (MixerParams::part)
+#pragma unroll
+      for (int i = 0; i < NV; ++i) {
+        const float4 bb = ldg4(p.part_bias + c0 + i * 128);
+        v[i] = make_float4(v[i].x + bb.x, v[i].y + bb.y, v[i].z + bb.z, v[i].w + bb.w);
+      }
+      for (int s = 0; s < p.n_part; ++s) {
+        const float* pr = p.part + (int64_t)s * p.part_plane + r * d + c0;
+#pragma unroll
+        for (int i = 0; i < NV; ++i) {
+          const float4 q = ld4(pr + i * 128);
+          v[i] = make_float4(v[i].x + q.x, v[i].y + q.y, v[i].z + q.z, v[i].w + q.w);
+        }
+      }
+    }
     float mean, rstd;
     row_stats_full<NV>(v, inv_d, p.eps, mean, rstd);
     const float nmr = -mean * rstd;                      // (x - mean) * rstd = x * rstd + nmr

@@ -301,8 +301,27 @@ size_t small_scratch_bytes(const srm_config& c) {
   return align_up((size_t)8 * sb::kMaxRows * c.d_model * 4, 256) + align_up((size_t)256 * sb::kMaxRows * 8, 256) + 256;
 }
 
+// Partial-product planes of a small pass's down projection (GemmArgs::k_slices): up to 8 planes of the pass's rows
+// (padded to whole 256-row tiles) x d floats, never more than one 256 x 256 fp32 tile per CTA pair of the largest
+// device (tiles x ranges stays within the pairs). Only for the models whose mixer adds them (mixer_stream_kernel).
+constexpr int kMaxKSlices = 8;
+bool kslice_model(const srm_config& c) {
+  const int d = c.d_model, nv = d / 128, se = c.state_dtype == SRM_DTYPE_FP32 ? 4 : 2;
+  return c.dtype == SRM_DTYPE_BF16 && !(c.flags & (SRM_FLAG_SIMT_GEMM | SRM_FLAG_NO_KSLICE | SRM_FLAG_HEAD_PROJ)) &&
+         c.mixer == SRM_MIXER_MIXED && d % 128 == 0 && (d / c.n_heads) % 128 == 0 && c.n_heads <= 8 &&
+         (nv == 4 || nv == 8 || nv == 12 || nv == 16) && mixer_stream_warps(d, se) >= 1 && ((size_t)c.ffn_mult * d) % 64 == 0;
+}
+size_t kslice_bytes(const srm_config& c, int64_t rows) {
+  if (!kslice_model(c)) return 0;
+  const size_t rows_pad = (size_t)(rows + tc::BM - 1) / tc::BM * tc::BM;
+  const size_t want = (size_t)kMaxKSlices * rows_pad * c.d_model * 4, cap = (size_t)96 * tc::BM * tc::BN * 4;
+  return align_up(want < cap ? want : cap, 256);
+}
+
 struct DecodeWs {
   float* x; void* a; void* H; float* logits;
+  float* part;            // kslice_bytes
+  size_t part_bytes;
   uint8_t* small;         // small_scratch_bytes
   float* q;               // head projections only
   int32_t* order;         // split-K down projection: one word per (tile of x, CTA of the pair, epilogue warp)
@@ -322,7 +341,8 @@ size_t decode_ws_bytes(const srm_model& m, int64_t rows) {
   const size_t d = m.cfg.d_model, F = m.F(), V = m.cfg.vocab, ab = m.act_bytes();
   return align_up(rows * d * 4, 256) + align_up(rows * d * ab, 256) + align_up(rows * F * ab, 256) +
          align_up(rows * V * 4, 256) + (m.head_proj() ? align_up(rows * d * 4, 256) : 0) +
-         (splitk_enabled(m.cfg) ? splitk_order_bytes(rows, m.cfg.d_model) : 0) + small_scratch_bytes(m.cfg);
+         (splitk_enabled(m.cfg) ? splitk_order_bytes(rows, m.cfg.d_model) : 0) + small_scratch_bytes(m.cfg) +
+         kslice_bytes(m.cfg, rows);
 }
 size_t prefill_ws_bytes(const srm_model& m, int64_t samples, int n) {
   const size_t d = m.cfg.d_model, F = m.F(), V = m.cfg.vocab, ab = m.act_bytes(), rows = (size_t)samples * n;
@@ -356,7 +376,9 @@ DecodeWs carve_decode(const srm_model& m, void* ws, int64_t rows) {
   w.order_bytes = splitk_enabled(m.cfg) ? splitk_order_bytes(rows, m.cfg.d_model) : 0;
   w.order = w.order_bytes ? reinterpret_cast<int32_t*>(p) : nullptr;
   p += w.order_bytes;
-  w.small = p;
+  w.small = p; p += small_scratch_bytes(m.cfg);
+  w.part_bytes = kslice_bytes(m.cfg, rows);
+  w.part = w.part_bytes ? reinterpret_cast<float*>(p) : nullptr;
   return w;
 }
 PrefillWs carve_prefill(const srm_model& m, void* ws, int64_t samples, int n) {

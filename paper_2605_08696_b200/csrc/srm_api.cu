@@ -45,6 +45,13 @@ size_t srm_workspace_bytes(const srm_config* cfg, int64_t B_chunk, int32_t n_pre
   return need;
 }
 
+size_t srm_prefill_workspace_bytes(const srm_config* cfg, int64_t samples, int32_t n) {
+  if (!config_ok(cfg) || samples < 1 || n < 1) return 0;
+  srm_model tmp;
+  tmp.cfg = *cfg;
+  return prefill_ws_bytes(tmp, samples, n);
+}
+
 int srm_create(const srm_config* cfg, const void* d_weights, size_t nbytes, srm_model** out) {
   if (out == nullptr || d_weights == nullptr) return SRM_ERR_INVALID_ARG;
   *out = nullptr;
