@@ -215,6 +215,8 @@ namespace {
 // (replicas == 1: the plain prefill). A prompt is run once; with replicas > 1 its per-layer cache goes to a
 // staging area at the end of the workspace and is then copied to the rows of its replicas, and every replica
 // selects its own first token from the prompt's last-position logits.
+constexpr int64_t kPrefillFfnRows = 8192;     // rows per feed-forward kernel of a prefill pass
+
 int prefill_impl(srm_model* m, srm_state* s, const int32_t* d_tokens, int64_t P, int32_t n, int64_t replicas,
                  const srm_sampling* samp, int32_t* d_first_tok, float* d_logits_last, void* d_ws, size_t ws_bytes,
                  cudaStream_t st, const int32_t* d_len = nullptr) {
@@ -253,8 +255,36 @@ int prefill_impl(srm_model* m, srm_state* s, const int32_t* d_tokens, int64_t P,
                                           nullptr, d_len ? d_len + p0 : nullptr))) return rc;
       } else if ((rc = launch_prefill_mixer(*m, l, np, n, l == 0 ? d_tokens + p0 * n : nullptr, w.x, Sl, w.a, s->status, st,
                                             d_len ? d_len + p0 : nullptr))) return rc;
-      if ((rc = launch_gemm(*m, kEpiBiasGelu, rows, F, d, w.a, m->ptr(l, SRM_T_W1), m->fptr(l, SRM_T_B1), w.H, s->status, st))) return rc;
-      if ((rc = launch_gemm(*m, kEpiBiasResidual, rows, d, F, w.H, m->ptr(l, SRM_T_W2), m->fptr(l, SRM_T_B2), w.x, s->status, st))) return rc;
+      // The feed-forward block over the rows of the pass: in slabs of kPrefillFfnRows rows, each as ONE kernel
+      // (ffn_fused.cuh: a slab's hidden activations, 64 MB for the mid model, are consumed from L2 as they are
+      // produced instead of crossing HBM twice), where the model's shape allows and the slab counters fit in the
+      // logits area (free until the LM head); else, and for a short last slab, up projection then down projection.
+      const size_t slab_ready = ffn_ready_bytes(kPrefillFfnRows, F);
+      const int64_t n_slabs = (rows + kPrefillFfnRows - 1) / kPrefillFfnRows;
+      bool slabs = !(c.flags & SRM_FLAG_NO_FUSED_FFN) && rows >= kPrefillFfnRows && ffn_fused_shape_ok(*m, kPrefillFfnRows) &&
+                   (size_t)n_slabs * slab_ready <= align_up((size_t)np * c.vocab * 4, 256);
+      if (slabs) {
+        if ((rc = ensure_tc_ready(*m))) return rc;
+        slabs = ffn_fused_worthwhile(*m, kPrefillFfnRows);
+      }
+      if (slabs) SRM_CUDA(cudaMemsetAsync(w.logits, 0, (size_t)n_slabs * slab_ready, st));
+      for (int64_t r0 = 0; slabs && r0 < rows; r0 += kPrefillFfnRows) {
+        const int64_t nr = rows - r0 < kPrefillFfnRows ? rows - r0 : kPrefillFfnRows;
+        uint8_t* a_s = static_cast<uint8_t*>(w.a) + (size_t)r0 * d * m->act_bytes();
+        uint8_t* H_s = static_cast<uint8_t*>(w.H) + (size_t)r0 * F * m->act_bytes();
+        float* x_s = w.x + (size_t)r0 * d;
+        int32_t* ready = reinterpret_cast<int32_t*>(reinterpret_cast<uint8_t*>(w.logits) + (size_t)(r0 / kPrefillFfnRows) * slab_ready);
+        rc = ffn_fused_worthwhile(*m, nr) ? launch_ffn_fused(*m, l, nr, a_s, H_s, x_s, ready, s->status, st) : SRM_ERR_UNSUPPORTED;
+        if (rc == SRM_ERR_UNSUPPORTED) {
+          if ((rc = launch_gemm(*m, kEpiBiasGelu, nr, F, d, a_s, m->ptr(l, SRM_T_W1), m->fptr(l, SRM_T_B1), H_s, s->status, st))) return rc;
+          rc = launch_gemm(*m, kEpiBiasResidual, nr, d, F, H_s, m->ptr(l, SRM_T_W2), m->fptr(l, SRM_T_B2), x_s, s->status, st);
+        }
+        if (rc) return rc;
+      }
+      if (!slabs) {
+        if ((rc = launch_gemm(*m, kEpiBiasGelu, rows, F, d, w.a, m->ptr(l, SRM_T_W1), m->fptr(l, SRM_T_B1), w.H, s->status, st))) return rc;
+        if ((rc = launch_gemm(*m, kEpiBiasResidual, rows, d, F, w.H, m->ptr(l, SRM_T_W2), m->fptr(l, SRM_T_B2), w.x, s->status, st))) return rc;
+      }
       for (int pl = 0; replicas > 1 && pl < planes; ++pl) {
         LaunchScope scope(*m, SRM_KERNEL_PREFILL_MIXER, st);
         const int64_t vpr = (int64_t)row_bytes / 16, total = nb * vpr;

@@ -147,3 +147,31 @@ def test_captured_step_with_the_fused_block_equals_launch_by_launch():
             assert prof["ffn"][0] == 6 * shape.n_layers        # (launches inside a replayed graph are not bracketed)
     for x_, y_ in zip(outs[0], outs[1]):
         assert torch.equal(x_, y_)
+
+
+def test_prefill_with_the_fused_block_in_slabs_equals_the_two_launches():
+    """A prefill pass of more than 8192 rows runs its feed-forward blocks slab by slab through the single kernel (a
+    whole slab, then a shorter one): logits of the last position, first tokens and the cache must equal the run with
+    SRM_FLAG_NO_FUSED_FFN, and the decode step that follows must agree as well."""
+    import paper_2605_08696_b200 as P
+    shape = custom_shape(n_layers=2, d_model=1024, vocab=2048, n_ctx=320, dtype="bf16", seed=12)
+    W = I.make_weights(shape, alpha_std=0.5, beta_std=0.5)
+    B, n = 40, 300                                             # 12000 rows: one slab of 8192 and one of 3808
+    prompts = torch.from_numpy(np.random.default_rng(5).integers(0, shape.vocab, size=(B, n)).astype(np.int32)).to(DEV)
+    outs = []
+    for flags in (0, P.FLAG_NO_FUSED_FFN):
+        m = P.SRM(shape, W, device=DEV, flags=flags | P.FLAG_NO_SMALL_BATCH)
+        st = m.new_state(B)
+        ws = m.new_workspace(B, n, prefill_samples=B)
+        m.profile(True)
+        m.profile_reset()
+        tok, lg = m.prefill(st, prompts, P.Sampling("greedy"), ws, want_logits=True)
+        prof = m.profile_read()
+        m.profile(False)
+        tok2, lg2 = m.decode_step(st, tok, P.Sampling("greedy"), 1, ws, want_logits=True)
+        assert st.status() == 0
+        outs.append((lg.clone(), tok.clone(), lg2.clone(), st.cache().clone(), prof))
+    assert outs[0][4]["ffn"][0] == 2 * shape.n_layers and outs[0][4]["gemm_up"][0] == 0
+    assert outs[1][4]["ffn"][0] == 0 and outs[1][4]["gemm_up"][0] == shape.n_layers
+    for a_, b_ in zip(outs[0][:4], outs[1][:4]):
+        assert torch.equal(a_, b_)
