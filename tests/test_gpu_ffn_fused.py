@@ -150,13 +150,13 @@ def test_captured_step_with_the_fused_block_equals_launch_by_launch():
 
 
 def test_prefill_with_the_fused_block_in_slabs_equals_the_two_launches():
-    """A prefill pass of more than 8192 rows runs its feed-forward blocks slab by slab through the single kernel (a
+    """A prefill pass of more than 16384 rows runs its feed-forward blocks slab by slab through the single kernel (a
     whole slab, then a shorter one): logits of the last position, first tokens and the cache must equal the run with
     SRM_FLAG_NO_FUSED_FFN, and the decode step that follows must agree as well."""
     import paper_2605_08696_b200 as P
     shape = custom_shape(n_layers=2, d_model=1024, vocab=2048, n_ctx=320, dtype="bf16", seed=12)
     W = I.make_weights(shape, alpha_std=0.5, beta_std=0.5)
-    B, n = 40, 300                                             # 12000 rows: one slab of 8192 and one of 3808
+    B, n = 68, 300                                             # 20400 rows: one slab of 16384 and one of 4016
     prompts = torch.from_numpy(np.random.default_rng(5).integers(0, shape.vocab, size=(B, n)).astype(np.int32)).to(DEV)
     outs = []
     for flags in (0, P.FLAG_NO_FUSED_FFN):
