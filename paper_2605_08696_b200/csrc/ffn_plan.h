@@ -134,7 +134,7 @@ inline double ffn_simulate(const FfnShape& s, const FfnPlan& P, const FfnCost& c
 // Lower bound of any plan under the cost model: all work shared out evenly, and at least one up and one down tile in a row.
 inline double ffn_ideal(const FfnShape& s, int pairs, const FfnCost& c = FfnCost()) {
   const double up = s.ku * c.up_kb + c.up_tile, dn = s.kd * c.dn_kb + c.dn_tile;
-  return std::max(((double)s.Rb * s.Cu * up + (double)s.Rb * s.Cd * dn) / pairs, up + kFfnKbPerHTile * c.dn_kb + dn - 0.0 * c.ready_lag);
+  return std::max(((double)s.Rb * s.Cu * up + (double)s.Rb * s.Cd * dn) / pairs, up + kFfnKbPerHTile * c.dn_kb + dn);
 }
 
 // The plan in which the last `n_half` up tiles placed (the first of the forward lists) go out as halves.

@@ -68,13 +68,6 @@ int launch_mixer_nv(const MixerParams& p, int num_sms, cudaStream_t st) {
   return SRM_OK;
 }
 
-// Whether the token-mixer step of this model runs on mixer_stream_kernel (whole 128-channel vectors per head).
-bool mixer_stream_shape(const srm_config& c, int state_elem) {
-  const int d = c.d_model, nv = d / 128;
-  return c.mixer == SRM_MIXER_MIXED && !(c.flags & SRM_FLAG_HEAD_PROJ) && d % 128 == 0 && (d / c.n_heads) % 128 == 0 &&
-         c.n_heads <= 8 && (nv == 4 || nv == 8 || nv == 12 || nv == 16) && mixer_stream_warps(d, state_elem) >= 1;
-}
-
 // ps: partial products of the previous layer's down projection still to be added into x (mixer_stream_kernel only).
 int launch_mixer(const srm_model& m, int layer, int t, int64_t R, const int32_t* tok, float* x, void* S, void* a,
                  uint32_t* status, cudaStream_t st, const int32_t* ctr = nullptr, const int32_t* pos = nullptr,
