@@ -78,7 +78,7 @@ enum {
                                         CTA pairs busy to the end); for comparison and measurement */
   SRM_FLAG_NO_FUSED_FFN = 256,       /* the feed-forward block of a decode step always runs as two launches, up projection
                                         then down projection (default, bf16 models whose d is a multiple of 256, passes
-                                        of at most 16384 rows with at least one and a half 256 x 256 tiles per CTA pair:
+                                        of at most 16384 rows with at least two 256 x 256 tiles per CTA pair:
                                         ONE kernel computes the tiles of both projections, see srm_k_ffn; same results
                                         bit for bit); for comparison and measurement */
   SRM_FLAG_NO_KSLICE = 512,          /* the down projection of a small decode pass always adds whole tiles into x (default,
@@ -427,7 +427,7 @@ int64_t srm_k_gemm_splitk_plan(int64_t M, int64_t N, int64_t K, int32_t pairs, i
  * one another: do not run it concurrently with other work on the same device (it then may time out: status bit
  * SRM_STATUS_WAIT_TIMEOUT, result invalid). SRM_ERR_UNSUPPORTED: not a bf16 tensor-core model, d or F not a multiple of
  * 256, more than 16384 rows or more than 2048 tiles. This is what srm_decode_step and srm_generate run per layer
- * for passes with at least one and a half tiles per CTA pair (mid model: from 1536 rows), unless
+ * for passes with at least two tiles per CTA pair (mid model: from 2048 rows), unless
  * SRM_FLAG_NO_FUSED_FFN is set. */
 size_t srm_k_ffn_ready_bytes(int64_t M, int64_t F);
 int srm_k_ffn(srm_model* m, int32_t layer, int64_t M, const void* d_a, void* d_H, float* d_x, void* d_ready,

@@ -295,13 +295,15 @@ bool ffn_fused_shape_ok(const srm_model& m, int64_t M) {
   return tc::ffn_shape_ok(ffn_shape(M, c.d_model, F), 2);
 }
 
-// Whether the decode step takes it for a pass of M rows: from one and a half tiles per CTA pair. With fewer the chain
-// up tile -> epilogue -> counter -> down tile is longer than two launches that overlap through programmatic dependent
-// launch. Measured on the mid model (74 pairs, 20 tiles per 256 rows), one kernel against two launches, ms per step:
-// 512 rows 0.73 / 0.64, 1024: 0.76 / 0.71, 1536: 0.80 / 0.81, 2048: 0.89 / 0.93, 3072: 1.14 / 1.24, 4096: 1.47 / 1.51.
+// Whether the decode step takes it for a pass of M rows: from two tiles per CTA pair. With fewer the chain up tile ->
+// epilogue -> counter -> down tile is longer than two launches that overlap through programmatic dependent launch,
+// and the down projection of such a pass runs over ranges of K instead (down_k_slices). Measured on the mid model
+// (74 pairs, 20 tiles per 256 rows), ms per step, one kernel / two launches / two launches with ranges of K: 512 rows
+// 0.73 / 0.64 / 0.50, 1024: 0.76 / 0.71 / 0.59, 1536: 0.80 / 0.81 / 0.75, 2048: 0.89 / 0.93 / 0.92, 2304: 0.94 / 0.99 /
+// 0.99, 3072: 1.14 / 1.24 / -, 4096: 1.47 / 1.51 / -.
 bool ffn_fused_worthwhile(const srm_model& m, int64_t M) {
   const tc::FfnShape s = ffn_shape(M, m.cfg.d_model, m.F());
-  return m.tc_clusters >= 2 && 2 * (int64_t)s.Rb * (s.Cu + s.Cd) >= 3 * (int64_t)m.tc_clusters;
+  return m.tc_clusters >= 2 && (int64_t)s.Rb * (s.Cu + s.Cd) >= 2 * (int64_t)m.tc_clusters;
 }
 
 // `ready`: ffn_ready_bytes(M, F) bytes of zeroed words. SRM_ERR_UNSUPPORTED: take the two launches.

@@ -80,11 +80,11 @@ def test_shapes_the_fused_block_does_not_take_are_refused():
     assert e.value.code == P.ERR_UNSUPPORTED
 
 
-@pytest.mark.parametrize("B,d,head_proj,fused", [(2500, 1024, False, True), (3100, 512, True, True), (300, 512, False, False)])
+@pytest.mark.parametrize("B,d,head_proj,fused", [(2500, 1024, False, True), (3900, 512, True, True), (300, 512, False, False)])
 def test_decode_steps_with_and_without_the_fused_block_are_equal(B, d, head_proj, fused):
     """Prefill and a few decode steps (logits requested, greedy) on two models over the same weights, one of them with
     SRM_FLAG_NO_FUSED_FFN: logits, tokens and cache must be equal, and the profile must show which path ran (the
-    step takes the single kernel from one and a half tiles per CTA pair; 300 rows of d = 512 are 20 tiles)."""
+    step takes the single kernel from two tiles per CTA pair; 300 rows of d = 512 are 20 tiles)."""
     import paper_2605_08696_b200 as P
     shape = custom_shape(n_layers=3, d_model=d, vocab=2048, n_ctx=24, dtype="bf16", seed=5, head_proj=head_proj)
     W = I.make_weights(shape, alpha_std=0.5, beta_std=0.5)
@@ -126,7 +126,7 @@ def test_captured_step_with_the_fused_block_equals_launch_by_launch():
     import paper_2605_08696_b200 as P
     shape = custom_shape(n_layers=3, d_model=512, vocab=2048, n_ctx=40, dtype="bf16", seed=8)
     W = I.make_weights(shape, alpha_std=0.5, beta_std=0.5)
-    B, n = 3100, 4
+    B, n = 3900, 4
     prompts = torch.from_numpy(np.random.default_rng(3).integers(0, shape.vocab, size=(B, n)).astype(np.int32)).to(DEV)
     samp = P.Sampling("topk", 20, 0.9, seed=4, sample_idx_base=11)
     outs = []
