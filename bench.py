@@ -358,7 +358,8 @@ def run_ours(args):
     model = P.SRM(shape, W, device=dev, state_dtype=args.state_dtype,
                   flags={"auto": 0, "on": P.FLAG_GRAPH, "off": P.FLAG_NO_GRAPH}[args.graph] |
                   (P.FLAG_NO_SPLITK if args.no_splitk else 0) | (P.FLAG_NO_TAIL_SPLIT if args.no_tail_split else 0) |
-                  (P.FLAG_NO_FUSED_FFN if args.no_fused_ffn else 0) | (P.FLAG_NO_KSLICE if args.no_kslice else 0))
+                  (P.FLAG_NO_FUSED_FFN if args.no_fused_ffn else 0) | (P.FLAG_NO_KSLICE if args.no_kslice else 0) |
+                  (P.FLAG_NO_SMALL_BATCH if args.no_small_batch else 0))
     sidx0 = rank_plan(rank, world, B)["sample_idx_base"]
     samp = {"greedy": lambda: P.Sampling("greedy"),
             "topk": lambda: P.Sampling("topk", w["top_k"], w["temperature"], seed=shape.seed, sample_idx_base=sidx0),
@@ -763,6 +764,8 @@ def main():
                     help="token mixer of the model: mixed heads (the hot path), linearly combined heads (twice the cache) "
                          "or kernels of size --kernel-size (Eq. 11; that many times the cache)")
     ap.add_argument("--kernel-size", type=int, default=4)
+    ap.add_argument("--no-small-batch", action="store_true",
+                    help="batches of at most 64 samples: one kernel per operation instead of the single-kernel step")
     ap.add_argument("--no-kslice", action="store_true",
                     help="small passes: down projection as whole tiles (no ranges of K with partial products)")
     ap.add_argument("--no-fused-ffn", action="store_true",
